@@ -1,0 +1,195 @@
+/*
+ * rattn.h -- C ABI of the RAttention operator for NVIDIA B200 (sm_100a).
+ *
+ * The operator is one attention layer's token mixing (Section 3.2 of the paper):
+ *
+ *     y_t = rmsnorm(o_swa_t; g_swa) + rmsnorm(o_rla_t; g_rla)
+ *
+ *   o_swa_t = softmax attention of q_t over the keys max(0,t-w) <= j <= t   (Section 2.1)
+ *   o_rla_t = phi(q_t) S_{t-w-1},  S_n = sum_{j<=n} phi(k_j)^T v_j          (Eq. 4)
+ *   phi     = softmax over the d head features, d' = d                      (Section 3.1)
+ *
+ * with K/V (and the state S) shared by the H_q/H_kv query heads of a group
+ * (Section 3.1, "Group-Query Variant": query head h reads K/V head h / (H_q/H_kv)).
+ *
+ * Conventions for every entry point
+ *   - Positions are 0-indexed.  The window holds w+1 keys including the current one.
+ *   - Tensors are dense, row-major, innermost dimension d:
+ *       q, out, dout, dq : [B, H_q,  T, d]      k, v, dk, dv : [B, H_kv, T, d]
+ *   - All data pointers are DEVICE pointers unless a parameter says "host".
+ *     They must be 16-byte aligned.  The caller owns every buffer; the library
+ *     keeps no reference after the call returns, allocates no device memory
+ *     (one documented exception: rattn_forward), and never synchronises
+ *     (exception: rattn_read_status): all work is enqueued on `stream` (a
+ *     cudaStream_t passed as void*; NULL is the legacy default stream).
+ *   - Return value: RATTN_OK (0) or a negative rattn_status.  Nothing is launched
+ *     when an argument check fails.  No C++ exception crosses this boundary.
+ *   - Device-side waits are bounded: if one expires the kernel stops early and
+ *     records RATTN_ERR_TIMEOUT in the status word inside the workspace
+ *     (see rattn_read_status).
+ */
+#ifndef RATTN_H_
+#define RATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum rattn_status {
+  RATTN_OK = 0,
+  RATTN_ERR_BAD_ARG = -1,        /* a size is out of range (B,H,T < 1, w < 1, H_q % H_kv != 0, ...) */
+  RATTN_ERR_NULL_PTR = -2,       /* a required pointer is NULL */
+  RATTN_ERR_MISALIGNED = -3,     /* a data pointer is not 16-byte aligned */
+  RATTN_ERR_UNSUPPORTED = -4,    /* d not in {64,128}, unknown dtype / mode */
+  RATTN_ERR_WORKSPACE = -5,      /* workspace missing or smaller than rattn_workspace_bytes() */
+  RATTN_ERR_CUDA = -6,           /* a CUDA call failed; see rattn_last_cuda_error() */
+  RATTN_ERR_TIMEOUT = -7         /* a bounded device-side wait expired (status word) */
+} rattn_status;
+
+typedef enum rattn_dtype { RATTN_BF16 = 0, RATTN_F32 = 1 } rattn_dtype;
+
+typedef enum rattn_mode {
+  RATTN_MODE_RATTN = 0,          /* SWA + RLA, the operator above */
+  RATTN_MODE_SWA_ONLY = 1,       /* y = rmsnorm(o_swa); the RLA branch is skipped */
+  RATTN_MODE_FULL_CAUSAL = 2     /* w := T: y = rmsnorm(causal softmax attention) */
+} rattn_mode;
+
+/* Path selection for rattn_params.flags. */
+#define RATTN_FLAG_FORCE_GENERIC 1u  /* use the portable fp32-FMA kernels even where the
+                                        tensor-core path applies (debugging / comparison) */
+#define RATTN_FLAG_SAVE_RESIDUALS 2u /* training mode: the forward also writes what the
+                                        backward needs (log-sum-exp and the two un-normalised
+                                        branch outputs) into the workspace */
+
+/*
+ * Parameter block of the *_ex entry points.  Zero-initialise it, then fill in.
+ *   dtype      I/O element type of q,k,v,out,dout,dq,dk,dv and the decode ring.
+ *              Accumulation, softmax, feature map, norms and the state are fp32.
+ *   scale      multiplies the SWA logits q.k only (the paper writes none: 1.0).
+ *   eps        added to mean(x^2) inside the RMS-norm square root.
+ *   gamma_swa, gamma_rla   fp32 [H_q, d] gains of the two norms, or NULL for ones.
+ *   workspace  scratch + saved residuals, rattn_workspace_bytes() bytes, 256-byte
+ *              aligned.  rattn_forward_ex writes it; rattn_backward_ex reads the
+ *              residuals the forward left there, so pass the same buffer, untouched,
+ *              with the same sizes.
+ *   state_out, k_ring_out, v_ring_out   optional prefill -> decode hand-off written by
+ *              rattn_forward_ex: state [B,H_kv,d,d] fp32 = sum over tokens j < T-w of
+ *              phi(k_j)^T v_j; rings [B,H_kv,w,d] (I/O dtype) holding token j at slot
+ *              j % w for the last min(w,T) tokens (other slots zero).
+ *   dgamma_swa, dgamma_rla   optional fp32 [H_q,d] outputs of rattn_backward_ex.
+ */
+typedef struct rattn_params {
+  const void* q;
+  const void* k;
+  const void* v;
+  void* out;
+  int32_t B, H_q, H_kv, T, d, w;
+  int32_t dtype;                 /* rattn_dtype */
+  int32_t mode;                  /* rattn_mode */
+  float scale;
+  float eps;
+  const float* gamma_swa;
+  const float* gamma_rla;
+  void* workspace;
+  size_t workspace_bytes;
+  float* state_out;
+  void* k_ring_out;
+  void* v_ring_out;
+  /* backward only */
+  const void* dout;
+  void* dq;
+  void* dk;
+  void* dv;
+  float* dgamma_swa;
+  float* dgamma_rla;
+  uint32_t flags;                /* RATTN_FLAG_* */
+  uint32_t reserved;
+} rattn_params;
+
+/*
+ * Forward, Section 3.2 (SWA of Section 2.1 + RLA of Eq. 4 + two RMS norms).
+ * bf16 I/O, scale = 1, unit gains, eps = 1e-6, mode RATTN, inference (no residuals).
+ * T need not be a multiple of any tile.  This is the one entry point that may take
+ * device memory on its own: where the tensor-core path applies (d = 128, w % 128 == 0)
+ * it needs scratch for the chunk states of the linear branch and obtains it with
+ * cudaMallocAsync / cudaFreeAsync on `stream` (the device's stream-ordered pool; no
+ * synchronisation).  Callers that must control every allocation use rattn_forward_ex
+ * with their own workspace.
+ */
+int rattn_forward(const void* q, const void* k, const void* v,
+                  int B, int H_q, int H_kv, int T, int d, int w,
+                  void* out, void* stream);
+
+/* Forward with the full parameter block (dtype, scale, gains, mode, workspace,
+ * residuals for the backward, prefill -> decode hand-off). */
+int rattn_forward_ex(const rattn_params* p, void* stream);
+
+/*
+ * Backward of the same operator: given dout = dL/dy, writes dq, dk, dv (I/O dtype;
+ * dk, dv summed over the query heads of each group).  The paper prints no backward
+ * formulas; these are the chain rule through Section 2.1, Eq. 4, the softmax feature
+ * map and the two RMS norms, using per-chunk states as the paper's kernel-design
+ * paragraph describes (states saved at chunk boundaries, intra-chunk terms recomputed).
+ * bf16, scale = 1, unit gains, eps = 1e-6.  `ws` must be the workspace a preceding
+ * rattn_forward_ex call with the same sizes filled.
+ */
+int rattn_backward(const void* q, const void* k, const void* v, const void* dout,
+                   void* ws, size_t ws_bytes,
+                   int B, int H_q, int H_kv, int T, int d, int w,
+                   void* dq, void* dk, void* dv, void* stream);
+
+int rattn_backward_ex(const rattn_params* p, void* stream);
+
+/*
+ * One decode step (Section 2.1: at most w+1 cached tokens; Eq. 4: constant-size state).
+ * For every batch entry, at position pos (the same for the whole batch):
+ *   SWA over the ring's tokens pos-w..pos-1 (those >= 0) plus the incoming token,
+ *   RLA read-out phi(q) . state  (state holds tokens j < pos-w),
+ *   y = rmsnorm(o_swa) + rmsnorm(o_rla) -> out [B,H_q,d];
+ * then the token leaving the window (pos-w, if >= 0) is folded into the state,
+ * state += phi(k_old)^T v_old, and the incoming k,v overwrite ring slot pos % w.
+ *   q [B,H_q,d]; k, v [B,H_kv,d]; k_ring, v_ring [B,H_kv,w,d] (same dtype as q);
+ *   state [B,H_kv,d,d] fp32 (rows: feature index of phi(k), columns: value index).
+ * Ring and state are updated in place.  bf16, scale = 1, unit gains, eps = 1e-6.
+ */
+int rattn_decode_step(const void* q, const void* k, const void* v,
+                      void* k_ring, void* v_ring, float* state, int pos,
+                      int B, int H_q, int H_kv, int d, int w,
+                      void* out, void* stream);
+
+/* Decode step with dtype / scale / eps / gains taken from `p` (p->q,k,v,out are the
+ * step's tensors; p->T is ignored).  k_ring, v_ring, state, pos as above. */
+int rattn_decode_step_ex(const rattn_params* p, void* k_ring, void* v_ring, float* state,
+                         int pos, void* stream);
+
+/*
+ * Bytes of workspace the forward (and the backward that follows it) needs for these
+ * sizes; dtype is a rattn_dtype.  Returns 0 for invalid sizes.  The first 256 bytes
+ * hold the device status word.
+ */
+size_t rattn_workspace_bytes(int B, int H_q, int H_kv, int T, int d, int w, int dtype);
+
+/* Reads the status word of a workspace (synchronises `stream` first, copies 4 bytes
+ * device -> host).  Returns RATTN_OK, RATTN_ERR_TIMEOUT, or RATTN_ERR_CUDA. */
+int rattn_read_status(const void* workspace, void* stream);
+
+/* Static string for a status code.  Host memory owned by the library. */
+const char* rattn_strerror(int status);
+
+/* The cudaError_t (as int) behind the calling thread's last RATTN_ERR_CUDA. */
+int rattn_last_cuda_error(void);
+
+/* Number of kernel launches this process has enqueued through the library so far
+ * (host counter; used by the benchmark to report its launch count). */
+uint64_t rattn_launch_count(void);
+
+/* 1 when the tensor-core (tcgen05) forward would be chosen for these sizes. */
+int rattn_uses_tensor_path(int d, int w, int dtype, int mode, unsigned flags);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RATTN_H_ */

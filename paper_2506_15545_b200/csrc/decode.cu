@@ -1,0 +1,445 @@
+// Single-token decode step and the prefill -> decode hand-off.
+//
+// Decode keeps, per K/V head, a ring of the last w keys/values (Section 2.1: the SWA
+// cache is at most w+1 tokens, the newest being the incoming one) and the fixed-size
+// fp32 state S of Eq. 4.  One step streams the ring once, reads S once and writes it
+// back with the evicted token folded in: the step is bound by HBM traffic, so all
+// global accesses are 16-byte vectors and every CTA keeps several loads in flight.
+#include "rattn_internal.h"
+
+namespace rattn {
+namespace {
+
+constexpr int DEC_THREADS = 512;
+constexpr int DEC_WARPS = DEC_THREADS / 32;
+constexpr int GH = 4;                       // query heads processed per pass over the ring
+
+template <typename T> struct Vec16;        // a 16-byte vector of I/O elements
+template <> struct Vec16<__nv_bfloat16> {
+  static constexpr int N = 8;
+  static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&f)[8]) {
+    uint4 u = *reinterpret_cast<const uint4*>(p);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float2 x = __bfloat1622float2(h[i]);
+      f[2 * i] = x.x;
+      f[2 * i + 1] = x.y;
+    }
+  }
+};
+template <> struct Vec16<float> {
+  static constexpr int N = 4;
+  static __device__ __forceinline__ void load(const float* p, float (&f)[4]) {
+    float4 u = *reinterpret_cast<const float4*>(p);
+    f[0] = u.x; f[1] = u.y; f[2] = u.z; f[3] = u.w;
+  }
+};
+
+__device__ __forceinline__ float to_f(float x) { return x; }
+__device__ __forceinline__ float to_f(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_f(float x);
+template <> __device__ __forceinline__ float from_f<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float x) {
+  return __float2bfloat16_rn(x);
+}
+
+__device__ __forceinline__ float warp_max(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+  return x;
+}
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+
+// softmax over D features by one warp: dst[a] = phi(src)[a]
+template <int D>
+__device__ __forceinline__ void warp_feature_map(float* dst, const float* src, int lane) {
+  float m = -INFINITY;
+  for (int a = lane; a < D; a += 32) m = fmaxf(m, src[a]);
+  m = warp_max(m);
+  float s = 0.f;
+  for (int a = lane; a < D; a += 32) {
+    float e = __expf(src[a] - m);
+    dst[a] = e;
+    s += e;
+  }
+  s = warp_sum(s);
+  const float inv = 1.f / s;
+  for (int a = lane; a < D; a += 32) dst[a] *= inv;
+}
+
+struct DecodeArgs {
+  const void* q; const void* k; const void* v;
+  void* k_ring; void* v_ring; float* state; void* out;
+  const float* gamma_swa; const float* gamma_rla;
+  int B, H_q, H_kv, w, pos, group;
+  float scale, eps;
+};
+
+template <typename TIO, int D>
+__global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecodeArgs a) {
+  constexpr int EPL = Vec16<TIO>::N;        // elements per lane per 16-byte load
+  constexpr int LPK = D / EPL;              // lanes that cover one key row
+  constexpr int KPW = 32 / LPK;             // key rows per warp per load
+  constexpr int C4 = D / 4;                 // float4 columns of a state row
+  constexpr int RP = DEC_THREADS / C4;      // state rows per pass
+
+  extern __shared__ __align__(16) float sm[];
+  const int g = a.group;
+  float* q_s = sm;                          // [g][D] raw q
+  float* fq_s = q_s + g * D;                // [g][D] phi(q)
+  float* k_new = fq_s + g * D;              // [D]
+  float* v_new = k_new + D;
+  float* k_old = v_new + D;
+  float* v_old = k_old + D;
+  float* fk_old = v_old + D;
+  float* s_new = fk_old + D;                // [GH] logit of the incoming token
+  float* part_m = s_new + GH;               // [WARPS][GH]
+  float* part_l = part_m + DEC_WARPS * GH;  // [WARPS][GH]
+  float* o_swa = part_l + DEC_WARPS * GH;   // [GH][D]
+  float* o_rla = o_swa + GH * D;            // [GH][D]
+  float* part_acc = o_rla + GH * D;         // [max(WARPS,RP)][GH][D]
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int b = blockIdx.x / a.H_kv, hk = blockIdx.x % a.H_kv;
+  const int w = a.w, pos = a.pos;
+  const bool evict = pos - w >= 0;
+  const int slot = pos % w;
+  const int n_valid = pos < w ? pos : w;
+
+  const TIO* qg = reinterpret_cast<const TIO*>(a.q) + ((size_t)b * a.H_q + (size_t)hk * g) * D;
+  const TIO* kg = reinterpret_cast<const TIO*>(a.k) + ((size_t)b * a.H_kv + hk) * D;
+  const TIO* vg = reinterpret_cast<const TIO*>(a.v) + ((size_t)b * a.H_kv + hk) * D;
+  TIO* kr = reinterpret_cast<TIO*>(a.k_ring) + ((size_t)b * a.H_kv + hk) * (size_t)w * D;
+  TIO* vr = reinterpret_cast<TIO*>(a.v_ring) + ((size_t)b * a.H_kv + hk) * (size_t)w * D;
+  float* S = a.state + ((size_t)b * a.H_kv + hk) * (size_t)D * D;
+  TIO* og = reinterpret_cast<TIO*>(a.out) + ((size_t)b * a.H_q + (size_t)hk * g) * D;
+
+  for (int i = tid; i < g * D; i += DEC_THREADS) q_s[i] = to_f(qg[i]);
+  if (tid < D) {
+    k_new[tid] = to_f(kg[tid]);
+    v_new[tid] = to_f(vg[tid]);
+    if (evict) {
+      k_old[tid] = to_f(kr[(size_t)slot * D + tid]);
+      v_old[tid] = to_f(vr[(size_t)slot * D + tid]);
+    }
+  }
+  __syncthreads();
+  for (int r = warp; r <= g; r += DEC_WARPS) {
+    if (r < g) warp_feature_map<D>(fq_s + r * D, q_s + r * D, lane);
+    else if (evict) warp_feature_map<D>(fk_old, k_old, lane);
+  }
+  __syncthreads();
+
+  const int sub = lane / LPK, chunk = lane % LPK;
+  for (int h0 = 0; h0 < g; h0 += GH) {
+    const int nh = (g - h0) < GH ? (g - h0) : GH;
+    // ---- SWA over the ring (Section 2.1), online softmax per warp -------------------
+    float qr[GH][EPL], m[GH], l[GH], acc[GH][EPL];
+#pragma unroll
+    for (int hh = 0; hh < GH; ++hh) {
+      m[hh] = -INFINITY;
+      l[hh] = 0.f;
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) {
+        qr[hh][e] = hh < nh ? q_s[(h0 + hh) * D + chunk * EPL + e] * a.scale : 0.f;
+        acc[hh][e] = 0.f;
+      }
+    }
+    constexpr int U = 4;                    // loads in flight per lane (x2 for K and V)
+    for (int s0 = warp * KPW; s0 < n_valid; s0 += DEC_WARPS * KPW * U) {
+      float kx[U][EPL], vx[U][EPL];
+      bool ok[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int s = s0 + u * DEC_WARPS * KPW + sub;
+        ok[u] = s < n_valid;
+        if (ok[u]) {
+          Vec16<TIO>::load(kr + (size_t)s * D + chunk * EPL, kx[u]);
+          Vec16<TIO>::load(vr + (size_t)s * D + chunk * EPL, vx[u]);
+        } else {
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) { kx[u][e] = 0.f; vx[u][e] = 0.f; }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+#pragma unroll
+        for (int hh = 0; hh < GH; ++hh) {
+          float dot = 0.f;
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) dot += qr[hh][e] * kx[u][e];
+#pragma unroll
+          for (int o = 1; o < LPK; o <<= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+          if (ok[u]) {
+            const float m_new = fmaxf(m[hh], dot);
+            const float corr = __expf(m[hh] - m_new);   // exp(-inf) = 0 on the first key
+            const float p = __expf(dot - m_new);
+            l[hh] = l[hh] * corr + p;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) acc[hh][e] = acc[hh][e] * corr + p * vx[u][e];
+            m[hh] = m_new;
+          }
+        }
+      }
+    }
+    // merge the KPW key sub-groups of the warp
+#pragma unroll
+    for (int o = LPK; o < 32; o <<= 1) {
+#pragma unroll
+      for (int hh = 0; hh < GH; ++hh) {
+        const float m_o = __shfl_xor_sync(0xffffffffu, m[hh], o);
+        const float l_o = __shfl_xor_sync(0xffffffffu, l[hh], o);
+        const float m_new = fmaxf(m[hh], m_o);
+        const float c0 = (m[hh] == -INFINITY) ? 0.f : __expf(m[hh] - m_new);
+        const float c1 = (m_o == -INFINITY) ? 0.f : __expf(m_o - m_new);
+        l[hh] = l[hh] * c0 + l_o * c1;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+          const float a_o = __shfl_xor_sync(0xffffffffu, acc[hh][e], o);
+          acc[hh][e] = acc[hh][e] * c0 + a_o * c1;
+        }
+        m[hh] = m_new;
+      }
+    }
+    if (sub == 0) {
+#pragma unroll
+      for (int hh = 0; hh < GH; ++hh) {
+        if (chunk == 0) {
+          part_m[warp * GH + hh] = m[hh];
+          part_l[warp * GH + hh] = l[hh];
+        }
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) part_acc[(warp * GH + hh) * D + chunk * EPL + e] = acc[hh][e];
+      }
+    }
+    if (warp < nh) {                        // logit of the incoming token for head h0+warp
+      float dot = 0.f;
+      for (int c = lane; c < D; c += 32) dot += q_s[(h0 + warp) * D + c] * k_new[c];
+      dot = warp_sum(dot) * a.scale;
+      if (lane == 0) s_new[warp] = dot;
+    }
+    __syncthreads();
+    for (int i = tid; i < nh * D; i += DEC_THREADS) {
+      const int hh = i / D, c = i % D;
+      float M = s_new[hh];
+      for (int wv = 0; wv < DEC_WARPS; ++wv) M = fmaxf(M, part_m[wv * GH + hh]);
+      float pn = __expf(s_new[hh] - M);
+      float L = pn, O = pn * v_new[c];
+      for (int wv = 0; wv < DEC_WARPS; ++wv) {
+        const float mw = part_m[wv * GH + hh];
+        if (mw == -INFINITY) continue;
+        const float cf = __expf(mw - M);
+        L += part_l[wv * GH + hh] * cf;
+        O += part_acc[(wv * GH + hh) * D + c] * cf;
+      }
+      o_swa[hh * D + c] = O / L;
+    }
+    __syncthreads();
+
+    // ---- RLA read-out phi(q) S and, once, the state update S += phi(k_old)^T v_old (Eq. 4)
+    {
+      const int c4 = tid % C4, rl = tid / C4;
+      float4 ar[GH];
+#pragma unroll
+      for (int hh = 0; hh < GH; ++hh) ar[hh] = make_float4(0.f, 0.f, 0.f, 0.f);
+      const bool update = evict && (h0 + GH >= g);   // fold the evicted token in on the last pass
+      float4 vo = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (update) vo = *reinterpret_cast<const float4*>(v_old + c4 * 4);
+#pragma unroll 4
+      for (int r = rl; r < D; r += RP) {
+        float4 s4 = *reinterpret_cast<const float4*>(S + (size_t)r * D + c4 * 4);
+#pragma unroll
+        for (int hh = 0; hh < GH; ++hh) {
+          const float f = hh < nh ? fq_s[(h0 + hh) * D + r] : 0.f;
+          ar[hh].x += f * s4.x; ar[hh].y += f * s4.y; ar[hh].z += f * s4.z; ar[hh].w += f * s4.w;
+        }
+        if (update) {
+          const float fk = fk_old[r];
+          s4.x += fk * vo.x; s4.y += fk * vo.y; s4.z += fk * vo.z; s4.w += fk * vo.w;
+          *reinterpret_cast<float4*>(S + (size_t)r * D + c4 * 4) = s4;
+        }
+      }
+#pragma unroll
+      for (int hh = 0; hh < GH; ++hh)
+        *reinterpret_cast<float4*>(part_acc + ((size_t)(rl * GH + hh)) * D + c4 * 4) = ar[hh];
+    }
+    __syncthreads();
+    for (int i = tid; i < nh * D; i += DEC_THREADS) {
+      const int hh = i / D, c = i % D;
+      float O = 0.f;
+      for (int r = 0; r < RP; ++r) O += part_acc[(r * GH + hh) * D + c];
+      o_rla[hh * D + c] = O;
+    }
+    __syncthreads();
+
+    // ---- Section 3.2: two RMS norms and the sum --------------------------------------
+    if (warp < nh) {
+      const int h = hk * g + h0 + warp;
+      float ss = 0.f, sr = 0.f;
+      for (int c = lane; c < D; c += 32) {
+        const float x = o_swa[warp * D + c], y = o_rla[warp * D + c];
+        ss += x * x;
+        sr += y * y;
+      }
+      ss = warp_sum(ss);
+      sr = warp_sum(sr);
+      const float is = rsqrtf(ss / D + a.eps), ir = rsqrtf(sr / D + a.eps);
+      for (int c = lane; c < D; c += 32) {
+        const float gs = a.gamma_swa ? a.gamma_swa[(size_t)h * D + c] : 1.f;
+        const float gr = a.gamma_rla ? a.gamma_rla[(size_t)h * D + c] : 1.f;
+        og[(size_t)(h0 + warp) * D + c] =
+            from_f<TIO>(gs * o_swa[warp * D + c] * is + gr * o_rla[warp * D + c] * ir);
+      }
+    }
+    __syncthreads();
+  }
+  // the incoming token takes the evicted token's slot
+  if (tid < D) {
+    kr[(size_t)slot * D + tid] = kg[tid];
+    vr[(size_t)slot * D + tid] = vg[tid];
+  }
+}
+
+template <int D> constexpr size_t decode_smem_floats(int g) {
+  constexpr int RP = DEC_THREADS / (D / 4);
+  constexpr int PR = RP > DEC_WARPS ? RP : DEC_WARPS;
+  return (size_t)2 * g * D + 5 * D + GH + 2 * DEC_WARPS * GH + 2 * GH * D + (size_t)PR * GH * D;
+}
+
+template <typename TIO, int D>
+cudaError_t launch_dec(const DecodeArgs& a, cudaStream_t s) {
+  const size_t smem = decode_smem_floats<D>(a.group) * sizeof(float);
+  if (smem > 227 * 1024) return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(decode_kernel<TIO, D>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  decode_kernel<TIO, D><<<a.B * a.H_kv, DEC_THREADS, smem, s>>>(a);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- prefill -> decode hand-off
+// state_out[b,hk] = sum_{j < T-w} phi(k_j)^T v_j  (Eq. 4), one CTA per 8 feature rows.
+template <typename TIO, int D>
+__global__ void __launch_bounds__(256) handoff_state_kernel(const TIO* __restrict__ k,
+                                                            const TIO* __restrict__ v,
+                                                            float* __restrict__ state, int T, int w) {
+  constexpr int ROWS = 8, TOK = 32;
+  __shared__ float fk[TOK][ROWS];
+  __shared__ float vs[TOK][D];
+  const int bh = blockIdx.y, r0 = blockIdx.x * ROWS;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const TIO* kg = k + (size_t)bh * T * D;
+  const TIO* vg = v + (size_t)bh * T * D;
+  const int n = T - w;                       // tokens 0..n-1 have left every window
+  // thread -> (row, column group): 8 rows x 32 column lanes, D/32 columns each
+  const int row = tid / 32, cl = tid % 32;
+  float acc[D / 32];
+#pragma unroll
+  for (int c = 0; c < D / 32; ++c) acc[c] = 0.f;
+  for (int j0 = 0; j0 < n; j0 += TOK) {
+    __syncthreads();
+    for (int jj = warp; jj < TOK; jj += 8) {   // warp-level softmax of k_j, keep rows r0..r0+7
+      const int j = j0 + jj;
+      float x[D / 32];
+      float m = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        x[c] = j < n ? to_f(kg[(size_t)j * D + lane + 32 * c]) : 0.f;
+        m = fmaxf(m, x[c]);
+      }
+      m = warp_max(m);
+      float s = 0.f;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) { x[c] = __expf(x[c] - m); s += x[c]; }
+      s = warp_sum(s);
+      const float inv = j < n ? 1.f / s : 0.f;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        const int col = lane + 32 * c;
+        if (col >= r0 && col < r0 + ROWS) fk[jj][col - r0] = x[c] * inv;
+        vs[jj][col] = j < n ? to_f(vg[(size_t)j * D + col]) : 0.f;
+      }
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int jj = 0; jj < TOK; ++jj) {
+      const float f = fk[jj][row];
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) acc[c] += f * vs[jj][cl + 32 * c];
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < D / 32; ++c) state[((size_t)bh * D + r0 + row) * D + cl + 32 * c] = acc[c];
+}
+
+// ring[b,hk, j % w] = x[b,hk, j] for the last min(w,T) tokens; other slots zero.
+template <typename TIO>
+__global__ void handoff_ring_kernel(const TIO* __restrict__ k, const TIO* __restrict__ v,
+                                    TIO* __restrict__ kr, TIO* __restrict__ vr, int T, int w, int D) {
+  const int bh = blockIdx.y;
+  const int slot = blockIdx.x;
+  // the newest token that maps to this slot
+  const int last = T - 1;
+  const int j = last - ((last - slot) % w + w) % w;
+  const bool valid = j >= 0 && j >= T - w;
+  for (int c = threadIdx.x; c < D; c += blockDim.x) {
+    const size_t dst = ((size_t)bh * w + slot) * D + c;
+    if (valid) {
+      kr[dst] = k[((size_t)bh * T + j) * D + c];
+      vr[dst] = v[((size_t)bh * T + j) * D + c];
+    } else {
+      kr[dst] = from_f<TIO>(0.f);
+      vr[dst] = from_f<TIO>(0.f);
+    }
+  }
+}
+
+template <typename TIO, int D>
+cudaError_t launch_handoff_t(const Args& a, cudaStream_t s) {
+  const int BH = a.B * a.H_kv;
+  if (a.state_out) {
+    dim3 grid(D / 8, BH);
+    handoff_state_kernel<TIO, D><<<grid, 256, 0, s>>>(reinterpret_cast<const TIO*>(a.k),
+                                                      reinterpret_cast<const TIO*>(a.v),
+                                                      a.state_out, a.T, a.w);
+    count_launches(1);
+  }
+  if (a.k_ring_out && a.v_ring_out) {
+    dim3 grid(a.w, BH);
+    handoff_ring_kernel<TIO><<<grid, 64, 0, s>>>(reinterpret_cast<const TIO*>(a.k),
+                                                 reinterpret_cast<const TIO*>(a.v),
+                                                 reinterpret_cast<TIO*>(a.k_ring_out),
+                                                 reinterpret_cast<TIO*>(a.v_ring_out), a.T, a.w, D);
+    count_launches(1);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_decode(const Args& p, void* k_ring, void* v_ring, float* state, int pos,
+                          cudaStream_t s) {
+  DecodeArgs a;
+  a.q = p.q; a.k = p.k; a.v = p.v; a.k_ring = k_ring; a.v_ring = v_ring; a.state = state;
+  a.out = p.out; a.gamma_swa = p.gamma_swa; a.gamma_rla = p.gamma_rla;
+  a.B = p.B; a.H_q = p.H_q; a.H_kv = p.H_kv; a.w = p.w; a.pos = pos; a.group = p.group;
+  a.scale = p.scale; a.eps = p.eps;
+  if (p.dtype == RATTN_F32)
+    return p.d == 64 ? launch_dec<float, 64>(a, s) : launch_dec<float, 128>(a, s);
+  return p.d == 64 ? launch_dec<__nv_bfloat16, 64>(a, s) : launch_dec<__nv_bfloat16, 128>(a, s);
+}
+
+cudaError_t launch_handoff(const Args& a, cudaStream_t s) {
+  if (a.dtype == RATTN_F32)
+    return a.d == 64 ? launch_handoff_t<float, 64>(a, s) : launch_handoff_t<float, 128>(a, s);
+  return a.d == 64 ? launch_handoff_t<__nv_bfloat16, 64>(a, s)
+                   : launch_handoff_t<__nv_bfloat16, 128>(a, s);
+}
+
+}  // namespace rattn

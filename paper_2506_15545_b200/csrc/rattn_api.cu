@@ -1,0 +1,273 @@
+// C ABI of librattn.so: argument checks, workspace carving, path selection.
+// See include/rattn.h for the contract of every entry point.
+#include <atomic>
+#include <cstring>
+
+#include "rattn_internal.h"
+
+namespace rattn {
+
+static std::atomic<uint64_t> g_launches{0};
+static thread_local int g_last_cuda_error = 0;
+
+void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+WorkspaceLayout workspace_layout(int B, int H_q, int H_kv, int T, int d, int w, int dtype) {
+  (void)w;
+  (void)dtype;
+  WorkspaceLayout L;
+  const size_t rows = (size_t)B * H_q * T;
+  size_t off = 0;
+  L.status = off;      off += 256;
+  L.lse = off;         off += align256(rows * sizeof(float));
+  L.o_swa = off;       off += align256(rows * d * sizeof(float));
+  L.o_rla = off;       off += align256(rows * d * sizeof(float));
+  L.do_swa = off;      off += align256(rows * d * sizeof(float));
+  L.do_rla = off;      off += align256(rows * d * sizeof(float));
+  L.delta = off;       off += align256(rows * sizeof(float));
+  L.n_chunks = (T + 127) / 128;
+  const size_t states = (size_t)B * H_kv * L.n_chunks * d * d;
+  L.chunk_delta = off; off += align256(states * sizeof(float));
+  L.chunk_state = off; off += align256(states * sizeof(__nv_bfloat16));
+  L.total = off;
+  return L;
+}
+
+static int fail_cuda(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  return RATTN_ERR_CUDA;
+}
+
+static bool misaligned(const void* p) { return ((uintptr_t)p & 15u) != 0; }
+
+// Common checks of the size fields; fills the resolved Args.
+static int resolve(const rattn_params* p, Args* a, bool need_T) {
+  if (!p) return RATTN_ERR_NULL_PTR;
+  if (p->B < 1 || p->H_q < 1 || p->H_kv < 1 || p->w < 1 || (need_T && p->T < 1)) return RATTN_ERR_BAD_ARG;
+  if (p->H_q % p->H_kv != 0) return RATTN_ERR_BAD_ARG;
+  if (p->d != 64 && p->d != 128) return RATTN_ERR_UNSUPPORTED;
+  if (p->dtype != RATTN_BF16 && p->dtype != RATTN_F32) return RATTN_ERR_UNSUPPORTED;
+  if (p->mode < RATTN_MODE_RATTN || p->mode > RATTN_MODE_FULL_CAUSAL) return RATTN_ERR_UNSUPPORTED;
+  if (!(p->eps > 0.f) || !(p->scale == p->scale)) return RATTN_ERR_BAD_ARG;
+  if (!p->q || !p->k || !p->v || !p->out) return RATTN_ERR_NULL_PTR;
+  if (misaligned(p->q) || misaligned(p->k) || misaligned(p->v) || misaligned(p->out) ||
+      misaligned(p->gamma_swa) || misaligned(p->gamma_rla))
+    return RATTN_ERR_MISALIGNED;
+  std::memset(a, 0, sizeof(*a));
+  a->q = p->q; a->k = p->k; a->v = p->v; a->out = p->out;
+  a->B = p->B; a->H_q = p->H_q; a->H_kv = p->H_kv; a->T = p->T; a->d = p->d;
+  a->w = (p->mode == RATTN_MODE_FULL_CAUSAL && need_T) ? p->T : p->w;
+  a->group = p->H_q / p->H_kv;
+  a->dtype = p->dtype; a->mode = p->mode;
+  a->scale = p->scale; a->eps = p->eps;
+  a->gamma_swa = p->gamma_swa; a->gamma_rla = p->gamma_rla;
+  return RATTN_OK;
+}
+
+static int bind_workspace(const rattn_params* p, Args* a, bool required) {
+  if (!p->workspace) return required ? RATTN_ERR_WORKSPACE : RATTN_OK;
+  if (((uintptr_t)p->workspace & 255u) != 0) return RATTN_ERR_MISALIGNED;
+  const WorkspaceLayout L = workspace_layout(p->B, p->H_q, p->H_kv, p->T, p->d, p->w, p->dtype);
+  if (p->workspace_bytes < L.total) return RATTN_ERR_WORKSPACE;
+  char* base = reinterpret_cast<char*>(p->workspace);
+  a->status = reinterpret_cast<int*>(base + L.status);
+  a->lse = reinterpret_cast<float*>(base + L.lse);
+  a->o_swa = reinterpret_cast<float*>(base + L.o_swa);
+  a->o_rla = reinterpret_cast<float*>(base + L.o_rla);
+  a->do_swa = reinterpret_cast<float*>(base + L.do_swa);
+  a->do_rla = reinterpret_cast<float*>(base + L.do_rla);
+  a->delta = reinterpret_cast<float*>(base + L.delta);
+  a->chunk_delta = reinterpret_cast<float*>(base + L.chunk_delta);
+  a->chunk_state = reinterpret_cast<__nv_bfloat16*>(base + L.chunk_state);
+  a->n_chunks = L.n_chunks;
+  return RATTN_OK;
+}
+
+static bool tensor_path(int d, int w, int dtype, int mode, unsigned flags) {
+#ifdef RATTN_HAVE_TC
+  if (flags & RATTN_FLAG_FORCE_GENERIC) return false;
+  if (dtype != RATTN_BF16 || d != 128) return false;
+  if (mode == RATTN_MODE_RATTN && (w % 128) != 0) return false;
+  return true;
+#else
+  (void)d; (void)w; (void)dtype; (void)mode; (void)flags;
+  return false;
+#endif
+}
+
+static int forward_impl(const rattn_params* p, cudaStream_t s) {
+  Args a;
+  int rc = resolve(p, &a, true);
+  if (rc != RATTN_OK) return rc;
+  const bool want_handoff = p->state_out || p->k_ring_out || p->v_ring_out;
+  if (want_handoff) {
+    if ((p->k_ring_out == nullptr) != (p->v_ring_out == nullptr)) return RATTN_ERR_NULL_PTR;
+    if (misaligned(p->state_out) || misaligned(p->k_ring_out) || misaligned(p->v_ring_out))
+      return RATTN_ERR_MISALIGNED;
+    if (p->mode != RATTN_MODE_RATTN) return RATTN_ERR_UNSUPPORTED;
+  }
+  const bool tc = tensor_path(p->d, a.w, p->dtype, p->mode, p->flags);
+  rc = bind_workspace(p, &a, tc);
+  if (rc != RATTN_OK) return rc;
+  if (!(p->flags & RATTN_FLAG_SAVE_RESIDUALS)) {
+    a.lse = nullptr; a.o_swa = nullptr; a.o_rla = nullptr;
+  } else if (!p->workspace) {
+    return RATTN_ERR_WORKSPACE;
+  }
+  a.state_out = p->state_out; a.k_ring_out = p->k_ring_out; a.v_ring_out = p->v_ring_out;
+  cudaError_t e;
+  if (a.status) {
+    e = cudaMemsetAsync(a.status, 0, 256, s);
+    if (e != cudaSuccess) return fail_cuda(e);
+  }
+#ifdef RATTN_HAVE_TC
+  if (tc) e = launch_tc_forward(a, s);
+  else
+#endif
+    e = launch_generic_forward(a, s);
+  if (e != cudaSuccess) return fail_cuda(e);
+  if (want_handoff) {
+    e = launch_handoff(a, s);
+    if (e != cudaSuccess) return fail_cuda(e);
+  }
+  return RATTN_OK;
+}
+
+static int backward_impl(const rattn_params* p, cudaStream_t s) {
+  Args a;
+  int rc = resolve(p, &a, true);
+  if (rc != RATTN_OK) return rc;
+  if (!p->dout || !p->dq || !p->dk || !p->dv) return RATTN_ERR_NULL_PTR;
+  if (misaligned(p->dout) || misaligned(p->dq) || misaligned(p->dk) || misaligned(p->dv) ||
+      misaligned(p->dgamma_swa) || misaligned(p->dgamma_rla))
+    return RATTN_ERR_MISALIGNED;
+  rc = bind_workspace(p, &a, true);
+  if (rc != RATTN_OK) return rc;
+  a.dout = p->dout; a.dq = p->dq; a.dk = p->dk; a.dv = p->dv;
+  a.dgamma_swa = p->dgamma_swa; a.dgamma_rla = p->dgamma_rla;
+  cudaError_t e = launch_generic_backward(a, s);
+  if (e != cudaSuccess) return fail_cuda(e);
+  return RATTN_OK;
+}
+
+}  // namespace rattn
+
+using namespace rattn;
+
+extern "C" {
+
+int rattn_forward_ex(const rattn_params* p, void* stream) {
+  return forward_impl(p, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int rattn_forward(const void* q, const void* k, const void* v, int B, int H_q, int H_kv, int T,
+                  int d, int w, void* out, void* stream) {
+  rattn_params p;
+  std::memset(&p, 0, sizeof(p));
+  p.q = q; p.k = k; p.v = v; p.out = out;
+  p.B = B; p.H_q = H_q; p.H_kv = H_kv; p.T = T; p.d = d; p.w = w;
+  p.dtype = RATTN_BF16; p.mode = RATTN_MODE_RATTN; p.scale = 1.f; p.eps = 1e-6f;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (!tensor_path(d, w, RATTN_BF16, RATTN_MODE_RATTN, 0)) return forward_impl(&p, s);
+  // The tensor-core path needs scratch for the chunk states of the linear branch: take it
+  // from the device's stream-ordered pool for the duration of this call's work.
+  Args chk;
+  int rc = resolve(&p, &chk, true);
+  if (rc != RATTN_OK) return rc;
+  const size_t bytes = rattn_workspace_bytes(B, H_q, H_kv, T, d, w, RATTN_BF16);
+  void* ws = nullptr;
+  cudaError_t e = cudaMallocAsync(&ws, bytes, s);
+  if (e != cudaSuccess) return fail_cuda(e);
+  p.workspace = ws;
+  p.workspace_bytes = bytes;
+  rc = forward_impl(&p, s);
+  e = cudaFreeAsync(ws, s);
+  if (rc == RATTN_OK && e != cudaSuccess) return fail_cuda(e);
+  return rc;
+}
+
+int rattn_backward_ex(const rattn_params* p, void* stream) {
+  return backward_impl(p, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int rattn_backward(const void* q, const void* k, const void* v, const void* dout, void* ws,
+                   size_t ws_bytes, int B, int H_q, int H_kv, int T, int d, int w, void* dq,
+                   void* dk, void* dv, void* stream) {
+  rattn_params p;
+  std::memset(&p, 0, sizeof(p));
+  p.q = q; p.k = k; p.v = v; p.out = dq;   /* `out` is not written by the backward */
+  p.B = B; p.H_q = H_q; p.H_kv = H_kv; p.T = T; p.d = d; p.w = w;
+  p.dtype = RATTN_BF16; p.mode = RATTN_MODE_RATTN; p.scale = 1.f; p.eps = 1e-6f;
+  p.workspace = ws; p.workspace_bytes = ws_bytes;
+  p.dout = dout; p.dq = dq; p.dk = dk; p.dv = dv;
+  return backward_impl(&p, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int rattn_decode_step_ex(const rattn_params* p, void* k_ring, void* v_ring, float* state, int pos,
+                         void* stream) {
+  Args a;
+  int rc = resolve(p, &a, false);
+  if (rc != RATTN_OK) return rc;
+  if (!k_ring || !v_ring || !state) return RATTN_ERR_NULL_PTR;
+  if (misaligned(k_ring) || misaligned(v_ring) || misaligned(state)) return RATTN_ERR_MISALIGNED;
+  if (pos < 0) return RATTN_ERR_BAD_ARG;
+  if (p->mode != RATTN_MODE_RATTN) return RATTN_ERR_UNSUPPORTED;
+  if (a.group > 64) return RATTN_ERR_UNSUPPORTED;
+  a.w = p->w;
+  cudaError_t e = launch_decode(a, k_ring, v_ring, state, pos, reinterpret_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return fail_cuda(e);
+  return RATTN_OK;
+}
+
+int rattn_decode_step(const void* q, const void* k, const void* v, void* k_ring, void* v_ring,
+                      float* state, int pos, int B, int H_q, int H_kv, int d, int w, void* out,
+                      void* stream) {
+  rattn_params p;
+  std::memset(&p, 0, sizeof(p));
+  p.q = q; p.k = k; p.v = v; p.out = out;
+  p.B = B; p.H_q = H_q; p.H_kv = H_kv; p.T = 1; p.d = d; p.w = w;
+  p.dtype = RATTN_BF16; p.mode = RATTN_MODE_RATTN; p.scale = 1.f; p.eps = 1e-6f;
+  return rattn_decode_step_ex(&p, k_ring, v_ring, state, pos, stream);
+}
+
+size_t rattn_workspace_bytes(int B, int H_q, int H_kv, int T, int d, int w, int dtype) {
+  if (B < 1 || H_q < 1 || H_kv < 1 || T < 1 || w < 1 || (d != 64 && d != 128)) return 0;
+  if (H_q % H_kv != 0) return 0;
+  return workspace_layout(B, H_q, H_kv, T, d, w, dtype).total;
+}
+
+int rattn_read_status(const void* workspace, void* stream) {
+  if (!workspace) return RATTN_ERR_NULL_PTR;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  int word = 0;
+  cudaError_t e = cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return fail_cuda(e);
+  return word == 0 ? RATTN_OK : RATTN_ERR_TIMEOUT;
+}
+
+const char* rattn_strerror(int status) {
+  switch (status) {
+    case RATTN_OK: return "ok";
+    case RATTN_ERR_BAD_ARG: return "size argument out of range";
+    case RATTN_ERR_NULL_PTR: return "required pointer is NULL";
+    case RATTN_ERR_MISALIGNED: return "pointer is not sufficiently aligned";
+    case RATTN_ERR_UNSUPPORTED: return "unsupported head size, dtype or mode";
+    case RATTN_ERR_WORKSPACE: return "workspace missing or too small";
+    case RATTN_ERR_CUDA: return "CUDA call failed (see rattn_last_cuda_error)";
+    case RATTN_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    default: return "unknown status";
+  }
+}
+
+int rattn_last_cuda_error(void) { return g_last_cuda_error; }
+
+uint64_t rattn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int rattn_uses_tensor_path(int d, int w, int dtype, int mode, unsigned flags) {
+  return tensor_path(d, w, dtype, mode, flags) ? 1 : 0;
+}
+
+}  // extern "C"

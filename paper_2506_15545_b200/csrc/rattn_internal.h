@@ -1,0 +1,78 @@
+// Internal declarations shared by the translation units of librattn.so.
+// Nothing here is part of the public ABI (include/rattn.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "rattn.h"
+
+namespace rattn {
+
+// Byte offsets inside the caller's workspace.  Every region is 256-byte aligned.
+struct WorkspaceLayout {
+  size_t status;        // 256 bytes; word 0 = device status, word 1 = detail code
+  size_t lse;           // fp32 [B,H_q,T]      log-sum-exp of the SWA logits (natural log)
+  size_t o_swa;         // fp32 [B,H_q,T,d]    un-normalised SWA branch output
+  size_t o_rla;         // fp32 [B,H_q,T,d]    un-normalised RLA branch output
+  size_t do_swa;        // fp32 [B,H_q,T,d]    backward scratch
+  size_t do_rla;        // fp32 [B,H_q,T,d]    backward scratch
+  size_t delta;         // fp32 [B,H_q,T]      backward scratch
+  size_t chunk_delta;   // fp32 [B,H_kv,n_chunks,d,d]  per-chunk phi(K)^T V
+  size_t chunk_state;   // bf16 [B,H_kv,n_chunks,d,d]  exclusive prefix over chunks
+  size_t total;
+  int n_chunks;         // ceil(T / 128)
+};
+
+WorkspaceLayout workspace_layout(int B, int H_q, int H_kv, int T, int d, int w, int dtype);
+
+// Resolved arguments handed to the kernel launchers (all device pointers).
+struct Args {
+  const void* q;
+  const void* k;
+  const void* v;
+  void* out;
+  int B, H_q, H_kv, T, d, w;   // w already replaced by T for FULL_CAUSAL
+  int group;                   // H_q / H_kv
+  int dtype, mode;
+  float scale, eps;
+  const float* gamma_swa;
+  const float* gamma_rla;
+  // residuals (may be null in inference mode)
+  float* lse;
+  float* o_swa;
+  float* o_rla;
+  // tensor-path scratch
+  float* chunk_delta;
+  __nv_bfloat16* chunk_state;
+  int n_chunks;
+  int* status;                 // device status word (may be null when no workspace)
+  // hand-off
+  float* state_out;
+  void* k_ring_out;
+  void* v_ring_out;
+  // backward
+  const void* dout;
+  void* dq;
+  void* dk;
+  void* dv;
+  float* dgamma_swa;
+  float* dgamma_rla;
+  float* do_swa;               // fp32 [B,H_q,T,d]  gradient w.r.t. the SWA branch output
+  float* do_rla;               // fp32 [B,H_q,T,d]  gradient w.r.t. the RLA branch output
+  float* delta;                // fp32 [B,H_q,T]    do_swa . o_swa per row
+};
+
+// Launchers; each returns the cudaError_t of its launches (cudaGetLastError).
+cudaError_t launch_generic_forward(const Args& a, cudaStream_t s);
+cudaError_t launch_generic_backward(const Args& a, cudaStream_t s);
+cudaError_t launch_decode(const Args& a, void* k_ring, void* v_ring, float* state, int pos,
+                          cudaStream_t s);
+cudaError_t launch_handoff(const Args& a, cudaStream_t s);
+cudaError_t launch_tc_forward(const Args& a, cudaStream_t s);
+
+void count_launches(int n);
+
+}  // namespace rattn

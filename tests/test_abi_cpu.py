@@ -1,0 +1,124 @@
+"""Host-side checks that need no GPU: the library builds, loads, exports every symbol the
+header declares, agrees with the binding on the parameter block, and rejects bad
+arguments before touching the device."""
+import ctypes
+import os
+import re
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "rattn.h")
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2506_15545_b200 import build, binding
+    build.build()
+    binding.lib()
+    return binding
+
+
+def _declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(rattn_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(B):
+    names = _declared_functions()
+    assert set(names) == set(B.EXPORTS)
+    for n in names:
+        assert hasattr(B.lib(), n), n
+
+
+def test_header_is_plain_c_and_struct_matches_binding(B, tmp_path):
+    src = tmp_path / "sz.c"
+    src.write_text('#include "rattn.h"\n#include <stdio.h>\n#include <stddef.h>\n'
+                   'int main(void){printf("%zu %zu %zu %zu\\n", sizeof(rattn_params),'
+                   'offsetof(rattn_params, workspace_bytes), offsetof(rattn_params, dout),'
+                   'offsetof(rattn_params, flags));return 0;}\n')
+    exe = tmp_path / "sz"
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"),
+                           str(src), "-o", str(exe)])
+    size, off_ws, off_dout, off_flags = map(int, subprocess.check_output([str(exe)]).split())
+    P = B.RattnParams
+    assert size == ctypes.sizeof(P)
+    assert off_ws == P.workspace_bytes.offset
+    assert off_dout == P.dout.offset
+    assert off_flags == P.flags.offset
+
+
+def test_strerror_and_workspace_bytes(B):
+    L = B.lib()
+    assert L.rattn_strerror(0) == b"ok"
+    for code in range(-7, 0):
+        assert L.rattn_strerror(code) not in (b"ok", b"unknown status")
+    assert L.rattn_strerror(-99) == b"unknown status"
+    n = B.rattn_workspace_bytes(4, 16, 16, 4096, 128, 512)
+    assert n > 0 and n % 256 == 0
+    assert B.rattn_workspace_bytes(4, 16, 16, 4096, 128, 512) == n          # pure function
+    assert B.rattn_workspace_bytes(8, 16, 16, 4096, 128, 512) > n
+    assert B.rattn_workspace_bytes(4, 16, 16, 4096, 96, 512) == 0           # unsupported d
+    assert B.rattn_workspace_bytes(4, 16, 5, 4096, 128, 512) == 0           # H_q % H_kv != 0
+    assert B.rattn_workspace_bytes(0, 16, 16, 4096, 128, 512) == 0
+
+
+def _p(bind, **kw):
+    p = bind.RattnParams()
+    fake = 0x10000                       # non-null, 16-byte aligned; never dereferenced
+    p.q = p.k = p.v = p.out = fake
+    p.B, p.H_q, p.H_kv, p.T, p.d, p.w = 1, 4, 2, 64, 64, 8
+    p.dtype, p.mode, p.scale, p.eps = bind.RATTN_F32, bind.MODE_RATTN, 1.0, 1e-6
+    for k, v in kw.items():
+        setattr(p, k, v)
+    return p
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(B=0), -1), (dict(T=0), -1), (dict(w=0), -1), (dict(H_kv=3), -1), (dict(eps=0.0), -1),
+    (dict(d=96), -4), (dict(dtype=7), -4), (dict(mode=5), -4),
+    (dict(q=0), -2), (dict(out=0), -2),
+    (dict(k=0x10008), -3), (dict(gamma_swa=0x10004), -3),
+    (dict(flags=2), -5),                                   # residuals wanted, no workspace
+    (dict(workspace=0x10100, workspace_bytes=16), -5),     # too small
+    (dict(workspace=0x10010, workspace_bytes=1 << 40), -3),  # workspace not 256-byte aligned
+    (dict(k_ring_out=0x10000), -2),                        # only one of the two rings
+])
+def test_forward_rejects_bad_arguments_without_launching(B, kw, code):
+    before = B.rattn_launch_count()
+    assert B.lib().rattn_forward_ex(ctypes.byref(_p(B, **kw)), None) == code
+    assert B.rattn_launch_count() == before
+
+
+def test_null_params_and_backward_and_decode_checks(B):
+    L = B.lib()
+    assert L.rattn_forward_ex(None, None) == -2
+    assert L.rattn_backward_ex(ctypes.byref(_p(B)), None) == -2           # no dout/dq/dk/dv
+    p = _p(B, dout=0x10000, dq=0x10000, dk=0x10000, dv=0x10000)
+    assert L.rattn_backward_ex(ctypes.byref(p), None) == -5               # no workspace
+    assert L.rattn_decode_step_ex(ctypes.byref(_p(B)), None, None, None, 0, None) == -2
+    assert L.rattn_decode_step_ex(ctypes.byref(_p(B)), 0x10000, 0x10000, 0x10000, -1, None) == -1
+    assert L.rattn_decode_step_ex(ctypes.byref(_p(B)), 0x10000, 0x10008, 0x10000, 0, None) == -3
+    assert L.rattn_read_status(None, None) == -2
+
+
+def test_path_selection_is_a_pure_host_decision(B):
+    assert not B.rattn_uses_tensor_path(64, 128)                         # d = 64: portable path
+    assert not B.rattn_uses_tensor_path(128, 100)                        # w not a tile multiple
+    assert not B.rattn_uses_tensor_path(128, 512, dtype=B.RATTN_F32)
+    assert not B.rattn_uses_tensor_path(128, 512, flags=B.FLAG_FORCE_GENERIC)
+
+
+def test_product_never_imports_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2506_15545_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower(), f
+    for f in os.listdir(os.path.join(ROOT, "oracle")):
+        if f.endswith(".py"):
+            assert "paper_2506_15545_b200" not in open(os.path.join(ROOT, "oracle", f)).read()
