@@ -186,6 +186,16 @@ int rattn_last_cuda_error(void);
  * (host counter; used by the benchmark to report its launch count). */
 uint64_t rattn_launch_count(void);
 
+/*
+ * Optional per-kernel device timing for benchmarks.  While enabled, every kernel the
+ * library launches is bracketed by a CUDA event pair on its stream.  Enabling or
+ * disabling clears the records.  rattn_timing_read waits for the recorded events, then
+ * writes one text line per kernel name, "name launches total_ms\n", NUL-terminated,
+ * into the HOST buffer `buf` (truncated to buf_bytes) and returns the bytes needed.
+ */
+int rattn_timing_enable(int on);
+size_t rattn_timing_read(char* buf, size_t buf_bytes);
+
 /* 1 when the tensor-core (tcgen05) forward would be chosen for these sizes. */
 int rattn_uses_tensor_path(int d, int w, int dtype, int mode, unsigned flags);
 

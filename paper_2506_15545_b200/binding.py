@@ -22,7 +22,7 @@ EXPORTS = (
     "rattn_forward", "rattn_forward_ex", "rattn_backward", "rattn_backward_ex",
     "rattn_decode_step", "rattn_decode_step_ex", "rattn_workspace_bytes",
     "rattn_read_status", "rattn_strerror", "rattn_last_cuda_error", "rattn_launch_count",
-    "rattn_uses_tensor_path",
+    "rattn_uses_tensor_path", "rattn_timing_enable", "rattn_timing_read",
 )
 
 
@@ -92,6 +92,10 @@ def lib() -> ctypes.CDLL:
     L.rattn_launch_count.restype = ctypes.c_uint64
     L.rattn_uses_tensor_path.argtypes = [ci, ci, ci, ci, ctypes.c_uint]
     L.rattn_uses_tensor_path.restype = ci
+    L.rattn_timing_enable.argtypes = [ci]
+    L.rattn_timing_enable.restype = ci
+    L.rattn_timing_read.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
+    L.rattn_timing_read.restype = ctypes.c_size_t
     _lib = L
     return L
 
@@ -242,3 +246,18 @@ def rattn_launch_count() -> int:
 
 def rattn_uses_tensor_path(d, w, dtype=RATTN_BF16, mode=MODE_RATTN, flags=0) -> bool:
     return bool(lib().rattn_uses_tensor_path(d, w, dtype, mode, flags))
+
+
+def rattn_timing_enable(on: bool) -> None:
+    lib().rattn_timing_enable(1 if on else 0)
+
+
+def rattn_timing_read() -> dict:
+    """{kernel name: (launches, total milliseconds)} since timing was enabled."""
+    buf = ctypes.create_string_buffer(1 << 16)
+    lib().rattn_timing_read(buf, len(buf))
+    out = {}
+    for line in buf.value.decode().splitlines():
+        name, n, ms = line.rsplit(" ", 2)
+        out[name] = (int(n), float(ms))
+    return out

@@ -318,7 +318,7 @@ cudaError_t launch_dec(const DecodeArgs& a, cudaStream_t s) {
   cudaError_t e = cudaFuncSetAttribute(decode_kernel<TIO, D>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  decode_kernel<TIO, D><<<a.B * a.H_kv, DEC_THREADS, smem, s>>>(a);
+  { KernelTimer kt("decode_step", s); decode_kernel<TIO, D><<<a.B * a.H_kv, DEC_THREADS, smem, s>>>(a); }
   count_launches(1);
   return cudaGetLastError();
 }

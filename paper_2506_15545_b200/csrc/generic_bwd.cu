@@ -377,7 +377,8 @@ cudaError_t launch_bwd(const Args& a, cudaStream_t s) {
     e = cudaMemsetAsync(a.dgamma_rla, 0, sizeof(float) * a.H_q * D, s);
     if (e != cudaSuccess) return e;
   }
-  bwd_preprocess_kernel<TIO, D><<<(unsigned)((n_rows + 7) / 8), 256, 0, s>>>(a, do_s, do_r, delta);
+  { KernelTimer kt("generic_bwd_preprocess", s);
+    bwd_preprocess_kernel<TIO, D><<<(unsigned)((n_rows + 7) / 8), 256, 0, s>>>(a, do_s, do_r, delta); }
   constexpr int LD = D + PAD;
   constexpr size_t smem_dq = (size_t)(4 * 32 * LD + 3 * 64 * LD + 32 * (64 + PAD) + 64) * sizeof(float);
   constexpr size_t smem_dkv = (size_t)(4 * 32 * LD + 3 * 64 * LD + 64 * (32 + PAD) + 64) * sizeof(float);
@@ -386,9 +387,9 @@ cudaError_t launch_bwd(const Args& a, cudaStream_t s) {
   e = cudaFuncSetAttribute(bwd_dkv_kernel<TIO, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_dkv);
   if (e != cudaSuccess) return e;
   dim3 gq((a.T + 31) / 32, a.B * a.H_q);
-  bwd_dq_kernel<TIO, D><<<gq, NT, smem_dq, s>>>(a, do_s, do_r, delta);
+  { KernelTimer kt("generic_bwd_dq", s); bwd_dq_kernel<TIO, D><<<gq, NT, smem_dq, s>>>(a, do_s, do_r, delta); }
   dim3 gk((a.T + 63) / 64, a.B * a.H_kv);
-  bwd_dkv_kernel<TIO, D><<<gk, NT, smem_dkv, s>>>(a, do_s, do_r, delta);
+  { KernelTimer kt("generic_bwd_dkv", s); bwd_dkv_kernel<TIO, D><<<gk, NT, smem_dkv, s>>>(a, do_s, do_r, delta); }
   count_launches(3);
   return cudaGetLastError();
 }

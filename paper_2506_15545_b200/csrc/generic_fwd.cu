@@ -176,7 +176,7 @@ cudaError_t launch_fwd(const Args& a, cudaStream_t s) {
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid((a.T + BM - 1) / BM, a.B * a.H_q);
-  generic_fwd_kernel<TIO, D><<<grid, NT, smem, s>>>(a);
+  { KernelTimer kt("generic_fwd", s); generic_fwd_kernel<TIO, D><<<grid, NT, smem, s>>>(a); }
   count_launches(1);
   return cudaGetLastError();
 }

@@ -1,7 +1,12 @@
 // C ABI of librattn.so: argument checks, workspace carving, path selection.
 // See include/rattn.h for the contract of every entry point.
 #include <atomic>
+#include <cstdio>
 #include <cstring>
+#include <map>
+#include <mutex>
+#include <string>
+#include <vector>
 
 #include "rattn_internal.h"
 
@@ -11,6 +16,36 @@ static std::atomic<uint64_t> g_launches{0};
 static thread_local int g_last_cuda_error = 0;
 
 void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+// ---- optional per-kernel timing ------------------------------------------------------
+struct TimingRecord { const char* name; cudaEvent_t begin, end; };
+static std::mutex g_timing_mu;
+static std::vector<TimingRecord> g_timing;
+static std::atomic<int> g_timing_on{0};
+constexpr size_t kMaxTimingRecords = 1 << 16;
+
+KernelTimer::KernelTimer(const char* name, cudaStream_t s) : stream_(s), slot_(-1) {
+  if (!g_timing_on.load(std::memory_order_relaxed)) return;
+  std::lock_guard<std::mutex> lk(g_timing_mu);
+  if (g_timing.size() >= kMaxTimingRecords) return;
+  TimingRecord r{name, nullptr, nullptr};
+  if (cudaEventCreate(&r.begin) != cudaSuccess) return;
+  if (cudaEventCreate(&r.end) != cudaSuccess) { cudaEventDestroy(r.begin); return; }
+  cudaEventRecord(r.begin, s);
+  g_timing.push_back(r);
+  slot_ = (int)g_timing.size() - 1;
+}
+
+KernelTimer::~KernelTimer() {
+  if (slot_ < 0) return;
+  std::lock_guard<std::mutex> lk(g_timing_mu);
+  if (slot_ < (int)g_timing.size()) cudaEventRecord(g_timing[slot_].end, stream_);
+}
+
+static void timing_clear_locked() {
+  for (auto& r : g_timing) { cudaEventDestroy(r.begin); cudaEventDestroy(r.end); }
+  g_timing.clear();
+}
 
 static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
@@ -89,7 +124,7 @@ static bool tensor_path(int d, int w, int dtype, int mode, unsigned flags) {
 #ifdef RATTN_HAVE_TC
   if (flags & RATTN_FLAG_FORCE_GENERIC) return false;
   if (dtype != RATTN_BF16 || d != 128) return false;
-  if (mode == RATTN_MODE_RATTN && (w % 128) != 0) return false;
+  if (mode != RATTN_MODE_FULL_CAUSAL && (w % 128) != 0) return false;
   return true;
 #else
   (void)d; (void)w; (void)dtype; (void)mode; (void)flags;
@@ -265,6 +300,38 @@ const char* rattn_strerror(int status) {
 int rattn_last_cuda_error(void) { return g_last_cuda_error; }
 
 uint64_t rattn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int rattn_timing_enable(int on) {
+  std::lock_guard<std::mutex> lk(g_timing_mu);
+  timing_clear_locked();
+  g_timing_on.store(on ? 1 : 0, std::memory_order_relaxed);
+  return RATTN_OK;
+}
+
+size_t rattn_timing_read(char* buf, size_t buf_bytes) {
+  std::lock_guard<std::mutex> lk(g_timing_mu);
+  std::map<std::string, std::pair<long, double>> acc;
+  for (auto& r : g_timing) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(r.end) != cudaSuccess) continue;
+    if (cudaEventElapsedTime(&ms, r.begin, r.end) != cudaSuccess) continue;
+    auto& e = acc[r.name];
+    e.first += 1;
+    e.second += ms;
+  }
+  std::string out;
+  char line[256];
+  for (auto& kv : acc) {
+    std::snprintf(line, sizeof(line), "%s %ld %.6f\n", kv.first.c_str(), kv.second.first, kv.second.second);
+    out += line;
+  }
+  if (buf && buf_bytes > 0) {
+    const size_t n = out.size() < buf_bytes - 1 ? out.size() : buf_bytes - 1;
+    std::memcpy(buf, out.data(), n);
+    buf[n] = 0;
+  }
+  return out.size() + 1;
+}
 
 int rattn_uses_tensor_path(int d, int w, int dtype, int mode, unsigned flags) {
   return tensor_path(d, w, dtype, mode, flags) ? 1 : 0;

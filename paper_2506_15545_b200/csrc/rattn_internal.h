@@ -75,4 +75,15 @@ cudaError_t launch_tc_forward(const Args& a, cudaStream_t s);
 
 void count_launches(int n);
 
+// Records a CUDA event pair around one kernel launch on its stream while per-kernel
+// timing is enabled (rattn_timing_enable); free otherwise.
+class KernelTimer {
+ public:
+  KernelTimer(const char* name, cudaStream_t s);
+  ~KernelTimer();
+ private:
+  cudaStream_t stream_;
+  int slot_;
+};
+
 }  // namespace rattn

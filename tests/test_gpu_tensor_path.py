@@ -1,0 +1,98 @@
+"""Parity of the tensor-core (tcgen05) forward against the fp64 oracle: bf16, d = 128,
+window a multiple of 128.  Same tolerances as the portable path: max-abs <= 2e-2,
+mean-abs <= 2e-3 on outputs that are the sum of two unit-RMS vectors."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import rattn_oracle as O
+from paper_2506_15545_b200 import binding as R
+from paper_2506_15545_b200 import workloads as W
+from test_gpu_parity import check, np64, small
+
+pytestmark = pytest.mark.gpu
+
+
+def run(wl, mode=R.MODE_RATTN, gains=True, save=False):
+    assert R.rattn_uses_tensor_path(wl.d, wl.w, R.RATTN_BF16, mode)
+    q, k, v = W.make_qkv(wl)
+    gs, gr = W.make_gains(wl) if gains else (None, None)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    ws = R.alloc_workspace(qd, kd, wl.w)
+    ws.zero_()
+    y = R.rattn_forward_ex(qd, kd, vd, wl.w, scale=wl.scale, mode=mode, workspace=ws,
+                           gamma_swa=None if gs is None else gs.cuda(),
+                           gamma_rla=None if gr is None else gr.cuda(), save_residuals=save)
+    torch.cuda.synchronize()
+    assert R.rattn_read_status(ws) == 0, "a device-side wait expired"
+    ref = O.forward(np64(q), np64(k), np64(v), wl.w, wl.scale, 1e-6,
+                    None if gs is None else np64(gs), None if gr is None else np64(gr), mode)
+    return y, ref, (qd, kd, vd, ws)
+
+
+@pytest.mark.parametrize("T,w,Hq,Hkv,unit", [
+    (128, 128, 1, 1, False),     # one tile, nothing outside the window
+    (256, 128, 1, 1, False),     # second tile reads chunk 0 in intra form, no stored state
+    (384, 128, 2, 1, True),      # third tile: stored state of chunk 0 + intra form of chunk 1
+    (1024, 256, 4, 2, True),     # window of two tiles, GQA
+    (1280, 512, 2, 2, False),    # the w = 512 band: five key tiles
+    (300, 128, 2, 1, False),     # ragged T: last tile partly beyond the sequence
+    (77, 128, 2, 2, False),      # T below one tile
+    (640, 1024, 2, 1, True),     # w > T: SWA covers everything
+])
+def test_tensor_forward_shapes(T, w, Hq, Hkv, unit):
+    wl = small("tc", 2, Hq, Hkv, T, 128, w, "bf16", 4000 + T + w, unit=unit)
+    y, ref, _ = run(wl)
+    check(y, ref, "bf16", f"T={T} w={w}")
+
+
+@pytest.mark.parametrize("mode", [R.MODE_SWA_ONLY, R.MODE_FULL_CAUSAL])
+def test_tensor_forward_control_modes(mode):
+    wl = small("tcm", 1, 4, 2, 896, 128, 256, "bf16", 4100, unit=True)
+    y, ref, _ = run(wl, mode=mode)
+    check(y, ref, "bf16", f"mode={mode}")
+
+
+def test_tensor_forward_large_logits_trigger_rescale():
+    """Un-normalised q, k with scale 1/4: logits of std ~ 30, so the running maximum moves by
+    far more than the lazy-rescale threshold between key tiles."""
+    wl = small("tcr", 1, 2, 2, 768, 128, 256, "bf16", 4200, unit=False, scale=0.25)
+    y, ref, _ = run(wl)
+    check(y, ref, "bf16", "large logits")
+
+
+def test_tensor_forward_c2_like_heads():
+    """Config 2's sequence (T=4096, w=512, unit-RMS q/k, scale 1/sqrt(128)) on two heads."""
+    wl = W.C2.replace(B=1, H_q=2, H_kv=2)
+    y, ref, _ = run(wl, gains=False)
+    check(y, ref, "bf16", "c2 heads")
+
+
+def test_tensor_residuals_match_portable_path():
+    wl = small("tcs", 1, 2, 1, 512, 128, 128, "bf16", 4300, unit=True)
+    y, ref, (q, k, v, ws) = run(wl, save=True)
+    ws2 = torch.zeros_like(ws)
+    y2 = R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws2, save_residuals=True,
+                            gamma_swa=W.make_gains(wl)[0].cuda(), gamma_rla=W.make_gains(wl)[1].cuda(),
+                            flags=R.FLAG_FORCE_GENERIC)
+    torch.cuda.synchronize()
+    n = 2 * 512
+    f1 = ws[256:].view(torch.float32)
+    f2 = ws2[256:].view(torch.float32)
+    lse1, lse2 = f1[:n], f2[:n]
+    assert (lse1 - lse2).abs().max() < 2e-2
+    off = ((n * 4 + 255) // 256 * 256) // 4
+    o1, o2 = f1[off:off + n * 128], f2[off:off + n * 128]
+    assert (o1 - o2).abs().max() < 3e-2
+    check(y, ref, "bf16")
+
+
+def test_tensor_run_to_run_determinism():
+    wl = small("tcd", 2, 2, 1, 1024, 128, 256, "bf16", 4400, unit=True)
+    q, k, v = (t.cuda() for t in W.make_qkv(wl))
+    ws = R.alloc_workspace(q, k, wl.w)
+    a = R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws).clone()
+    b = R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws)
+    assert torch.equal(a, b)
