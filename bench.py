@@ -1,0 +1,405 @@
+#!/usr/bin/env python
+"""Benchmark of the RAttention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one training step of one RAttention layer on the "c4_train_step" workload
+(B=8, H_q=H_kv=16, T=4096, d=128, w=512, bf16): forward with residuals + backward
+(dq, dk, dv), through the C ABI.  `value` is algorithmic TFLOP/s of that step (band pairs
+and recurrent-form RLA only: masked tile halves and recomputation are not counted).
+The forward-only configuration (c2) and one decode step (c5 shapes) are timed beside it
+and reported under "extra".  Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2506_15545_b200 import workloads as W  # noqa: E402
+
+METRIC = "RAttention fwd+bwd TFLOP/s (T=4096,w=512,d=128,bf16)"
+
+
+# --------------------------------------------------------------------------- work model
+def n_swa_pairs(T, w):
+    w = min(w, T - 1)
+    return (w + 1) * T - w * (w + 1) // 2
+
+
+def flops(wl, what):
+    """Algorithmic FLOPs.  SWA fwd 4*d per band pair and query head; RLA fwd 2*d^2 per
+    residual row and query head (read-out) + 2*d^2 per absorbed token and K/V head (state
+    update); backward: SWA 10*d per pair (five products), RLA 4*d^2 + 4*d^2."""
+    d, T, w = wl.d, wl.T, wl.w
+    n = n_swa_pairs(T, w)
+    rows = max(0, T - w - 1)
+    bq, bkv = wl.B * wl.H_q, wl.B * wl.H_kv
+    fwd_swa = 4 * d * n * bq
+    fwd_read = 2 * d * d * rows * bq
+    fwd_upd = 2 * d * d * rows * bkv
+    parts = {
+        "fwd": fwd_swa + fwd_read + fwd_upd,
+        "fwd_main": fwd_swa + fwd_read,
+        "fwd_state": fwd_upd,
+        "bwd": 10 * d * n * bq + 4 * d * d * rows * bq + 4 * d * d * rows * bkv,
+        "bwd_dq": 4 * d * n * bq + 2 * d * d * rows * bq,
+        "bwd_dkv": 6 * d * n * bq + 2 * d * d * rows * bq + 4 * d * d * rows * bkv,
+    }
+    parts["step"] = parts["fwd"] + parts["bwd"]
+    return parts[what]
+
+
+def io_bytes_fwd(wl):
+    e = 2 if wl.dtype == "bf16" else 4
+    return e * wl.d * wl.T * wl.B * (2 * wl.H_q + 2 * wl.H_kv)
+
+
+def decode_bytes(wl):
+    e = 2
+    ring = 2 * wl.B * wl.H_kv * wl.w * wl.d * e
+    state = 2 * wl.B * wl.H_kv * wl.d * wl.d * 4
+    tok = wl.B * (2 * wl.H_q + 2 * wl.H_kv) * wl.d * e
+    return ring + state + tok
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return dict(hbm=j["hbm_gbs"], tf_burst=j["bf16_tflops"], tf_sus=j["bf16_tflops_sustained"],
+                    src="measured")
+    return dict(hbm=6650.0, tf_burst=1590.0, tf_sus=1400.0, src="fallback")
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(index)], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1]))
+                mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        os.unlink(self.f.name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------ reference arm
+def oracle_step(wl, q, k, v, dy, head):
+    """One bounded sample of the workload through the fp64 oracle: forward + backward of one
+    (batch, head) pair at the full sequence length."""
+    from oracle import rattn_oracle as O
+    b, h = divmod(head, wl.H_q)
+    g = wl.H_q // wl.H_kv
+    q64, k64, v64, dy64 = (t.to(torch.float64).numpy() for t in (q[b, h], k[b, h // g], v[b, h // g], dy[b, h]))
+    O.forward_head(q64, k64, v64, wl.w, wl.scale)
+    O.backward_head(q64, k64, v64, dy64, wl.w, wl.scale)
+
+
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return len(os.sched_getaffinity(0))
+
+
+def head_flops(wl):
+    one = wl.replace(B=1, H_q=1, H_kv=1)
+    return flops(one, "step")
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    small = wl.replace(B=1, H_q=min(4, wl.H_q), H_kv=min(4, wl.H_kv))
+    q, k, v = W.make_qkv(small)
+    dy = W.make_dout(small)
+    for i in range(args.warmup):
+        oracle_step(small, q, k, v, dy, i % small.H_q)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        oracle_step(small, q, k, v, dy, i % small.H_q)
+    dt = time.perf_counter() - t0
+    val = head_flops(wl) * args.steps / dt / 1e12
+    cores = oracle_threads()
+    sample = "each step = forward+backward of one (batch, head) pair at T=4096 through the fp64 oracle"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": workload_name(wl), "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_name(wl):
+    return (f"{wl.name}: B={wl.B},H_q={wl.H_q},H_kv={wl.H_kv},T={wl.T},d={wl.d},w={wl.w},{wl.dtype} "
+            "forward(with residuals)+backward")
+
+
+# ----------------------------------------------------------------------------- our arm
+def timed(fn, steps, warmup, sync):
+    for _ in range(warmup):
+        fn()
+    sync()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(steps):
+        fn()
+    b.record()
+    sync()
+    return a.elapsed_time(b) / steps
+
+
+def run_ours(args, wl):
+    from paper_2506_15545_b200 import binding as R
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    R.lib()
+    pk = peaks()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # every rank runs the same per-GPU workload (independent replicas of the layer's batch)
+    wl_r = wl.replace(seed=wl.seed + rank)
+    q, k, v = W.make_qkv(wl_r, dev)
+    dy = W.make_dout(wl_r, dev)
+    ws = R.alloc_workspace(q, k, wl.w)
+    out = torch.empty_like(q)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+
+    def step():
+        R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws, save_residuals=True, out=out)
+        R.rattn_backward_ex(q, k, v, dy, wl.w, ws, scale=wl.scale, dq=dq, dk=dk, dv=dv)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    R.rattn_timing_enable(True)
+    launches0 = R.rattn_launch_count()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        step()
+    b.record()
+    barrier()
+    ms = a.elapsed_time(b) / args.steps
+    launches = R.rattn_launch_count() - launches0
+    kernel_ms = R.rattn_timing_read()
+    R.rattn_timing_enable(False)
+    clocks = sampler.stop() if sampler else None
+    assert R.rattn_read_status(ws) == 0, "device-side wait expired"
+    if dist is not None:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = flops(wl, "step") * world / (ms * 1e-3) / 1e12
+
+    # ---- dominant kernel and its roofline -------------------------------------------
+    per_launch = {n: tot / cnt for n, (cnt, tot) in kernel_ms.items() if cnt}
+    share = {n: tot for n, (cnt, tot) in kernel_ms.items()}
+    top = max(share, key=share.get)
+    kflops = {"tc_fwd": "fwd_main", "tc_chunk_delta": "fwd_state", "generic_fwd": "fwd",
+              "generic_bwd_dq": "bwd_dq", "generic_bwd_dkv": "bwd_dkv"}
+    roof = None
+    if top in kflops:
+        ach = flops(wl, kflops[top]) / (per_launch[top] * 1e-3) / 1e12
+        roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": pk["tf_sus"], "unit": "TFLOP/s",
+                "frac": ach / pk["tf_sus"], "traffic": None, "peak_source": pk["src"] + " (sustained bf16)",
+                "ms_per_launch": per_launch[top]}
+    total_k = sum(share.values())
+    kernels = {n: {"launches": kernel_ms[n][0], "ms_per_launch": per_launch[n], "share": share[n] / total_k}
+               for n in share}
+
+    result = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": workload_name(wl), "global_batch": wl.B * world,
+                   "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                   "l2": "inputs larger than L2 (q,k,v,dO,residuals > 1 GB per step)"},
+        "tokens_per_s": wl.B * wl.T * world / (ms * 1e-3),
+        "gpu_launches": int(launches), "kernels": kernels, "roofline": roof, "clocks": clocks,
+    }
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- extra: forward-only (c2) and decode (c5 shapes), device-resident -----------
+    extra = {}
+    sync = torch.cuda.synchronize
+    del dq, dk, dv, dy
+    c2 = W.C2
+    q2, k2, v2 = W.make_qkv(c2, dev)
+    ws2 = R.alloc_workspace(q2, k2, c2.w)
+    # rotate three input sets (3 x 268 MB > L2) so no launch finds its inputs in L2
+    sets = [(q2, k2, v2)] + [tuple(t.clone() for t in (q2, k2, v2)) for _ in range(2)]
+    o2 = torch.empty_like(q2)
+    it = [0]
+
+    def fwd_only():
+        s = sets[it[0] % 3]
+        it[0] += 1
+        R.rattn_forward_ex(s[0], s[1], s[2], c2.w, scale=c2.scale, workspace=ws2, out=o2)
+
+    R.rattn_timing_enable(True)
+    ms_f = timed(fwd_only, 30, 5, sync)
+    kf = R.rattn_timing_read()
+    R.rattn_timing_enable(False)
+    t_roof = max(flops(c2, "fwd") / (pk["tf_burst"] * 1e12), io_bytes_fwd(c2) / (pk["hbm"] * 1e9))
+    extra["fwd_c2"] = {
+        "workload": "c2_3b_fwd: B=4,H=16/16,T=4096,d=128,w=512 forward only, 3 rotating input sets",
+        "ms": ms_f, "tflops": flops(c2, "fwd") / (ms_f * 1e-3) / 1e12,
+        "tokens_per_s": c2.B * c2.T / (ms_f * 1e-3),
+        "roofline_ms": t_roof * 1e3, "roofline_frac": t_roof * 1e3 / ms_f,
+        "roofline_denominator": f"max(FLOPs/{pk['tf_burst']} TF/s burst, bytes/{pk['hbm']} GB/s), {pk['src']}",
+        "kernels_ms_per_launch": {n: tot / cnt for n, (cnt, tot) in kf.items() if cnt},
+    }
+    del sets, q2, k2, v2, ws2, o2
+
+    c5 = W.C5
+    rings = []
+    for i in range(2):      # two cache sets: 2 x (67 MB ring + 17 MB state) > L2 together with q,k,v
+        rings.append((torch.randn(c5.B, c5.H_kv, c5.w, c5.d, device=dev).to(torch.bfloat16),
+                      torch.randn(c5.B, c5.H_kv, c5.w, c5.d, device=dev).to(torch.bfloat16),
+                      torch.zeros(c5.B, c5.H_kv, c5.d, c5.d, device=dev)))
+    qd, kd, vd = W.make_decode_token(c5, 0, dev)
+    od = torch.empty_like(qd)
+    pos = [c5.T]
+
+    def dec():
+        r = rings[pos[0] & 1]
+        R.rattn_decode_step_ex(qd, kd, vd, r[0], r[1], r[2], pos[0], scale=c5.scale, out=od)
+        pos[0] += 1
+
+    ms_d = timed(dec, 100, 10, sync)
+    extra["decode_c5"] = {
+        "workload": "one decode step, B=32,H=32/8,d=128,w=512, two rotating cache sets",
+        "ms": ms_d, "gb_per_s": decode_bytes(c5) / (ms_d * 1e-3) / 1e9,
+        "roofline_frac": decode_bytes(c5) / (ms_d * 1e-3) / 1e9 / pk["hbm"],
+        "tokens_per_s": c5.B / (ms_d * 1e-3),
+        "roofline_denominator": f"{pk['hbm']} GB/s HBM copy, {pk['src']}",
+    }
+    del rings
+    result["extra"] = extra
+
+    # ---- end to end: host buffers in, gradients out, through the same calls ----------
+    hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
+    hdy = W.make_dout(wl_r, "cpu").pin_memory()
+    dy_d = torch.empty_like(q)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    h_dq, h_dk, h_dv = (torch.empty_like(t, device="cpu").pin_memory() for t in (dq, dk, dv))
+
+    def e2e_step():
+        q.copy_(hq, non_blocking=True)
+        k.copy_(hk, non_blocking=True)
+        v.copy_(hv, non_blocking=True)
+        dy_d.copy_(hdy, non_blocking=True)
+        R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws, save_residuals=True, out=out)
+        R.rattn_backward_ex(q, k, v, dy_d, wl.w, ws, scale=wl.scale, dq=dq, dk=dk, dv=dv)
+        h_dq.copy_(dq, non_blocking=True)
+        h_dk.copy_(dk, non_blocking=True)
+        h_dv.copy_(dv, non_blocking=True)
+
+    ms_e = timed(e2e_step, max(2, min(args.steps, 5)), 1, sync)
+    nbytes = lambda *ts: int(sum(t.numel() * t.element_size() for t in ts))
+    result["e2e"] = {"value": flops(wl, "step") / (ms_e * 1e-3) / 1e12, "unit": "TFLOP/s",
+                     "ms_per_step": ms_e, "h2d_bytes_per_step": nbytes(hq, hk, hv, hdy),
+                     "d2h_bytes_per_step": nbytes(h_dq, h_dk, h_dv)}
+
+    # ---- CPU baseline: the oracle, as it stands, on a bounded sample ------------------
+    if world == 1:
+        n_heads = 6
+        qc, kc, vc, dyc = hq, hk, hv, hdy
+        t0 = time.perf_counter()
+        for i in range(n_heads):
+            oracle_step(wl, qc, kc, vc, dyc, i * 7 % (wl.B * wl.H_q))
+        dt = time.perf_counter() - t0
+        result["cpu_baseline"] = {
+            "value": head_flops(wl) * n_heads / dt / 1e12, "unit": "TFLOP/s", "cores": oracle_threads(),
+            "kind": "oracle", "seconds": dt,
+            "sample": f"{n_heads} of {wl.B * wl.H_q} (batch, head) pairs, forward+backward at full T=4096",
+        }
+    print(json.dumps(result))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    wl = W.C4
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()
