@@ -46,7 +46,8 @@ typedef enum rattn_status {
   RATTN_ERR_UNSUPPORTED = -4,    /* d not in {64,128}, unknown dtype / mode */
   RATTN_ERR_WORKSPACE = -5,      /* workspace missing or smaller than rattn_workspace_bytes() */
   RATTN_ERR_CUDA = -6,           /* a CUDA call failed; see rattn_last_cuda_error() */
-  RATTN_ERR_TIMEOUT = -7         /* a bounded device-side wait expired (status word) */
+  RATTN_ERR_TIMEOUT = -7,        /* a bounded device-side wait expired (status word) */
+  RATTN_ERR_STATIC_LIMIT = -8    /* rattn_forward_static: sizes exceed its fixed scratch */
 } rattn_status;
 
 typedef enum rattn_dtype { RATTN_BF16 = 0, RATTN_F32 = 1 } rattn_dtype;
@@ -122,6 +123,34 @@ typedef struct rattn_params {
 int rattn_forward(const void* q, const void* k, const void* v,
                   int B, int H_q, int H_kv, int T, int d, int w,
                   void* out, void* stream);
+
+/*
+ * Forward that allocates nothing (the paper has no counterpart; this exists for the sake
+ * of callers, not of the method).  Same operator and conventions as rattn_forward (bf16,
+ * unit gains, eps = 1e-6, inference) with an explicit logit `scale`.
+ *
+ * Who needs it: code that is not in a position to obtain device memory at call time and
+ * has no workspace to pass -- a server whose own cache manager already owns all of the
+ * GPU's memory, an operator plugged into another framework that cannot reach that
+ * framework's allocator, a latency-bound loop that must stay clear of the driver's
+ * allocation lock.  Where the tensor-core path applies (d = 128, w % 128 == 0) its chunk
+ * states go into a fixed array inside the library instead: RATTN_STATIC_MAX_CHUNK_STATES
+ * matrices of 128 x 128 (6 MiB in all, held by every GPU that loads the library until the
+ * process exits).  The call is refused with RATTN_ERR_STATIC_LIMIT when
+ * B * H_kv * ceil(T / 128) exceeds that number; other shapes run the portable kernel,
+ * which needs no scratch, so they are never refused for size.
+ *
+ * The call itself makes no cudaMalloc / cudaFree / pool allocation.  The first call on
+ * each device looks up the array's device address (a one-time set-up step; make that
+ * first call outside any stream capture).  All calls on a device share the one array and
+ * it keeps the previous call's contents (the library clears the part that must start at
+ * zero): two calls whose kernels may overlap on the GPU -- different streams, no ordering
+ * between them -- race on it, so serialise them.
+ */
+#define RATTN_STATIC_MAX_CHUNK_STATES 64
+int rattn_forward_static(const void* q, const void* k, const void* v,
+                         int B, int H_q, int H_kv, int T, int d, int w, float scale,
+                         void* out, void* stream);
 
 /* Forward with the full parameter block (dtype, scale, gains, mode, workspace,
  * residuals for the backward, prefill -> decode hand-off). */

@@ -23,6 +23,7 @@ EXPORTS = (
     "rattn_decode_step", "rattn_decode_step_ex", "rattn_workspace_bytes",
     "rattn_read_status", "rattn_strerror", "rattn_last_cuda_error", "rattn_launch_count",
     "rattn_uses_tensor_path", "rattn_timing_enable", "rattn_timing_read",
+    "rattn_forward_static",
 )
 
 
@@ -92,6 +93,8 @@ def lib() -> ctypes.CDLL:
     L.rattn_launch_count.restype = ctypes.c_uint64
     L.rattn_uses_tensor_path.argtypes = [ci, ci, ci, ci, ctypes.c_uint]
     L.rattn_uses_tensor_path.restype = ci
+    L.rattn_forward_static.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp]
+    L.rattn_forward_static.restype = ci
     L.rattn_timing_enable.argtypes = [ci]
     L.rattn_timing_enable.restype = ci
     L.rattn_timing_read.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
@@ -168,6 +171,18 @@ def rattn_forward(q, k, v, w, out=None, stream=None):
     out = torch.empty_like(q) if out is None else out
     _check(lib().rattn_forward(_ptr(q), _ptr(k), _ptr(v), B, H_q, k.shape[1], T, d, w, _ptr(out),
                                _stream(stream)), "rattn_forward")
+    return out
+
+
+def rattn_forward_static(q, k, v, w, scale=1.0, out=None, stream=None):
+    """rattn_forward_static: the forward that allocates nothing on the library side (its
+    scratch is a fixed array inside the library).  `out` may be passed in so that the call
+    allocates nothing on the Python side either."""
+    _dense(q, k, v, out)
+    B, H_q, T, d = q.shape
+    out = torch.empty_like(q) if out is None else out
+    _check(lib().rattn_forward_static(_ptr(q), _ptr(k), _ptr(v), B, H_q, k.shape[1], T, d, w, scale,
+                                      _ptr(out), _stream(stream)), "rattn_forward_static")
     return out
 
 

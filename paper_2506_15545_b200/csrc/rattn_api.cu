@@ -16,6 +16,7 @@ static std::atomic<uint64_t> g_launches{0};
 static thread_local int g_last_cuda_error = 0;
 
 void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+void set_last_cuda_error(int cuda_error) { g_last_cuda_error = cuda_error; }
 
 // ---- optional per-kernel timing ------------------------------------------------------
 struct TimingRecord { const char* name; cudaEvent_t begin, end; };
@@ -293,6 +294,7 @@ const char* rattn_strerror(int status) {
     case RATTN_ERR_WORKSPACE: return "workspace missing or too small";
     case RATTN_ERR_CUDA: return "CUDA call failed (see rattn_last_cuda_error)";
     case RATTN_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    case RATTN_ERR_STATIC_LIMIT: return "problem needs more chunk states than rattn_forward_static's fixed scratch holds";
     default: return "unknown status";
   }
 }

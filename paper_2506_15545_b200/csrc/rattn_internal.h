@@ -74,6 +74,7 @@ cudaError_t launch_handoff(const Args& a, cudaStream_t s);
 cudaError_t launch_tc_forward(const Args& a, cudaStream_t s);
 
 void count_launches(int n);
+void set_last_cuda_error(int cuda_error);   // what rattn_last_cuda_error() reports for this thread
 
 // Records a CUDA event pair around one kernel launch on its stream while per-kernel
 // timing is enabled (rattn_timing_enable); free otherwise.
