@@ -387,13 +387,64 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
+def run_case(args):
+    """One small, single-kernel-family case for profiler captures (`--case`): a few launches
+    of one entry point on inputs a little larger than L2, no clocks sampling, no oracle."""
+    from paper_2506_15545_b200 import binding as R
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    sync = torch.cuda.synchronize
+    if args.case in ("fwd", "train"):
+        wl = W.C2.replace(B=2)          # q,k,v,out = 134 MB
+        q, k, v = W.make_qkv(wl, dev)
+        ws = R.alloc_workspace(q, k, wl.w)
+        out = torch.empty_like(q)
+        if args.case == "fwd":
+            fn = lambda: R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws, out=out)
+            fl = flops(wl, "fwd")
+        else:
+            dy = W.make_dout(wl, dev)
+            dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+
+            def fn():
+                R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws, save_residuals=True, out=out)
+                R.rattn_backward_ex(q, k, v, dy, wl.w, ws, scale=wl.scale, dq=dq, dk=dk, dv=dv)
+            fl = flops(wl, "step")
+        R.rattn_timing_enable(True)
+        ms = timed(fn, args.steps, args.warmup, sync)
+        km = R.rattn_timing_read()
+        assert R.rattn_read_status(ws) == 0
+        print(json.dumps({"case": args.case, "workload": workload_name(wl), "ms": ms,
+                          "tflops": fl / (ms * 1e-3) / 1e12,
+                          "kernels_ms_per_launch": {n: t / c for n, (c, t) in km.items() if c}}))
+    else:
+        c5 = W.C5
+        kr = torch.randn(c5.B, c5.H_kv, c5.w, c5.d, device=dev).to(torch.bfloat16)
+        vr = torch.randn(c5.B, c5.H_kv, c5.w, c5.d, device=dev).to(torch.bfloat16)
+        st = torch.zeros(c5.B, c5.H_kv, c5.d, c5.d, device=dev)
+        qd, kd, vd = W.make_decode_token(c5, 0, dev)
+        od = torch.empty_like(qd)
+        pos = [c5.T]
+
+        def fn():
+            R.rattn_decode_step_ex(qd, kd, vd, kr, vr, st, pos[0], scale=c5.scale, out=od)
+            pos[0] += 1
+        ms = timed(fn, args.steps, args.warmup, sync)
+        print(json.dumps({"case": "decode", "ms": ms, "gb_per_s": decode_bytes(c5) / (ms * 1e-3) / 1e9}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--case", default=None, choices=["fwd", "train", "decode"],
+                    help="run one small case (for profiler captures) instead of the benchmark")
     args = ap.parse_args()
+    if args.case:
+        run_case(args)
+        return
     wl = W.C4
     if args.impl == "reference":
         run_reference(args, wl)

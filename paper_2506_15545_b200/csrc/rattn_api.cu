@@ -67,6 +67,7 @@ WorkspaceLayout workspace_layout(int B, int H_q, int H_kv, int T, int d, int w, 
   const size_t states = (size_t)B * H_kv * L.n_chunks * d * d;
   L.chunk_delta = off; off += align256(states * sizeof(float));
   L.chunk_state = off; off += align256(states * sizeof(__nv_bfloat16));
+  L.rstate = off;      off += align256(states * sizeof(__nv_bfloat16));
   L.total = off;
   return L;
 }
@@ -117,6 +118,7 @@ static int bind_workspace(const rattn_params* p, Args* a, bool required) {
   a->delta = reinterpret_cast<float*>(base + L.delta);
   a->chunk_delta = reinterpret_cast<float*>(base + L.chunk_delta);
   a->chunk_state = reinterpret_cast<__nv_bfloat16*>(base + L.chunk_state);
+  a->rstate = reinterpret_cast<__nv_bfloat16*>(base + L.rstate);
   a->n_chunks = L.n_chunks;
   return RATTN_OK;
 }
@@ -183,7 +185,14 @@ static int backward_impl(const rattn_params* p, cudaStream_t s) {
   if (rc != RATTN_OK) return rc;
   a.dout = p->dout; a.dq = p->dq; a.dk = p->dk; a.dv = p->dv;
   a.dgamma_swa = p->dgamma_swa; a.dgamma_rla = p->dgamma_rla;
-  cudaError_t e = launch_generic_backward(a, s);
+  cudaError_t e;
+#ifdef RATTN_HAVE_TC
+  // The tensor-core backward reads the chunk states the tensor-core forward left in the
+  // workspace: both calls must take the same path (same sizes, mode and flags).
+  if (tensor_path(p->d, a.w, p->dtype, p->mode, p->flags)) e = launch_tc_backward(a, s);
+  else
+#endif
+    e = launch_generic_backward(a, s);
   if (e != cudaSuccess) return fail_cuda(e);
   return RATTN_OK;
 }

@@ -17,11 +17,12 @@ struct WorkspaceLayout {
   size_t lse;           // fp32 [B,H_q,T]      log-sum-exp of the SWA logits (natural log)
   size_t o_swa;         // fp32 [B,H_q,T,d]    un-normalised SWA branch output
   size_t o_rla;         // fp32 [B,H_q,T,d]    un-normalised RLA branch output
-  size_t do_swa;        // fp32 [B,H_q,T,d]    backward scratch
-  size_t do_rla;        // fp32 [B,H_q,T,d]    backward scratch
+  size_t do_swa;        // fp32 [B,H_q,T,d]    backward scratch (the tensor-core path keeps bf16 there)
+  size_t do_rla;        // fp32 [B,H_q,T,d]    backward scratch (likewise)
   size_t delta;         // fp32 [B,H_q,T]      backward scratch
   size_t chunk_delta;   // fp32 [B,H_kv,n_chunks,d,d]  per-chunk phi(K)^T V
   size_t chunk_state;   // bf16 [B,H_kv,n_chunks,d,d]  exclusive prefix over chunks
+  size_t rstate;        // bf16 [B,H_kv,n_chunks,d,d]  backward: suffix sums of phi(Q)^T g_r
   size_t total;
   int n_chunks;         // ceil(T / 128)
 };
@@ -47,6 +48,7 @@ struct Args {
   // tensor-path scratch
   float* chunk_delta;
   __nv_bfloat16* chunk_state;
+  __nv_bfloat16* rstate;
   int n_chunks;
   int* status;                 // device status word (may be null when no workspace)
   // hand-off
@@ -72,6 +74,7 @@ cudaError_t launch_decode(const Args& a, void* k_ring, void* v_ring, float* stat
                           cudaStream_t s);
 cudaError_t launch_handoff(const Args& a, cudaStream_t s);
 cudaError_t launch_tc_forward(const Args& a, cudaStream_t s);
+cudaError_t launch_tc_backward(const Args& a, cudaStream_t s);
 
 void count_launches(int n);
 void set_last_cuda_error(int cuda_error);   // what rattn_last_cuda_error() reports for this thread

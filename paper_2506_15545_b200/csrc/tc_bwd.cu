@@ -1,0 +1,986 @@
+// Tensor-core backward for bf16, d = 128, window a multiple of 128 (sm_100a: TMA + tcgen05 + TMEM).
+//
+// The paper prints no backward formulas; these follow from its definitions by the chain rule
+// (Section 2.1 for the window branch, Eq. 4 in the chunkwise form of Eq. 2-3 for the residual
+// branch, Section 3.1 for the feature map, Section 3.2 for the two norms).  With 128-token
+// tiles, chunk c = key tile c, lag wt = w / 128, and for query tile i the "boundary" chunk
+// cb = i - wt (the chunk the residual branch reads in intra form, masked to j < t - w):
+//
+//   prep      per row: gradients g_s, g_r of the two un-normalised branch outputs (through the
+//             RMS norms and gains), D_t = g_s . o_swa, all from the forward's residuals.
+//   window    P = exp(scale q.k - lse),  dP = g_s V^T,  dS = P * (dP - D) * scale,
+//             dQ += dS K,   dK += dS^T Q,   dV += P^T g_s.
+//   residual  forward states S_c = sum_{c' < c} phi(K_c')^T V_c' (saved by the forward) and
+//             reverse states R_c = sum_{i > c + wt} phi(Q_i)^T g_r,i (summed over the query
+//             heads of the group; computed here by an outer-product kernel and a suffix scan):
+//               dphi_q = g_r S_cb^T + ((g_r V_cb^T) masked) phi(K_cb)
+//               dphi_k = V_c R_c^T  + ((V_c g_r^T) masked) phi(Q_{c+wt})
+//               dV    += phi(K_c) R_c + ((phi(K_c) phi(Q_{c+wt})^T) masked) g_r
+//   feature   dq += phi(q) * (dphi_q - <dphi_q, phi(q)>), the same for k.
+//
+// Two main kernels, so that every output tile has one owner and nothing is accumulated with
+// atomics (results are deterministic):
+//   tc_bwd_dq_kernel   one CTA per (query tile, query head): loops over the key tiles of the band.
+//   tc_bwd_dkv_kernel  one CTA per (key tile, K/V head): loops over the group's query heads and,
+//                      for each, over the query tiles whose band contains the key tile.
+// In both, 128 threads own one accumulator row each (row = TMEM lane), one thread issues every
+// TMA load and tcgen05.mma, all products are 128 x 128 x 128 with fp32 accumulation in TMEM,
+// and the two weight matrices of each tile pair are rounded to bf16 in shared memory.
+#include "tc_common.cuh"
+
+namespace rattn {
+namespace {
+
+using namespace ptx;
+using namespace tc;
+
+constexpr float LOG2E = 1.4426950408889634f;
+
+struct BwdArgs {
+  __nv_bfloat16* dq;
+  __nv_bfloat16* dk;
+  __nv_bfloat16* dv;
+  const float* lse;     // [B,H_q,T]  natural-log log-sum-exp of the window logits
+  const float* delta;   // [B,H_q,T]  D_t
+  int* status;
+  int T, w, H_q, group, mode, n_chunks;
+  float scale, scale_log2;
+};
+
+#define WAIT_OR_RETURN(bar, parity) \
+  do { if (!mbar_wait(&(bar), (parity), &bars->abort)) return false; } while (0)
+
+__device__ __forceinline__ void load_tile(unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int row, int z) {
+  tma_load_3d(dst, tm, bar, 0, row, z);
+  tma_load_3d(dst + HALF_BYTES, tm, bar, 64, row, z);
+}
+
+__device__ __forceinline__ void named_sync_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// ------------------------------------------------------------------------------ prep
+// One warp per row; lane owns 4 consecutive features.  Writes g_s, g_r (bf16), D and, when
+// asked, accumulates the gain gradients.
+__global__ void __launch_bounds__(256)
+tc_bwd_prep_kernel(const __nv_bfloat16* __restrict__ dy, const float* __restrict__ o_s,
+                   const float* __restrict__ o_r, const float* __restrict__ gamma_s,
+                   const float* __restrict__ gamma_r, __nv_bfloat16* __restrict__ g_s,
+                   __nv_bfloat16* __restrict__ g_r, float* __restrict__ delta, float* __restrict__ dgamma_s,
+                   float* __restrict__ dgamma_r, size_t n_rows, int T, int H_q, float eps, int rla_on) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  constexpr int ROWS_PER_CTA = 64;
+  const size_t row0 = (size_t)blockIdx.x * ROWS_PER_CTA;
+  float acc_s[4] = {0.f, 0.f, 0.f, 0.f}, acc_r[4] = {0.f, 0.f, 0.f, 0.f};
+  int acc_h = -1;
+  auto flush = [&]() {
+    if (acc_h < 0) return;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (dgamma_s) atomicAdd(dgamma_s + (size_t)acc_h * 128 + 4 * lane + e, acc_s[e]);
+      if (dgamma_r && rla_on) atomicAdd(dgamma_r + (size_t)acc_h * 128 + 4 * lane + e, acc_r[e]);
+      acc_s[e] = 0.f;
+      acc_r[e] = 0.f;
+    }
+  };
+  for (int rr = warp; rr < ROWS_PER_CTA; rr += 8) {
+    const size_t row = row0 + rr;
+    if (row >= n_rows) break;
+    const int h = (int)((row / T) % H_q);
+    const float4 xs = *reinterpret_cast<const float4*>(o_s + row * 128 + 4 * lane);
+    const float4 xr = *reinterpret_cast<const float4*>(o_r + row * 128 + 4 * lane);
+    const uint2 gy = *reinterpret_cast<const uint2*>(dy + row * 128 + 4 * lane);
+    const float2 g01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gy.x));
+    const float2 g23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gy.y));
+    const float g[4] = {g01.x, g01.y, g23.x, g23.y};
+    const float vs[4] = {xs.x, xs.y, xs.z, xs.w}, vr[4] = {xr.x, xr.y, xr.z, xr.w};
+    float ss = 0.f, sr = 0.f;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      ss += vs[e] * vs[e];
+      sr += vr[e] * vr[e];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      sr += __shfl_xor_sync(0xffffffffu, sr, o);
+    }
+    const float is = rsqrtf(ss * (1.f / 128.f) + eps), ir = rsqrtf(sr * (1.f / 128.f) + eps);
+    float ghs[4], ghr[4], ms = 0.f, mr = 0.f;
+    if ((dgamma_s || dgamma_r) && h != acc_h) {
+      flush();
+      acc_h = h;
+    }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float gs = gamma_s ? __ldg(gamma_s + (size_t)h * 128 + 4 * lane + e) : 1.f;
+      const float gr = gamma_r ? __ldg(gamma_r + (size_t)h * 128 + 4 * lane + e) : 1.f;
+      ghs[e] = g[e] * gs;
+      ghr[e] = g[e] * gr;
+      ms += ghs[e] * vs[e] * is;
+      mr += ghr[e] * vr[e] * ir;
+      acc_s[e] += g[e] * vs[e] * is;
+      acc_r[e] += g[e] * vr[e] * ir;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      ms += __shfl_xor_sync(0xffffffffu, ms, o);
+      mr += __shfl_xor_sync(0xffffffffu, mr, o);
+    }
+    ms *= (1.f / 128.f);
+    mr *= (1.f / 128.f);
+    float ds[4], dr[4], dl = 0.f;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      ds[e] = (ghs[e] - vs[e] * is * ms) * is;
+      dr[e] = (ghr[e] - vr[e] * ir * mr) * ir;
+      dl += ds[e] * vs[e];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) dl += __shfl_xor_sync(0xffffffffu, dl, o);
+    *reinterpret_cast<uint2*>(g_s + row * 128 + 4 * lane) = make_uint2(pack_bf16(ds[0], ds[1]), pack_bf16(ds[2], ds[3]));
+    *reinterpret_cast<uint2*>(g_r + row * 128 + 4 * lane) = make_uint2(pack_bf16(dr[0], dr[1]), pack_bf16(dr[2], dr[3]));
+    if (lane == 0) delta[row] = dl;
+  }
+  if (dgamma_s || dgamma_r) flush();
+}
+
+// --------------------------------------------------------------- reverse chunk states
+// delta[kv][c] = sum over the group's query heads of phi(Q_c)^T G_c  (fp32, 128 x 128),
+// for c = chunk0 + blockIdx.x.
+constexpr int RD_SMEM = 2 * TILE_BYTES + 64;
+
+__global__ void __launch_bounds__(128)
+tc_bwd_rdelta_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_g,
+                     float* __restrict__ delta, int n_chunks, int chunk0, int group, int* status) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  struct Bars { uint64_t full, done; uint32_t tmem_base; int abort; };
+  Bars* bars = reinterpret_cast<Bars*>(smem + 2 * TILE_BYTES);
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int c = chunk0 + blockIdx.x, kv = blockIdx.y;
+  if ((smem_u32(smem) & 1023u) != 0) {       // the swizzled tile layout needs a 1024-byte aligned base
+    if (tid == 0 && status) atomicExch(status, 2);
+    return;
+  }
+  if (tid == 0) {
+    mbar_init(&bars->full, 1);
+    mbar_init(&bars->done, 1);
+    bars->abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(&bars->tmem_base, 128);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_base;
+  bool ok = true;
+  for (int hh = 0; hh < group; ++hh) {         // every thread runs every iteration (block-wide barriers inside)
+    const int z = kv * group + hh;
+    if (tid == 0 && !bars->abort) {
+      mbar_arrive_expect_tx(&bars->full, 2 * TILE_BYTES);
+      load_tile(smem, &tm_q, &bars->full, c * TILE, z);
+      load_tile(smem + TILE_BYTES, &tm_g, &bars->full, c * TILE, z);
+    }
+    ok = ok && mbar_wait(&bars->full, hh & 1, &bars->abort);
+    if (ok) {
+      feature_map_row_inplace(smem, tid);
+      fence_proxy_async_smem();
+    }
+    __syncthreads();
+    if (tid == 0 && !bars->abort) {
+      tc_fence_after();
+      mma_mnmn(tmem, smem_u32(smem), smem_u32(smem + TILE_BYTES), hh > 0);
+      mma_commit(&bars->done);
+    }
+    ok = ok && mbar_wait(&bars->done, hh & 1, &bars->abort);   // shared memory is reused by the next head
+  }
+  if (ok) {
+    tc_fence_after();
+    float* dst = delta + (((size_t)kv * n_chunks + c) * 128 + tid) * 128;
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc) {
+      float x[32];
+      tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + 32 * cc, x);
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 8; ++e)
+        *reinterpret_cast<float4*>(dst + 32 * cc + 4 * e) = make_float4(x[4 * e], x[4 * e + 1], x[4 * e + 2], x[4 * e + 3]);
+    }
+  } else if (status) {
+    atomicExch(status, 1);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 128);
+  }
+}
+
+// rstate[kv][c] = sum_{i >= c + lag} delta[kv][i],  c = 0 .. n_r-1, i up to n_qt-1  (bf16).
+__global__ void __launch_bounds__(256)
+tc_bwd_rscan_kernel(const float* __restrict__ delta, __nv_bfloat16* __restrict__ rstate, int n_chunks,
+                    int n_qt, int lag) {
+  const int kv = blockIdx.x;
+  const int idx = blockIdx.y * 256 + threadIdx.x;
+  const float4* src = reinterpret_cast<const float4*>(delta) + (size_t)kv * n_chunks * 4096 + idx;
+  uint2* dst = reinterpret_cast<uint2*>(rstate) + (size_t)kv * n_chunks * 4096 + idx;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int i = n_qt - 1; i >= lag; --i) {
+    const float4 x = src[(size_t)i * 4096];
+    acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+    dst[(size_t)(i - lag) * 4096] = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
+  }
+}
+
+// ================================================================================ dq
+constexpr int DQ_OFF_Q = 0;
+constexpr int DQ_OFF_G = 1 * TILE_BYTES;
+constexpr int DQ_OFF_K = 2 * TILE_BYTES;   // 2 stages
+constexpr int DQ_OFF_V = 4 * TILE_BYTES;   // 2 stages
+constexpr int DQ_OFF_D = 6 * TILE_BYTES;
+constexpr int DQ_OFF_BAR = 7 * TILE_BYTES;
+constexpr int DQ_SMEM = DQ_OFF_BAR + 256;
+
+struct DqBars {
+  uint64_t qg_full, kv_full[2], s_full, s_empty, ds_full, dq_done, x_full, phik_ready, o_done, drain;
+  uint32_t tmem_base;
+  int abort;
+};
+
+__device__ bool dq_control(const CUtensorMap* tm_q, const CUtensorMap* tm_k, const CUtensorMap* tm_v,
+                           const CUtensorMap* tm_gs, const CUtensorMap* tm_gr, const CUtensorMap* tm_st,
+                           unsigned char* smem, DqBars* bars, uint32_t tmem, int q0, int bh_q, int bh_kv,
+                           int n_kt, bool has_rla, bool has_state, int st_index) {
+  const uint32_t sQ = smem_u32(smem + DQ_OFF_Q), sG = smem_u32(smem + DQ_OFF_G);
+  const uint32_t sK = smem_u32(smem + DQ_OFF_K), sV = smem_u32(smem + DQ_OFF_V), sD = smem_u32(smem + DQ_OFF_D);
+  const uint32_t tS = tmem, tP = tmem + 128, tQ = tmem + 256, tF = tmem + 384;
+
+  mbar_arrive_expect_tx(&bars->qg_full, 2 * TILE_BYTES);
+  load_tile(smem + DQ_OFF_Q, tm_q, &bars->qg_full, q0, bh_q);
+  load_tile(smem + DQ_OFF_G, tm_gs, &bars->qg_full, q0, bh_q);
+  for (int i = 0; i < (n_kt < 2 ? n_kt : 2); ++i) {
+    mbar_arrive_expect_tx(&bars->kv_full[i], 2 * TILE_BYTES);
+    load_tile(smem + DQ_OFF_K + i * TILE_BYTES, tm_k, &bars->kv_full[i], q0 - i * TILE, bh_kv);
+    load_tile(smem + DQ_OFF_V + i * TILE_BYTES, tm_v, &bars->kv_full[i], q0 - i * TILE, bh_kv);
+  }
+  WAIT_OR_RETURN(bars->qg_full, 0);
+  for (int i = 0; i < n_kt; ++i) {
+    const int b = i & 1;
+    WAIT_OR_RETURN(bars->kv_full[b], (i >> 1) & 1);
+    if (i > 0) WAIT_OR_RETURN(bars->s_empty, (i - 1) & 1);
+    tc_fence_after();
+    mma_kk(tS, sQ, sK + b * TILE_BYTES, false);          // S  = Q K^T
+    mma_kk(tP, sG, sV + b * TILE_BYTES, false);          // dP = g_s V^T
+    mma_commit(&bars->s_full);
+    if (i > 0) {
+      const int pb = (i - 1) & 1;
+      WAIT_OR_RETURN(bars->ds_full, (i - 1) & 1);
+      tc_fence_after();
+      mma_kmn<1>(tQ, sD, sK + pb * TILE_BYTES, i - 1 > 0); // dQ += dS K
+      mma_commit(&bars->dq_done);
+      WAIT_OR_RETURN(bars->dq_done, (i - 1) & 1);          // stage pb is free again
+      if (i + 1 < n_kt) {
+        mbar_arrive_expect_tx(&bars->kv_full[pb], 2 * TILE_BYTES);
+        load_tile(smem + DQ_OFF_K + pb * TILE_BYTES, tm_k, &bars->kv_full[pb], q0 - (i + 1) * TILE, bh_kv);
+        load_tile(smem + DQ_OFF_V + pb * TILE_BYTES, tm_v, &bars->kv_full[pb], q0 - (i + 1) * TILE, bh_kv);
+      } else if (has_rla) {
+        // the free stage receives the residual branch's operands: g_r and the stored state
+        mbar_arrive_expect_tx(&bars->x_full, (has_state ? 2 : 1) * TILE_BYTES);
+        load_tile(smem + DQ_OFF_V + pb * TILE_BYTES, tm_gr, &bars->x_full, q0, bh_q);
+        if (has_state) load_tile(smem + DQ_OFF_K + pb * TILE_BYTES, tm_st, &bars->x_full, 0, st_index);
+      }
+    }
+  }
+  const int last = (n_kt - 1) & 1, other = last ^ 1;
+  WAIT_OR_RETURN(bars->ds_full, (n_kt - 1) & 1);
+  tc_fence_after();
+  mma_kmn<1>(tQ, sD, sK + last * TILE_BYTES, n_kt - 1 > 0);
+  mma_commit(&bars->dq_done);
+  if (has_rla) {
+    const uint32_t sG2 = sV + other * TILE_BYTES, sSt = sK + other * TILE_BYTES;
+    WAIT_OR_RETURN(bars->x_full, 0);
+    WAIT_OR_RETURN(bars->s_empty, (n_kt - 1) & 1);
+    tc_fence_after();
+    mma_kk(tS, sG2, sV + last * TILE_BYTES, false);        // dA = g_r V_cb^T
+    if (has_state) mma_kk(tF, sG2, sSt, false);            // g_r S_cb^T
+    mma_commit(&bars->s_full);
+    WAIT_OR_RETURN(bars->phik_ready, 0);
+    WAIT_OR_RETURN(bars->ds_full, n_kt & 1);
+    tc_fence_after();
+    mma_kmn<1>(tF, sD, sK + last * TILE_BYTES, has_state); // (dA masked) phi(K_cb)
+  }
+  mma_commit(&bars->o_done);
+  return true;
+}
+
+__device__ bool dq_rows(const BwdArgs& a, unsigned char* smem, DqBars* bars, uint32_t tmem, int r, int q0,
+                        int bh_q, int n_kt, bool has_boundary, bool has_rla) {
+  const uint32_t lane_off = (uint32_t)((r & ~31) << 16);
+  const uint32_t tS = tmem + lane_off, tP = tmem + 128 + lane_off, tQ = tmem + 256 + lane_off,
+                 tF = tmem + 384 + lane_off;
+  unsigned char* sD = smem + DQ_OFF_D;
+  const int t = q0 + r;
+  const bool live = t < a.T;
+  const size_t row = (size_t)bh_q * a.T + t;
+  const float l2 = live ? a.lse[row] * LOG2E : INFINITY;
+  const float Dr = live ? a.delta[row] : 0.f;
+
+  for (int i = 0; i < n_kt; ++i) {
+    WAIT_OR_RETURN(bars->s_full, i & 1);
+    tc_fence_after();
+    const bool diag = (i == 0), bound = has_boundary && (i == n_kt - 1);
+    uint32_t pk[64];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      float s[32], dp[32];
+      tmem_ld32(tS + 32 * c, s);
+      tmem_ld32(tP + 32 * c, dp);
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 32; e += 2) {
+        const int j = 32 * c + e;
+        const float p0 = ex2(s[e] * a.scale_log2 - l2), p1 = ex2(s[e + 1] * a.scale_log2 - l2);
+        const bool ok0 = !((diag && j > r) || (bound && j < r));
+        const bool ok1 = !((diag && j + 1 > r) || (bound && j + 1 < r));
+        const float d0 = ok0 ? p0 * (dp[e] - Dr) * a.scale : 0.f;
+        const float d1 = ok1 ? p1 * (dp[e + 1] - Dr) * a.scale : 0.f;
+        pk[16 * c + (e >> 1)] = pack_bf16(d0, d1);
+      }
+    }
+    tc_fence_before();
+    mbar_arrive(&bars->s_empty);
+    if (i > 0) WAIT_OR_RETURN(bars->dq_done, (i - 1) & 1);   // the previous dS has been consumed
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+      *reinterpret_cast<uint4*>(sD + swz(r, c)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+    fence_proxy_async_smem();
+    mbar_arrive(&bars->ds_full);
+  }
+
+  if (has_rla) {
+    const int last = (n_kt - 1) & 1;
+    WAIT_OR_RETURN(bars->dq_done, (n_kt - 1) & 1);           // K_cb is no longer read raw
+    feature_map_row_inplace(smem + DQ_OFF_K + last * TILE_BYTES, r);
+    fence_proxy_async_smem();
+    mbar_arrive(&bars->phik_ready);
+    WAIT_OR_RETURN(bars->s_full, n_kt & 1);
+    tc_fence_after();
+    uint32_t pk[64];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      float x[32];
+      tmem_ld32(tS + 32 * c, x);
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 32; e += 2) {
+        const int j = 32 * c + e;                            // residual keys of row r in this chunk: j < r
+        pk[16 * c + (e >> 1)] = pack_bf16(j < r ? x[e] : 0.f, j + 1 < r ? x[e + 1] : 0.f);
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+      *reinterpret_cast<uint4*>(sD + swz(r, c)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+    fence_proxy_async_smem();
+    tc_fence_before();
+    mbar_arrive(&bars->ds_full);
+  }
+
+  // ---- dq = dQ + phi(q) * (dphi_q - <dphi_q, phi(q)>) -----------------------------------
+  WAIT_OR_RETURN(bars->o_done, 0);
+  tc_fence_after();
+  const unsigned char* sQ = smem + DQ_OFF_Q;
+  float m = 0.f, inv = 0.f, dot = 0.f;
+  if (has_rla) {
+    m = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+      const uint4 u = *reinterpret_cast<const uint4*>(sQ + swz(r, c));
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 f = __bfloat1622float2(h[e]);
+        m = fmaxf(m, fmaxf(f.x, f.y));
+      }
+    }
+    const float ml = m * LOG2E;
+    float sum = 0.f, du = 0.f;
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+      float df[32];
+      tmem_ld32(tF + 32 * c, df);
+      tmem_wait_ld();
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        const uint4 u = *reinterpret_cast<const uint4*>(sQ + swz(r, 4 * c + cc));
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 f = __bfloat1622float2(h[e]);
+          const float e0 = ex2(f.x * LOG2E - ml), e1 = ex2(f.y * LOG2E - ml);
+          sum += e0 + e1;
+          du += e0 * df[8 * cc + 2 * e] + e1 * df[8 * cc + 2 * e + 1];
+        }
+      }
+    }
+    inv = 1.f / sum;
+    dot = du * inv;
+    m = ml;
+  }
+  __nv_bfloat16* orow = a.dq + row * 128;
+#pragma unroll 1
+  for (int c = 0; c < 4; ++c) {
+    float x[32], df[32];
+    tmem_ld32(tQ + 32 * c, x);
+    if (has_rla) tmem_ld32(tF + 32 * c, df);
+    tmem_wait_ld();
+    if (has_rla) {
+#pragma unroll
+      for (int cc = 0; cc < 4; ++cc) {
+        const uint4 u = *reinterpret_cast<const uint4*>(sQ + swz(r, 4 * c + cc));
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 f = __bfloat1622float2(h[e]);
+          const float e0 = ex2(f.x * LOG2E - m) * inv, e1 = ex2(f.y * LOG2E - m) * inv;
+          x[8 * cc + 2 * e] += e0 * (df[8 * cc + 2 * e] - dot);
+          x[8 * cc + 2 * e + 1] += e1 * (df[8 * cc + 2 * e + 1] - dot);
+        }
+      }
+    }
+    if (live) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        uint4 u;
+        u.x = pack_bf16(x[8 * e + 0], x[8 * e + 1]);
+        u.y = pack_bf16(x[8 * e + 2], x[8 * e + 3]);
+        u.z = pack_bf16(x[8 * e + 4], x[8 * e + 5]);
+        u.w = pack_bf16(x[8 * e + 6], x[8 * e + 7]);
+        *reinterpret_cast<uint4*>(orow + 32 * c + 8 * e) = u;
+      }
+    }
+  }
+  tc_fence_before();
+  return true;
+}
+
+__global__ void __launch_bounds__(160, 1)
+tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_gs,
+                 const __grid_constant__ CUtensorMap tm_gr, const __grid_constant__ CUtensorMap tm_st, BwdArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  DqBars* bars = reinterpret_cast<DqBars*>(smem + DQ_OFF_BAR);
+  const int tid = threadIdx.x, warp = tid >> 5;
+  if ((smem_u32(smem) & 1023u) != 0) {
+    if (tid == 0 && a.status) atomicExch(a.status, 2);
+    return;
+  }
+  const int n_qt = (a.T + TILE - 1) / TILE;
+  const int qt = n_qt - 1 - (int)blockIdx.x;
+  const int q0 = qt * TILE;
+  const int bh_q = blockIdx.y;
+  const int b = bh_q / a.H_q, h = bh_q % a.H_q;
+  const int bh_kv = b * (a.H_q / a.group) + h / a.group;
+  const int wt = a.w / TILE;
+  const bool has_boundary = (a.mode != RATTN_MODE_FULL_CAUSAL) && (qt - wt >= 0);
+  const int n_kt = (has_boundary ? wt : qt) + 1;
+  const bool has_rla = has_boundary && (a.mode == RATTN_MODE_RATTN);
+  const int cb = qt - wt;
+  const bool has_state = has_rla && cb > 0;
+  const int st_index = bh_kv * a.n_chunks + (cb > 0 ? cb : 0);
+
+  if (tid == 0) {
+    mbar_init(&bars->qg_full, 1);
+    mbar_init(&bars->kv_full[0], 1);
+    mbar_init(&bars->kv_full[1], 1);
+    mbar_init(&bars->s_full, 1);
+    mbar_init(&bars->s_empty, 128);
+    mbar_init(&bars->ds_full, 128);
+    mbar_init(&bars->dq_done, 1);
+    mbar_init(&bars->x_full, 1);
+    mbar_init(&bars->phik_ready, 128);
+    mbar_init(&bars->o_done, 1);
+    mbar_init(&bars->drain, 1);
+    bars->abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 4) {
+    tmem_alloc(&bars->tmem_base, 512);
+    tmem_relinquish();
+    if (tid == 128) {
+      prefetch_tensormap(&tm_q);
+      prefetch_tensormap(&tm_k);
+      prefetch_tensormap(&tm_v);
+      prefetch_tensormap(&tm_gs);
+      prefetch_tensormap(&tm_gr);
+      prefetch_tensormap(&tm_st);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_base;
+
+  bool ok = true;
+  if (warp < 4) {
+    ok = dq_rows(a, smem, bars, tmem, tid, q0, bh_q, n_kt, has_boundary, has_rla);
+  } else if (tid == 128) {
+    ok = dq_control(&tm_q, &tm_k, &tm_v, &tm_gs, &tm_gr, &tm_st, smem, bars, tmem, q0, bh_q, bh_kv, n_kt,
+                    has_rla, has_state, st_index);
+    if (!ok) {
+      mma_commit(&bars->drain);
+      for (int it = 0; it < (1 << 16) && !mbar_try_wait(&bars->drain, 0); ++it) {}
+    }
+  }
+  if (!ok && a.status) atomicExch(a.status, 1);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// =============================================================================== dkv
+constexpr int KV_OFF_K = 0;
+constexpr int KV_OFF_V = 1 * TILE_BYTES;
+constexpr int KV_OFF_Q = 2 * TILE_BYTES;   // 2 stages
+constexpr int KV_OFF_G = 4 * TILE_BYTES;   // 2 stages
+constexpr int KV_OFF_D = 6 * TILE_BYTES;
+constexpr int KV_OFF_STAT = 7 * TILE_BYTES;            // 2 stages x (lse2[128], D*scale[128]) fp32
+constexpr int KV_OFF_BAR = KV_OFF_STAT + 2 * 2 * 128 * 4;
+constexpr int KV_SMEM = KV_OFF_BAR + 256;
+
+struct KvBars {
+  uint64_t kv_full, k2_full, r_full, kphi_ready, inter_done, qg_full[2], phi_ready, s_full, s_empty,
+      d1_full, acc1_done, d2_full, acc2_done, xform_done, drain;
+  uint32_t tmem_base;
+  int abort;
+};
+
+// The work of one CTA is a list of items, each one (query head of the group, query tile):
+// first the residual-branch items (one per head, query tile j + wt), then the window items.
+struct KvPlan {
+  int j, n_qt, wt, group, n_r, n_s_tiles, N;
+  bool windowed, has_inter;
+  __device__ bool is_r(int n) const { return n < n_r; }
+  __device__ int head(int n) const { return n < n_r ? n : (n - n_r) / n_s_tiles; }
+  __device__ int qtile(int n) const { return n < n_r ? j + wt : j + (n - n_r) % n_s_tiles; }
+};
+
+__device__ bool kv_control(const CUtensorMap* tm_q, const CUtensorMap* tm_k, const CUtensorMap* tm_v,
+                           const CUtensorMap* tm_gs, const CUtensorMap* tm_gr, const CUtensorMap* tm_rs,
+                           unsigned char* smem, KvBars* bars, uint32_t tmem, const KvPlan& pl, int bh_kv,
+                           int rs_index) {
+  const uint32_t sK = smem_u32(smem + KV_OFF_K), sV = smem_u32(smem + KV_OFF_V);
+  const uint32_t sQ = smem_u32(smem + KV_OFF_Q), sG = smem_u32(smem + KV_OFF_G), sD = smem_u32(smem + KV_OFF_D);
+  const uint32_t tS = tmem, tP = tmem + 128, tV = tmem + 256, tK = tmem + 384;
+  const int j0 = pl.j * TILE;
+
+  auto load_item = [&](int n) {
+    const int st = n & 1;
+    const int z = bh_kv * pl.group + pl.head(n);
+    const int row = pl.qtile(n) * TILE;
+    mbar_arrive_expect_tx(&bars->qg_full[st], 2 * TILE_BYTES);
+    load_tile(smem + KV_OFF_Q + st * TILE_BYTES, tm_q, &bars->qg_full[st], row, z);
+    load_tile(smem + KV_OFF_G + st * TILE_BYTES, pl.is_r(n) ? tm_gr : tm_gs, &bars->qg_full[st], row, z);
+  };
+
+  mbar_arrive_expect_tx(&bars->kv_full, 2 * TILE_BYTES);
+  load_tile(smem + KV_OFF_K, tm_k, &bars->kv_full, j0, bh_kv);
+  load_tile(smem + KV_OFF_V, tm_v, &bars->kv_full, j0, bh_kv);
+  if (pl.has_inter) {
+    mbar_arrive_expect_tx(&bars->r_full, TILE_BYTES);
+    load_tile(smem + KV_OFF_D, tm_rs, &bars->r_full, 0, rs_index);
+  }
+  load_item(0);
+  if (pl.N > 1) load_item(1);
+
+  bool accV = false, accK = false;
+  if (pl.n_r > 0) {
+    WAIT_OR_RETURN(bars->kphi_ready, 0);                   // phi(K_j) is in place (implies K, V landed)
+    if (pl.has_inter) {
+      WAIT_OR_RETURN(bars->r_full, 0);
+      tc_fence_after();
+      mma_kk(tK, sV, sD, false);                           // dphi_k  = V_j R_j^T
+      mma_kmn<1>(tV, sK, sD, false);                       // dV      = phi(K_j) R_j
+      mma_commit(&bars->inter_done);
+      accV = accK = true;
+    }
+  } else {
+    WAIT_OR_RETURN(bars->kv_full, 0);
+  }
+
+  auto issue_scores = [&](int n) -> bool {
+    const int st = n & 1;
+    if (n == pl.n_r && pl.n_r > 0) {
+      // residual phase over: phi(K_j) has been consumed and folded; fetch K_j again for the window phase
+      WAIT_OR_RETURN(bars->xform_done, 0);
+      mbar_arrive_expect_tx(&bars->k2_full, TILE_BYTES);
+      load_tile(smem + KV_OFF_K, tm_k, &bars->k2_full, j0, bh_kv);
+      WAIT_OR_RETURN(bars->k2_full, 0);
+    }
+    WAIT_OR_RETURN(bars->qg_full[st], (n >> 1) & 1);
+    if (pl.is_r(n)) WAIT_OR_RETURN(bars->phi_ready, n & 1);
+    if (n > 0) WAIT_OR_RETURN(bars->s_empty, (n - 1) & 1);
+    tc_fence_after();
+    mma_kk(tS, sK, sQ + st * TILE_BYTES, false);           // S^T  = K Q^T      (or phi(K) phi(Q)^T)
+    mma_kk(tP, sV, sG + st * TILE_BYTES, false);           // dP^T = V g^T
+    mma_commit(&bars->s_full);
+    return true;
+  };
+
+  int issued = -1;
+  for (int n = 0; n < pl.N; ++n) {
+    const int st = n & 1;
+    if (issued < n) {
+      if (!issue_scores(n)) return false;
+      issued = n;
+    }
+    // run ahead: the next item's scores, unless it needs this item's results first
+    if (n + 1 < pl.N && !pl.is_r(n + 1) && !(n + 1 == pl.n_r && pl.n_r > 0)) {
+      if (!issue_scores(n + 1)) return false;
+      issued = n + 1;
+    }
+    WAIT_OR_RETURN(bars->d1_full, n & 1);
+    tc_fence_after();
+    mma_kmn<1>(tV, sD, sG + st * TILE_BYTES, accV);        // dV += P^T g_s      (or A^T g_r)
+    mma_commit(&bars->acc1_done);
+    accV = true;
+    WAIT_OR_RETURN(bars->d2_full, n & 1);
+    tc_fence_after();
+    mma_kmn<1>(tK, sD, sQ + st * TILE_BYTES, accK);        // dK += dS^T Q       (or dphi_k += dA^T phi(Q))
+    mma_commit(&bars->acc2_done);
+    accK = true;
+    WAIT_OR_RETURN(bars->acc2_done, n & 1);                // stage st is free again
+    if (n + 2 < pl.N) load_item(n + 2);
+  }
+  return true;
+}
+
+__device__ bool kv_rows(const BwdArgs& a, unsigned char* smem, KvBars* bars, uint32_t tmem, const KvPlan& pl,
+                        int r, int bh_kv) {
+  const uint32_t lane_off = (uint32_t)((r & ~31) << 16);
+  const uint32_t tS = tmem + lane_off, tP = tmem + 128 + lane_off, tV = tmem + 256 + lane_off,
+                 tK = tmem + 384 + lane_off;
+  unsigned char* sD = smem + KV_OFF_D;
+  unsigned char* sK = smem + KV_OFF_K;
+  float* stat = reinterpret_cast<float*>(smem + KV_OFF_STAT);
+
+  WAIT_OR_RETURN(bars->kv_full, 0);
+  if (pl.n_r > 0) {
+    feature_map_row_inplace(sK, r);
+    fence_proxy_async_smem();
+    mbar_arrive(&bars->kphi_ready);
+  }
+
+  for (int n = 0; n < pl.N; ++n) {
+    const int st = n & 1;
+    const bool is_r = pl.is_r(n);
+    const int i = pl.qtile(n);
+    if (is_r) {
+      WAIT_OR_RETURN(bars->qg_full[st], (n >> 1) & 1);
+      feature_map_row_inplace(smem + KV_OFF_Q + st * TILE_BYTES, r);
+      fence_proxy_async_smem();
+      mbar_arrive(&bars->phi_ready);
+    } else {
+      const int bq = bh_kv * a.group + pl.head(n);        // (batch, query head) index of this item
+      const int t = i * TILE + r;
+      const size_t row = (size_t)bq * a.T + t;
+      stat[st * 256 + r] = t < a.T ? a.lse[row] * LOG2E : INFINITY;
+      stat[st * 256 + 128 + r] = t < a.T ? a.delta[row] * a.scale : 0.f;
+      named_sync_128();
+    }
+    WAIT_OR_RETURN(bars->s_full, n & 1);
+    tc_fence_after();
+    const bool diag = !is_r && (i == pl.j), bound = !is_r && pl.windowed && (i == pl.j + pl.wt);
+    const float* l2 = stat + st * 256;
+    const float* Ds = l2 + 128;
+    uint32_t pk1[64], pk2[64];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      float s[32], dp[32];
+      tmem_ld32(tS + 32 * c, s);
+      tmem_ld32(tP + 32 * c, dp);
+      tmem_wait_ld();
+      if (is_r) {
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+          const int q = 32 * c + e;                          // query column; keep key r < query q
+          pk1[16 * c + (e >> 1)] = pack_bf16(q > r ? s[e] : 0.f, q + 1 > r ? s[e + 1] : 0.f);
+          pk2[16 * c + (e >> 1)] = pack_bf16(q > r ? dp[e] : 0.f, q + 1 > r ? dp[e + 1] : 0.f);
+        }
+      } else {
+#pragma unroll
+        for (int e4 = 0; e4 < 32; e4 += 4) {
+          const float4 lv = *reinterpret_cast<const float4*>(l2 + 32 * c + e4);
+          const float4 dv = *reinterpret_cast<const float4*>(Ds + 32 * c + e4);
+          const float lq[4] = {lv.x, lv.y, lv.z, lv.w}, dq4[4] = {dv.x, dv.y, dv.z, dv.w};
+          float p[4], d[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int q = 32 * c + e4 + u;
+            const bool ok = !((diag && q < r) || (bound && q > r));
+            const float pv = ex2(s[e4 + u] * a.scale_log2 - lq[u]);
+            p[u] = ok ? pv : 0.f;
+            d[u] = ok ? pv * (dp[e4 + u] * a.scale - dq4[u]) : 0.f;
+          }
+          pk1[16 * c + (e4 >> 1)] = pack_bf16(p[0], p[1]);
+          pk1[16 * c + (e4 >> 1) + 1] = pack_bf16(p[2], p[3]);
+          pk2[16 * c + (e4 >> 1)] = pack_bf16(d[0], d[1]);
+          pk2[16 * c + (e4 >> 1) + 1] = pack_bf16(d[2], d[3]);
+        }
+      }
+    }
+    tc_fence_before();
+    mbar_arrive(&bars->s_empty);
+    // the staging tile is free once the previous product that read it has completed
+    if (n > 0) WAIT_OR_RETURN(bars->acc2_done, (n - 1) & 1);
+    else if (pl.has_inter) WAIT_OR_RETURN(bars->inter_done, 0);
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+      *reinterpret_cast<uint4*>(sD + swz(r, c)) = make_uint4(pk1[4 * c], pk1[4 * c + 1], pk1[4 * c + 2], pk1[4 * c + 3]);
+    fence_proxy_async_smem();
+    mbar_arrive(&bars->d1_full);
+    WAIT_OR_RETURN(bars->acc1_done, n & 1);
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+      *reinterpret_cast<uint4*>(sD + swz(r, c)) = make_uint4(pk2[4 * c], pk2[4 * c + 1], pk2[4 * c + 2], pk2[4 * c + 3]);
+    fence_proxy_async_smem();
+    mbar_arrive(&bars->d2_full);
+
+    if (n == pl.n_r - 1) {
+      // end of the residual phase: fold the feature-map Jacobian into the dK accumulator,
+      // dK := phi(k) * (dphi_k - <dphi_k, phi(k)>), so that the window phase accumulates on top
+      WAIT_OR_RETURN(bars->acc2_done, n & 1);
+      tc_fence_after();
+      float dot = 0.f;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        float df[32];
+        tmem_ld32(tK + 32 * c, df);
+        tmem_wait_ld();
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          const uint4 u = *reinterpret_cast<const uint4*>(sK + swz(r, 4 * c + cc));
+          const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(h2[e]);
+            dot += f.x * df[8 * cc + 2 * e] + f.y * df[8 * cc + 2 * e + 1];
+          }
+        }
+      }
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        float df[32];
+        tmem_ld32(tK + 32 * c, df);
+        tmem_wait_ld();
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          const uint4 u = *reinterpret_cast<const uint4*>(sK + swz(r, 4 * c + cc));
+          const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(h2[e]);
+            df[8 * cc + 2 * e] = f.x * (df[8 * cc + 2 * e] - dot);
+            df[8 * cc + 2 * e + 1] = f.y * (df[8 * cc + 2 * e + 1] - dot);
+          }
+        }
+        tmem_st32(tK + 32 * c, df);
+      }
+      tmem_wait_st();
+      fence_proxy_async_smem();
+      tc_fence_before();
+      mbar_arrive(&bars->xform_done);
+    }
+  }
+
+  WAIT_OR_RETURN(bars->acc2_done, (pl.N - 1) & 1);
+  tc_fence_after();
+  const int jj = pl.j * TILE + r;
+  const size_t row = (size_t)bh_kv * a.T + jj;
+#pragma unroll 1
+  for (int c = 0; c < 4; ++c) {
+    float xk[32], xv[32];
+    tmem_ld32(tK + 32 * c, xk);
+    tmem_ld32(tV + 32 * c, xv);
+    tmem_wait_ld();
+    if (jj < a.T) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        uint4 u;
+        u.x = pack_bf16(xk[8 * e + 0], xk[8 * e + 1]);
+        u.y = pack_bf16(xk[8 * e + 2], xk[8 * e + 3]);
+        u.z = pack_bf16(xk[8 * e + 4], xk[8 * e + 5]);
+        u.w = pack_bf16(xk[8 * e + 6], xk[8 * e + 7]);
+        *reinterpret_cast<uint4*>(a.dk + row * 128 + 32 * c + 8 * e) = u;
+        u.x = pack_bf16(xv[8 * e + 0], xv[8 * e + 1]);
+        u.y = pack_bf16(xv[8 * e + 2], xv[8 * e + 3]);
+        u.z = pack_bf16(xv[8 * e + 4], xv[8 * e + 5]);
+        u.w = pack_bf16(xv[8 * e + 6], xv[8 * e + 7]);
+        *reinterpret_cast<uint4*>(a.dv + row * 128 + 32 * c + 8 * e) = u;
+      }
+    }
+  }
+  tc_fence_before();
+  return true;
+}
+
+__global__ void __launch_bounds__(160, 1)
+tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_gs,
+                  const __grid_constant__ CUtensorMap tm_gr, const __grid_constant__ CUtensorMap tm_rs, BwdArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  KvBars* bars = reinterpret_cast<KvBars*>(smem + KV_OFF_BAR);
+  const int tid = threadIdx.x, warp = tid >> 5;
+  if ((smem_u32(smem) & 1023u) != 0) {
+    if (tid == 0 && a.status) atomicExch(a.status, 2);
+    return;
+  }
+  KvPlan pl;
+  pl.n_qt = (a.T + TILE - 1) / TILE;
+  pl.j = blockIdx.x;
+  pl.wt = a.w / TILE;
+  pl.group = a.group;
+  pl.windowed = (a.mode != RATTN_MODE_FULL_CAUSAL);
+  const int i_hi = (pl.windowed && pl.j + pl.wt < pl.n_qt - 1) ? pl.j + pl.wt : pl.n_qt - 1;
+  pl.n_s_tiles = i_hi - pl.j + 1;
+  const bool r_tile = pl.windowed && (a.mode == RATTN_MODE_RATTN) && (pl.j + pl.wt <= pl.n_qt - 1);
+  pl.n_r = r_tile ? a.group : 0;
+  pl.has_inter = r_tile && (pl.j + pl.wt + 1 <= pl.n_qt - 1);
+  pl.N = pl.n_r + a.group * pl.n_s_tiles;
+  const int bh_kv = blockIdx.y;
+  const int rs_index = bh_kv * a.n_chunks + pl.j;
+
+  if (tid == 0) {
+    mbar_init(&bars->kv_full, 1);
+    mbar_init(&bars->k2_full, 1);
+    mbar_init(&bars->r_full, 1);
+    mbar_init(&bars->kphi_ready, 128);
+    mbar_init(&bars->inter_done, 1);
+    mbar_init(&bars->qg_full[0], 1);
+    mbar_init(&bars->qg_full[1], 1);
+    mbar_init(&bars->phi_ready, 128);
+    mbar_init(&bars->s_full, 1);
+    mbar_init(&bars->s_empty, 128);
+    mbar_init(&bars->d1_full, 128);
+    mbar_init(&bars->acc1_done, 1);
+    mbar_init(&bars->d2_full, 128);
+    mbar_init(&bars->acc2_done, 1);
+    mbar_init(&bars->xform_done, 128);
+    mbar_init(&bars->drain, 1);
+    bars->abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 4) {
+    tmem_alloc(&bars->tmem_base, 512);
+    tmem_relinquish();
+    if (tid == 128) {
+      prefetch_tensormap(&tm_q);
+      prefetch_tensormap(&tm_k);
+      prefetch_tensormap(&tm_v);
+      prefetch_tensormap(&tm_gs);
+      prefetch_tensormap(&tm_gr);
+      prefetch_tensormap(&tm_rs);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_base;
+
+  bool ok = true;
+  if (warp < 4) {
+    ok = kv_rows(a, smem, bars, tmem, pl, tid, bh_kv);
+  } else if (tid == 128) {
+    ok = kv_control(&tm_q, &tm_k, &tm_v, &tm_gs, &tm_gr, &tm_rs, smem, bars, tmem, pl, bh_kv, rs_index);
+    if (!ok) {
+      mma_commit(&bars->drain);
+      for (int it = 0; it < (1 << 16) && !mbar_try_wait(&bars->drain, 0); ++it) {}
+    }
+  }
+  if (!ok && a.status) atomicExch(a.status, 1);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
+  const size_t n_rows = (size_t)a.B * a.H_q * a.T;
+  __nv_bfloat16* g_s = reinterpret_cast<__nv_bfloat16*>(a.do_swa);
+  __nv_bfloat16* g_r = reinterpret_cast<__nv_bfloat16*>(a.do_rla);
+  const bool rla_on = (a.mode == RATTN_MODE_RATTN);
+  const int n_qt = (a.T + TILE - 1) / TILE;
+  const int wt = a.w / TILE;
+  cudaError_t e;
+  if (a.dgamma_swa) {
+    e = cudaMemsetAsync(a.dgamma_swa, 0, sizeof(float) * a.H_q * 128, s);
+    if (e != cudaSuccess) return e;
+  }
+  if (a.dgamma_rla) {
+    e = cudaMemsetAsync(a.dgamma_rla, 0, sizeof(float) * a.H_q * 128, s);
+    if (e != cudaSuccess) return e;
+  }
+  {
+    KernelTimer kt("tc_bwd_prep", s);
+    tc_bwd_prep_kernel<<<(unsigned)((n_rows + 63) / 64), 256, 0, s>>>(
+        reinterpret_cast<const __nv_bfloat16*>(a.dout), a.o_swa, a.o_rla, a.gamma_swa, a.gamma_rla, g_s, g_r,
+        a.delta, a.dgamma_swa, a.dgamma_rla, n_rows, a.T, a.H_q, a.eps, rla_on ? 1 : 0);
+  }
+  count_launches(1);
+
+  CUtensorMap tm_q, tm_k, tm_v, tm_gs, tm_gr, tm_st, tm_rs;
+  const uint64_t nq = (uint64_t)a.B * a.H_q, nkv = (uint64_t)a.B * a.H_kv;
+  if (!make_map(&tm_q, a.q, a.T, nq) || !make_map(&tm_k, a.k, a.T, nkv) || !make_map(&tm_v, a.v, a.T, nkv) ||
+      !make_map(&tm_gs, g_s, a.T, nq) || !make_map(&tm_gr, g_r, a.T, nq) ||
+      !make_map(&tm_st, a.chunk_state, 128, nkv * a.n_chunks) || !make_map(&tm_rs, a.rstate, 128, nkv * a.n_chunks))
+    return cudaErrorInvalidValue;
+
+  // reverse states of the residual branch: chunks c with a query tile beyond c + wt
+  const int n_r = rla_on && a.mode != RATTN_MODE_FULL_CAUSAL ? n_qt - wt - 1 : 0;
+  if (n_r > 0) {
+    e = cudaFuncSetAttribute(tc_bwd_rdelta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, RD_SMEM);
+    if (e != cudaSuccess) return e;
+    {
+      KernelTimer kt("tc_bwd_rdelta", s);
+      tc_bwd_rdelta_kernel<<<dim3(n_r, (unsigned)nkv), 128, RD_SMEM, s>>>(tm_q, tm_gr, a.chunk_delta, a.n_chunks,
+                                                                          wt + 1, a.group, a.status);
+    }
+    {
+      KernelTimer kt("tc_bwd_rscan", s);
+      tc_bwd_rscan_kernel<<<dim3((unsigned)nkv, 16), 256, 0, s>>>(a.chunk_delta, a.rstate, a.n_chunks, n_qt, wt + 1);
+    }
+    count_launches(2);
+  }
+
+  BwdArgs t;
+  t.dq = reinterpret_cast<__nv_bfloat16*>(a.dq);
+  t.dk = reinterpret_cast<__nv_bfloat16*>(a.dk);
+  t.dv = reinterpret_cast<__nv_bfloat16*>(a.dv);
+  t.lse = a.lse; t.delta = a.delta; t.status = a.status;
+  t.T = a.T; t.w = a.w; t.H_q = a.H_q; t.group = a.group; t.mode = a.mode; t.n_chunks = a.n_chunks;
+  t.scale = a.scale; t.scale_log2 = a.scale * LOG2E;
+  e = cudaFuncSetAttribute(tc_bwd_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DQ_SMEM);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(tc_bwd_dkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, KV_SMEM);
+  if (e != cudaSuccess) return e;
+  {
+    KernelTimer kt("tc_bwd_dq", s);
+    tc_bwd_dq_kernel<<<dim3(n_qt, (unsigned)nq), 160, DQ_SMEM, s>>>(tm_q, tm_k, tm_v, tm_gs, tm_gr, tm_st, t);
+  }
+  {
+    KernelTimer kt("tc_bwd_dkv", s);
+    tc_bwd_dkv_kernel<<<dim3(n_qt, (unsigned)nkv), 160, KV_SMEM, s>>>(tm_q, tm_k, tm_v, tm_gs, tm_gr, tm_rs, t);
+  }
+  count_launches(2);
+  return cudaGetLastError();
+}
+
+}  // namespace rattn

@@ -1,0 +1,118 @@
+// Pieces shared by the tensor-core kernels (forward and backward): the shared-memory tile
+// layout a 128-byte-swizzled TMA load produces, the tcgen05 operand descriptors for it, the
+// 128 x 128 x 128 MMA chains, the in-place feature map and the host-side tensor maps.
+#pragma once
+
+#include "rattn_internal.h"
+#include "tc_ptx.cuh"
+
+namespace rattn {
+namespace tc {
+
+using namespace ptx;
+
+constexpr int TILE = 128;
+constexpr int HALF_BYTES = TILE * 64 * 2;   // one [128 x 64] bf16 sub-tile, 128-byte rows
+constexpr int TILE_BYTES = 2 * HALF_BYTES;
+
+// K-major operand: [128 rows x 128 reduction] as two 64-wide halves; 16 reduction elements
+// per MMA = 32 bytes along the 128-byte row.
+__device__ __forceinline__ uint64_t kmajor_desc(uint32_t base, int kstep) {
+  return smem_desc(base + (kstep >> 2) * HALF_BYTES + (kstep & 3) * 32, 16, 1024);
+}
+// MN-major operand: rows are the reduction index (128-byte rows of 64 columns, two column
+// halves 16 KB apart); 16 reduction rows per MMA = 2048 bytes.
+__device__ __forceinline__ uint64_t mnmajor_desc(uint32_t base, int kstep) {
+  return smem_desc(base + kstep * 2048, HALF_BYTES, 1024);
+}
+
+// D[128x128] (+)= A B^T-style products over a reduction of 128, 8 MMAs of K = 16.
+__device__ __forceinline__ void mma_kk(uint32_t d, uint32_t a_base, uint32_t b_base, bool acc) {
+  constexpr uint32_t idesc = instr_desc(128, 128, 0, 0);
+#pragma unroll
+  for (int k = 0; k < 8; ++k) mma_bf16(d, kmajor_desc(a_base, k), kmajor_desc(b_base, k), idesc, (acc || k > 0) ? 1u : 0u);
+}
+template <int AB_BF16>
+__device__ __forceinline__ void mma_kmn(uint32_t d, uint32_t a_base, uint32_t b_base, bool acc) {
+  constexpr uint32_t idesc = instr_desc(128, 128, 0, 1, AB_BF16);
+#pragma unroll
+  for (int k = 0; k < 8; ++k) mma_bf16(d, kmajor_desc(a_base, k), mnmajor_desc(b_base, k), idesc, (acc || k > 0) ? 1u : 0u);
+}
+__device__ __forceinline__ void mma_mnmn(uint32_t d, uint32_t a_base, uint32_t b_base, bool acc) {
+  constexpr uint32_t idesc = instr_desc(128, 128, 1, 1);
+#pragma unroll
+  for (int k = 0; k < 8; ++k) mma_bf16(d, mnmajor_desc(a_base, k), mnmajor_desc(b_base, k), idesc, (acc || k > 0) ? 1u : 0u);
+}
+
+// byte offset of 16-byte chunk c (0..15) of row r inside a swizzled [128 x 128] bf16 tile
+__device__ __forceinline__ uint32_t swz(int r, int c) {
+  return (uint32_t)((c >> 3) * HALF_BYTES + r * 128 + (((c & 7) ^ (r & 7)) << 4));
+}
+
+// phi (softmax over the 128 features) of row r of a swizzled bf16 tile, in place.
+__device__ __forceinline__ void feature_map_row_inplace(unsigned char* tile, int r) {
+  float x[128];
+  float m = -INFINITY;
+#pragma unroll
+  for (int c = 0; c < 16; ++c) {
+    uint4 u = *reinterpret_cast<const uint4*>(tile + swz(r, c));
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      float2 f = __bfloat1622float2(h[e]);
+      x[c * 8 + 2 * e] = f.x;
+      x[c * 8 + 2 * e + 1] = f.y;
+      m = fmaxf(m, fmaxf(f.x, f.y));
+    }
+  }
+  float sum = 0.f;
+  const float ml = m * 1.4426950408889634f;
+#pragma unroll
+  for (int i = 0; i < 128; ++i) {
+    x[i] = ex2(x[i] * 1.4426950408889634f - ml);
+    sum += x[i];
+  }
+  const float inv = 1.f / sum;
+#pragma unroll
+  for (int c = 0; c < 16; ++c) {
+    uint4 u;
+    u.x = pack_bf16(x[c * 8 + 0] * inv, x[c * 8 + 1] * inv);
+    u.y = pack_bf16(x[c * 8 + 2] * inv, x[c * 8 + 3] * inv);
+    u.z = pack_bf16(x[c * 8 + 4] * inv, x[c * 8 + 5] * inv);
+    u.w = pack_bf16(x[c * 8 + 6] * inv, x[c * 8 + 7] * inv);
+    *reinterpret_cast<uint4*>(tile + swz(r, c)) = u;
+  }
+}
+
+
+// ------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess) return (EncodeTiledFn) nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// [n_mats, rows, 128] bf16, box = 64 columns x 128 rows x 1, 128-byte swizzle, zero fill.
+inline bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t n_mats) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {128, rows, n_mats};
+  const cuuint64_t strides[2] = {128 * 2, rows * 128 * 2};
+  const cuuint32_t box[3] = {64, 128, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+
+}  // namespace tc
+}  // namespace rattn

@@ -10,7 +10,7 @@ import torch
 from oracle import rattn_oracle as O
 from paper_2506_15545_b200 import binding as R
 from paper_2506_15545_b200 import workloads as W
-from test_gpu_parity import check, np64, small
+from test_gpu_parity import GRAD_TOL, check, np64, rel_fro, small
 
 pytestmark = pytest.mark.gpu
 
@@ -96,3 +96,92 @@ def test_tensor_run_to_run_determinism():
     a = R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws).clone()
     b = R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws)
     assert torch.equal(a, b)
+
+
+# ------------------------------------------------------------------ backward (tcgen05)
+
+def run_bwd(wl, mode=R.MODE_RATTN, gains=True):
+    """Tensor-core forward (saving residuals) + tensor-core backward against the oracle's
+    analytic fp64 gradients; returns the relative Frobenius errors per tensor."""
+    assert R.rattn_uses_tensor_path(wl.d, wl.w, R.RATTN_BF16, mode)
+    q, k, v = W.make_qkv(wl)
+    dy = W.make_dout(wl)
+    gs, gr = W.make_gains(wl) if gains else (None, None)
+    gsd = None if gs is None else gs.cuda()
+    grd = None if gr is None else gr.cuda()
+    qd, kd, vd, dyd = q.cuda(), k.cuda(), v.cuda(), dy.cuda()
+    ws = R.alloc_workspace(qd, kd, wl.w)
+    ws.zero_()
+    R.rattn_forward_ex(qd, kd, vd, wl.w, scale=wl.scale, mode=mode, workspace=ws, gamma_swa=gsd,
+                       gamma_rla=grd, save_residuals=True)
+    dgs = torch.empty(wl.H_q, wl.d, device="cuda")
+    dgr = torch.empty(wl.H_q, wl.d, device="cuda")
+    dq = torch.full_like(qd, float("nan"))
+    dk = torch.full_like(kd, float("nan"))
+    dv = torch.full_like(vd, float("nan"))
+    R.rattn_backward_ex(qd, kd, vd, dyd, wl.w, ws, scale=wl.scale, mode=mode, gamma_swa=gsd,
+                        gamma_rla=grd, dq=dq, dk=dk, dv=dv, dgamma_swa=dgs, dgamma_rla=dgr)
+    torch.cuda.synchronize()
+    assert R.rattn_read_status(ws) == 0, "a device-side wait expired"
+    ref = O.backward(np64(q), np64(k), np64(v), np64(dy), wl.w, wl.scale, 1e-6,
+                     None if gs is None else np64(gs), None if gr is None else np64(gr), mode)
+    errs = {}
+    for name, got, want in zip(("dq", "dk", "dv", "dgamma_swa"), (dq, dk, dv, dgs), ref):
+        assert np.isfinite(np64(got)).all(), name
+        errs[name] = rel_fro(np64(got), want)
+    if mode == R.MODE_RATTN and wl.w < wl.T - 1:
+        errs["dgamma_rla"] = rel_fro(np64(dgr), ref[4])
+    return errs
+
+
+@pytest.mark.parametrize("T,w,Hq,Hkv,unit", [
+    (128, 128, 1, 1, False),     # one tile: window branch only, diagonal mask only
+    (256, 128, 1, 1, True),      # residual branch in intra form only (no stored state either way)
+    (384, 128, 2, 1, True),      # forward state S_1 and reverse state R_0 both in play, group of 2
+    (640, 256, 4, 2, True),      # window of two tiles, GQA
+    (1280, 512, 2, 2, True),     # the w = 512 band
+    (300, 128, 2, 1, False),     # ragged T
+    (77, 128, 2, 2, False),      # T below one tile
+    (640, 1024, 2, 1, True),     # w > T: window branch covers everything
+])
+def test_tensor_backward_shapes(T, w, Hq, Hkv, unit):
+    wl = small("tcb", 2, Hq, Hkv, T, 128, w, "bf16", 5000 + T + w, unit=unit)
+    errs = run_bwd(wl)
+    for name, e in errs.items():
+        assert e <= GRAD_TOL, (name, e, errs)
+
+
+@pytest.mark.parametrize("mode", [R.MODE_SWA_ONLY, R.MODE_FULL_CAUSAL])
+def test_tensor_backward_control_modes(mode):
+    wl = small("tcbm", 1, 4, 2, 600, 128, 256, "bf16", 5100, unit=True)
+    errs = run_bwd(wl, mode=mode)
+    for name, e in errs.items():
+        assert e <= GRAD_TOL, (name, e, errs)
+
+
+def test_tensor_backward_matches_portable_backward():
+    """Same residuals, both backward paths: the two CUDA implementations agree far inside the
+    bound either has against the oracle."""
+    wl = small("tcbp", 1, 2, 1, 512, 128, 128, "bf16", 5200, unit=True)
+    q, k, v = (t.cuda() for t in W.make_qkv(wl))
+    dy = W.make_dout(wl).cuda()
+    ws = R.alloc_workspace(q, k, wl.w)
+    R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws, save_residuals=True)
+    a = R.rattn_backward_ex(q, k, v, dy, wl.w, ws, scale=wl.scale)
+    a = [t.clone() for t in a]
+    b = R.rattn_backward_ex(q, k, v, dy, wl.w, ws, scale=wl.scale, flags=R.FLAG_FORCE_GENERIC)
+    torch.cuda.synchronize()
+    for x, y in zip(a, b):
+        assert rel_fro(np64(x), np64(y)) <= 2e-2
+
+
+def test_tensor_backward_determinism():
+    wl = small("tcbd", 1, 4, 2, 768, 128, 256, "bf16", 5300, unit=True)
+    q, k, v = (t.cuda() for t in W.make_qkv(wl))
+    dy = W.make_dout(wl).cuda()
+    ws = R.alloc_workspace(q, k, wl.w)
+    R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws, save_residuals=True)
+    a = [t.clone() for t in R.rattn_backward_ex(q, k, v, dy, wl.w, ws, scale=wl.scale)]
+    b = R.rattn_backward_ex(q, k, v, dy, wl.w, ws, scale=wl.scale)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
