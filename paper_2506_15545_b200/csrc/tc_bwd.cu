@@ -55,8 +55,6 @@ __device__ __forceinline__ void load_tile(unsigned char* dst, const CUtensorMap*
   tma_load_3d(dst + HALF_BYTES, tm, bar, 64, row, z);
 }
 
-__device__ __forceinline__ void named_sync_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
 // ------------------------------------------------------------------------------ prep
 // One warp per row; lane owns 4 consecutive features.  Writes g_s, g_r (bf16), D and, when
 // asked, accumulates the gain gradients.
@@ -315,7 +313,7 @@ __device__ bool dq_control(const CUtensorMap* tm_q, const CUtensorMap* tm_k, con
   return true;
 }
 
-__device__ bool dq_rows(const BwdArgs& a, unsigned char* smem, DqBars* bars, uint32_t tmem, int r, int q0,
+__device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned char* smem, DqBars* bars, uint32_t tmem, int r, int q0,
                         int bh_q, int n_kt, bool has_boundary, bool has_rla) {
   const uint32_t lane_off = (uint32_t)((r & ~31) << 16);
   const uint32_t tS = tmem + lane_off, tP = tmem + 128 + lane_off, tQ = tmem + 256 + lane_off,
@@ -428,7 +426,7 @@ __device__ bool dq_rows(const BwdArgs& a, unsigned char* smem, DqBars* bars, uin
     dot = du * inv;
     m = ml;
   }
-  __nv_bfloat16* orow = a.dq + row * 128;
+  // every product has completed: the dS tile is free and stages the output for one TMA store
 #pragma unroll 1
   for (int c = 0; c < 4; ++c) {
     float x[32], df[32];
@@ -449,17 +447,22 @@ __device__ bool dq_rows(const BwdArgs& a, unsigned char* smem, DqBars* bars, uin
         }
       }
     }
-    if (live) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        uint4 u;
-        u.x = pack_bf16(x[8 * e + 0], x[8 * e + 1]);
-        u.y = pack_bf16(x[8 * e + 2], x[8 * e + 3]);
-        u.z = pack_bf16(x[8 * e + 4], x[8 * e + 5]);
-        u.w = pack_bf16(x[8 * e + 6], x[8 * e + 7]);
-        *reinterpret_cast<uint4*>(orow + 32 * c + 8 * e) = u;
-      }
+    for (int e = 0; e < 4; ++e) {
+      uint4 u;
+      u.x = pack_bf16(x[8 * e + 0], x[8 * e + 1]);
+      u.y = pack_bf16(x[8 * e + 2], x[8 * e + 3]);
+      u.z = pack_bf16(x[8 * e + 4], x[8 * e + 5]);
+      u.w = pack_bf16(x[8 * e + 6], x[8 * e + 7]);
+      *reinterpret_cast<uint4*>(sD + swz(r, 4 * c + e)) = u;
     }
+  }
+  fence_proxy_async_smem();
+  rows_sync();
+  if (r == 0) {
+    store_tile(tm_dq, sD, q0, bh_q);
+    tma_store_commit();
+    tma_store_wait_read();
   }
   tc_fence_before();
   return true;
@@ -468,7 +471,8 @@ __device__ bool dq_rows(const BwdArgs& a, unsigned char* smem, DqBars* bars, uin
 __global__ void __launch_bounds__(160, 1)
 tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_gs,
-                 const __grid_constant__ CUtensorMap tm_gr, const __grid_constant__ CUtensorMap tm_st, BwdArgs a) {
+                 const __grid_constant__ CUtensorMap tm_gr, const __grid_constant__ CUtensorMap tm_st,
+                 const __grid_constant__ CUtensorMap tm_dq, BwdArgs a) {
   extern __shared__ __align__(1024) unsigned char smem[];
   DqBars* bars = reinterpret_cast<DqBars*>(smem + DQ_OFF_BAR);
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -515,6 +519,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       prefetch_tensormap(&tm_gs);
       prefetch_tensormap(&tm_gr);
       prefetch_tensormap(&tm_st);
+      prefetch_tensormap(&tm_dq);
     }
   }
   tc_fence_before();
@@ -524,7 +529,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
   bool ok = true;
   if (warp < 4) {
-    ok = dq_rows(a, smem, bars, tmem, tid, q0, bh_q, n_kt, has_boundary, has_rla);
+    ok = dq_rows(a, &tm_dq, smem, bars, tmem, tid, q0, bh_q, n_kt, has_boundary, has_rla);
   } else if (tid == 128) {
     ok = dq_control(&tm_q, &tm_k, &tm_v, &tm_gs, &tm_gr, &tm_st, smem, bars, tmem, q0, bh_q, bh_kv, n_kt,
                     has_rla, has_state, st_index);
@@ -659,7 +664,7 @@ __device__ bool kv_control(const CUtensorMap* tm_q, const CUtensorMap* tm_k, con
   return true;
 }
 
-__device__ bool kv_rows(const BwdArgs& a, unsigned char* smem, KvBars* bars, uint32_t tmem, const KvPlan& pl,
+__device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtensorMap* tm_dv, unsigned char* smem, KvBars* bars, uint32_t tmem, const KvPlan& pl,
                         int r, int bh_kv) {
   const uint32_t lane_off = (uint32_t)((r & ~31) << 16);
   const uint32_t tS = tmem + lane_off, tP = tmem + 128 + lane_off, tV = tmem + 256 + lane_off,
@@ -690,7 +695,7 @@ __device__ bool kv_rows(const BwdArgs& a, unsigned char* smem, KvBars* bars, uin
       const size_t row = (size_t)bq * a.T + t;
       stat[st * 256 + r] = t < a.T ? a.lse[row] * LOG2E : INFINITY;
       stat[st * 256 + 128 + r] = t < a.T ? a.delta[row] * a.scale : 0.f;
-      named_sync_128();
+      rows_sync();
     }
     WAIT_OR_RETURN(bars->s_full, n & 1);
     tc_fence_after();
@@ -799,30 +804,36 @@ __device__ bool kv_rows(const BwdArgs& a, unsigned char* smem, KvBars* bars, uin
 
   WAIT_OR_RETURN(bars->acc2_done, (pl.N - 1) & 1);
   tc_fence_after();
-  const int jj = pl.j * TILE + r;
-  const size_t row = (size_t)bh_kv * a.T + jj;
+  // every product has completed: dK is staged in the dS tile, dV in the first query stage
+  unsigned char* sOutV = smem + KV_OFF_Q;
 #pragma unroll 1
   for (int c = 0; c < 4; ++c) {
     float xk[32], xv[32];
     tmem_ld32(tK + 32 * c, xk);
     tmem_ld32(tV + 32 * c, xv);
     tmem_wait_ld();
-    if (jj < a.T) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        uint4 u;
-        u.x = pack_bf16(xk[8 * e + 0], xk[8 * e + 1]);
-        u.y = pack_bf16(xk[8 * e + 2], xk[8 * e + 3]);
-        u.z = pack_bf16(xk[8 * e + 4], xk[8 * e + 5]);
-        u.w = pack_bf16(xk[8 * e + 6], xk[8 * e + 7]);
-        *reinterpret_cast<uint4*>(a.dk + row * 128 + 32 * c + 8 * e) = u;
-        u.x = pack_bf16(xv[8 * e + 0], xv[8 * e + 1]);
-        u.y = pack_bf16(xv[8 * e + 2], xv[8 * e + 3]);
-        u.z = pack_bf16(xv[8 * e + 4], xv[8 * e + 5]);
-        u.w = pack_bf16(xv[8 * e + 6], xv[8 * e + 7]);
-        *reinterpret_cast<uint4*>(a.dv + row * 128 + 32 * c + 8 * e) = u;
-      }
+    for (int e = 0; e < 4; ++e) {
+      uint4 u;
+      u.x = pack_bf16(xk[8 * e + 0], xk[8 * e + 1]);
+      u.y = pack_bf16(xk[8 * e + 2], xk[8 * e + 3]);
+      u.z = pack_bf16(xk[8 * e + 4], xk[8 * e + 5]);
+      u.w = pack_bf16(xk[8 * e + 6], xk[8 * e + 7]);
+      *reinterpret_cast<uint4*>(sD + swz(r, 4 * c + e)) = u;
+      u.x = pack_bf16(xv[8 * e + 0], xv[8 * e + 1]);
+      u.y = pack_bf16(xv[8 * e + 2], xv[8 * e + 3]);
+      u.z = pack_bf16(xv[8 * e + 4], xv[8 * e + 5]);
+      u.w = pack_bf16(xv[8 * e + 6], xv[8 * e + 7]);
+      *reinterpret_cast<uint4*>(sOutV + swz(r, 4 * c + e)) = u;
     }
+  }
+  fence_proxy_async_smem();
+  rows_sync();
+  if (r == 0) {
+    store_tile(tm_dk, sD, pl.j * TILE, bh_kv);
+    store_tile(tm_dv, sOutV, pl.j * TILE, bh_kv);
+    tma_store_commit();
+    tma_store_wait_read();
   }
   tc_fence_before();
   return true;
@@ -831,7 +842,8 @@ __device__ bool kv_rows(const BwdArgs& a, unsigned char* smem, KvBars* bars, uin
 __global__ void __launch_bounds__(160, 1)
 tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_gs,
-                  const __grid_constant__ CUtensorMap tm_gr, const __grid_constant__ CUtensorMap tm_rs, BwdArgs a) {
+                  const __grid_constant__ CUtensorMap tm_gr, const __grid_constant__ CUtensorMap tm_rs,
+                  const __grid_constant__ CUtensorMap tm_dk, const __grid_constant__ CUtensorMap tm_dv, BwdArgs a) {
   extern __shared__ __align__(1024) unsigned char smem[];
   KvBars* bars = reinterpret_cast<KvBars*>(smem + KV_OFF_BAR);
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -884,6 +896,8 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       prefetch_tensormap(&tm_gs);
       prefetch_tensormap(&tm_gr);
       prefetch_tensormap(&tm_rs);
+      prefetch_tensormap(&tm_dk);
+      prefetch_tensormap(&tm_dv);
     }
   }
   tc_fence_before();
@@ -893,7 +907,7 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
   bool ok = true;
   if (warp < 4) {
-    ok = kv_rows(a, smem, bars, tmem, pl, tid, bh_kv);
+    ok = kv_rows(a, &tm_dk, &tm_dv, smem, bars, tmem, pl, tid, bh_kv);
   } else if (tid == 128) {
     ok = kv_control(&tm_q, &tm_k, &tm_v, &tm_gs, &tm_gr, &tm_rs, smem, bars, tmem, pl, bh_kv, rs_index);
     if (!ok) {
@@ -936,10 +950,11 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
   }
   count_launches(1);
 
-  CUtensorMap tm_q, tm_k, tm_v, tm_gs, tm_gr, tm_st, tm_rs;
+  CUtensorMap tm_q, tm_k, tm_v, tm_gs, tm_gr, tm_st, tm_rs, tm_dq, tm_dk, tm_dv;
   const uint64_t nq = (uint64_t)a.B * a.H_q, nkv = (uint64_t)a.B * a.H_kv;
   if (!make_map(&tm_q, a.q, a.T, nq) || !make_map(&tm_k, a.k, a.T, nkv) || !make_map(&tm_v, a.v, a.T, nkv) ||
       !make_map(&tm_gs, g_s, a.T, nq) || !make_map(&tm_gr, g_r, a.T, nq) ||
+      !make_map(&tm_dq, a.dq, a.T, nq) || !make_map(&tm_dk, a.dk, a.T, nkv) || !make_map(&tm_dv, a.dv, a.T, nkv) ||
       !make_map(&tm_st, a.chunk_state, 128, nkv * a.n_chunks) || !make_map(&tm_rs, a.rstate, 128, nkv * a.n_chunks))
     return cudaErrorInvalidValue;
 
@@ -973,11 +988,11 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
   if (e != cudaSuccess) return e;
   {
     KernelTimer kt("tc_bwd_dq", s);
-    tc_bwd_dq_kernel<<<dim3(n_qt, (unsigned)nq), 160, DQ_SMEM, s>>>(tm_q, tm_k, tm_v, tm_gs, tm_gr, tm_st, t);
+    tc_bwd_dq_kernel<<<dim3(n_qt, (unsigned)nq), 160, DQ_SMEM, s>>>(tm_q, tm_k, tm_v, tm_gs, tm_gr, tm_st, tm_dq, t);
   }
   {
     KernelTimer kt("tc_bwd_dkv", s);
-    tc_bwd_dkv_kernel<<<dim3(n_qt, (unsigned)nkv), 160, KV_SMEM, s>>>(tm_q, tm_k, tm_v, tm_gs, tm_gr, tm_rs, t);
+    tc_bwd_dkv_kernel<<<dim3(n_qt, (unsigned)nkv), 160, KV_SMEM, s>>>(tm_q, tm_k, tm_v, tm_gs, tm_gr, tm_rs, tm_dk, tm_dv, t);
   }
   count_launches(2);
   return cudaGetLastError();

@@ -49,6 +49,33 @@ __device__ __forceinline__ uint32_t swz(int r, int c) {
   return (uint32_t)((c >> 3) * HALF_BYTES + r * 128 + (((c & 7) ^ (r & 7)) << 4));
 }
 
+// One [128 x 128] bf16 tile staged in shared memory (swizzled like a loaded tile) goes to
+// rows row0.. of matrix z of a tensor map: two 64-column boxes; rows past the end are clipped.
+__device__ __forceinline__ void store_tile(const CUtensorMap* tm, const unsigned char* tile, int row0, int z) {
+  tma_store_3d(tm, tile, 0, row0, z);
+  tma_store_3d(tm, tile + HALF_BYTES, 64, row0, z);
+}
+
+// Row-owner r holds 32 fp32 values (columns 32*c .. 32*c+31 of its row).  Stages them in a
+// 16 KB region ([128 rows x 128 bytes], 16-byte chunks XOR-swizzled by row) so that the 128
+// row owners can then write the [128 x 32] block to global memory with full 128-byte segments.
+__device__ __forceinline__ void stage_f32_block(unsigned char* stage, int r, const float (&x)[32]) {
+#pragma unroll
+  for (int e = 0; e < 8; ++e)
+    *reinterpret_cast<float4*>(stage + r * 128 + ((e ^ (r & 7)) << 4)) =
+        make_float4(x[4 * e], x[4 * e + 1], x[4 * e + 2], x[4 * e + 3]);
+}
+// dst points at column 32*c of the tile's first row (row pitch 128 floats); rows >= n_rows are skipped.
+__device__ __forceinline__ void flush_f32_block(const unsigned char* stage, int r, float* dst, int n_rows) {
+  const int sub = r & 7;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const int row = (r >> 5) * 32 + 4 * k + ((r & 31) >> 3);
+    const float4 v = *reinterpret_cast<const float4*>(stage + row * 128 + ((sub ^ (row & 7)) << 4));
+    if (row < n_rows) *reinterpret_cast<float4*>(dst + (size_t)row * 128 + 4 * sub) = v;
+  }
+}
+
 // phi (softmax over the 128 features) of row r of a swizzled bf16 tile, in place.
 __device__ __forceinline__ void feature_map_row_inplace(unsigned char* tile, int r) {
   float x[128];

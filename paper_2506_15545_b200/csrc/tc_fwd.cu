@@ -136,7 +136,7 @@ __device__ bool control_role(const CUtensorMap* tm_q, const CUtensorMap* tm_k, c
 }
 
 // ------------------------------------------------------------------ softmax / epilogue
-__device__ bool softmax_role(const TcArgs& a, unsigned char* smem, FwdBars* bars, uint32_t tmem, int r,
+__device__ bool softmax_role(const TcArgs& a, const CUtensorMap* tm_out, unsigned char* smem, FwdBars* bars, uint32_t tmem, int r,
                              int q0, int bh_q, int h, int n_kt, bool has_boundary, bool has_rla) {
   const uint32_t lane_off = (uint32_t)((r & ~31) << 16);   // this warp's 32 TMEM lanes
   const uint32_t tS[2] = {tmem + lane_off, tmem + 128 + lane_off};
@@ -261,44 +261,58 @@ __device__ bool softmax_role(const TcArgs& a, unsigned char* smem, FwdBars* bars
   const int t = q0 + r;
   const bool live = t < a.T;
   const size_t row = (size_t)bh_q * a.T + t;
-  __nv_bfloat16* orow = a.out + row * 128;
-#pragma unroll
+  // Every product has completed, so the operand tiles are free: y is staged in the P tile
+  // (bf16, swizzled) for one TMA store, the fp32 residuals in the K stages, 32 columns at a
+  // time, so that each warp writes whole 128-byte segments of its own 32 rows.
+  unsigned char* sY = smem + OFF_P;
+  unsigned char* stage_s = smem + OFF_K;
+  unsigned char* stage_r = smem + OFF_K + 16384;
+  const size_t tile_row0 = (size_t)bh_q * a.T + q0;
+#pragma unroll 1
   for (int c = 0; c < 4; ++c) {
     float os[32], orl[32];
     tmem_ld32(tOs + 32 * c, os);
     if (has_rla) tmem_ld32(tOr + 32 * c, orl);
     tmem_wait_ld();
-    if (live) {
-      float y[32];
+    float y[32];
 #pragma unroll
-      for (int e = 0; e < 32; ++e) {
-        const float gs = a.gamma_swa ? __ldg(a.gamma_swa + (size_t)h * 128 + 32 * c + e) : 1.f;
-        y[e] = gs * os[e] * rs;
-        if (has_rla) {
-          const float gr = a.gamma_rla ? __ldg(a.gamma_rla + (size_t)h * 128 + 32 * c + e) : 1.f;
-          y[e] += gr * orl[e] * rr;
-        }
-      }
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        uint4 u;
-        u.x = pack_bf16(y[8 * e + 0], y[8 * e + 1]);
-        u.y = pack_bf16(y[8 * e + 2], y[8 * e + 3]);
-        u.z = pack_bf16(y[8 * e + 4], y[8 * e + 5]);
-        u.w = pack_bf16(y[8 * e + 6], y[8 * e + 7]);
-        *reinterpret_cast<uint4*>(orow + 32 * c + 8 * e) = u;
-      }
-      if (a.o_swa) {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          *reinterpret_cast<float4*>(a.o_swa + row * 128 + 32 * c + 4 * e) =
-              make_float4(os[4 * e] * inv_l, os[4 * e + 1] * inv_l, os[4 * e + 2] * inv_l, os[4 * e + 3] * inv_l);
-          *reinterpret_cast<float4*>(a.o_rla + row * 128 + 32 * c + 4 * e) =
-              has_rla ? make_float4(orl[4 * e], orl[4 * e + 1], orl[4 * e + 2], orl[4 * e + 3])
-                      : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
+    for (int e = 0; e < 32; ++e) {
+      const float gs = a.gamma_swa ? __ldg(a.gamma_swa + (size_t)h * 128 + 32 * c + e) : 1.f;
+      y[e] = gs * os[e] * rs;
+      if (has_rla) {
+        const float gr = a.gamma_rla ? __ldg(a.gamma_rla + (size_t)h * 128 + 32 * c + e) : 1.f;
+        y[e] += gr * orl[e] * rr;
       }
     }
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      uint4 u;
+      u.x = pack_bf16(y[8 * e + 0], y[8 * e + 1]);
+      u.y = pack_bf16(y[8 * e + 2], y[8 * e + 3]);
+      u.z = pack_bf16(y[8 * e + 4], y[8 * e + 5]);
+      u.w = pack_bf16(y[8 * e + 6], y[8 * e + 7]);
+      *reinterpret_cast<uint4*>(sY + swz(r, 4 * c + e)) = u;
+    }
+    if (a.o_swa) {
+#pragma unroll
+      for (int e = 0; e < 32; ++e) {
+        os[e] *= inv_l;
+        if (!has_rla) orl[e] = 0.f;
+      }
+      __syncwarp();
+      stage_f32_block(stage_s, r, os);
+      stage_f32_block(stage_r, r, orl);
+      __syncwarp();
+      flush_f32_block(stage_s, r, a.o_swa + tile_row0 * 128 + 32 * c, a.T - q0);
+      flush_f32_block(stage_r, r, a.o_rla + tile_row0 * 128 + 32 * c, a.T - q0);
+    }
+  }
+  fence_proxy_async_smem();
+  rows_sync();
+  if (r == 0) {
+    store_tile(tm_out, sY, q0, bh_q);
+    tma_store_commit();
+    tma_store_wait_read();
   }
   if (live && a.lse) a.lse[row] = (m_ref + log2f(l)) * 0.6931471805599453f;
   tc_fence_before();
@@ -327,7 +341,8 @@ __device__ bool convert_role(unsigned char* smem, FwdBars* bars, int cid, int n_
 
 __global__ void __launch_bounds__(256, 1)
 tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-              const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_st, TcArgs a) {
+              const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_st,
+              const __grid_constant__ CUtensorMap tm_out, TcArgs a) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   FwdBars* bars = reinterpret_cast<FwdBars*>(smem + OFF_BAR);
@@ -373,6 +388,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
       prefetch_tensormap(&tm_k);
       prefetch_tensormap(&tm_v);
       prefetch_tensormap(&tm_st);
+      prefetch_tensormap(&tm_out);
     }
   }
   tc_fence_before();
@@ -382,7 +398,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 
   bool ok = true;
   if (warp < 4) {
-    ok = softmax_role(a, smem, bars, tmem, tid, q0, bh_q, h, n_kt, has_boundary, has_rla);
+    ok = softmax_role(a, &tm_out, smem, bars, tmem, tid, q0, bh_q, h, n_kt, has_boundary, has_rla);
   } else if (tid == 128) {
     ok = control_role(&tm_q, &tm_k, &tm_v, &tm_st, smem, bars, tmem, q0, bh_q, bh_kv, n_kt, has_rla,
                       has_state, st_index);
@@ -490,10 +506,11 @@ tc_chunk_scan_kernel(const float* __restrict__ delta, __nv_bfloat16* __restrict_
 }  // namespace
 
 cudaError_t launch_tc_forward(const Args& a, cudaStream_t s) {
-  CUtensorMap tm_q, tm_k, tm_v, tm_st;
+  CUtensorMap tm_q, tm_k, tm_v, tm_st, tm_out;
   if (!make_map(&tm_q, a.q, a.T, (uint64_t)a.B * a.H_q)) return cudaErrorInvalidValue;
   if (!make_map(&tm_k, a.k, a.T, (uint64_t)a.B * a.H_kv)) return cudaErrorInvalidValue;
   if (!make_map(&tm_v, a.v, a.T, (uint64_t)a.B * a.H_kv)) return cudaErrorInvalidValue;
+  if (!make_map(&tm_out, a.out, a.T, (uint64_t)a.B * a.H_q)) return cudaErrorInvalidValue;
   if (!make_map(&tm_st, a.chunk_state, 128, (uint64_t)a.B * a.H_kv * a.n_chunks)) return cudaErrorInvalidValue;
 
   const int n_qt = (a.T + TILE - 1) / TILE;
@@ -522,7 +539,7 @@ cudaError_t launch_tc_forward(const Args& a, cudaStream_t s) {
   if (e != cudaSuccess) return e;
   {
     KernelTimer kt("tc_fwd", s);
-    tc_fwd_kernel<<<dim3(n_qt, a.B * a.H_q), 256, FWD_SMEM, s>>>(tm_q, tm_k, tm_v, tm_st, t);
+    tc_fwd_kernel<<<dim3(n_qt, a.B * a.H_q), 256, FWD_SMEM, s>>>(tm_q, tm_k, tm_v, tm_st, tm_out, t);
   }
   count_launches(1);
   return cudaGetLastError();
