@@ -68,6 +68,9 @@ WorkspaceLayout workspace_layout(int B, int H_q, int H_kv, int T, int d, int w, 
   L.chunk_delta = off; off += align256(states * sizeof(float));
   L.chunk_state = off; off += align256(states * sizeof(__nv_bfloat16));
   L.rstate = off;      off += align256(states * sizeof(__nv_bfloat16));
+  const size_t rows_pad = (size_t)B * H_q * L.n_chunks * 128;
+  L.lse2p = off;       off += align256(rows_pad * sizeof(float));
+  L.dscp = off;        off += align256(rows_pad * sizeof(float));
   L.total = off;
   return L;
 }
@@ -119,6 +122,8 @@ static int bind_workspace(const rattn_params* p, Args* a, bool required) {
   a->chunk_delta = reinterpret_cast<float*>(base + L.chunk_delta);
   a->chunk_state = reinterpret_cast<__nv_bfloat16*>(base + L.chunk_state);
   a->rstate = reinterpret_cast<__nv_bfloat16*>(base + L.rstate);
+  a->lse2p = reinterpret_cast<float*>(base + L.lse2p);
+  a->dscp = reinterpret_cast<float*>(base + L.dscp);
   a->n_chunks = L.n_chunks;
   return RATTN_OK;
 }

@@ -23,6 +23,8 @@ struct WorkspaceLayout {
   size_t chunk_delta;   // fp32 [B,H_kv,n_chunks,d,d]  per-chunk phi(K)^T V
   size_t chunk_state;   // bf16 [B,H_kv,n_chunks,d,d]  exclusive prefix over chunks
   size_t rstate;        // bf16 [B,H_kv,n_chunks,d,d]  backward: suffix sums of phi(Q)^T g_r
+  size_t lse2p;         // fp32 [B*H_q, n_chunks*128]  backward: lse * log2(e), +inf in the padding
+  size_t dscp;          // fp32 [B*H_q, n_chunks*128]  backward: D_t * scale, 0 in the padding
   size_t total;
   int n_chunks;         // ceil(T / 128)
 };
@@ -49,6 +51,8 @@ struct Args {
   float* chunk_delta;
   __nv_bfloat16* chunk_state;
   __nv_bfloat16* rstate;
+  float* lse2p;
+  float* dscp;
   int n_chunks;
   int* status;                 // device status word (may be null when no workspace)
   // hand-off

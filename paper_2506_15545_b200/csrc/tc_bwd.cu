@@ -42,6 +42,9 @@ struct BwdArgs {
   __nv_bfloat16* dv;
   const float* lse;     // [B,H_q,T]  natural-log log-sum-exp of the window logits
   const float* delta;   // [B,H_q,T]  D_t
+  const float* lse2p;   // [B*H_q, t_pad]  lse * log2(e), +inf beyond T   (t_pad = T rounded up to 128)
+  const float* dscp;    // [B*H_q, t_pad]  D_t * scale, 0 beyond T
+  int t_pad;
   int* status;
   int T, w, H_q, group, mode, n_chunks;
   float scale, scale_log2;
@@ -49,11 +52,6 @@ struct BwdArgs {
 
 #define WAIT_OR_RETURN(bar, parity) \
   do { if (!mbar_wait(&(bar), (parity), &bars->abort)) return false; } while (0)
-
-__device__ __forceinline__ void load_tile(unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int row, int z) {
-  tma_load_3d(dst, tm, bar, 0, row, z);
-  tma_load_3d(dst + HALF_BYTES, tm, bar, 64, row, z);
-}
 
 // ------------------------------------------------------------------------------ prep
 // One warp per row; lane owns 4 consecutive features.  Writes g_s, g_r (bf16), D and, when
@@ -63,7 +61,9 @@ tc_bwd_prep_kernel(const __nv_bfloat16* __restrict__ dy, const float* __restrict
                    const float* __restrict__ o_r, const float* __restrict__ gamma_s,
                    const float* __restrict__ gamma_r, __nv_bfloat16* __restrict__ g_s,
                    __nv_bfloat16* __restrict__ g_r, float* __restrict__ delta, float* __restrict__ dgamma_s,
-                   float* __restrict__ dgamma_r, size_t n_rows, int T, int H_q, float eps, int rla_on) {
+                   float* __restrict__ dgamma_r, const float* __restrict__ lse, float* __restrict__ lse2p,
+                   float* __restrict__ dscp, size_t n_rows_pad, int T, int t_pad, int H_q, float eps, float scale,
+                   int rla_on) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   constexpr int ROWS_PER_CTA = 64;
   const size_t row0 = (size_t)blockIdx.x * ROWS_PER_CTA;
@@ -80,9 +80,19 @@ tc_bwd_prep_kernel(const __nv_bfloat16* __restrict__ dy, const float* __restrict
     }
   };
   for (int rr = warp; rr < ROWS_PER_CTA; rr += 8) {
-    const size_t row = row0 + rr;
-    if (row >= n_rows) break;
-    const int h = (int)((row / T) % H_q);
+    const size_t prow = row0 + rr;                 // row of the padded [B*H_q, t_pad] index space
+    if (prow >= n_rows_pad) break;
+    const size_t bq = prow / t_pad;
+    const int t = (int)(prow % t_pad);
+    if (t >= T) {                                  // padding: statistics that make every weight zero
+      if (lane == 0) {
+        lse2p[prow] = INFINITY;
+        dscp[prow] = 0.f;
+      }
+      continue;
+    }
+    const size_t row = bq * T + t;
+    const int h = (int)(bq % H_q);
     const float4 xs = *reinterpret_cast<const float4*>(o_s + row * 128 + 4 * lane);
     const float4 xr = *reinterpret_cast<const float4*>(o_r + row * 128 + 4 * lane);
     const uint2 gy = *reinterpret_cast<const uint2*>(dy + row * 128 + 4 * lane);
@@ -136,7 +146,11 @@ tc_bwd_prep_kernel(const __nv_bfloat16* __restrict__ dy, const float* __restrict
     for (int o = 16; o > 0; o >>= 1) dl += __shfl_xor_sync(0xffffffffu, dl, o);
     *reinterpret_cast<uint2*>(g_s + row * 128 + 4 * lane) = make_uint2(pack_bf16(ds[0], ds[1]), pack_bf16(ds[2], ds[3]));
     *reinterpret_cast<uint2*>(g_r + row * 128 + 4 * lane) = make_uint2(pack_bf16(dr[0], dr[1]), pack_bf16(dr[2], dr[3]));
-    if (lane == 0) delta[row] = dl;
+    if (lane == 0) {
+      delta[row] = dl;
+      lse2p[prow] = lse[row] * LOG2E;
+      dscp[prow] = dl * scale;
+    }
   }
   if (dgamma_s || dgamma_r) flush();
 }
@@ -264,42 +278,35 @@ __device__ bool dq_control(const CUtensorMap* tm_q, const CUtensorMap* tm_k, con
     load_tile(smem + DQ_OFF_V + i * TILE_BYTES, tm_v, &bars->kv_full[i], q0 - i * TILE, bh_kv);
   }
   WAIT_OR_RETURN(bars->qg_full, 0);
+  constexpr uint32_t idesc_ts = instr_desc(128, 128, 0, 1);
+  const int last = (n_kt - 1) & 1, other = last ^ 1;
   for (int i = 0; i < n_kt; ++i) {
     const int b = i & 1;
     WAIT_OR_RETURN(bars->kv_full[b], (i >> 1) & 1);
-    if (i > 0) WAIT_OR_RETURN(bars->s_empty, (i - 1) & 1);
     tc_fence_after();
     mma_kk(tS, sQ, sK + b * TILE_BYTES, false);          // S  = Q K^T
     mma_kk(tP, sG, sV + b * TILE_BYTES, false);          // dP = g_s V^T
     mma_commit(&bars->s_full);
-    if (i > 0) {
-      const int pb = (i - 1) & 1;
-      WAIT_OR_RETURN(bars->ds_full, (i - 1) & 1);
-      tc_fence_after();
-      mma_kmn<1>(tQ, sD, sK + pb * TILE_BYTES, i - 1 > 0); // dQ += dS K
-      mma_commit(&bars->dq_done);
-      WAIT_OR_RETURN(bars->dq_done, (i - 1) & 1);          // stage pb is free again
-      if (i + 1 < n_kt) {
-        mbar_arrive_expect_tx(&bars->kv_full[pb], 2 * TILE_BYTES);
-        load_tile(smem + DQ_OFF_K + pb * TILE_BYTES, tm_k, &bars->kv_full[pb], q0 - (i + 1) * TILE, bh_kv);
-        load_tile(smem + DQ_OFF_V + pb * TILE_BYTES, tm_v, &bars->kv_full[pb], q0 - (i + 1) * TILE, bh_kv);
-      } else if (has_rla) {
-        // the free stage receives the residual branch's operands: g_r and the stored state
-        mbar_arrive_expect_tx(&bars->x_full, (has_state ? 2 : 1) * TILE_BYTES);
-        load_tile(smem + DQ_OFF_V + pb * TILE_BYTES, tm_gr, &bars->x_full, q0, bh_q);
-        if (has_state) load_tile(smem + DQ_OFF_K + pb * TILE_BYTES, tm_st, &bars->x_full, 0, st_index);
-      }
+    WAIT_OR_RETURN(bars->ds_full, i & 1);
+    tc_fence_after();
+#pragma unroll
+    for (int k = 0; k < 8; ++k)                           // dQ += dS K, dS read from TMEM
+      mma_bf16_ts(tQ, tS + 8 * k, mnmajor_desc(sK + b * TILE_BYTES, k), idesc_ts, (i > 0 || k > 0) ? 1u : 0u);
+    mma_commit(&bars->dq_done);
+    WAIT_OR_RETURN(bars->dq_done, i & 1);
+    if (i + 2 < n_kt) {
+      mbar_arrive_expect_tx(&bars->kv_full[b], 2 * TILE_BYTES);
+      load_tile(smem + DQ_OFF_K + b * TILE_BYTES, tm_k, &bars->kv_full[b], q0 - (i + 2) * TILE, bh_kv);
+      load_tile(smem + DQ_OFF_V + b * TILE_BYTES, tm_v, &bars->kv_full[b], q0 - (i + 2) * TILE, bh_kv);
+    } else if (has_rla && i + 2 == n_kt) {
+      mbar_arrive_expect_tx(&bars->x_full, (has_state ? 2 : 1) * TILE_BYTES);
+      load_tile(smem + DQ_OFF_V + b * TILE_BYTES, tm_gr, &bars->x_full, q0, bh_q);
+      if (has_state) load_tile(smem + DQ_OFF_K + b * TILE_BYTES, tm_st, &bars->x_full, 0, st_index);
     }
   }
-  const int last = (n_kt - 1) & 1, other = last ^ 1;
-  WAIT_OR_RETURN(bars->ds_full, (n_kt - 1) & 1);
-  tc_fence_after();
-  mma_kmn<1>(tQ, sD, sK + last * TILE_BYTES, n_kt - 1 > 0);
-  mma_commit(&bars->dq_done);
   if (has_rla) {
     const uint32_t sG2 = sV + other * TILE_BYTES, sSt = sK + other * TILE_BYTES;
     WAIT_OR_RETURN(bars->x_full, 0);
-    WAIT_OR_RETURN(bars->s_empty, (n_kt - 1) & 1);
     tc_fence_after();
     mma_kk(tS, sG2, sV + last * TILE_BYTES, false);        // dA = g_r V_cb^T
     if (has_state) mma_kk(tF, sG2, sSt, false);            // g_r S_cb^T
@@ -307,7 +314,9 @@ __device__ bool dq_control(const CUtensorMap* tm_q, const CUtensorMap* tm_k, con
     WAIT_OR_RETURN(bars->phik_ready, 0);
     WAIT_OR_RETURN(bars->ds_full, n_kt & 1);
     tc_fence_after();
-    mma_kmn<1>(tF, sD, sK + last * TILE_BYTES, has_state); // (dA masked) phi(K_cb)
+#pragma unroll
+    for (int k = 0; k < 8; ++k)                           // (dA masked) phi(K_cb)
+      mma_bf16_ts(tF, tS + 8 * k, mnmajor_desc(sK + last * TILE_BYTES, k), idesc_ts, (has_state || k > 0) ? 1u : 0u);
   }
   mma_commit(&bars->o_done);
   return true;
@@ -329,13 +338,13 @@ __device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned cha
     WAIT_OR_RETURN(bars->s_full, i & 1);
     tc_fence_after();
     const bool diag = (i == 0), bound = has_boundary && (i == n_kt - 1);
-    uint32_t pk[64];
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
       float s[32], dp[32];
       tmem_ld32(tS + 32 * c, s);
       tmem_ld32(tP + 32 * c, dp);
       tmem_wait_ld();
+      uint32_t pk[16];
 #pragma unroll
       for (int e = 0; e < 32; e += 2) {
         const int j = 32 * c + e;
@@ -344,16 +353,13 @@ __device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned cha
         const bool ok1 = !((diag && j + 1 > r) || (bound && j + 1 < r));
         const float d0 = ok0 ? p0 * (dp[e] - Dr) * a.scale : 0.f;
         const float d1 = ok1 ? p1 * (dp[e + 1] - Dr) * a.scale : 0.f;
-        pk[16 * c + (e >> 1)] = pack_bf16(d0, d1);
+        pk[e >> 1] = pack_bf16(d0, d1);
       }
+      // dS (bf16, two per column) overwrites the S columns already consumed: 16c..16c+15 < 32c+32
+      tmem_st16(tS + 16 * c, pk);
     }
+    tmem_wait_st();
     tc_fence_before();
-    mbar_arrive(&bars->s_empty);
-    if (i > 0) WAIT_OR_RETURN(bars->dq_done, (i - 1) & 1);   // the previous dS has been consumed
-#pragma unroll
-    for (int c = 0; c < 16; ++c)
-      *reinterpret_cast<uint4*>(sD + swz(r, c)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-    fence_proxy_async_smem();
     mbar_arrive(&bars->ds_full);
   }
 
@@ -365,22 +371,20 @@ __device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned cha
     mbar_arrive(&bars->phik_ready);
     WAIT_OR_RETURN(bars->s_full, n_kt & 1);
     tc_fence_after();
-    uint32_t pk[64];
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
       float x[32];
       tmem_ld32(tS + 32 * c, x);
       tmem_wait_ld();
+      uint32_t pk[16];
 #pragma unroll
       for (int e = 0; e < 32; e += 2) {
         const int j = 32 * c + e;                            // residual keys of row r in this chunk: j < r
-        pk[16 * c + (e >> 1)] = pack_bf16(j < r ? x[e] : 0.f, j + 1 < r ? x[e + 1] : 0.f);
+        pk[e >> 1] = pack_bf16(j < r ? x[e] : 0.f, j + 1 < r ? x[e + 1] : 0.f);
       }
+      tmem_st16(tS + 16 * c, pk);
     }
-#pragma unroll
-    for (int c = 0; c < 16; ++c)
-      *reinterpret_cast<uint4*>(sD + swz(r, c)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-    fence_proxy_async_smem();
+    tmem_wait_st();
     tc_fence_before();
     mbar_arrive(&bars->ds_full);
   }
@@ -548,173 +552,175 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 }
 
 // =============================================================================== dkv
+// One CTA per (key tile j, K/V head).  K_j, V_j (and phi(K_j)) stay in shared memory, the dV
+// and dK accumulators in TMEM.  The work is a list of items, one per (query head of the
+// group, query half tile of 64 rows): first the residual-branch items (query tile j + wt),
+// then the window items (query tiles j .. j + wt).  Two row groups of 128 threads (thread =
+// key row = TMEM lane) take the items alternately, each with its own TMEM slot, so that one
+// group's exponentials overlap the other group's products:
+//   loader thread   TMA: K, V, [R_j], then per item Q_h, g_h and the query-side row statistics
+//   MMA thread      per item: S^T = K Q_h^T and dP^T = V g_h^T into the slot (128 x 64 each);
+//                   after the row group has overwritten them with bf16 P^T and dS^T:
+//                   dV += P^T g_h, dK += dS^T Q_h with the A operand read from TMEM
+//   row group       P^T = exp2(S^T * scale_log2 - lse2[q]), dS^T = P^T (dP^T scale - D[q] scale)
+// The residual items run first and leave dphi_k in the dK accumulator; row group 0 then folds
+// the feature-map Jacobian into it (dK := phi(k) (dphi_k - <dphi_k, phi(k)>)) and the window
+// items accumulate on top.
+constexpr int KV_NS = 4;                                   // item stages
 constexpr int KV_OFF_K = 0;
 constexpr int KV_OFF_V = 1 * TILE_BYTES;
-constexpr int KV_OFF_Q = 2 * TILE_BYTES;   // 2 stages
-constexpr int KV_OFF_G = 4 * TILE_BYTES;   // 2 stages
-constexpr int KV_OFF_D = 6 * TILE_BYTES;
-constexpr int KV_OFF_STAT = 7 * TILE_BYTES;            // 2 stages x (lse2[128], D*scale[128]) fp32
-constexpr int KV_OFF_BAR = KV_OFF_STAT + 2 * 2 * 128 * 4;
+constexpr int KV_OFF_KPHI = 2 * TILE_BYTES;
+constexpr int KV_OFF_STAGE = 3 * TILE_BYTES;               // KV_NS x [Q_h 16 KB | g_h 16 KB]
+constexpr int KV_OFF_STAT = KV_OFF_STAGE + KV_NS * TILE_BYTES;   // KV_NS x (lse2[64], D*scale[64]) fp32
+constexpr int KV_OFF_BAR = KV_OFF_STAT + KV_NS * 512;
 constexpr int KV_SMEM = KV_OFF_BAR + 256;
+constexpr int KV_THREADS = 320;                            // 2 row groups, MMA warp, loader warp
 
 struct KvBars {
-  uint64_t kv_full, k2_full, r_full, kphi_ready, inter_done, qg_full[2], phi_ready, s_full, s_empty,
-      d1_full, acc1_done, d2_full, acc2_done, xform_done, drain;
+  uint64_t kv_full, kphi_ready, full[KV_NS], acc_done[KV_NS], s_full[2], p_ready[2], phiq_ready[2],
+      r_acc_done, fold_done, all_done, drain;
   uint32_t tmem_base;
   int abort;
 };
 
-// The work of one CTA is a list of items, each one (query head of the group, query tile):
-// first the residual-branch items (one per head, query tile j + wt), then the window items.
 struct KvPlan {
-  int j, n_qt, wt, group, n_r, n_s_tiles, N;
+  int j, n_qt, wt, group, n_R, n_s_tiles, N, off;
   bool windowed, has_inter;
-  __device__ bool is_r(int n) const { return n < n_r; }
-  __device__ int head(int n) const { return n < n_r ? n : (n - n_r) / n_s_tiles; }
-  __device__ int qtile(int n) const { return n < n_r ? j + wt : j + (n - n_r) % n_s_tiles; }
+  __device__ bool is_r(int n) const { return n < n_R; }
+  __device__ int head(int n) const { return n < n_R ? (n >> 1) : (n - n_R) / (2 * n_s_tiles); }
+  __device__ int qtile(int n) const { return n < n_R ? j + wt : j + (((n - n_R) % (2 * n_s_tiles)) >> 1); }
+  __device__ int half(int n) const { return n < n_R ? (n & 1) : ((n - n_R) & 1); }
+  __device__ int stage(int n) const { return (n + off) % KV_NS; }
+  __device__ int use(int n) const { return (n + off) / KV_NS; }
 };
 
-__device__ bool kv_control(const CUtensorMap* tm_q, const CUtensorMap* tm_k, const CUtensorMap* tm_v,
-                           const CUtensorMap* tm_gs, const CUtensorMap* tm_gr, const CUtensorMap* tm_rs,
-                           unsigned char* smem, KvBars* bars, uint32_t tmem, const KvPlan& pl, int bh_kv,
-                           int rs_index) {
-  const uint32_t sK = smem_u32(smem + KV_OFF_K), sV = smem_u32(smem + KV_OFF_V);
-  const uint32_t sQ = smem_u32(smem + KV_OFF_Q), sG = smem_u32(smem + KV_OFF_G), sD = smem_u32(smem + KV_OFF_D);
-  const uint32_t tS = tmem, tP = tmem + 128, tV = tmem + 256, tK = tmem + 384;
+__device__ bool kv_loader(const CUtensorMap* tm_k, const CUtensorMap* tm_v, const CUtensorMap* tm_rs,
+                          const CUtensorMap* tm_qh, const CUtensorMap* tm_gsh, const CUtensorMap* tm_grh,
+                          const float* lse2p, const float* dscp, int t_pad, unsigned char* smem, KvBars* bars,
+                          const KvPlan& pl, int bh_kv, int rs_index) {
   const int j0 = pl.j * TILE;
-
-  auto load_item = [&](int n) {
-    const int st = n & 1;
-    const int z = bh_kv * pl.group + pl.head(n);
-    const int row = pl.qtile(n) * TILE;
-    mbar_arrive_expect_tx(&bars->qg_full[st], 2 * TILE_BYTES);
-    load_tile(smem + KV_OFF_Q + st * TILE_BYTES, tm_q, &bars->qg_full[st], row, z);
-    load_tile(smem + KV_OFF_G + st * TILE_BYTES, pl.is_r(n) ? tm_gr : tm_gs, &bars->qg_full[st], row, z);
-  };
-
   mbar_arrive_expect_tx(&bars->kv_full, 2 * TILE_BYTES);
   load_tile(smem + KV_OFF_K, tm_k, &bars->kv_full, j0, bh_kv);
   load_tile(smem + KV_OFF_V, tm_v, &bars->kv_full, j0, bh_kv);
   if (pl.has_inter) {
-    mbar_arrive_expect_tx(&bars->r_full, TILE_BYTES);
-    load_tile(smem + KV_OFF_D, tm_rs, &bars->r_full, 0, rs_index);
+    mbar_arrive_expect_tx(&bars->full[0], TILE_BYTES);
+    load_tile(smem + KV_OFF_STAGE, tm_rs, &bars->full[0], 0, rs_index);
   }
-  load_item(0);
-  if (pl.N > 1) load_item(1);
-
-  bool accV = false, accK = false;
-  if (pl.n_r > 0) {
-    WAIT_OR_RETURN(bars->kphi_ready, 0);                   // phi(K_j) is in place (implies K, V landed)
-    if (pl.has_inter) {
-      WAIT_OR_RETURN(bars->r_full, 0);
-      tc_fence_after();
-      mma_kk(tK, sV, sD, false);                           // dphi_k  = V_j R_j^T
-      mma_kmn<1>(tV, sK, sD, false);                       // dV      = phi(K_j) R_j
-      mma_commit(&bars->inter_done);
-      accV = accK = true;
-    }
-  } else {
-    WAIT_OR_RETURN(bars->kv_full, 0);
-  }
-
-  auto issue_scores = [&](int n) -> bool {
-    const int st = n & 1;
-    if (n == pl.n_r && pl.n_r > 0) {
-      // residual phase over: phi(K_j) has been consumed and folded; fetch K_j again for the window phase
-      WAIT_OR_RETURN(bars->xform_done, 0);
-      mbar_arrive_expect_tx(&bars->k2_full, TILE_BYTES);
-      load_tile(smem + KV_OFF_K, tm_k, &bars->k2_full, j0, bh_kv);
-      WAIT_OR_RETURN(bars->k2_full, 0);
-    }
-    WAIT_OR_RETURN(bars->qg_full[st], (n >> 1) & 1);
-    if (pl.is_r(n)) WAIT_OR_RETURN(bars->phi_ready, n & 1);
-    if (n > 0) WAIT_OR_RETURN(bars->s_empty, (n - 1) & 1);
-    tc_fence_after();
-    mma_kk(tS, sK, sQ + st * TILE_BYTES, false);           // S^T  = K Q^T      (or phi(K) phi(Q)^T)
-    mma_kk(tP, sV, sG + st * TILE_BYTES, false);           // dP^T = V g^T
-    mma_commit(&bars->s_full);
-    return true;
-  };
-
-  int issued = -1;
   for (int n = 0; n < pl.N; ++n) {
-    const int st = n & 1;
-    if (issued < n) {
-      if (!issue_scores(n)) return false;
-      issued = n;
+    const int st = pl.stage(n), u = pl.use(n);
+    if (u >= 1) WAIT_OR_RETURN(bars->acc_done[st], (u - 1) & 1);
+    unsigned char* dst = smem + KV_OFF_STAGE + st * TILE_BYTES;
+    const int z = bh_kv * pl.group + pl.head(n);
+    const int row = pl.qtile(n) * TILE + 64 * pl.half(n);
+    if (pl.is_r(n)) {
+      mbar_arrive_expect_tx(&bars->full[st], 2 * HT_BYTES);
+      load_half_tile(dst, tm_qh, &bars->full[st], row, z);
+      load_half_tile(dst + HT_BYTES, tm_grh, &bars->full[st], row, z);
+    } else {
+      mbar_arrive_expect_tx(&bars->full[st], 2 * HT_BYTES + 512);
+      load_half_tile(dst, tm_qh, &bars->full[st], row, z);
+      load_half_tile(dst + HT_BYTES, tm_gsh, &bars->full[st], row, z);
+      float* stat = reinterpret_cast<float*>(smem + KV_OFF_STAT + st * 512);
+      bulk_load_1d(stat, lse2p + (size_t)z * t_pad + row, 256, &bars->full[st]);
+      bulk_load_1d(stat + 64, dscp + (size_t)z * t_pad + row, 256, &bars->full[st]);
     }
-    // run ahead: the next item's scores, unless it needs this item's results first
-    if (n + 1 < pl.N && !pl.is_r(n + 1) && !(n + 1 == pl.n_r && pl.n_r > 0)) {
-      if (!issue_scores(n + 1)) return false;
-      issued = n + 1;
-    }
-    WAIT_OR_RETURN(bars->d1_full, n & 1);
-    tc_fence_after();
-    mma_kmn<1>(tV, sD, sG + st * TILE_BYTES, accV);        // dV += P^T g_s      (or A^T g_r)
-    mma_commit(&bars->acc1_done);
-    accV = true;
-    WAIT_OR_RETURN(bars->d2_full, n & 1);
-    tc_fence_after();
-    mma_kmn<1>(tK, sD, sQ + st * TILE_BYTES, accK);        // dK += dS^T Q       (or dphi_k += dA^T phi(Q))
-    mma_commit(&bars->acc2_done);
-    accK = true;
-    WAIT_OR_RETURN(bars->acc2_done, n & 1);                // stage st is free again
-    if (n + 2 < pl.N) load_item(n + 2);
   }
   return true;
 }
 
-__device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtensorMap* tm_dv, unsigned char* smem, KvBars* bars, uint32_t tmem, const KvPlan& pl,
-                        int r, int bh_kv) {
-  const uint32_t lane_off = (uint32_t)((r & ~31) << 16);
-  const uint32_t tS = tmem + lane_off, tP = tmem + 128 + lane_off, tV = tmem + 256 + lane_off,
-                 tK = tmem + 384 + lane_off;
-  unsigned char* sD = smem + KV_OFF_D;
-  unsigned char* sK = smem + KV_OFF_K;
-  float* stat = reinterpret_cast<float*>(smem + KV_OFF_STAT);
+__device__ bool kv_mma(unsigned char* smem, KvBars* bars, uint32_t tmem, const KvPlan& pl) {
+  const uint32_t sK = smem_u32(smem + KV_OFF_K), sV = smem_u32(smem + KV_OFF_V), sKphi = smem_u32(smem + KV_OFF_KPHI);
+  const uint32_t sStage = smem_u32(smem + KV_OFF_STAGE);
+  const uint32_t tV = tmem, tK = tmem + 128;
+  const uint32_t tS[2] = {tmem + 256, tmem + 384}, tP[2] = {tmem + 320, tmem + 448};
+  bool accV = false, accK = false;
 
   WAIT_OR_RETURN(bars->kv_full, 0);
-  if (pl.n_r > 0) {
-    feature_map_row_inplace(sK, r);
+  if (pl.n_R > 0) WAIT_OR_RETURN(bars->kphi_ready, 0);
+  if (pl.has_inter) {
+    WAIT_OR_RETURN(bars->full[0], 0);
+    tc_fence_after();
+    mma_kk(tK, sV, sStage, false);                         // dphi_k = V_j R_j^T
+    mma_kmn<1>(tV, sKphi, sStage, false);                  // dV     = phi(K_j) R_j
+    mma_commit(&bars->acc_done[0]);
+    accV = accK = true;
+  }
+  for (int n = 0; n <= pl.N; ++n) {
+    if (n < pl.N) {
+      const int st = pl.stage(n), slot = n & 1;
+      const uint32_t sQh = sStage + st * TILE_BYTES, sGh = sQh + HT_BYTES;
+      WAIT_OR_RETURN(bars->full[st], pl.use(n) & 1);
+      if (pl.is_r(n)) WAIT_OR_RETURN(bars->phiq_ready[slot], (n >> 1) & 1);
+      if (n >= 2) WAIT_OR_RETURN(bars->acc_done[pl.stage(n - 2)], pl.use(n - 2) & 1);   // the slot is free
+      tc_fence_after();
+      mma_k_kh(tS[slot], pl.is_r(n) ? sKphi : sK, sQh);   // S^T  = K Q_h^T   (phi(K) phi(Q_h)^T)
+      mma_k_kh(tP[slot], sV, sGh);                         // dP^T = V g_h^T
+      mma_commit(&bars->s_full[slot]);
+    }
+    if (n >= 1) {
+      const int m = n - 1, st = pl.stage(m), slot = m & 1;
+      const uint32_t sQh = sStage + st * TILE_BYTES, sGh = sQh + HT_BYTES;
+      WAIT_OR_RETURN(bars->p_ready[slot], (m >> 1) & 1);
+      if (m == pl.n_R && pl.n_R > 0) WAIT_OR_RETURN(bars->fold_done, 0);
+      tc_fence_after();
+      mma_ts_h(tV, tS[slot], sGh, accV);                   // dV += P^T g_h
+      mma_ts_h(tK, tP[slot], sQh, accK);                   // dK += dS^T Q_h   (dphi_k += dA^T phi(Q_h))
+      accV = accK = true;
+      mma_commit(&bars->acc_done[st]);
+      if (m == pl.n_R - 1) mma_commit(&bars->r_acc_done);
+    }
+  }
+  mma_commit(&bars->all_done);
+  return true;
+}
+
+__device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtensorMap* tm_dv, unsigned char* smem,
+                        KvBars* bars, uint32_t tmem, const KvPlan& pl, int g, int r, int bh_kv) {
+  const uint32_t lane_off = (uint32_t)((r & ~31) << 16);
+  const uint32_t tV = tmem + lane_off, tK = tmem + 128 + lane_off;
+  const uint32_t tS = tmem + 256 + 128 * g + lane_off, tP = tS + 64;
+  const unsigned char* sKphi = smem + KV_OFF_KPHI;
+
+  WAIT_OR_RETURN(bars->kv_full, 0);
+  if (pl.n_R > 0) {
+    // phi(K_j) into its own tile: 256 threads, two per row
+    const int t2 = g * 128 + r, row = t2 >> 1, hf = t2 & 1;
+    feature_map_pair(smem + KV_OFF_K + hf * HALF_BYTES, smem + KV_OFF_KPHI + hf * HALF_BYTES, row);
     fence_proxy_async_smem();
     mbar_arrive(&bars->kphi_ready);
   }
 
-  for (int n = 0; n < pl.N; ++n) {
-    const int st = n & 1;
+  for (int n = g; n < pl.N; n += 2) {
+    const int st = pl.stage(n);
     const bool is_r = pl.is_r(n);
-    const int i = pl.qtile(n);
+    const int i = pl.qtile(n), hf = pl.half(n);
+    unsigned char* sQh = smem + KV_OFF_STAGE + st * TILE_BYTES;
+    WAIT_OR_RETURN(bars->full[st], pl.use(n) & 1);
     if (is_r) {
-      WAIT_OR_RETURN(bars->qg_full[st], (n >> 1) & 1);
-      feature_map_row_inplace(smem + KV_OFF_Q + st * TILE_BYTES, r);
+      // phi(Q_h) in place: 64 rows, two threads per row
+      const int row = r >> 1, ch = r & 1;
+      feature_map_pair(sQh + ch * HT_HALF, sQh + ch * HT_HALF, row);
       fence_proxy_async_smem();
-      mbar_arrive(&bars->phi_ready);
-    } else {
-      const int bq = bh_kv * a.group + pl.head(n);        // (batch, query head) index of this item
-      const int t = i * TILE + r;
-      const size_t row = (size_t)bq * a.T + t;
-      stat[st * 256 + r] = t < a.T ? a.lse[row] * LOG2E : INFINITY;
-      stat[st * 256 + 128 + r] = t < a.T ? a.delta[row] * a.scale : 0.f;
-      rows_sync();
+      mbar_arrive(&bars->phiq_ready[g]);
     }
-    WAIT_OR_RETURN(bars->s_full, n & 1);
+    WAIT_OR_RETURN(bars->s_full[g], (n >> 1) & 1);
     tc_fence_after();
     const bool diag = !is_r && (i == pl.j), bound = !is_r && pl.windowed && (i == pl.j + pl.wt);
-    const float* l2 = stat + st * 256;
-    const float* Ds = l2 + 128;
-    uint32_t pk1[64], pk2[64];
+    const float* l2 = reinterpret_cast<const float*>(smem + KV_OFF_STAT + st * 512);
+    const float* Ds = l2 + 64;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
+    for (int c = 0; c < 2; ++c) {
       float s[32], dp[32];
       tmem_ld32(tS + 32 * c, s);
       tmem_ld32(tP + 32 * c, dp);
       tmem_wait_ld();
+      uint32_t pk1[16], pk2[16];
       if (is_r) {
 #pragma unroll
         for (int e = 0; e < 32; e += 2) {
-          const int q = 32 * c + e;                          // query column; keep key r < query q
-          pk1[16 * c + (e >> 1)] = pack_bf16(q > r ? s[e] : 0.f, q + 1 > r ? s[e + 1] : 0.f);
-          pk2[16 * c + (e >> 1)] = pack_bf16(q > r ? dp[e] : 0.f, q + 1 > r ? dp[e + 1] : 0.f);
+          const int q = 64 * hf + 32 * c + e;              // query row inside its tile; keep key r < query q
+          pk1[e >> 1] = pack_bf16(q > r ? s[e] : 0.f, q + 1 > r ? s[e + 1] : 0.f);
+          pk2[e >> 1] = pack_bf16(q > r ? dp[e] : 0.f, q + 1 > r ? dp[e + 1] : 0.f);
         }
       } else {
 #pragma unroll
@@ -725,40 +731,29 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
           float p[4], d[4];
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
-            const int q = 32 * c + e4 + u;
+            const int q = 64 * hf + 32 * c + e4 + u;
             const bool ok = !((diag && q < r) || (bound && q > r));
             const float pv = ex2(s[e4 + u] * a.scale_log2 - lq[u]);
             p[u] = ok ? pv : 0.f;
             d[u] = ok ? pv * (dp[e4 + u] * a.scale - dq4[u]) : 0.f;
           }
-          pk1[16 * c + (e4 >> 1)] = pack_bf16(p[0], p[1]);
-          pk1[16 * c + (e4 >> 1) + 1] = pack_bf16(p[2], p[3]);
-          pk2[16 * c + (e4 >> 1)] = pack_bf16(d[0], d[1]);
-          pk2[16 * c + (e4 >> 1) + 1] = pack_bf16(d[2], d[3]);
+          pk1[e4 >> 1] = pack_bf16(p[0], p[1]);
+          pk1[(e4 >> 1) + 1] = pack_bf16(p[2], p[3]);
+          pk2[e4 >> 1] = pack_bf16(d[0], d[1]);
+          pk2[(e4 >> 1) + 1] = pack_bf16(d[2], d[3]);
         }
       }
+      // bf16 results (two per column) overwrite columns of S^T / dP^T that have been consumed
+      tmem_st16(tS + 16 * c, pk1);
+      tmem_st16(tP + 16 * c, pk2);
     }
+    tmem_wait_st();
     tc_fence_before();
-    mbar_arrive(&bars->s_empty);
-    // the staging tile is free once the previous product that read it has completed
-    if (n > 0) WAIT_OR_RETURN(bars->acc2_done, (n - 1) & 1);
-    else if (pl.has_inter) WAIT_OR_RETURN(bars->inter_done, 0);
-#pragma unroll
-    for (int c = 0; c < 16; ++c)
-      *reinterpret_cast<uint4*>(sD + swz(r, c)) = make_uint4(pk1[4 * c], pk1[4 * c + 1], pk1[4 * c + 2], pk1[4 * c + 3]);
-    fence_proxy_async_smem();
-    mbar_arrive(&bars->d1_full);
-    WAIT_OR_RETURN(bars->acc1_done, n & 1);
-#pragma unroll
-    for (int c = 0; c < 16; ++c)
-      *reinterpret_cast<uint4*>(sD + swz(r, c)) = make_uint4(pk2[4 * c], pk2[4 * c + 1], pk2[4 * c + 2], pk2[4 * c + 3]);
-    fence_proxy_async_smem();
-    mbar_arrive(&bars->d2_full);
+    mbar_arrive(&bars->p_ready[g]);
 
-    if (n == pl.n_r - 1) {
-      // end of the residual phase: fold the feature-map Jacobian into the dK accumulator,
-      // dK := phi(k) * (dphi_k - <dphi_k, phi(k)>), so that the window phase accumulates on top
-      WAIT_OR_RETURN(bars->acc2_done, n & 1);
+    if (g == 0 && pl.n_R > 0 && n == pl.n_R - 2) {
+      // end of the residual items: dK := phi(k) (dphi_k - <dphi_k, phi(k)>)
+      WAIT_OR_RETURN(bars->r_acc_done, 0);
       tc_fence_after();
       float dot = 0.f;
 #pragma unroll 1
@@ -768,7 +763,7 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
         tmem_wait_ld();
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) {
-          const uint4 u = *reinterpret_cast<const uint4*>(sK + swz(r, 4 * c + cc));
+          const uint4 u = *reinterpret_cast<const uint4*>(sKphi + swz(r, 4 * c + cc));
           const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
@@ -784,7 +779,7 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
         tmem_wait_ld();
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) {
-          const uint4 u = *reinterpret_cast<const uint4*>(sK + swz(r, 4 * c + cc));
+          const uint4 u = *reinterpret_cast<const uint4*>(sKphi + swz(r, 4 * c + cc));
           const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
@@ -796,42 +791,36 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
         tmem_st32(tK + 32 * c, df);
       }
       tmem_wait_st();
-      fence_proxy_async_smem();
       tc_fence_before();
-      mbar_arrive(&bars->xform_done);
+      mbar_arrive(&bars->fold_done);
     }
   }
 
-  WAIT_OR_RETURN(bars->acc2_done, (pl.N - 1) & 1);
+  // every product has completed: row group 0 stores dK, row group 1 dV, each staged in one of
+  // the (now free) item stages and written by one TMA store
+  WAIT_OR_RETURN(bars->all_done, 0);
   tc_fence_after();
-  // every product has completed: dK is staged in the dS tile, dV in the first query stage
-  unsigned char* sOutV = smem + KV_OFF_Q;
+  unsigned char* sOut = smem + KV_OFF_STAGE + g * TILE_BYTES;
+  const uint32_t tOut = g == 0 ? tK : tV;
 #pragma unroll 1
   for (int c = 0; c < 4; ++c) {
-    float xk[32], xv[32];
-    tmem_ld32(tK + 32 * c, xk);
-    tmem_ld32(tV + 32 * c, xv);
+    float x[32];
+    tmem_ld32(tOut + 32 * c, x);
     tmem_wait_ld();
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       uint4 u;
-      u.x = pack_bf16(xk[8 * e + 0], xk[8 * e + 1]);
-      u.y = pack_bf16(xk[8 * e + 2], xk[8 * e + 3]);
-      u.z = pack_bf16(xk[8 * e + 4], xk[8 * e + 5]);
-      u.w = pack_bf16(xk[8 * e + 6], xk[8 * e + 7]);
-      *reinterpret_cast<uint4*>(sD + swz(r, 4 * c + e)) = u;
-      u.x = pack_bf16(xv[8 * e + 0], xv[8 * e + 1]);
-      u.y = pack_bf16(xv[8 * e + 2], xv[8 * e + 3]);
-      u.z = pack_bf16(xv[8 * e + 4], xv[8 * e + 5]);
-      u.w = pack_bf16(xv[8 * e + 6], xv[8 * e + 7]);
-      *reinterpret_cast<uint4*>(sOutV + swz(r, 4 * c + e)) = u;
+      u.x = pack_bf16(x[8 * e + 0], x[8 * e + 1]);
+      u.y = pack_bf16(x[8 * e + 2], x[8 * e + 3]);
+      u.z = pack_bf16(x[8 * e + 4], x[8 * e + 5]);
+      u.w = pack_bf16(x[8 * e + 6], x[8 * e + 7]);
+      *reinterpret_cast<uint4*>(sOut + swz(r, 4 * c + e)) = u;
     }
   }
   fence_proxy_async_smem();
-  rows_sync();
+  group_sync(g);
   if (r == 0) {
-    store_tile(tm_dk, sD, pl.j * TILE, bh_kv);
-    store_tile(tm_dv, sOutV, pl.j * TILE, bh_kv);
+    store_tile(g == 0 ? tm_dk : tm_dv, sOut, pl.j * TILE, bh_kv);
     tma_store_commit();
     tma_store_wait_read();
   }
@@ -839,11 +828,12 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
   return true;
 }
 
-__global__ void __launch_bounds__(160, 1)
-tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_gs,
-                  const __grid_constant__ CUtensorMap tm_gr, const __grid_constant__ CUtensorMap tm_rs,
-                  const __grid_constant__ CUtensorMap tm_dk, const __grid_constant__ CUtensorMap tm_dv, BwdArgs a) {
+struct KvMaps {
+  CUtensorMap k, v, rs, qh, gsh, grh, dk, dv;
+};
+
+__global__ void __launch_bounds__(KV_THREADS, 1)
+tc_bwd_dkv_kernel(const __grid_constant__ KvMaps tm, BwdArgs a) {
   extern __shared__ __align__(1024) unsigned char smem[];
   KvBars* bars = reinterpret_cast<KvBars*>(smem + KV_OFF_BAR);
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -860,45 +850,43 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   const int i_hi = (pl.windowed && pl.j + pl.wt < pl.n_qt - 1) ? pl.j + pl.wt : pl.n_qt - 1;
   pl.n_s_tiles = i_hi - pl.j + 1;
   const bool r_tile = pl.windowed && (a.mode == RATTN_MODE_RATTN) && (pl.j + pl.wt <= pl.n_qt - 1);
-  pl.n_r = r_tile ? a.group : 0;
+  pl.n_R = r_tile ? 2 * a.group : 0;
   pl.has_inter = r_tile && (pl.j + pl.wt + 1 <= pl.n_qt - 1);
-  pl.N = pl.n_r + a.group * pl.n_s_tiles;
+  pl.off = pl.has_inter ? 1 : 0;
+  pl.N = pl.n_R + 2 * a.group * pl.n_s_tiles;
   const int bh_kv = blockIdx.y;
   const int rs_index = bh_kv * a.n_chunks + pl.j;
 
   if (tid == 0) {
     mbar_init(&bars->kv_full, 1);
-    mbar_init(&bars->k2_full, 1);
-    mbar_init(&bars->r_full, 1);
-    mbar_init(&bars->kphi_ready, 128);
-    mbar_init(&bars->inter_done, 1);
-    mbar_init(&bars->qg_full[0], 1);
-    mbar_init(&bars->qg_full[1], 1);
-    mbar_init(&bars->phi_ready, 128);
-    mbar_init(&bars->s_full, 1);
-    mbar_init(&bars->s_empty, 128);
-    mbar_init(&bars->d1_full, 128);
-    mbar_init(&bars->acc1_done, 1);
-    mbar_init(&bars->d2_full, 128);
-    mbar_init(&bars->acc2_done, 1);
-    mbar_init(&bars->xform_done, 128);
+    mbar_init(&bars->kphi_ready, 256);
+    for (int i = 0; i < KV_NS; ++i) {
+      mbar_init(&bars->full[i], 1);
+      mbar_init(&bars->acc_done[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bars->s_full[i], 1);
+      mbar_init(&bars->p_ready[i], 128);
+      mbar_init(&bars->phiq_ready[i], 128);
+    }
+    mbar_init(&bars->r_acc_done, 1);
+    mbar_init(&bars->fold_done, 128);
+    mbar_init(&bars->all_done, 1);
     mbar_init(&bars->drain, 1);
     bars->abort = 0;
     fence_mbar_init();
   }
-  if (warp == 4) {
+  if (warp == 8) {
     tmem_alloc(&bars->tmem_base, 512);
     tmem_relinquish();
-    if (tid == 128) {
-      prefetch_tensormap(&tm_q);
-      prefetch_tensormap(&tm_k);
-      prefetch_tensormap(&tm_v);
-      prefetch_tensormap(&tm_gs);
-      prefetch_tensormap(&tm_gr);
-      prefetch_tensormap(&tm_rs);
-      prefetch_tensormap(&tm_dk);
-      prefetch_tensormap(&tm_dv);
-    }
+  }
+  if (tid == 288) {
+    prefetch_tensormap(&tm.k);
+    prefetch_tensormap(&tm.v);
+    prefetch_tensormap(&tm.rs);
+    prefetch_tensormap(&tm.qh);
+    prefetch_tensormap(&tm.gsh);
+    prefetch_tensormap(&tm.grh);
   }
   tc_fence_before();
   __syncthreads();
@@ -906,19 +894,22 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   const uint32_t tmem = bars->tmem_base;
 
   bool ok = true;
-  if (warp < 4) {
-    ok = kv_rows(a, &tm_dk, &tm_dv, smem, bars, tmem, pl, tid, bh_kv);
-  } else if (tid == 128) {
-    ok = kv_control(&tm_q, &tm_k, &tm_v, &tm_gs, &tm_gr, &tm_rs, smem, bars, tmem, pl, bh_kv, rs_index);
+  if (warp < 8) {
+    ok = kv_rows(a, &tm.dk, &tm.dv, smem, bars, tmem, pl, warp >> 2, tid & 127, bh_kv);
+  } else if (tid == 256) {
+    ok = kv_mma(smem, bars, tmem, pl);
     if (!ok) {
       mma_commit(&bars->drain);
       for (int it = 0; it < (1 << 16) && !mbar_try_wait(&bars->drain, 0); ++it) {}
     }
+  } else if (tid == 288) {
+    ok = kv_loader(&tm.k, &tm.v, &tm.rs, &tm.qh, &tm.gsh, &tm.grh, a.lse2p, a.dscp, a.t_pad, smem, bars, pl,
+                   bh_kv, rs_index);
   }
   if (!ok && a.status) atomicExch(a.status, 1);
   tc_fence_before();
   __syncthreads();
-  if (warp == 4) {
+  if (warp == 8) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
   }
@@ -927,7 +918,6 @@ tc_bwd_dkv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 }  // namespace
 
 cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
-  const size_t n_rows = (size_t)a.B * a.H_q * a.T;
   __nv_bfloat16* g_s = reinterpret_cast<__nv_bfloat16*>(a.do_swa);
   __nv_bfloat16* g_r = reinterpret_cast<__nv_bfloat16*>(a.do_rla);
   const bool rla_on = (a.mode == RATTN_MODE_RATTN);
@@ -942,11 +932,14 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
     e = cudaMemsetAsync(a.dgamma_rla, 0, sizeof(float) * a.H_q * 128, s);
     if (e != cudaSuccess) return e;
   }
+  const int t_pad = a.n_chunks * TILE;
+  const size_t n_rows_pad = (size_t)a.B * a.H_q * t_pad;
   {
     KernelTimer kt("tc_bwd_prep", s);
-    tc_bwd_prep_kernel<<<(unsigned)((n_rows + 63) / 64), 256, 0, s>>>(
+    tc_bwd_prep_kernel<<<(unsigned)((n_rows_pad + 63) / 64), 256, 0, s>>>(
         reinterpret_cast<const __nv_bfloat16*>(a.dout), a.o_swa, a.o_rla, a.gamma_swa, a.gamma_rla, g_s, g_r,
-        a.delta, a.dgamma_swa, a.dgamma_rla, n_rows, a.T, a.H_q, a.eps, rla_on ? 1 : 0);
+        a.delta, a.dgamma_swa, a.dgamma_rla, a.lse, a.lse2p, a.dscp, n_rows_pad, a.T, t_pad, a.H_q, a.eps, a.scale,
+        rla_on ? 1 : 0);
   }
   count_launches(1);
 
@@ -980,6 +973,7 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
   t.dk = reinterpret_cast<__nv_bfloat16*>(a.dk);
   t.dv = reinterpret_cast<__nv_bfloat16*>(a.dv);
   t.lse = a.lse; t.delta = a.delta; t.status = a.status;
+  t.lse2p = a.lse2p; t.dscp = a.dscp; t.t_pad = t_pad;
   t.T = a.T; t.w = a.w; t.H_q = a.H_q; t.group = a.group; t.mode = a.mode; t.n_chunks = a.n_chunks;
   t.scale = a.scale; t.scale_log2 = a.scale * LOG2E;
   e = cudaFuncSetAttribute(tc_bwd_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DQ_SMEM);
@@ -990,9 +984,13 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
     KernelTimer kt("tc_bwd_dq", s);
     tc_bwd_dq_kernel<<<dim3(n_qt, (unsigned)nq), 160, DQ_SMEM, s>>>(tm_q, tm_k, tm_v, tm_gs, tm_gr, tm_st, tm_dq, t);
   }
+  KvMaps km;
+  km.k = tm_k; km.v = tm_v; km.rs = tm_rs; km.dk = tm_dk; km.dv = tm_dv;
+  if (!make_map(&km.qh, a.q, a.T, nq, 64) || !make_map(&km.gsh, g_s, a.T, nq, 64) || !make_map(&km.grh, g_r, a.T, nq, 64))
+    return cudaErrorInvalidValue;
   {
     KernelTimer kt("tc_bwd_dkv", s);
-    tc_bwd_dkv_kernel<<<dim3(n_qt, (unsigned)nkv), 160, KV_SMEM, s>>>(tm_q, tm_k, tm_v, tm_gs, tm_gr, tm_rs, tm_dk, tm_dv, t);
+    tc_bwd_dkv_kernel<<<dim3(n_qt, (unsigned)nkv), KV_THREADS, KV_SMEM, s>>>(km, t);
   }
   count_launches(2);
   return cudaGetLastError();

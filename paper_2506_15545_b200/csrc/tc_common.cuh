@@ -44,6 +44,78 @@ __device__ __forceinline__ void mma_mnmn(uint32_t d, uint32_t a_base, uint32_t b
   for (int k = 0; k < 8; ++k) mma_bf16(d, mnmajor_desc(a_base, k), mnmajor_desc(b_base, k), idesc, (acc || k > 0) ? 1u : 0u);
 }
 
+// ---- half tiles: [64 rows x 128 columns] bf16 as two [64 x 64] boxes of 8 KB ------------
+constexpr int HT_HALF = 64 * 64 * 2;
+constexpr int HT_BYTES = 2 * HT_HALF;
+// B operand, K-major: the half tile's 64 rows are N, its 128 columns the reduction (8 steps)
+__device__ __forceinline__ uint64_t kmajor_desc_h(uint32_t base, int kstep) {
+  return smem_desc(base + (kstep >> 2) * HT_HALF + (kstep & 3) * 32, 16, 1024);
+}
+// B operand, MN-major: the half tile's 128 columns are N, its 64 rows the reduction (4 steps)
+__device__ __forceinline__ uint64_t mnmajor_desc_h(uint32_t base, int kstep) {
+  return smem_desc(base + kstep * 2048, HT_HALF, 1024);
+}
+// D[128 x 64] = A[128 x 128] (K-major full tile) . B[64 x 128]^T (K-major half tile)
+__device__ __forceinline__ void mma_k_kh(uint32_t d, uint32_t a_base, uint32_t b_base) {
+  constexpr uint32_t idesc = instr_desc(128, 64, 0, 0);
+#pragma unroll
+  for (int k = 0; k < 8; ++k) mma_bf16(d, kmajor_desc(a_base, k), kmajor_desc_h(b_base, k), idesc, k > 0 ? 1u : 0u);
+}
+// D[128 x 128] (+)= A[128 x 64] (bf16 in TMEM, 32 columns) . B[64 x 128] (MN-major half tile)
+__device__ __forceinline__ void mma_ts_h(uint32_t d, uint32_t a_tmem, uint32_t b_base, bool acc) {
+  constexpr uint32_t idesc = instr_desc(128, 128, 0, 1);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) mma_bf16_ts(d, a_tmem + 8 * k, mnmajor_desc_h(b_base, k), idesc, (acc || k > 0) ? 1u : 0u);
+}
+__device__ __forceinline__ void load_tile(unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int row, int z) {
+  tma_load_3d(dst, tm, bar, 0, row, z);
+  tma_load_3d(dst + HALF_BYTES, tm, bar, 64, row, z);
+}
+// `tm` must have a [64 columns x 64 rows] box
+__device__ __forceinline__ void load_half_tile(unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int row, int z) {
+  tma_load_3d(dst, tm, bar, 0, row, z);
+  tma_load_3d(dst + HT_HALF, tm, bar, 64, row, z);
+}
+
+// phi over the 128 features of one row by a pair of adjacent lanes: this lane owns the 64
+// columns of column half `half` (eight 16-byte chunks at src + row * 128 within that half's box).
+// src_half / dst_half point at the [rows x 64] box of this lane's column half.
+__device__ __forceinline__ void feature_map_pair(const unsigned char* src_half, unsigned char* dst_half, int row) {
+  float x[64];
+  float m = -INFINITY;
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    const uint4 u = *reinterpret_cast<const uint4*>(src_half + row * 128 + ((c ^ (row & 7)) << 4));
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 f = __bfloat1622float2(h[e]);
+      x[c * 8 + 2 * e] = f.x;
+      x[c * 8 + 2 * e + 1] = f.y;
+      m = fmaxf(m, fmaxf(f.x, f.y));
+    }
+  }
+  m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+  const float ml = m * 1.4426950408889634f;
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < 64; ++i) {
+    x[i] = ex2(x[i] * 1.4426950408889634f - ml);
+    sum += x[i];
+  }
+  sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+  const float inv = 1.f / sum;
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    uint4 u;
+    u.x = pack_bf16(x[c * 8 + 0] * inv, x[c * 8 + 1] * inv);
+    u.y = pack_bf16(x[c * 8 + 2] * inv, x[c * 8 + 3] * inv);
+    u.z = pack_bf16(x[c * 8 + 4] * inv, x[c * 8 + 5] * inv);
+    u.w = pack_bf16(x[c * 8 + 6] * inv, x[c * 8 + 7] * inv);
+    *reinterpret_cast<uint4*>(dst_half + row * 128 + ((c ^ (row & 7)) << 4)) = u;
+  }
+}
+
 // byte offset of 16-byte chunk c (0..15) of row r inside a swizzled [128 x 128] bf16 tile
 __device__ __forceinline__ uint32_t swz(int r, int c) {
   return (uint32_t)((c >> 3) * HALF_BYTES + r * 128 + (((c & 7) ^ (r & 7)) << 4));
@@ -128,12 +200,12 @@ inline EncodeTiledFn encode_fn() {
 }
 
 // [n_mats, rows, 128] bf16, box = 64 columns x 128 rows x 1, 128-byte swizzle, zero fill.
-inline bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t n_mats) {
+inline bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t n_mats, uint32_t box_rows = 128) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[3] = {128, rows, n_mats};
   const cuuint64_t strides[2] = {128 * 2, rows * 128 * 2};
-  const cuuint32_t box[3] = {64, 128, 1};
+  const cuuint32_t box[3] = {64, box_rows, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
