@@ -52,6 +52,9 @@ struct BwdArgs {
 
 #define WAIT_OR_RETURN(bar, parity) \
   do { if (!mbar_wait(&(bar), (parity), &bars->abort)) return false; } while (0)
+// for roles run by a whole converged warp
+#define WAIT_OR_RETURN_W(bar, parity) \
+  do { if (!mbar_wait_warp(&(bar), (parity), &bars->abort)) return false; } while (0)
 
 // ------------------------------------------------------------------------------ prep
 // One warp per row; lane owns 4 consecutive features.  Writes g_s, g_r (bf16), D and, when
@@ -189,7 +192,8 @@ tc_bwd_rdelta_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
   bool ok = true;
   for (int hh = 0; hh < group; ++hh) {         // every thread runs every iteration (block-wide barriers inside)
     const int z = kv * group + hh;
-    if (tid == 0 && !bars->abort) {
+    __syncwarp();
+    if (warp == 0 && !__any_sync(0xffffffffu, bars->abort != 0)) {
       mbar_arrive_expect_tx(&bars->full, 2 * TILE_BYTES);
       load_tile(smem, &tm_q, &bars->full, c * TILE, z);
       load_tile(smem + TILE_BYTES, &tm_g, &bars->full, c * TILE, z);
@@ -200,7 +204,7 @@ tc_bwd_rdelta_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
       fence_proxy_async_smem();
     }
     __syncthreads();
-    if (tid == 0 && !bars->abort) {
+    if (warp == 0 && !__any_sync(0xffffffffu, bars->abort != 0)) {
       tc_fence_after();
       mma_mnmn(tmem, smem_u32(smem), smem_u32(smem + TILE_BYTES), hh > 0);
       mma_commit(&bars->done);
@@ -277,23 +281,23 @@ __device__ bool dq_control(const CUtensorMap* tm_q, const CUtensorMap* tm_k, con
     load_tile(smem + DQ_OFF_K + i * TILE_BYTES, tm_k, &bars->kv_full[i], q0 - i * TILE, bh_kv);
     load_tile(smem + DQ_OFF_V + i * TILE_BYTES, tm_v, &bars->kv_full[i], q0 - i * TILE, bh_kv);
   }
-  WAIT_OR_RETURN(bars->qg_full, 0);
+  WAIT_OR_RETURN_W(bars->qg_full, 0);
   constexpr uint32_t idesc_ts = instr_desc(128, 128, 0, 1);
   const int last = (n_kt - 1) & 1, other = last ^ 1;
   for (int i = 0; i < n_kt; ++i) {
     const int b = i & 1;
-    WAIT_OR_RETURN(bars->kv_full[b], (i >> 1) & 1);
+    WAIT_OR_RETURN_W(bars->kv_full[b], (i >> 1) & 1);
     tc_fence_after();
     mma_kk(tS, sQ, sK + b * TILE_BYTES, false);          // S  = Q K^T
     mma_kk(tP, sG, sV + b * TILE_BYTES, false);          // dP = g_s V^T
     mma_commit(&bars->s_full);
-    WAIT_OR_RETURN(bars->ds_full, i & 1);
+    WAIT_OR_RETURN_W(bars->ds_full, i & 1);
     tc_fence_after();
 #pragma unroll
     for (int k = 0; k < 8; ++k)                           // dQ += dS K, dS read from TMEM
       mma_bf16_ts(tQ, tS + 8 * k, mnmajor_desc(sK + b * TILE_BYTES, k), idesc_ts, (i > 0 || k > 0) ? 1u : 0u);
     mma_commit(&bars->dq_done);
-    WAIT_OR_RETURN(bars->dq_done, i & 1);
+    WAIT_OR_RETURN_W(bars->dq_done, i & 1);
     if (i + 2 < n_kt) {
       mbar_arrive_expect_tx(&bars->kv_full[b], 2 * TILE_BYTES);
       load_tile(smem + DQ_OFF_K + b * TILE_BYTES, tm_k, &bars->kv_full[b], q0 - (i + 2) * TILE, bh_kv);
@@ -306,13 +310,13 @@ __device__ bool dq_control(const CUtensorMap* tm_q, const CUtensorMap* tm_k, con
   }
   if (has_rla) {
     const uint32_t sG2 = sV + other * TILE_BYTES, sSt = sK + other * TILE_BYTES;
-    WAIT_OR_RETURN(bars->x_full, 0);
+    WAIT_OR_RETURN_W(bars->x_full, 0);
     tc_fence_after();
     mma_kk(tS, sG2, sV + last * TILE_BYTES, false);        // dA = g_r V_cb^T
     if (has_state) mma_kk(tF, sG2, sSt, false);            // g_r S_cb^T
     mma_commit(&bars->s_full);
-    WAIT_OR_RETURN(bars->phik_ready, 0);
-    WAIT_OR_RETURN(bars->ds_full, n_kt & 1);
+    WAIT_OR_RETURN_W(bars->phik_ready, 0);
+    WAIT_OR_RETURN_W(bars->ds_full, n_kt & 1);
     tc_fence_after();
 #pragma unroll
     for (int k = 0; k < 8; ++k)                           // (dA masked) phi(K_cb)
@@ -534,7 +538,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   bool ok = true;
   if (warp < 4) {
     ok = dq_rows(a, &tm_dq, smem, bars, tmem, tid, q0, bh_q, n_kt, has_boundary, has_rla);
-  } else if (tid == 128) {
+  } else if (warp == 4) {
     ok = dq_control(&tm_q, &tm_k, &tm_v, &tm_gs, &tm_gr, &tm_st, smem, bars, tmem, q0, bh_q, bh_kv, n_kt,
                     has_rla, has_state, st_index);
     if (!ok) {
@@ -608,7 +612,7 @@ __device__ bool kv_loader(const CUtensorMap* tm_k, const CUtensorMap* tm_v, cons
   }
   for (int n = 0; n < pl.N; ++n) {
     const int st = pl.stage(n), u = pl.use(n);
-    if (u >= 1) WAIT_OR_RETURN(bars->acc_done[st], (u - 1) & 1);
+    if (u >= 1) WAIT_OR_RETURN_W(bars->acc_done[st], (u - 1) & 1);
     unsigned char* dst = smem + KV_OFF_STAGE + st * TILE_BYTES;
     const int z = bh_kv * pl.group + pl.head(n);
     const int row = pl.qtile(n) * TILE + 64 * pl.half(n);
@@ -635,10 +639,10 @@ __device__ bool kv_mma(unsigned char* smem, KvBars* bars, uint32_t tmem, const K
   const uint32_t tS[2] = {tmem + 256, tmem + 384}, tP[2] = {tmem + 320, tmem + 448};
   bool accV = false, accK = false;
 
-  WAIT_OR_RETURN(bars->kv_full, 0);
-  if (pl.n_R > 0) WAIT_OR_RETURN(bars->kphi_ready, 0);
+  WAIT_OR_RETURN_W(bars->kv_full, 0);
+  if (pl.n_R > 0) WAIT_OR_RETURN_W(bars->kphi_ready, 0);
   if (pl.has_inter) {
-    WAIT_OR_RETURN(bars->full[0], 0);
+    WAIT_OR_RETURN_W(bars->full[0], 0);
     tc_fence_after();
     mma_kk(tK, sV, sStage, false);                         // dphi_k = V_j R_j^T
     mma_kmn<1>(tV, sKphi, sStage, false);                  // dV     = phi(K_j) R_j
@@ -649,9 +653,9 @@ __device__ bool kv_mma(unsigned char* smem, KvBars* bars, uint32_t tmem, const K
     if (n < pl.N) {
       const int st = pl.stage(n), slot = n & 1;
       const uint32_t sQh = sStage + st * TILE_BYTES, sGh = sQh + HT_BYTES;
-      WAIT_OR_RETURN(bars->full[st], pl.use(n) & 1);
-      if (pl.is_r(n)) WAIT_OR_RETURN(bars->phiq_ready[slot], (n >> 1) & 1);
-      if (n >= 2) WAIT_OR_RETURN(bars->acc_done[pl.stage(n - 2)], pl.use(n - 2) & 1);   // the slot is free
+      WAIT_OR_RETURN_W(bars->full[st], pl.use(n) & 1);
+      if (pl.is_r(n)) WAIT_OR_RETURN_W(bars->phiq_ready[slot], (n >> 1) & 1);
+      if (n >= 2) WAIT_OR_RETURN_W(bars->acc_done[pl.stage(n - 2)], pl.use(n - 2) & 1);   // the slot is free
       tc_fence_after();
       mma_k_kh(tS[slot], pl.is_r(n) ? sKphi : sK, sQh);   // S^T  = K Q_h^T   (phi(K) phi(Q_h)^T)
       mma_k_kh(tP[slot], sV, sGh);                         // dP^T = V g_h^T
@@ -660,8 +664,8 @@ __device__ bool kv_mma(unsigned char* smem, KvBars* bars, uint32_t tmem, const K
     if (n >= 1) {
       const int m = n - 1, st = pl.stage(m), slot = m & 1;
       const uint32_t sQh = sStage + st * TILE_BYTES, sGh = sQh + HT_BYTES;
-      WAIT_OR_RETURN(bars->p_ready[slot], (m >> 1) & 1);
-      if (m == pl.n_R && pl.n_R > 0) WAIT_OR_RETURN(bars->fold_done, 0);
+      WAIT_OR_RETURN_W(bars->p_ready[slot], (m >> 1) & 1);
+      if (m == pl.n_R && pl.n_R > 0) WAIT_OR_RETURN_W(bars->fold_done, 0);
       tc_fence_after();
       mma_ts_h(tV, tS[slot], sGh, accV);                   // dV += P^T g_h
       mma_ts_h(tK, tP[slot], sQh, accK);                   // dK += dS^T Q_h   (dphi_k += dA^T phi(Q_h))
@@ -896,13 +900,13 @@ tc_bwd_dkv_kernel(const __grid_constant__ KvMaps tm, BwdArgs a) {
   bool ok = true;
   if (warp < 8) {
     ok = kv_rows(a, &tm.dk, &tm.dv, smem, bars, tmem, pl, warp >> 2, tid & 127, bh_kv);
-  } else if (tid == 256) {
+  } else if (warp == 8) {
     ok = kv_mma(smem, bars, tmem, pl);
     if (!ok) {
       mma_commit(&bars->drain);
       for (int it = 0; it < (1 << 16) && !mbar_try_wait(&bars->drain, 0); ++it) {}
     }
-  } else if (tid == 288) {
+  } else if (warp == 9) {
     ok = kv_loader(&tm.k, &tm.v, &tm.rs, &tm.qh, &tm.gsh, &tm.grh, a.lse2p, a.dscp, a.t_pad, smem, bars, pl,
                    bh_kv, rs_index);
   }

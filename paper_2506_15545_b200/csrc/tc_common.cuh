@@ -15,57 +15,63 @@ constexpr int TILE = 128;
 constexpr int HALF_BYTES = TILE * 64 * 2;   // one [128 x 64] bf16 sub-tile, 128-byte rows
 constexpr int TILE_BYTES = 2 * HALF_BYTES;
 
-// K-major operand: [128 rows x 128 reduction] as two 64-wide halves; 16 reduction elements
-// per MMA = 32 bytes along the 128-byte row.
-__device__ __forceinline__ uint64_t kmajor_desc(uint32_t base, int kstep) {
-  return smem_desc(base + (kstep >> 2) * HALF_BYTES + (kstep & 3) * 32, 16, 1024);
-}
-// MN-major operand: rows are the reduction index (128-byte rows of 64 columns, two column
-// halves 16 KB apart); 16 reduction rows per MMA = 2048 bytes.
-__device__ __forceinline__ uint64_t mnmajor_desc(uint32_t base, int kstep) {
-  return smem_desc(base + kstep * 2048, HALF_BYTES, 1024);
-}
+// Operand descriptors.  The descriptor of a tile is built once from its base address; the
+// eight (or four) reduction steps of a product then only add a constant to its start-address
+// field (bytes / 16; shared-memory addresses stay below 2^18, so the field never carries).
+//   K-major operand: [128 rows x 128 reduction] as two 64-wide halves; 16 reduction elements
+//   per MMA = 32 bytes along the 128-byte row.
+//   MN-major operand: rows are the reduction index (128-byte rows of 64 columns, two column
+//   halves 16 KB apart); 16 reduction rows per MMA = 2048 bytes.
+__device__ __forceinline__ uint64_t kmajor_base(uint32_t base) { return smem_desc(base, 16, 1024); }
+__device__ __forceinline__ uint64_t mnmajor_base(uint32_t base) { return smem_desc(base, HALF_BYTES, 1024); }
+__host__ __device__ constexpr uint32_t kstep_k(int k, int half_bytes) { return (uint32_t)(((k >> 2) * half_bytes + (k & 3) * 32) >> 4); }
+__host__ __device__ constexpr uint32_t kstep_mn(int k) { return (uint32_t)((k * 2048) >> 4); }
+__device__ __forceinline__ uint64_t kmajor_desc(uint32_t base, int kstep) { return kmajor_base(base) + kstep_k(kstep, HALF_BYTES); }
+__device__ __forceinline__ uint64_t mnmajor_desc(uint32_t base, int kstep) { return mnmajor_base(base) + kstep_mn(kstep); }
 
 // D[128x128] (+)= A B^T-style products over a reduction of 128, 8 MMAs of K = 16.
 __device__ __forceinline__ void mma_kk(uint32_t d, uint32_t a_base, uint32_t b_base, bool acc) {
   constexpr uint32_t idesc = instr_desc(128, 128, 0, 0);
+  const uint64_t a0 = kmajor_base(a_base), b0 = kmajor_base(b_base);
 #pragma unroll
-  for (int k = 0; k < 8; ++k) mma_bf16(d, kmajor_desc(a_base, k), kmajor_desc(b_base, k), idesc, (acc || k > 0) ? 1u : 0u);
+  for (int k = 0; k < 8; ++k)
+    mma_bf16(d, a0 + kstep_k(k, HALF_BYTES), b0 + kstep_k(k, HALF_BYTES), idesc, (acc || k > 0) ? 1u : 0u);
 }
 template <int AB_BF16>
 __device__ __forceinline__ void mma_kmn(uint32_t d, uint32_t a_base, uint32_t b_base, bool acc) {
   constexpr uint32_t idesc = instr_desc(128, 128, 0, 1, AB_BF16);
+  const uint64_t a0 = kmajor_base(a_base), b0 = mnmajor_base(b_base);
 #pragma unroll
-  for (int k = 0; k < 8; ++k) mma_bf16(d, kmajor_desc(a_base, k), mnmajor_desc(b_base, k), idesc, (acc || k > 0) ? 1u : 0u);
+  for (int k = 0; k < 8; ++k) mma_bf16(d, a0 + kstep_k(k, HALF_BYTES), b0 + kstep_mn(k), idesc, (acc || k > 0) ? 1u : 0u);
 }
 __device__ __forceinline__ void mma_mnmn(uint32_t d, uint32_t a_base, uint32_t b_base, bool acc) {
   constexpr uint32_t idesc = instr_desc(128, 128, 1, 1);
+  const uint64_t a0 = mnmajor_base(a_base), b0 = mnmajor_base(b_base);
 #pragma unroll
-  for (int k = 0; k < 8; ++k) mma_bf16(d, mnmajor_desc(a_base, k), mnmajor_desc(b_base, k), idesc, (acc || k > 0) ? 1u : 0u);
+  for (int k = 0; k < 8; ++k) mma_bf16(d, a0 + kstep_mn(k), b0 + kstep_mn(k), idesc, (acc || k > 0) ? 1u : 0u);
 }
 
 // ---- half tiles: [64 rows x 128 columns] bf16 as two [64 x 64] boxes of 8 KB ------------
 constexpr int HT_HALF = 64 * 64 * 2;
 constexpr int HT_BYTES = 2 * HT_HALF;
 // B operand, K-major: the half tile's 64 rows are N, its 128 columns the reduction (8 steps)
-__device__ __forceinline__ uint64_t kmajor_desc_h(uint32_t base, int kstep) {
-  return smem_desc(base + (kstep >> 2) * HT_HALF + (kstep & 3) * 32, 16, 1024);
-}
+__device__ __forceinline__ uint64_t kmajor_base_h(uint32_t base) { return smem_desc(base, 16, 1024); }
 // B operand, MN-major: the half tile's 128 columns are N, its 64 rows the reduction (4 steps)
-__device__ __forceinline__ uint64_t mnmajor_desc_h(uint32_t base, int kstep) {
-  return smem_desc(base + kstep * 2048, HT_HALF, 1024);
-}
+__device__ __forceinline__ uint64_t mnmajor_base_h(uint32_t base) { return smem_desc(base, HT_HALF, 1024); }
 // D[128 x 64] = A[128 x 128] (K-major full tile) . B[64 x 128]^T (K-major half tile)
 __device__ __forceinline__ void mma_k_kh(uint32_t d, uint32_t a_base, uint32_t b_base) {
   constexpr uint32_t idesc = instr_desc(128, 64, 0, 0);
+  const uint64_t a0 = kmajor_base(a_base), b0 = kmajor_base_h(b_base);
 #pragma unroll
-  for (int k = 0; k < 8; ++k) mma_bf16(d, kmajor_desc(a_base, k), kmajor_desc_h(b_base, k), idesc, k > 0 ? 1u : 0u);
+  for (int k = 0; k < 8; ++k)
+    mma_bf16(d, a0 + kstep_k(k, HALF_BYTES), b0 + kstep_k(k, HT_HALF), idesc, k > 0 ? 1u : 0u);
 }
 // D[128 x 128] (+)= A[128 x 64] (bf16 in TMEM, 32 columns) . B[64 x 128] (MN-major half tile)
 __device__ __forceinline__ void mma_ts_h(uint32_t d, uint32_t a_tmem, uint32_t b_base, bool acc) {
   constexpr uint32_t idesc = instr_desc(128, 128, 0, 1);
+  const uint64_t b0 = mnmajor_base_h(b_base);
 #pragma unroll
-  for (int k = 0; k < 4; ++k) mma_bf16_ts(d, a_tmem + 8 * k, mnmajor_desc_h(b_base, k), idesc, (acc || k > 0) ? 1u : 0u);
+  for (int k = 0; k < 4; ++k) mma_bf16_ts(d, a_tmem + 8 * k, b0 + kstep_mn(k), idesc, (acc || k > 0) ? 1u : 0u);
 }
 __device__ __forceinline__ void load_tile(unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int row, int z) {
   tma_load_3d(dst, tm, bar, 0, row, z);

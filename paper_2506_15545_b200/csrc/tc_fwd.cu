@@ -61,8 +61,11 @@ struct TcArgs {
 
 #define WAIT_OR_RETURN(bar, parity) \
   do { if (!mbar_wait(&(bar), (parity), &bars->abort)) return false; } while (0)
+// for roles run by a whole converged warp
+#define WAIT_OR_RETURN_W(bar, parity) \
+  do { if (!mbar_wait_warp(&(bar), (parity), &bars->abort)) return false; } while (0)
 
-// ------------------------------------------------------------------ control thread
+// ------------------------------------------------------------------ control warp (all 32 lanes)
 __device__ bool control_role(const CUtensorMap* tm_q, const CUtensorMap* tm_k, const CUtensorMap* tm_v,
                              const CUtensorMap* tm_st, unsigned char* smem, FwdBars* bars, uint32_t tmem,
                              int q0, int bh_q, int bh_kv, int n_kt, bool has_rla, bool has_state, int st_index) {
@@ -83,8 +86,8 @@ __device__ bool control_role(const CUtensorMap* tm_q, const CUtensorMap* tm_k, c
   }
   if (has_state) load_tile(tm_st, OFF_ST, &bars->st_full, 0, st_index);
 
-  WAIT_OR_RETURN(bars->q_full, 0);
-  WAIT_OR_RETURN(bars->k_full[0], 0);
+  WAIT_OR_RETURN_W(bars->q_full, 0);
+  WAIT_OR_RETURN_W(bars->k_full[0], 0);
   tc_fence_after();
   mma_kk(tS[0], sQ, sK, false);
   mma_commit(&bars->s_full[0]);
@@ -92,22 +95,22 @@ __device__ bool control_role(const CUtensorMap* tm_q, const CUtensorMap* tm_k, c
   for (int i = 0; i < n_kt; ++i) {
     if (i + 1 < n_kt) {                       // scores of the next tile into the other buffer
       const int b = (i + 1) & 1;
-      WAIT_OR_RETURN(bars->k_full[b], ((i + 1) >> 1) & 1);
-      if (i + 1 >= 2) WAIT_OR_RETURN(bars->s_empty[b], (((i + 1) >> 1) - 1) & 1);
+      WAIT_OR_RETURN_W(bars->k_full[b], ((i + 1) >> 1) & 1);
+      if (i + 1 >= 2) WAIT_OR_RETURN_W(bars->s_empty[b], (((i + 1) >> 1) - 1) & 1);
       tc_fence_after();
       mma_kk(tS[b], sQ, sK + b * TILE_BYTES, false);
       mma_commit(&bars->s_full[b]);
     }
     if (i >= 1 && i + 1 < n_kt) {             // V of tile i+1 replaces V of tile i-1
-      WAIT_OR_RETURN(bars->pv_done, (i - 1) & 1);
+      WAIT_OR_RETURN_W(bars->pv_done, (i - 1) & 1);
       load_tile(tm_v, OFF_V + ((i + 1) & 1) * TILE_BYTES, &bars->v_full[(i + 1) & 1], q0 - (i + 1) * TILE, bh_kv);
     }
     if (i + 2 < n_kt) {                       // K of tile i+2 replaces K of tile i
-      WAIT_OR_RETURN(bars->s_full[i & 1], (i >> 1) & 1);
+      WAIT_OR_RETURN_W(bars->s_full[i & 1], (i >> 1) & 1);
       load_tile(tm_k, OFF_K + (i & 1) * TILE_BYTES, &bars->k_full[i & 1], q0 - (i + 2) * TILE, bh_kv);
     }
-    WAIT_OR_RETURN(bars->p_full, i & 1);
-    WAIT_OR_RETURN(bars->v_ready[i & 1], (i >> 1) & 1);
+    WAIT_OR_RETURN_W(bars->p_full, i & 1);
+    WAIT_OR_RETURN_W(bars->v_ready[i & 1], (i >> 1) & 1);
     tc_fence_after();
     mma_kmn<0>(tOs, sP, sV + (i & 1) * TILE_BYTES, i > 0);
     mma_commit(&bars->pv_done);
@@ -117,17 +120,17 @@ __device__ bool control_role(const CUtensorMap* tm_q, const CUtensorMap* tm_k, c
     const int last = (n_kt - 1) & 1;          // stage of the oldest tile of the band
     const int ba = n_kt & 1;                  // score buffer for phi(Q) phi(K)^T
     const int uses = (n_kt - ba + 1) >> 1;    // earlier uses of that buffer
-    WAIT_OR_RETURN(bars->phi_ready, 0);
-    if (uses > 0) WAIT_OR_RETURN(bars->s_empty[ba], (uses - 1) & 1);
+    WAIT_OR_RETURN_W(bars->phi_ready, 0);
+    if (uses > 0) WAIT_OR_RETURN_W(bars->s_empty[ba], (uses - 1) & 1);
     tc_fence_after();
     mma_kk(tS[ba], sQ, sK + last * TILE_BYTES, false);
     mma_commit(&bars->s_full[ba]);
     if (has_state) {
-      WAIT_OR_RETURN(bars->st_full, 0);
+      WAIT_OR_RETURN_W(bars->st_full, 0);
       tc_fence_after();
       mma_kmn<1>(tOr, sQ, sST, false);
     }
-    WAIT_OR_RETURN(bars->p_full, n_kt & 1);
+    WAIT_OR_RETURN_W(bars->p_full, n_kt & 1);
     tc_fence_after();
     mma_kmn<0>(tOr, sP, sV + last * TILE_BYTES, has_state);
   }
@@ -383,7 +386,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   if (warp == 4) {
     tmem_alloc(&bars->tmem_base, 512);
     tmem_relinquish();
-    if (tid == 128) {
+    if (tid == 128) {   // one lane is enough for the prefetches
       prefetch_tensormap(&tm_q);
       prefetch_tensormap(&tm_k);
       prefetch_tensormap(&tm_v);
@@ -399,7 +402,7 @@ tc_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   bool ok = true;
   if (warp < 4) {
     ok = softmax_role(a, &tm_out, smem, bars, tmem, tid, q0, bh_q, h, n_kt, has_boundary, has_rla);
-  } else if (tid == 128) {
+  } else if (warp == 4) {
     ok = control_role(&tm_q, &tm_k, &tm_v, &tm_st, smem, bars, tmem, q0, bh_q, bh_kv, n_kt, has_rla,
                       has_state, st_index);
     if (!ok) {
@@ -445,7 +448,7 @@ tc_chunk_delta_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
-  if (tid == 0) {
+  if (warp == 0) {
     mbar_arrive_expect_tx(&bars->full, 2 * TILE_BYTES);
     tma_load_3d(smem, &tm_k, &bars->full, 0, c * TILE, kv);
     tma_load_3d(smem + HALF_BYTES, &tm_k, &bars->full, 64, c * TILE, kv);
@@ -458,7 +461,7 @@ tc_chunk_delta_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_con
     fence_proxy_async_smem();
   }
   __syncthreads();
-  if (tid == 0 && !bars->abort) {
+  if (warp == 0 && !__any_sync(0xffffffffu, bars->abort != 0)) {
     tc_fence_after();
     mma_mnmn(tmem, smem_u32(smem), smem_u32(smem + TILE_BYTES), false);   // phi(K)^T V  (Eq. 2)
     mma_commit(&bars->done);
