@@ -77,7 +77,8 @@ cudaError_t launch_generic_backward(const Args& a, cudaStream_t s);
 cudaError_t launch_decode(const Args& a, void* k_ring, void* v_ring, float* state, int pos,
                           cudaStream_t s);
 cudaError_t launch_handoff(const Args& a, cudaStream_t s);
-cudaError_t launch_tc_forward(const Args& a, cudaStream_t s);
+cudaError_t launch_tc_forward(const Args& a, cudaStream_t s);        // chunk states, then the main kernel
+cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s);
 cudaError_t launch_tc_backward(const Args& a, cudaStream_t s);
 
 void count_launches(int n);

@@ -3,6 +3,8 @@
 // 128 x 128 x 128 MMA chains, the in-place feature map and the host-side tensor maps.
 #pragma once
 
+#include <cuda_fp16.h>
+
 #include "rattn_internal.h"
 #include "tc_ptx.cuh"
 
@@ -151,6 +153,73 @@ __device__ __forceinline__ void flush_f32_block(const unsigned char* stage, int 
     const int row = (r >> 5) * 32 + 4 * k + ((r & 31) >> 3);
     const float4 v = *reinterpret_cast<const float4*>(stage + row * 128 + ((sub ^ (row & 7)) << 4));
     if (row < n_rows) *reinterpret_cast<float4*>(dst + (size_t)row * 128 + 4 * sub) = v;
+  }
+}
+
+// Row maximum of row r of a swizzled bf16 tile.
+__device__ __forceinline__ float row_max_bf16(const unsigned char* tile, int r) {
+  float m = -INFINITY;
+#pragma unroll
+  for (int c = 0; c < 16; ++c) {
+    const uint4 u = *reinterpret_cast<const uint4*>(tile + swz(r, c));
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 f = __bfloat1622float2(h[e]);
+      m = fmaxf(m, fmaxf(f.x, f.y));
+    }
+  }
+  return m;
+}
+// Un-normalised feature map of row r, in place: x -> exp(x - max) (bf16); returns 1 / sum so
+// that the caller can scale whatever is linear in this row afterwards.  Few live registers.
+__device__ __forceinline__ float feature_map_row_unnorm_inplace(unsigned char* tile, int r) {
+  const float ml = row_max_bf16(tile, r) * 1.4426950408889634f;
+  float sum = 0.f;
+#pragma unroll
+  for (int c = 0; c < 16; ++c) {
+    uint4 u = *reinterpret_cast<const uint4*>(tile + swz(r, c));
+    uint32_t* w = reinterpret_cast<uint32_t*>(&u);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
+      const float e0 = ex2(f.x * 1.4426950408889634f - ml), e1 = ex2(f.y * 1.4426950408889634f - ml);
+      sum += e0 + e1;
+      w[e] = pack_bf16(e0, e1);
+    }
+    *reinterpret_cast<uint4*>(tile + swz(r, c)) = u;
+  }
+  return 1.f / sum;
+}
+// phi of row r, in place, with few live registers: the exponentials are parked in the tile
+// itself as fp16 between the summation and the normalisation (one bf16 rounding in the end).
+__device__ __forceinline__ void feature_map_row_inplace_lr(unsigned char* tile, int r) {
+  const float ml = row_max_bf16(tile, r) * 1.4426950408889634f;
+  float sum = 0.f;
+#pragma unroll
+  for (int c = 0; c < 16; ++c) {
+    uint4 u = *reinterpret_cast<const uint4*>(tile + swz(r, c));
+    uint32_t* w = reinterpret_cast<uint32_t*>(&u);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
+      const float e0 = ex2(f.x * 1.4426950408889634f - ml), e1 = ex2(f.y * 1.4426950408889634f - ml);
+      sum += e0 + e1;
+      w[e] = pack_f16(e0, e1);
+    }
+    *reinterpret_cast<uint4*>(tile + swz(r, c)) = u;
+  }
+  const float inv = 1.f / sum;
+#pragma unroll
+  for (int c = 0; c < 16; ++c) {
+    uint4 u = *reinterpret_cast<const uint4*>(tile + swz(r, c));
+    uint32_t* w = reinterpret_cast<uint32_t*>(&u);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w[e]));
+      w[e] = pack_bf16(f.x * inv, f.y * inv);
+    }
+    *reinterpret_cast<uint4*>(tile + swz(r, c)) = u;
   }
 }
 

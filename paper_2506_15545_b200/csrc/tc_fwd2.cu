@@ -1,0 +1,642 @@
+// Tensor-core forward for bf16, d = 128, window a multiple of 128 (sm_100a: TMA + tcgen05 + TMEM).
+//
+// Persistent kernel, one CTA per SM.  A work unit is a pair of adjacent query tiles (A = 2p,
+// B = 2p+1, 128 rows each) of one query head; the two tiles share one descending stream of
+// key tiles (2p+1 down to 2p - w/128), so every K/V tile is fetched once for both.
+//
+//   row group A / B (4 warps each, thread = query row = TMEM lane)
+//       SWA (Section 2.1): online softmax straight out of TMEM; P (fp16) is written back over
+//       the score columns and read from there by the P V product, so it never touches shared
+//       memory.  While one group exponentiates, the tensor pipe works for the other group.
+//   MMA warp      S = Q K^T, O += P V (A operand from TMEM), the residual-branch products
+//   loader warp   TMA: Q tiles, K/V stages, the stored chunk state
+//   2 helper warps re-encode each V tile bf16 -> fp16 in place (tcgen05 needs A and B of one type)
+//
+//   RLA (Eq. 4 in the chunkwise form of Eq. 2-3 with the window lag): when a tile's window loop
+//   ends, its normalised window output is parked in registers (fp16) and the same accumulator
+//   is reused.  With cA = 2p - w/128 the chunk tile A reads in "intra" form and S_[cA] the stored
+//   state (sum over the chunks before cA of phi(K)^T V):
+//       O_rla(A) = phi(Q_A) S_[cA] + ((phi(Q_A) phi(K_cA)^T) masked to j < t - w) V_cA
+//       O_rla(B) = phi(Q_B) S_[cA] +  (phi(Q_B) phi(K_cA)^T) V_cA                       (chunk cA whole)
+//                                  + ((phi(Q_B) phi(K_cB)^T) masked) V_cB,   cB = cA + 1
+//   so one stored state serves both tiles.  phi (softmax over the head features, Section 3.1)
+//   is applied to the Q and K tiles in shared memory, in place: it never goes to HBM.
+//   Section 3.2: y = g_s * o_swa / rms(o_swa) + g_r * o_rla / rms(o_rla), staged in the tile's Q
+//   buffer and written by one TMA store.
+#include "tc_common.cuh"
+
+namespace rattn {
+namespace {
+
+using namespace ptx;
+using namespace tc;
+
+constexpr int F_OFF_Q = 0;                       // Q_A, Q_B
+constexpr int F_OFF_KV = 2 * TILE_BYTES;         // 2 stages x [K | V]
+constexpr int F_OFF_X = 6 * TILE_BYTES;          // stored chunk state
+constexpr int F_OFF_BAR = 7 * TILE_BYTES;
+constexpr int F_SMEM = F_OFF_BAR + 512;
+constexpr int F_THREADS = 384;
+constexpr float LOG2E = 1.4426950408889634f;
+
+struct FBars {
+  uint64_t q_full[2], q_free[2], kv_full[2], v_ready[2], kv_free[2], x_full, x_free;
+  uint64_t s_full[2], p_ready[2], o_ready[2], stash_done[2], phiq_ready[2], phik_ready[2], o_free[2], drain;
+  uint32_t tmem_base;
+  int abort;
+};
+
+struct FArgs {
+  float* lse;
+  float* o_swa;
+  float* o_rla;
+  const float* gamma_swa;
+  const float* gamma_rla;
+  int* status;
+  int T, w, H_q, group, mode, n_chunks, n_qt, n_pairs, n_units, n_bh;
+  float scale_log2, eps;
+};
+
+struct FMaps {
+  CUtensorMap q, k, v, st, out;
+};
+
+// What one unit consists of; every role derives the same plan from the unit index.
+struct Unit {
+  int bh_q, bh_kv, h;
+  int t[2];                 // tile index of A, B (B: -1 when the sequence ends after A)
+  int kt_hi, n;             // key tiles kt_hi, kt_hi-1, ..., kt_hi-n+1
+  int i0[2], i1[2];         // stream positions each tile is active on (inclusive)
+  bool rla[2];
+  bool has_state;           // cA > 0: a stored state exists
+  int cA;
+  bool windowed;
+  int wt;
+};
+
+__device__ __forceinline__ Unit make_unit(const FArgs& a, int u) {
+  Unit un;
+  const int pr = u / a.n_bh;                     // heaviest pairs first
+  un.bh_q = u % a.n_bh;
+  const int p = a.n_pairs - 1 - pr;
+  const int b = un.bh_q / a.H_q;
+  un.h = un.bh_q % a.H_q;
+  un.bh_kv = b * (a.H_q / a.group) + un.h / a.group;
+  un.wt = a.w / TILE;
+  un.windowed = (a.mode != RATTN_MODE_FULL_CAUSAL);
+  un.t[0] = 2 * p;
+  un.t[1] = (2 * p + 1 < a.n_qt) ? 2 * p + 1 : -1;
+  un.kt_hi = un.t[1] >= 0 ? un.t[1] : un.t[0];
+  const int loA = un.windowed ? max(0, un.t[0] - un.wt) : 0;
+  un.n = un.kt_hi - loA + 1;
+  un.i0[0] = un.kt_hi - un.t[0];
+  un.i1[0] = un.n - 1;
+  un.i0[1] = 0;
+  un.i1[1] = un.t[1] >= 0 ? un.kt_hi - (un.windowed ? max(0, un.t[1] - un.wt) : 0) : -1;
+  const bool rla_mode = un.windowed && a.mode == RATTN_MODE_RATTN;
+  un.rla[0] = rla_mode && un.t[0] - un.wt >= 0;
+  un.rla[1] = rla_mode && un.t[1] >= 0 && un.t[1] - un.wt >= 0;
+  un.cA = un.t[0] - un.wt;
+  un.has_state = un.rla[0] && un.cA > 0;
+  return un;
+}
+
+__device__ __forceinline__ bool active(const Unit& un, int X, int i) { return un.t[X] >= 0 && i >= un.i0[X] && i <= un.i1[X]; }
+
+#define WAIT_OR_RETURN(bar, parity) \
+  do { if (!mbar_wait(&(bar), (parity), &bars->abort)) return false; } while (0)
+#define WAIT_OR_RETURN_W(bar, parity) \
+  do { if (!mbar_wait_warp(&(bar), (parity), &bars->abort)) return false; } while (0)
+
+// D[128x128] (+)= P[128 x 128 keys] (fp16 in TMEM, 64 columns) . V[128 keys x 128] (fp16, MN-major)
+__device__ __forceinline__ void mma_pv(uint32_t d, uint32_t p_tmem, uint32_t v_base, bool acc) {
+  constexpr uint32_t idesc = instr_desc(128, 128, 0, 1, 0);
+  const uint64_t b0 = mnmajor_base(v_base);
+#pragma unroll
+  for (int k = 0; k < 8; ++k) mma_bf16_ts(d, p_tmem + 8 * k, b0 + kstep_mn(k), idesc, (acc || k > 0) ? 1u : 0u);
+}
+
+// ----------------------------------------------------------------------------- loader
+__device__ bool fwd_loader(const FMaps& tm, const FArgs& a, unsigned char* smem, FBars* bars) {
+  int kv_count = 0, cntU[2] = {0, 0}, cntX = 0;
+  for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+    const Unit un = make_unit(a, u);
+#pragma unroll
+    for (int X = 0; X < 2; ++X) {
+      if (un.t[X] < 0) continue;
+      if (cntU[X] >= 1) WAIT_OR_RETURN_W(bars->q_free[X], (cntU[X] - 1) & 1);
+      mbar_arrive_expect_tx(&bars->q_full[X], TILE_BYTES);
+      load_tile(smem + F_OFF_Q + X * TILE_BYTES, &tm.q, &bars->q_full[X], un.t[X] * TILE, un.bh_q);
+      ++cntU[X];
+    }
+    for (int i = 0; i < un.n; ++i, ++kv_count) {
+      const int st = kv_count & 1, use = kv_count >> 1;
+      if (use >= 1) WAIT_OR_RETURN_W(bars->kv_free[st], (use - 1) & 1);
+      unsigned char* dst = smem + F_OFF_KV + st * 2 * TILE_BYTES;
+      mbar_arrive_expect_tx(&bars->kv_full[st], 2 * TILE_BYTES);
+      load_tile(dst, &tm.k, &bars->kv_full[st], (un.kt_hi - i) * TILE, un.bh_kv);
+      load_tile(dst + TILE_BYTES, &tm.v, &bars->kv_full[st], (un.kt_hi - i) * TILE, un.bh_kv);
+    }
+    if (un.has_state) {
+      if (cntX >= 1) WAIT_OR_RETURN_W(bars->x_free, (cntX - 1) & 1);
+      mbar_arrive_expect_tx(&bars->x_full, TILE_BYTES);
+      load_tile(smem + F_OFF_X, &tm.st, &bars->x_full, 0, un.bh_kv * a.n_chunks + un.cA);
+      ++cntX;
+    }
+  }
+  return true;
+}
+
+// -------------------------------------------------------------------------- V re-encoding
+__device__ bool fwd_convert(const FArgs& a, unsigned char* smem, FBars* bars, int cid) {
+  int kv_count = 0;
+  for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+    const Unit un = make_unit(a, u);
+    for (int i = 0; i < un.n; ++i, ++kv_count) {
+      const int st = kv_count & 1, use = kv_count >> 1;
+      WAIT_OR_RETURN(bars->kv_full[st], use & 1);
+      unsigned char* tile = smem + F_OFF_KV + st * 2 * TILE_BYTES + TILE_BYTES;
+#pragma unroll 4
+      for (int c = cid; c < TILE_BYTES / 16; c += 64) {
+        uint4 x = *reinterpret_cast<uint4*>(tile + c * 16);
+        x.x = bf16x2_to_f16x2(x.x);
+        x.y = bf16x2_to_f16x2(x.y);
+        x.z = bf16x2_to_f16x2(x.z);
+        x.w = bf16x2_to_f16x2(x.w);
+        *reinterpret_cast<uint4*>(tile + c * 16) = x;
+      }
+      fence_proxy_async_smem();
+      mbar_arrive(&bars->v_ready[st]);
+    }
+  }
+  return true;
+}
+
+// ----------------------------------------------------------------------------- MMA warp
+__device__ bool fwd_mma(const FArgs& a, unsigned char* smem, FBars* bars, uint32_t tmem) {
+  const uint32_t sQ[2] = {smem_u32(smem + F_OFF_Q), smem_u32(smem + F_OFF_Q + TILE_BYTES)};
+  const uint32_t sKV = smem_u32(smem + F_OFF_KV), sX = smem_u32(smem + F_OFF_X);
+  const uint32_t tS[2] = {tmem, tmem + 128}, tO[2] = {tmem + 256, tmem + 384};
+  int kv_count = 0, cntU[2] = {0, 0}, cntX = 0, cntP[2] = {0, 0}, cntR[2] = {0, 0}, cntK[2] = {0, 0};
+
+  for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+    const Unit un = make_unit(a, u);
+    const int kv0 = kv_count;
+    auto stage_of = [&](int i) { return (kv0 + i) & 1; };
+    auto use_of = [&](int i) { return (kv0 + i) >> 1; };
+    auto sK = [&](int i) { return sKV + stage_of(i) * 2 * TILE_BYTES; };
+    auto sV = [&](int i) { return sKV + stage_of(i) * 2 * TILE_BYTES + TILE_BYTES; };
+#pragma unroll
+    for (int X = 0; X < 2; ++X) {
+      if (un.t[X] < 0) continue;
+      if (cntU[X] >= 1) WAIT_OR_RETURN_W(bars->o_free[X], (cntU[X] - 1) & 1);   // previous unit has read O_X
+      WAIT_OR_RETURN_W(bars->q_full[X], cntU[X] & 1);
+      ++cntU[X];
+    }
+    // first scores of each tile
+    WAIT_OR_RETURN_W(bars->kv_full[stage_of(0)], use_of(0) & 1);
+    tc_fence_after();
+#pragma unroll
+    for (int X = 1; X >= 0; --X) {
+      if (active(un, X, 0)) {
+        mma_kk(tS[X], sQ[X], sK(0), false);
+        mma_commit(&bars->s_full[X]);
+      }
+    }
+    for (int i = 0; i < un.n; ++i) {
+#pragma unroll
+      for (int X = 0; X < 2; ++X) {
+        if (active(un, X, i)) {
+          WAIT_OR_RETURN_W(bars->p_ready[X], cntP[X] & 1);
+          ++cntP[X];
+          WAIT_OR_RETURN_W(bars->v_ready[stage_of(i)], use_of(i) & 1);
+          tc_fence_after();
+          mma_pv(tO[X], tS[X], sV(i), i > un.i0[X]);                             // O_X += P V
+          if (i == un.i1[X]) mma_commit(&bars->o_ready[X]);
+        }
+        if (i + 1 < un.n && active(un, X, i + 1)) {
+          WAIT_OR_RETURN_W(bars->kv_full[stage_of(i + 1)], use_of(i + 1) & 1);
+          tc_fence_after();
+          mma_kk(tS[X], sQ[X], sK(i + 1), false);                                // S_X = Q_X K^T (after P V in pipe order)
+          mma_commit(&bars->s_full[X]);
+        }
+      }
+      // the stage is released here unless the residual branch still reads it
+      const bool keep = (un.rla[0] && i == un.n - 1) || (un.rla[1] && i == un.i1[1]);
+      if (!keep) mma_commit(&bars->kv_free[stage_of(i)]);
+    }
+    // ---- residual branch ---------------------------------------------------------------
+    const int iA = un.n - 1, iB = un.i1[1];          // stream positions of chunks cA, cB
+    if (un.rla[0] || un.rla[1]) {
+      if (un.has_state) {
+        WAIT_OR_RETURN_W(bars->x_full, cntX & 1);
+        ++cntX;
+      }
+      if (un.rla[0]) {
+        WAIT_OR_RETURN_W(bars->stash_done[0], cntR[0] & 1);
+        WAIT_OR_RETURN_W(bars->phiq_ready[0], cntR[0] & 1);
+        WAIT_OR_RETURN_W(bars->phik_ready[0], cntK[0] & 1);
+        tc_fence_after();
+        if (un.has_state) mma_kmn<1>(tO[0], sQ[0], sX, false);                   // phi(Q_A) S_[cA]
+        mma_kk(tS[0], sQ[0], sK(iA), false);                                     // phi(Q_A) phi(K_cA)^T
+        mma_commit(&bars->s_full[0]);
+      }
+      if (un.rla[1]) {
+        WAIT_OR_RETURN_W(bars->stash_done[1], cntR[1] & 1);
+        WAIT_OR_RETURN_W(bars->phiq_ready[1], cntR[1] & 1);
+        tc_fence_after();
+        if (un.rla[0]) {
+          if (un.has_state) mma_kmn<1>(tO[1], sQ[1], sX, false);                 // phi(Q_B) S_[cA]
+          mma_kk(tS[1], sQ[1], sK(iA), false);                                   // phi(Q_B) phi(K_cA)^T, whole chunk
+          mma_commit(&bars->s_full[1]);
+        }
+      }
+      if (un.rla[0]) {
+        WAIT_OR_RETURN_W(bars->p_ready[0], cntP[0] & 1);
+        ++cntP[0];
+        tc_fence_after();
+        mma_pv(tO[0], tS[0], sV(iA), un.has_state);
+        mma_commit(&bars->o_ready[0]);
+      }
+      if (un.rla[1]) {
+        if (un.rla[0]) {
+          WAIT_OR_RETURN_W(bars->p_ready[1], cntP[1] & 1);
+          ++cntP[1];
+          tc_fence_after();
+          mma_pv(tO[1], tS[1], sV(iA), un.has_state);
+        }
+        WAIT_OR_RETURN_W(bars->phik_ready[1], cntK[1] & 1);
+        tc_fence_after();
+        mma_kk(tS[1], sQ[1], sK(iB), false);                                     // phi(Q_B) phi(K_cB)^T
+        mma_commit(&bars->s_full[1]);
+        WAIT_OR_RETURN_W(bars->p_ready[1], cntP[1] & 1);
+        ++cntP[1];
+        tc_fence_after();
+        mma_pv(tO[1], tS[1], sV(iB), un.rla[0]);
+        mma_commit(&bars->o_ready[1]);
+      }
+      if (un.has_state) mma_commit(&bars->x_free);
+      if (un.rla[0]) { ++cntR[0]; ++cntK[0]; }
+      if (un.rla[1]) { ++cntR[1]; ++cntK[1]; }
+      // the chunk stages
+      if (un.rla[0]) mma_commit(&bars->kv_free[stage_of(iA)]);
+      if (un.rla[1] && !(un.rla[0] && iB == iA)) mma_commit(&bars->kv_free[stage_of(iB)]);
+    }
+    kv_count += un.n;
+  }
+  return true;
+}
+
+// ------------------------------------------------------------------------------ row groups
+__device__ __forceinline__ uint32_t lane_base(int r) { return (uint32_t)((r & ~31) << 16); }
+
+template <int X>
+__device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, FBars* bars, uint32_t tmem, int r) {
+  const uint32_t tS = tmem + 128 * X + lane_base(r), tO = tmem + 256 + 128 * X + lane_base(r);
+  unsigned char* sQ = smem + F_OFF_Q + X * TILE_BYTES;
+  int kv_count = 0, cntS = 0, cntO = 0;
+
+  for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+    const Unit un = make_unit(a, u);
+    const int kv0 = kv_count;
+    kv_count += un.n;
+    if (un.t[X] < 0) continue;
+    const int q0 = un.t[X] * TILE;
+    const int t = q0 + r;
+
+    // ---- window branch: online softmax over the key tiles of the band -------------------
+    float m_ref = -INFINITY, l = 0.f;
+    for (int i = un.i0[X]; i <= un.i1[X]; ++i) {
+      const int kt = un.kt_hi - i;
+      WAIT_OR_RETURN(bars->s_full[X], cntS & 1);
+      ++cntS;
+      tc_fence_after();
+      const bool diag = (kt == un.t[X]), bound = un.windowed && (kt == un.t[X] - un.wt);
+      // pass 1 over the scores: row maximum (32 columns at a time keeps the register count low)
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float x[32];
+        tmem_ld32(tS + 32 * c, x);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const int j = 32 * c + e;
+          const bool ok = !((diag && j > r) || (bound && j < r));
+          mx = fmaxf(mx, ok ? x[e] : -INFINITY);
+        }
+      }
+      mx *= a.scale_log2;                                              // scale > 0
+      // lazy rescale: the reference maximum only moves when the row maximum grew by more than 2^8
+      const float m_new = fmaxf(m_ref, mx);
+      bool rescale = false;
+      if (i == un.i0[X]) m_ref = m_new;
+      else rescale = __any_sync(0xffffffffu, m_new > m_ref + 8.f);
+      if (rescale) {
+        // P V of the previous tile has completed (the commit behind these scores covers it)
+        const float f = ex2(m_ref - m_new);
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          float o[32];
+          tmem_ld32(tO + 32 * c, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o[e] *= f;
+          tmem_st32(tO + 32 * c, o);
+        }
+        l *= f;
+        m_ref = m_new;
+      }
+      // pass 2: weights, written back (fp16, two per column) over score columns already consumed
+      float psum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float x[32];
+        tmem_ld32(tS + 32 * c, x);
+        tmem_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const int j = 32 * c + 2 * e;
+          const bool ok0 = !((diag && j > r) || (bound && j < r));
+          const bool ok1 = !((diag && j + 1 > r) || (bound && j + 1 < r));
+          const float p0 = ok0 ? ex2(x[2 * e] * a.scale_log2 - m_ref) : 0.f;
+          const float p1 = ok1 ? ex2(x[2 * e + 1] * a.scale_log2 - m_ref) : 0.f;
+          psum += p0 + p1;
+          pk[e] = pack_f16(p0, p1);
+        }
+        tmem_st16(tS + 16 * c, pk);
+      }
+      l += psum;
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bars->p_ready[X]);
+    }
+
+    // ---- park the normalised window output (Section 3.2, first norm) in registers ---------
+    WAIT_OR_RETURN(bars->o_ready[X], cntO & 1);
+    ++cntO;
+    tc_fence_after();
+    const float inv_l = 1.f / l;
+    uint32_t stash[64];
+    float ss = 0.f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      float o[32];
+      tmem_ld32(tO + 32 * c, o);
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 32; ++e) ss += o[e] * o[e];
+    }
+    const float ms = ss * inv_l * inv_l * (1.f / 128.f) + a.eps;     // mean square of o_swa, plus eps
+    const float rs = rsqrtf(ms);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      float o[32];
+      tmem_ld32(tO + 32 * c, o);
+      tmem_wait_ld();
+#pragma unroll
+      for (int e = 0; e < 16; ++e) stash[16 * c + e] = pack_f16(o[2 * e] * inv_l * rs, o[2 * e + 1] * inv_l * rs);
+    }
+    float rr = 0.f, sr = 0.f, inv_q = 1.f;
+
+    // ---- residual branch ------------------------------------------------------------------
+    if (un.rla[X]) {
+      tc_fence_before();
+      mbar_arrive(&bars->stash_done[X]);
+      // phi(Q_X) without its normalisation: everything that follows is linear in this row,
+      // so 1/sum is applied to the accumulator row at the end
+      inv_q = feature_map_row_unnorm_inplace(sQ, r);                   // every Q_X K^T has completed
+      fence_proxy_async_smem();
+      mbar_arrive(&bars->phiq_ready[X]);
+      // this tile's own chunk: A -> last stream position, B -> its last active position
+      const int ic = (X == 0) ? un.n - 1 : un.i1[1];
+      feature_map_row_inplace_lr(smem + F_OFF_KV + ((kv0 + ic) & 1) * 2 * TILE_BYTES, r);
+      fence_proxy_async_smem();
+      mbar_arrive(&bars->phik_ready[X]);
+      const int n_terms = (X == 1 && un.rla[0]) ? 2 : 1;
+      for (int term = 0; term < n_terms; ++term) {
+        const bool masked = (term == n_terms - 1);                     // B's first term takes chunk cA whole
+        WAIT_OR_RETURN(bars->s_full[X], cntS & 1);
+        ++cntS;
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          float x[32];
+          tmem_ld32(tS + 32 * c, x);
+          tmem_wait_ld();
+          uint32_t pk[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const int j = 32 * c + 2 * e;                              // residual keys of row r in its chunk: j < r
+            const float p0 = (!masked || j < r) ? x[2 * e] : 0.f;
+            const float p1 = (!masked || j + 1 < r) ? x[2 * e + 1] : 0.f;
+            pk[e] = pack_f16(p0, p1);
+          }
+          tmem_st16(tS + 16 * c, pk);                                  // columns already consumed
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&bars->p_ready[X]);
+      }
+      WAIT_OR_RETURN(bars->o_ready[X], cntO & 1);
+      ++cntO;
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float o[32];
+        tmem_ld32(tO + 32 * c, o);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) sr += o[e] * o[e];
+      }
+      rr = inv_q * rsqrtf(sr * inv_q * inv_q * (1.f / 128.f) + a.eps);     // o_rla = inv_q * accumulator
+    }
+
+    // ---- Section 3.2: gains, sum; outputs leave through the tile's Q buffer ---------------
+    const size_t tile_row0 = (size_t)un.bh_q * a.T + q0;
+    const float rms_s = ms * rs;                                       // sqrt(mean square + eps)
+    if (a.o_swa) {
+      // training mode: un-normalised branch outputs (fp32), 32 columns at a time, staged so
+      // that each warp writes whole 128-byte segments of its own 32 rows
+      unsigned char* stage = sQ;
+      if (un.rla[X]) group_sync(X);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float x[32];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&stash[16 * c + e]));
+          x[2 * e] = f.x * rms_s;
+          x[2 * e + 1] = f.y * rms_s;
+        }
+        __syncwarp();
+        stage_f32_block(stage, r, x);
+        __syncwarp();
+        flush_f32_block(stage, r, a.o_swa + tile_row0 * 128 + 32 * c, a.T - q0);
+        if (un.rla[X]) {
+          tmem_ld32(tO + 32 * c, x);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) x[e] *= inv_q;
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) x[e] = 0.f;
+        }
+        __syncwarp();
+        stage_f32_block(stage, r, x);
+        __syncwarp();
+        flush_f32_block(stage, r, a.o_rla + tile_row0 * 128 + 32 * c, a.T - q0);
+      }
+      group_sync(X);
+    }
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {                                      // 16 columns at a time
+      float orl[16];
+      if (un.rla[X]) {
+        tmem_ld16(tO + 16 * c, orl);
+        tmem_wait_ld();
+      }
+      uint32_t yk[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&stash[8 * c + e]));
+        const int col = 16 * c + 2 * e;
+        float y0 = f.x, y1 = f.y;
+        if (a.gamma_swa) {
+          y0 *= __ldg(a.gamma_swa + (size_t)un.h * 128 + col);
+          y1 *= __ldg(a.gamma_swa + (size_t)un.h * 128 + col + 1);
+        }
+        if (un.rla[X]) {
+          float r0 = orl[2 * e] * rr, r1 = orl[2 * e + 1] * rr;
+          if (a.gamma_rla) {
+            r0 *= __ldg(a.gamma_rla + (size_t)un.h * 128 + col);
+            r1 *= __ldg(a.gamma_rla + (size_t)un.h * 128 + col + 1);
+          }
+          y0 += r0;
+          y1 += r1;
+        }
+        yk[e] = pack_bf16(y0, y1);
+      }
+      *reinterpret_cast<uint4*>(sQ + swz(r, 2 * c)) = make_uint4(yk[0], yk[1], yk[2], yk[3]);
+      *reinterpret_cast<uint4*>(sQ + swz(r, 2 * c + 1)) = make_uint4(yk[4], yk[5], yk[6], yk[7]);
+    }
+    if (t < a.T && a.lse) a.lse[(size_t)un.bh_q * a.T + t] = (m_ref + log2f(l)) * 0.6931471805599453f;
+    fence_proxy_async_smem();
+    tc_fence_before();
+    group_sync(X);
+    if (r == 0) {
+      store_tile(&tm.out, sQ, q0, un.bh_q);
+      tma_store_commit();
+      tma_store_wait_read();
+    }
+    group_sync(X);
+    mbar_arrive(&bars->q_free[X]);       // the Q buffer may be refilled
+    mbar_arrive(&bars->o_free[X]);       // the score and output columns may be overwritten
+  }
+  return true;
+}
+
+__global__ void __launch_bounds__(F_THREADS, 1)
+tc_fwd2_kernel(const __grid_constant__ FMaps tm, FArgs a) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  FBars* bars = reinterpret_cast<FBars*>(smem + F_OFF_BAR);
+  const int tid = threadIdx.x, warp = tid >> 5;
+  if ((smem_u32(smem) & 1023u) != 0) {
+    if (tid == 0 && a.status) atomicExch(a.status, 2);
+    return;
+  }
+  if (tid == 0) {
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bars->q_full[i], 1);
+      mbar_init(&bars->q_free[i], 128);
+      mbar_init(&bars->kv_full[i], 1);
+      mbar_init(&bars->v_ready[i], 64);
+      mbar_init(&bars->kv_free[i], 1);
+      mbar_init(&bars->s_full[i], 1);
+      mbar_init(&bars->p_ready[i], 128);
+      mbar_init(&bars->o_ready[i], 1);
+      mbar_init(&bars->stash_done[i], 128);
+      mbar_init(&bars->phiq_ready[i], 128);
+      mbar_init(&bars->phik_ready[i], 128);
+      mbar_init(&bars->o_free[i], 128);
+    }
+    mbar_init(&bars->x_full, 1);
+    mbar_init(&bars->x_free, 1);
+    mbar_init(&bars->drain, 1);
+    bars->abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 8) {
+    tmem_alloc(&bars->tmem_base, 512);
+    tmem_relinquish();
+  }
+  if (tid == 288) {
+    prefetch_tensormap(&tm.q);
+    prefetch_tensormap(&tm.k);
+    prefetch_tensormap(&tm.v);
+    prefetch_tensormap(&tm.st);
+    prefetch_tensormap(&tm.out);
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_base;
+
+  bool ok = true;
+  if (warp < 8) {
+    ok = (warp < 4) ? fwd_rows<0>(tm, a, smem, bars, tmem, tid & 127) : fwd_rows<1>(tm, a, smem, bars, tmem, tid & 127);
+  } else if (warp == 8) {
+    ok = fwd_mma(a, smem, bars, tmem);
+    if (!ok) {
+      mma_commit(&bars->drain);
+      for (int it = 0; it < (1 << 16) && !mbar_try_wait(&bars->drain, 0); ++it) {}
+    }
+  } else if (warp == 9) {
+    ok = fwd_loader(tm, a, smem, bars);
+  } else {
+    ok = fwd_convert(a, smem, bars, tid - 320);
+  }
+  if (!ok && a.status) atomicExch(a.status, 1);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s) {
+  FMaps tm;
+  if (!make_map(&tm.q, a.q, a.T, (uint64_t)a.B * a.H_q) || !make_map(&tm.k, a.k, a.T, (uint64_t)a.B * a.H_kv) ||
+      !make_map(&tm.v, a.v, a.T, (uint64_t)a.B * a.H_kv) || !make_map(&tm.out, a.out, a.T, (uint64_t)a.B * a.H_q) ||
+      !make_map(&tm.st, a.chunk_state, 128, (uint64_t)a.B * a.H_kv * a.n_chunks))
+    return cudaErrorInvalidValue;
+  FArgs t;
+  t.lse = a.lse; t.o_swa = a.o_swa; t.o_rla = a.o_rla;
+  t.gamma_swa = a.gamma_swa; t.gamma_rla = a.gamma_rla; t.status = a.status;
+  t.T = a.T; t.w = a.w; t.H_q = a.H_q; t.group = a.group; t.mode = a.mode; t.n_chunks = a.n_chunks;
+  t.n_qt = (a.T + TILE - 1) / TILE;
+  t.n_pairs = (t.n_qt + 1) / 2;
+  t.n_bh = a.B * a.H_q;
+  t.n_units = t.n_pairs * t.n_bh;
+  t.scale_log2 = a.scale * LOG2E; t.eps = a.eps;
+  int dev = 0, n_sm = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(tc_fwd2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, F_SMEM);
+  if (e != cudaSuccess) return e;
+  const int grid = t.n_units < n_sm ? t.n_units : n_sm;
+  {
+    KernelTimer kt("tc_fwd", s);
+    tc_fwd2_kernel<<<grid, F_THREADS, F_SMEM, s>>>(tm, t);
+  }
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+}  // namespace rattn
