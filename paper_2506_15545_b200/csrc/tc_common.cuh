@@ -156,10 +156,12 @@ __device__ __forceinline__ void flush_f32_block(const unsigned char* stage, int 
   }
 }
 
+// The helpers below walk a row in sixteen 16-byte steps with a rolled loop: compact code
+// matters more than loop overhead here (large unrolled kernels are instruction-fetch bound).
 // Row maximum of row r of a swizzled bf16 tile.
 __device__ __forceinline__ float row_max_bf16(const unsigned char* tile, int r) {
   float m = -INFINITY;
-#pragma unroll
+#pragma unroll 1
   for (int c = 0; c < 16; ++c) {
     const uint4 u = *reinterpret_cast<const uint4*>(tile + swz(r, c));
     const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
@@ -171,12 +173,11 @@ __device__ __forceinline__ float row_max_bf16(const unsigned char* tile, int r) 
   }
   return m;
 }
-// Un-normalised feature map of row r, in place: x -> exp(x - max) (bf16); returns 1 / sum so
-// that the caller can scale whatever is linear in this row afterwards.  Few live registers.
-__device__ __forceinline__ float feature_map_row_unnorm_inplace(unsigned char* tile, int r) {
-  const float ml = row_max_bf16(tile, r) * 1.4426950408889634f;
+// x -> exp(x - max) over row r, in place, as fp16 (FP16 = true) or bf16; returns the row sum.
+template <bool FP16>
+__device__ __forceinline__ float row_exp_inplace(unsigned char* tile, int r, float ml) {
   float sum = 0.f;
-#pragma unroll
+#pragma unroll 1
   for (int c = 0; c < 16; ++c) {
     uint4 u = *reinterpret_cast<const uint4*>(tile + swz(r, c));
     uint32_t* w = reinterpret_cast<uint32_t*>(&u);
@@ -185,32 +186,24 @@ __device__ __forceinline__ float feature_map_row_unnorm_inplace(unsigned char* t
       const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
       const float e0 = ex2(f.x * 1.4426950408889634f - ml), e1 = ex2(f.y * 1.4426950408889634f - ml);
       sum += e0 + e1;
-      w[e] = pack_bf16(e0, e1);
+      w[e] = FP16 ? pack_f16(e0, e1) : pack_bf16(e0, e1);
     }
     *reinterpret_cast<uint4*>(tile + swz(r, c)) = u;
   }
-  return 1.f / sum;
+  return sum;
+}
+// Un-normalised feature map of row r, in place: x -> exp(x - max) (bf16); returns 1 / sum so
+// that the caller can scale whatever is linear in this row afterwards.
+__device__ __forceinline__ float feature_map_row_unnorm_inplace(unsigned char* tile, int r) {
+  const float ml = row_max_bf16(tile, r) * 1.4426950408889634f;
+  return 1.f / row_exp_inplace<false>(tile, r, ml);
 }
 // phi of row r, in place, with few live registers: the exponentials are parked in the tile
 // itself as fp16 between the summation and the normalisation (one bf16 rounding in the end).
 __device__ __forceinline__ void feature_map_row_inplace_lr(unsigned char* tile, int r) {
   const float ml = row_max_bf16(tile, r) * 1.4426950408889634f;
-  float sum = 0.f;
-#pragma unroll
-  for (int c = 0; c < 16; ++c) {
-    uint4 u = *reinterpret_cast<const uint4*>(tile + swz(r, c));
-    uint32_t* w = reinterpret_cast<uint32_t*>(&u);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
-      const float e0 = ex2(f.x * 1.4426950408889634f - ml), e1 = ex2(f.y * 1.4426950408889634f - ml);
-      sum += e0 + e1;
-      w[e] = pack_f16(e0, e1);
-    }
-    *reinterpret_cast<uint4*>(tile + swz(r, c)) = u;
-  }
-  const float inv = 1.f / sum;
-#pragma unroll
+  const float inv = 1.f / row_exp_inplace<true>(tile, r, ml);
+#pragma unroll 1
   for (int c = 0; c < 16; ++c) {
     uint4 u = *reinterpret_cast<const uint4*>(tile + swz(r, c));
     uint32_t* w = reinterpret_cast<uint32_t*>(&u);

@@ -290,8 +290,20 @@ __device__ bool fwd_mma(const FArgs& a, unsigned char* smem, FBars* bars, uint32
 // ------------------------------------------------------------------------------ row groups
 __device__ __forceinline__ uint32_t lane_base(int r) { return (uint32_t)((r & ~31) << 16); }
 
-template <int X>
-__device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, FBars* bars, uint32_t tmem, int r) {
+// Bit e of the result says whether column 32*c + e of a [128 x 128] score tile is kept for row
+// r: on the diagonal tile the keys j <= r, on the oldest tile of the band the keys j >= r.
+__device__ __forceinline__ uint32_t keep_bits(int r, int c, bool diag, bool bound) {
+  const int rd = r - 32 * c;                       // column of the row's own position in this chunk
+  uint32_t m = 0xffffffffu;
+  if (diag) m &= rd >= 31 ? 0xffffffffu : (rd < 0 ? 0u : ((2u << rd) - 1u));
+  if (bound) m &= rd <= 0 ? 0xffffffffu : (rd > 31 ? 0u : ~((1u << rd) - 1u));
+  return m;
+}
+
+// The per-tile loops below are rolled over 32-column chunks on purpose: with everything
+// unrolled the kernel was ~390 KB of code and ran instruction-fetch bound.
+__device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, FBars* bars, uint32_t tmem, int X,
+                         int r) {
   const uint32_t tS = tmem + 128 * X + lane_base(r), tO = tmem + 256 + 128 * X + lane_base(r);
   unsigned char* sQ = smem + F_OFF_Q + X * TILE_BYTES;
   int kv_count = 0, cntS = 0, cntO = 0;
@@ -300,37 +312,37 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     const Unit un = make_unit(a, u);
     const int kv0 = kv_count;
     kv_count += un.n;
-    if (un.t[X] < 0) continue;
-    const int q0 = un.t[X] * TILE;
+    const int tX = X ? un.t[1] : un.t[0], i0 = X ? un.i0[1] : un.i0[0], i1 = X ? un.i1[1] : un.i1[0];
+    const bool rlaX = X ? un.rla[1] : un.rla[0];
+    if (tX < 0) continue;
+    const int q0 = tX * TILE;
     const int t = q0 + r;
 
     // ---- window branch: online softmax over the key tiles of the band -------------------
     float m_ref = -INFINITY, l = 0.f;
-    for (int i = un.i0[X]; i <= un.i1[X]; ++i) {
+#pragma unroll 1
+    for (int i = i0; i <= i1; ++i) {
       const int kt = un.kt_hi - i;
       WAIT_OR_RETURN(bars->s_full[X], cntS & 1);
       ++cntS;
       tc_fence_after();
-      const bool diag = (kt == un.t[X]), bound = un.windowed && (kt == un.t[X] - un.wt);
-      // pass 1 over the scores: row maximum (32 columns at a time keeps the register count low)
+      const bool diag = (kt == tX), bound = un.windowed && (kt == tX - un.wt);
+      // pass 1 over the scores: row maximum
       float mx = -INFINITY;
-#pragma unroll
+#pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         float x[32];
         tmem_ld32(tS + 32 * c, x);
         tmem_wait_ld();
+        const uint32_t keep = keep_bits(r, c, diag, bound);
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int j = 32 * c + e;
-          const bool ok = !((diag && j > r) || (bound && j < r));
-          mx = fmaxf(mx, ok ? x[e] : -INFINITY);
-        }
+        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, (keep >> e) & 1u ? x[e] : -INFINITY);
       }
       mx *= a.scale_log2;                                              // scale > 0
       // lazy rescale: the reference maximum only moves when the row maximum grew by more than 2^8
       const float m_new = fmaxf(m_ref, mx);
       bool rescale = false;
-      if (i == un.i0[X]) m_ref = m_new;
+      if (i == i0) m_ref = m_new;
       else rescale = __any_sync(0xffffffffu, m_new > m_ref + 8.f);
       if (rescale) {
         // P V of the previous tile has completed (the commit behind these scores covers it)
@@ -349,19 +361,17 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
       }
       // pass 2: weights, written back (fp16, two per column) over score columns already consumed
       float psum = 0.f;
-#pragma unroll
+#pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         float x[32];
         tmem_ld32(tS + 32 * c, x);
         tmem_wait_ld();
+        const uint32_t keep = keep_bits(r, c, diag, bound);
         uint32_t pk[16];
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
-          const int j = 32 * c + 2 * e;
-          const bool ok0 = !((diag && j > r) || (bound && j < r));
-          const bool ok1 = !((diag && j + 1 > r) || (bound && j + 1 < r));
-          const float p0 = ok0 ? ex2(x[2 * e] * a.scale_log2 - m_ref) : 0.f;
-          const float p1 = ok1 ? ex2(x[2 * e + 1] * a.scale_log2 - m_ref) : 0.f;
+          const float p0 = (keep >> (2 * e)) & 1u ? ex2(x[2 * e] * a.scale_log2 - m_ref) : 0.f;
+          const float p1 = (keep >> (2 * e + 1)) & 1u ? ex2(x[2 * e + 1] * a.scale_log2 - m_ref) : 0.f;
           psum += p0 + p1;
           pk[e] = pack_f16(p0, p1);
         }
@@ -380,7 +390,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     const float inv_l = 1.f / l;
     uint32_t stash[64];
     float ss = 0.f;
-#pragma unroll
+#pragma unroll 1
     for (int c = 0; c < 4; ++c) {
       float o[32];
       tmem_ld32(tO + 32 * c, o);
@@ -401,7 +411,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     float rr = 0.f, sr = 0.f, inv_q = 1.f;
 
     // ---- residual branch ------------------------------------------------------------------
-    if (un.rla[X]) {
+    if (rlaX) {
       tc_fence_before();
       mbar_arrive(&bars->stash_done[X]);
       // phi(Q_X) without its normalisation: everything that follows is linear in this row,
@@ -415,24 +425,24 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
       fence_proxy_async_smem();
       mbar_arrive(&bars->phik_ready[X]);
       const int n_terms = (X == 1 && un.rla[0]) ? 2 : 1;
+#pragma unroll 1
       for (int term = 0; term < n_terms; ++term) {
         const bool masked = (term == n_terms - 1);                     // B's first term takes chunk cA whole
         WAIT_OR_RETURN(bars->s_full[X], cntS & 1);
         ++cntS;
         tc_fence_after();
-#pragma unroll
+#pragma unroll 1
         for (int c = 0; c < 4; ++c) {
           float x[32];
           tmem_ld32(tS + 32 * c, x);
           tmem_wait_ld();
+          // residual keys of row r in its chunk: j < r
+          const int rd = r - 32 * c;
+          const uint32_t keep = !masked ? 0xffffffffu : (rd >= 32 ? 0xffffffffu : (rd <= 0 ? 0u : ((1u << rd) - 1u)));
           uint32_t pk[16];
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const int j = 32 * c + 2 * e;                              // residual keys of row r in its chunk: j < r
-            const float p0 = (!masked || j < r) ? x[2 * e] : 0.f;
-            const float p1 = (!masked || j + 1 < r) ? x[2 * e + 1] : 0.f;
-            pk[e] = pack_f16(p0, p1);
-          }
+          for (int e = 0; e < 16; ++e)
+            pk[e] = pack_f16((keep >> (2 * e)) & 1u ? x[2 * e] : 0.f, (keep >> (2 * e + 1)) & 1u ? x[2 * e + 1] : 0.f);
           tmem_st16(tS + 16 * c, pk);                                  // columns already consumed
         }
         tmem_wait_st();
@@ -442,7 +452,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
       WAIT_OR_RETURN(bars->o_ready[X], cntO & 1);
       ++cntO;
       tc_fence_after();
-#pragma unroll
+#pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         float o[32];
         tmem_ld32(tO + 32 * c, o);
@@ -460,7 +470,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
       // training mode: un-normalised branch outputs (fp32), 32 columns at a time, staged so
       // that each warp writes whole 128-byte segments of its own 32 rows
       unsigned char* stage = sQ;
-      if (un.rla[X]) group_sync(X);
+      if (rlaX) group_sync(X);
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         float x[32];
@@ -474,7 +484,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
         stage_f32_block(stage, r, x);
         __syncwarp();
         flush_f32_block(stage, r, a.o_swa + tile_row0 * 128 + 32 * c, a.T - q0);
-        if (un.rla[X]) {
+        if (rlaX) {
           tmem_ld32(tO + 32 * c, x);
           tmem_wait_ld();
 #pragma unroll
@@ -490,10 +500,12 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
       }
       group_sync(X);
     }
+    const float* gs = a.gamma_swa ? a.gamma_swa + (size_t)un.h * 128 : nullptr;
+    const float* gr = a.gamma_rla ? a.gamma_rla + (size_t)un.h * 128 : nullptr;
 #pragma unroll
     for (int c = 0; c < 8; ++c) {                                      // 16 columns at a time
       float orl[16];
-      if (un.rla[X]) {
+      if (rlaX) {
         tmem_ld16(tO + 16 * c, orl);
         tmem_wait_ld();
       }
@@ -503,15 +515,15 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
         const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&stash[8 * c + e]));
         const int col = 16 * c + 2 * e;
         float y0 = f.x, y1 = f.y;
-        if (a.gamma_swa) {
-          y0 *= __ldg(a.gamma_swa + (size_t)un.h * 128 + col);
-          y1 *= __ldg(a.gamma_swa + (size_t)un.h * 128 + col + 1);
+        if (gs) {
+          y0 *= __ldg(gs + col);
+          y1 *= __ldg(gs + col + 1);
         }
-        if (un.rla[X]) {
+        if (rlaX) {
           float r0 = orl[2 * e] * rr, r1 = orl[2 * e + 1] * rr;
-          if (a.gamma_rla) {
-            r0 *= __ldg(a.gamma_rla + (size_t)un.h * 128 + col);
-            r1 *= __ldg(a.gamma_rla + (size_t)un.h * 128 + col + 1);
+          if (gr) {
+            r0 *= __ldg(gr + col);
+            r1 *= __ldg(gr + col + 1);
           }
           y0 += r0;
           y1 += r1;
@@ -585,7 +597,7 @@ tc_fwd2_kernel(const __grid_constant__ FMaps tm, FArgs a) {
 
   bool ok = true;
   if (warp < 8) {
-    ok = (warp < 4) ? fwd_rows<0>(tm, a, smem, bars, tmem, tid & 127) : fwd_rows<1>(tm, a, smem, bars, tmem, tid & 127);
+    ok = fwd_rows(tm, a, smem, bars, tmem, warp >> 2, tid & 127);
   } else if (warp == 8) {
     ok = fwd_mma(a, smem, bars, tmem);
     if (!ok) {
