@@ -336,27 +336,25 @@ __device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned cha
   const bool live = t < a.T;
   const size_t row = (size_t)bh_q * a.T + t;
   const float l2 = live ? a.lse[row] * LOG2E : INFINITY;
-  const float Dr = live ? a.delta[row] : 0.f;
+  const float Drs = live ? a.delta[row] * a.scale : 0.f;
 
   for (int i = 0; i < n_kt; ++i) {
     WAIT_OR_RETURN(bars->s_full, i & 1);
     tc_fence_after();
     const bool diag = (i == 0), bound = has_boundary && (i == n_kt - 1);
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {                              // rolled: compact code
       float s[32], dp[32];
       tmem_ld32(tS + 32 * c, s);
       tmem_ld32(tP + 32 * c, dp);
       tmem_wait_ld();
+      const uint32_t keep = keep_bits(r, c, diag, bound);
       uint32_t pk[16];
 #pragma unroll
       for (int e = 0; e < 32; e += 2) {
-        const int j = 32 * c + e;
         const float p0 = ex2(s[e] * a.scale_log2 - l2), p1 = ex2(s[e + 1] * a.scale_log2 - l2);
-        const bool ok0 = !((diag && j > r) || (bound && j < r));
-        const bool ok1 = !((diag && j + 1 > r) || (bound && j + 1 < r));
-        const float d0 = ok0 ? p0 * (dp[e] - Dr) * a.scale : 0.f;
-        const float d1 = ok1 ? p1 * (dp[e + 1] - Dr) * a.scale : 0.f;
+        const float d0 = (keep >> e) & 1u ? p0 * (dp[e] * a.scale - Drs) : 0.f;
+        const float d1 = (keep >> (e + 1)) & 1u ? p1 * (dp[e + 1] * a.scale - Drs) : 0.f;
         pk[e >> 1] = pack_bf16(d0, d1);
       }
       // dS (bf16, two per column) overwrites the S columns already consumed: 16c..16c+15 < 32c+32
@@ -370,22 +368,21 @@ __device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned cha
   if (has_rla) {
     const int last = (n_kt - 1) & 1;
     WAIT_OR_RETURN(bars->dq_done, (n_kt - 1) & 1);           // K_cb is no longer read raw
-    feature_map_row_inplace(smem + DQ_OFF_K + last * TILE_BYTES, r);
+    feature_map_row_inplace_lr(smem + DQ_OFF_K + last * TILE_BYTES, r);
     fence_proxy_async_smem();
     mbar_arrive(&bars->phik_ready);
     WAIT_OR_RETURN(bars->s_full, n_kt & 1);
     tc_fence_after();
-#pragma unroll
+#pragma unroll 1
     for (int c = 0; c < 4; ++c) {
       float x[32];
       tmem_ld32(tS + 32 * c, x);
       tmem_wait_ld();
+      const uint32_t keep = bits_lt(r - 32 * c);               // residual keys of row r in this chunk: j < r
       uint32_t pk[16];
 #pragma unroll
-      for (int e = 0; e < 32; e += 2) {
-        const int j = 32 * c + e;                            // residual keys of row r in this chunk: j < r
-        pk[e >> 1] = pack_bf16(j < r ? x[e] : 0.f, j + 1 < r ? x[e + 1] : 0.f);
-      }
+      for (int e = 0; e < 32; e += 2)
+        pk[e >> 1] = pack_bf16((keep >> e) & 1u ? x[e] : 0.f, (keep >> (e + 1)) & 1u ? x[e + 1] : 0.f);
       tmem_st16(tS + 16 * c, pk);
     }
     tmem_wait_st();
@@ -712,21 +709,25 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
     const bool diag = !is_r && (i == pl.j), bound = !is_r && pl.windowed && (i == pl.j + pl.wt);
     const float* l2 = reinterpret_cast<const float*>(smem + KV_OFF_STAT + st * 512);
     const float* Ds = l2 + 64;
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
+#pragma unroll 1
+    for (int c = 0; c < 2; ++c) {                              // rolled: compact code
       float s[32], dp[32];
       tmem_ld32(tS + 32 * c, s);
       tmem_ld32(tP + 32 * c, dp);
       tmem_wait_ld();
+      const int rd = r - (64 * hf + 32 * c);                   // key row relative to this chunk's first query
       uint32_t pk1[16], pk2[16];
       if (is_r) {
+        const uint32_t keep = bits_gt(rd);                     // keep key r < query q
 #pragma unroll
         for (int e = 0; e < 32; e += 2) {
-          const int q = 64 * hf + 32 * c + e;              // query row inside its tile; keep key r < query q
-          pk1[e >> 1] = pack_bf16(q > r ? s[e] : 0.f, q + 1 > r ? s[e + 1] : 0.f);
-          pk2[e >> 1] = pack_bf16(q > r ? dp[e] : 0.f, q + 1 > r ? dp[e + 1] : 0.f);
+          const bool k0 = (keep >> e) & 1u, k1 = (keep >> (e + 1)) & 1u;
+          pk1[e >> 1] = pack_bf16(k0 ? s[e] : 0.f, k1 ? s[e + 1] : 0.f);
+          pk2[e >> 1] = pack_bf16(k0 ? dp[e] : 0.f, k1 ? dp[e + 1] : 0.f);
         }
       } else {
+        // diagonal tile: queries q >= r; oldest tile of the band: queries q <= r
+        const uint32_t keep = (diag ? bits_ge(rd) : 0xffffffffu) & (bound ? bits_le(rd) : 0xffffffffu);
 #pragma unroll
         for (int e4 = 0; e4 < 32; e4 += 4) {
           const float4 lv = *reinterpret_cast<const float4*>(l2 + 32 * c + e4);
@@ -735,8 +736,7 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
           float p[4], d[4];
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
-            const int q = 64 * hf + 32 * c + e4 + u;
-            const bool ok = !((diag && q < r) || (bound && q > r));
+            const bool ok = (keep >> (e4 + u)) & 1u;
             const float pv = ex2(s[e4 + u] * a.scale_log2 - lq[u]);
             p[u] = ok ? pv : 0.f;
             d[u] = ok ? pv * (dp[e4 + u] * a.scale - dq4[u]) : 0.f;

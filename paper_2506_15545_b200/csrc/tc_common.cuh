@@ -156,6 +156,22 @@ __device__ __forceinline__ void flush_f32_block(const unsigned char* stage, int 
   }
 }
 
+// Bit e of the result says whether column 32*c + e of a [128 x 128] score tile is kept for row
+// r: on the diagonal tile the keys j <= r, on the oldest tile of the band the keys j >= r.
+__device__ __forceinline__ uint32_t keep_bits(int r, int c, bool diag, bool bound) {
+  const int rd = r - 32 * c;                      // column of the row's own position in this chunk
+  uint32_t m = 0xffffffffu;
+  if (diag) m &= rd >= 31 ? 0xffffffffu : (rd < 0 ? 0u : ((2u << rd) - 1u));
+  if (bound) m &= rd <= 0 ? 0xffffffffu : (rd > 31 ? 0u : ~((1u << rd) - 1u));
+  return m;
+}
+
+// bits e >= rd, e > rd, e <= rd of a 32-bit chunk mask (any integer rd)
+__device__ __forceinline__ uint32_t bits_ge(int rd) { return rd <= 0 ? 0xffffffffu : (rd > 31 ? 0u : ~((1u << rd) - 1u)); }
+__device__ __forceinline__ uint32_t bits_gt(int rd) { return bits_ge(rd + 1); }
+__device__ __forceinline__ uint32_t bits_le(int rd) { return ~bits_gt(rd); }
+__device__ __forceinline__ uint32_t bits_lt(int rd) { return ~bits_ge(rd); }
+
 // The helpers below walk a row in sixteen 16-byte steps with a rolled loop: compact code
 // matters more than loop overhead here (large unrolled kernels are instruction-fetch bound).
 // Row maximum of row r of a swizzled bf16 tile.

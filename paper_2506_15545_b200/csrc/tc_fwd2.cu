@@ -290,16 +290,6 @@ __device__ bool fwd_mma(const FArgs& a, unsigned char* smem, FBars* bars, uint32
 // ------------------------------------------------------------------------------ row groups
 __device__ __forceinline__ uint32_t lane_base(int r) { return (uint32_t)((r & ~31) << 16); }
 
-// Bit e of the result says whether column 32*c + e of a [128 x 128] score tile is kept for row
-// r: on the diagonal tile the keys j <= r, on the oldest tile of the band the keys j >= r.
-__device__ __forceinline__ uint32_t keep_bits(int r, int c, bool diag, bool bound) {
-  const int rd = r - 32 * c;                       // column of the row's own position in this chunk
-  uint32_t m = 0xffffffffu;
-  if (diag) m &= rd >= 31 ? 0xffffffffu : (rd < 0 ? 0u : ((2u << rd) - 1u));
-  if (bound) m &= rd <= 0 ? 0xffffffffu : (rd > 31 ? 0u : ~((1u << rd) - 1u));
-  return m;
-}
-
 // The per-tile loops below are rolled over 32-column chunks on purpose: with everything
 // unrolled the kernel was ~390 KB of code and ran instruction-fetch bound.
 __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, FBars* bars, uint32_t tmem, int X,
