@@ -261,7 +261,8 @@ def run_ours(args, wl):
     share = {n: tot for n, (cnt, tot) in kernel_ms.items()}
     top = max(share, key=share.get)
     kflops = {"tc_fwd": "fwd_main", "tc_chunk_delta": "fwd_state", "generic_fwd": "fwd",
-              "generic_bwd_dq": "bwd_dq", "generic_bwd_dkv": "bwd_dkv"}
+              "generic_bwd_dq": "bwd_dq", "generic_bwd_dkv": "bwd_dkv",
+              "tc_bwd_dq": "bwd_dq", "tc_bwd_dkv": "bwd_dkv"}
     roof = None
     if top in kflops:
         ach = flops(wl, kflops[top]) / (per_launch[top] * 1e-3) / 1e12
