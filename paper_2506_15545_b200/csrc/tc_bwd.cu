@@ -575,7 +575,7 @@ constexpr int KV_OFF_STAGE = 3 * TILE_BYTES;               // KV_NS x [Q_h 16 KB
 constexpr int KV_OFF_STAT = KV_OFF_STAGE + KV_NS * TILE_BYTES;   // KV_NS x (lse2[64], D*scale[64]) fp32
 constexpr int KV_OFF_BAR = KV_OFF_STAT + KV_NS * 512;
 constexpr int KV_SMEM = KV_OFF_BAR + 256;
-constexpr int KV_THREADS = 320;                            // 2 row groups, MMA warp, loader warp
+constexpr int KV_THREADS = 576;                            // 4 row groups, MMA warp, loader warp
 
 struct KvBars {
   uint64_t kv_full, kphi_ready, full[KV_NS], acc_done[KV_NS], s_full[2], p_ready[2], phiq_ready[2],
@@ -676,16 +676,20 @@ __device__ bool kv_mma(unsigned char* smem, KvBars* bars, uint32_t tmem, const K
 }
 
 __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtensorMap* tm_dv, unsigned char* smem,
-                        KvBars* bars, uint32_t tmem, const KvPlan& pl, int g, int r, int bh_kv) {
+                        KvBars* bars, uint32_t tmem, const KvPlan& pl, int gg, int r, int bh_kv) {
+  // four groups of 128 threads (thread = key row = TMEM lane): groups 0,1 serve TMEM slot 0,
+  // groups 2,3 slot 1; within a slot the even group takes query columns 0..31 of the item,
+  // the odd group columns 32..63
+  const int g = gg >> 1, c = gg & 1;
   const uint32_t lane_off = (uint32_t)((r & ~31) << 16);
   const uint32_t tV = tmem + lane_off, tK = tmem + 128 + lane_off;
   const uint32_t tS = tmem + 256 + 128 * g + lane_off, tP = tS + 64;
   const unsigned char* sKphi = smem + KV_OFF_KPHI;
 
   WAIT_OR_RETURN(bars->kv_full, 0);
-  if (pl.n_R > 0) {
+  if (pl.n_R > 0 && gg < 2) {
     // phi(K_j) into its own tile: 256 threads, two per row
-    const int t2 = g * 128 + r, row = t2 >> 1, hf = t2 & 1;
+    const int t2 = gg * 128 + r, row = t2 >> 1, hf = t2 & 1;
     feature_map_pair(smem + KV_OFF_K + hf * HALF_BYTES, smem + KV_OFF_KPHI + hf * HALF_BYTES, row);
     fence_proxy_async_smem();
     mbar_arrive(&bars->kphi_ready);
@@ -697,8 +701,8 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
     const int i = pl.qtile(n), hf = pl.half(n);
     unsigned char* sQh = smem + KV_OFF_STAGE + st * TILE_BYTES;
     WAIT_OR_RETURN(bars->full[st], pl.use(n) & 1);
-    if (is_r) {
-      // phi(Q_h) in place: 64 rows, two threads per row
+    if (is_r && c == 0) {
+      // phi(Q_h) in place: 64 rows, two threads per row (the slot's even group)
       const int row = r >> 1, ch = r & 1;
       feature_map_pair(sQh + ch * HT_HALF, sQh + ch * HT_HALF, row);
       fence_proxy_async_smem();
@@ -709,8 +713,7 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
     const bool diag = !is_r && (i == pl.j), bound = !is_r && pl.windowed && (i == pl.j + pl.wt);
     const float* l2 = reinterpret_cast<const float*>(smem + KV_OFF_STAT + st * 512);
     const float* Ds = l2 + 64;
-#pragma unroll 1
-    for (int c = 0; c < 2; ++c) {                              // rolled: compact code
+    {
       float s[32], dp[32];
       tmem_ld32(tS + 32 * c, s);
       tmem_ld32(tP + 32 * c, dp);
@@ -747,15 +750,15 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
           pk2[(e4 >> 1) + 1] = pack_bf16(d[2], d[3]);
         }
       }
-      // bf16 results (two per column) overwrite columns of S^T / dP^T that have been consumed
-      tmem_st16(tS + 16 * c, pk1);
-      tmem_st16(tP + 16 * c, pk2);
+      // bf16 results (two per column) overwrite the first half of this group's own columns
+      tmem_st16(tS + 32 * c, pk1);
+      tmem_st16(tP + 32 * c, pk2);
     }
     tmem_wait_st();
     tc_fence_before();
     mbar_arrive(&bars->p_ready[g]);
 
-    if (g == 0 && pl.n_R > 0 && n == pl.n_R - 2) {
+    if (gg == 0 && pl.n_R > 0 && n == pl.n_R - 2) {
       // end of the residual items: dK := phi(k) (dphi_k - <dphi_k, phi(k)>)
       WAIT_OR_RETURN(bars->r_acc_done, 0);
       tc_fence_after();
@@ -800,12 +803,13 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
     }
   }
 
-  // every product has completed: row group 0 stores dK, row group 1 dV, each staged in one of
+  // every product has completed: group 0 stores dK, group 1 dV, each staged in one of
   // the (now free) item stages and written by one TMA store
+  if (gg >= 2) return true;
   WAIT_OR_RETURN(bars->all_done, 0);
   tc_fence_after();
-  unsigned char* sOut = smem + KV_OFF_STAGE + g * TILE_BYTES;
-  const uint32_t tOut = g == 0 ? tK : tV;
+  unsigned char* sOut = smem + KV_OFF_STAGE + gg * TILE_BYTES;
+  const uint32_t tOut = gg == 0 ? tK : tV;
 #pragma unroll 1
   for (int c = 0; c < 4; ++c) {
     float x[32];
@@ -822,9 +826,9 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
     }
   }
   fence_proxy_async_smem();
-  group_sync(g);
+  group_sync(gg);
   if (r == 0) {
-    store_tile(g == 0 ? tm_dk : tm_dv, sOut, pl.j * TILE, bh_kv);
+    store_tile(gg == 0 ? tm_dk : tm_dv, sOut, pl.j * TILE, bh_kv);
     tma_store_commit();
     tma_store_wait_read();
   }
@@ -870,7 +874,7 @@ tc_bwd_dkv_kernel(const __grid_constant__ KvMaps tm, BwdArgs a) {
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bars->s_full[i], 1);
-      mbar_init(&bars->p_ready[i], 128);
+      mbar_init(&bars->p_ready[i], 256);
       mbar_init(&bars->phiq_ready[i], 128);
     }
     mbar_init(&bars->r_acc_done, 1);
@@ -880,11 +884,11 @@ tc_bwd_dkv_kernel(const __grid_constant__ KvMaps tm, BwdArgs a) {
     bars->abort = 0;
     fence_mbar_init();
   }
-  if (warp == 8) {
+  if (warp == 16) {
     tmem_alloc(&bars->tmem_base, 512);
     tmem_relinquish();
   }
-  if (tid == 288) {
+  if (tid == 544) {
     prefetch_tensormap(&tm.k);
     prefetch_tensormap(&tm.v);
     prefetch_tensormap(&tm.rs);
@@ -898,22 +902,22 @@ tc_bwd_dkv_kernel(const __grid_constant__ KvMaps tm, BwdArgs a) {
   const uint32_t tmem = bars->tmem_base;
 
   bool ok = true;
-  if (warp < 8) {
+  if (warp < 16) {
     ok = kv_rows(a, &tm.dk, &tm.dv, smem, bars, tmem, pl, warp >> 2, tid & 127, bh_kv);
-  } else if (warp == 8) {
+  } else if (warp == 16) {
     ok = kv_mma(smem, bars, tmem, pl);
     if (!ok) {
       mma_commit(&bars->drain);
       for (int it = 0; it < (1 << 16) && !mbar_try_wait(&bars->drain, 0); ++it) {}
     }
-  } else if (warp == 9) {
+  } else if (warp == 17) {
     ok = kv_loader(&tm.k, &tm.v, &tm.rs, &tm.qh, &tm.gsh, &tm.grh, a.lse2p, a.dscp, a.t_pad, smem, bars, pl,
                    bh_kv, rs_index);
   }
   if (!ok && a.status) atomicExch(a.status, 1);
   tc_fence_before();
   __syncthreads();
-  if (warp == 8) {
+  if (warp == 16) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
   }

@@ -68,12 +68,15 @@ __device__ __forceinline__ void mma_k_kh(uint32_t d, uint32_t a_base, uint32_t b
   for (int k = 0; k < 8; ++k)
     mma_bf16(d, a0 + kstep_k(k, HALF_BYTES), b0 + kstep_k(k, HT_HALF), idesc, k > 0 ? 1u : 0u);
 }
-// D[128 x 128] (+)= A[128 x 64] (bf16 in TMEM, 32 columns) . B[64 x 128] (MN-major half tile)
+// D[128 x 128] (+)= A[128 x 64] (bf16 in TMEM) . B[64 x 128] (MN-major half tile).  A sits where
+// the row groups left it: reduction elements 0..31 in columns 0..15 and 32..63 in columns
+// 32..47 of the slot (each group packs its 32 fp32 columns into the first 16 of them).
 __device__ __forceinline__ void mma_ts_h(uint32_t d, uint32_t a_tmem, uint32_t b_base, bool acc) {
   constexpr uint32_t idesc = instr_desc(128, 128, 0, 1);
   const uint64_t b0 = mnmajor_base_h(b_base);
 #pragma unroll
-  for (int k = 0; k < 4; ++k) mma_bf16_ts(d, a_tmem + 8 * k, b0 + kstep_mn(k), idesc, (acc || k > 0) ? 1u : 0u);
+  for (int k = 0; k < 4; ++k)
+    mma_bf16_ts(d, a_tmem + (k < 2 ? 8 * k : 32 + 8 * (k - 2)), b0 + kstep_mn(k), idesc, (acc || k > 0) ? 1u : 0u);
 }
 __device__ __forceinline__ void load_tile(unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int row, int z) {
   tma_load_3d(dst, tm, bar, 0, row, z);
