@@ -19,7 +19,7 @@ BUILD = os.path.join(ROOT, "_build")
 LIB = os.path.join(HERE, "librattn.so")
 
 SOURCES = ["rattn_api.cu", "generic_fwd.cu", "generic_bwd.cu", "decode.cu", "tc_fwd.cu",
-           "tc_fwd2.cu", "tc_bwd.cu", "static_scratch.cu"]
+           "tc_fwd2.cu", "tc_state.cu", "tc_bwd.cu", "static_scratch.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC",
               "-I" + os.path.join(ROOT, "include"), "-I" + CSRC]

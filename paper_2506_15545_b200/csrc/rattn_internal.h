@@ -79,6 +79,11 @@ cudaError_t launch_decode(const Args& a, void* k_ring, void* v_ring, float* stat
 cudaError_t launch_handoff(const Args& a, cudaStream_t s);
 cudaError_t launch_tc_forward(const Args& a, cudaStream_t s);        // chunk states, then the main kernel
 cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s);
+// running sums of phi(X_c)^T Y_c over the chunks first, first+dir, ... (n_steps of them), the sum
+// after step s written to matrix out_first + dir*s of each K/V head; `name` labels the timing record
+cudaError_t launch_tc_states(const void* x, const void* y, void* out, int T, int n_kv, int group, int n_chunks,
+                             int n_steps, int first, int dir, int out_first, int* status, const char* name,
+                             cudaStream_t s);
 cudaError_t launch_tc_backward(const Args& a, cudaStream_t s);
 
 void count_launches(int n);

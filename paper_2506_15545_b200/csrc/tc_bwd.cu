@@ -158,98 +158,6 @@ tc_bwd_prep_kernel(const __nv_bfloat16* __restrict__ dy, const float* __restrict
   if (dgamma_s || dgamma_r) flush();
 }
 
-// --------------------------------------------------------------- reverse chunk states
-// delta[kv][c] = sum over the group's query heads of phi(Q_c)^T G_c  (fp32, 128 x 128),
-// for c = chunk0 + blockIdx.x.
-constexpr int RD_SMEM = 2 * TILE_BYTES + 64;
-
-__global__ void __launch_bounds__(128)
-tc_bwd_rdelta_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_g,
-                     float* __restrict__ delta, int n_chunks, int chunk0, int group, int* status) {
-  extern __shared__ __align__(1024) unsigned char smem[];
-  struct Bars { uint64_t full, done; uint32_t tmem_base; int abort; };
-  Bars* bars = reinterpret_cast<Bars*>(smem + 2 * TILE_BYTES);
-  const int tid = threadIdx.x, warp = tid >> 5;
-  const int c = chunk0 + blockIdx.x, kv = blockIdx.y;
-  if ((smem_u32(smem) & 1023u) != 0) {       // the swizzled tile layout needs a 1024-byte aligned base
-    if (tid == 0 && status) atomicExch(status, 2);
-    return;
-  }
-  if (tid == 0) {
-    mbar_init(&bars->full, 1);
-    mbar_init(&bars->done, 1);
-    bars->abort = 0;
-    fence_mbar_init();
-  }
-  if (warp == 0) {
-    tmem_alloc(&bars->tmem_base, 128);
-    tmem_relinquish();
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = bars->tmem_base;
-  bool ok = true;
-  for (int hh = 0; hh < group; ++hh) {         // every thread runs every iteration (block-wide barriers inside)
-    const int z = kv * group + hh;
-    __syncwarp();
-    if (warp == 0 && !__any_sync(0xffffffffu, bars->abort != 0)) {
-      mbar_arrive_expect_tx(&bars->full, 2 * TILE_BYTES);
-      load_tile(smem, &tm_q, &bars->full, c * TILE, z);
-      load_tile(smem + TILE_BYTES, &tm_g, &bars->full, c * TILE, z);
-    }
-    ok = ok && mbar_wait(&bars->full, hh & 1, &bars->abort);
-    if (ok) {
-      feature_map_row_inplace(smem, tid);
-      fence_proxy_async_smem();
-    }
-    __syncthreads();
-    if (warp == 0 && !__any_sync(0xffffffffu, bars->abort != 0)) {
-      tc_fence_after();
-      mma_mnmn(tmem, smem_u32(smem), smem_u32(smem + TILE_BYTES), hh > 0);
-      mma_commit(&bars->done);
-    }
-    ok = ok && mbar_wait(&bars->done, hh & 1, &bars->abort);   // shared memory is reused by the next head
-  }
-  if (ok) {
-    tc_fence_after();
-    float* dst = delta + (((size_t)kv * n_chunks + c) * 128 + tid) * 128;
-#pragma unroll
-    for (int cc = 0; cc < 4; ++cc) {
-      float x[32];
-      tmem_ld32(tmem + ((uint32_t)(warp * 32) << 16) + 32 * cc, x);
-      tmem_wait_ld();
-#pragma unroll
-      for (int e = 0; e < 8; ++e)
-        *reinterpret_cast<float4*>(dst + 32 * cc + 4 * e) = make_float4(x[4 * e], x[4 * e + 1], x[4 * e + 2], x[4 * e + 3]);
-    }
-  } else if (status) {
-    atomicExch(status, 1);
-  }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 0) {
-    tc_fence_after();
-    tmem_dealloc(tmem, 128);
-  }
-}
-
-// rstate[kv][c] = sum_{i >= c + lag} delta[kv][i],  c = 0 .. n_r-1, i up to n_qt-1  (bf16).
-__global__ void __launch_bounds__(256)
-tc_bwd_rscan_kernel(const float* __restrict__ delta, __nv_bfloat16* __restrict__ rstate, int n_chunks,
-                    int n_qt, int lag) {
-  const int kv = blockIdx.x;
-  const int idx = blockIdx.y * 256 + threadIdx.x;
-  const float4* src = reinterpret_cast<const float4*>(delta) + (size_t)kv * n_chunks * 4096 + idx;
-  uint2* dst = reinterpret_cast<uint2*>(rstate) + (size_t)kv * n_chunks * 4096 + idx;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int i = n_qt - 1; i >= lag; --i) {
-    const float4 x = src[(size_t)i * 4096];
-    acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
-    dst[(size_t)(i - lag) * 4096] = make_uint2(pack_bf16(acc.x, acc.y), pack_bf16(acc.z, acc.w));
-  }
-}
-
 // ================================================================================ dq
 constexpr int DQ_OFF_Q = 0;
 constexpr int DQ_OFF_G = 1 * TILE_BYTES;
@@ -961,20 +869,10 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
 
   // reverse states of the residual branch: chunks c with a query tile beyond c + wt
   const int n_r = rla_on && a.mode != RATTN_MODE_FULL_CAUSAL ? n_qt - wt - 1 : 0;
-  if (n_r > 0) {
-    e = cudaFuncSetAttribute(tc_bwd_rdelta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, RD_SMEM);
-    if (e != cudaSuccess) return e;
-    {
-      KernelTimer kt("tc_bwd_rdelta", s);
-      tc_bwd_rdelta_kernel<<<dim3(n_r, (unsigned)nkv), 128, RD_SMEM, s>>>(tm_q, tm_gr, a.chunk_delta, a.n_chunks,
-                                                                          wt + 1, a.group, a.status);
-    }
-    {
-      KernelTimer kt("tc_bwd_rscan", s);
-      tc_bwd_rscan_kernel<<<dim3((unsigned)nkv, 16), 256, 0, s>>>(a.chunk_delta, a.rstate, a.n_chunks, n_qt, wt + 1);
-    }
-    count_launches(2);
-  }
+  // R_c for c = 0 .. n_r-1: walk the query tiles from the last one down to wt+1
+  e = launch_tc_states(a.q, g_r, a.rstate, a.T, (int)nkv, a.group, a.n_chunks, n_r, n_qt - 1, -1, n_qt - wt - 2,
+                       a.status, "tc_state_bwd", s);
+  if (e != cudaSuccess) return e;
 
   BwdArgs t;
   t.dq = reinterpret_cast<__nv_bfloat16*>(a.dq);
