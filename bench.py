@@ -434,6 +434,64 @@ def run_case(args):
         print(json.dumps({"case": "decode", "ms": ms, "gb_per_s": decode_bytes(c5) / (ms * 1e-3) / 1e9}))
 
 
+def run_all_configs(args):
+    """Forward timings of the five named configurations (window sweep and the two control
+    modes for config 3, prefill and decode for config 5), one JSON line.  Device-resident
+    inputs, CUDA events, each configuration's working set larger than L2 except config 1."""
+    from paper_2506_15545_b200 import binding as R
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    sync = torch.cuda.synchronize
+    pk = peaks()
+    out = {"peaks": pk, "configs": []}
+
+    def roof_ms(wl, fl):
+        return 1e3 * max(fl / (pk["tf_burst"] * 1e12), io_bytes_fwd(wl) / (pk["hbm"] * 1e9))
+
+    def time_fwd(wl, mode=R.MODE_RATTN, label=None, steps=20):
+        q, k, v = W.make_qkv(wl, dev)
+        ws = R.alloc_workspace(q, k, wl.w)
+        o = torch.empty_like(q)
+        ms = timed(lambda: R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, mode=mode, workspace=ws, out=o),
+                   steps, 3, sync)
+        assert R.rattn_read_status(ws) == 0
+        eff = wl if mode == R.MODE_RATTN else wl.replace(w=wl.T if mode == R.MODE_FULL_CAUSAL else wl.w)
+        fl = flops(eff, "fwd") if mode == R.MODE_RATTN else flops(eff, "fwd_main") - 2 * wl.d * wl.d * max(0, eff.T - eff.w - 1) * wl.B * wl.H_q
+        rec = {"config": label or wl.name, "B": wl.B, "H_q": wl.H_q, "H_kv": wl.H_kv, "T": wl.T, "w": wl.w,
+               "mode": ["rattn", "swa_only", "full_causal"][mode], "ms": ms, "tflops": fl / (ms * 1e-3) / 1e12,
+               "tokens_per_s": wl.B * wl.T / (ms * 1e-3), "roofline_ms": roof_ms(wl, fl),
+               "roofline_frac": roof_ms(wl, fl) / ms, "tensor_path": bool(R.rattn_uses_tensor_path(wl.d, wl.w, R.RATTN_BF16 if wl.dtype == "bf16" else R.RATTN_F32, mode))}
+        out["configs"].append(rec)
+        del q, k, v, ws, o
+        torch.cuda.empty_cache()
+
+    time_fwd(W.C1, label="c1 (fp32, portable kernels)")
+    time_fwd(W.C2)
+    for w in W.C3_WINDOWS:
+        time_fwd(W.C3.replace(w=w), label=f"c3 w={w}")
+    for w in W.C3_WINDOWS:
+        time_fwd(W.C3.replace(w=w), mode=R.MODE_SWA_ONLY, label=f"c3 w={w} swa-only")
+    time_fwd(W.C3, mode=R.MODE_FULL_CAUSAL, label="c3 full-causal")
+    time_fwd(W.C4, label="c4 forward only")
+    c5 = W.C5.replace(B=args.c5_batch)
+    time_fwd(c5, label=f"c5 prefill (B={c5.B} of 32)", steps=3)
+    kr = torch.randn(W.C5.B, W.C5.H_kv, W.C5.w, W.C5.d, device=dev).to(torch.bfloat16)
+    vr = torch.randn(W.C5.B, W.C5.H_kv, W.C5.w, W.C5.d, device=dev).to(torch.bfloat16)
+    st = torch.zeros(W.C5.B, W.C5.H_kv, W.C5.d, W.C5.d, device=dev)
+    qd, kd, vd = W.make_decode_token(W.C5, 0, dev)
+    od = torch.empty_like(qd)
+    pos = [W.C5.T]
+
+    def dec():
+        R.rattn_decode_step_ex(qd, kd, vd, kr, vr, st, pos[0], scale=W.C5.scale, out=od)
+        pos[0] += 1
+    ms_d = timed(dec, 256, 10, sync)
+    out["configs"].append({"config": "c5 decode step (B=32)", "ms": ms_d, "gb_per_s": decode_bytes(W.C5) / (ms_d * 1e-3) / 1e9,
+                           "roofline_frac": decode_bytes(W.C5) / (ms_d * 1e-3) / 1e9 / pk["hbm"],
+                           "tokens_per_s": W.C5.B / (ms_d * 1e-3), "note": "one cache set (84 MB, below L2 size)"})
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -442,7 +500,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--case", default=None, choices=["fwd", "train", "decode"],
                     help="run one small case (for profiler captures) instead of the benchmark")
+    ap.add_argument("--all-configs", action="store_true",
+                    help="time the forward of all five named configurations instead of the benchmark")
+    ap.add_argument("--c5-batch", type=int, default=8, help="batch entries of config 5's prefill to time")
     args = ap.parse_args()
+    if args.all_configs:
+        run_all_configs(args)
+        return
     if args.case:
         run_case(args)
         return
