@@ -560,7 +560,9 @@ __device__ bool kv_mma(unsigned char* smem, KvBars* bars, uint32_t tmem, const K
       const uint32_t sQh = sStage + st * TILE_BYTES, sGh = sQh + HT_BYTES;
       WAIT_OR_RETURN_W(bars->full[st], pl.use(n) & 1);
       if (pl.is_r(n)) WAIT_OR_RETURN_W(bars->phiq_ready[slot], (n >> 1) & 1);
-      if (n >= 2) WAIT_OR_RETURN_W(bars->acc_done[pl.stage(n - 2)], pl.use(n - 2) & 1);   // the slot is free
+      // The slot's previous user (item n-2) needs no wait here: its row groups were waited for
+      // before its accumulate products were issued, and those precede these scores in the
+      // tensor pipe, which executes in issue order.
       tc_fence_after();
       mma_k_kh(tS[slot], pl.is_r(n) ? sKphi : sK, sQh);   // S^T  = K Q_h^T   (phi(K) phi(Q_h)^T)
       mma_k_kh(tP[slot], sV, sGh);                         // dP^T = V g_h^T
