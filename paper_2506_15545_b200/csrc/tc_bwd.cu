@@ -199,22 +199,28 @@ __device__ bool dq_control(const CUtensorMap* tm_q, const CUtensorMap* tm_k, con
     mma_kk(tS, sQ, sK + b * TILE_BYTES, false);          // S  = Q K^T
     mma_kk(tP, sG, sV + b * TILE_BYTES, false);          // dP = g_s V^T
     mma_commit(&bars->s_full);
+    if (i >= 1) {
+      // while the row groups work on tile i: the stage of tile i-1 is free once its dQ product
+      // has completed; refill it with tile i+1 (or, after the last tile, the residual operands)
+      const int pb = (i - 1) & 1;
+      WAIT_OR_RETURN_W(bars->dq_done, (i - 1) & 1);
+      if (i + 1 < n_kt) {
+        mbar_arrive_expect_tx(&bars->kv_full[pb], 2 * TILE_BYTES);
+        load_tile(smem + DQ_OFF_K + pb * TILE_BYTES, tm_k, &bars->kv_full[pb], q0 - (i + 1) * TILE, bh_kv);
+        load_tile(smem + DQ_OFF_V + pb * TILE_BYTES, tm_v, &bars->kv_full[pb], q0 - (i + 1) * TILE, bh_kv);
+      } else if (has_rla) {
+        mbar_arrive_expect_tx(&bars->x_full, (has_state ? 2 : 1) * TILE_BYTES);
+        load_tile(smem + DQ_OFF_V + pb * TILE_BYTES, tm_gr, &bars->x_full, q0, bh_q);
+        if (has_state) load_tile(smem + DQ_OFF_K + pb * TILE_BYTES, tm_st, &bars->x_full, 0, st_index);
+      }
+    }
     WAIT_OR_RETURN_W(bars->ds_full, i & 1);
     tc_fence_after();
 #pragma unroll
     for (int k = 0; k < 8; ++k)                           // dQ += dS K, dS read from TMEM
-      mma_bf16_ts(tQ, tS + 8 * k, mnmajor_desc(sK + b * TILE_BYTES, k), idesc_ts, (i > 0 || k > 0) ? 1u : 0u);
+      mma_bf16_ts(tQ, tS + (k < 4 ? 8 * k : 64 + 8 * (k - 4)), mnmajor_desc(sK + b * TILE_BYTES, k), idesc_ts, (i > 0 || k > 0) ? 1u : 0u);
     mma_commit(&bars->dq_done);
-    WAIT_OR_RETURN_W(bars->dq_done, i & 1);
-    if (i + 2 < n_kt) {
-      mbar_arrive_expect_tx(&bars->kv_full[b], 2 * TILE_BYTES);
-      load_tile(smem + DQ_OFF_K + b * TILE_BYTES, tm_k, &bars->kv_full[b], q0 - (i + 2) * TILE, bh_kv);
-      load_tile(smem + DQ_OFF_V + b * TILE_BYTES, tm_v, &bars->kv_full[b], q0 - (i + 2) * TILE, bh_kv);
-    } else if (has_rla && i + 2 == n_kt) {
-      mbar_arrive_expect_tx(&bars->x_full, (has_state ? 2 : 1) * TILE_BYTES);
-      load_tile(smem + DQ_OFF_V + b * TILE_BYTES, tm_gr, &bars->x_full, q0, bh_q);
-      if (has_state) load_tile(smem + DQ_OFF_K + b * TILE_BYTES, tm_st, &bars->x_full, 0, st_index);
-    }
+    // the next tile's scores follow these products in the tensor pipe, which runs in issue order
   }
   if (has_rla) {
     const uint32_t sG2 = sV + other * TILE_BYTES, sSt = sK + other * TILE_BYTES;
@@ -228,14 +234,17 @@ __device__ bool dq_control(const CUtensorMap* tm_q, const CUtensorMap* tm_k, con
     tc_fence_after();
 #pragma unroll
     for (int k = 0; k < 8; ++k)                           // (dA masked) phi(K_cb)
-      mma_bf16_ts(tF, tS + 8 * k, mnmajor_desc(sK + last * TILE_BYTES, k), idesc_ts, (has_state || k > 0) ? 1u : 0u);
+      mma_bf16_ts(tF, tS + (k < 4 ? 8 * k : 64 + 8 * (k - 4)), mnmajor_desc(sK + last * TILE_BYTES, k), idesc_ts, (has_state || k > 0) ? 1u : 0u);
   }
   mma_commit(&bars->o_done);
   return true;
 }
 
-__device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned char* smem, DqBars* bars, uint32_t tmem, int r, int q0,
-                        int bh_q, int n_kt, bool has_boundary, bool has_rla) {
+// Two row groups of 128 threads (thread = query row = TMEM lane): group g takes key columns
+// 64g .. 64g+63 of every score tile and leaves its 64 bf16 results in the first 32 columns of
+// its own half, where the dQ product reads them.  Group 0 alone runs the epilogue.
+__device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned char* smem, DqBars* bars, uint32_t tmem, int g, int r,
+                        int q0, int bh_q, int n_kt, bool has_boundary, bool has_rla) {
   const uint32_t lane_off = (uint32_t)((r & ~31) << 16);
   const uint32_t tS = tmem + lane_off, tP = tmem + 128 + lane_off, tQ = tmem + 256 + lane_off,
                  tF = tmem + 384 + lane_off;
@@ -251,7 +260,7 @@ __device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned cha
     tc_fence_after();
     const bool diag = (i == 0), bound = has_boundary && (i == n_kt - 1);
 #pragma unroll 1
-    for (int c = 0; c < 4; ++c) {                              // rolled: compact code
+    for (int c = 2 * g; c < 2 * g + 2; ++c) {                   // rolled: compact code
       float s[32], dp[32];
       tmem_ld32(tS + 32 * c, s);
       tmem_ld32(tP + 32 * c, dp);
@@ -265,8 +274,8 @@ __device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned cha
         const float d1 = (keep >> (e + 1)) & 1u ? p1 * (dp[e + 1] * a.scale - Drs) : 0.f;
         pk[e >> 1] = pack_bf16(d0, d1);
       }
-      // dS (bf16, two per column) overwrites the S columns already consumed: 16c..16c+15 < 32c+32
-      tmem_st16(tS + 16 * c, pk);
+      // dS (bf16, two per column) overwrites this group's own S columns already consumed
+      tmem_st16(tS + 64 * g + 16 * (c - 2 * g), pk);
     }
     tmem_wait_st();
     tc_fence_before();
@@ -276,13 +285,17 @@ __device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned cha
   if (has_rla) {
     const int last = (n_kt - 1) & 1;
     WAIT_OR_RETURN(bars->dq_done, (n_kt - 1) & 1);           // K_cb is no longer read raw
-    feature_map_row_inplace_lr(smem + DQ_OFF_K + last * TILE_BYTES, r);
+    {
+      const int t2 = g * 128 + r;                              // two threads per key row
+      unsigned char* kh = smem + DQ_OFF_K + last * TILE_BYTES + (t2 & 1) * HALF_BYTES;
+      feature_map_pair(kh, kh, t2 >> 1);
+    }
     fence_proxy_async_smem();
     mbar_arrive(&bars->phik_ready);
     WAIT_OR_RETURN(bars->s_full, n_kt & 1);
     tc_fence_after();
 #pragma unroll 1
-    for (int c = 0; c < 4; ++c) {
+    for (int c = 2 * g; c < 2 * g + 2; ++c) {
       float x[32];
       tmem_ld32(tS + 32 * c, x);
       tmem_wait_ld();
@@ -291,7 +304,7 @@ __device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned cha
 #pragma unroll
       for (int e = 0; e < 32; e += 2)
         pk[e >> 1] = pack_bf16((keep >> e) & 1u ? x[e] : 0.f, (keep >> (e + 1)) & 1u ? x[e + 1] : 0.f);
-      tmem_st16(tS + 16 * c, pk);
+      tmem_st16(tS + 64 * g + 16 * (c - 2 * g), pk);
     }
     tmem_wait_st();
     tc_fence_before();
@@ -299,6 +312,7 @@ __device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned cha
   }
 
   // ---- dq = dQ + phi(q) * (dphi_q - <dphi_q, phi(q)>) -----------------------------------
+  if (g != 0) return true;
   WAIT_OR_RETURN(bars->o_done, 0);
   tc_fence_after();
   const unsigned char* sQ = smem + DQ_OFF_Q;
@@ -381,7 +395,7 @@ __device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned cha
   return true;
 }
 
-__global__ void __launch_bounds__(160, 1)
+__global__ void __launch_bounds__(288, 1)
 tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_gs,
                  const __grid_constant__ CUtensorMap tm_gr, const __grid_constant__ CUtensorMap tm_st,
@@ -413,19 +427,19 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     mbar_init(&bars->kv_full[1], 1);
     mbar_init(&bars->s_full, 1);
     mbar_init(&bars->s_empty, 128);
-    mbar_init(&bars->ds_full, 128);
+    mbar_init(&bars->ds_full, 256);
     mbar_init(&bars->dq_done, 1);
     mbar_init(&bars->x_full, 1);
-    mbar_init(&bars->phik_ready, 128);
+    mbar_init(&bars->phik_ready, 256);
     mbar_init(&bars->o_done, 1);
     mbar_init(&bars->drain, 1);
     bars->abort = 0;
     fence_mbar_init();
   }
-  if (warp == 4) {
+  if (warp == 8) {
     tmem_alloc(&bars->tmem_base, 512);
     tmem_relinquish();
-    if (tid == 128) {
+    if (tid == 256) {
       prefetch_tensormap(&tm_q);
       prefetch_tensormap(&tm_k);
       prefetch_tensormap(&tm_v);
@@ -441,9 +455,9 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const uint32_t tmem = bars->tmem_base;
 
   bool ok = true;
-  if (warp < 4) {
-    ok = dq_rows(a, &tm_dq, smem, bars, tmem, tid, q0, bh_q, n_kt, has_boundary, has_rla);
-  } else if (warp == 4) {
+  if (warp < 8) {
+    ok = dq_rows(a, &tm_dq, smem, bars, tmem, warp >> 2, tid & 127, q0, bh_q, n_kt, has_boundary, has_rla);
+  } else if (warp == 8) {
     ok = dq_control(&tm_q, &tm_k, &tm_v, &tm_gs, &tm_gr, &tm_st, smem, bars, tmem, q0, bh_q, bh_kv, n_kt,
                     has_rla, has_state, st_index);
     if (!ok) {
@@ -454,7 +468,7 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   if (!ok && a.status) atomicExch(a.status, 1);
   tc_fence_before();
   __syncthreads();
-  if (warp == 4) {
+  if (warp == 8) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
   }
@@ -890,7 +904,7 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
   if (e != cudaSuccess) return e;
   {
     KernelTimer kt("tc_bwd_dq", s);
-    tc_bwd_dq_kernel<<<dim3(n_qt, (unsigned)nq), 160, DQ_SMEM, s>>>(tm_q, tm_k, tm_v, tm_gs, tm_gr, tm_st, tm_dq, t);
+    tc_bwd_dq_kernel<<<dim3(n_qt, (unsigned)nq), 288, DQ_SMEM, s>>>(tm_q, tm_k, tm_v, tm_gs, tm_gr, tm_st, tm_dq, t);
   }
   KvMaps km;
   km.k = tm_k; km.v = tm_v; km.rs = tm_rs; km.dk = tm_dk; km.dv = tm_dv;
