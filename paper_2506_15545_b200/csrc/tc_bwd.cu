@@ -265,14 +265,22 @@ __device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned cha
       tmem_ld32(tS + 32 * c, s);
       tmem_ld32(tP + 32 * c, dp);
       tmem_wait_ld();
-      const uint32_t keep = keep_bits(r, c, diag, bound);
       uint32_t pk[16];
+      if (diag || bound) {                         // only the two edge tiles of the band need a mask
+        const uint32_t keep = keep_bits(r, c, diag, bound);
 #pragma unroll
-      for (int e = 0; e < 32; e += 2) {
-        const float p0 = ex2(s[e] * a.scale_log2 - l2), p1 = ex2(s[e + 1] * a.scale_log2 - l2);
-        const float d0 = (keep >> e) & 1u ? p0 * (dp[e] * a.scale - Drs) : 0.f;
-        const float d1 = (keep >> (e + 1)) & 1u ? p1 * (dp[e + 1] * a.scale - Drs) : 0.f;
-        pk[e >> 1] = pack_bf16(d0, d1);
+        for (int e = 0; e < 32; e += 2) {
+          const float p0 = ex2(s[e] * a.scale_log2 - l2), p1 = ex2(s[e + 1] * a.scale_log2 - l2);
+          const float d0 = (keep >> e) & 1u ? p0 * (dp[e] * a.scale - Drs) : 0.f;
+          const float d1 = (keep >> (e + 1)) & 1u ? p1 * (dp[e + 1] * a.scale - Drs) : 0.f;
+          pk[e >> 1] = pack_bf16(d0, d1);
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+          const float p0 = ex2(s[e] * a.scale_log2 - l2), p1 = ex2(s[e + 1] * a.scale_log2 - l2);
+          pk[e >> 1] = pack_bf16(p0 * (dp[e] * a.scale - Drs), p1 * (dp[e + 1] * a.scale - Drs));
+        }
       }
       // dS (bf16, two per column) overwrites this group's own S columns already consumed
       tmem_st16(tS + 64 * g + 16 * (c - 2 * g), pk);
@@ -655,6 +663,24 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
       } else {
         // diagonal tile: queries q >= r; oldest tile of the band: queries q <= r
         const uint32_t keep = (diag ? bits_ge(rd) : 0xffffffffu) & (bound ? bits_le(rd) : 0xffffffffu);
+        if (!diag && !bound) {                     // interior tiles of the band: no mask
+#pragma unroll
+          for (int e4 = 0; e4 < 32; e4 += 4) {
+            const float4 lv = *reinterpret_cast<const float4*>(l2 + 32 * c + e4);
+            const float4 dv = *reinterpret_cast<const float4*>(Ds + 32 * c + e4);
+            const float lq[4] = {lv.x, lv.y, lv.z, lv.w}, dq4[4] = {dv.x, dv.y, dv.z, dv.w};
+            float p[4], d[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              p[u] = ex2(s[e4 + u] * a.scale_log2 - lq[u]);
+              d[u] = p[u] * (dp[e4 + u] * a.scale - dq4[u]);
+            }
+            pk1[e4 >> 1] = pack_bf16(p[0], p[1]);
+            pk1[(e4 >> 1) + 1] = pack_bf16(p[2], p[3]);
+            pk2[e4 >> 1] = pack_bf16(d[0], d[1]);
+            pk2[(e4 >> 1) + 1] = pack_bf16(d[2], d[3]);
+          }
+        } else
 #pragma unroll
         for (int e4 = 0; e4 < 32; e4 += 4) {
           const float4 lv = *reinterpret_cast<const float4*>(l2 + 32 * c + e4);

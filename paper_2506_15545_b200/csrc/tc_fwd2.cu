@@ -324,9 +324,14 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
         float x[32];
         tmem_ld32(tS + 32 * c, x);
         tmem_wait_ld();
-        const uint32_t keep = keep_bits(r, c, diag, bound);
+        if (diag || bound) {                       // only the two edge tiles of the band need a mask
+          const uint32_t keep = keep_bits(r, c, diag, bound);
 #pragma unroll
-        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, (keep >> e) & 1u ? x[e] : -INFINITY);
+          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, (keep >> e) & 1u ? x[e] : -INFINITY);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, x[e]);
+        }
       }
       mx *= a.scale_log2;                                              // scale > 0
       // lazy rescale: the reference maximum only moves when the row maximum grew by more than 2^8
@@ -356,14 +361,23 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
         float x[32];
         tmem_ld32(tS + 32 * c, x);
         tmem_wait_ld();
-        const uint32_t keep = keep_bits(r, c, diag, bound);
         uint32_t pk[16];
+        if (diag || bound) {
+          const uint32_t keep = keep_bits(r, c, diag, bound);
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          const float p0 = (keep >> (2 * e)) & 1u ? ex2(x[2 * e] * a.scale_log2 - m_ref) : 0.f;
-          const float p1 = (keep >> (2 * e + 1)) & 1u ? ex2(x[2 * e + 1] * a.scale_log2 - m_ref) : 0.f;
-          psum += p0 + p1;
-          pk[e] = pack_f16(p0, p1);
+          for (int e = 0; e < 16; ++e) {
+            const float p0 = (keep >> (2 * e)) & 1u ? ex2(x[2 * e] * a.scale_log2 - m_ref) : 0.f;
+            const float p1 = (keep >> (2 * e + 1)) & 1u ? ex2(x[2 * e + 1] * a.scale_log2 - m_ref) : 0.f;
+            psum += p0 + p1;
+            pk[e] = pack_f16(p0, p1);
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const float p0 = ex2(x[2 * e] * a.scale_log2 - m_ref), p1 = ex2(x[2 * e + 1] * a.scale_log2 - m_ref);
+            psum += p0 + p1;
+            pk[e] = pack_f16(p0, p1);
+          }
         }
         tmem_st16(tS + 16 * c, pk);
       }
