@@ -31,6 +31,12 @@ from paper_2506_15545_b200 import workloads as W  # noqa: E402
 
 METRIC = "RAttention fwd+bwd TFLOP/s (T=4096,w=512,d=128,bf16)"
 
+# DRAM traffic per launch of the main kernels (dram__bytes_read.sum + dram__bytes_write.sum, one
+# ncu capture each on the small training case `--case train`, B = 2), in MB per batch entry of
+# this head configuration; it scales with the batch.  See profiles/.  Set an entry to None when
+# its kernel changes after the capture.
+NCU_TRAFFIC_MB_PER_BATCH_ENTRY = {"tc_fwd": None, "tc_bwd_dq": None, "tc_bwd_dkv": None}
+
 
 # --------------------------------------------------------------------------- work model
 def n_swa_pairs(T, w):
@@ -93,7 +99,7 @@ class ClockSampler:
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                       "-lms", "100", "-i", str(index)], stdout=self.f,
+                                       "-lms", "50", "-i", str(index)], stdout=self.f,
                                       stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
@@ -266,8 +272,11 @@ def run_ours(args, wl):
     roof = None
     if top in kflops:
         ach = flops(wl, kflops[top]) / (per_launch[top] * 1e-3) / 1e12
+        mb = NCU_TRAFFIC_MB_PER_BATCH_ENTRY.get(top)
         roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": pk["tf_sus"], "unit": "TFLOP/s",
-                "frac": ach / pk["tf_sus"], "traffic": None, "peak_source": pk["src"] + " (sustained bf16)",
+                "frac": ach / pk["tf_sus"], "traffic": None if mb is None else mb * 1e6 * wl.B,
+                "traffic_unit": "bytes per launch (ncu capture at B=2, scaled by the batch)",
+                "peak_source": pk["src"] + " (sustained bf16: the kernel is timed inside a long step)",
                 "ms_per_launch": per_launch[top]}
     total_k = sum(share.values())
     kernels = {n: {"launches": kernel_ms[n][0], "ms_per_launch": per_launch[n], "share": share[n] / total_k}
@@ -495,7 +504,7 @@ def run_all_configs(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--case", default=None, choices=["fwd", "train", "decode"],
