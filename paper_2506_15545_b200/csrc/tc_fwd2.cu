@@ -23,6 +23,8 @@
 //   is applied to the Q and K tiles in shared memory, in place: it never goes to HBM.
 //   Section 3.2: y = g_s * o_swa / rms(o_swa) + g_r * o_rla / rms(o_rla), staged in the tile's Q
 //   buffer and written by one TMA store.
+#include <type_traits>
+
 #include "tc_common.cuh"
 
 namespace rattn {
@@ -506,36 +508,48 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     }
     const float* gs = a.gamma_swa ? a.gamma_swa + (size_t)un.h * 128 : nullptr;
     const float* gr = a.gamma_rla ? a.gamma_rla + (size_t)un.h * 128 : nullptr;
+    // the branches on "gains given" and "tile has a residual branch" are taken once, outside the loop
+    auto emit_y = [&](auto has_gains_t, auto has_rla_t) {
+      constexpr bool has_gains = decltype(has_gains_t)::value, has_rla = decltype(has_rla_t)::value;
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {                                      // 16 columns at a time
-      float orl[16];
-      if (rlaX) {
-        tmem_ld16(tO + 16 * c, orl);
-        tmem_wait_ld();
-      }
-      uint32_t yk[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&stash[8 * c + e]));
-        const int col = 16 * c + 2 * e;
-        float y0 = f.x, y1 = f.y;
-        if (gs) {
-          y0 *= __ldg(gs + col);
-          y1 *= __ldg(gs + col + 1);
+      for (int c = 0; c < 8; ++c) {                                    // 16 columns at a time
+        float orl[16];
+        if constexpr (has_rla) {
+          tmem_ld16(tO + 16 * c, orl);
+          tmem_wait_ld();
         }
-        if (rlaX) {
-          float r0 = orl[2 * e] * rr, r1 = orl[2 * e + 1] * rr;
-          if (gr) {
-            r0 *= __ldg(gr + col);
-            r1 *= __ldg(gr + col + 1);
+        uint32_t yk[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&stash[8 * c + e]));
+          const int col = 16 * c + 2 * e;
+          float y0 = f.x, y1 = f.y;
+          if constexpr (has_gains) {
+            y0 *= gs ? __ldg(gs + col) : 1.f;
+            y1 *= gs ? __ldg(gs + col + 1) : 1.f;
           }
-          y0 += r0;
-          y1 += r1;
+          if constexpr (has_rla) {
+            float r0 = orl[2 * e] * rr, r1 = orl[2 * e + 1] * rr;
+            if constexpr (has_gains) {
+              r0 *= gr ? __ldg(gr + col) : 1.f;
+              r1 *= gr ? __ldg(gr + col + 1) : 1.f;
+            }
+            y0 += r0;
+            y1 += r1;
+          }
+          yk[e] = pack_bf16(y0, y1);
         }
-        yk[e] = pack_bf16(y0, y1);
+        *reinterpret_cast<uint4*>(sQ + swz(r, 2 * c)) = make_uint4(yk[0], yk[1], yk[2], yk[3]);
+        *reinterpret_cast<uint4*>(sQ + swz(r, 2 * c + 1)) = make_uint4(yk[4], yk[5], yk[6], yk[7]);
       }
-      *reinterpret_cast<uint4*>(sQ + swz(r, 2 * c)) = make_uint4(yk[0], yk[1], yk[2], yk[3]);
-      *reinterpret_cast<uint4*>(sQ + swz(r, 2 * c + 1)) = make_uint4(yk[4], yk[5], yk[6], yk[7]);
+    };
+    const bool gains = gs != nullptr || gr != nullptr;
+    if (gains) {
+      if (rlaX) emit_y(std::true_type{}, std::true_type{});
+      else emit_y(std::true_type{}, std::false_type{});
+    } else {
+      if (rlaX) emit_y(std::false_type{}, std::true_type{});
+      else emit_y(std::false_type{}, std::false_type{});
     }
     if (t < a.T && a.lse) a.lse[(size_t)un.bh_q * a.T + t] = (m_ref + log2f(l)) * 0.6931471805599453f;
     fence_proxy_async_smem();
