@@ -67,95 +67,99 @@ tc_bwd_prep_kernel(const __nv_bfloat16* __restrict__ dy, const float* __restrict
                    float* __restrict__ dgamma_r, const float* __restrict__ lse, float* __restrict__ lse2p,
                    float* __restrict__ dscp, size_t n_rows_pad, int T, int t_pad, int H_q, float eps, float scale,
                    int rla_on) {
+  // Half a warp per row, a lane owns 8 consecutive features; the 64 rows of a CTA lie inside one
+  // (batch, head) pair because t_pad is a multiple of 128.  With n = o / r (r the rms incl. eps),
+  // gh = dy * gain, A = gh . o:   g = (gh - n * (A / (128 r))) / r,   D = g . o = (A - A ss / (128 r^2)) / r,
+  // so each branch needs two row sums (ss = o . o and A), all four reduced in one shuffle round.
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int sub = lane >> 4, l16 = lane & 15;
   constexpr int ROWS_PER_CTA = 64;
   const size_t row0 = (size_t)blockIdx.x * ROWS_PER_CTA;
-  float acc_s[4] = {0.f, 0.f, 0.f, 0.f}, acc_r[4] = {0.f, 0.f, 0.f, 0.f};
-  int acc_h = -1;
-  auto flush = [&]() {
-    if (acc_h < 0) return;
+  if (row0 >= n_rows_pad) return;
+  const size_t bq = row0 / t_pad;
+  const int t0 = (int)(row0 - bq * t_pad);
+  const int h = (int)(bq % H_q);
+  float gs[8], gr[8], acc_s[8], acc_r[8];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      if (dgamma_s) atomicAdd(dgamma_s + (size_t)acc_h * 128 + 4 * lane + e, acc_s[e]);
-      if (dgamma_r && rla_on) atomicAdd(dgamma_r + (size_t)acc_h * 128 + 4 * lane + e, acc_r[e]);
-      acc_s[e] = 0.f;
-      acc_r[e] = 0.f;
-    }
-  };
-  for (int rr = warp; rr < ROWS_PER_CTA; rr += 8) {
-    const size_t prow = row0 + rr;                 // row of the padded [B*H_q, t_pad] index space
-    if (prow >= n_rows_pad) break;
-    const size_t bq = prow / t_pad;
-    const int t = (int)(prow % t_pad);
+  for (int e = 0; e < 8; ++e) {
+    gs[e] = gamma_s ? __ldg(gamma_s + (size_t)h * 128 + 8 * l16 + e) : 1.f;
+    gr[e] = gamma_r ? __ldg(gamma_r + (size_t)h * 128 + 8 * l16 + e) : 1.f;
+    acc_s[e] = 0.f;
+    acc_r[e] = 0.f;
+  }
+#pragma unroll 2
+  for (int rr = 2 * warp + sub; rr < ROWS_PER_CTA; rr += 16) {
+    const int t = t0 + rr;
+    const size_t prow = bq * t_pad + t;
     if (t >= T) {                                  // padding: statistics that make every weight zero
-      if (lane == 0) {
+      if (l16 == 0) {
         lse2p[prow] = INFINITY;
         dscp[prow] = 0.f;
       }
       continue;
     }
     const size_t row = bq * T + t;
-    const int h = (int)(bq % H_q);
-    const float4 xs = *reinterpret_cast<const float4*>(o_s + row * 128 + 4 * lane);
-    const float4 xr = *reinterpret_cast<const float4*>(o_r + row * 128 + 4 * lane);
-    const uint2 gy = *reinterpret_cast<const uint2*>(dy + row * 128 + 4 * lane);
-    const float2 g01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gy.x));
-    const float2 g23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gy.y));
-    const float g[4] = {g01.x, g01.y, g23.x, g23.y};
-    const float vs[4] = {xs.x, xs.y, xs.z, xs.w}, vr[4] = {xr.x, xr.y, xr.z, xr.w};
-    float ss = 0.f, sr = 0.f;
+    const float4 s0 = *reinterpret_cast<const float4*>(o_s + row * 128 + 8 * l16);
+    const float4 s1 = *reinterpret_cast<const float4*>(o_s + row * 128 + 8 * l16 + 4);
+    const float4 r0 = *reinterpret_cast<const float4*>(o_r + row * 128 + 8 * l16);
+    const float4 r1 = *reinterpret_cast<const float4*>(o_r + row * 128 + 8 * l16 + 4);
+    const uint4 gy = *reinterpret_cast<const uint4*>(dy + row * 128 + 8 * l16);
+    const float vs[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+    const float vr[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+    float g[8];
+    {
+      const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&gy);
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
+      for (int e = 0; e < 4; ++e) {
+        const float2 f = __bfloat1622float2(hp[e]);
+        g[2 * e] = f.x;
+        g[2 * e + 1] = f.y;
+      }
+    }
+    float ss = 0.f, sr = 0.f, As = 0.f, Ar = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
       ss += vs[e] * vs[e];
       sr += vr[e] * vr[e];
+      As += g[e] * gs[e] * vs[e];
+      Ar += g[e] * gr[e] * vr[e];
     }
+    const unsigned half_mask = sub ? 0xffff0000u : 0x0000ffffu;   // the other half may be on a padding row
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      ss += __shfl_xor_sync(0xffffffffu, ss, o);
-      sr += __shfl_xor_sync(0xffffffffu, sr, o);
+    for (int o = 8; o > 0; o >>= 1) {
+      ss += __shfl_xor_sync(half_mask, ss, o);
+      sr += __shfl_xor_sync(half_mask, sr, o);
+      As += __shfl_xor_sync(half_mask, As, o);
+      Ar += __shfl_xor_sync(half_mask, Ar, o);
     }
     const float is = rsqrtf(ss * (1.f / 128.f) + eps), ir = rsqrtf(sr * (1.f / 128.f) + eps);
-    float ghs[4], ghr[4], ms = 0.f, mr = 0.f;
-    if ((dgamma_s || dgamma_r) && h != acc_h) {
-      flush();
-      acc_h = h;
-    }
+    const float cs = As * is * is * (1.f / 128.f), cr = Ar * ir * ir * (1.f / 128.f);   // mean(gh n) / r
+    uint32_t ws[4], wr[4];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const float gs = gamma_s ? __ldg(gamma_s + (size_t)h * 128 + 4 * lane + e) : 1.f;
-      const float gr = gamma_r ? __ldg(gamma_r + (size_t)h * 128 + 4 * lane + e) : 1.f;
-      ghs[e] = g[e] * gs;
-      ghr[e] = g[e] * gr;
-      ms += ghs[e] * vs[e] * is;
-      mr += ghr[e] * vr[e] * ir;
+    for (int e = 0; e < 8; e += 2) {
+      ws[e >> 1] = pack_bf16((g[e] * gs[e] - vs[e] * cs) * is, (g[e + 1] * gs[e + 1] - vs[e + 1] * cs) * is);
+      wr[e >> 1] = pack_bf16((g[e] * gr[e] - vr[e] * cr) * ir, (g[e + 1] * gr[e + 1] - vr[e + 1] * cr) * ir);
       acc_s[e] += g[e] * vs[e] * is;
+      acc_s[e + 1] += g[e + 1] * vs[e + 1] * is;
       acc_r[e] += g[e] * vr[e] * ir;
+      acc_r[e + 1] += g[e + 1] * vr[e + 1] * ir;
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      ms += __shfl_xor_sync(0xffffffffu, ms, o);
-      mr += __shfl_xor_sync(0xffffffffu, mr, o);
-    }
-    ms *= (1.f / 128.f);
-    mr *= (1.f / 128.f);
-    float ds[4], dr[4], dl = 0.f;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      ds[e] = (ghs[e] - vs[e] * is * ms) * is;
-      dr[e] = (ghr[e] - vr[e] * ir * mr) * ir;
-      dl += ds[e] * vs[e];
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) dl += __shfl_xor_sync(0xffffffffu, dl, o);
-    *reinterpret_cast<uint2*>(g_s + row * 128 + 4 * lane) = make_uint2(pack_bf16(ds[0], ds[1]), pack_bf16(ds[2], ds[3]));
-    *reinterpret_cast<uint2*>(g_r + row * 128 + 4 * lane) = make_uint2(pack_bf16(dr[0], dr[1]), pack_bf16(dr[2], dr[3]));
-    if (lane == 0) {
+    *reinterpret_cast<uint4*>(g_s + row * 128 + 8 * l16) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
+    *reinterpret_cast<uint4*>(g_r + row * 128 + 8 * l16) = make_uint4(wr[0], wr[1], wr[2], wr[3]);
+    if (l16 == 0) {
+      const float dl = (As - cs * ss) * is;        // D_t = g_s . o_swa
       delta[row] = dl;
       lse2p[prow] = lse[row] * LOG2E;
       dscp[prow] = dl * scale;
     }
   }
-  if (dgamma_s || dgamma_r) flush();
+  if (dgamma_s || dgamma_r) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      if (dgamma_s) atomicAdd(dgamma_s + (size_t)h * 128 + 8 * l16 + e, acc_s[e]);
+      if (dgamma_r && rla_on) atomicAdd(dgamma_r + (size_t)h * 128 + 8 * l16 + e, acc_r[e]);
+    }
+  }
 }
 
 // ================================================================================ dq
