@@ -206,6 +206,17 @@ def timed(fn, steps, warmup, sync):
     return a.elapsed_time(b) / steps
 
 
+def whole_job(ms_local, units_per_rank, dist=None, device="cpu"):
+    """Replicas only: every rank runs the same per-GPU workload with no data-path exchange.
+    The job's time is the slowest rank's (MAX over ranks), its work the sum over ranks.
+    Returns (ms, total units)."""
+    if dist is None:
+        return ms_local, units_per_rank
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item()), units_per_rank * dist.get_world_size()
+
+
 def run_ours(args, wl):
     from paper_2506_15545_b200 import binding as R
     rank = int(os.environ.get("RANK", "0"))
@@ -256,11 +267,8 @@ def run_ours(args, wl):
     R.rattn_timing_enable(False)
     clocks = sampler.stop() if sampler else None
     assert R.rattn_read_status(ws) == 0, "device-side wait expired"
-    if dist is not None:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = flops(wl, "step") * world / (ms * 1e-3) / 1e12
+    ms, total_flops = whole_job(ms, flops(wl, "step"), dist, dev)
+    value = total_flops / (ms * 1e-3) / 1e12
 
     # ---- dominant kernel and its roofline -------------------------------------------
     per_launch = {n: tot / cnt for n, (cnt, tot) in kernel_ms.items() if cnt}
