@@ -163,255 +163,323 @@ tc_bwd_prep_kernel(const __nv_bfloat16* __restrict__ dy, const float* __restrict
 }
 
 // ================================================================================ dq
-constexpr int DQ_OFF_Q = 0;
+// Persistent: one CTA per SM walks a list of (query head, query tile) items, so that an item's
+// first loads are in flight while the previous item's epilogue drains (at w = 512 the fixed
+// cost per tile -- first TMA touch, output staging -- is larger than the band itself).
+//   loader warp   Q (two buffers, alternating), g_s, K/V tiles through a ring of two stages;
+//                 the residual operands (g_r, stored state) take one more slot of that ring
+//   MMA warp      per key tile S = Q K^T, dP = g_s V^T; after the row groups have overwritten S
+//                 with dS (bf16, in TMEM): dQ += dS K.  Then the residual part.
+//   row groups    two groups of 128 threads (thread = query row = TMEM lane), group g takes the
+//                 key columns 64g .. 64g+63 of every tile; group 0 runs the epilogue
+// All barriers run on with phase counters that every role advances in the same way.
+constexpr int DQ_OFF_Q = 0;                 // Q buffer 0
 constexpr int DQ_OFF_G = 1 * TILE_BYTES;
 constexpr int DQ_OFF_K = 2 * TILE_BYTES;   // 2 stages
 constexpr int DQ_OFF_V = 4 * TILE_BYTES;   // 2 stages
-constexpr int DQ_OFF_D = 6 * TILE_BYTES;
+constexpr int DQ_OFF_Q1 = 6 * TILE_BYTES;  // Q buffer 1
 constexpr int DQ_OFF_BAR = 7 * TILE_BYTES;
 constexpr int DQ_SMEM = DQ_OFF_BAR + 256;
+constexpr int DQ_THREADS = 320;            // 2 row groups, MMA warp, loader warp
 
 struct DqBars {
-  uint64_t qg_full, kv_full[2], s_full, s_empty, ds_full, dq_done, x_full, phik_ready, o_done, drain;
+  uint64_t qg_full, kv_full[2], kv_free[2], s_full, ds_full, phik_ready, o_done, acc_free, drain;
   uint32_t tmem_base;
   int abort;
 };
 
-__device__ bool dq_control(const CUtensorMap* tm_q, const CUtensorMap* tm_k, const CUtensorMap* tm_v,
-                           const CUtensorMap* tm_gs, const CUtensorMap* tm_gr, const CUtensorMap* tm_st,
-                           unsigned char* smem, DqBars* bars, uint32_t tmem, int q0, int bh_q, int bh_kv,
-                           int n_kt, bool has_rla, bool has_state, int st_index) {
-  const uint32_t sQ = smem_u32(smem + DQ_OFF_Q), sG = smem_u32(smem + DQ_OFF_G);
-  const uint32_t sK = smem_u32(smem + DQ_OFF_K), sV = smem_u32(smem + DQ_OFF_V), sD = smem_u32(smem + DQ_OFF_D);
-  const uint32_t tS = tmem, tP = tmem + 128, tQ = tmem + 256, tF = tmem + 384;
+struct DqItem {
+  int q0, bh_q, bh_kv, n_kt, st_index;
+  bool has_boundary, has_rla, has_state;
+};
 
-  mbar_arrive_expect_tx(&bars->qg_full, 2 * TILE_BYTES);
-  load_tile(smem + DQ_OFF_Q, tm_q, &bars->qg_full, q0, bh_q);
-  load_tile(smem + DQ_OFF_G, tm_gs, &bars->qg_full, q0, bh_q);
-  for (int i = 0; i < (n_kt < 2 ? n_kt : 2); ++i) {
-    mbar_arrive_expect_tx(&bars->kv_full[i], 2 * TILE_BYTES);
-    load_tile(smem + DQ_OFF_K + i * TILE_BYTES, tm_k, &bars->kv_full[i], q0 - i * TILE, bh_kv);
-    load_tile(smem + DQ_OFF_V + i * TILE_BYTES, tm_v, &bars->kv_full[i], q0 - i * TILE, bh_kv);
-  }
-  WAIT_OR_RETURN_W(bars->qg_full, 0);
-  constexpr uint32_t idesc_ts = instr_desc(128, 128, 0, 1);
-  const int last = (n_kt - 1) & 1, other = last ^ 1;
-  for (int i = 0; i < n_kt; ++i) {
-    const int b = i & 1;
-    WAIT_OR_RETURN_W(bars->kv_full[b], (i >> 1) & 1);
-    tc_fence_after();
-    mma_kk(tS, sQ, sK + b * TILE_BYTES, false);          // S  = Q K^T
-    mma_kk(tP, sG, sV + b * TILE_BYTES, false);          // dP = g_s V^T
-    mma_commit(&bars->s_full);
-    if (i >= 1) {
-      // while the row groups work on tile i: the stage of tile i-1 is free once its dQ product
-      // has completed; refill it with tile i+1 (or, after the last tile, the residual operands)
-      const int pb = (i - 1) & 1;
-      WAIT_OR_RETURN_W(bars->dq_done, (i - 1) & 1);
-      if (i + 1 < n_kt) {
-        mbar_arrive_expect_tx(&bars->kv_full[pb], 2 * TILE_BYTES);
-        load_tile(smem + DQ_OFF_K + pb * TILE_BYTES, tm_k, &bars->kv_full[pb], q0 - (i + 1) * TILE, bh_kv);
-        load_tile(smem + DQ_OFF_V + pb * TILE_BYTES, tm_v, &bars->kv_full[pb], q0 - (i + 1) * TILE, bh_kv);
-      } else if (has_rla) {
-        mbar_arrive_expect_tx(&bars->x_full, (has_state ? 2 : 1) * TILE_BYTES);
-        load_tile(smem + DQ_OFF_V + pb * TILE_BYTES, tm_gr, &bars->x_full, q0, bh_q);
-        if (has_state) load_tile(smem + DQ_OFF_K + pb * TILE_BYTES, tm_st, &bars->x_full, 0, st_index);
-      }
+__device__ __forceinline__ DqItem dq_item(const BwdArgs& a, int idx, int n_qt) {
+  DqItem it;
+  it.bh_q = idx / n_qt;
+  const int qt = n_qt - 1 - idx % n_qt;                    // long bands first within a head
+  it.q0 = qt * TILE;
+  const int b = it.bh_q / a.H_q, h = it.bh_q % a.H_q;
+  it.bh_kv = b * (a.H_q / a.group) + h / a.group;
+  const int wt = a.w / TILE;
+  it.has_boundary = (a.mode != RATTN_MODE_FULL_CAUSAL) && (qt - wt >= 0);
+  it.n_kt = (it.has_boundary ? wt : qt) + 1;
+  it.has_rla = it.has_boundary && (a.mode == RATTN_MODE_RATTN);
+  const int cb = qt - wt;
+  it.has_state = it.has_rla && cb > 0;
+  it.st_index = it.bh_kv * a.n_chunks + (cb > 0 ? cb : 0);
+  return it;
+}
+
+struct DqMaps {
+  CUtensorMap q, k, v, gs, gr, st, dq;
+};
+
+__device__ bool dq_loader(const DqMaps& tm, const BwdArgs& a, unsigned char* smem, DqBars* bars, int n_items, int n_qt) {
+  int kc = 0, n = 0, co = 0;                               // ring uses, items, o_done completions so far
+  for (int idx = blockIdx.x; idx < n_items; idx += gridDim.x, ++n) {
+    const DqItem it = dq_item(a, idx, n_qt);
+    auto ring_wait = [&]() -> bool {                       // the slot's previous user has been consumed
+      const int st = kc & 1, use = kc >> 1;
+      if (use >= 1) WAIT_OR_RETURN_W(bars->kv_free[st], (use - 1) & 1);
+      return true;
+    };
+    // The barrier's previous phase must be over before this item arrives on it: after a short
+    // item the loader gets here while that item's Q and g_s are still in flight.
+    if (n >= 1) WAIT_OR_RETURN_W(bars->qg_full, (n - 1) & 1);
+    mbar_arrive_expect_tx(&bars->qg_full, 2 * TILE_BYTES);
+    // Q into the buffer last used two items ago: free once that item's epilogue has left it
+    if (n >= 2) WAIT_OR_RETURN_W(bars->acc_free, (n - 2) & 1);
+    load_tile(smem + ((n & 1) ? DQ_OFF_Q1 : DQ_OFF_Q), &tm.q, &bars->qg_full, it.q0, it.bh_q);
+    // g_s: its one buffer is free once every product of the previous item has completed
+    // (o_done completes twice for an item with a residual part, once otherwise)
+    if (n >= 1) WAIT_OR_RETURN_W(bars->o_done, (co - 1) & 1);
+    co += it.has_rla ? 2 : 1;
+    load_tile(smem + DQ_OFF_G, &tm.gs, &bars->qg_full, it.q0, it.bh_q);
+    for (int i = 0; i < it.n_kt; ++i, ++kc) {
+      if (!ring_wait()) return false;
+      const int st = kc & 1;
+      mbar_arrive_expect_tx(&bars->kv_full[st], 2 * TILE_BYTES);
+      load_tile(smem + DQ_OFF_K + st * TILE_BYTES, &tm.k, &bars->kv_full[st], it.q0 - i * TILE, it.bh_kv);
+      load_tile(smem + DQ_OFF_V + st * TILE_BYTES, &tm.v, &bars->kv_full[st], it.q0 - i * TILE, it.bh_kv);
     }
-    WAIT_OR_RETURN_W(bars->ds_full, i & 1);
-    tc_fence_after();
-#pragma unroll
-    for (int k = 0; k < 8; ++k)                           // dQ += dS K, dS read from TMEM
-      mma_bf16_ts(tQ, tS + (k < 4 ? 8 * k : 64 + 8 * (k - 4)), mnmajor_desc(sK + b * TILE_BYTES, k), idesc_ts, (i > 0 || k > 0) ? 1u : 0u);
-    mma_commit(&bars->dq_done);
-    // the next tile's scores follow these products in the tensor pipe, which runs in issue order
+    if (it.has_rla) {                                      // g_r in the V half of the slot, the state in the K half
+      if (!ring_wait()) return false;
+      const int st = kc & 1;
+      mbar_arrive_expect_tx(&bars->kv_full[st], (it.has_state ? 2 : 1) * TILE_BYTES);
+      load_tile(smem + DQ_OFF_V + st * TILE_BYTES, &tm.gr, &bars->kv_full[st], it.q0, it.bh_q);
+      if (it.has_state) load_tile(smem + DQ_OFF_K + st * TILE_BYTES, &tm.st, &bars->kv_full[st], 0, it.st_index);
+      ++kc;
+    }
   }
-  if (has_rla) {
-    const uint32_t sG2 = sV + other * TILE_BYTES, sSt = sK + other * TILE_BYTES;
-    WAIT_OR_RETURN_W(bars->x_full, 0);
-    tc_fence_after();
-    mma_kk(tS, sG2, sV + last * TILE_BYTES, false);        // dA = g_r V_cb^T
-    if (has_state) mma_kk(tF, sG2, sSt, false);            // g_r S_cb^T
-    mma_commit(&bars->s_full);
-    WAIT_OR_RETURN_W(bars->phik_ready, 0);
-    WAIT_OR_RETURN_W(bars->ds_full, n_kt & 1);
-    tc_fence_after();
-#pragma unroll
-    for (int k = 0; k < 8; ++k)                           // (dA masked) phi(K_cb)
-      mma_bf16_ts(tF, tS + (k < 4 ? 8 * k : 64 + 8 * (k - 4)), mnmajor_desc(sK + last * TILE_BYTES, k), idesc_ts, (has_state || k > 0) ? 1u : 0u);
-  }
-  mma_commit(&bars->o_done);
   return true;
 }
 
-// Two row groups of 128 threads (thread = query row = TMEM lane): group g takes key columns
-// 64g .. 64g+63 of every score tile and leaves its 64 bf16 results in the first 32 columns of
-// its own half, where the dQ product reads them.  Group 0 alone runs the epilogue.
-__device__ bool dq_rows(const BwdArgs& a, const CUtensorMap* tm_dq, unsigned char* smem, DqBars* bars, uint32_t tmem, int g, int r,
-                        int q0, int bh_q, int n_kt, bool has_boundary, bool has_rla) {
+__device__ bool dq_mma(const BwdArgs& a, unsigned char* smem, DqBars* bars, uint32_t tmem, int n_items, int n_qt) {
+  const uint32_t sG = smem_u32(smem + DQ_OFF_G), sK = smem_u32(smem + DQ_OFF_K), sV = smem_u32(smem + DQ_OFF_V);
+  const uint32_t tS = tmem, tP = tmem + 128, tQ = tmem + 256, tF = tmem + 384;
+  constexpr uint32_t idesc_ts = instr_desc(128, 128, 0, 1);
+  int kc = 0, n = 0, cs = 0, cr = 0;                       // ring uses, items, score hand-overs, residual items
+  for (int idx = blockIdx.x; idx < n_items; idx += gridDim.x, ++n) {
+    const DqItem it = dq_item(a, idx, n_qt);
+    const uint32_t sQ = smem_u32(smem + ((n & 1) ? DQ_OFF_Q1 : DQ_OFF_Q));
+    WAIT_OR_RETURN_W(bars->qg_full, n & 1);
+    int last_st = 0;
+    for (int i = 0; i < it.n_kt; ++i, ++kc, ++cs) {
+      const int st = kc & 1;
+      last_st = st;
+      WAIT_OR_RETURN_W(bars->kv_full[st], (kc >> 1) & 1);
+      tc_fence_after();
+      mma_kk(tS, sQ, sK + st * TILE_BYTES, false);         // S  = Q K^T
+      mma_kk(tP, sG, sV + st * TILE_BYTES, false);         // dP = g_s V^T
+      mma_commit(&bars->s_full);
+      WAIT_OR_RETURN_W(bars->ds_full, cs & 1);
+      if (i == 0 && n >= 1) WAIT_OR_RETURN_W(bars->acc_free, (n - 1) & 1);   // the previous item's epilogue has read dQ
+      tc_fence_after();
+#pragma unroll
+      for (int k = 0; k < 8; ++k)                          // dQ += dS K, dS read from TMEM
+        mma_bf16_ts(tQ, tS + (k < 4 ? 8 * k : 64 + 8 * (k - 4)), mnmajor_desc(sK + st * TILE_BYTES, k), idesc_ts, (i > 0 || k > 0) ? 1u : 0u);
+      // the last tile's K turns into phi(K) for the residual part: its slot is released there
+      if (!(it.has_rla && i == it.n_kt - 1)) mma_commit(&bars->kv_free[st]);
+      // the next tile's scores follow these products in the tensor pipe, which runs in issue order
+    }
+    if (it.has_rla) {
+      const int xs = kc & 1;                               // slot of g_r and the stored state
+      const uint32_t sG2 = sV + xs * TILE_BYTES, sSt = sK + xs * TILE_BYTES;
+      mma_commit(&bars->o_done);                           // (interim) every window product done: K_cb may be rewritten
+      WAIT_OR_RETURN_W(bars->kv_full[xs], (kc >> 1) & 1);
+      tc_fence_after();
+      mma_kk(tS, sG2, sV + last_st * TILE_BYTES, false);   // dA = g_r V_cb^T
+      if (it.has_state) mma_kk(tF, sG2, sSt, false);       // g_r S_cb^T
+      mma_commit(&bars->s_full);
+      WAIT_OR_RETURN_W(bars->phik_ready, cr & 1);
+      WAIT_OR_RETURN_W(bars->ds_full, cs & 1);
+      tc_fence_after();
+#pragma unroll
+      for (int k = 0; k < 8; ++k)                          // (dA masked) phi(K_cb)
+        mma_bf16_ts(tF, tS + (k < 4 ? 8 * k : 64 + 8 * (k - 4)), mnmajor_desc(sK + last_st * TILE_BYTES, k), idesc_ts, (it.has_state || k > 0) ? 1u : 0u);
+      mma_commit(&bars->kv_free[last_st]);
+      mma_commit(&bars->kv_free[xs]);
+      ++kc; ++cs; ++cr;
+    }
+    mma_commit(&bars->o_done);
+  }
+  return true;
+}
+
+__device__ bool dq_rows(const DqMaps& tm, const BwdArgs& a, unsigned char* smem, DqBars* bars, uint32_t tmem, int g, int r,
+                        int n_items, int n_qt) {
   const uint32_t lane_off = (uint32_t)((r & ~31) << 16);
   const uint32_t tS = tmem + lane_off, tP = tmem + 128 + lane_off, tQ = tmem + 256 + lane_off,
                  tF = tmem + 384 + lane_off;
-  unsigned char* sD = smem + DQ_OFF_D;
-  const int t = q0 + r;
-  const bool live = t < a.T;
-  const size_t row = (size_t)bh_q * a.T + t;
-  const float l2 = live ? a.lse[row] * LOG2E : INFINITY;
-  const float Drs = live ? a.delta[row] * a.scale : 0.f;
+  int kc = 0, n = 0, cs = 0, co = 0;                       // ring uses, items, score hand-overs, o_done completions
+  for (int idx = blockIdx.x; idx < n_items; idx += gridDim.x, ++n) {
+    const DqItem it = dq_item(a, idx, n_qt);
+    const int n_kt = it.n_kt;
+    unsigned char* sQ = smem + ((n & 1) ? DQ_OFF_Q1 : DQ_OFF_Q);
+    const int t = it.q0 + r;
+    const bool live = t < a.T;
+    const size_t row = (size_t)it.bh_q * a.T + t;
+    const float l2 = live ? a.lse[row] * LOG2E : INFINITY;
+    const float Drs = live ? a.delta[row] * a.scale : 0.f;
 
-  for (int i = 0; i < n_kt; ++i) {
-    WAIT_OR_RETURN(bars->s_full, i & 1);
-    tc_fence_after();
-    const bool diag = (i == 0), bound = has_boundary && (i == n_kt - 1);
+    for (int i = 0; i < n_kt; ++i, ++cs) {
+      WAIT_OR_RETURN(bars->s_full, cs & 1);
+      tc_fence_after();
+      const bool diag = (i == 0), bound = it.has_boundary && (i == n_kt - 1);
 #pragma unroll 1
-    for (int c = 2 * g; c < 2 * g + 2; ++c) {                   // rolled: compact code
-      float s[32], dp[32];
-      tmem_ld32(tS + 32 * c, s);
-      tmem_ld32(tP + 32 * c, dp);
-      tmem_wait_ld();
-      uint32_t pk[16];
-      if (diag || bound) {                         // only the two edge tiles of the band need a mask
-        const uint32_t keep = keep_bits(r, c, diag, bound);
+      for (int c = 2 * g; c < 2 * g + 2; ++c) {                 // rolled: compact code
+        float s[32], dp[32];
+        tmem_ld32(tS + 32 * c, s);
+        tmem_ld32(tP + 32 * c, dp);
+        tmem_wait_ld();
+        uint32_t pk[16];
+        if (diag || bound) {                       // only the two edge tiles of the band need a mask
+          const uint32_t keep = keep_bits(r, c, diag, bound);
 #pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          const float p0 = ex2(s[e] * a.scale_log2 - l2), p1 = ex2(s[e + 1] * a.scale_log2 - l2);
-          const float d0 = (keep >> e) & 1u ? p0 * (dp[e] * a.scale - Drs) : 0.f;
-          const float d1 = (keep >> (e + 1)) & 1u ? p1 * (dp[e + 1] * a.scale - Drs) : 0.f;
-          pk[e >> 1] = pack_bf16(d0, d1);
+          for (int e = 0; e < 32; e += 2) {
+            const float p0 = ex2(s[e] * a.scale_log2 - l2), p1 = ex2(s[e + 1] * a.scale_log2 - l2);
+            const float d0 = (keep >> e) & 1u ? p0 * (dp[e] * a.scale - Drs) : 0.f;
+            const float d1 = (keep >> (e + 1)) & 1u ? p1 * (dp[e + 1] * a.scale - Drs) : 0.f;
+            pk[e >> 1] = pack_bf16(d0, d1);
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float p0 = ex2(s[e] * a.scale_log2 - l2), p1 = ex2(s[e + 1] * a.scale_log2 - l2);
+            pk[e >> 1] = pack_bf16(p0 * (dp[e] * a.scale - Drs), p1 * (dp[e + 1] * a.scale - Drs));
+          }
         }
-      } else {
+        // dS (bf16, two per column) overwrites this group's own S columns already consumed
+        tmem_st16(tS + 64 * g + 16 * (c - 2 * g), pk);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bars->ds_full);
+    }
+    kc += n_kt;
+
+    if (it.has_rla) {
+      const int last = (kc - 1) & 1;
+      WAIT_OR_RETURN(bars->o_done, co & 1);                    // every window product done: K_cb is no longer read raw
+      ++co;
+      {
+        const int t2 = g * 128 + r;                              // two threads per key row
+        unsigned char* kh = smem + DQ_OFF_K + last * TILE_BYTES + (t2 & 1) * HALF_BYTES;
+        feature_map_pair(kh, kh, t2 >> 1);
+      }
+      fence_proxy_async_smem();
+      mbar_arrive(&bars->phik_ready);
+      WAIT_OR_RETURN(bars->s_full, cs & 1);
+      tc_fence_after();
+#pragma unroll 1
+      for (int c = 2 * g; c < 2 * g + 2; ++c) {
+        float x[32];
+        tmem_ld32(tS + 32 * c, x);
+        tmem_wait_ld();
+        const uint32_t keep = bits_lt(r - 32 * c);               // residual keys of row r in this chunk: j < r
+        uint32_t pk[16];
 #pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          const float p0 = ex2(s[e] * a.scale_log2 - l2), p1 = ex2(s[e + 1] * a.scale_log2 - l2);
-          pk[e >> 1] = pack_bf16(p0 * (dp[e] * a.scale - Drs), p1 * (dp[e + 1] * a.scale - Drs));
+        for (int e = 0; e < 32; e += 2)
+          pk[e >> 1] = pack_bf16((keep >> e) & 1u ? x[e] : 0.f, (keep >> (e + 1)) & 1u ? x[e + 1] : 0.f);
+        tmem_st16(tS + 64 * g + 16 * (c - 2 * g), pk);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bars->ds_full);
+      ++cs;
+      ++kc;
+    }
+
+    // ---- dq = dQ + phi(q) * (dphi_q - <dphi_q, phi(q)>) -----------------------------------
+    const int co_final = co++;
+    if (g != 0) continue;                                      // group 0 alone runs the epilogue
+    WAIT_OR_RETURN(bars->o_done, co_final & 1);
+    tc_fence_after();
+    float m = 0.f, inv = 0.f, dot = 0.f;
+    if (it.has_rla) {
+      m = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        const uint4 u = *reinterpret_cast<const uint4*>(sQ + swz(r, c));
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float2 f = __bfloat1622float2(h[e]);
+          m = fmaxf(m, fmaxf(f.x, f.y));
         }
       }
-      // dS (bf16, two per column) overwrites this group's own S columns already consumed
-      tmem_st16(tS + 64 * g + 16 * (c - 2 * g), pk);
-    }
-    tmem_wait_st();
-    tc_fence_before();
-    mbar_arrive(&bars->ds_full);
-  }
-
-  if (has_rla) {
-    const int last = (n_kt - 1) & 1;
-    WAIT_OR_RETURN(bars->dq_done, (n_kt - 1) & 1);           // K_cb is no longer read raw
-    {
-      const int t2 = g * 128 + r;                              // two threads per key row
-      unsigned char* kh = smem + DQ_OFF_K + last * TILE_BYTES + (t2 & 1) * HALF_BYTES;
-      feature_map_pair(kh, kh, t2 >> 1);
-    }
-    fence_proxy_async_smem();
-    mbar_arrive(&bars->phik_ready);
-    WAIT_OR_RETURN(bars->s_full, n_kt & 1);
-    tc_fence_after();
+      const float ml = m * LOG2E;
+      float sum = 0.f, du = 0.f;
 #pragma unroll 1
-    for (int c = 2 * g; c < 2 * g + 2; ++c) {
-      float x[32];
-      tmem_ld32(tS + 32 * c, x);
-      tmem_wait_ld();
-      const uint32_t keep = bits_lt(r - 32 * c);               // residual keys of row r in this chunk: j < r
-      uint32_t pk[16];
+      for (int c = 0; c < 4; ++c) {
+        float df[32];
+        tmem_ld32(tF + 32 * c, df);
+        tmem_wait_ld();
 #pragma unroll
-      for (int e = 0; e < 32; e += 2)
-        pk[e >> 1] = pack_bf16((keep >> e) & 1u ? x[e] : 0.f, (keep >> (e + 1)) & 1u ? x[e + 1] : 0.f);
-      tmem_st16(tS + 64 * g + 16 * (c - 2 * g), pk);
-    }
-    tmem_wait_st();
-    tc_fence_before();
-    mbar_arrive(&bars->ds_full);
-  }
-
-  // ---- dq = dQ + phi(q) * (dphi_q - <dphi_q, phi(q)>) -----------------------------------
-  if (g != 0) return true;
-  WAIT_OR_RETURN(bars->o_done, 0);
-  tc_fence_after();
-  const unsigned char* sQ = smem + DQ_OFF_Q;
-  float m = 0.f, inv = 0.f, dot = 0.f;
-  if (has_rla) {
-    m = -INFINITY;
+        for (int cc = 0; cc < 4; ++cc) {
+          const uint4 u = *reinterpret_cast<const uint4*>(sQ + swz(r, 4 * c + cc));
+          const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
-    for (int c = 0; c < 16; ++c) {
-      const uint4 u = *reinterpret_cast<const uint4*>(sQ + swz(r, c));
-      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 f = __bfloat1622float2(h[e]);
-        m = fmaxf(m, fmaxf(f.x, f.y));
+          for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(h[e]);
+            const float e0 = ex2(f.x * LOG2E - ml), e1 = ex2(f.y * LOG2E - ml);
+            sum += e0 + e1;
+            du += e0 * df[8 * cc + 2 * e] + e1 * df[8 * cc + 2 * e + 1];
+          }
+        }
       }
+      inv = 1.f / sum;
+      dot = du * inv;
+      m = ml;
     }
-    const float ml = m * LOG2E;
-    float sum = 0.f, du = 0.f;
+    // every product has completed: this item's Q buffer stages the output, each thread
+    // rewriting its own row in place, for one TMA store
 #pragma unroll 1
     for (int c = 0; c < 4; ++c) {
-      float df[32];
-      tmem_ld32(tF + 32 * c, df);
+      float x[32], df[32];
+      tmem_ld32(tQ + 32 * c, x);
+      if (it.has_rla) tmem_ld32(tF + 32 * c, df);
       tmem_wait_ld();
+      if (it.has_rla) {
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        const uint4 u = *reinterpret_cast<const uint4*>(sQ + swz(r, 4 * c + cc));
-        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+        for (int cc = 0; cc < 4; ++cc) {
+          const uint4 u = *reinterpret_cast<const uint4*>(sQ + swz(r, 4 * c + cc));
+          const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float2 f = __bfloat1622float2(h[e]);
-          const float e0 = ex2(f.x * LOG2E - ml), e1 = ex2(f.y * LOG2E - ml);
-          sum += e0 + e1;
-          du += e0 * df[8 * cc + 2 * e] + e1 * df[8 * cc + 2 * e + 1];
+          for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(h[e]);
+            const float e0 = ex2(f.x * LOG2E - m) * inv, e1 = ex2(f.y * LOG2E - m) * inv;
+            x[8 * cc + 2 * e] += e0 * (df[8 * cc + 2 * e] - dot);
+            x[8 * cc + 2 * e + 1] += e1 * (df[8 * cc + 2 * e + 1] - dot);
+          }
         }
       }
-    }
-    inv = 1.f / sum;
-    dot = du * inv;
-    m = ml;
-  }
-  // every product has completed: the dS tile is free and stages the output for one TMA store
-#pragma unroll 1
-  for (int c = 0; c < 4; ++c) {
-    float x[32], df[32];
-    tmem_ld32(tQ + 32 * c, x);
-    if (has_rla) tmem_ld32(tF + 32 * c, df);
-    tmem_wait_ld();
-    if (has_rla) {
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        const uint4 u = *reinterpret_cast<const uint4*>(sQ + swz(r, 4 * c + cc));
-        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float2 f = __bfloat1622float2(h[e]);
-          const float e0 = ex2(f.x * LOG2E - m) * inv, e1 = ex2(f.y * LOG2E - m) * inv;
-          x[8 * cc + 2 * e] += e0 * (df[8 * cc + 2 * e] - dot);
-          x[8 * cc + 2 * e + 1] += e1 * (df[8 * cc + 2 * e + 1] - dot);
-        }
+      for (int e = 0; e < 4; ++e) {
+        uint4 u;
+        u.x = pack_bf16(x[8 * e + 0], x[8 * e + 1]);
+        u.y = pack_bf16(x[8 * e + 2], x[8 * e + 3]);
+        u.z = pack_bf16(x[8 * e + 4], x[8 * e + 5]);
+        u.w = pack_bf16(x[8 * e + 6], x[8 * e + 7]);
+        *reinterpret_cast<uint4*>(sQ + swz(r, 4 * c + e)) = u;
       }
     }
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      uint4 u;
-      u.x = pack_bf16(x[8 * e + 0], x[8 * e + 1]);
-      u.y = pack_bf16(x[8 * e + 2], x[8 * e + 3]);
-      u.z = pack_bf16(x[8 * e + 4], x[8 * e + 5]);
-      u.w = pack_bf16(x[8 * e + 6], x[8 * e + 7]);
-      *reinterpret_cast<uint4*>(sD + swz(r, 4 * c + e)) = u;
+    fence_proxy_async_smem();
+    tc_fence_before();
+    rows_sync();
+    if (r == 0) {
+      store_tile(&tm.dq, sQ, it.q0, it.bh_q);
+      tma_store_commit();
+      tma_store_wait_read();
     }
+    rows_sync();
+    mbar_arrive(&bars->acc_free);          // dQ / dphi_q columns and this Q buffer may be reused
   }
-  fence_proxy_async_smem();
-  rows_sync();
-  if (r == 0) {
-    store_tile(tm_dq, sD, q0, bh_q);
-    tma_store_commit();
-    tma_store_wait_read();
-  }
-  tc_fence_before();
   return true;
 }
 
-__global__ void __launch_bounds__(288, 1)
-tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_gs,
-                 const __grid_constant__ CUtensorMap tm_gr, const __grid_constant__ CUtensorMap tm_st,
-                 const __grid_constant__ CUtensorMap tm_dq, BwdArgs a) {
+__global__ void __launch_bounds__(DQ_THREADS, 1)
+tc_bwd_dq_kernel(const __grid_constant__ DqMaps tm, BwdArgs a, int n_items, int n_qt) {
   extern __shared__ __align__(1024) unsigned char smem[];
   DqBars* bars = reinterpret_cast<DqBars*>(smem + DQ_OFF_BAR);
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -419,31 +487,17 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     if (tid == 0 && a.status) atomicExch(a.status, 2);
     return;
   }
-  const int n_qt = (a.T + TILE - 1) / TILE;
-  const int qt = n_qt - 1 - (int)blockIdx.x;
-  const int q0 = qt * TILE;
-  const int bh_q = blockIdx.y;
-  const int b = bh_q / a.H_q, h = bh_q % a.H_q;
-  const int bh_kv = b * (a.H_q / a.group) + h / a.group;
-  const int wt = a.w / TILE;
-  const bool has_boundary = (a.mode != RATTN_MODE_FULL_CAUSAL) && (qt - wt >= 0);
-  const int n_kt = (has_boundary ? wt : qt) + 1;
-  const bool has_rla = has_boundary && (a.mode == RATTN_MODE_RATTN);
-  const int cb = qt - wt;
-  const bool has_state = has_rla && cb > 0;
-  const int st_index = bh_kv * a.n_chunks + (cb > 0 ? cb : 0);
-
   if (tid == 0) {
     mbar_init(&bars->qg_full, 1);
-    mbar_init(&bars->kv_full[0], 1);
-    mbar_init(&bars->kv_full[1], 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bars->kv_full[i], 1);
+      mbar_init(&bars->kv_free[i], 1);
+    }
     mbar_init(&bars->s_full, 1);
-    mbar_init(&bars->s_empty, 128);
     mbar_init(&bars->ds_full, 256);
-    mbar_init(&bars->dq_done, 1);
-    mbar_init(&bars->x_full, 1);
     mbar_init(&bars->phik_ready, 256);
     mbar_init(&bars->o_done, 1);
+    mbar_init(&bars->acc_free, 128);
     mbar_init(&bars->drain, 1);
     bars->abort = 0;
     fence_mbar_init();
@@ -451,15 +505,15 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   if (warp == 8) {
     tmem_alloc(&bars->tmem_base, 512);
     tmem_relinquish();
-    if (tid == 256) {
-      prefetch_tensormap(&tm_q);
-      prefetch_tensormap(&tm_k);
-      prefetch_tensormap(&tm_v);
-      prefetch_tensormap(&tm_gs);
-      prefetch_tensormap(&tm_gr);
-      prefetch_tensormap(&tm_st);
-      prefetch_tensormap(&tm_dq);
-    }
+  }
+  if (tid == 288) {
+    prefetch_tensormap(&tm.q);
+    prefetch_tensormap(&tm.k);
+    prefetch_tensormap(&tm.v);
+    prefetch_tensormap(&tm.gs);
+    prefetch_tensormap(&tm.gr);
+    prefetch_tensormap(&tm.st);
+    prefetch_tensormap(&tm.dq);
   }
   tc_fence_before();
   __syncthreads();
@@ -468,14 +522,15 @@ tc_bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 
   bool ok = true;
   if (warp < 8) {
-    ok = dq_rows(a, &tm_dq, smem, bars, tmem, warp >> 2, tid & 127, q0, bh_q, n_kt, has_boundary, has_rla);
+    ok = dq_rows(tm, a, smem, bars, tmem, warp >> 2, tid & 127, n_items, n_qt);
   } else if (warp == 8) {
-    ok = dq_control(&tm_q, &tm_k, &tm_v, &tm_gs, &tm_gr, &tm_st, smem, bars, tmem, q0, bh_q, bh_kv, n_kt,
-                    has_rla, has_state, st_index);
+    ok = dq_mma(a, smem, bars, tmem, n_items, n_qt);
     if (!ok) {
       mma_commit(&bars->drain);
       for (int it = 0; it < (1 << 16) && !mbar_try_wait(&bars->drain, 0); ++it) {}
     }
+  } else {
+    ok = dq_loader(tm, a, smem, bars, n_items, n_qt);
   }
   if (!ok && a.status) atomicExch(a.status, 1);
   tc_fence_before();
@@ -933,8 +988,16 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
   e = cudaFuncSetAttribute(tc_bwd_dkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, KV_SMEM);
   if (e != cudaSuccess) return e;
   {
+    DqMaps dm;
+    dm.q = tm_q; dm.k = tm_k; dm.v = tm_v; dm.gs = tm_gs; dm.gr = tm_gr; dm.st = tm_st; dm.dq = tm_dq;
+    int dev = 0, n_sm = 0;
+    e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    const int n_items = n_qt * (int)nq;
     KernelTimer kt("tc_bwd_dq", s);
-    tc_bwd_dq_kernel<<<dim3(n_qt, (unsigned)nq), 288, DQ_SMEM, s>>>(tm_q, tm_k, tm_v, tm_gs, tm_gr, tm_st, tm_dq, t);
+    tc_bwd_dq_kernel<<<n_items < n_sm ? n_items : n_sm, DQ_THREADS, DQ_SMEM, s>>>(dm, t, n_items, n_qt);
   }
   KvMaps km;
   km.k = tm_k; km.v = tm_v; km.rs = tm_rs; km.dk = tm_dk; km.dv = tm_dv;
