@@ -556,155 +556,224 @@ tc_bwd_dq_kernel(const __grid_constant__ DqMaps tm, BwdArgs a, int n_items, int 
 // The residual items run first and leave dphi_k in the dK accumulator; row group 0 then folds
 // the feature-map Jacobian into it (dK := phi(k) (dphi_k - <dphi_k, phi(k)>)) and the window
 // items accumulate on top.
-constexpr int KV_NS = 4;                                   // item stages
+constexpr int KV_NS = 3;                                   // item stages
 constexpr int KV_OFF_K = 0;
 constexpr int KV_OFF_V = 1 * TILE_BYTES;
-constexpr int KV_OFF_KPHI = 2 * TILE_BYTES;
-constexpr int KV_OFF_STAGE = 3 * TILE_BYTES;               // KV_NS x [Q_h 16 KB | g_h 16 KB]
+constexpr int KV_OFF_KPHI = 2 * TILE_BYTES;                // phi(K_j); stages dK at the end of an item
+constexpr int KV_OFF_OUT = 3 * TILE_BYTES;                 // stages dV at the end of an item
+constexpr int KV_OFF_STAGE = 4 * TILE_BYTES;               // KV_NS x [Q_h 16 KB | g_h 16 KB]
 constexpr int KV_OFF_STAT = KV_OFF_STAGE + KV_NS * TILE_BYTES;   // KV_NS x (lse2[64], D*scale[64]) fp32
 constexpr int KV_OFF_BAR = KV_OFF_STAT + KV_NS * 512;
 constexpr int KV_SMEM = KV_OFF_BAR + 256;
-constexpr int KV_THREADS = 576;                            // 4 row groups, MMA warp, loader warp
+constexpr int KV_THREADS = 320;                            // 2 row groups, MMA warp, loader warp
 
 struct KvBars {
   uint64_t kv_full, kphi_ready, full[KV_NS], acc_done[KV_NS], s_full[2], p_ready[2], phiq_ready[2],
-      r_acc_done, fold_done, all_done, drain;
+      r_acc_done, fold_done, all_done, acc_free, drain;
   uint32_t tmem_base;
   int abort;
 };
 
+struct KvMaps {
+  CUtensorMap k, v, rs, qh, gsh, grh, dk, dv;
+};
+
+// One key tile (j, K/V head) of the persistent CTA's work list, and how its half-tile items
+// are numbered.  Counters that run on across key tiles (ring slots, TMEM slots, barrier
+// phases) are kept by every role in the same way.
 struct KvPlan {
-  int j, n_qt, wt, group, n_R, n_s_tiles, N, off;
+  int j, bh_kv, rs_index, n_qt, wt, group, n_R, n_s_tiles, N;
   bool windowed, has_inter;
   __device__ bool is_r(int n) const { return n < n_R; }
   __device__ int head(int n) const { return n < n_R ? (n >> 1) : (n - n_R) / (2 * n_s_tiles); }
   __device__ int qtile(int n) const { return n < n_R ? j + wt : j + (((n - n_R) % (2 * n_s_tiles)) >> 1); }
   __device__ int half(int n) const { return n < n_R ? (n & 1) : ((n - n_R) & 1); }
-  __device__ int stage(int n) const { return (n + off) % KV_NS; }
-  __device__ int use(int n) const { return (n + off) / KV_NS; }
 };
 
-__device__ bool kv_loader(const CUtensorMap* tm_k, const CUtensorMap* tm_v, const CUtensorMap* tm_rs,
-                          const CUtensorMap* tm_qh, const CUtensorMap* tm_gsh, const CUtensorMap* tm_grh,
-                          const float* lse2p, const float* dscp, int t_pad, unsigned char* smem, KvBars* bars,
-                          const KvPlan& pl, int bh_kv, int rs_index) {
-  const int j0 = pl.j * TILE;
-  mbar_arrive_expect_tx(&bars->kv_full, 2 * TILE_BYTES);
-  load_tile(smem + KV_OFF_K, tm_k, &bars->kv_full, j0, bh_kv);
-  load_tile(smem + KV_OFF_V, tm_v, &bars->kv_full, j0, bh_kv);
-  if (pl.has_inter) {
-    mbar_arrive_expect_tx(&bars->full[0], TILE_BYTES);
-    load_tile(smem + KV_OFF_STAGE, tm_rs, &bars->full[0], 0, rs_index);
-  }
-  for (int n = 0; n < pl.N; ++n) {
-    const int st = pl.stage(n), u = pl.use(n);
-    if (u >= 1) WAIT_OR_RETURN_W(bars->acc_done[st], (u - 1) & 1);
-    unsigned char* dst = smem + KV_OFF_STAGE + st * TILE_BYTES;
-    const int z = bh_kv * pl.group + pl.head(n);
-    const int row = pl.qtile(n) * TILE + 64 * pl.half(n);
-    if (pl.is_r(n)) {
-      mbar_arrive_expect_tx(&bars->full[st], 2 * HT_BYTES);
-      load_half_tile(dst, tm_qh, &bars->full[st], row, z);
-      load_half_tile(dst + HT_BYTES, tm_grh, &bars->full[st], row, z);
-    } else {
-      mbar_arrive_expect_tx(&bars->full[st], 2 * HT_BYTES + 512);
-      load_half_tile(dst, tm_qh, &bars->full[st], row, z);
-      load_half_tile(dst + HT_BYTES, tm_gsh, &bars->full[st], row, z);
-      float* stat = reinterpret_cast<float*>(smem + KV_OFF_STAT + st * 512);
-      bulk_load_1d(stat, lse2p + (size_t)z * t_pad + row, 256, &bars->full[st]);
-      bulk_load_1d(stat + 64, dscp + (size_t)z * t_pad + row, 256, &bars->full[st]);
+__device__ __forceinline__ KvPlan kv_plan(const BwdArgs& a, int idx) {
+  KvPlan pl;
+  pl.n_qt = (a.T + TILE - 1) / TILE;
+  pl.bh_kv = idx / pl.n_qt;
+  pl.j = idx % pl.n_qt;
+  pl.rs_index = pl.bh_kv * a.n_chunks + pl.j;
+  pl.wt = a.w / TILE;
+  pl.group = a.group;
+  pl.windowed = (a.mode != RATTN_MODE_FULL_CAUSAL);
+  const int i_hi = (pl.windowed && pl.j + pl.wt < pl.n_qt - 1) ? pl.j + pl.wt : pl.n_qt - 1;
+  pl.n_s_tiles = i_hi - pl.j + 1;
+  const bool r_tile = pl.windowed && (a.mode == RATTN_MODE_RATTN) && (pl.j + pl.wt <= pl.n_qt - 1);
+  pl.n_R = r_tile ? 2 * a.group : 0;
+  pl.has_inter = r_tile && (pl.j + pl.wt + 1 <= pl.n_qt - 1);
+  pl.N = pl.n_R + 2 * a.group * pl.n_s_tiles;
+  return pl;
+}
+
+// running counters shared by the three roles: key tiles done, ring slots used, half-tile items
+// done, key tiles with residual items done
+struct KvCount {
+  int it, seq, gi, cr;
+};
+
+__device__ bool kv_loader(const KvMaps& tm, const BwdArgs& a, unsigned char* smem, KvBars* bars, int n_items) {
+  KvCount c = {0, 0, 0, 0};
+  for (int idx = blockIdx.x; idx < n_items; idx += gridDim.x, ++c.it) {
+    const KvPlan pl = kv_plan(a, idx);
+    const int j0 = pl.j * TILE;
+    // K_j, V_j replace the previous key tile's once every product that read them has completed
+    if (c.it >= 1) WAIT_OR_RETURN_W(bars->all_done, (c.it - 1) & 1);
+    mbar_arrive_expect_tx(&bars->kv_full, 2 * TILE_BYTES);
+    load_tile(smem + KV_OFF_K, &tm.k, &bars->kv_full, j0, pl.bh_kv);
+    load_tile(smem + KV_OFF_V, &tm.v, &bars->kv_full, j0, pl.bh_kv);
+    auto ring = [&](int& st) -> bool {                     // next ring slot, once its previous user is consumed
+      st = c.seq % KV_NS;
+      const int use = c.seq / KV_NS;
+      if (use >= 1) WAIT_OR_RETURN_W(bars->acc_done[st], (use - 1) & 1);
+      ++c.seq;
+      return true;
+    };
+    if (pl.has_inter) {
+      int st;
+      if (!ring(st)) return false;
+      mbar_arrive_expect_tx(&bars->full[st], TILE_BYTES);
+      load_tile(smem + KV_OFF_STAGE + st * TILE_BYTES, &tm.rs, &bars->full[st], 0, pl.rs_index);
+    }
+    for (int n = 0; n < pl.N; ++n) {
+      int st;
+      if (!ring(st)) return false;
+      unsigned char* dst = smem + KV_OFF_STAGE + st * TILE_BYTES;
+      const int z = pl.bh_kv * pl.group + pl.head(n);
+      const int row = pl.qtile(n) * TILE + 64 * pl.half(n);
+      if (pl.is_r(n)) {
+        mbar_arrive_expect_tx(&bars->full[st], 2 * HT_BYTES);
+        load_half_tile(dst, &tm.qh, &bars->full[st], row, z);
+        load_half_tile(dst + HT_BYTES, &tm.grh, &bars->full[st], row, z);
+      } else {
+        mbar_arrive_expect_tx(&bars->full[st], 2 * HT_BYTES + 512);
+        load_half_tile(dst, &tm.qh, &bars->full[st], row, z);
+        load_half_tile(dst + HT_BYTES, &tm.gsh, &bars->full[st], row, z);
+        float* stat = reinterpret_cast<float*>(smem + KV_OFF_STAT + st * 512);
+        bulk_load_1d(stat, a.lse2p + (size_t)z * a.t_pad + row, 256, &bars->full[st]);
+        bulk_load_1d(stat + 64, a.dscp + (size_t)z * a.t_pad + row, 256, &bars->full[st]);
+      }
     }
   }
   return true;
 }
 
-__device__ bool kv_mma(unsigned char* smem, KvBars* bars, uint32_t tmem, const KvPlan& pl) {
+__device__ bool kv_mma(const BwdArgs& a, unsigned char* smem, KvBars* bars, uint32_t tmem, int n_items) {
   const uint32_t sK = smem_u32(smem + KV_OFF_K), sV = smem_u32(smem + KV_OFF_V), sKphi = smem_u32(smem + KV_OFF_KPHI);
   const uint32_t sStage = smem_u32(smem + KV_OFF_STAGE);
   const uint32_t tV = tmem, tK = tmem + 128;
   const uint32_t tS[2] = {tmem + 256, tmem + 384}, tP[2] = {tmem + 320, tmem + 448};
-  bool accV = false, accK = false;
+  KvCount c = {0, 0, 0, 0};
+  int cq[2] = {0, 0};                                      // phi(Q_h) hand-overs per TMEM slot
 
-  WAIT_OR_RETURN_W(bars->kv_full, 0);
-  if (pl.n_R > 0) WAIT_OR_RETURN_W(bars->kphi_ready, 0);
-  if (pl.has_inter) {
-    WAIT_OR_RETURN_W(bars->full[0], 0);
-    tc_fence_after();
-    mma_kk(tK, sV, sStage, false);                         // dphi_k = V_j R_j^T
-    mma_kmn<1>(tV, sKphi, sStage, false);                  // dV     = phi(K_j) R_j
-    mma_commit(&bars->acc_done[0]);
-    accV = accK = true;
-  }
-  for (int n = 0; n <= pl.N; ++n) {
-    if (n < pl.N) {
-      const int st = pl.stage(n), slot = n & 1;
-      const uint32_t sQh = sStage + st * TILE_BYTES, sGh = sQh + HT_BYTES;
-      WAIT_OR_RETURN_W(bars->full[st], pl.use(n) & 1);
-      if (pl.is_r(n)) WAIT_OR_RETURN_W(bars->phiq_ready[slot], (n >> 1) & 1);
-      // The slot's previous user (item n-2) needs no wait here: its row groups were waited for
-      // before its accumulate products were issued, and those precede these scores in the
-      // tensor pipe, which executes in issue order.
+  for (int idx = blockIdx.x; idx < n_items; idx += gridDim.x, ++c.it) {
+    const KvPlan pl = kv_plan(a, idx);
+    bool accV = false, accK = false;
+    WAIT_OR_RETURN_W(bars->kv_full, c.it & 1);
+    if (pl.n_R > 0) WAIT_OR_RETURN_W(bars->kphi_ready, c.cr & 1);
+    // the previous key tile's epilogue has read the two accumulators
+    bool acc_ok = (c.it == 0);
+    if (pl.has_inter) {
+      const int st = c.seq % KV_NS, use = c.seq / KV_NS;
+      ++c.seq;
+      WAIT_OR_RETURN_W(bars->full[st], use & 1);
+      if (!acc_ok) { WAIT_OR_RETURN_W(bars->acc_free, (c.it - 1) & 1); acc_ok = true; }
       tc_fence_after();
-      mma_k_kh(tS[slot], pl.is_r(n) ? sKphi : sK, sQh);   // S^T  = K Q_h^T   (phi(K) phi(Q_h)^T)
-      mma_k_kh(tP[slot], sV, sGh);                         // dP^T = V g_h^T
-      mma_commit(&bars->s_full[slot]);
-    }
-    if (n >= 1) {
-      const int m = n - 1, st = pl.stage(m), slot = m & 1;
-      const uint32_t sQh = sStage + st * TILE_BYTES, sGh = sQh + HT_BYTES;
-      WAIT_OR_RETURN_W(bars->p_ready[slot], (m >> 1) & 1);
-      if (m == pl.n_R && pl.n_R > 0) WAIT_OR_RETURN_W(bars->fold_done, 0);
-      tc_fence_after();
-      mma_ts_h(tV, tS[slot], sGh, accV);                   // dV += P^T g_h
-      mma_ts_h(tK, tP[slot], sQh, accK);                   // dK += dS^T Q_h   (dphi_k += dA^T phi(Q_h))
-      accV = accK = true;
+      mma_kk(tK, sV, sStage + st * TILE_BYTES, false);     // dphi_k = V_j R_j^T
+      mma_kmn<1>(tV, sKphi, sStage + st * TILE_BYTES, false);   // dV     = phi(K_j) R_j
       mma_commit(&bars->acc_done[st]);
-      if (m == pl.n_R - 1) mma_commit(&bars->r_acc_done);
+      accV = accK = true;
     }
+    const int seq0 = c.seq, gi0 = c.gi;
+    for (int n = 0; n <= pl.N; ++n) {
+      if (n < pl.N) {
+        const int st = (seq0 + n) % KV_NS, use = (seq0 + n) / KV_NS, slot = (gi0 + n) & 1;
+        const uint32_t sQh = sStage + st * TILE_BYTES, sGh = sQh + HT_BYTES;
+        WAIT_OR_RETURN_W(bars->full[st], use & 1);
+        if (pl.is_r(n)) {
+          WAIT_OR_RETURN_W(bars->phiq_ready[slot], cq[slot] & 1);
+          ++cq[slot];
+        }
+        // The slot's previous user needs no wait here: its row groups were waited for before its
+        // accumulate products were issued, and those precede these scores in the tensor pipe,
+        // which executes in issue order.
+        tc_fence_after();
+        mma_k_kh(tS[slot], pl.is_r(n) ? sKphi : sK, sQh);   // S^T  = K Q_h^T   (phi(K) phi(Q_h)^T)
+        mma_k_kh(tP[slot], sV, sGh);                         // dP^T = V g_h^T
+        mma_commit(&bars->s_full[slot]);
+      }
+      if (n >= 1) {
+        const int m = n - 1, st = (seq0 + m) % KV_NS, slot = (gi0 + m) & 1;
+        const uint32_t sQh = sStage + st * TILE_BYTES, sGh = sQh + HT_BYTES;
+        WAIT_OR_RETURN_W(bars->p_ready[slot], ((gi0 + m) >> 1) & 1);
+        if (m == pl.n_R && pl.n_R > 0) WAIT_OR_RETURN_W(bars->fold_done, c.cr & 1);
+        if (!acc_ok) { WAIT_OR_RETURN_W(bars->acc_free, (c.it - 1) & 1); acc_ok = true; }
+        tc_fence_after();
+        mma_ts_h(tV, tS[slot], sGh, accV);                   // dV += P^T g_h
+        mma_ts_h(tK, tP[slot], sQh, accK);                   // dK += dS^T Q_h   (dphi_k += dA^T phi(Q_h))
+        accV = accK = true;
+        mma_commit(&bars->acc_done[st]);
+        if (m == pl.n_R - 1) mma_commit(&bars->r_acc_done);
+      }
+    }
+    c.seq += pl.N;
+    c.gi += pl.N;
+    if (pl.n_R > 0) ++c.cr;
+    mma_commit(&bars->all_done);
   }
-  mma_commit(&bars->all_done);
   return true;
 }
 
-__device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtensorMap* tm_dv, unsigned char* smem,
-                        KvBars* bars, uint32_t tmem, const KvPlan& pl, int gg, int r, int bh_kv) {
-  // four groups of 128 threads (thread = key row = TMEM lane): groups 0,1 serve TMEM slot 0,
-  // groups 2,3 slot 1; within a slot the even group takes query columns 0..31 of the item,
-  // the odd group columns 32..63
-  const int g = gg >> 1, c = gg & 1;
+__device__ bool kv_rows(const KvMaps& tm, const BwdArgs& a, unsigned char* smem, KvBars* bars, uint32_t tmem, int gg,
+                        int r, int n_items) {
+  // two groups of 128 threads (thread = key row = TMEM lane), one per TMEM slot; a thread takes
+  // all 64 query columns of its item, 32 at a time (more row groups per slot measured no faster
+  // and cost registers)
+  const int g = gg;
   const uint32_t lane_off = (uint32_t)((r & ~31) << 16);
   const uint32_t tV = tmem + lane_off, tK = tmem + 128 + lane_off;
   const uint32_t tS = tmem + 256 + 128 * g + lane_off, tP = tS + 64;
   const unsigned char* sKphi = smem + KV_OFF_KPHI;
+  KvCount cnt = {0, 0, 0, 0};
 
-  WAIT_OR_RETURN(bars->kv_full, 0);
-  if (pl.n_R > 0 && gg < 2) {
-    // phi(K_j) into its own tile: 256 threads, two per row
-    const int t2 = gg * 128 + r, row = t2 >> 1, hf = t2 & 1;
-    feature_map_pair(smem + KV_OFF_K + hf * HALF_BYTES, smem + KV_OFF_KPHI + hf * HALF_BYTES, row);
-    fence_proxy_async_smem();
-    mbar_arrive(&bars->kphi_ready);
+  for (int idx = blockIdx.x; idx < n_items; idx += gridDim.x) {
+  const KvPlan pl = kv_plan(a, idx);
+  const int bh_kv = pl.bh_kv;
+  if (gg < 2) {
+    WAIT_OR_RETURN(bars->kv_full, cnt.it & 1);
+    if (pl.n_R > 0) {
+      // phi(K_j) into its own tile: 256 threads, two per row
+      const int t2 = gg * 128 + r, row = t2 >> 1, hf = t2 & 1;
+      feature_map_pair(smem + KV_OFF_K + hf * HALF_BYTES, smem + KV_OFF_KPHI + hf * HALF_BYTES, row);
+      fence_proxy_async_smem();
+      mbar_arrive(&bars->kphi_ready);
+    }
   }
+  const int seq0 = cnt.seq + (pl.has_inter ? 1 : 0), gi0 = cnt.gi;
 
-  for (int n = g; n < pl.N; n += 2) {
-    const int st = pl.stage(n);
+  for (int n = 0; n < pl.N; ++n) {
+    if (((gi0 + n) & 1) != g) continue;                       // the other TMEM slot's item
+    const int st = (seq0 + n) % KV_NS, use = (seq0 + n) / KV_NS;
     const bool is_r = pl.is_r(n);
     const int i = pl.qtile(n), hf = pl.half(n);
     unsigned char* sQh = smem + KV_OFF_STAGE + st * TILE_BYTES;
-    WAIT_OR_RETURN(bars->full[st], pl.use(n) & 1);
-    if (is_r && c == 0) {
-      // phi(Q_h) in place: 64 rows, two threads per row (the slot's even group)
+    WAIT_OR_RETURN(bars->full[st], use & 1);
+    if (is_r) {
+      // phi(Q_h) in place: 64 rows, two threads per row
       const int row = r >> 1, ch = r & 1;
       feature_map_pair(sQh + ch * HT_HALF, sQh + ch * HT_HALF, row);
       fence_proxy_async_smem();
       mbar_arrive(&bars->phiq_ready[g]);
     }
-    WAIT_OR_RETURN(bars->s_full[g], (n >> 1) & 1);
+    WAIT_OR_RETURN(bars->s_full[g], ((gi0 + n) >> 1) & 1);
     tc_fence_after();
     const bool diag = !is_r && (i == pl.j), bound = !is_r && pl.windowed && (i == pl.j + pl.wt);
     const float* l2 = reinterpret_cast<const float*>(smem + KV_OFF_STAT + st * 512);
     const float* Ds = l2 + 64;
-    {
+#pragma unroll 1
+    for (int c = 0; c < 2; ++c) {                              // rolled: compact code
       float s[32], dp[32];
       tmem_ld32(tS + 32 * c, s);
       tmem_ld32(tP + 32 * c, dp);
@@ -759,7 +828,7 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
           pk2[(e4 >> 1) + 1] = pack_bf16(d[2], d[3]);
         }
       }
-      // bf16 results (two per column) overwrite the first half of this group's own columns
+      // bf16 results (two per column) overwrite the first half of the chunk just consumed
       tmem_st16(tS + 32 * c, pk1);
       tmem_st16(tP + 32 * c, pk2);
     }
@@ -767,9 +836,9 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
     tc_fence_before();
     mbar_arrive(&bars->p_ready[g]);
 
-    if (gg == 0 && pl.n_R > 0 && n == pl.n_R - 2) {
+    if (gg == 0 && is_r && n + 2 >= pl.n_R) {                   // group 0's last residual item of this key tile
       // end of the residual items: dK := phi(k) (dphi_k - <dphi_k, phi(k)>)
-      WAIT_OR_RETURN(bars->r_acc_done, 0);
+      WAIT_OR_RETURN(bars->r_acc_done, cnt.cr & 1);
       tc_fence_after();
       float dot = 0.f;
 #pragma unroll 1
@@ -812,45 +881,51 @@ __device__ bool kv_rows(const BwdArgs& a, const CUtensorMap* tm_dk, const CUtens
     }
   }
 
-  // every product has completed: group 0 stores dK, group 1 dV, each staged in one of
-  // the (now free) item stages and written by one TMA store
-  if (gg >= 2) return true;
-  WAIT_OR_RETURN(bars->all_done, 0);
-  tc_fence_after();
-  unsigned char* sOut = smem + KV_OFF_STAGE + gg * TILE_BYTES;
-  const uint32_t tOut = gg == 0 ? tK : tV;
+  // every product has completed: group 0 stores dK (staged in the phi(K) tile), group 1 dV
+  // (staged in its own tile), each written by one TMA store
+  if (gg < 2) {
+    WAIT_OR_RETURN(bars->all_done, cnt.it & 1);
+    tc_fence_after();
+    unsigned char* sOut = smem + (gg == 0 ? KV_OFF_KPHI : KV_OFF_OUT);
+    const uint32_t tOut = gg == 0 ? tK : tV;
 #pragma unroll 1
-  for (int c = 0; c < 4; ++c) {
-    float x[32];
-    tmem_ld32(tOut + 32 * c, x);
-    tmem_wait_ld();
+    for (int cc = 0; cc < 4; ++cc) {
+      float x[32];
+      tmem_ld32(tOut + 32 * cc, x);
+      tmem_wait_ld();
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      uint4 u;
-      u.x = pack_bf16(x[8 * e + 0], x[8 * e + 1]);
-      u.y = pack_bf16(x[8 * e + 2], x[8 * e + 3]);
-      u.z = pack_bf16(x[8 * e + 4], x[8 * e + 5]);
-      u.w = pack_bf16(x[8 * e + 6], x[8 * e + 7]);
-      *reinterpret_cast<uint4*>(sOut + swz(r, 4 * c + e)) = u;
+      for (int e = 0; e < 4; ++e) {
+        uint4 u;
+        u.x = pack_bf16(x[8 * e + 0], x[8 * e + 1]);
+        u.y = pack_bf16(x[8 * e + 2], x[8 * e + 3]);
+        u.z = pack_bf16(x[8 * e + 4], x[8 * e + 5]);
+        u.w = pack_bf16(x[8 * e + 6], x[8 * e + 7]);
+        *reinterpret_cast<uint4*>(sOut + swz(r, 4 * cc + e)) = u;
+      }
     }
+    fence_proxy_async_smem();
+    tc_fence_before();
+    group_sync(gg);
+    if (r == 0) {
+      store_tile(gg == 0 ? &tm.dk : &tm.dv, sOut, pl.j * TILE, bh_kv);
+      tma_store_commit();
+      tma_store_wait_read();
+    }
+    // both staging tiles have been read by their stores before either group goes on (the next
+    // key tile's phi(K) is written by both groups into the tile that staged dK)
+    asm volatile("bar.sync 6, 256;" ::: "memory");
+    mbar_arrive(&bars->acc_free);
   }
-  fence_proxy_async_smem();
-  group_sync(gg);
-  if (r == 0) {
-    store_tile(gg == 0 ? tm_dk : tm_dv, sOut, pl.j * TILE, bh_kv);
-    tma_store_commit();
-    tma_store_wait_read();
+  cnt.seq = seq0 + pl.N;
+  cnt.gi += pl.N;
+  if (pl.n_R > 0) ++cnt.cr;
+  ++cnt.it;
   }
-  tc_fence_before();
   return true;
 }
 
-struct KvMaps {
-  CUtensorMap k, v, rs, qh, gsh, grh, dk, dv;
-};
-
 __global__ void __launch_bounds__(KV_THREADS, 1)
-tc_bwd_dkv_kernel(const __grid_constant__ KvMaps tm, BwdArgs a) {
+tc_bwd_dkv_kernel(const __grid_constant__ KvMaps tm, BwdArgs a, int n_items) {
   extern __shared__ __align__(1024) unsigned char smem[];
   KvBars* bars = reinterpret_cast<KvBars*>(smem + KV_OFF_BAR);
   const int tid = threadIdx.x, warp = tid >> 5;
@@ -858,22 +933,6 @@ tc_bwd_dkv_kernel(const __grid_constant__ KvMaps tm, BwdArgs a) {
     if (tid == 0 && a.status) atomicExch(a.status, 2);
     return;
   }
-  KvPlan pl;
-  pl.n_qt = (a.T + TILE - 1) / TILE;
-  pl.j = blockIdx.x;
-  pl.wt = a.w / TILE;
-  pl.group = a.group;
-  pl.windowed = (a.mode != RATTN_MODE_FULL_CAUSAL);
-  const int i_hi = (pl.windowed && pl.j + pl.wt < pl.n_qt - 1) ? pl.j + pl.wt : pl.n_qt - 1;
-  pl.n_s_tiles = i_hi - pl.j + 1;
-  const bool r_tile = pl.windowed && (a.mode == RATTN_MODE_RATTN) && (pl.j + pl.wt <= pl.n_qt - 1);
-  pl.n_R = r_tile ? 2 * a.group : 0;
-  pl.has_inter = r_tile && (pl.j + pl.wt + 1 <= pl.n_qt - 1);
-  pl.off = pl.has_inter ? 1 : 0;
-  pl.N = pl.n_R + 2 * a.group * pl.n_s_tiles;
-  const int bh_kv = blockIdx.y;
-  const int rs_index = bh_kv * a.n_chunks + pl.j;
-
   if (tid == 0) {
     mbar_init(&bars->kv_full, 1);
     mbar_init(&bars->kphi_ready, 256);
@@ -883,27 +942,30 @@ tc_bwd_dkv_kernel(const __grid_constant__ KvMaps tm, BwdArgs a) {
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bars->s_full[i], 1);
-      mbar_init(&bars->p_ready[i], 256);
+      mbar_init(&bars->p_ready[i], 128);
       mbar_init(&bars->phiq_ready[i], 128);
     }
     mbar_init(&bars->r_acc_done, 1);
     mbar_init(&bars->fold_done, 128);
     mbar_init(&bars->all_done, 1);
+    mbar_init(&bars->acc_free, 256);
     mbar_init(&bars->drain, 1);
     bars->abort = 0;
     fence_mbar_init();
   }
-  if (warp == 16) {
+  if (warp == 8) {
     tmem_alloc(&bars->tmem_base, 512);
     tmem_relinquish();
   }
-  if (tid == 544) {
+  if (tid == 288) {
     prefetch_tensormap(&tm.k);
     prefetch_tensormap(&tm.v);
     prefetch_tensormap(&tm.rs);
     prefetch_tensormap(&tm.qh);
     prefetch_tensormap(&tm.gsh);
     prefetch_tensormap(&tm.grh);
+    prefetch_tensormap(&tm.dk);
+    prefetch_tensormap(&tm.dv);
   }
   tc_fence_before();
   __syncthreads();
@@ -911,22 +973,21 @@ tc_bwd_dkv_kernel(const __grid_constant__ KvMaps tm, BwdArgs a) {
   const uint32_t tmem = bars->tmem_base;
 
   bool ok = true;
-  if (warp < 16) {
-    ok = kv_rows(a, &tm.dk, &tm.dv, smem, bars, tmem, pl, warp >> 2, tid & 127, bh_kv);
-  } else if (warp == 16) {
-    ok = kv_mma(smem, bars, tmem, pl);
+  if (warp < 8) {
+    ok = kv_rows(tm, a, smem, bars, tmem, warp >> 2, tid & 127, n_items);
+  } else if (warp == 8) {
+    ok = kv_mma(a, smem, bars, tmem, n_items);
     if (!ok) {
       mma_commit(&bars->drain);
       for (int it = 0; it < (1 << 16) && !mbar_try_wait(&bars->drain, 0); ++it) {}
     }
-  } else if (warp == 17) {
-    ok = kv_loader(&tm.k, &tm.v, &tm.rs, &tm.qh, &tm.gsh, &tm.grh, a.lse2p, a.dscp, a.t_pad, smem, bars, pl,
-                   bh_kv, rs_index);
+  } else if (warp == 9) {
+    ok = kv_loader(tm, a, smem, bars, n_items);
   }
   if (!ok && a.status) atomicExch(a.status, 1);
   tc_fence_before();
   __syncthreads();
-  if (warp == 16) {
+  if (warp == 8) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
   }
@@ -1004,8 +1065,14 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
   if (!make_map(&km.qh, a.q, a.T, nq, 64) || !make_map(&km.gsh, g_s, a.T, nq, 64) || !make_map(&km.grh, g_r, a.T, nq, 64))
     return cudaErrorInvalidValue;
   {
+    int dev = 0, n_sm = 0;
+    e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    const int n_items = n_qt * (int)nkv;
     KernelTimer kt("tc_bwd_dkv", s);
-    tc_bwd_dkv_kernel<<<dim3(n_qt, (unsigned)nkv), KV_THREADS, KV_SMEM, s>>>(km, t);
+    tc_bwd_dkv_kernel<<<n_items < n_sm ? n_items : n_sm, KV_THREADS, KV_SMEM, s>>>(km, t, n_items);
   }
   count_launches(2);
   return cudaGetLastError();
