@@ -185,3 +185,15 @@ def test_tensor_backward_determinism():
     b = R.rattn_backward_ex(q, k, v, dy, wl.w, ws, scale=wl.scale)
     for x, y in zip(a, b):
         assert torch.equal(x, y)
+
+
+def test_tensor_paths_with_several_items_per_cta():
+    """More (head, tile) items than the GPU has SMs, ragged T, a group of four query heads per
+    K/V head: the persistent kernels walk several items per CTA with their barriers running on
+    (the small shapes above give every CTA at most one item)."""
+    wl = small("tcp", 6, 8, 2, 700, 128, 256, "bf16", 5400, unit=True)      # 6 tiles x 48 heads = 288 items
+    y, ref, _ = run(wl)
+    check(y, ref, "bf16", "persistent forward")
+    errs = run_bwd(wl)
+    for name, e in errs.items():
+        assert e <= GRAD_TOL, (name, e, errs)
