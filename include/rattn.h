@@ -75,7 +75,8 @@ typedef enum rattn_mode {
  *   workspace  scratch + saved residuals, rattn_workspace_bytes() bytes, 256-byte
  *              aligned.  rattn_forward_ex writes it; rattn_backward_ex reads the
  *              residuals the forward left there, so pass the same buffer, untouched,
- *              with the same sizes.
+ *              with the same sizes, mode and flags (the tensor-core and the portable
+ *              kernels keep their residuals in different forms).
  *   state_out, k_ring_out, v_ring_out   optional prefill -> decode hand-off written by
  *              rattn_forward_ex: state [B,H_kv,d,d] fp32 = sum over tokens j < T-w of
  *              phi(k_j)^T v_j; rings [B,H_kv,w,d] (I/O dtype) holding token j at slot

@@ -15,8 +15,8 @@ namespace rattn {
 struct WorkspaceLayout {
   size_t status;        // 256 bytes; word 0 = device status, word 1 = detail code
   size_t lse;           // fp32 [B,H_q,T]      log-sum-exp of the SWA logits (natural log)
-  size_t o_swa;         // fp32 [B,H_q,T,d]    un-normalised SWA branch output
-  size_t o_rla;         // fp32 [B,H_q,T,d]    un-normalised RLA branch output
+  size_t o_swa;         // fp32 [B,H_q,T,d]    un-normalised SWA branch output (bf16 on the tensor-core path)
+  size_t o_rla;         // fp32 [B,H_q,T,d]    un-normalised RLA branch output (likewise)
   size_t do_swa;        // fp32 [B,H_q,T,d]    backward scratch (the tensor-core path keeps bf16 there)
   size_t do_rla;        // fp32 [B,H_q,T,d]    backward scratch (likewise)
   size_t delta;         // fp32 [B,H_q,T]      backward scratch

@@ -60,8 +60,8 @@ struct BwdArgs {
 // One warp per row; lane owns 4 consecutive features.  Writes g_s, g_r (bf16), D and, when
 // asked, accumulates the gain gradients.
 __global__ void __launch_bounds__(256)
-tc_bwd_prep_kernel(const __nv_bfloat16* __restrict__ dy, const float* __restrict__ o_s,
-                   const float* __restrict__ o_r, const float* __restrict__ gamma_s,
+tc_bwd_prep_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat16* __restrict__ o_s,
+                   const __nv_bfloat16* __restrict__ o_r, const float* __restrict__ gamma_s,
                    const float* __restrict__ gamma_r, __nv_bfloat16* __restrict__ g_s,
                    __nv_bfloat16* __restrict__ g_r, float* __restrict__ delta, float* __restrict__ dgamma_s,
                    float* __restrict__ dgamma_r, const float* __restrict__ lse, float* __restrict__ lse2p,
@@ -99,21 +99,20 @@ tc_bwd_prep_kernel(const __nv_bfloat16* __restrict__ dy, const float* __restrict
       continue;
     }
     const size_t row = bq * T + t;
-    const float4 s0 = *reinterpret_cast<const float4*>(o_s + row * 128 + 8 * l16);
-    const float4 s1 = *reinterpret_cast<const float4*>(o_s + row * 128 + 8 * l16 + 4);
-    const float4 r0 = *reinterpret_cast<const float4*>(o_r + row * 128 + 8 * l16);
-    const float4 r1 = *reinterpret_cast<const float4*>(o_r + row * 128 + 8 * l16 + 4);
+    const uint4 us = *reinterpret_cast<const uint4*>(o_s + row * 128 + 8 * l16);
+    const uint4 ur = *reinterpret_cast<const uint4*>(o_r + row * 128 + 8 * l16);
     const uint4 gy = *reinterpret_cast<const uint4*>(dy + row * 128 + 8 * l16);
-    const float vs[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-    const float vr[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
-    float g[8];
+    float vs[8], vr[8], g[8];
     {
+      const __nv_bfloat162* ps = reinterpret_cast<const __nv_bfloat162*>(&us);
+      const __nv_bfloat162* pr = reinterpret_cast<const __nv_bfloat162*>(&ur);
       const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&gy);
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const float2 f = __bfloat1622float2(hp[e]);
-        g[2 * e] = f.x;
-        g[2 * e + 1] = f.y;
+        const float2 fs = __bfloat1622float2(ps[e]), fr = __bfloat1622float2(pr[e]), f = __bfloat1622float2(hp[e]);
+        vs[2 * e] = fs.x; vs[2 * e + 1] = fs.y;
+        vr[2 * e] = fr.x; vr[2 * e + 1] = fr.y;
+        g[2 * e] = f.x;   g[2 * e + 1] = f.y;
       }
     }
     float ss = 0.f, sr = 0.f, As = 0.f, Ar = 0.f;
@@ -1015,7 +1014,8 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
   {
     KernelTimer kt("tc_bwd_prep", s);
     tc_bwd_prep_kernel<<<(unsigned)((n_rows_pad + 63) / 64), 256, 0, s>>>(
-        reinterpret_cast<const __nv_bfloat16*>(a.dout), a.o_swa, a.o_rla, a.gamma_swa, a.gamma_rla, g_s, g_r,
+        reinterpret_cast<const __nv_bfloat16*>(a.dout), reinterpret_cast<const __nv_bfloat16*>(a.o_swa),
+        reinterpret_cast<const __nv_bfloat16*>(a.o_rla), a.gamma_swa, a.gamma_rla, g_s, g_r,
         a.delta, a.dgamma_swa, a.dgamma_rla, a.lse, a.lse2p, a.dscp, n_rows_pad, a.T, t_pad, a.H_q, a.eps, a.scale,
         rla_on ? 1 : 0);
   }

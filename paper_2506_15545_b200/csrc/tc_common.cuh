@@ -88,6 +88,26 @@ __device__ __forceinline__ void load_half_tile(unsigned char* dst, const CUtenso
   tma_load_3d(dst + HT_HALF, tm, bar, 64, row, z);
 }
 
+// The same for bf16 output: 32 values of row r become one 64-byte row of an 8 KB region
+// (16-byte chunks XOR-swizzled by row pair), flushed in 64-byte segments, eight rows per
+// instruction.  dst points at column 32*c of the tile's first row (row pitch 128 bf16).
+__device__ __forceinline__ void stage_bf16_block(unsigned char* stage, int r, const float (&x)[32]) {
+#pragma unroll
+  for (int e = 0; e < 4; ++e)
+    *reinterpret_cast<uint4*>(stage + r * 64 + ((e ^ ((r >> 1) & 3)) << 4)) =
+        make_uint4(pack_bf16(x[8 * e], x[8 * e + 1]), pack_bf16(x[8 * e + 2], x[8 * e + 3]),
+                   pack_bf16(x[8 * e + 4], x[8 * e + 5]), pack_bf16(x[8 * e + 6], x[8 * e + 7]));
+}
+__device__ __forceinline__ void flush_bf16_block(const unsigned char* stage, int r, __nv_bfloat16* dst, int n_rows) {
+  const int sub = r & 3;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int row = (r >> 5) * 32 + 8 * k + ((r & 31) >> 2);
+    const uint4 v = *reinterpret_cast<const uint4*>(stage + row * 64 + ((sub ^ ((row >> 1) & 3)) << 4));
+    if (row < n_rows) *reinterpret_cast<uint4*>(dst + (size_t)row * 128 + 8 * sub) = v;
+  }
+}
+
 // phi over the 128 features of one row by a pair of adjacent lanes: this lane owns the 64
 // columns of column half `half` (eight 16-byte chunks at src + row * 128 within that half's box).
 // src_half / dst_half point at the [rows x 64] box of this lane's column half.

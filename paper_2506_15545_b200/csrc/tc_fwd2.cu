@@ -50,8 +50,8 @@ struct FBars {
 
 struct FArgs {
   float* lse;
-  float* o_swa;
-  float* o_rla;
+  __nv_bfloat16* o_swa;   // training mode: un-normalised branch outputs [B*H_q, T, 128] as bf16
+  __nv_bfloat16* o_rla;   // (the tensor-core backward reads them in that form)
   const float* gamma_swa;
   const float* gamma_rla;
   int* status;
@@ -473,8 +473,8 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     const size_t tile_row0 = (size_t)un.bh_q * a.T + q0;
     const float rms_s = ms * rs;                                       // sqrt(mean square + eps)
     if (a.o_swa) {
-      // training mode: un-normalised branch outputs (fp32), 32 columns at a time, staged so
-      // that each warp writes whole 128-byte segments of its own 32 rows
+      // training mode: un-normalised branch outputs (bf16), 32 columns at a time, staged so
+      // that each warp writes whole 64-byte segments of its own 32 rows
       unsigned char* stage = sQ;
       if (rlaX) group_sync(X);
 #pragma unroll
@@ -487,9 +487,9 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
           x[2 * e + 1] = f.y * rms_s;
         }
         __syncwarp();
-        stage_f32_block(stage, r, x);
+        stage_bf16_block(stage, r, x);
         __syncwarp();
-        flush_f32_block(stage, r, a.o_swa + tile_row0 * 128 + 32 * c, a.T - q0);
+        flush_bf16_block(stage, r, a.o_swa + tile_row0 * 128 + 32 * c, a.T - q0);
         if (rlaX) {
           tmem_ld32(tO + 32 * c, x);
           tmem_wait_ld();
@@ -500,9 +500,9 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
           for (int e = 0; e < 32; ++e) x[e] = 0.f;
         }
         __syncwarp();
-        stage_f32_block(stage, r, x);
+        stage_bf16_block(stage, r, x);
         __syncwarp();
-        flush_f32_block(stage, r, a.o_rla + tile_row0 * 128 + 32 * c, a.T - q0);
+        flush_bf16_block(stage, r, a.o_rla + tile_row0 * 128 + 32 * c, a.T - q0);
       }
       group_sync(X);
     }
@@ -645,7 +645,9 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s) {
       !make_map(&tm.st, a.chunk_state, 128, (uint64_t)a.B * a.H_kv * a.n_chunks))
     return cudaErrorInvalidValue;
   FArgs t;
-  t.lse = a.lse; t.o_swa = a.o_swa; t.o_rla = a.o_rla;
+  t.lse = a.lse;
+  t.o_swa = reinterpret_cast<__nv_bfloat16*>(a.o_swa);   // the fp32-sized regions of the workspace hold bf16 here
+  t.o_rla = reinterpret_cast<__nv_bfloat16*>(a.o_rla);
   t.gamma_swa = a.gamma_swa; t.gamma_rla = a.gamma_rla; t.status = a.status;
   t.T = a.T; t.w = a.w; t.H_q = a.H_q; t.group = a.group; t.mode = a.mode; t.n_chunks = a.n_chunks;
   t.n_qt = (a.T + TILE - 1) / TILE;

@@ -71,6 +71,9 @@ def test_tensor_forward_c2_like_heads():
 
 
 def test_tensor_residuals_match_portable_path():
+    """The residuals the training-mode forward leaves for the backward: log-sum-exp (fp32, first
+    region after the 256-byte status block) and the un-normalised window output (second region;
+    fp32 on the portable path, bf16 on the tensor-core path) agree between the two paths."""
     wl = small("tcs", 1, 2, 1, 512, 128, 128, "bf16", 4300, unit=True)
     y, ref, (q, k, v, ws) = run(wl, save=True)
     ws2 = torch.zeros_like(ws)
@@ -83,8 +86,9 @@ def test_tensor_residuals_match_portable_path():
     f2 = ws2[256:].view(torch.float32)
     lse1, lse2 = f1[:n], f2[:n]
     assert (lse1 - lse2).abs().max() < 2e-2
-    off = ((n * 4 + 255) // 256 * 256) // 4
-    o1, o2 = f1[off:off + n * 128], f2[off:off + n * 128]
+    off = (n * 4 + 255) // 256 * 256
+    o1 = ws[256 + off:256 + off + n * 128 * 2].view(torch.bfloat16).float()
+    o2 = f2[off // 4:off // 4 + n * 128]
     assert (o1 - o2).abs().max() < 3e-2
     check(y, ref, "bf16")
 
@@ -160,15 +164,17 @@ def test_tensor_backward_control_modes(mode):
 
 
 def test_tensor_backward_matches_portable_backward():
-    """Same residuals, both backward paths: the two CUDA implementations agree far inside the
-    bound either has against the oracle."""
+    """Forward + backward on the tensor-core path against forward + backward on the portable
+    path (each backward reads the residuals its own forward left): the two CUDA
+    implementations agree far inside the bound either has against the oracle."""
     wl = small("tcbp", 1, 2, 1, 512, 128, 128, "bf16", 5200, unit=True)
     q, k, v = (t.cuda() for t in W.make_qkv(wl))
     dy = W.make_dout(wl).cuda()
     ws = R.alloc_workspace(q, k, wl.w)
     R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws, save_residuals=True)
-    a = R.rattn_backward_ex(q, k, v, dy, wl.w, ws, scale=wl.scale)
-    a = [t.clone() for t in a]
+    a = [t.clone() for t in R.rattn_backward_ex(q, k, v, dy, wl.w, ws, scale=wl.scale)]
+    R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws, save_residuals=True,
+                       flags=R.FLAG_FORCE_GENERIC)
     b = R.rattn_backward_ex(q, k, v, dy, wl.w, ws, scale=wl.scale, flags=R.FLAG_FORCE_GENERIC)
     torch.cuda.synchronize()
     for x, y in zip(a, b):
