@@ -87,7 +87,7 @@ tc_bwd_prep_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat16* __
     acc_s[e] = 0.f;
     acc_r[e] = 0.f;
   }
-#pragma unroll 2
+#pragma unroll 1
   for (int rr = 2 * warp + sub; rr < ROWS_PER_CTA; rr += 16) {
     const int t = t0 + rr;
     const size_t prow = bq * t_pad + t;
