@@ -20,12 +20,14 @@
 //
 // Two main kernels, so that every output tile has one owner and nothing is accumulated with
 // atomics (results are deterministic):
-//   tc_bwd_dq_kernel   one CTA per (query tile, query head): loops over the key tiles of the band.
-//   tc_bwd_dkv_kernel  one CTA per (key tile, K/V head): loops over the group's query heads and,
-//                      for each, over the query tiles whose band contains the key tile.
-// In both, 128 threads own one accumulator row each (row = TMEM lane), one thread issues every
-// TMA load and tcgen05.mma, all products are 128 x 128 x 128 with fp32 accumulation in TMEM,
-// and the two weight matrices of each tile pair are rounded to bf16 in shared memory.
+//   tc_bwd_dq_kernel   a (query head, query tile) item loops over the key tiles of its band;
+//   tc_bwd_dkv_kernel  a (K/V head, key tile) item loops over the group's query heads and, for
+//                      each, over the query half tiles whose band contains the key tile.
+// Both are persistent (one CTA per SM walks its items, the next item's loads in flight while
+// the current one's epilogue drains) and warp-specialised: row groups of 128 threads own one
+// accumulator row each (row = TMEM lane), a loader warp issues the TMA loads, an MMA warp the
+// tcgen05 products; all accumulation is fp32 in TMEM, and the weight matrices of each tile
+// pair (P, dS) are rounded to bf16 and handed to the tensor core through TMEM.
 #include "tc_common.cuh"
 
 namespace rattn {
