@@ -166,25 +166,52 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecodeArgs a) {
           for (int e = 0; e < EPL; ++e) { kx[u][e] = 0.f; vx[u][e] = 0.f; }
         }
       }
+      // Scores of the whole batch first, then one running-maximum update and one rescale of
+      // the accumulator per batch and head (rescaling per key costs twice the arithmetic and
+      // chains every key behind the previous one).
+      float dot[U][GH];
 #pragma unroll
       for (int u = 0; u < U; ++u) {
 #pragma unroll
         for (int hh = 0; hh < GH; ++hh) {
-          float dot = 0.f;
+          float x = 0.f;
 #pragma unroll
-          for (int e = 0; e < EPL; ++e) dot += qr[hh][e] * kx[u][e];
-#pragma unroll
-          for (int o = 1; o < LPK; o <<= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-          if (ok[u]) {
-            const float m_new = fmaxf(m[hh], dot);
-            const float corr = __expf(m[hh] - m_new);   // exp(-inf) = 0 on the first key
-            const float p = __expf(dot - m_new);
-            l[hh] = l[hh] * corr + p;
-#pragma unroll
-            for (int e = 0; e < EPL; ++e) acc[hh][e] = acc[hh][e] * corr + p * vx[u][e];
-            m[hh] = m_new;
-          }
+          for (int e = 0; e < EPL; ++e) x += qr[hh][e] * kx[u][e];
+          dot[u][hh] = x;
         }
+      }
+#pragma unroll
+      for (int o = 1; o < LPK; o <<= 1) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+#pragma unroll
+          for (int hh = 0; hh < GH; ++hh) dot[u][hh] += __shfl_xor_sync(0xffffffffu, dot[u][hh], o);
+        }
+      }
+#pragma unroll
+      for (int hh = 0; hh < GH; ++hh) {
+        float mb = -INFINITY;
+#pragma unroll
+        for (int u = 0; u < U; ++u) mb = fmaxf(mb, ok[u] ? dot[u][hh] : -INFINITY);
+        if (mb == -INFINITY) continue;                       // no valid key in this batch for this lane group
+        const float m_new = fmaxf(m[hh], mb);
+        const float corr = __expf(m[hh] - m_new);            // exp(-inf) = 0 on the first batch
+        float p[U];
+        float ps = 0.f;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          p[u] = ok[u] ? __expf(dot[u][hh] - m_new) : 0.f;
+          ps += p[u];
+        }
+        l[hh] = l[hh] * corr + ps;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+          float x = acc[hh][e] * corr;
+#pragma unroll
+          for (int u = 0; u < U; ++u) x += p[u] * vx[u][e];
+          acc[hh][e] = x;
+        }
+        m[hh] = m_new;
       }
     }
     // merge the KPW key sub-groups of the warp
