@@ -490,6 +490,9 @@ def run_all_configs(args):
         time_fwd(W.C3.replace(w=w), mode=R.MODE_SWA_ONLY, label=f"c3 w={w} swa-only")
     time_fwd(W.C3, mode=R.MODE_FULL_CAUSAL, label="c3 full-causal")
     time_fwd(W.C4, label="c4 forward only")
+    # the paper's own head shapes (Table 1): 3B = 16 query / 4 K/V heads, 12B = 40 / 8 (groups of 4 and 5)
+    time_fwd(W.C2.replace(H_q=16, H_kv=4), label="paper 3B heads 16/4, B=4, T=4096, w=512")
+    time_fwd(W.C3.replace(H_q=40, H_kv=8, w=1024), label="paper 12B heads 40/8, B=2, T=8192, w=1024")
     c5 = W.C5.replace(B=args.c5_batch)
     time_fwd(c5, label=f"c5 prefill (B={c5.B} of 32)", steps=3)
     kr = torch.randn(W.C5.B, W.C5.H_kv, W.C5.w, W.C5.d, device=dev).to(torch.bfloat16)

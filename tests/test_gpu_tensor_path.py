@@ -203,3 +203,15 @@ def test_tensor_paths_with_several_items_per_cta():
     errs = run_bwd(wl)
     for name, e in errs.items():
         assert e <= GRAD_TOL, (name, e, errs)
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(16, 4), (40, 8)])
+def test_paper_head_shapes(Hq, Hkv):
+    """Head counts of the paper's 3B (16 query / 4 K/V heads) and 12B (40 / 8: a group of five,
+    not a power of two) models (Table 1), head size 128, forward and backward."""
+    wl = small("tab1", 1, Hq, Hkv, 768, 128, 256, "bf16", 5500 + Hq, unit=True)
+    y, ref, _ = run(wl)
+    check(y, ref, "bf16", f"H={Hq}/{Hkv}")
+    errs = run_bwd(wl)
+    for name, e in errs.items():
+        assert e <= GRAD_TOL, (name, e, errs)
