@@ -256,7 +256,11 @@ __device__ __forceinline__ void feature_map_row_inplace_lr(unsigned char* tile, 
 }
 
 // phi (softmax over the 128 features) of row r of a swizzled bf16 tile, in place.
-__device__ __forceinline__ void feature_map_row_inplace(unsigned char* tile, int r) {
+// NORMALISE = false leaves exp(x - max) (bf16) and returns 1 / sum, for callers that scale
+// whatever is linear in this row afterwards.  The row lives in 128 registers in between: one
+// read and one write of shared memory.
+template <bool NORMALISE = true>
+__device__ __forceinline__ float feature_map_row_inplace(unsigned char* tile, int r) {
   float x[128];
   float m = -INFINITY;
 #pragma unroll
@@ -278,16 +282,17 @@ __device__ __forceinline__ void feature_map_row_inplace(unsigned char* tile, int
     x[i] = ex2(x[i] * 1.4426950408889634f - ml);
     sum += x[i];
   }
-  const float inv = 1.f / sum;
+  const float inv = 1.f / sum, sc = NORMALISE ? inv : 1.f;
 #pragma unroll
   for (int c = 0; c < 16; ++c) {
     uint4 u;
-    u.x = pack_bf16(x[c * 8 + 0] * inv, x[c * 8 + 1] * inv);
-    u.y = pack_bf16(x[c * 8 + 2] * inv, x[c * 8 + 3] * inv);
-    u.z = pack_bf16(x[c * 8 + 4] * inv, x[c * 8 + 5] * inv);
-    u.w = pack_bf16(x[c * 8 + 6] * inv, x[c * 8 + 7] * inv);
+    u.x = pack_bf16(x[c * 8 + 0] * sc, x[c * 8 + 1] * sc);
+    u.y = pack_bf16(x[c * 8 + 2] * sc, x[c * 8 + 3] * sc);
+    u.z = pack_bf16(x[c * 8 + 4] * sc, x[c * 8 + 5] * sc);
+    u.w = pack_bf16(x[c * 8 + 6] * sc, x[c * 8 + 7] * sc);
     *reinterpret_cast<uint4*>(tile + swz(r, c)) = u;
   }
+  return inv;
 }
 
 

@@ -234,26 +234,36 @@ __device__ bool fwd_mma(const FArgs& a, unsigned char* smem, FBars* bars, uint32
         WAIT_OR_RETURN_W(bars->x_full, cntX & 1);
         ++cntX;
       }
+      // scores first (they only need the feature maps), the products into the accumulators once
+      // the row groups have parked the window outputs
       if (un.rla[0]) {
-        WAIT_OR_RETURN_W(bars->stash_done[0], cntR[0] & 1);
         WAIT_OR_RETURN_W(bars->phiq_ready[0], cntR[0] & 1);
         WAIT_OR_RETURN_W(bars->phik_ready[0], cntK[0] & 1);
         tc_fence_after();
-        if (un.has_state) mma_kmn<1>(tO[0], sQ[0], sX, false);                   // phi(Q_A) S_[cA]
         mma_kk(tS[0], sQ[0], sK(iA), false);                                     // phi(Q_A) phi(K_cA)^T
         mma_commit(&bars->s_full[0]);
       }
-      if (un.rla[1]) {
-        WAIT_OR_RETURN_W(bars->stash_done[1], cntR[1] & 1);
+      if (un.rla[1] && un.rla[0]) {
         WAIT_OR_RETURN_W(bars->phiq_ready[1], cntR[1] & 1);
         tc_fence_after();
-        if (un.rla[0]) {
-          if (un.has_state) mma_kmn<1>(tO[1], sQ[1], sX, false);                 // phi(Q_B) S_[cA]
-          mma_kk(tS[1], sQ[1], sK(iA), false);                                   // phi(Q_B) phi(K_cA)^T, whole chunk
-          mma_commit(&bars->s_full[1]);
+        mma_kk(tS[1], sQ[1], sK(iA), false);                                     // phi(Q_B) phi(K_cA)^T, whole chunk
+        mma_commit(&bars->s_full[1]);
+      }
+      if (un.rla[0] && un.has_state) {
+        WAIT_OR_RETURN_W(bars->stash_done[0], cntR[0] & 1);
+        tc_fence_after();
+        mma_kmn<1>(tO[0], sQ[0], sX, false);                                     // phi(Q_A) S_[cA]
+      }
+      if (un.rla[1]) {
+        if (!un.rla[0]) WAIT_OR_RETURN_W(bars->phiq_ready[1], cntR[1] & 1);
+        if (un.rla[0] && un.has_state) {
+          WAIT_OR_RETURN_W(bars->stash_done[1], cntR[1] & 1);
+          tc_fence_after();
+          mma_kmn<1>(tO[1], sQ[1], sX, false);                                   // phi(Q_B) S_[cA]
         }
       }
       if (un.rla[0]) {
+        if (!un.has_state) WAIT_OR_RETURN_W(bars->stash_done[0], cntR[0] & 1);   // O_A is free
         WAIT_OR_RETURN_W(bars->p_ready[0], cntP[0] & 1);
         ++cntP[0];
         tc_fence_after();
@@ -261,6 +271,7 @@ __device__ bool fwd_mma(const FArgs& a, unsigned char* smem, FBars* bars, uint32
         mma_commit(&bars->o_ready[0]);
       }
       if (un.rla[1]) {
+        if (!(un.rla[0] && un.has_state)) WAIT_OR_RETURN_W(bars->stash_done[1], cntR[1] & 1);   // O_B is free
         if (un.rla[0]) {
           WAIT_OR_RETURN_W(bars->p_ready[1], cntP[1] & 1);
           ++cntP[1];
@@ -389,6 +400,25 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
       mbar_arrive(&bars->p_ready[X]);
     }
 
+    // ---- residual branch, first part: feature maps ------------------------------------------
+    // Done right here, while the last P V of the window loop is still running and before the
+    // parked output takes 64 registers: the row fits in registers, so phi is one read and one
+    // write of shared memory.  Every Q_X K^T and every product reading the raw chunk K has
+    // completed (the commit behind this tile's last scores covers them).
+    float rr = 0.f, sr = 0.f, inv_q = 1.f;
+    if (rlaX) {
+      // phi(Q_X) without its normalisation: everything that follows is linear in this row,
+      // so 1/sum is applied to the accumulator row at the end
+      inv_q = feature_map_row_inplace<false>(sQ, r);
+      fence_proxy_async_smem();
+      mbar_arrive(&bars->phiq_ready[X]);
+      // this tile's own chunk: A -> last stream position, B -> its last active position
+      const int ic = (X == 0) ? un.n - 1 : un.i1[1];
+      feature_map_row_inplace<true>(smem + F_OFF_KV + ((kv0 + ic) & 1) * 2 * TILE_BYTES, r);
+      fence_proxy_async_smem();
+      mbar_arrive(&bars->phik_ready[X]);
+    }
+
     // ---- park the normalised window output (Section 3.2, first norm) in registers ---------
     WAIT_OR_RETURN(bars->o_ready[X], cntO & 1);
     ++cntO;
@@ -414,22 +444,11 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
 #pragma unroll
       for (int e = 0; e < 16; ++e) stash[16 * c + e] = pack_f16(o[2 * e] * inv_l * rs, o[2 * e + 1] * inv_l * rs);
     }
-    float rr = 0.f, sr = 0.f, inv_q = 1.f;
 
-    // ---- residual branch ------------------------------------------------------------------
+    // ---- residual branch, second part -------------------------------------------------------
     if (rlaX) {
       tc_fence_before();
       mbar_arrive(&bars->stash_done[X]);
-      // phi(Q_X) without its normalisation: everything that follows is linear in this row,
-      // so 1/sum is applied to the accumulator row at the end
-      inv_q = feature_map_row_unnorm_inplace(sQ, r);                   // every Q_X K^T has completed
-      fence_proxy_async_smem();
-      mbar_arrive(&bars->phiq_ready[X]);
-      // this tile's own chunk: A -> last stream position, B -> its last active position
-      const int ic = (X == 0) ? un.n - 1 : un.i1[1];
-      feature_map_row_inplace_lr(smem + F_OFF_KV + ((kv0 + ic) & 1) * 2 * TILE_BYTES, r);
-      fence_proxy_async_smem();
-      mbar_arrive(&bars->phik_ready[X]);
       const int n_terms = (X == 1 && un.rla[0]) ? 2 : 1;
 #pragma unroll 1
       for (int term = 0; term < n_terms; ++term) {
