@@ -43,7 +43,7 @@ constexpr float LOG2E = 1.4426950408889634f;
 
 struct FBars {
   uint64_t q_full[2], q_free[2], kv_full[2], v_ready[2], kv_free[2], x_full, x_free;
-  uint64_t s_full[2], p_ready[2], o_ready[2], stash_done[2], phiq_ready[2], phik_ready[2], o_free[2], drain;
+  uint64_t s_full[2], p_ready[2], o_ready[2], stash_done[2], phiq_ready[2], phik_ready[2], o_free[2], y_done[2], drain;
   uint32_t tmem_base;
   int abort;
 };
@@ -141,6 +141,12 @@ __device__ bool fwd_loader(const FMaps& tm, const FArgs& a, unsigned char* smem,
     }
     if (un.has_state) {
       if (cntX >= 1) WAIT_OR_RETURN_W(bars->x_free, (cntX - 1) & 1);
+      // the same buffer stages the outputs: every tile of the units before has left it
+#pragma unroll
+      for (int X = 0; X < 2; ++X) {
+        const int done_before = cntU[X] - (un.t[X] >= 0 ? 1 : 0);      // epilogues of tile X before this unit
+        if (done_before >= 1) WAIT_OR_RETURN_W(bars->y_done[X], (done_before - 1) & 1);
+      }
       mbar_arrive_expect_tx(&bars->x_full, TILE_BYTES);
       load_tile(smem + F_OFF_X, &tm.st, &bars->x_full, 0, un.bh_kv * a.n_chunks + un.cA);
       ++cntX;
@@ -527,39 +533,60 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     }
     const float* gs = a.gamma_swa ? a.gamma_swa + (size_t)un.h * 128 : nullptr;
     const float* gr = a.gamma_rla ? a.gamma_rla + (size_t)un.h * 128 : nullptr;
-    // the branches on "gains given" and "tile has a residual branch" are taken once, outside the loop
+    // y leaves through the state tile's buffer (free once this unit's residual products are done;
+    // 16 KB per row group), one 64-column half at a time, so that the tile's Q buffer and the
+    // K/V stages can take the next unit's loads while the epilogue runs.  The branches on "gains
+    // given" and "tile has a residual branch" are taken once, outside the loops.
+    unsigned char* sY = smem + F_OFF_X + X * HALF_BYTES;
+    mbar_arrive(&bars->q_free[X]);         // phi(Q_X) has been consumed: the Q buffer may be refilled
     auto emit_y = [&](auto has_gains_t, auto has_rla_t) {
       constexpr bool has_gains = decltype(has_gains_t)::value, has_rla = decltype(has_rla_t)::value;
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {                                    // 16 columns at a time
-        float orl[16];
-        if constexpr (has_rla) {
-          tmem_ld16(tO + 16 * c, orl);
-          tmem_wait_ld();
-        }
-        uint32_t yk[8];
+      for (int hf = 0; hf < 2; ++hf) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&stash[8 * c + e]));
-          const int col = 16 * c + 2 * e;
-          float y0 = f.x, y1 = f.y;
-          if constexpr (has_gains) {
-            y0 *= gs ? __ldg(gs + col) : 1.f;
-            y1 *= gs ? __ldg(gs + col + 1) : 1.f;
-          }
+        for (int c4 = 0; c4 < 4; ++c4) {                               // 16 columns at a time
+          const int c = 4 * hf + c4;
+          float orl[16];
           if constexpr (has_rla) {
-            float r0 = orl[2 * e] * rr, r1 = orl[2 * e + 1] * rr;
-            if constexpr (has_gains) {
-              r0 *= gr ? __ldg(gr + col) : 1.f;
-              r1 *= gr ? __ldg(gr + col + 1) : 1.f;
-            }
-            y0 += r0;
-            y1 += r1;
+            tmem_ld16(tO + 16 * c, orl);
+            tmem_wait_ld();
           }
-          yk[e] = pack_bf16(y0, y1);
+          uint32_t yk[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&stash[8 * c + e]));
+            const int col = 16 * c + 2 * e;
+            float y0 = f.x, y1 = f.y;
+            if constexpr (has_gains) {
+              y0 *= gs ? __ldg(gs + col) : 1.f;
+              y1 *= gs ? __ldg(gs + col + 1) : 1.f;
+            }
+            if constexpr (has_rla) {
+              float r0 = orl[2 * e] * rr, r1 = orl[2 * e + 1] * rr;
+              if constexpr (has_gains) {
+                r0 *= gr ? __ldg(gr + col) : 1.f;
+                r1 *= gr ? __ldg(gr + col + 1) : 1.f;
+              }
+              y0 += r0;
+              y1 += r1;
+            }
+            yk[e] = pack_bf16(y0, y1);
+          }
+          *reinterpret_cast<uint4*>(sY + swz(r, 2 * c4)) = make_uint4(yk[0], yk[1], yk[2], yk[3]);
+          *reinterpret_cast<uint4*>(sY + swz(r, 2 * c4 + 1)) = make_uint4(yk[4], yk[5], yk[6], yk[7]);
         }
-        *reinterpret_cast<uint4*>(sQ + swz(r, 2 * c)) = make_uint4(yk[0], yk[1], yk[2], yk[3]);
-        *reinterpret_cast<uint4*>(sQ + swz(r, 2 * c + 1)) = make_uint4(yk[4], yk[5], yk[6], yk[7]);
+        if (hf == 1) {
+          tc_fence_before();
+          mbar_arrive(&bars->o_free[X]);   // last read of the accumulator: scores and output columns may be overwritten
+        }
+        fence_proxy_async_smem();
+        group_sync(X);
+        if (r == 0) {
+          tma_store_3d(&tm.out, sY, 64 * hf, q0, un.bh_q);
+          tma_store_commit();
+          tma_store_wait_read();
+        }
+        group_sync(X);
       }
     };
     const bool gains = gs != nullptr || gr != nullptr;
@@ -571,17 +598,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
       else emit_y(std::false_type{}, std::false_type{});
     }
     if (t < a.T && a.lse) a.lse[(size_t)un.bh_q * a.T + t] = (m_ref + log2f(l)) * 0.6931471805599453f;
-    fence_proxy_async_smem();
-    tc_fence_before();
-    group_sync(X);
-    if (r == 0) {
-      store_tile(&tm.out, sQ, q0, un.bh_q);
-      tma_store_commit();
-      tma_store_wait_read();
-    }
-    group_sync(X);
-    mbar_arrive(&bars->q_free[X]);       // the Q buffer may be refilled
-    mbar_arrive(&bars->o_free[X]);       // the score and output columns may be overwritten
+    mbar_arrive(&bars->y_done[X]);         // the staging buffer may take the next state tile
   }
   return true;
 }
@@ -609,6 +626,7 @@ tc_fwd2_kernel(const __grid_constant__ FMaps tm, FArgs a) {
       mbar_init(&bars->phiq_ready[i], 128);
       mbar_init(&bars->phik_ready[i], 128);
       mbar_init(&bars->o_free[i], 128);
+      mbar_init(&bars->y_done[i], 128);
     }
     mbar_init(&bars->x_full, 1);
     mbar_init(&bars->x_free, 1);
