@@ -538,7 +538,6 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     // K/V stages can take the next unit's loads while the epilogue runs.  The branches on "gains
     // given" and "tile has a residual branch" are taken once, outside the loops.
     unsigned char* sY = smem + F_OFF_X + X * HALF_BYTES;
-    mbar_arrive(&bars->q_free[X]);         // phi(Q_X) has been consumed: the Q buffer may be refilled
     auto emit_y = [&](auto has_gains_t, auto has_rla_t) {
       constexpr bool has_gains = decltype(has_gains_t)::value, has_rla = decltype(has_rla_t)::value;
 #pragma unroll
@@ -584,8 +583,12 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
         if (r == 0) {
           tma_store_3d(&tm.out, sY, 64 * hf, q0, un.bh_q);
           tma_store_commit();
-          tma_store_wait_read();
         }
+        // The Q buffer (phi(Q_X) has long been consumed) is released only once the last store is
+        // in the TMA queue: the next unit's loads, issued the moment it is released, would
+        // otherwise sit in front of the stores and hold the staging buffer for thousands of cycles.
+        if (hf == 1) mbar_arrive(&bars->q_free[X]);
+        if (r == 0) tma_store_wait_read();
         group_sync(X);
       }
     };
