@@ -72,6 +72,13 @@ def io_bytes_fwd(wl):
     return e * wl.d * wl.T * wl.B * (2 * wl.H_q + 2 * wl.H_kv)
 
 
+def io_bytes_step(wl):
+    """Algorithmic bytes of a training step: q, k, v, dO read; out, dq, dk, dv written (the
+    residuals the forward leaves for the backward are implementation traffic, not counted)."""
+    e = 2 if wl.dtype == "bf16" else 4
+    return e * wl.d * wl.T * wl.B * (4 * wl.H_q + 4 * wl.H_kv)
+
+
 def decode_bytes(wl):
     e = 2
     ring = 2 * wl.B * wl.H_kv * wl.w * wl.d * e
@@ -99,14 +106,14 @@ class ClockSampler:
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                       "-lms", "50", "-i", str(index)], stdout=self.f,
+                                       "-lms", "20", "-i", str(index)], stdout=self.f,
                                       stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
 
     def stop(self):
         if self.p is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["nvidia-smi unavailable"]}
         self.p.terminate()
         try:
             self.p.wait(timeout=5)
@@ -129,7 +136,7 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         os.unlink(self.f.name)
-        return {"sm_mhz": statistics.median(sm) if sm else None,
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_min_mhz": min(sm) if sm else None,
                 "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
@@ -178,7 +185,8 @@ def run_reference(args, wl):
     cores = oracle_threads()
     sample = "each step = forward+backward of one (batch, head) pair at T=4096 through the fp64 oracle"
     print(json.dumps({
-        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s",
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic", "config": {"workload": workload_name(wl), "sample": sample},
@@ -241,7 +249,7 @@ def run_ours(args, wl):
     wl_r = wl.replace(seed=wl.seed + rank)
     q, k, v = W.make_qkv(wl_r, dev)
     dy = W.make_dout(wl_r, dev)
-    ws = R.alloc_workspace(q, k, wl.w)
+    ws = R.alloc_workspace(q, k, wl.w, R.MODE_RATTN, R.FLAG_SAVE_RESIDUALS)
     out = torch.empty_like(q)
     dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
 
@@ -265,7 +273,27 @@ def run_ours(args, wl):
     launches = R.rattn_launch_count() - launches0
     kernel_ms = R.rattn_timing_read()
     R.rattn_timing_enable(False)
+    # The K timed steps last tens of milliseconds, too short for more than a sample or two of
+    # nvidia-smi.  The same step is therefore repeated under the same sampler for about two
+    # seconds more (timed on its own, reported as "sustained"): the clock record then has
+    # dozens of samples of this very load, and the two times show whether the short region ran
+    # in the burst regime (same time per step) or ahead of a power-capped steady state.
+    sustained = None
+    if rank == 0 and args.clock_seconds > 0:
+        n_more = max(args.steps, int(args.clock_seconds * 1e3 / max(ms, 1e-3)))
+        c, d = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c.record()
+        for _ in range(n_more):
+            step()
+        d.record()
+        torch.cuda.synchronize()
+        sustained = {"steps": n_more, "ms_per_step": c.elapsed_time(d) / n_more}
     clocks = sampler.stop() if sampler else None
+    if clocks is not None and sustained is not None:
+        clocks["sustained_loop"] = sustained
+        if clocks.get("sm_mhz"):
+            clocks["ms_per_step_x_sm_mhz"] = ms * clocks["sm_mhz"]
+    barrier()
     assert R.rattn_read_status(ws) == 0, "device-side wait expired"
     ms, total_flops = whole_job(ms, flops(wl, "step"), dist, dev)
     value = total_flops / (ms * 1e-3) / 1e12
@@ -277,15 +305,30 @@ def run_ours(args, wl):
     kflops = {"tc_fwd": "fwd_main", "tc_chunk_delta": "fwd_state", "generic_fwd": "fwd",
               "generic_bwd_dq": "bwd_dq", "generic_bwd_dkv": "bwd_dkv",
               "tc_bwd_dq": "bwd_dq", "tc_bwd_dkv": "bwd_dkv"}
+    # Which measured bf16 peak applies is read off the run: the burst figure when the timed
+    # region is short and the sampled SM clock sat at its maximum, the sustained one for a
+    # region of seconds or a clock held down by the power cap.  Both fractions are printed.
+    region_s = ms * args.steps * 1e-3
+    at_max = bool(clocks and clocks.get("sm_mhz") and clocks["sm_mhz"] >= 0.97 * clocks["sm_max_mhz"])
+    regime = "burst" if (region_s < 1.0 and (at_max or not clocks or not clocks.get("sm_mhz"))) else "sustained"
+    peak = pk["tf_burst"] if regime == "burst" else pk["tf_sus"]
     roof = None
     if top in kflops:
         ach = flops(wl, kflops[top]) / (per_launch[top] * 1e-3) / 1e12
         mb = NCU_TRAFFIC_MB_PER_BATCH_ENTRY.get(top)
-        roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": pk["tf_sus"], "unit": "TFLOP/s",
-                "frac": ach / pk["tf_sus"], "traffic": None if mb is None else mb * 1e6 * wl.B,
+        roof = {"kernel": top, "bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s",
+                "frac": ach / peak, "frac_of_burst_peak": ach / pk["tf_burst"],
+                "frac_of_sustained_peak": ach / pk["tf_sus"],
+                "traffic": None if mb is None else mb * 1e6 * wl.B,
                 "traffic_unit": "bytes per launch (ncu capture at B=2, scaled by the batch)",
-                "peak_source": pk["src"] + " (sustained bf16: the kernel is timed inside a long step)",
+                "peak_source": f"{pk['src']} {regime} bf16 peak (timed region {region_s * 1e3:.0f} ms, "
+                               f"median SM clock {clocks['sm_mhz'] if clocks else None} MHz)",
+                "algorithmic_flops_per_launch": flops(wl, kflops[top]),
                 "ms_per_launch": per_launch[top]}
+    t_roof_step = max(flops(wl, "step") / (peak * 1e12), io_bytes_step(wl) / (pk["hbm"] * 1e9)) * 1e3
+    step_roof = {"roofline_ms": t_roof_step, "frac": t_roof_step / (ms if world == 1 else ms),
+                 "flops_per_step": flops(wl, "step"), "bytes_per_step": io_bytes_step(wl),
+                 "denominator": f"max(FLOPs / {peak} TF/s, bytes / {pk['hbm']} GB/s), {pk['src']} {regime}"}
     total_k = sum(share.values())
     kernels = {n: {"launches": kernel_ms[n][0], "ms_per_launch": per_launch[n], "share": share[n] / total_k}
                for n in share}
@@ -298,7 +341,8 @@ def run_ours(args, wl):
                    "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                    "l2": "inputs larger than L2 (q,k,v,dO,residuals > 1 GB per step)"},
         "tokens_per_s": wl.B * wl.T * world / (ms * 1e-3),
-        "gpu_launches": int(launches), "kernels": kernels, "roofline": roof, "clocks": clocks,
+        "gpu_launches": int(launches), "kernels": kernels, "roofline": roof, "step_roofline": step_roof,
+        "clocks": clocks,
     }
     if rank != 0:
         if dist is not None:
@@ -311,7 +355,7 @@ def run_ours(args, wl):
     del dq, dk, dv, dy
     c2 = W.C2
     q2, k2, v2 = W.make_qkv(c2, dev)
-    ws2 = R.alloc_workspace(q2, k2, c2.w)
+    ws2 = R.alloc_workspace(q2, k2, c2.w, R.MODE_RATTN, 0)
     # rotate three input sets (3 x 268 MB > L2) so no launch finds its inputs in L2
     sets = [(q2, k2, v2)] + [tuple(t.clone() for t in (q2, k2, v2)) for _ in range(2)]
     o2 = torch.empty_like(q2)
@@ -381,10 +425,22 @@ def run_ours(args, wl):
         h_dk.copy_(dk, non_blocking=True)
         h_dv.copy_(dv, non_blocking=True)
 
-    ms_e = timed(e2e_step, max(2, min(args.steps, 5)), 1, sync)
+    n_e2e = max(10, min(args.steps, 20))
+    e2e_step()
+    sync()
+    per = []
+    for _ in range(n_e2e):
+        ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ea.record()
+        e2e_step()
+        eb.record()
+        sync()
+        per.append(ea.elapsed_time(eb))
+    ms_e = statistics.median(per)
     nbytes = lambda *ts: int(sum(t.numel() * t.element_size() for t in ts))
     result["e2e"] = {"value": flops(wl, "step") / (ms_e * 1e-3) / 1e12, "unit": "TFLOP/s",
-                     "ms_per_step": ms_e, "h2d_bytes_per_step": nbytes(hq, hk, hv, hdy),
+                     "ms_per_step": ms_e, "ms_per_step_min": min(per), "steps": n_e2e,
+                     "h2d_bytes_per_step": nbytes(hq, hk, hv, hdy),
                      "d2h_bytes_per_step": nbytes(h_dq, h_dk, h_dv)}
 
     # ---- CPU baseline: the oracle, as it stands, on a bounded sample ------------------
@@ -415,7 +471,7 @@ def run_case(args):
     if args.case in ("fwd", "train"):
         wl = W.C2.replace(B=2)          # q,k,v,out = 134 MB
         q, k, v = W.make_qkv(wl, dev)
-        ws = R.alloc_workspace(q, k, wl.w)
+        ws = R.alloc_workspace(q, k, wl.w, R.MODE_RATTN, R.FLAG_SAVE_RESIDUALS if args.case == "train" else 0)
         out = torch.empty_like(q)
         if args.case == "fwd":
             fn = lambda: R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws, out=out)
@@ -467,7 +523,7 @@ def run_all_configs(args):
 
     def time_fwd(wl, mode=R.MODE_RATTN, label=None, steps=20):
         q, k, v = W.make_qkv(wl, dev)
-        ws = R.alloc_workspace(q, k, wl.w)
+        ws = R.alloc_workspace(q, k, wl.w, mode, 0)
         o = torch.empty_like(q)
         ms = timed(lambda: R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, mode=mode, workspace=ws, out=o),
                    steps, 3, sync)
@@ -495,6 +551,25 @@ def run_all_configs(args):
     time_fwd(W.C3.replace(H_q=40, H_kv=8, w=1024), label="paper 12B heads 40/8, B=2, T=8192, w=1024")
     c5 = W.C5.replace(B=args.c5_batch)
     time_fwd(c5, label=f"c5 prefill (B={c5.B} of 32)", steps=3)
+    # prefill -> decode hand-off (ring + state out of the prefill's K/V): the library's own
+    # per-kernel events around one forward that asks for it
+    q, k, v = W.make_qkv(c5, dev)
+    ws = R.alloc_workspace(q, k, c5.w, R.MODE_RATTN, 0)
+    o = torch.empty_like(q)
+    st_o = torch.zeros(c5.B, c5.H_kv, c5.d, c5.d, device=dev)
+    kr_o = torch.zeros(c5.B, c5.H_kv, c5.w, c5.d, device=dev, dtype=torch.bfloat16)
+    vr_o = torch.zeros_like(kr_o)
+    hand = lambda: R.rattn_forward_ex(q, k, v, c5.w, scale=c5.scale, workspace=ws, out=o, state_out=st_o,
+                                      k_ring_out=kr_o, v_ring_out=vr_o)
+    hand()
+    R.rattn_timing_enable(True)
+    hand()
+    km = R.rattn_timing_read()
+    R.rattn_timing_enable(False)
+    out["configs"].append({"config": f"c5 prefill + hand-off (B={c5.B}), per kernel",
+                           "kernels_ms_per_launch": {n: t / c for n, (c, t) in km.items() if c}})
+    del q, k, v, ws, o, st_o, kr_o, vr_o
+    torch.cuda.empty_cache()
     kr = torch.randn(W.C5.B, W.C5.H_kv, W.C5.w, W.C5.d, device=dev).to(torch.bfloat16)
     vr = torch.randn(W.C5.B, W.C5.H_kv, W.C5.w, W.C5.d, device=dev).to(torch.bfloat16)
     st = torch.zeros(W.C5.B, W.C5.H_kv, W.C5.d, W.C5.d, device=dev)
@@ -512,18 +587,56 @@ def run_all_configs(args):
     print(json.dumps(out))
 
 
+def free_port():
+    import socket
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        return so.getsockname()[1]
+
+
+def launch_replicas(argv, n):
+    """`bench.py --gpus N` started as a plain process: start the N replica ranks itself (one
+    process per GPU under torch.distributed.run on this node) and hand back their exit code.
+    Rank 0 of the children prints the JSON line."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__), *argv]
+    return subprocess.call(cmd)
+
+
+def run_replicas_selftest(args):
+    """The replica plumbing without a GPU: gloo ranks that pretend to have measured
+    10 + 5 * rank milliseconds for 7 units of work each; rank 0 prints the aggregate."""
+    import torch.distributed as dist
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    ms, units = whole_job(10.0 + 5.0 * rank, 7.0, dist if world > 1 else None, "cpu")
+    if rank == 0:
+        print(json.dumps({"impl": "replicas-selftest", "n_gpus": world, "ms_per_step": ms, "units": units}))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "replicas-selftest"])
     ap.add_argument("--case", default=None, choices=["fwd", "train", "decode"],
                     help="run one small case (for profiler captures) instead of the benchmark")
     ap.add_argument("--all-configs", action="store_true",
                     help="time the forward of all five named configurations instead of the benchmark")
-    ap.add_argument("--c5-batch", type=int, default=8, help="batch entries of config 5's prefill to time")
+    ap.add_argument("--c5-batch", type=int, default=32, help="batch entries of config 5's prefill to time")
+    ap.add_argument("--clock-seconds", type=float, default=2.0,
+                    help="after the K timed steps, repeat the step for about this long under the clock sampler")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.all_configs or args.case):
+        sys.exit(launch_replicas(sys.argv[1:], args.gpus))
+    if args.impl == "replicas-selftest":
+        run_replicas_selftest(args)
+        return
     if args.all_configs:
         run_all_configs(args)
         return

@@ -69,11 +69,16 @@ typedef enum rattn_mode {
  * Parameter block of the *_ex entry points.  Zero-initialise it, then fill in.
  *   dtype      I/O element type of q,k,v,out,dout,dq,dk,dv and the decode ring.
  *              Accumulation, softmax, feature map, norms and the state are fp32.
- *   scale      multiplies the SWA logits q.k only (the paper writes none: 1.0).
+ *   scale      multiplies the SWA logits q.k only (the paper writes none: 1.0).  The
+ *              tensor-core kernels need scale > 0 and return RATTN_ERR_UNSUPPORTED
+ *              otherwise; the portable kernels (RATTN_FLAG_FORCE_GENERIC) take any finite
+ *              value.
  *   eps        added to mean(x^2) inside the RMS-norm square root.
  *   gamma_swa, gamma_rla   fp32 [H_q, d] gains of the two norms, or NULL for ones.
- *   workspace  scratch + saved residuals, rattn_workspace_bytes() bytes, 256-byte
- *              aligned.  rattn_forward_ex writes it; rattn_backward_ex reads the
+ *   workspace  scratch + saved residuals, rattn_workspace_bytes_ex() bytes for this
+ *              call's sizes, mode and flags, 256-byte aligned.  May be NULL where that
+ *              size is 256 (nothing but the status word would live there).
+ *              rattn_forward_ex writes it; rattn_backward_ex reads the
  *              residuals the forward left there, so pass the same buffer, untouched,
  *              with the same sizes, mode and flags (the tensor-core and the portable
  *              kernels keep their residuals in different forms).
@@ -116,7 +121,8 @@ typedef struct rattn_params {
  * bf16 I/O, scale = 1, unit gains, eps = 1e-6, mode RATTN, inference (no residuals).
  * T need not be a multiple of any tile.  This is the one entry point that may take
  * device memory on its own: where the tensor-core path applies (d = 128, w % 128 == 0)
- * it needs scratch for the chunk states of the linear branch and obtains it with
+ * it needs scratch for the chunk states of the linear branch
+ * (rattn_workspace_bytes_ex(..., RATTN_MODE_RATTN, 0) bytes) and obtains it with
  * cudaMallocAsync / cudaFreeAsync on `stream` (the device's stream-ordered pool; no
  * synchronisation).  Callers that must control every allocation use rattn_forward_ex
  * with their own workspace.
@@ -152,6 +158,12 @@ int rattn_forward(const void* q, const void* k, const void* v,
 int rattn_forward_static(const void* q, const void* k, const void* v,
                          int B, int H_q, int H_kv, int T, int d, int w, float scale,
                          void* out, void* stream);
+
+/* The device status word of rattn_forward_static's calls on the current device (it sits at
+ * the head of the fixed array, which the caller cannot name): synchronises `stream`, then
+ * returns RATTN_OK, RATTN_ERR_TIMEOUT (a bounded device-side wait of the last call expired)
+ * or RATTN_ERR_CUDA.  Allocates nothing. */
+int rattn_static_status(void* stream);
 
 /* Forward with the full parameter block (dtype, scale, gains, mode, workspace,
  * residuals for the backward, prefill -> decode hand-off). */
@@ -196,10 +208,25 @@ int rattn_decode_step_ex(const rattn_params* p, void* k_ring, void* v_ring, floa
                          int pos, void* stream);
 
 /*
- * Bytes of workspace the forward (and the backward that follows it) needs for these
- * sizes; dtype is a rattn_dtype.  Returns 0 for invalid sizes.  The first 256 bytes
- * hold the device status word.
+ * Bytes of workspace a call with these sizes, mode (rattn_mode) and flags (RATTN_FLAG_*)
+ * needs; dtype is a rattn_dtype.  Returns 0 for invalid arguments.  The first 256 bytes hold
+ * the device status word.  What the rest holds depends on the call:
+ *   inference, portable kernels        nothing more (256 bytes in all);
+ *   inference, tensor-core kernels     the chunk states of the linear branch (Eq. 2; the
+ *                                      paper's stored states): bf16 [B,H_kv,ceil(T/128),d,d],
+ *                                      mode RATTN only;
+ *   RATTN_FLAG_SAVE_RESIDUALS          in addition the residuals of Section 3.2's two branches
+ *                                      (log-sum-exp, un-normalised o_swa and o_rla: bf16 on the
+ *                                      tensor-core path, fp32 on the portable one) and the
+ *                                      backward's scratch of the same shapes.
+ * The backward needs the size of its forward (same sizes, mode, flags with
+ * RATTN_FLAG_SAVE_RESIDUALS set).  A larger buffer is always accepted.
  */
+size_t rattn_workspace_bytes_ex(int B, int H_q, int H_kv, int T, int d, int w, int dtype,
+                                int mode, unsigned flags);
+
+/* An upper bound of rattn_workspace_bytes_ex over every mode and every flag combination for
+ * these sizes (the training layout of the larger kernel family). */
 size_t rattn_workspace_bytes(int B, int H_q, int H_kv, int T, int d, int w, int dtype);
 
 /* Reads the status word of a workspace (synchronises `stream` first, copies 4 bytes

@@ -21,9 +21,10 @@ FLAG_FORCE_GENERIC, FLAG_SAVE_RESIDUALS = 1, 2
 EXPORTS = (
     "rattn_forward", "rattn_forward_ex", "rattn_backward", "rattn_backward_ex",
     "rattn_decode_step", "rattn_decode_step_ex", "rattn_workspace_bytes",
+    "rattn_workspace_bytes_ex",
     "rattn_read_status", "rattn_strerror", "rattn_last_cuda_error", "rattn_launch_count",
     "rattn_uses_tensor_path", "rattn_timing_enable", "rattn_timing_read",
-    "rattn_forward_static",
+    "rattn_forward_static", "rattn_static_status",
 )
 
 
@@ -83,6 +84,8 @@ def lib() -> ctypes.CDLL:
     L.rattn_decode_step_ex.restype = ci
     L.rattn_workspace_bytes.argtypes = [ci, ci, ci, ci, ci, ci, ci]
     L.rattn_workspace_bytes.restype = ctypes.c_size_t
+    L.rattn_workspace_bytes_ex.argtypes = [ci, ci, ci, ci, ci, ci, ci, ci, ctypes.c_uint]
+    L.rattn_workspace_bytes_ex.restype = ctypes.c_size_t
     L.rattn_read_status.argtypes = [vp, vp]
     L.rattn_read_status.restype = ci
     L.rattn_strerror.argtypes = [ci]
@@ -95,6 +98,8 @@ def lib() -> ctypes.CDLL:
     L.rattn_uses_tensor_path.restype = ci
     L.rattn_forward_static.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, vp, vp]
     L.rattn_forward_static.restype = ci
+    L.rattn_static_status.argtypes = [vp]
+    L.rattn_static_status.restype = ci
     L.rattn_timing_enable.argtypes = [ci]
     L.rattn_timing_enable.restype = ci
     L.rattn_timing_read.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
@@ -135,10 +140,18 @@ def rattn_workspace_bytes(B, H_q, H_kv, T, d, w, dtype=RATTN_BF16) -> int:
     return int(lib().rattn_workspace_bytes(B, H_q, H_kv, T, d, w, dtype))
 
 
-def alloc_workspace(q, k, w) -> torch.Tensor:
-    """A uint8 device tensor of rattn_workspace_bytes() bytes for these shapes."""
+def rattn_workspace_bytes_ex(B, H_q, H_kv, T, d, w, dtype=RATTN_BF16, mode=MODE_RATTN, flags=0) -> int:
+    return int(lib().rattn_workspace_bytes_ex(B, H_q, H_kv, T, d, w, dtype, mode, flags))
+
+
+def alloc_workspace(q, k, w, mode=None, flags=None) -> torch.Tensor:
+    """A uint8 device tensor for these shapes: exactly rattn_workspace_bytes_ex() bytes when
+    mode and flags are given, else rattn_workspace_bytes() (enough for any mode and flags)."""
     B, H_q, T, d = q.shape
-    n = rattn_workspace_bytes(B, H_q, k.shape[1], T, d, w, _dtype_code(q))
+    if mode is None and flags is None:
+        n = rattn_workspace_bytes(B, H_q, k.shape[1], T, d, w, _dtype_code(q))
+    else:
+        n = rattn_workspace_bytes_ex(B, H_q, k.shape[1], T, d, w, _dtype_code(q), mode or 0, flags or 0)
     return torch.empty(n, dtype=torch.uint8, device=q.device)
 
 
@@ -253,6 +266,11 @@ def rattn_decode_step_ex(q, k, v, k_ring, v_ring, state, pos, *, scale=1.0, eps=
 
 def rattn_read_status(workspace, stream=None) -> int:
     return int(lib().rattn_read_status(_ptr(workspace), _stream(stream)))
+
+
+def rattn_static_status(stream=None) -> int:
+    """Status word of rattn_forward_static's last call on the current device."""
+    return int(lib().rattn_static_status(_stream(stream)))
 
 
 def rattn_launch_count() -> int:

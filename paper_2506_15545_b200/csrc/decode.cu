@@ -432,6 +432,7 @@ cudaError_t launch_handoff_t(const Args& a, cudaStream_t s) {
   const int BH = a.B * a.H_kv;
   if (a.state_out) {
     dim3 grid(D / 8, BH);
+    KernelTimer kt("handoff_state", s);
     handoff_state_kernel<TIO, D><<<grid, 256, 0, s>>>(reinterpret_cast<const TIO*>(a.k),
                                                       reinterpret_cast<const TIO*>(a.v),
                                                       a.state_out, a.T, a.w);
@@ -439,6 +440,7 @@ cudaError_t launch_handoff_t(const Args& a, cudaStream_t s) {
   }
   if (a.k_ring_out && a.v_ring_out) {
     dim3 grid(a.w, BH);
+    KernelTimer kt("handoff_ring", s);
     handoff_ring_kernel<TIO><<<grid, 64, 0, s>>>(reinterpret_cast<const TIO*>(a.k),
                                                  reinterpret_cast<const TIO*>(a.v),
                                                  reinterpret_cast<TIO*>(a.k_ring_out),

@@ -50,27 +50,53 @@ static void timing_clear_locked() {
 
 static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
-WorkspaceLayout workspace_layout(int B, int H_q, int H_kv, int T, int d, int w, int dtype) {
-  (void)w;
-  (void)dtype;
+static bool tensor_path(int d, int w, int dtype, int mode, unsigned flags) {
+#ifdef RATTN_HAVE_TC
+  if (flags & RATTN_FLAG_FORCE_GENERIC) return false;
+  if (dtype != RATTN_BF16 || d != 128) return false;
+  if (mode != RATTN_MODE_FULL_CAUSAL && (w % 128) != 0) return false;
+  return true;
+#else
+  (void)d; (void)w; (void)dtype; (void)mode; (void)flags;
+  return false;
+#endif
+}
+
+// What a call with these sizes, mode and flags keeps in its workspace.  Inference on the
+// portable kernels: the status block only.  Inference on the tensor-core kernels: the status
+// block and the chunk states of the linear branch.  Training (RATTN_FLAG_SAVE_RESIDUALS) adds the
+// residuals the backward reads and the backward's own scratch, in the element type the chosen
+// kernels keep them in (bf16 on the tensor-core path, fp32 on the portable one).
+WorkspaceLayout workspace_layout(int B, int H_q, int H_kv, int T, int d, int w, int dtype, int mode,
+                                 unsigned flags) {
   WorkspaceLayout L;
+  const bool tc = tensor_path(d, mode == RATTN_MODE_FULL_CAUSAL ? T : w, dtype, mode, flags);
+  const bool train = (flags & RATTN_FLAG_SAVE_RESIDUALS) != 0;
+  const bool rla = (mode == RATTN_MODE_RATTN);
   const size_t rows = (size_t)B * H_q * T;
+  const size_t branch_elem = tc ? sizeof(__nv_bfloat16) : sizeof(float);
   size_t off = 0;
-  L.status = off;      off += 256;
-  L.lse = off;         off += align256(rows * sizeof(float));
-  L.o_swa = off;       off += align256(rows * d * sizeof(float));
-  L.o_rla = off;       off += align256(rows * d * sizeof(float));
-  L.do_swa = off;      off += align256(rows * d * sizeof(float));
-  L.do_rla = off;      off += align256(rows * d * sizeof(float));
-  L.delta = off;       off += align256(rows * sizeof(float));
+  auto take = [&](bool present, size_t bytes) -> size_t {
+    if (!present) return kAbsent;
+    const size_t at = off;
+    off += align256(bytes);
+    return at;
+  };
   L.n_chunks = (T + 127) / 128;
   const size_t states = (size_t)B * H_kv * L.n_chunks * d * d;
-  L.chunk_delta = off; off += align256(states * sizeof(float));
-  L.chunk_state = off; off += align256(states * sizeof(__nv_bfloat16));
-  L.rstate = off;      off += align256(states * sizeof(__nv_bfloat16));
   const size_t rows_pad = (size_t)B * H_q * L.n_chunks * 128;
-  L.lse2p = off;       off += align256(rows_pad * sizeof(float));
-  L.dscp = off;        off += align256(rows_pad * sizeof(float));
+  L.status = take(true, 256);
+  L.lse = take(train, rows * sizeof(float));
+  L.o_swa = take(train, rows * d * branch_elem);
+  L.o_rla = take(train, rows * d * branch_elem);
+  L.do_swa = take(train, rows * d * branch_elem);
+  L.do_rla = take(train, rows * d * branch_elem);
+  L.delta = take(train, rows * sizeof(float));
+  L.chunk_state = take(tc && rla, states * sizeof(__nv_bfloat16));
+  L.chunk_delta = take(tc && rla && tc_parallel_states(B * H_kv), states * sizeof(float));
+  L.rstate = take(tc && rla && train, states * sizeof(__nv_bfloat16));
+  L.lse2p = take(tc && train, rows_pad * sizeof(float));
+  L.dscp = take(tc && train, rows_pad * sizeof(float));
   L.total = off;
   return L;
 }
@@ -106,38 +132,27 @@ static int resolve(const rattn_params* p, Args* a, bool need_T) {
   return RATTN_OK;
 }
 
-static int bind_workspace(const rattn_params* p, Args* a, bool required) {
+static int bind_workspace(const rattn_params* p, Args* a, bool required, unsigned flags) {
   if (!p->workspace) return required ? RATTN_ERR_WORKSPACE : RATTN_OK;
   if (((uintptr_t)p->workspace & 255u) != 0) return RATTN_ERR_MISALIGNED;
-  const WorkspaceLayout L = workspace_layout(p->B, p->H_q, p->H_kv, p->T, p->d, p->w, p->dtype);
+  const WorkspaceLayout L = workspace_layout(p->B, p->H_q, p->H_kv, p->T, p->d, p->w, p->dtype, p->mode, flags);
   if (p->workspace_bytes < L.total) return RATTN_ERR_WORKSPACE;
   char* base = reinterpret_cast<char*>(p->workspace);
-  a->status = reinterpret_cast<int*>(base + L.status);
-  a->lse = reinterpret_cast<float*>(base + L.lse);
-  a->o_swa = reinterpret_cast<float*>(base + L.o_swa);
-  a->o_rla = reinterpret_cast<float*>(base + L.o_rla);
-  a->do_swa = reinterpret_cast<float*>(base + L.do_swa);
-  a->do_rla = reinterpret_cast<float*>(base + L.do_rla);
-  a->delta = reinterpret_cast<float*>(base + L.delta);
-  a->chunk_delta = reinterpret_cast<float*>(base + L.chunk_delta);
-  a->chunk_state = reinterpret_cast<__nv_bfloat16*>(base + L.chunk_state);
-  a->rstate = reinterpret_cast<__nv_bfloat16*>(base + L.rstate);
-  a->lse2p = reinterpret_cast<float*>(base + L.lse2p);
-  a->dscp = reinterpret_cast<float*>(base + L.dscp);
+  auto at = [&](size_t off) -> char* { return off == kAbsent ? nullptr : base + off; };
+  a->status = reinterpret_cast<int*>(at(L.status));
+  a->lse = reinterpret_cast<float*>(at(L.lse));
+  a->o_swa = reinterpret_cast<float*>(at(L.o_swa));
+  a->o_rla = reinterpret_cast<float*>(at(L.o_rla));
+  a->do_swa = reinterpret_cast<float*>(at(L.do_swa));
+  a->do_rla = reinterpret_cast<float*>(at(L.do_rla));
+  a->delta = reinterpret_cast<float*>(at(L.delta));
+  a->chunk_delta = reinterpret_cast<float*>(at(L.chunk_delta));
+  a->chunk_state = reinterpret_cast<__nv_bfloat16*>(at(L.chunk_state));
+  a->rstate = reinterpret_cast<__nv_bfloat16*>(at(L.rstate));
+  a->lse2p = reinterpret_cast<float*>(at(L.lse2p));
+  a->dscp = reinterpret_cast<float*>(at(L.dscp));
   a->n_chunks = L.n_chunks;
   return RATTN_OK;
-}
-
-static bool tensor_path(int d, int w, int dtype, int mode, unsigned flags) {
-#ifdef RATTN_HAVE_TC
-  if (flags & RATTN_FLAG_FORCE_GENERIC) return false;
-  if (dtype != RATTN_BF16 || d != 128) return false;
-  if (mode != RATTN_MODE_FULL_CAUSAL && (w % 128) != 0) return false;
-  return true;
-#else
-  (void)d; (void)w; (void)dtype; (void)mode; (void)flags;
-  return false;
-#endif
 }
 
 static int forward_impl(const rattn_params* p, cudaStream_t s) {
@@ -152,13 +167,12 @@ static int forward_impl(const rattn_params* p, cudaStream_t s) {
     if (p->mode != RATTN_MODE_RATTN) return RATTN_ERR_UNSUPPORTED;
   }
   const bool tc = tensor_path(p->d, a.w, p->dtype, p->mode, p->flags);
-  rc = bind_workspace(p, &a, tc);
+  // the tensor-core kernels take the row maximum before multiplying by the scale
+  if (tc && !(p->scale > 0.f)) return RATTN_ERR_UNSUPPORTED;
+  const bool train = (p->flags & RATTN_FLAG_SAVE_RESIDUALS) != 0;
+  // a workspace is needed for the residuals and for the chunk states of the tensor-core path
+  rc = bind_workspace(p, &a, train || (tc && p->mode == RATTN_MODE_RATTN), p->flags);
   if (rc != RATTN_OK) return rc;
-  if (!(p->flags & RATTN_FLAG_SAVE_RESIDUALS)) {
-    a.lse = nullptr; a.o_swa = nullptr; a.o_rla = nullptr;
-  } else if (!p->workspace) {
-    return RATTN_ERR_WORKSPACE;
-  }
   a.state_out = p->state_out; a.k_ring_out = p->k_ring_out; a.v_ring_out = p->v_ring_out;
   cudaError_t e;
   if (a.status) {
@@ -186,7 +200,9 @@ static int backward_impl(const rattn_params* p, cudaStream_t s) {
   if (misaligned(p->dout) || misaligned(p->dq) || misaligned(p->dk) || misaligned(p->dv) ||
       misaligned(p->dgamma_swa) || misaligned(p->dgamma_rla))
     return RATTN_ERR_MISALIGNED;
-  rc = bind_workspace(p, &a, true);
+  const bool tc = tensor_path(p->d, a.w, p->dtype, p->mode, p->flags);
+  if (tc && !(p->scale > 0.f)) return RATTN_ERR_UNSUPPORTED;
+  rc = bind_workspace(p, &a, true, p->flags | RATTN_FLAG_SAVE_RESIDUALS);
   if (rc != RATTN_OK) return rc;
   a.dout = p->dout; a.dq = p->dq; a.dk = p->dk; a.dv = p->dv;
   a.dgamma_swa = p->dgamma_swa; a.dgamma_rla = p->dgamma_rla;
@@ -194,7 +210,7 @@ static int backward_impl(const rattn_params* p, cudaStream_t s) {
 #ifdef RATTN_HAVE_TC
   // The tensor-core backward reads the chunk states the tensor-core forward left in the
   // workspace: both calls must take the same path (same sizes, mode and flags).
-  if (tensor_path(p->d, a.w, p->dtype, p->mode, p->flags)) e = launch_tc_backward(a, s);
+  if (tc) e = launch_tc_backward(a, s);
   else
 #endif
     e = launch_generic_backward(a, s);
@@ -226,7 +242,7 @@ int rattn_forward(const void* q, const void* k, const void* v, int B, int H_q, i
   Args chk;
   int rc = resolve(&p, &chk, true);
   if (rc != RATTN_OK) return rc;
-  const size_t bytes = rattn_workspace_bytes(B, H_q, H_kv, T, d, w, RATTN_BF16);
+  const size_t bytes = rattn_workspace_bytes_ex(B, H_q, H_kv, T, d, w, RATTN_BF16, RATTN_MODE_RATTN, 0);
   void* ws = nullptr;
   cudaError_t e = cudaMallocAsync(&ws, bytes, s);
   if (e != cudaSuccess) return fail_cuda(e);
@@ -282,10 +298,22 @@ int rattn_decode_step(const void* q, const void* k, const void* v, void* k_ring,
   return rattn_decode_step_ex(&p, k_ring, v_ring, state, pos, stream);
 }
 
-size_t rattn_workspace_bytes(int B, int H_q, int H_kv, int T, int d, int w, int dtype) {
+size_t rattn_workspace_bytes_ex(int B, int H_q, int H_kv, int T, int d, int w, int dtype, int mode,
+                                unsigned flags) {
   if (B < 1 || H_q < 1 || H_kv < 1 || T < 1 || w < 1 || (d != 64 && d != 128)) return 0;
   if (H_q % H_kv != 0) return 0;
-  return workspace_layout(B, H_q, H_kv, T, d, w, dtype).total;
+  if (dtype != RATTN_BF16 && dtype != RATTN_F32) return 0;
+  if (mode < RATTN_MODE_RATTN || mode > RATTN_MODE_FULL_CAUSAL) return 0;
+  return workspace_layout(B, H_q, H_kv, T, d, w, dtype, mode, flags).total;
+}
+
+size_t rattn_workspace_bytes(int B, int H_q, int H_kv, int T, int d, int w, int dtype) {
+  // enough for any mode and any flags: the training layout of either kernel family
+  const unsigned train = RATTN_FLAG_SAVE_RESIDUALS;
+  const size_t a = rattn_workspace_bytes_ex(B, H_q, H_kv, T, d, w, dtype, RATTN_MODE_RATTN, train);
+  const size_t b = rattn_workspace_bytes_ex(B, H_q, H_kv, T, d, w, dtype, RATTN_MODE_RATTN,
+                                            train | RATTN_FLAG_FORCE_GENERIC);
+  return a > b ? a : b;
 }
 
 int rattn_read_status(const void* workspace, void* stream) {

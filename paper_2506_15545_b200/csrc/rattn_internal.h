@@ -11,7 +11,8 @@
 
 namespace rattn {
 
-// Byte offsets inside the caller's workspace.  Every region is 256-byte aligned.
+// Byte offsets inside the caller's workspace.  Every region is 256-byte aligned; a region the
+// call's mode and flags do not need has offset kAbsent and takes no room.
 struct WorkspaceLayout {
   size_t status;        // 256 bytes; word 0 = device status, word 1 = detail code
   size_t lse;           // fp32 [B,H_q,T]      log-sum-exp of the SWA logits (natural log)
@@ -29,7 +30,15 @@ struct WorkspaceLayout {
   int n_chunks;         // ceil(T / 128)
 };
 
-WorkspaceLayout workspace_layout(int B, int H_q, int H_kv, int T, int d, int w, int dtype);
+// Offset of a region the call does not use.
+constexpr size_t kAbsent = ~(size_t)0;
+
+// The forward computes the chunk states in parallel form (a block per chunk, then a prefix sum)
+// when there are too few K/V heads to give every SM a serial chain of its own.
+inline bool tc_parallel_states(int n_kv) { return n_kv < 64; }
+
+WorkspaceLayout workspace_layout(int B, int H_q, int H_kv, int T, int d, int w, int dtype, int mode,
+                                 unsigned flags);
 
 // Resolved arguments handed to the kernel launchers (all device pointers).
 struct Args {

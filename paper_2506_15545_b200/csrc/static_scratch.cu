@@ -96,3 +96,10 @@ extern "C" int rattn_forward_static(const void* q, const void* k, const void* v,
   e = launch_tc_forward(a, s);
   return e == cudaSuccess ? RATTN_OK : cuda_failure(e);
 }
+
+extern "C" int rattn_static_status(void* stream) {
+  unsigned char* base = nullptr;
+  cudaError_t e = scratch_address(&base);
+  if (e != cudaSuccess) return cuda_failure(e);
+  return rattn_read_status(base, stream);
+}

@@ -1028,7 +1028,7 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
   if (!make_map(&tm_q, a.q, a.T, nq) || !make_map(&tm_k, a.k, a.T, nkv) || !make_map(&tm_v, a.v, a.T, nkv) ||
       !make_map(&tm_gs, g_s, a.T, nq) || !make_map(&tm_gr, g_r, a.T, nq) ||
       !make_map(&tm_dq, a.dq, a.T, nq) || !make_map(&tm_dk, a.dk, a.T, nkv) || !make_map(&tm_dv, a.dv, a.T, nkv) ||
-      !make_map(&tm_st, a.chunk_state, 128, nkv * a.n_chunks) || !make_map(&tm_rs, a.rstate, 128, nkv * a.n_chunks))
+      !make_state_map(&tm_st, a.chunk_state, a.k, nkv * a.n_chunks) || !make_state_map(&tm_rs, a.rstate, a.k, nkv * a.n_chunks))
     return cudaErrorInvalidValue;
 
   // reverse states of the residual branch: chunks c with a query tile beyond c + wt

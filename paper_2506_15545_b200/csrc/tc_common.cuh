@@ -323,7 +323,12 @@ inline bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t n
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-
+// [n_mats, 128, 128] bf16 chunk states.  Modes without a linear branch keep none: the kernels
+// then never use the map, which is encoded over one matrix of `any` (some valid bf16 buffer of
+// at least 128 x 128 elements) so that it is well formed.
+inline bool make_state_map(CUtensorMap* m, const void* states, const void* any, uint64_t n_mats) {
+  return states ? make_map(m, states, 128, n_mats) : make_map(m, any, 128, 1);
+}
 
 }  // namespace tc
 }  // namespace rattn

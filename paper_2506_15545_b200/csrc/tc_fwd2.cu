@@ -682,7 +682,7 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s) {
   FMaps tm;
   if (!make_map(&tm.q, a.q, a.T, (uint64_t)a.B * a.H_q) || !make_map(&tm.k, a.k, a.T, (uint64_t)a.B * a.H_kv) ||
       !make_map(&tm.v, a.v, a.T, (uint64_t)a.B * a.H_kv) || !make_map(&tm.out, a.out, a.T, (uint64_t)a.B * a.H_q) ||
-      !make_map(&tm.st, a.chunk_state, 128, (uint64_t)a.B * a.H_kv * a.n_chunks))
+      !make_state_map(&tm.st, a.chunk_state, a.k, (uint64_t)a.B * a.H_kv * a.n_chunks))
     return cudaErrorInvalidValue;
   FArgs t;
   t.lse = a.lse;

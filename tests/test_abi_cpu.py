@@ -66,6 +66,26 @@ def test_strerror_and_workspace_bytes(B):
     assert B.rattn_workspace_bytes(0, 16, 16, 4096, 128, 512) == 0
 
 
+def test_workspace_size_follows_mode_and_flags(B):
+    """An inference forward keeps only what it uses: the status block on the portable kernels,
+    status + bf16 chunk states on the tensor-core kernels; training adds the residuals."""
+    c5 = (32, 32, 8, 32768, 128, 512)
+    infer = B.rattn_workspace_bytes_ex(*c5, B.RATTN_BF16, B.MODE_RATTN, 0)
+    states = 32 * 8 * 256 * 128 * 128 * 2
+    assert infer == 256 + states                                         # 2.1 GB, not 78 GB
+    assert B.rattn_workspace_bytes_ex(*c5, B.RATTN_BF16, B.MODE_SWA_ONLY, 0) == 256
+    assert B.rattn_workspace_bytes_ex(*c5, B.RATTN_BF16, B.MODE_RATTN, B.FLAG_FORCE_GENERIC) == 256
+    train = B.rattn_workspace_bytes_ex(*c5, B.RATTN_BF16, B.MODE_RATTN, B.FLAG_SAVE_RESIDUALS)
+    train_generic = B.rattn_workspace_bytes_ex(*c5, B.RATTN_BF16, B.MODE_RATTN,
+                                               B.FLAG_SAVE_RESIDUALS | B.FLAG_FORCE_GENERIC)
+    assert infer < train < train_generic                                 # bf16 against fp32 residuals
+    assert B.rattn_workspace_bytes(*c5) == max(train, train_generic)     # the bound covers every case
+    assert B.rattn_workspace_bytes_ex(*c5, B.RATTN_BF16, 7, 0) == 0      # unknown mode
+    # few K/V heads: the parallel state form keeps its fp32 blocks too
+    few = (1, 4, 2, 1024, 128, 128)
+    assert B.rattn_workspace_bytes_ex(*few, B.RATTN_BF16, B.MODE_RATTN, 0) == 256 + 2 * 8 * 128 * 128 * (2 + 4)
+
+
 def _p(bind, **kw):
     p = bind.RattnParams()
     fake = 0x10000                       # non-null, 16-byte aligned; never dereferenced
@@ -86,6 +106,10 @@ def _p(bind, **kw):
     (dict(workspace=0x10100, workspace_bytes=16), -5),     # too small
     (dict(workspace=0x10010, workspace_bytes=1 << 40), -3),  # workspace not 256-byte aligned
     (dict(k_ring_out=0x10000), -2),                        # only one of the two rings
+    # shapes of the tensor-core path: it needs a workspace for its chunk states and a positive scale
+    (dict(d=128, w=128, dtype=0), -5),
+    (dict(d=128, w=128, dtype=0, scale=-1.0, workspace=0x10100, workspace_bytes=1 << 40), -4),
+    (dict(d=128, w=128, dtype=0, scale=0.0, workspace=0x10100, workspace_bytes=1 << 40), -4),
 ])
 def test_forward_rejects_bad_arguments_without_launching(B, kw, code):
     before = B.rattn_launch_count()

@@ -40,6 +40,21 @@ def test_two_replicas_take_the_slowest_time_and_sum_the_work():
         assert units == 14.0       # whole-job work
 
 
+def test_gpus_flag_starts_its_own_replica_processes():
+    """`python bench.py --gpus 2` run as a plain process (no torchrun around it, WORLD_SIZE
+    unset) starts two ranks itself; the line rank 0 prints says n_gpus 2, the slowest rank's
+    time and the summed work."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "replicas-selftest"],
+                       capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    assert lines[0]["n_gpus"] == 2 and lines[0]["ms_per_step"] == 15.0 and lines[0]["units"] == 14.0
+
+
 def test_single_process_is_the_identity():
     import bench
     assert bench.whole_job(3.5, 2.0) == (3.5, 2.0)

@@ -45,7 +45,8 @@ def check_sampled_forward(wl, y, q, k, v, pairs, mode=R.MODE_RATTN, n_random=48)
 def forward_full(wl, mode=R.MODE_RATTN, save=False):
     assert R.rattn_uses_tensor_path(wl.d, wl.w, R.RATTN_BF16, mode)
     q, k, v = W.make_qkv(wl, "cuda")
-    ws = R.alloc_workspace(q, k, wl.w)
+    # exactly what this call needs: an inference forward keeps only the chunk states
+    ws = R.alloc_workspace(q, k, wl.w, mode, R.FLAG_SAVE_RESIDUALS if save else 0)
     y = R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, mode=mode, workspace=ws, save_residuals=save)
     torch.cuda.synchronize()
     assert R.rattn_read_status(ws) == 0, "a device-side wait expired"
@@ -59,10 +60,11 @@ def test_config2_forward_full_size():
     check_sampled_forward(wl, y, q, k, v, [(0, 0), (1, 7), (3, 15)])
 
 
-@pytest.mark.parametrize("w,mode", [(128, R.MODE_RATTN), (512, R.MODE_RATTN), (4096, R.MODE_RATTN),
-                                    (512, R.MODE_SWA_ONLY), (512, R.MODE_FULL_CAUSAL)])
+@pytest.mark.parametrize("w,mode", [(128, R.MODE_RATTN), (256, R.MODE_RATTN), (512, R.MODE_RATTN),
+                                    (1024, R.MODE_RATTN), (2048, R.MODE_RATTN), (4096, R.MODE_RATTN),
+                                    (512, R.MODE_SWA_ONLY), (2048, R.MODE_SWA_ONLY), (512, R.MODE_FULL_CAUSAL)])
 def test_config3_gqa_windows_and_controls(w, mode):
-    """B=2, H=32/8, T=8192: window sweep ends and middle, SWA-only and full-causal controls."""
+    """B=2, H=32/8, T=8192: every window of the sweep, SWA-only and full-causal controls."""
     wl = W.C3.replace(w=w)
     q, k, v, y, _ = forward_full(wl, mode)
     check_sampled_forward(wl, y, q, k, v, [(0, 0), (1, 29)], mode=mode, n_random=32)
@@ -84,25 +86,24 @@ def test_config4_training_step_full_size():
             assert rel_fro(np64(got), want) <= GRAD_TOL, (name, b, h, rel_fro(np64(got), want))
 
 
-def test_config5_long_prefill_then_decode():
-    """H=32/8, d=128, w=512, prefill T=32768 then 256 decode steps (ring + state hand-off).
-    The batch is 4 of the configuration's 32 (the per-head problem is the same; the full
-    batch only repeats it and needs ~100 GB with the training-sized workspace)."""
-    wl = W.C5.replace(B=4)
+def _prefill_then_decode(wl, pairs, n_random=32):
     q, k, v, y, ws = forward_full(wl)
-    pairs = [(0, 0), (3, 31)]
-    check_sampled_forward(wl, y, q, k, v, pairs, n_random=32)
+    check_sampled_forward(wl, y, q, k, v, pairs, n_random=n_random)
+    del y
     # hand-off, then decode with fresh tokens
     state = torch.zeros(wl.B, wl.H_kv, wl.d, wl.d, device="cuda")
     k_ring = torch.zeros(wl.B, wl.H_kv, wl.w, wl.d, device="cuda", dtype=torch.bfloat16)
     v_ring = torch.zeros_like(k_ring)
+    out = torch.empty_like(q)
     R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws, state_out=state, k_ring_out=k_ring,
-                       v_ring_out=v_ring)
+                       v_ring_out=v_ring, out=out)
+    del out
     steps = wl.decode_steps
     toks = [W.make_decode_token(wl, s, "cuda") for s in range(steps)]
     outs = [R.rattn_decode_step_ex(tq, tk, tv, k_ring, v_ring, state, wl.T + s, scale=wl.scale)
             for s, (tq, tk, tv) in enumerate(toks)]
     torch.cuda.synchronize()
+    assert R.rattn_read_status(ws) == 0
     yd = torch.stack(outs, dim=2)                              # [B, H_q, steps, d]
     g = wl.H_q // wl.H_kv
     errs = []
@@ -116,3 +117,17 @@ def test_config5_long_prefill_then_decode():
     err = np.concatenate(errs)
     assert err.max() <= TOL["bf16"]["max_abs"], err.max()
     assert err.mean() <= TOL["bf16"]["mean_abs"], err.mean()
+
+
+def test_config5_long_prefill_then_decode_full_batch():
+    """The configuration as stated: B=32, H=32/8, d=128, w=512, prefill T=32768 (q, k, v, out
+    21.5 GB, chunk states 2.1 GB), then 256 decode steps with the ring and state the prefill
+    hands over.  256 K/V heads: the chunk states come from the serial one-CTA-per-head chain,
+    255 steps long.  Oracle on sampled rows of three heads and on all 256 decode rows."""
+    _prefill_then_decode(W.C5, [(0, 0), (13, 6), (31, 31)], n_random=24)
+
+
+def test_config5_few_heads_take_the_parallel_state_form():
+    """Four batch entries of the same configuration (32 K/V heads in all): too few heads for a
+    chain per SM, so the chunk states are formed per chunk in parallel and prefix-summed."""
+    _prefill_then_decode(W.C5.replace(B=4), [(0, 0), (3, 31)])

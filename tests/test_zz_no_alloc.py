@@ -26,11 +26,18 @@ def _both(wl):
     ws = R.alloc_workspace(q, k, wl.w)
     want = R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws)
     out = torch.empty_like(q)
+    # A first call may still load the kernels' code and look up the array's address; the
+    # property is checked on the call after it.  Free device memory as the driver reports it
+    # covers every kind of allocation (cudaMalloc, a growing stream-ordered pool), not only
+    # those made through torch's caching allocator.
+    R.rattn_forward_static(q, k, v, wl.w, wl.scale, out=out)
     torch.cuda.synchronize()
-    before = torch.cuda.memory_allocated()
+    before, free_before = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
     got = R.rattn_forward_static(q, k, v, wl.w, wl.scale, out=out)
     torch.cuda.synchronize()
     assert torch.cuda.memory_allocated() == before
+    assert torch.cuda.mem_get_info()[0] >= free_before
+    assert R.rattn_static_status() == 0          # no bounded device-side wait expired
     return got, want
 
 
