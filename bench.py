@@ -98,7 +98,7 @@ def peaks():
 
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -111,7 +111,9 @@ class ClockSampler:
         except OSError:
             self.p = None
 
-    def stop(self):
+    def stop(self, window=None):
+        """Summary of the samples; `window` = (t0, t1) wall-clock seconds of the timed region,
+        whose own samples are summarised under "timed_region"."""
         if self.p is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["nvidia-smi unavailable"]}
         self.p.terminate()
@@ -121,7 +123,8 @@ class ClockSampler:
             self.p.kill()
         self.f.flush()
         self.f.seek(0)
-        sm, mx, reasons = [], [], set()
+        import datetime
+        sm, mx, pw, ts, reasons = [], [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.f.read().splitlines():
             c = [x.strip() for x in line.split(",")]
@@ -132,12 +135,25 @@ class ClockSampler:
                 mx.append(float(c[2]))
             except ValueError:
                 continue
+            try:
+                pw.append(float(c[3]))
+            except ValueError:
+                pw.append(float("nan"))
+            try:
+                ts.append(datetime.datetime.strptime(c[0], "%Y/%m/%d %H:%M:%S.%f").timestamp())
+            except ValueError:
+                ts.append(None)
             for n, v in zip(names, c[5:9]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         os.unlink(self.f.name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_min_mhz": min(sm) if sm else None,
-                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "reasons": sorted(reasons)}
+        out = {"sm_mhz": statistics.median(sm) if sm else None, "sm_min_mhz": min(sm) if sm else None,
+               "sm_max_mhz": max(mx) if mx else None, "power_w_max": max(pw) if pw else None,
+               "samples": len(sm), "reasons": sorted(reasons)}
+        if window is not None:
+            inside = [x for x, t in zip(sm, ts) if t is not None and window[0] <= t <= window[1]]
+            out["timed_region"] = {"samples": len(inside), "sm_mhz": statistics.median(inside) if inside else None}
+        return out
 
 
 # ------------------------------------------------------------------------ reference arm
@@ -264,11 +280,13 @@ def run_ours(args, wl):
     R.rattn_timing_enable(True)
     launches0 = R.rattn_launch_count()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wall0 = time.time()
     a.record()
     for _ in range(args.steps):
         step()
     b.record()
     barrier()
+    wall1 = time.time()
     ms = a.elapsed_time(b) / args.steps
     launches = R.rattn_launch_count() - launches0
     kernel_ms = R.rattn_timing_read()
@@ -288,7 +306,7 @@ def run_ours(args, wl):
         d.record()
         torch.cuda.synchronize()
         sustained = {"steps": n_more, "ms_per_step": c.elapsed_time(d) / n_more}
-    clocks = sampler.stop() if sampler else None
+    clocks = sampler.stop((wall0, wall1)) if sampler else None
     if clocks is not None and sustained is not None:
         clocks["sustained_loop"] = sustained
         if clocks.get("sm_mhz"):
@@ -309,8 +327,12 @@ def run_ours(args, wl):
     # region is short and the sampled SM clock sat at its maximum, the sustained one for a
     # region of seconds or a clock held down by the power cap.  Both fractions are printed.
     region_s = ms * args.steps * 1e-3
-    at_max = bool(clocks and clocks.get("sm_mhz") and clocks["sm_mhz"] >= 0.97 * clocks["sm_max_mhz"])
-    regime = "burst" if (region_s < 1.0 and (at_max or not clocks or not clocks.get("sm_mhz"))) else "sustained"
+    # clock of the timed region itself where nvidia-smi caught a sample inside it, else the loop's
+    mhz = None
+    if clocks:
+        mhz = (clocks.get("timed_region") or {}).get("sm_mhz") or clocks.get("sm_mhz")
+    at_max = bool(mhz and mhz >= 0.97 * clocks["sm_max_mhz"])
+    regime = "burst" if (region_s < 1.0 and (at_max or not mhz)) else "sustained"
     peak = pk["tf_burst"] if regime == "burst" else pk["tf_sus"]
     roof = None
     if top in kflops:
@@ -322,7 +344,7 @@ def run_ours(args, wl):
                 "traffic": None if mb is None else mb * 1e6 * wl.B,
                 "traffic_unit": "bytes per launch (ncu capture at B=2, scaled by the batch)",
                 "peak_source": f"{pk['src']} {regime} bf16 peak (timed region {region_s * 1e3:.0f} ms, "
-                               f"median SM clock {clocks['sm_mhz'] if clocks else None} MHz)",
+                               f"SM clock there {mhz} MHz)",
                 "algorithmic_flops_per_launch": flops(wl, kflops[top]),
                 "ms_per_launch": per_launch[top]}
     t_roof_step = max(flops(wl, "step") / (peak * 1e12), io_bytes_step(wl) / (pk["hbm"] * 1e9)) * 1e3
