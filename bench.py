@@ -277,7 +277,6 @@ def run_ours(args, wl):
         step()
     barrier()
     sampler = ClockSampler(local) if rank == 0 else None
-    R.rattn_timing_enable(True)
     launches0 = R.rattn_launch_count()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     wall0 = time.time()
@@ -289,6 +288,14 @@ def run_ours(args, wl):
     wall1 = time.time()
     ms = a.elapsed_time(b) / args.steps
     launches = R.rattn_launch_count() - launches0
+    # Per-kernel durations: the same K steps once more with the library's event pair around every
+    # launch.  (An event between two kernels makes the second wait for the first to finish, so in
+    # this pass the forward's main kernel does not overlap the chunk-state kernel as it does in
+    # the timed region above; the sum of the kernels is therefore a little above ms_per_step.)
+    R.rattn_timing_enable(True)
+    for _ in range(args.steps):
+        step()
+    torch.cuda.synchronize()
     kernel_ms = R.rattn_timing_read()
     R.rattn_timing_enable(False)
     # The K timed steps last tens of milliseconds, too short for more than a sample or two of
@@ -388,8 +395,9 @@ def run_ours(args, wl):
         it[0] += 1
         R.rattn_forward_ex(s[0], s[1], s[2], c2.w, scale=c2.scale, workspace=ws2, out=o2)
 
-    R.rattn_timing_enable(True)
-    ms_f = timed(fwd_only, 30, 5, sync)
+    ms_f = timed(fwd_only, 60, 5, sync)
+    R.rattn_timing_enable(True)      # per-kernel events serialise the two kernels: a second pass
+    timed(fwd_only, 12, 0, sync)
     kf = R.rattn_timing_read()
     R.rattn_timing_enable(False)
     t_roof = max(flops(c2, "fwd") / (pk["tf_burst"] * 1e12), io_bytes_fwd(c2) / (pk["hbm"] * 1e9))
@@ -506,9 +514,11 @@ def run_case(args):
                 R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws, save_residuals=True, out=out)
                 R.rattn_backward_ex(q, k, v, dy, wl.w, ws, scale=wl.scale, dq=dq, dk=dk, dv=dv)
             fl = flops(wl, "step")
-        R.rattn_timing_enable(True)
         ms = timed(fn, args.steps, args.warmup, sync)
+        R.rattn_timing_enable(True)
+        timed(fn, args.steps, 0, sync)
         km = R.rattn_timing_read()
+        R.rattn_timing_enable(False)
         assert R.rattn_read_status(ws) == 0
         print(json.dumps({"case": args.case, "workload": workload_name(wl), "ms": ms,
                           "tflops": fl / (ms * 1e-3) / 1e12,

@@ -142,8 +142,8 @@ int rattn_forward(const void* q, const void* k, const void* v,
  * framework's allocator, a latency-bound loop that must stay clear of the driver's
  * allocation lock.  Where the tensor-core path applies (d = 128, w % 128 == 0) its chunk
  * states go into a fixed array inside the library instead: RATTN_STATIC_MAX_CHUNK_STATES
- * matrices of 128 x 128 (6 MiB in all, held by every GPU that loads the library until the
- * process exits).  The call is refused with RATTN_ERR_STATIC_LIMIT when
+ * matrices of 128 x 128 bf16 (2 MiB in all, held by every GPU that loads the library until
+ * the process exits).  The call is refused with RATTN_ERR_STATIC_LIMIT when
  * B * H_kv * ceil(T / 128) exceeds that number; other shapes run the portable kernel,
  * which needs no scratch, so they are never refused for size.
  *

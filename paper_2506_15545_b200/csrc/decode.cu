@@ -428,9 +428,9 @@ __global__ void handoff_ring_kernel(const TIO* __restrict__ k, const TIO* __rest
 }
 
 template <typename TIO, int D>
-cudaError_t launch_handoff_t(const Args& a, cudaStream_t s) {
+cudaError_t launch_handoff_t(const Args& a, cudaStream_t s, bool state_too) {
   const int BH = a.B * a.H_kv;
-  if (a.state_out) {
+  if (a.state_out && state_too) {
     dim3 grid(D / 8, BH);
     KernelTimer kt("handoff_state", s);
     handoff_state_kernel<TIO, D><<<grid, 256, 0, s>>>(reinterpret_cast<const TIO*>(a.k),
@@ -464,11 +464,11 @@ cudaError_t launch_decode(const Args& p, void* k_ring, void* v_ring, float* stat
   return p.d == 64 ? launch_dec<__nv_bfloat16, 64>(a, s) : launch_dec<__nv_bfloat16, 128>(a, s);
 }
 
-cudaError_t launch_handoff(const Args& a, cudaStream_t s) {
+cudaError_t launch_handoff(const Args& a, cudaStream_t s, bool state_too) {
   if (a.dtype == RATTN_F32)
-    return a.d == 64 ? launch_handoff_t<float, 64>(a, s) : launch_handoff_t<float, 128>(a, s);
-  return a.d == 64 ? launch_handoff_t<__nv_bfloat16, 64>(a, s)
-                   : launch_handoff_t<__nv_bfloat16, 128>(a, s);
+    return a.d == 64 ? launch_handoff_t<float, 64>(a, s, state_too) : launch_handoff_t<float, 128>(a, s, state_too);
+  return a.d == 64 ? launch_handoff_t<__nv_bfloat16, 64>(a, s, state_too)
+                   : launch_handoff_t<__nv_bfloat16, 128>(a, s, state_too);
 }
 
 }  // namespace rattn

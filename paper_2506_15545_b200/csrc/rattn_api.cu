@@ -93,7 +93,6 @@ WorkspaceLayout workspace_layout(int B, int H_q, int H_kv, int T, int d, int w, 
   L.do_rla = take(train, rows * d * branch_elem);
   L.delta = take(train, rows * sizeof(float));
   L.chunk_state = take(tc && rla, states * sizeof(__nv_bfloat16));
-  L.chunk_delta = take(tc && rla && tc_parallel_states(B * H_kv), states * sizeof(float));
   L.rstate = take(tc && rla && train, states * sizeof(__nv_bfloat16));
   L.lse2p = take(tc && train, rows_pad * sizeof(float));
   L.dscp = take(tc && train, rows_pad * sizeof(float));
@@ -146,7 +145,6 @@ static int bind_workspace(const rattn_params* p, Args* a, bool required, unsigne
   a->do_swa = reinterpret_cast<float*>(at(L.do_swa));
   a->do_rla = reinterpret_cast<float*>(at(L.do_rla));
   a->delta = reinterpret_cast<float*>(at(L.delta));
-  a->chunk_delta = reinterpret_cast<float*>(at(L.chunk_delta));
   a->chunk_state = reinterpret_cast<__nv_bfloat16*>(at(L.chunk_state));
   a->rstate = reinterpret_cast<__nv_bfloat16*>(at(L.rstate));
   a->lse2p = reinterpret_cast<float*>(at(L.lse2p));
@@ -174,6 +172,7 @@ static int forward_impl(const rattn_params* p, cudaStream_t s) {
   rc = bind_workspace(p, &a, train || (tc && p->mode == RATTN_MODE_RATTN), p->flags);
   if (rc != RATTN_OK) return rc;
   a.state_out = p->state_out; a.k_ring_out = p->k_ring_out; a.v_ring_out = p->v_ring_out;
+  a.training = train;
   cudaError_t e;
   if (a.status) {
     e = cudaMemsetAsync(a.status, 0, 256, s);
@@ -186,7 +185,7 @@ static int forward_impl(const rattn_params* p, cudaStream_t s) {
     e = launch_generic_forward(a, s);
   if (e != cudaSuccess) return fail_cuda(e);
   if (want_handoff) {
-    e = launch_handoff(a, s);
+    e = launch_handoff(a, s, !tc);      // the tensor-core forward has left the state itself
     if (e != cudaSuccess) return fail_cuda(e);
   }
   return RATTN_OK;

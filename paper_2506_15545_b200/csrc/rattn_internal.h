@@ -21,7 +21,6 @@ struct WorkspaceLayout {
   size_t do_swa;        // fp32 [B,H_q,T,d]    backward scratch (the tensor-core path keeps bf16 there)
   size_t do_rla;        // fp32 [B,H_q,T,d]    backward scratch (likewise)
   size_t delta;         // fp32 [B,H_q,T]      backward scratch
-  size_t chunk_delta;   // fp32 [B,H_kv,n_chunks,d,d]  per-chunk phi(K)^T V
   size_t chunk_state;   // bf16 [B,H_kv,n_chunks,d,d]  exclusive prefix over chunks
   size_t rstate;        // bf16 [B,H_kv,n_chunks,d,d]  backward: suffix sums of phi(Q)^T g_r
   size_t lse2p;         // fp32 [B*H_q, n_chunks*128]  backward: lse * log2(e), +inf in the padding
@@ -32,10 +31,6 @@ struct WorkspaceLayout {
 
 // Offset of a region the call does not use.
 constexpr size_t kAbsent = ~(size_t)0;
-
-// The forward computes the chunk states in parallel form (a block per chunk, then a prefix sum)
-// when there are too few K/V heads to give every SM a serial chain of its own.
-inline bool tc_parallel_states(int n_kv) { return n_kv < 64; }
 
 WorkspaceLayout workspace_layout(int B, int H_q, int H_kv, int T, int d, int w, int dtype, int mode,
                                  unsigned flags);
@@ -57,13 +52,14 @@ struct Args {
   float* o_swa;
   float* o_rla;
   // tensor-path scratch
-  float* chunk_delta;
   __nv_bfloat16* chunk_state;
   __nv_bfloat16* rstate;
   float* lse2p;
   float* dscp;
   int n_chunks;
-  int* status;                 // device status word (may be null when no workspace)
+  int* status;                 // device status block (may be null when no workspace): word 0 status,
+                               // word 1 detail, word 2 the forward's work counter
+  bool training;               // the backward will read every chunk state
   // hand-off
   float* state_out;
   void* k_ring_out;
@@ -85,14 +81,29 @@ cudaError_t launch_generic_forward(const Args& a, cudaStream_t s);
 cudaError_t launch_generic_backward(const Args& a, cudaStream_t s);
 cudaError_t launch_decode(const Args& a, void* k_ring, void* v_ring, float* state, int pos,
                           cudaStream_t s);
-cudaError_t launch_handoff(const Args& a, cudaStream_t s);
+// prefill -> decode hand-off: the rings, and (state_too) the state by the portable kernel
+cudaError_t launch_handoff(const Args& a, cudaStream_t s, bool state_too);
 cudaError_t launch_tc_forward(const Args& a, cudaStream_t s);        // chunk states, then the main kernel
-cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s);
-// running sums of phi(X_c)^T Y_c over the chunks first, first+dir, ... (n_steps of them), the sum
-// after step s written to matrix out_first + dir*s of each K/V head; `name` labels the timing record
-cudaError_t launch_tc_states(const void* x, const void* y, void* out, int T, int n_kv, int group, int n_chunks,
-                             int n_steps, int first, int dir, int out_first, int* status, const char* name,
-                             cudaStream_t s);
+// after_states: a chunk-state kernel was launched just before on the same stream
+cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_states);
+// Running sums of phi(X_c)^T Y_c over the chunks first, first+dir, ... (n_steps of them) for every
+// K/V head (tc_state.cu).  The sum after step s goes, as bf16, to matrix out_first + dir*s of the
+// head when that index is congruent to store_phase modulo store_every; the sum after the last
+// step also goes to final_out (fp32 [n_kv,128,128]) when that is given.  Tokens at positions
+// >= row_limit (0: no limit) contribute nothing.
+struct StateLaunch {
+  const void* x;            // [n_kv * group, T, 128] bf16, mapped through phi
+  const void* y;            // [n_kv * group, T, 128] bf16
+  void* out;                // [n_kv * n_chunks, 128, 128] bf16
+  int T, n_kv, group, n_chunks;
+  int n_steps, first, dir, out_first;
+  int store_every, store_phase;
+  int row_limit;
+  float* final_out;
+  int* status;
+  const char* name;         // label of the timing record
+};
+cudaError_t launch_tc_states(const StateLaunch& L, cudaStream_t s);
 cudaError_t launch_tc_backward(const Args& a, cudaStream_t s);
 
 void count_launches(int n);

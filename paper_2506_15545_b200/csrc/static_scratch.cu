@@ -18,11 +18,10 @@ namespace {
 
 constexpr size_t kMatrices = RATTN_STATIC_MAX_CHUNK_STATES;
 constexpr size_t kStatusBytes = 256;
-constexpr size_t kDeltaBytes = kMatrices * 128 * 128 * sizeof(float);
 constexpr size_t kStateBytes = kMatrices * 128 * 128 * sizeof(__nv_bfloat16);
 
-// [status word, 256 B | per-chunk phi(K)^T V, fp32 | prefix states, bf16]
-static __device__ __align__(256) unsigned char g_static_scratch[kStatusBytes + kDeltaBytes + kStateBytes];
+// [status block, 256 B | chunk states, bf16]
+static __device__ __align__(256) unsigned char g_static_scratch[kStatusBytes + kStateBytes];
 
 constexpr int kMaxDevices = 64;
 std::mutex g_mu;
@@ -86,11 +85,11 @@ extern "C" int rattn_forward_static(const void* q, const void* k, const void* v,
   e = scratch_address(&base);
   if (e != cudaSuccess) return cuda_failure(e);
   a.status = reinterpret_cast<int*>(base);
-  a.chunk_delta = reinterpret_cast<float*>(base + kStatusBytes);
-  a.chunk_state = reinterpret_cast<__nv_bfloat16*>(base + kStatusBytes + kDeltaBytes);
+  a.chunk_state = reinterpret_cast<__nv_bfloat16*>(base + kStatusBytes);
   a.n_chunks = n_chunks;
-  // The array keeps whatever the previous call left.  Only the status word has to start at
-  // zero: every state the forward reads is rewritten by this call's own pre-pass first.
+  // The array keeps whatever the previous call left.  Only the status block (status word and
+  // the forward's work counter) has to start at zero: every state the forward reads is rewritten
+  // by this call's own pre-pass first.
   e = cudaMemsetAsync(base, 0, kStatusBytes, s);
   if (e != cudaSuccess) return cuda_failure(e);
   e = launch_tc_forward(a, s);

@@ -1034,8 +1034,15 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
   // reverse states of the residual branch: chunks c with a query tile beyond c + wt
   const int n_r = rla_on && a.mode != RATTN_MODE_FULL_CAUSAL ? n_qt - wt - 1 : 0;
   // R_c for c = 0 .. n_r-1: walk the query tiles from the last one down to wt+1
-  e = launch_tc_states(a.q, g_r, a.rstate, a.T, (int)nkv, a.group, a.n_chunks, n_r, n_qt - 1, -1, n_qt - wt - 2,
-                       a.status, "tc_state_bwd", s);
+  {
+    StateLaunch L;
+    L.x = a.q; L.y = g_r; L.out = a.rstate;
+    L.T = a.T; L.n_kv = (int)nkv; L.group = a.group; L.n_chunks = a.n_chunks;
+    L.n_steps = n_r; L.first = n_qt - 1; L.dir = -1; L.out_first = n_qt - wt - 2;
+    L.store_every = 1; L.store_phase = 0; L.row_limit = 0; L.final_out = nullptr;
+    L.status = a.status; L.name = "tc_state_bwd";
+    e = launch_tc_states(L, s);
+  }
   if (e != cudaSuccess) return e;
 
   BwdArgs t;

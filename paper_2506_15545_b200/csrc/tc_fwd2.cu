@@ -41,9 +41,14 @@ constexpr int F_SMEM = F_OFF_BAR + 512;
 constexpr int F_THREADS = 384;
 constexpr float LOG2E = 1.4426950408889634f;
 
+constexpr int SCHED_SLOTS = 4;
+constexpr int SCHED_READERS = 256 + 1 + 64;      // row threads, the MMA warp's lane 0, the converter threads
+
 struct FBars {
   uint64_t q_full[2], q_free[2], kv_full[2], v_ready[2], kv_free[2], x_full, x_free;
   uint64_t s_full[2], p_ready[2], o_ready[2], stash_done[2], phiq_ready[2], phik_ready[2], o_free[2], y_done[2], drain;
+  uint64_t sched_full[SCHED_SLOTS], sched_free[SCHED_SLOTS];
+  int sched_unit[SCHED_SLOTS];
   uint32_t tmem_base;
   int abort;
 };
@@ -55,7 +60,10 @@ struct FArgs {
   const float* gamma_swa;
   const float* gamma_rla;
   int* status;
+  int* work_counter;      // next unit to hand out (device memory, zero at launch); null: static round-robin
   int T, w, H_q, group, mode, n_chunks, n_qt, n_pairs, n_units, n_bh;
+  int n_stateless;        // pairs whose tiles read no stored state; their units come first
+  int wait_for_states;    // a chunk-state kernel runs ahead of this one: wait for it before the first state load
   float scale_log2, eps;
 };
 
@@ -78,9 +86,11 @@ struct Unit {
 
 __device__ __forceinline__ Unit make_unit(const FArgs& a, int u) {
   Unit un;
-  const int pr = u / a.n_bh;                     // heaviest pairs first
+  // Order: first the pairs that read no stored state (they can run while the chunk-state kernel
+  // is still at work), then the others, heaviest first.
+  const int pr = u / a.n_bh;
   un.bh_q = u % a.n_bh;
-  const int p = a.n_pairs - 1 - pr;
+  const int p = pr < a.n_stateless ? pr : a.n_pairs - 1 - (pr - a.n_stateless);
   const int b = un.bh_q / a.H_q;
   un.h = un.bh_q % a.H_q;
   un.bh_kv = b * (a.H_q / a.group) + un.h / a.group;
@@ -118,10 +128,47 @@ __device__ __forceinline__ void mma_pv(uint32_t d, uint32_t p_tmem, uint32_t v_b
   for (int k = 0; k < 8; ++k) mma_bf16_ts(d, p_tmem + 8 * k, b0 + kstep_mn(k), idesc, (acc || k > 0) ? 1u : 0u);
 }
 
+// ------------------------------------------------------------------------------ work units
+// The loader warp draws the CTA's next unit (from a device-wide counter, so that CTAs that start
+// late -- their SM was still running the chunk-state kernel -- simply take fewer units) and
+// publishes it in a small ring; the other roles read the ring in order.  A slot is rewritten
+// only after every reader has read it.
+__device__ __forceinline__ bool sched_next_producer(const FArgs& a, FBars* bars, int n, int* u_out) {
+  const int slot = n % SCHED_SLOTS, use = n / SCHED_SLOTS;
+  if (use >= 1) { if (!mbar_wait_warp(&bars->sched_free[slot], (use - 1) & 1, &bars->abort)) return false; }
+  int u = 0;
+  if (a.work_counter) {
+    if ((threadIdx.x & 31) == 0) u = atomicAdd(a.work_counter, 1);
+    u = __shfl_sync(0xffffffffu, u, 0);
+  } else {
+    u = blockIdx.x + n * gridDim.x;
+  }
+  if (u >= a.n_units) u = -1;
+  if ((threadIdx.x & 31) == 0) {
+    bars->sched_unit[slot] = u;
+    mbar_arrive(&bars->sched_full[slot]);
+  }
+  __syncwarp();
+  *u_out = u;
+  return true;
+}
+// every reading thread calls this; `arrives` says whether this thread is one of the counted readers
+__device__ __forceinline__ bool sched_next(FBars* bars, int n, bool arrives, int* u_out) {
+  const int slot = n % SCHED_SLOTS, use = n / SCHED_SLOTS;
+  if (!mbar_wait(&bars->sched_full[slot], use & 1, &bars->abort)) return false;
+  *u_out = bars->sched_unit[slot];
+  if (arrives) mbar_arrive(&bars->sched_free[slot]);
+  return true;
+}
+
 // ----------------------------------------------------------------------------- loader
 __device__ bool fwd_loader(const FMaps& tm, const FArgs& a, unsigned char* smem, FBars* bars) {
   int kv_count = 0, cntU[2] = {0, 0}, cntX = 0;
-  for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+  bool states_ready = (a.wait_for_states == 0);
+  for (int n = 0;; ++n) {
+    int u;
+    if (!sched_next_producer(a, bars, n, &u)) return false;
+    if (u < 0) break;
     const Unit un = make_unit(a, u);
 #pragma unroll
     for (int X = 0; X < 2; ++X) {
@@ -147,6 +194,11 @@ __device__ bool fwd_loader(const FMaps& tm, const FArgs& a, unsigned char* smem,
         const int done_before = cntU[X] - (un.t[X] >= 0 ? 1 : 0);      // epilogues of tile X before this unit
         if (done_before >= 1) WAIT_OR_RETURN_W(bars->y_done[X], (done_before - 1) & 1);
       }
+      if (!states_ready) {
+        // the chunk-state kernel launched ahead of this one has completed and its stores are visible
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        states_ready = true;
+      }
       mbar_arrive_expect_tx(&bars->x_full, TILE_BYTES);
       load_tile(smem + F_OFF_X, &tm.st, &bars->x_full, 0, un.bh_kv * a.n_chunks + un.cA);
       ++cntX;
@@ -158,7 +210,10 @@ __device__ bool fwd_loader(const FMaps& tm, const FArgs& a, unsigned char* smem,
 // -------------------------------------------------------------------------- V re-encoding
 __device__ bool fwd_convert(const FArgs& a, unsigned char* smem, FBars* bars, int cid) {
   int kv_count = 0;
-  for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+  for (int n = 0;; ++n) {
+    int u;
+    if (!sched_next(bars, n, true, &u)) return false;
+    if (u < 0) break;
     const Unit un = make_unit(a, u);
     for (int i = 0; i < un.n; ++i, ++kv_count) {
       const int st = kv_count & 1, use = kv_count >> 1;
@@ -187,7 +242,11 @@ __device__ bool fwd_mma(const FArgs& a, unsigned char* smem, FBars* bars, uint32
   const uint32_t tS[2] = {tmem, tmem + 128}, tO[2] = {tmem + 256, tmem + 384};
   int kv_count = 0, cntU[2] = {0, 0}, cntX = 0, cntP[2] = {0, 0}, cntR[2] = {0, 0}, cntK[2] = {0, 0};
 
-  for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+  for (int n = 0;; ++n) {
+    int u;
+    if (!sched_next(bars, n, (threadIdx.x & 31) == 0, &u)) return false;
+    u = __shfl_sync(0xffffffffu, u, 0);
+    if (u < 0) break;
     const Unit un = make_unit(a, u);
     const int kv0 = kv_count;
     auto stage_of = [&](int i) { return (kv0 + i) & 1; };
@@ -317,7 +376,10 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
   unsigned char* sQ = smem + F_OFF_Q + X * TILE_BYTES;
   int kv_count = 0, cntS = 0, cntO = 0;
 
-  for (int u = blockIdx.x; u < a.n_units; u += gridDim.x) {
+  for (int n = 0;; ++n) {
+    int u;
+    if (!sched_next(bars, n, true, &u)) return false;
+    if (u < 0) break;
     const Unit un = make_unit(a, u);
     const int kv0 = kv_count;
     kv_count += un.n;
@@ -634,6 +696,10 @@ tc_fwd2_kernel(const __grid_constant__ FMaps tm, FArgs a) {
     mbar_init(&bars->x_full, 1);
     mbar_init(&bars->x_free, 1);
     mbar_init(&bars->drain, 1);
+    for (int i = 0; i < SCHED_SLOTS; ++i) {
+      mbar_init(&bars->sched_full[i], 1);
+      mbar_init(&bars->sched_free[i], SCHED_READERS);
+    }
     bars->abort = 0;
     fence_mbar_init();
   }
@@ -678,7 +744,7 @@ tc_fwd2_kernel(const __grid_constant__ FMaps tm, FArgs a) {
 
 }  // namespace
 
-cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s) {
+cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_states) {
   FMaps tm;
   if (!make_map(&tm.q, a.q, a.T, (uint64_t)a.B * a.H_q) || !make_map(&tm.k, a.k, a.T, (uint64_t)a.B * a.H_kv) ||
       !make_map(&tm.v, a.v, a.T, (uint64_t)a.B * a.H_kv) || !make_map(&tm.out, a.out, a.T, (uint64_t)a.B * a.H_q) ||
@@ -695,6 +761,14 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s) {
   t.n_bh = a.B * a.H_q;
   t.n_units = t.n_pairs * t.n_bh;
   t.scale_log2 = a.scale * LOG2E; t.eps = a.eps;
+  // pairs p with 2p - w/128 <= 0 read no stored state
+  t.n_stateless = 0;
+  if (a.mode == RATTN_MODE_RATTN && after_states) {
+    t.n_stateless = (a.w / TILE) / 2 + 1;
+    if (t.n_stateless > t.n_pairs) t.n_stateless = t.n_pairs;
+  }
+  t.wait_for_states = after_states ? 1 : 0;
+  t.work_counter = a.status ? a.status + 2 : nullptr;
   int dev = 0, n_sm = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
@@ -705,7 +779,21 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s) {
   const int grid = t.n_units < n_sm ? t.n_units : n_sm;
   {
     KernelTimer kt("tc_fwd", s);
-    tc_fwd2_kernel<<<grid, F_THREADS, F_SMEM, s>>>(tm, t);
+    // Programmatic dependent launch: when a chunk-state kernel precedes it on the stream, this
+    // kernel may begin while that one is still running; its loader waits (griddepcontrol.wait)
+    // before the first state load.  Without a preceding state kernel the attribute changes nothing.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(F_THREADS);
+    cfg.dynamicSmemBytes = F_SMEM;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = after_states ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, tc_fwd2_kernel, tm, t);
+    if (e != cudaSuccess) return e;
   }
   count_launches(1);
   return cudaGetLastError();

@@ -81,9 +81,8 @@ def test_workspace_size_follows_mode_and_flags(B):
     assert infer < train < train_generic                                 # bf16 against fp32 residuals
     assert B.rattn_workspace_bytes(*c5) == max(train, train_generic)     # the bound covers every case
     assert B.rattn_workspace_bytes_ex(*c5, B.RATTN_BF16, 7, 0) == 0      # unknown mode
-    # few K/V heads: the parallel state form keeps its fp32 blocks too
     few = (1, 4, 2, 1024, 128, 128)
-    assert B.rattn_workspace_bytes_ex(*few, B.RATTN_BF16, B.MODE_RATTN, 0) == 256 + 2 * 8 * 128 * 128 * (2 + 4)
+    assert B.rattn_workspace_bytes_ex(*few, B.RATTN_BF16, B.MODE_RATTN, 0) == 256 + 2 * 8 * 128 * 128 * 2
 
 
 def _p(bind, **kw):

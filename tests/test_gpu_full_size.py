@@ -122,12 +122,12 @@ def _prefill_then_decode(wl, pairs, n_random=32):
 def test_config5_long_prefill_then_decode_full_batch():
     """The configuration as stated: B=32, H=32/8, d=128, w=512, prefill T=32768 (q, k, v, out
     21.5 GB, chunk states 2.1 GB), then 256 decode steps with the ring and state the prefill
-    hands over.  256 K/V heads: the chunk states come from the serial one-CTA-per-head chain,
-    255 steps long.  Oracle on sampled rows of three heads and on all 256 decode rows."""
+    hands over.  256 K/V heads, each a chain of 256 chunk steps in the state kernel (two waves of CTAs),
+    which also leaves the fp32 decode state.  Oracle on sampled rows of three heads and on all 256 decode rows."""
     _prefill_then_decode(W.C5, [(0, 0), (13, 6), (31, 31)], n_random=24)
 
 
-def test_config5_few_heads_take_the_parallel_state_form():
-    """Four batch entries of the same configuration (32 K/V heads in all): too few heads for a
-    chain per SM, so the chunk states are formed per chunk in parallel and prefix-summed."""
+def test_config5_few_heads():
+    """Four batch entries of the same configuration (32 K/V heads in all): the chunk-state chains
+    occupy only 32 SMs while the main kernel already runs on the others."""
     _prefill_then_decode(W.C5.replace(B=4), [(0, 0), (3, 31)])
