@@ -15,7 +15,8 @@ What it computes, for one query head (row vectors, 0-indexed positions t, j):
   that ends at token ``t-w-1``.  It is evaluated as the explicit quadratic sum; no
   recurrence, no chunking;
 * the feature map ``phi`` (Section 3.1, "Parameterization"): a softmax over the head
-  features, same map for q and k, ``d' = d``;
+  features, same map for q and k, ``d' = d``; the two alternatives of the paper's ablation
+  (Table 6: ReLU, identity) are selectable and change nothing else;
 * the combination (Section 3.2): ``y_t = rmsnorm(o_swa_t; g_swa) + rmsnorm(o_rla_t; g_rla)``
   with two separate per-head RMS norms, ``eps`` inside the square root;
 * grouped-query sharing (Section 3.1, "Group-Query Variant"): query head ``h`` reads
@@ -43,10 +44,20 @@ MODE_FULL_CAUSAL = 2
 
 DEFAULT_EPS = 1e-6
 
+PHI_SOFTMAX = 0      # the paper's choice (Section 3.1)
+PHI_RELU = 1         # ablation, Table 6
+PHI_IDENTITY = 2     # ablation, Table 6
 
-def feature_map(x: np.ndarray) -> np.ndarray:
-    """phi(x): softmax over the last axis (Section 3.1, softmax-based feature map)."""
+
+def feature_map(x: np.ndarray, phi: int = PHI_SOFTMAX) -> np.ndarray:
+    """phi(x) over the last axis: softmax (Section 3.1, softmax-based feature map), or one
+    of the ablation's element-wise maps: max(x, 0), x (Table 6)."""
     x = np.asarray(x, dtype=np.float64)
+    if phi == PHI_RELU:
+        return np.maximum(x, 0.0)
+    if phi == PHI_IDENTITY:
+        return x.copy()
+    assert phi == PHI_SOFTMAX
     e = np.exp(x - x.max(axis=-1, keepdims=True))
     return e / e.sum(axis=-1, keepdims=True)
 
@@ -90,17 +101,17 @@ def swa_rows(q_rows, rows, k, v, w, scale):
     return p @ v, p
 
 
-def rla_rows(q_rows, rows, k, v, w):
+def rla_rows(q_rows, rows, k, v, w, phi=PHI_SOFTMAX):
     """RLA outputs for the listed query rows of one head: Eq. 4 unrolled into the
     explicit sum over residual tokens.  Returns (o_rla [n, d], a [n, T])."""
     T = k.shape[0]
-    a = feature_map(q_rows) @ feature_map(k).T
+    a = feature_map(q_rows, phi) @ feature_map(k, phi).T
     a = np.where(rla_mask(rows, T, w), a, 0.0)
     return a @ v, a
 
 
 def forward_head(q, k, v, w, scale=1.0, eps=DEFAULT_EPS, gamma_swa=None, gamma_rla=None,
-                 mode=MODE_RATTN, rows=None, row_block=512, parts=False):
+                 mode=MODE_RATTN, rows=None, row_block=512, parts=False, phi=PHI_SOFTMAX):
     """The operator for one query head.  q, k, v: [T, d].  ``rows`` selects output rows
     (default all).  Returns y [n, d], or (y, o_swa, o_rla) when ``parts`` is set."""
     q = np.asarray(q, dtype=np.float64)
@@ -116,7 +127,7 @@ def forward_head(q, k, v, w, scale=1.0, eps=DEFAULT_EPS, gamma_swa=None, gamma_r
         r = rows[lo:lo + row_block]
         o_s[lo:lo + len(r)], _ = swa_rows(q[r], r, k, v, w, scale)
         if mode == MODE_RATTN:
-            o_r[lo:lo + len(r)], _ = rla_rows(q[r], r, k, v, w)
+            o_r[lo:lo + len(r)], _ = rla_rows(q[r], r, k, v, w, phi)
     y = rmsnorm(o_s, gamma_swa, eps)
     if mode == MODE_RATTN:
         y = y + rmsnorm(o_r, gamma_rla, eps)
@@ -128,7 +139,7 @@ def _gain(gamma, h):
 
 
 def forward(q, k, v, w, scale=1.0, eps=DEFAULT_EPS, gamma_swa=None, gamma_rla=None,
-            mode=MODE_RATTN):
+            mode=MODE_RATTN, phi=PHI_SOFTMAX):
     """The operator for a batch.  q [B, H_q, T, d]; k, v [B, H_kv, T, d]; gains [H_q, d]
     or None.  Query head h uses K/V head h // (H_q // H_kv)."""
     q = np.asarray(q, dtype=np.float64)
@@ -140,25 +151,25 @@ def forward(q, k, v, w, scale=1.0, eps=DEFAULT_EPS, gamma_swa=None, gamma_rla=No
     for b in range(B):
         for h in range(Hq):
             y[b, h] = forward_head(q[b, h], k[b, h // g], v[b, h // g], w, scale, eps,
-                                   _gain(gamma_swa, h), _gain(gamma_rla, h), mode)
+                                   _gain(gamma_swa, h), _gain(gamma_rla, h), mode, phi=phi)
     return y
 
 
 def forward_rows(q_head, k_head, v_head, rows, w, scale=1.0, eps=DEFAULT_EPS,
-                 gamma_swa=None, gamma_rla=None, mode=MODE_RATTN):
+                 gamma_swa=None, gamma_rla=None, mode=MODE_RATTN, phi=PHI_SOFTMAX):
     """Selected output rows of one head, each from the full definition (rows are
     independent of one another, so sampling rows is exact)."""
     return forward_head(q_head, k_head, v_head, w, scale, eps, gamma_swa, gamma_rla,
-                        mode, rows=rows)
+                        mode, rows=rows, phi=phi)
 
 
 def decode_row(q_hist, k_hist, v_hist, pos, w, scale=1.0, eps=DEFAULT_EPS,
-               gamma_swa=None, gamma_rla=None):
+               gamma_swa=None, gamma_rla=None, phi=PHI_SOFTMAX):
     """Output of the decode step at position ``pos``: the same definition evaluated on
     the full history [0..pos] -- no ring buffer, no running state."""
     n = pos + 1
     return forward_head(q_hist[:n], k_hist[:n], v_hist[:n], w, scale, eps, gamma_swa,
-                        gamma_rla, rows=np.array([pos]))[0]
+                        gamma_rla, rows=np.array([pos]), phi=phi)[0]
 
 
 def _rmsnorm_bwd(x, gamma, eps, dy):
@@ -172,13 +183,18 @@ def _rmsnorm_bwd(x, gamma, eps, dy):
     return dx, dgamma
 
 
-def _feature_map_bwd(phi, dphi):
-    """Gradient through the softmax feature map: dx = phi * (dphi - <dphi, phi>)."""
-    return phi * (dphi - (dphi * phi).sum(axis=-1, keepdims=True))
+def _feature_map_bwd(f, df, x=None, phi=PHI_SOFTMAX):
+    """Gradient through the feature map, f = phi(x), df = dL/df.
+    softmax: dx = f * (df - <df, f>);  ReLU: dx = df where x > 0;  identity: dx = df."""
+    if phi == PHI_RELU:
+        return np.where(np.asarray(x) > 0.0, df, 0.0)
+    if phi == PHI_IDENTITY:
+        return df
+    return f * (df - (df * f).sum(axis=-1, keepdims=True))
 
 
 def backward_head(q, k, v, dy, w, scale=1.0, eps=DEFAULT_EPS, gamma_swa=None,
-                  gamma_rla=None, mode=MODE_RATTN):
+                  gamma_rla=None, mode=MODE_RATTN, phi=PHI_SOFTMAX):
     """Gradients of L = sum(y * dy) for one query head, by the chain rule through the
     dense [T, T] weight matrices of both branches.  Returns dq, dk, dv (this head's
     contribution to its K/V head), dgamma_swa, dgamma_rla."""
@@ -205,19 +221,19 @@ def backward_head(q, k, v, dy, w, scale=1.0, eps=DEFAULT_EPS, gamma_swa=None,
 
     if mode == MODE_RATTN:
         # RLA branch: y_r = rmsnorm(A V), A = (phi(q) phi(k)^T) masked to j < t-w
-        fq = feature_map(q)
-        fk = feature_map(k)
-        o_r, a = rla_rows(q, rows, k, v, w)
+        fq = feature_map(q, phi)
+        fk = feature_map(k, phi)
+        o_r, a = rla_rows(q, rows, k, v, w, phi)
         do_r, dgr = _rmsnorm_bwd(o_r, gr, eps, dy)
         dv = dv + a.T @ do_r
         da = np.where(rla_mask(rows, T, w), do_r @ v.T, 0.0)
-        dq = dq + _feature_map_bwd(fq, da @ fk)
-        dk = dk + _feature_map_bwd(fk, da.T @ fq)
+        dq = dq + _feature_map_bwd(fq, da @ fk, q, phi)
+        dk = dk + _feature_map_bwd(fk, da.T @ fq, k, phi)
     return dq, dk, dv, dgs, dgr
 
 
 def backward(q, k, v, dy, w, scale=1.0, eps=DEFAULT_EPS, gamma_swa=None, gamma_rla=None,
-             mode=MODE_RATTN):
+             mode=MODE_RATTN, phi=PHI_SOFTMAX):
     """Batch gradients.  dk, dv of a K/V head sum over the query heads of its group.
     Returns dq [B,H_q,T,d], dk, dv [B,H_kv,T,d], dgamma_swa, dgamma_rla [H_q,d]."""
     q = np.asarray(q, dtype=np.float64)
@@ -234,7 +250,7 @@ def backward(q, k, v, dy, w, scale=1.0, eps=DEFAULT_EPS, gamma_swa=None, gamma_r
     for b in range(B):
         for h in range(Hq):
             r = backward_head(q[b, h], k[b, h // g], v[b, h // g], dy[b, h], w, scale, eps,
-                              _gain(gamma_swa, h), _gain(gamma_rla, h), mode)
+                              _gain(gamma_swa, h), _gain(gamma_rla, h), mode, phi)
             dq[b, h] = r[0]
             dk[b, h // g] += r[1]
             dv[b, h // g] += r[2]
@@ -243,10 +259,10 @@ def backward(q, k, v, dy, w, scale=1.0, eps=DEFAULT_EPS, gamma_swa=None, gamma_r
     return dq, dk, dv, dgs, dgr
 
 
-def rla_state(k, v, n_tokens):
+def rla_state(k, v, n_tokens, phi=PHI_SOFTMAX):
     """S = sum_{j < n_tokens} phi(k_j)^T v_j, the [d, d] state of Eq. 4 after n_tokens
     tokens (zero for n_tokens <= 0).  Used to check the state a prefill hands to decode."""
     k = np.asarray(k, dtype=np.float64)
     v = np.asarray(v, dtype=np.float64)
     n = max(0, min(int(n_tokens), k.shape[0]))
-    return feature_map(k[:n]).T @ v[:n]
+    return feature_map(k[:n], phi).T @ v[:n]

@@ -195,41 +195,76 @@ __device__ __forceinline__ uint32_t bits_gt(int rd) { return bits_ge(rd + 1); }
 __device__ __forceinline__ uint32_t bits_le(int rd) { return ~bits_gt(rd); }
 __device__ __forceinline__ uint32_t bits_lt(int rd) { return ~bits_ge(rd); }
 
+// Maximum of 32 registers as four independent chains (the row threads run two or three warps per
+// scheduler, so a 32-long dependent chain would sit exposed at full latency).
+__device__ __forceinline__ float max32(const float (&x)[32]) {
+  float m0 = x[0], m1 = x[1], m2 = x[2], m3 = x[3];
+#pragma unroll
+  for (int e = 4; e < 32; e += 4) {
+    m0 = fmaxf(m0, x[e]);
+    m1 = fmaxf(m1, x[e + 1]);
+    m2 = fmaxf(m2, x[e + 2]);
+    m3 = fmaxf(m3, x[e + 3]);
+  }
+  return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+}
+__device__ __forceinline__ float max32_masked(const float (&x)[32], uint32_t keep) {
+  float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+  for (int e = 0; e < 32; e += 4) {
+    m0 = fmaxf(m0, (keep >> e) & 1u ? x[e] : -INFINITY);
+    m1 = fmaxf(m1, (keep >> (e + 1)) & 1u ? x[e + 1] : -INFINITY);
+    m2 = fmaxf(m2, (keep >> (e + 2)) & 1u ? x[e + 2] : -INFINITY);
+    m3 = fmaxf(m3, (keep >> (e + 3)) & 1u ? x[e + 3] : -INFINITY);
+  }
+  return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+}
+
 // The helpers below walk a row in sixteen 16-byte steps with a rolled loop: compact code
 // matters more than loop overhead here (large unrolled kernels are instruction-fetch bound).
 // Row maximum of row r of a swizzled bf16 tile.
 __device__ __forceinline__ float row_max_bf16(const unsigned char* tile, int r) {
-  float m = -INFINITY;
-#pragma unroll 1
-  for (int c = 0; c < 16; ++c) {
+  // packed bf16 maxima (two values per instruction), four independent chains
+  __nv_bfloat162 m[4];
+  {
+    const uint4 u = *reinterpret_cast<const uint4*>(tile + swz(r, 0));
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) m[e] = h[e];
+  }
+#pragma unroll 3
+  for (int c = 1; c < 16; ++c) {
     const uint4 u = *reinterpret_cast<const uint4*>(tile + swz(r, c));
     const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const float2 f = __bfloat1622float2(h[e]);
-      m = fmaxf(m, fmaxf(f.x, f.y));
-    }
+    for (int e = 0; e < 4; ++e) m[e] = __hmax2(m[e], h[e]);
   }
-  return m;
+  const float2 f = __bfloat1622float2(__hmax2(__hmax2(m[0], m[1]), __hmax2(m[2], m[3])));
+  return fmaxf(f.x, f.y);
 }
 // x -> exp(x - max) over row r, in place, as fp16 (FP16 = true) or bf16; returns the row sum.
 template <bool FP16>
 __device__ __forceinline__ float row_exp_inplace(unsigned char* tile, int r, float ml) {
-  float sum = 0.f;
-#pragma unroll 1
+  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll 2
   for (int c = 0; c < 16; ++c) {
     uint4 u = *reinterpret_cast<const uint4*>(tile + swz(r, c));
     uint32_t* w = reinterpret_cast<uint32_t*>(&u);
+    float ex[8];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[e]));
-      const float e0 = ex2(f.x * 1.4426950408889634f - ml), e1 = ex2(f.y * 1.4426950408889634f - ml);
-      sum += e0 + e1;
-      w[e] = FP16 ? pack_f16(e0, e1) : pack_bf16(e0, e1);
+      ex[2 * e] = ex2(f.x * 1.4426950408889634f - ml);
+      ex[2 * e + 1] = ex2(f.y * 1.4426950408889634f - ml);
+      w[e] = FP16 ? pack_f16(ex[2 * e], ex[2 * e + 1]) : pack_bf16(ex[2 * e], ex[2 * e + 1]);
     }
+    s0 += ex[0] + ex[4];
+    s1 += ex[1] + ex[5];
+    s2 += ex[2] + ex[6];
+    s3 += ex[3] + ex[7];
     *reinterpret_cast<uint4*>(tile + swz(r, c)) = u;
   }
-  return sum;
+  return (s0 + s1) + (s2 + s3);
 }
 // Un-normalised feature map of row r, in place: x -> exp(x - max) (bf16); returns 1 / sum so
 // that the caller can scale whatever is linear in this row afterwards.

@@ -115,6 +115,19 @@ __device__ __forceinline__ Unit make_unit(const FArgs& a, int u) {
 
 __device__ __forceinline__ bool active(const Unit& un, int X, int i) { return un.t[X] >= 0 && i >= un.i0[X] && i <= un.i1[X]; }
 
+// Optional timeline for tuning (compiled in only with -DRATTN_TIMELINE): one CTA records
+// (event id, clock) pairs per role.
+#ifdef RATTN_TIMELINE
+__device__ unsigned long long g_timeline[4][2048];
+__device__ int g_timeline_n[4];
+#define TL_DECL(on_expr) const bool tl_on = (on_expr); int tl_i = 0; (void)tl_on; (void)tl_i
+#define TL(role, id) do { if (tl_on && tl_i < 1000) { unsigned long long c_; asm volatile("mov.u64 %0, %%clock64;" : "=l"(c_) :: "memory"); \
+    g_timeline[role][2 * tl_i] = (unsigned long long)(id); g_timeline[role][2 * tl_i + 1] = c_; ++tl_i; g_timeline_n[role] = tl_i; } } while (0)
+#else
+#define TL_DECL(on_expr) do { } while (0)
+#define TL(role, id) do { } while (0)
+#endif
+
 #define WAIT_OR_RETURN(bar, parity) \
   do { if (!mbar_wait(&(bar), (parity), &bars->abort)) return false; } while (0)
 #define WAIT_OR_RETURN_W(bar, parity) \
@@ -375,6 +388,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
   const uint32_t tS = tmem + 128 * X + lane_base(r), tO = tmem + 256 + 128 * X + lane_base(r);
   unsigned char* sQ = smem + F_OFF_Q + X * TILE_BYTES;
   int kv_count = 0, cntS = 0, cntO = 0;
+  TL_DECL(blockIdx.x == 7 && r == 0);
 
   for (int n = 0;; ++n) {
     int u;
@@ -390,29 +404,29 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     const int t = q0 + r;
 
     // ---- window branch: online softmax over the key tiles of the band -------------------
+    // On the two edge tiles of the band a warp's 32 rows keep whole 32-column chunks, drop whole
+    // chunks (no score reads, no exponentials: zero weights) and mask exactly one chunk, the one
+    // their own positions fall into: diagonal tile -> chunks 0 .. wq, oldest tile -> chunks wq .. 3.
     float m_ref = -INFINITY, l = 0.f;
+    const int wq = r >> 5;                         // this warp's quarter of the tile's rows
 #pragma unroll 1
     for (int i = i0; i <= i1; ++i) {
       const int kt = un.kt_hi - i;
+      TL(X, 100 + i);
       WAIT_OR_RETURN(bars->s_full[X], cntS & 1);
+      TL(X, 200 + i);
       ++cntS;
       tc_fence_after();
       const bool diag = (kt == tX), bound = un.windowed && (kt == tX - un.wt);
+      const int c_lo = bound ? wq : 0, c_hi = diag ? wq : 3;     // chunks with kept columns
       // pass 1 over the scores: row maximum
       float mx = -INFINITY;
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
+      for (int c = c_lo; c <= c_hi; ++c) {
         float x[32];
         tmem_ld32(tS + 32 * c, x);
         tmem_wait_ld();
-        if (diag || bound) {                       // only the two edge tiles of the band need a mask
-          const uint32_t keep = keep_bits(r, c, diag, bound);
-#pragma unroll
-          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, (keep >> e) & 1u ? x[e] : -INFINITY);
-        } else {
-#pragma unroll
-          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, x[e]);
-        }
+        mx = fmaxf(mx, ((diag || bound) && c == wq) ? max32_masked(x, keep_bits(r, c, diag, bound)) : max32(x));
       }
       mx *= a.scale_log2;                                              // scale > 0
       // lazy rescale: the reference maximum only moves when the row maximum grew by more than 2^8
@@ -435,30 +449,40 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
         l *= f;
         m_ref = m_new;
       }
+      TL(X, 300 + i);
       // pass 2: weights, written back (fp16, two per column) over score columns already consumed
       float psum = 0.f;
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
-        float x[32];
-        tmem_ld32(tS + 32 * c, x);
-        tmem_wait_ld();
         uint32_t pk[16];
-        if (diag || bound) {
-          const uint32_t keep = keep_bits(r, c, diag, bound);
+        if (c < c_lo || c > c_hi) {
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const float p0 = (keep >> (2 * e)) & 1u ? ex2(x[2 * e] * a.scale_log2 - m_ref) : 0.f;
-            const float p1 = (keep >> (2 * e + 1)) & 1u ? ex2(x[2 * e + 1] * a.scale_log2 - m_ref) : 0.f;
-            psum += p0 + p1;
-            pk[e] = pack_f16(p0, p1);
-          }
+          for (int e = 0; e < 16; ++e) pk[e] = 0u;
         } else {
+          float x[32];
+          tmem_ld32(tS + 32 * c, x);
+          tmem_wait_ld();
+          float ps[4] = {0.f, 0.f, 0.f, 0.f};
+          if ((diag || bound) && c == wq) {
+            const uint32_t keep = keep_bits(r, c, diag, bound);
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const float p0 = ex2(x[2 * e] * a.scale_log2 - m_ref), p1 = ex2(x[2 * e + 1] * a.scale_log2 - m_ref);
-            psum += p0 + p1;
-            pk[e] = pack_f16(p0, p1);
+            for (int e = 0; e < 16; ++e) {
+              const float p0 = (keep >> (2 * e)) & 1u ? ex2(x[2 * e] * a.scale_log2 - m_ref) : 0.f;
+              const float p1 = (keep >> (2 * e + 1)) & 1u ? ex2(x[2 * e + 1] * a.scale_log2 - m_ref) : 0.f;
+              ps[2 * (e & 1)] += p0;
+              ps[2 * (e & 1) + 1] += p1;
+              pk[e] = pack_f16(p0, p1);
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const float p0 = ex2(x[2 * e] * a.scale_log2 - m_ref), p1 = ex2(x[2 * e + 1] * a.scale_log2 - m_ref);
+              ps[2 * (e & 1)] += p0;
+              ps[2 * (e & 1) + 1] += p1;
+              pk[e] = pack_f16(p0, p1);
+            }
           }
+          psum += (ps[0] + ps[1]) + (ps[2] + ps[3]);
         }
         tmem_st16(tS + 16 * c, pk);
       }
@@ -466,6 +490,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&bars->p_ready[X]);
+      TL(X, 400 + i);
     }
 
     // ---- residual branch, first part: feature maps ------------------------------------------
@@ -743,6 +768,16 @@ tc_fwd2_kernel(const __grid_constant__ FMaps tm, FArgs a) {
 }
 
 }  // namespace
+
+#ifdef RATTN_TIMELINE
+extern "C" int rattn_timeline_read(unsigned long long* out, int* n) {
+  cudaMemcpyFromSymbol(out, g_timeline, sizeof(g_timeline));
+  cudaMemcpyFromSymbol(n, g_timeline_n, sizeof(g_timeline_n));
+  int z[4] = {0, 0, 0, 0};
+  cudaMemcpyToSymbol(g_timeline_n, z, sizeof(z));
+  return 0;
+}
+#endif
 
 cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_states) {
   FMaps tm;

@@ -403,3 +403,83 @@ def test_pins_would_catch_an_off_by_one_window(monkeypatch):
     bad, _ = O.rla_rows(q, np.arange(T), k, v, w)
     assert np.abs(bad - _rla_recurrent(q, k, v, w)).max() > 1e-3
     np.testing.assert_allclose(good, _rla_recurrent(q, k, v, w), atol=1e-12)
+
+
+# ------------------------------------------------------------------ ablation feature maps (Table 6)
+
+def _rla_recurrent_phi(q, k, v, w, f):
+    """Eq. 4 as printed, with an arbitrary element-wise map f."""
+    T, d = q.shape
+    S = [np.zeros((d, d))]
+    for t in range(T):
+        S.append(S[-1] + np.outer(f(k[t]), v[t]))
+    out = np.zeros((T, d))
+    for t in range(T):
+        if t - w > 0:
+            out[t] = f(q[t]) @ S[t - w]
+    return out
+
+
+@pytest.mark.parametrize("phi,f", [(O.PHI_RELU, lambda x: np.array([max(a, 0.0) for a in x])),
+                                   (O.PHI_IDENTITY, lambda x: np.array(list(x)))])
+def test_other_feature_maps_quadratic_equals_recurrence(phi, f):
+    """ReLU and identity maps of the paper's ablation: the explicit quadratic sum equals the
+    printed recurrence with the same element-wise map (scalar max / copy written out here),
+    and the library routine agrees on the map itself."""
+    T, d, w = 48, 8, 7
+    q, k, v = _rand(T, d, 31)
+    o, _ = O.rla_rows(q, np.arange(T), k, v, w, phi)
+    np.testing.assert_allclose(o, _rla_recurrent_phi(q, k, v, w, f), atol=1e-12)
+    ref = torch.relu(torch.from_numpy(q)).numpy() if phi == O.PHI_RELU else q
+    assert np.array_equal(O.feature_map(q, phi), ref)
+    np.testing.assert_allclose(O.rla_state(k, v, 13, phi), sum(np.outer(f(k[t]), v[t]) for t in range(13)), atol=1e-13)
+
+
+def test_identity_map_closed_form_with_one_hot_keys():
+    """Identity map, keys k_j = e_{a_j} (one-hot): phi(q_t).phi(k_j) = q_t[a_j], so
+    o_rla_t = sum_{j < t-w} q_t[a_j] v_j.  The same keys under ReLU give the same sum with
+    max(q_t[a_j], 0)."""
+    T, d, w = 30, 8, 4
+    rng = np.random.default_rng(32)
+    q, v = rng.standard_normal((T, d)), rng.standard_normal((T, d))
+    a = rng.integers(0, d, T)
+    k = np.eye(d)[a]
+    for phi, g in ((O.PHI_IDENTITY, lambda x: x), (O.PHI_RELU, lambda x: max(x, 0.0))):
+        _, _, o_r = O.forward_head(q, k, v, w, parts=True, phi=phi)
+        for t in range(T):
+            want = sum((g(q[t, a[j]]) * v[j] for j in range(max(0, t - w))), np.zeros(d))
+            np.testing.assert_allclose(o_r[t], want, atol=1e-13)
+
+
+@pytest.mark.parametrize("phi", [O.PHI_RELU, O.PHI_IDENTITY])
+def test_other_feature_maps_backward_matches_central_differences(phi):
+    rng = np.random.default_rng(33 + phi)
+    B, Hq, Hkv, T, d, w = 1, 2, 1, 96, 8, 9
+    q = rng.standard_normal((B, Hq, T, d))
+    k = rng.standard_normal((B, Hkv, T, d))
+    v = rng.standard_normal((B, Hkv, T, d))
+    dy = rng.standard_normal((B, Hq, T, d))
+    dq, dk, dv, _, _ = O.backward(q, k, v, dy, w, 0.5, phi=phi)
+    loss = lambda q_, k_, v_: float((O.forward(q_, k_, v_, w, 0.5, phi=phi) * dy).sum())
+    h = 1e-6
+    for name, x, g in (("q", q, dq), ("k", k, dk), ("v", v, dv)):
+        for _ in range(3):
+            u = rng.standard_normal(x.shape)
+            args_p = {"q": q, "k": k, "v": v}
+            args_m = dict(args_p)
+            args_p[name] = x + h * u
+            args_m[name] = x - h * u
+            fd = (loss(args_p["q"], args_p["k"], args_p["v"]) - loss(args_m["q"], args_m["k"], args_m["v"])) / (2 * h)
+            an = float((g * u).sum())
+            assert abs(fd - an) <= 2e-6 * max(1.0, abs(an)) + 1e-6, (name, fd, an)
+
+
+def test_other_feature_maps_keep_the_window_branch_and_differ_from_softmax():
+    T, d, w = 40, 8, 5
+    q, k, v = _rand(T, d, 35)
+    base = O.forward_head(q, k, v, w, parts=True)
+    for phi in (O.PHI_RELU, O.PHI_IDENTITY):
+        y, o_s, o_r = O.forward_head(q, k, v, w, parts=True, phi=phi)
+        assert np.array_equal(o_s, base[1])                   # the map touches the linear branch only
+        assert np.all(o_r[:w + 1] == 0)
+        assert np.abs(o_r[w + 1:] - base[2][w + 1:]).max() > 1e-3
