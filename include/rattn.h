@@ -58,6 +58,14 @@ typedef enum rattn_mode {
   RATTN_MODE_FULL_CAUSAL = 2     /* w := T: y = rmsnorm(causal softmax attention) */
 } rattn_mode;
 
+/* The feature map phi of the linear branch (Section 3.1, "Parameterization").  The paper's
+ * models use the softmax map; its ablation (Table 6) also tries ReLU and the identity. */
+typedef enum rattn_feature_map {
+  RATTN_PHI_SOFTMAX = 0,         /* softmax over the d head features */
+  RATTN_PHI_RELU = 1,            /* max(x, 0), element-wise */
+  RATTN_PHI_IDENTITY = 2         /* x */
+} rattn_feature_map;
+
 /* Path selection for rattn_params.flags. */
 #define RATTN_FLAG_FORCE_GENERIC 1u  /* use the portable fp32-FMA kernels even where the
                                         tensor-core path applies (debugging / comparison) */
@@ -87,6 +95,7 @@ typedef enum rattn_mode {
  *              phi(k_j)^T v_j; rings [B,H_kv,w,d] (I/O dtype) holding token j at slot
  *              j % w for the last min(w,T) tokens (other slots zero).
  *   dgamma_swa, dgamma_rla   optional fp32 [H_q,d] outputs of rattn_backward_ex.
+ *   feature_map   phi of the linear branch (forward, backward and decode must agree).
  */
 typedef struct rattn_params {
   const void* q;
@@ -113,7 +122,7 @@ typedef struct rattn_params {
   float* dgamma_swa;
   float* dgamma_rla;
   uint32_t flags;                /* RATTN_FLAG_* */
-  uint32_t reserved;
+  int32_t feature_map;           /* rattn_feature_map; 0 = the paper's softmax map */
 } rattn_params;
 
 /*

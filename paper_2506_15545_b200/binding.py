@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "librattn.so")
 RATTN_BF16, RATTN_F32 = 0, 1
 MODE_RATTN, MODE_SWA_ONLY, MODE_FULL_CAUSAL = 0, 1, 2
 FLAG_FORCE_GENERIC, FLAG_SAVE_RESIDUALS = 1, 2
+PHI_SOFTMAX, PHI_RELU, PHI_IDENTITY = 0, 1, 2
 
 EXPORTS = (
     "rattn_forward", "rattn_forward_ex", "rattn_backward", "rattn_backward_ex",
@@ -43,7 +44,7 @@ class RattnParams(ctypes.Structure):
         ("dout", ctypes.c_void_p), ("dq", ctypes.c_void_p), ("dk", ctypes.c_void_p),
         ("dv", ctypes.c_void_p), ("dgamma_swa", ctypes.c_void_p),
         ("dgamma_rla", ctypes.c_void_p),
-        ("flags", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+        ("flags", ctypes.c_uint32), ("feature_map", ctypes.c_int32),
     ]
 
 
@@ -155,8 +156,9 @@ def alloc_workspace(q, k, w, mode=None, flags=None) -> torch.Tensor:
     return torch.empty(n, dtype=torch.uint8, device=q.device)
 
 
-def _params(q, k, v, out, w, scale, eps, gamma_swa, gamma_rla, mode, workspace, flags):
+def _params(q, k, v, out, w, scale, eps, gamma_swa, gamma_rla, mode, workspace, flags, phi=PHI_SOFTMAX):
     p = RattnParams()
+    p.feature_map = phi
     p.q, p.k, p.v, p.out = q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr()
     if q.dim() == 4:
         p.B, p.H_q, p.T, p.d = q.shape
@@ -201,12 +203,12 @@ def rattn_forward_static(q, k, v, w, scale=1.0, out=None, stream=None):
 
 def rattn_forward_ex(q, k, v, w, *, scale=1.0, eps=1e-6, gamma_swa=None, gamma_rla=None,
                      mode=MODE_RATTN, workspace=None, save_residuals=False, state_out=None,
-                     k_ring_out=None, v_ring_out=None, out=None, flags=0, stream=None):
+                     k_ring_out=None, v_ring_out=None, out=None, flags=0, phi=PHI_SOFTMAX, stream=None):
     _dense(q, k, v, out, gamma_swa, gamma_rla, workspace, state_out, k_ring_out, v_ring_out)
     out = torch.empty_like(q) if out is None else out
     if save_residuals:
         flags |= FLAG_SAVE_RESIDUALS
-    p = _params(q, k, v, out, w, scale, eps, gamma_swa, gamma_rla, mode, workspace, flags)
+    p = _params(q, k, v, out, w, scale, eps, gamma_swa, gamma_rla, mode, workspace, flags, phi)
     p.state_out = None if state_out is None else state_out.data_ptr()
     p.k_ring_out = None if k_ring_out is None else k_ring_out.data_ptr()
     p.v_ring_out = None if v_ring_out is None else v_ring_out.data_ptr()
@@ -229,12 +231,12 @@ def rattn_backward(q, k, v, dout, workspace, w, dq=None, dk=None, dv=None, strea
 
 def rattn_backward_ex(q, k, v, dout, w, workspace, *, scale=1.0, eps=1e-6, gamma_swa=None,
                       gamma_rla=None, mode=MODE_RATTN, dq=None, dk=None, dv=None,
-                      dgamma_swa=None, dgamma_rla=None, flags=0, stream=None):
+                      dgamma_swa=None, dgamma_rla=None, flags=0, phi=PHI_SOFTMAX, stream=None):
     _dense(q, k, v, dout, workspace, gamma_swa, gamma_rla, dq, dk, dv, dgamma_swa, dgamma_rla)
     dq = torch.empty_like(q) if dq is None else dq
     dk = torch.empty_like(k) if dk is None else dk
     dv = torch.empty_like(v) if dv is None else dv
-    p = _params(q, k, v, dq, w, scale, eps, gamma_swa, gamma_rla, mode, workspace, flags)
+    p = _params(q, k, v, dq, w, scale, eps, gamma_swa, gamma_rla, mode, workspace, flags, phi)
     p.dout, p.dq, p.dk, p.dv = dout.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr()
     p.dgamma_swa = None if dgamma_swa is None else dgamma_swa.data_ptr()
     p.dgamma_rla = None if dgamma_rla is None else dgamma_rla.data_ptr()
@@ -254,11 +256,11 @@ def rattn_decode_step(q, k, v, k_ring, v_ring, state, pos, out=None, stream=None
 
 
 def rattn_decode_step_ex(q, k, v, k_ring, v_ring, state, pos, *, scale=1.0, eps=1e-6,
-                         gamma_swa=None, gamma_rla=None, out=None, stream=None):
+                         gamma_swa=None, gamma_rla=None, out=None, phi=PHI_SOFTMAX, stream=None):
     _dense(q, k, v, k_ring, v_ring, state, out, gamma_swa, gamma_rla)
     out = torch.empty_like(q) if out is None else out
     p = _params(q, k, v, out, k_ring.shape[2], scale, eps, gamma_swa, gamma_rla, MODE_RATTN,
-                None, 0)
+                None, 0, phi)
     _check(lib().rattn_decode_step_ex(ctypes.byref(p), _ptr(k_ring), _ptr(v_ring), _ptr(state),
                                       pos, _stream(stream)), "rattn_decode_step_ex")
     return out

@@ -55,9 +55,13 @@ __device__ __forceinline__ float warp_sum(float x) {
   return x;
 }
 
-// softmax over D features by one warp: dst[a] = phi(src)[a]
+// phi over D features by one warp: dst[a] = phi(src)[a] (softmax, or an element-wise map)
 template <int D>
-__device__ __forceinline__ void warp_feature_map(float* dst, const float* src, int lane) {
+__device__ __forceinline__ void warp_feature_map(float* dst, const float* src, int lane, int phi) {
+  if (phi != RATTN_PHI_SOFTMAX) {
+    for (int a = lane; a < D; a += 32) dst[a] = phi == RATTN_PHI_RELU ? fmaxf(src[a], 0.f) : src[a];
+    return;
+  }
   float m = -INFINITY;
   for (int a = lane; a < D; a += 32) m = fmaxf(m, src[a]);
   m = warp_max(m);
@@ -76,7 +80,7 @@ struct DecodeArgs {
   const void* q; const void* k; const void* v;
   void* k_ring; void* v_ring; float* state; void* out;
   const float* gamma_swa; const float* gamma_rla;
-  int B, H_q, H_kv, w, pos, group;
+  int B, H_q, H_kv, w, pos, group, phi;
   float scale, eps;
 };
 
@@ -130,8 +134,8 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecodeArgs a) {
   }
   __syncthreads();
   for (int r = warp; r <= g; r += DEC_WARPS) {
-    if (r < g) warp_feature_map<D>(fq_s + r * D, q_s + r * D, lane);
-    else if (evict) warp_feature_map<D>(fk_old, k_old, lane);
+    if (r < g) warp_feature_map<D>(fq_s + r * D, q_s + r * D, lane, a.phi);
+    else if (evict) warp_feature_map<D>(fk_old, k_old, lane, a.phi);
   }
   __syncthreads();
 
@@ -355,7 +359,7 @@ cudaError_t launch_dec(const DecodeArgs& a, cudaStream_t s) {
 template <typename TIO, int D>
 __global__ void __launch_bounds__(256) handoff_state_kernel(const TIO* __restrict__ k,
                                                             const TIO* __restrict__ v,
-                                                            float* __restrict__ state, int T, int w) {
+                                                            float* __restrict__ state, int T, int w, int phi) {
   constexpr int ROWS = 8, TOK = 32;
   __shared__ float fk[TOK][ROWS];
   __shared__ float vs[TOK][D];
@@ -382,9 +386,17 @@ __global__ void __launch_bounds__(256) handoff_state_kernel(const TIO* __restric
       }
       m = warp_max(m);
       float s = 0.f;
+      if (phi == RATTN_PHI_SOFTMAX) {
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) { x[c] = __expf(x[c] - m); s += x[c]; }
-      s = warp_sum(s);
+        for (int c = 0; c < D / 32; ++c) { x[c] = __expf(x[c] - m); s += x[c]; }
+        s = warp_sum(s);
+      } else {
+        s = 1.f;
+        if (phi == RATTN_PHI_RELU) {
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) x[c] = fmaxf(x[c], 0.f);
+        }
+      }
       const float inv = j < n ? 1.f / s : 0.f;
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
@@ -435,7 +447,7 @@ cudaError_t launch_handoff_t(const Args& a, cudaStream_t s, bool state_too) {
     KernelTimer kt("handoff_state", s);
     handoff_state_kernel<TIO, D><<<grid, 256, 0, s>>>(reinterpret_cast<const TIO*>(a.k),
                                                       reinterpret_cast<const TIO*>(a.v),
-                                                      a.state_out, a.T, a.w);
+                                                      a.state_out, a.T, a.w, a.phi);
     count_launches(1);
   }
   if (a.k_ring_out && a.v_ring_out) {
@@ -457,7 +469,7 @@ cudaError_t launch_decode(const Args& p, void* k_ring, void* v_ring, float* stat
   DecodeArgs a;
   a.q = p.q; a.k = p.k; a.v = p.v; a.k_ring = k_ring; a.v_ring = v_ring; a.state = state;
   a.out = p.out; a.gamma_swa = p.gamma_swa; a.gamma_rla = p.gamma_rla;
-  a.B = p.B; a.H_q = p.H_q; a.H_kv = p.H_kv; a.w = p.w; a.pos = pos; a.group = p.group;
+  a.B = p.B; a.H_q = p.H_q; a.H_kv = p.H_kv; a.w = p.w; a.pos = pos; a.group = p.group; a.phi = p.phi;
   a.scale = p.scale; a.eps = p.eps;
   if (p.dtype == RATTN_F32)
     return p.d == 64 ? launch_dec<float, 64>(a, s) : launch_dec<float, 128>(a, s);

@@ -122,7 +122,7 @@ __global__ void __launch_bounds__(NT) bwd_dq_kernel(Args a, const float* __restr
     del_s[tid] = t < T ? delta[row_base + t] : 0.f;
   }
   __syncthreads();
-  if (rla_on) feature_map_tile<D, BQ>(Fq, Qs, tid);
+  if (rla_on) feature_map_tile<D, BQ>(Fq, Qs, tid, a.phi);
 
   float4 dq[2][D / 64], dfq[2][D / 64];
 #pragma unroll
@@ -144,7 +144,7 @@ __global__ void __launch_bounds__(NT) bwd_dq_kernel(Args a, const float* __restr
     load_tile<TIO, D, BK>(Ks, kg, j0, T, tid);
     load_tile<TIO, D, BK>(Vs, vg, j0, T, tid);
     __syncthreads();
-    if (need_rla) feature_map_tile<D, BK>(Fk, Ks, tid);
+    if (need_rla) feature_map_tile<D, BK>(Fk, Ks, tid, a.phi);
     if (need_swa) {
       float s[2][4], dp[2][4];
       tile_scores<D, 2, 4>(s, Qs, Ks, ty, tx);
@@ -180,7 +180,7 @@ __global__ void __launch_bounds__(NT) bwd_dq_kernel(Args a, const float* __restr
       tile_pv<D, 2, BK>(dfq, Ps, Fk, ty, tx);
     }
   }
-  // dq += phi(q) * (dphi_q - <dphi_q, phi(q)>)
+  // dq += gradient through phi: phi(q) * (dphi_q - <dphi_q, phi(q)>) for the softmax map
   TIO* dqg = reinterpret_cast<TIO*>(a.dq) + row_base * D;
 #pragma unroll
   for (int i = 0; i < 2; ++i) {
@@ -200,10 +200,10 @@ __global__ void __launch_bounds__(NT) bwd_dq_kernel(Args a, const float* __restr
       for (int c = 0; c < D / 64; ++c) {
         float4 o = dq[i][c];
         if (rla_on) {
-          o.x += f[c].x * (dfq[i][c].x - dot);
-          o.y += f[c].y * (dfq[i][c].y - dot);
-          o.z += f[c].z * (dfq[i][c].z - dot);
-          o.w += f[c].w * (dfq[i][c].w - dot);
+          o.x += feature_map_grad(a.phi, f[c].x, dfq[i][c].x, dot);
+          o.y += feature_map_grad(a.phi, f[c].y, dfq[i][c].y, dot);
+          o.z += feature_map_grad(a.phi, f[c].z, dfq[i][c].z, dot);
+          o.w += feature_map_grad(a.phi, f[c].w, dfq[i][c].w, dot);
         }
         store4<TIO>(dqg + (size_t)t * D + tx * 4 + 64 * c, o);
       }
@@ -241,7 +241,7 @@ __global__ void __launch_bounds__(NT) bwd_dkv_kernel(Args a, const float* __rest
   load_tile<TIO, D, BK>(Ks, kg, j0, T, tid);
   load_tile<TIO, D, BK>(Vs, vg, j0, T, tid);
   __syncthreads();
-  if (rla_on) feature_map_tile<D, BK>(Fk, Ks, tid);
+  if (rla_on) feature_map_tile<D, BK>(Fk, Ks, tid, a.phi);
 
   float4 dk[4][D / 64], dv[4][D / 64], dfk[4][D / 64];
 #pragma unroll
@@ -273,7 +273,7 @@ __global__ void __launch_bounds__(NT) bwd_dkv_kernel(Args a, const float* __rest
         del_s[tid] = t < T ? delta[row_base + t] : 0.f;
       }
       __syncthreads();
-      if (need_rla) feature_map_tile<D, BQ>(Fq, Qs, tid);
+      if (need_rla) feature_map_tile<D, BQ>(Fq, Qs, tid, a.phi);
       if (need_swa) {
         float s[4][2], dp[4][2];
         tile_scores<D, 4, 2>(s, Ks, Qs, ty, tx);
@@ -350,10 +350,10 @@ __global__ void __launch_bounds__(NT) bwd_dkv_kernel(Args a, const float* __rest
       for (int c = 0; c < D / 64; ++c) {
         float4 o = dk[i][c];
         if (rla_on) {
-          o.x += f[c].x * (dfk[i][c].x - dot);
-          o.y += f[c].y * (dfk[i][c].y - dot);
-          o.z += f[c].z * (dfk[i][c].z - dot);
-          o.w += f[c].w * (dfk[i][c].w - dot);
+          o.x += feature_map_grad(a.phi, f[c].x, dfk[i][c].x, dot);
+          o.y += feature_map_grad(a.phi, f[c].y, dfk[i][c].y, dot);
+          o.z += feature_map_grad(a.phi, f[c].z, dfk[i][c].z, dot);
+          o.w += feature_map_grad(a.phi, f[c].w, dfk[i][c].w, dot);
         }
         store4<TIO>(dkg + (size_t)jj * D + tx * 4 + 64 * c, o);
         store4<TIO>(dvg + (size_t)jj * D + tx * 4 + 64 * c, dv[i][c]);

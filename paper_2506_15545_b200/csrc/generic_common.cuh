@@ -47,14 +47,19 @@ __device__ __forceinline__ void load_tile(float* dst, const TIO* src, int row0, 
   }
 }
 
-// phi = softmax over the D features of each of the ROWS (<= 64) rows of src, written to
-// dst (Section 3.1).  Four threads per row.
+// phi of each of the ROWS (<= 64) rows of src, written to dst (Section 3.1): softmax over the
+// D features, or one of the element-wise maps of the paper's ablation.  Four threads per row.
 template <int D, int ROWS>
-__device__ __forceinline__ void feature_map_tile(float* dst, const float* src, int tid) {
+__device__ __forceinline__ void feature_map_tile(float* dst, const float* src, int tid, int phi) {
   constexpr int LD = D + PAD;
   int r = tid >> 2, part = tid & 3;
   if (r >= ROWS) return;            // whole warps drop out (ROWS is a multiple of 8)
   const float* s = src + r * LD;
+  if (phi != RATTN_PHI_SOFTMAX) {
+    float* o = dst + r * LD;
+    for (int a = part; a < D; a += 4) o[a] = phi == RATTN_PHI_RELU ? fmaxf(s[a], 0.f) : s[a];
+    return;
+  }
   float m = -INFINITY;
   for (int a = part; a < D; a += 4) m = fmaxf(m, s[a]);
   m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
@@ -70,6 +75,14 @@ __device__ __forceinline__ void feature_map_tile(float* dst, const float* src, i
   sum += __shfl_xor_sync(0xffffffffu, sum, 2);
   float inv = 1.f / sum;
   for (int a = part; a < D; a += 4) o[a] *= inv;
+}
+
+// Gradient through the feature map for one element: f = phi(x), df = dL/df, dot = <df, f> over
+// the row (used by the softmax map only).
+__device__ __forceinline__ float feature_map_grad(int phi, float f, float df, float dot) {
+  if (phi == RATTN_PHI_SOFTMAX) return f * (df - dot);
+  if (phi == RATTN_PHI_RELU) return f > 0.f ? df : 0.f;       // relu(x) > 0 exactly where x > 0
+  return df;
 }
 
 __device__ __forceinline__ float group16_max(float x) {

@@ -40,7 +40,7 @@ __global__ void __launch_bounds__(NT) generic_fwd_kernel(Args a) {
 
   load_tile<TIO, D, 64>(Qs, qg, q0, T, tid);
   __syncthreads();
-  if (rla_on) feature_map_tile<D, 64>(Fq, Qs, tid);
+  if (rla_on) feature_map_tile<D, 64>(Fq, Qs, tid, a.phi);
 
   float m_run[4], l_run[4];
   float4 acc_s[4][D / 64], acc_r[4][D / 64];
@@ -67,7 +67,7 @@ __global__ void __launch_bounds__(NT) generic_fwd_kernel(Args a) {
     load_tile<TIO, D, 64>(Ks, kg, j0, T, tid);
     load_tile<TIO, D, 64>(Vs, vg, j0, T, tid);
     __syncthreads();
-    if (need_rla) feature_map_tile<D, 64>(Fk, Ks, tid);
+    if (need_rla) feature_map_tile<D, 64>(Fk, Ks, tid, a.phi);
 
     if (need_swa) {
       float s[4][4];

@@ -115,6 +115,7 @@ static int resolve(const rattn_params* p, Args* a, bool need_T) {
   if (p->d != 64 && p->d != 128) return RATTN_ERR_UNSUPPORTED;
   if (p->dtype != RATTN_BF16 && p->dtype != RATTN_F32) return RATTN_ERR_UNSUPPORTED;
   if (p->mode < RATTN_MODE_RATTN || p->mode > RATTN_MODE_FULL_CAUSAL) return RATTN_ERR_UNSUPPORTED;
+  if (p->feature_map < RATTN_PHI_SOFTMAX || p->feature_map > RATTN_PHI_IDENTITY) return RATTN_ERR_UNSUPPORTED;
   if (!(p->eps > 0.f) || !(p->scale == p->scale)) return RATTN_ERR_BAD_ARG;
   if (!p->q || !p->k || !p->v || !p->out) return RATTN_ERR_NULL_PTR;
   if (misaligned(p->q) || misaligned(p->k) || misaligned(p->v) || misaligned(p->out) ||
@@ -126,6 +127,7 @@ static int resolve(const rattn_params* p, Args* a, bool need_T) {
   a->w = (p->mode == RATTN_MODE_FULL_CAUSAL && need_T) ? p->T : p->w;
   a->group = p->H_q / p->H_kv;
   a->dtype = p->dtype; a->mode = p->mode;
+  a->phi = p->feature_map;
   a->scale = p->scale; a->eps = p->eps;
   a->gamma_swa = p->gamma_swa; a->gamma_rla = p->gamma_rla;
   return RATTN_OK;

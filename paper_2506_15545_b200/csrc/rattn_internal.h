@@ -44,6 +44,7 @@ struct Args {
   int B, H_q, H_kv, T, d, w;   // w already replaced by T for FULL_CAUSAL
   int group;                   // H_q / H_kv
   int dtype, mode;
+  int phi;                     // rattn_feature_map
   float scale, eps;
   const float* gamma_swa;
   const float* gamma_rla;
@@ -100,6 +101,7 @@ struct StateLaunch {
   int store_every, store_phase;
   int row_limit;
   float* final_out;
+  int phi;                  // rattn_feature_map applied to x
   int* status;
   const char* name;         // label of the timing record
 };

@@ -49,6 +49,7 @@ struct BwdArgs {
   int t_pad;
   int* status;
   int T, w, H_q, group, mode, n_chunks;
+  int phi;              // rattn_feature_map
   float scale, scale_log2;
 };
 
@@ -366,7 +367,7 @@ __device__ bool dq_rows(const DqMaps& tm, const BwdArgs& a, unsigned char* smem,
       {
         const int t2 = g * 128 + r;                              // two threads per key row
         unsigned char* kh = smem + DQ_OFF_K + last * TILE_BYTES + (t2 & 1) * HALF_BYTES;
-        feature_map_pair(kh, kh, t2 >> 1);
+        feature_map_pair_any(kh, kh, t2 >> 1, a.phi);
       }
       fence_proxy_async_smem();
       mbar_arrive(&bars->phik_ready);
@@ -397,7 +398,8 @@ __device__ bool dq_rows(const DqMaps& tm, const BwdArgs& a, unsigned char* smem,
     WAIT_OR_RETURN(bars->o_done, co_final & 1);
     tc_fence_after();
     float m = 0.f, inv = 0.f, dot = 0.f;
-    if (it.has_rla) {
+    const bool soft = (a.phi == RATTN_PHI_SOFTMAX);
+    if (it.has_rla && soft) {
       m = -INFINITY;
 #pragma unroll
       for (int c = 0; c < 16; ++c) {
@@ -449,9 +451,16 @@ __device__ bool dq_rows(const DqMaps& tm, const BwdArgs& a, unsigned char* smem,
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const float2 f = __bfloat1622float2(h[e]);
-            const float e0 = ex2(f.x * LOG2E - m) * inv, e1 = ex2(f.y * LOG2E - m) * inv;
-            x[8 * cc + 2 * e] += e0 * (df[8 * cc + 2 * e] - dot);
-            x[8 * cc + 2 * e + 1] += e1 * (df[8 * cc + 2 * e + 1] - dot);
+            if (soft) {
+              const float e0 = ex2(f.x * LOG2E - m) * inv, e1 = ex2(f.y * LOG2E - m) * inv;
+              x[8 * cc + 2 * e] += e0 * (df[8 * cc + 2 * e] - dot);
+              x[8 * cc + 2 * e + 1] += e1 * (df[8 * cc + 2 * e + 1] - dot);
+            } else {
+              // element-wise maps: ReLU passes the gradient where q > 0, the identity everywhere
+              const bool relu = (a.phi == RATTN_PHI_RELU);
+              x[8 * cc + 2 * e] += (relu && !(f.x > 0.f)) ? 0.f : df[8 * cc + 2 * e];
+              x[8 * cc + 2 * e + 1] += (relu && !(f.y > 0.f)) ? 0.f : df[8 * cc + 2 * e + 1];
+            }
           }
         }
       }
@@ -747,7 +756,7 @@ __device__ bool kv_rows(const KvMaps& tm, const BwdArgs& a, unsigned char* smem,
     if (pl.n_R > 0) {
       // phi(K_j) into its own tile: 256 threads, two per row
       const int t2 = gg * 128 + r, row = t2 >> 1, hf = t2 & 1;
-      feature_map_pair(smem + KV_OFF_K + hf * HALF_BYTES, smem + KV_OFF_KPHI + hf * HALF_BYTES, row);
+      feature_map_pair_any(smem + KV_OFF_K + hf * HALF_BYTES, smem + KV_OFF_KPHI + hf * HALF_BYTES, row, a.phi);
       fence_proxy_async_smem();
       mbar_arrive(&bars->kphi_ready);
     }
@@ -764,7 +773,7 @@ __device__ bool kv_rows(const KvMaps& tm, const BwdArgs& a, unsigned char* smem,
     if (is_r) {
       // phi(Q_h) in place: 64 rows, two threads per row
       const int row = r >> 1, ch = r & 1;
-      feature_map_pair(sQh + ch * HT_HALF, sQh + ch * HT_HALF, row);
+      feature_map_pair_any(sQh + ch * HT_HALF, sQh + ch * HT_HALF, row, a.phi);
       fence_proxy_async_smem();
       mbar_arrive(&bars->phiq_ready[g]);
     }
@@ -838,43 +847,55 @@ __device__ bool kv_rows(const KvMaps& tm, const BwdArgs& a, unsigned char* smem,
     mbar_arrive(&bars->p_ready[g]);
 
     if (gg == 0 && is_r && n + 2 >= pl.n_R) {                   // group 0's last residual item of this key tile
-      // end of the residual items: dK := phi(k) (dphi_k - <dphi_k, phi(k)>)
+      // end of the residual items: dK := dphi_k through the feature map's gradient
+      // (softmax map: phi(k) (dphi_k - <dphi_k, phi(k)>))
       WAIT_OR_RETURN(bars->r_acc_done, cnt.cr & 1);
       tc_fence_after();
+      const bool soft = (a.phi == RATTN_PHI_SOFTMAX);
       float dot = 0.f;
+      if (soft) {
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        float df[32];
-        tmem_ld32(tK + 32 * c, df);
-        tmem_wait_ld();
+        for (int c = 0; c < 4; ++c) {
+          float df[32];
+          tmem_ld32(tK + 32 * c, df);
+          tmem_wait_ld();
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          const uint4 u = *reinterpret_cast<const uint4*>(sKphi + swz(r, 4 * c + cc));
-          const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&u);
+          for (int cc = 0; cc < 4; ++cc) {
+            const uint4 u = *reinterpret_cast<const uint4*>(sKphi + swz(r, 4 * c + cc));
+            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float2 f = __bfloat1622float2(h2[e]);
-            dot += f.x * df[8 * cc + 2 * e] + f.y * df[8 * cc + 2 * e + 1];
+            for (int e = 0; e < 4; ++e) {
+              const float2 f = __bfloat1622float2(h2[e]);
+              dot += f.x * df[8 * cc + 2 * e] + f.y * df[8 * cc + 2 * e + 1];
+            }
           }
         }
       }
+      // the identity map leaves dphi_k as it is
+      if (a.phi != RATTN_PHI_IDENTITY) {
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        float df[32];
-        tmem_ld32(tK + 32 * c, df);
-        tmem_wait_ld();
+        for (int c = 0; c < 4; ++c) {
+          float df[32];
+          tmem_ld32(tK + 32 * c, df);
+          tmem_wait_ld();
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          const uint4 u = *reinterpret_cast<const uint4*>(sKphi + swz(r, 4 * c + cc));
-          const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&u);
+          for (int cc = 0; cc < 4; ++cc) {
+            const uint4 u = *reinterpret_cast<const uint4*>(sKphi + swz(r, 4 * c + cc));
+            const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float2 f = __bfloat1622float2(h2[e]);
-            df[8 * cc + 2 * e] = f.x * (df[8 * cc + 2 * e] - dot);
-            df[8 * cc + 2 * e + 1] = f.y * (df[8 * cc + 2 * e + 1] - dot);
+            for (int e = 0; e < 4; ++e) {
+              const float2 f = __bfloat1622float2(h2[e]);
+              if (soft) {
+                df[8 * cc + 2 * e] = f.x * (df[8 * cc + 2 * e] - dot);
+                df[8 * cc + 2 * e + 1] = f.y * (df[8 * cc + 2 * e + 1] - dot);
+              } else {                                   // ReLU: relu(k) > 0 exactly where k > 0
+                df[8 * cc + 2 * e] = f.x > 0.f ? df[8 * cc + 2 * e] : 0.f;
+                df[8 * cc + 2 * e + 1] = f.y > 0.f ? df[8 * cc + 2 * e + 1] : 0.f;
+              }
+            }
           }
+          tmem_st32(tK + 32 * c, df);
         }
-        tmem_st32(tK + 32 * c, df);
       }
       tmem_wait_st();
       tc_fence_before();
@@ -1040,6 +1061,7 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
     L.T = a.T; L.n_kv = (int)nkv; L.group = a.group; L.n_chunks = a.n_chunks;
     L.n_steps = n_r; L.first = n_qt - 1; L.dir = -1; L.out_first = n_qt - wt - 2;
     L.store_every = 1; L.store_phase = 0; L.row_limit = 0; L.final_out = nullptr;
+    L.phi = a.phi;
     L.status = a.status; L.name = "tc_state_bwd";
     e = launch_tc_states(L, s);
   }
@@ -1053,6 +1075,7 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
   t.lse2p = a.lse2p; t.dscp = a.dscp; t.t_pad = t_pad;
   t.T = a.T; t.w = a.w; t.H_q = a.H_q; t.group = a.group; t.mode = a.mode; t.n_chunks = a.n_chunks;
   t.scale = a.scale; t.scale_log2 = a.scale * LOG2E;
+  t.phi = a.phi;
   e = cudaFuncSetAttribute(tc_bwd_dq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DQ_SMEM);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(tc_bwd_dkv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, KV_SMEM);

@@ -147,6 +147,30 @@ __device__ __forceinline__ void feature_map_pair(const unsigned char* src_half, 
   }
 }
 
+// The element-wise maps of the paper's ablation (Table 6) on packed bf16 pairs: ReLU; the
+// identity needs no arithmetic at all.
+__device__ __forceinline__ uint4 relu_bf16x8(uint4 u) {
+  __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&u);
+  const __nv_bfloat162 z = __floats2bfloat162_rn(0.f, 0.f);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) h[e] = __hmax2(h[e], z);
+  return u;
+}
+// feature_map_pair for any map: softmax as above; ReLU / identity element-wise (src may differ from dst)
+__device__ __forceinline__ void feature_map_pair_any(const unsigned char* src_half, unsigned char* dst_half, int row, int phi) {
+  if (phi == RATTN_PHI_SOFTMAX) {
+    feature_map_pair(src_half, dst_half, row);
+    return;
+  }
+  if (phi == RATTN_PHI_IDENTITY && src_half == dst_half) return;
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    const int off = row * 128 + ((c ^ (row & 7)) << 4);
+    const uint4 u = *reinterpret_cast<const uint4*>(src_half + off);
+    *reinterpret_cast<uint4*>(dst_half + off) = phi == RATTN_PHI_RELU ? relu_bf16x8(u) : u;
+  }
+}
+
 // byte offset of 16-byte chunk c (0..15) of row r inside a swizzled [128 x 128] bf16 tile
 __device__ __forceinline__ uint32_t swz(int r, int c) {
   return (uint32_t)((c >> 3) * HALF_BYTES + r * 128 + (((c & 7) ^ (r & 7)) << 4));
@@ -330,6 +354,21 @@ __device__ __forceinline__ float feature_map_row_inplace(unsigned char* tile, in
   return inv;
 }
 
+// phi of row r of a swizzled bf16 tile, in place, for any map.  NORMALISE = false: the softmax
+// map leaves exp(x - max) and returns 1 / sum (see feature_map_row_inplace); the element-wise
+// maps have no normalisation and return 1.
+template <bool NORMALISE>
+__device__ __forceinline__ float feature_map_row_any(unsigned char* tile, int r, int phi) {
+  if (phi == RATTN_PHI_SOFTMAX) return feature_map_row_inplace<NORMALISE>(tile, r);
+  if (phi == RATTN_PHI_RELU) {
+#pragma unroll 4
+    for (int c = 0; c < 16; ++c) {
+      uint4* p = reinterpret_cast<uint4*>(tile + swz(r, c));
+      *p = relu_bf16x8(*p);
+    }
+  }
+  return 1.f;
+}
 
 // ------------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,

@@ -38,6 +38,7 @@ cudaError_t launch_tc_forward(const Args& a, cudaStream_t s) {
     L.store_phase = a.training ? 0 : (wt & 1);
     L.row_limit = want_state ? a.T - a.w : 0;
     L.final_out = want_state ? a.state_out : nullptr;
+    L.phi = a.phi;
     L.status = a.status; L.name = "tc_state_fwd";
     cudaError_t e = launch_tc_states(L, s);
     if (e != cudaSuccess) return e;

@@ -62,6 +62,7 @@ struct FArgs {
   int* status;
   int* work_counter;      // next unit to hand out (device memory, zero at launch); null: static round-robin
   int T, w, H_q, group, mode, n_chunks, n_qt, n_pairs, n_units, n_bh;
+  int phi;                // rattn_feature_map
   int n_stateless;        // pairs whose tiles read no stored state; their units come first
   int wait_for_states;    // a chunk-state kernel runs ahead of this one: wait for it before the first state load
   float scale_log2, eps;
@@ -502,12 +503,12 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     if (rlaX) {
       // phi(Q_X) without its normalisation: everything that follows is linear in this row,
       // so 1/sum is applied to the accumulator row at the end
-      inv_q = feature_map_row_inplace<false>(sQ, r);
+      inv_q = feature_map_row_any<false>(sQ, r, a.phi);
       fence_proxy_async_smem();
       mbar_arrive(&bars->phiq_ready[X]);
       // this tile's own chunk: A -> last stream position, B -> its last active position
       const int ic = (X == 0) ? un.n - 1 : un.i1[1];
-      feature_map_row_inplace<true>(smem + F_OFF_KV + ((kv0 + ic) & 1) * 2 * TILE_BYTES, r);
+      feature_map_row_any<true>(smem + F_OFF_KV + ((kv0 + ic) & 1) * 2 * TILE_BYTES, r, a.phi);
       fence_proxy_async_smem();
       mbar_arrive(&bars->phik_ready[X]);
     }
@@ -796,6 +797,7 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_sta
   t.n_bh = a.B * a.H_q;
   t.n_units = t.n_pairs * t.n_bh;
   t.scale_log2 = a.scale * LOG2E; t.eps = a.eps;
+  t.phi = a.phi;
   // pairs p with 2p - w/128 <= 0 read no stored state
   t.n_stateless = 0;
   if (a.mode == RATTN_MODE_RATTN && after_states) {

@@ -43,6 +43,7 @@ struct StateArgs {
   int store_phase;
   int row_limit;    // tokens at positions >= row_limit contribute nothing (INT_MAX: no limit)
   float* final_out; // optional fp32 [n_kv, 128, 128]: the sum after the last step
+  int phi;          // rattn_feature_map
   int* status;
 };
 
@@ -109,9 +110,10 @@ tc_state_scan_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       unsigned char* xh = smem + st * ST_STAGE + (tid & 1) * HALF_BYTES;
       const int row = tid >> 1;
       const int token = (a.first + a.dir * (it / a.group)) * TILE + row;
-      if (token < a.row_limit) {
-        feature_map_pair(xh, xh, row);
-      } else {
+      // every lane maps its row (the softmax map exchanges partial results between the two lanes
+      // of a row with full-warp shuffles, so no lane may skip it); rows past the limit are then cleared
+      feature_map_pair_any(xh, xh, row, a.phi);
+      if (token >= a.row_limit) {
 #pragma unroll
         for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(xh + row * 128 + (c << 4)) = make_uint4(0, 0, 0, 0);
       }
@@ -227,6 +229,7 @@ cudaError_t launch_tc_states(const StateLaunch& L, cudaStream_t s) {
   a.store_phase = L.store_phase;
   a.row_limit = L.row_limit > 0 ? L.row_limit : INT_MAX;
   a.final_out = L.final_out;
+  a.phi = L.phi;
   cudaError_t e = cudaFuncSetAttribute(tc_state_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ST_SMEM);
   if (e != cudaSuccess) return e;
   {
