@@ -17,6 +17,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(ROOT, "_build")
 LIB = os.path.join(HERE, "librattn.so")
+LIB_DEBUG = os.path.join(HERE, "librattn_dbg.so")      # same sources with -DRATTN_DEBUG_KNOBS (include/rattn_debug.h)
 
 SOURCES = ["rattn_api.cu", "generic_fwd.cu", "generic_bwd.cu", "decode.cu", "tc_fwd.cu",
            "tc_fwd2.cu", "tc_state.cu", "tc_bwd.cu", "static_scratch.cu"]
@@ -33,15 +34,17 @@ def _nvcc() -> str:
 
 
 def _newest_dep_mtime() -> float:
-    m = os.path.getmtime(os.path.join(ROOT, "include", "rattn.h"))
+    m = max(os.path.getmtime(os.path.join(ROOT, "include", f)) for f in ("rattn.h", "rattn_debug.h"))
     for f in os.listdir(CSRC):
         m = max(m, os.path.getmtime(os.path.join(CSRC, f)))
     return max(m, os.path.getmtime(__file__))
 
 
-def _compile(src: str, verbose: bool) -> str:
-    obj = os.path.join(BUILD, src.replace(".cu", ".o"))
+def _compile(src: str, verbose: bool, debug: bool = False) -> str:
+    obj = os.path.join(BUILD, src.replace(".cu", ".dbg.o" if debug else ".o"))
     cmd = [_nvcc(), *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
+    if debug:
+        cmd.insert(1, "-DRATTN_DEBUG_KNOBS")
     if os.path.exists(os.path.join(CSRC, "tc_fwd.cu")):
         cmd.insert(1, "-DRATTN_HAVE_TC")
     if verbose:
@@ -55,20 +58,22 @@ def _compile(src: str, verbose: bool) -> str:
     return obj
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every source and link librattn.so; returns its path."""
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Compile every source and link librattn.so (debug: librattn_dbg.so); returns its path."""
+    lib = LIB_DEBUG if debug else LIB
     sources = [s for s in SOURCES if os.path.exists(os.path.join(CSRC, s))]
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_dep_mtime():
-        return LIB
+    if not force and os.path.exists(lib) and os.path.getmtime(lib) >= _newest_dep_mtime():
+        return lib
     os.makedirs(BUILD, exist_ok=True)
     with concurrent.futures.ThreadPoolExecutor(max_workers=len(sources)) as ex:
-        objs = list(ex.map(lambda s: _compile(s, verbose), sources))
-    cmd = [_nvcc(), "-shared", "-o", LIB, *objs, "-cudart", "static"]
+        objs = list(ex.map(lambda s: _compile(s, verbose, debug), sources))
+    cmd = [_nvcc(), "-shared", "-o", lib, *objs, "-cudart", "static"]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, debug=True))

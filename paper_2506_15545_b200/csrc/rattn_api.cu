@@ -9,11 +9,23 @@
 #include <vector>
 
 #include "rattn_internal.h"
+#ifdef RATTN_DEBUG_KNOBS
+#include "rattn_debug.h"
+#endif
 
 namespace rattn {
 
 static std::atomic<uint64_t> g_launches{0};
 static thread_local int g_last_cuda_error = 0;
+
+static std::atomic<int> g_debug_skip_arrive{0};
+int debug_skip_arrive() {
+#ifdef RATTN_DEBUG_KNOBS
+  return g_debug_skip_arrive.load(std::memory_order_relaxed);
+#else
+  return 0;
+#endif
+}
 
 void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 void set_last_cuda_error(int cuda_error) { g_last_cuda_error = cuda_error; }
@@ -377,6 +389,13 @@ size_t rattn_timing_read(char* buf, size_t buf_bytes) {
   }
   return out.size() + 1;
 }
+
+#ifdef RATTN_DEBUG_KNOBS
+int rattn_debug_withhold_arrival(int on) {
+  g_debug_skip_arrive.store(on ? 1 : 0, std::memory_order_relaxed);
+  return RATTN_OK;
+}
+#endif
 
 int rattn_uses_tensor_path(int d, int w, int dtype, int mode, unsigned flags) {
   return tensor_path(d, w, dtype, mode, flags) ? 1 : 0;

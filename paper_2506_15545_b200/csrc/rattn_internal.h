@@ -108,6 +108,7 @@ struct StateLaunch {
 cudaError_t launch_tc_states(const StateLaunch& L, cudaStream_t s);
 cudaError_t launch_tc_backward(const Args& a, cudaStream_t s);
 
+int debug_skip_arrive();                    // always 0 outside the debug build
 void count_launches(int n);
 void set_last_cuda_error(int cuda_error);   // what rattn_last_cuda_error() reports for this thread
 

@@ -65,6 +65,7 @@ struct FArgs {
   int phi;                // rattn_feature_map
   int n_stateless;        // pairs whose tiles read no stored state; their units come first
   int wait_for_states;    // a chunk-state kernel runs ahead of this one: wait for it before the first state load
+  int debug_skip_arrive;  // debug build only: tile A's row group withholds its first hand-over (a wait then runs out)
   float scale_log2, eps;
 };
 
@@ -490,6 +491,11 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
       l += psum;
       tmem_wait_st();
       tc_fence_before();
+#ifdef RATTN_DEBUG_KNOBS
+      // failure injection for the time-out test: an arrival that nothing else depends on is left
+      // out, so the MMA warp's bounded wait expires and every role takes the abort path
+      if (!(a.debug_skip_arrive && X == 0 && n == 0 && i == i0))
+#endif
       mbar_arrive(&bars->p_ready[X]);
       TL(X, 400 + i);
     }
@@ -805,6 +811,7 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_sta
     if (t.n_stateless > t.n_pairs) t.n_stateless = t.n_pairs;
   }
   t.wait_for_states = after_states ? 1 : 0;
+  t.debug_skip_arrive = debug_skip_arrive();
   t.work_counter = a.status ? a.status + 2 : nullptr;
   int dev = 0, n_sm = 0;
   cudaError_t e = cudaGetDevice(&dev);

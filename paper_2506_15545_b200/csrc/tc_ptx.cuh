@@ -58,9 +58,15 @@ __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, v
 }
 // Bounded wait.  Returns false when the limit is hit (and raises *abort so that every other
 // waiter of the CTA gives up too) or when another thread has already raised it.
+// (The debug build, which exists to make a wait run out in a test, gives up much sooner.)
+#ifdef RATTN_DEBUG_KNOBS
+constexpr int kWaitPolls = 1 << 15;
+#else
+constexpr int kWaitPolls = 1 << 21;
+#endif
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
 #pragma unroll 1
-  for (int it = 0; it < (1 << 21); ++it) {
+  for (int it = 0; it < kWaitPolls; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 63) == 63 && *abort) return false;
   }

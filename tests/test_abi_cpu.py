@@ -34,6 +34,18 @@ def test_every_declared_symbol_is_exported(B):
         assert hasattr(B.lib(), n), n
 
 
+def test_debug_library_exports_its_one_extra_entry_point(B):
+    """include/rattn_debug.h: declared there, exported by librattn_dbg.so only."""
+    from paper_2506_15545_b200 import build
+    dbg = ctypes.CDLL(build.build(debug=True))
+    text = re.sub(r"/\*.*?\*/", "", open(os.path.join(ROOT, "include", "rattn_debug.h")).read(), flags=re.S)
+    names = sorted(set(re.findall(r"\b(rattn_[a-z_]+)\s*\(", text)))
+    assert names == ["rattn_debug_withhold_arrival"]
+    assert hasattr(dbg, names[0]) and not hasattr(B.lib(), names[0])
+    for n in B.EXPORTS:
+        assert hasattr(dbg, n), n
+
+
 def test_header_is_plain_c_and_struct_matches_binding(B, tmp_path):
     src = tmp_path / "sz.c"
     src.write_text('#include "rattn.h"\n#include <stdio.h>\n#include <stddef.h>\n'
