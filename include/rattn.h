@@ -96,6 +96,18 @@ typedef enum rattn_feature_map {
  *              j % w for the last min(w,T) tokens (other slots zero).
  *   dgamma_swa, dgamma_rla   optional fp32 [H_q,d] outputs of rattn_backward_ex.
  *   feature_map   phi of the linear branch (forward, backward and decode must agree).
+ *   state_in, k_ring_in, v_ring_in, pos0   chunked prefill: this call's q, k, v are the tokens
+ *              pos0 .. pos0+T-1 of a longer sequence; the rings and the state are what an
+ *              earlier rattn_forward_ex call on the tokens before them handed out (state_out,
+ *              k_ring_out, v_ring_out -- the same buffers may be passed as both in and out).
+ *              out holds the T rows of this chunk, identical to rows pos0.. of one call on
+ *              the whole sequence.  Needs pos0 >= w (a first chunk of at least w tokens) and a
+ *              workspace (rattn_workspace_bytes_chunked); forward only.
+ *   seq_lens   variable-length batches: entry b has seq_lens[b] valid tokens.  Its valid rows
+ *              are what a call on that entry alone would give (the operator is causal, so
+ *              nothing behind an entry's end reaches them); tiles that lie wholly beyond an
+ *              entry's end are skipped, the other rows of out beyond it hold unspecified
+ *              values, and the hand-off (state_out, rings) is taken at each entry's own length.
  */
 typedef struct rattn_params {
   const void* q;
@@ -123,6 +135,17 @@ typedef struct rattn_params {
   float* dgamma_rla;
   uint32_t flags;                /* RATTN_FLAG_* */
   int32_t feature_map;           /* rattn_feature_map; 0 = the paper's softmax map */
+  /* chunked prefill (forward only): resume a sequence whose first pos0 tokens were processed
+   * by earlier calls.  pos0 = 0 with the three pointers NULL is a fresh sequence. */
+  const float* state_in;         /* [B,H_kv,d,d] fp32: state over the tokens j < pos0 - w */
+  const void* k_ring_in;         /* [B,H_kv,w,d]: tokens pos0-w .. pos0-1 at slot j % w */
+  const void* v_ring_in;
+  int32_t pos0;                  /* tokens that precede this call's T tokens; 0 or >= w */
+  int32_t reserved;
+  const int32_t* seq_lens;       /* optional device [B]: valid tokens of each batch entry, 1 <= len <= T
+                                    (fresh sequences only); NULL: all T */
+  const int32_t* pos;            /* decode only: optional device [B] positions, one per batch entry
+                                    (overrides the pos argument) */
 } rattn_params;
 
 /*
@@ -233,6 +256,11 @@ int rattn_decode_step_ex(const rattn_params* p, void* k_ring, void* v_ring, floa
  */
 size_t rattn_workspace_bytes_ex(int B, int H_q, int H_kv, int T, int d, int w, int dtype,
                                 int mode, unsigned flags);
+
+/* The same for a forward that resumes a sequence (rattn_params.pos0 > 0): in addition the
+ * history + chunk keys and values in time order, 2 x [B,H_kv,w+T,d] elements. */
+size_t rattn_workspace_bytes_chunked(int B, int H_q, int H_kv, int T, int d, int w, int dtype,
+                                     unsigned flags);
 
 /* An upper bound of rattn_workspace_bytes_ex over every mode and every flag combination for
  * these sizes (the training layout of the larger kernel family). */

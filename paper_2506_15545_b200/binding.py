@@ -22,7 +22,7 @@ PHI_SOFTMAX, PHI_RELU, PHI_IDENTITY = 0, 1, 2
 EXPORTS = (
     "rattn_forward", "rattn_forward_ex", "rattn_backward", "rattn_backward_ex",
     "rattn_decode_step", "rattn_decode_step_ex", "rattn_workspace_bytes",
-    "rattn_workspace_bytes_ex",
+    "rattn_workspace_bytes_ex", "rattn_workspace_bytes_chunked",
     "rattn_read_status", "rattn_strerror", "rattn_last_cuda_error", "rattn_launch_count",
     "rattn_uses_tensor_path", "rattn_timing_enable", "rattn_timing_read",
     "rattn_forward_static", "rattn_static_status",
@@ -45,6 +45,9 @@ class RattnParams(ctypes.Structure):
         ("dv", ctypes.c_void_p), ("dgamma_swa", ctypes.c_void_p),
         ("dgamma_rla", ctypes.c_void_p),
         ("flags", ctypes.c_uint32), ("feature_map", ctypes.c_int32),
+        ("state_in", ctypes.c_void_p), ("k_ring_in", ctypes.c_void_p), ("v_ring_in", ctypes.c_void_p),
+        ("pos0", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("seq_lens", ctypes.c_void_p), ("pos", ctypes.c_void_p),
     ]
 
 
@@ -87,6 +90,8 @@ def lib() -> ctypes.CDLL:
     L.rattn_workspace_bytes.restype = ctypes.c_size_t
     L.rattn_workspace_bytes_ex.argtypes = [ci, ci, ci, ci, ci, ci, ci, ci, ctypes.c_uint]
     L.rattn_workspace_bytes_ex.restype = ctypes.c_size_t
+    L.rattn_workspace_bytes_chunked.argtypes = [ci, ci, ci, ci, ci, ci, ci, ctypes.c_uint]
+    L.rattn_workspace_bytes_chunked.restype = ctypes.c_size_t
     L.rattn_read_status.argtypes = [vp, vp]
     L.rattn_read_status.restype = ci
     L.rattn_strerror.argtypes = [ci]
@@ -143,6 +148,17 @@ def rattn_workspace_bytes(B, H_q, H_kv, T, d, w, dtype=RATTN_BF16) -> int:
 
 def rattn_workspace_bytes_ex(B, H_q, H_kv, T, d, w, dtype=RATTN_BF16, mode=MODE_RATTN, flags=0) -> int:
     return int(lib().rattn_workspace_bytes_ex(B, H_q, H_kv, T, d, w, dtype, mode, flags))
+
+
+def rattn_workspace_bytes_chunked(B, H_q, H_kv, T, d, w, dtype=RATTN_BF16, flags=0) -> int:
+    return int(lib().rattn_workspace_bytes_chunked(B, H_q, H_kv, T, d, w, dtype, flags))
+
+
+def alloc_workspace_chunked(q, k, w, flags=0) -> torch.Tensor:
+    """Workspace of a forward that resumes a sequence (pos0 > 0)."""
+    B, H_q, T, d = q.shape
+    n = rattn_workspace_bytes_chunked(B, H_q, k.shape[1], T, d, w, _dtype_code(q), flags)
+    return torch.empty(n, dtype=torch.uint8, device=q.device)
 
 
 def alloc_workspace(q, k, w, mode=None, flags=None) -> torch.Tensor:
@@ -203,8 +219,10 @@ def rattn_forward_static(q, k, v, w, scale=1.0, out=None, stream=None):
 
 def rattn_forward_ex(q, k, v, w, *, scale=1.0, eps=1e-6, gamma_swa=None, gamma_rla=None,
                      mode=MODE_RATTN, workspace=None, save_residuals=False, state_out=None,
-                     k_ring_out=None, v_ring_out=None, out=None, flags=0, phi=PHI_SOFTMAX, stream=None):
-    _dense(q, k, v, out, gamma_swa, gamma_rla, workspace, state_out, k_ring_out, v_ring_out)
+                     k_ring_out=None, v_ring_out=None, out=None, flags=0, phi=PHI_SOFTMAX, state_in=None,
+                     k_ring_in=None, v_ring_in=None, pos0=0, seq_lens=None, stream=None):
+    _dense(q, k, v, out, gamma_swa, gamma_rla, workspace, state_out, k_ring_out, v_ring_out, state_in,
+           k_ring_in, v_ring_in, seq_lens)
     out = torch.empty_like(q) if out is None else out
     if save_residuals:
         flags |= FLAG_SAVE_RESIDUALS
@@ -212,6 +230,11 @@ def rattn_forward_ex(q, k, v, w, *, scale=1.0, eps=1e-6, gamma_swa=None, gamma_r
     p.state_out = None if state_out is None else state_out.data_ptr()
     p.k_ring_out = None if k_ring_out is None else k_ring_out.data_ptr()
     p.v_ring_out = None if v_ring_out is None else v_ring_out.data_ptr()
+    p.state_in = None if state_in is None else state_in.data_ptr()
+    p.k_ring_in = None if k_ring_in is None else k_ring_in.data_ptr()
+    p.v_ring_in = None if v_ring_in is None else v_ring_in.data_ptr()
+    p.pos0 = pos0
+    p.seq_lens = None if seq_lens is None else seq_lens.data_ptr()
     _check(lib().rattn_forward_ex(ctypes.byref(p), _stream(stream)), "rattn_forward_ex")
     return out
 
@@ -256,11 +279,13 @@ def rattn_decode_step(q, k, v, k_ring, v_ring, state, pos, out=None, stream=None
 
 
 def rattn_decode_step_ex(q, k, v, k_ring, v_ring, state, pos, *, scale=1.0, eps=1e-6,
-                         gamma_swa=None, gamma_rla=None, out=None, phi=PHI_SOFTMAX, stream=None):
-    _dense(q, k, v, k_ring, v_ring, state, out, gamma_swa, gamma_rla)
+                         gamma_swa=None, gamma_rla=None, out=None, phi=PHI_SOFTMAX, pos_dev=None, stream=None):
+    """pos_dev: optional int32 device tensor [B], one position per batch entry (then `pos` is ignored)."""
+    _dense(q, k, v, k_ring, v_ring, state, out, gamma_swa, gamma_rla, pos_dev)
     out = torch.empty_like(q) if out is None else out
     p = _params(q, k, v, out, k_ring.shape[2], scale, eps, gamma_swa, gamma_rla, MODE_RATTN,
                 None, 0, phi)
+    p.pos = None if pos_dev is None else pos_dev.data_ptr()
     _check(lib().rattn_decode_step_ex(ctypes.byref(p), _ptr(k_ring), _ptr(v_ring), _ptr(state),
                                       pos, _stream(stream)), "rattn_decode_step_ex")
     return out

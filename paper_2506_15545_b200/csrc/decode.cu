@@ -80,6 +80,7 @@ struct DecodeArgs {
   const void* q; const void* k; const void* v;
   void* k_ring; void* v_ring; float* state; void* out;
   const float* gamma_swa; const float* gamma_rla;
+  const int* pos_dev;                       // optional [B]: one position per batch entry
   int B, H_q, H_kv, w, pos, group, phi;
   float scale, eps;
 };
@@ -110,7 +111,7 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecodeArgs a) {
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = blockIdx.x / a.H_kv, hk = blockIdx.x % a.H_kv;
-  const int w = a.w, pos = a.pos;
+  const int w = a.w, pos = a.pos_dev ? a.pos_dev[b] : a.pos;
   const bool evict = pos - w >= 0;
   const int slot = pos % w;
   const int n_valid = pos < w ? pos : w;
@@ -356,10 +357,14 @@ cudaError_t launch_dec(const DecodeArgs& a, cudaStream_t s) {
 
 // ---------------------------------------------------------------- prefill -> decode hand-off
 // state_out[b,hk] = sum_{j < T-w} phi(k_j)^T v_j  (Eq. 4), one CTA per 8 feature rows.
+// T: key rows per head in memory; len[b] (optional): valid rows of entry b; state_in (optional):
+// the sum over the tokens before row 0.
 template <typename TIO, int D>
 __global__ void __launch_bounds__(256) handoff_state_kernel(const TIO* __restrict__ k,
                                                             const TIO* __restrict__ v,
-                                                            float* __restrict__ state, int T, int w, int phi) {
+                                                            float* __restrict__ state, int T, int w, int phi,
+                                                            const int* __restrict__ len, int H_kv,
+                                                            const float* __restrict__ state_in) {
   constexpr int ROWS = 8, TOK = 32;
   __shared__ float fk[TOK][ROWS];
   __shared__ float vs[TOK][D];
@@ -367,12 +372,13 @@ __global__ void __launch_bounds__(256) handoff_state_kernel(const TIO* __restric
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const TIO* kg = k + (size_t)bh * T * D;
   const TIO* vg = v + (size_t)bh * T * D;
-  const int n = T - w;                       // tokens 0..n-1 have left every window
+  const int n = (len ? min(T, len[bh / H_kv]) : T) - w;   // tokens 0..n-1 have left every window
   // thread -> (row, column group): 8 rows x 32 column lanes, D/32 columns each
   const int row = tid / 32, cl = tid % 32;
   float acc[D / 32];
 #pragma unroll
-  for (int c = 0; c < D / 32; ++c) acc[c] = 0.f;
+  for (int c = 0; c < D / 32; ++c)
+    acc[c] = state_in ? state_in[((size_t)bh * D + r0 + row) * D + cl + 32 * c] : 0.f;
   for (int j0 = 0; j0 < n; j0 += TOK) {
     __syncthreads();
     for (int jj = warp; jj < TOK; jj += 8) {   // warp-level softmax of k_j, keep rows r0..r0+7
@@ -420,13 +426,16 @@ __global__ void __launch_bounds__(256) handoff_state_kernel(const TIO* __restric
 // ring[b,hk, j % w] = x[b,hk, j] for the last min(w,T) tokens; other slots zero.
 template <typename TIO>
 __global__ void handoff_ring_kernel(const TIO* __restrict__ k, const TIO* __restrict__ v,
-                                    TIO* __restrict__ kr, TIO* __restrict__ vr, int T, int w, int D) {
+                                    TIO* __restrict__ kr, TIO* __restrict__ vr, int T, int w, int D,
+                                    const int* __restrict__ len, int H_kv, int pos_shift) {
   const int bh = blockIdx.y;
   const int slot = blockIdx.x;
-  // the newest token that maps to this slot
-  const int last = T - 1;
-  const int j = last - ((last - slot) % w + w) % w;
-  const bool valid = j >= 0 && j >= T - w;
+  // Row j of k, v is the token at sequence position j + pos_shift (a resumed sequence's rows start
+  // before the chunk); the ring keeps position p at slot p % w.  The newest row that maps to this slot:
+  const int Tb = len ? min(T, len[bh / H_kv]) : T;
+  const int last = Tb - 1;
+  const int j = last - ((last + pos_shift - slot) % w + w) % w;
+  const bool valid = j >= 0 && j >= Tb - w;
   for (int c = threadIdx.x; c < D; c += blockDim.x) {
     const size_t dst = ((size_t)bh * w + slot) * D + c;
     if (valid) {
@@ -447,7 +456,7 @@ cudaError_t launch_handoff_t(const Args& a, cudaStream_t s, bool state_too) {
     KernelTimer kt("handoff_state", s);
     handoff_state_kernel<TIO, D><<<grid, 256, 0, s>>>(reinterpret_cast<const TIO*>(a.k),
                                                       reinterpret_cast<const TIO*>(a.v),
-                                                      a.state_out, a.T, a.w, a.phi);
+                                                      a.state_out, a.Tk, a.w, a.phi, a.seq_lens, a.H_kv, a.state_in);
     count_launches(1);
   }
   if (a.k_ring_out && a.v_ring_out) {
@@ -456,17 +465,57 @@ cudaError_t launch_handoff_t(const Args& a, cudaStream_t s, bool state_too) {
     handoff_ring_kernel<TIO><<<grid, 64, 0, s>>>(reinterpret_cast<const TIO*>(a.k),
                                                  reinterpret_cast<const TIO*>(a.v),
                                                  reinterpret_cast<TIO*>(a.k_ring_out),
-                                                 reinterpret_cast<TIO*>(a.v_ring_out), a.T, a.w, D);
+                                                 reinterpret_cast<TIO*>(a.v_ring_out), a.Tk, a.w, D, a.seq_lens,
+                                                 a.H_kv, a.pos_shift);
     count_launches(1);
   }
   return cudaGetLastError();
 }
 
+// k_ext[bh, e] = e < w ? ring[bh, (pos0 - w + e) % w] : chunk[bh, e - w]   (16-byte vectors)
+__global__ void gather_history_kernel(const uint4* __restrict__ k_chunk, const uint4* __restrict__ v_chunk,
+                                      const uint4* __restrict__ k_ring, const uint4* __restrict__ v_ring,
+                                      uint4* __restrict__ k_ext, uint4* __restrict__ v_ext, int T, int w, int pos0,
+                                      int vec_per_row) {
+  const int bh = blockIdx.y;
+  const size_t n_ext = (size_t)(w + T) * vec_per_row;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_ext; i += (size_t)gridDim.x * blockDim.x) {
+    const int e = (int)(i / vec_per_row), c = (int)(i % vec_per_row);
+    uint4 kk, vv;
+    if (e < w) {
+      const int slot = (pos0 - w + e) % w;
+      kk = k_ring[((size_t)bh * w + slot) * vec_per_row + c];
+      vv = v_ring[((size_t)bh * w + slot) * vec_per_row + c];
+    } else {
+      kk = k_chunk[((size_t)bh * T + (e - w)) * vec_per_row + c];
+      vv = v_chunk[((size_t)bh * T + (e - w)) * vec_per_row + c];
+    }
+    k_ext[(size_t)bh * n_ext + i] = kk;
+    v_ext[(size_t)bh * n_ext + i] = vv;
+  }
+}
+
 }  // namespace
 
-cudaError_t launch_decode(const Args& p, void* k_ring, void* v_ring, float* state, int pos,
+cudaError_t launch_gather_history(const Args& a, const void* k_chunk, const void* v_chunk, const void* k_ring,
+                                  const void* v_ring, void* k_ext, void* v_ext, int pos0, cudaStream_t s) {
+  const int elem = a.dtype == RATTN_F32 ? 4 : 2;
+  const int vec_per_row = a.d * elem / 16;
+  const size_t n_ext = (size_t)(a.w + a.T) * vec_per_row;
+  dim3 grid((unsigned)((n_ext + 255) / 256 < 1024 ? (n_ext + 255) / 256 : 1024), a.B * a.H_kv);
+  KernelTimer kt("gather_history", s);
+  gather_history_kernel<<<grid, 256, 0, s>>>(
+      reinterpret_cast<const uint4*>(k_chunk), reinterpret_cast<const uint4*>(v_chunk),
+      reinterpret_cast<const uint4*>(k_ring), reinterpret_cast<const uint4*>(v_ring),
+      reinterpret_cast<uint4*>(k_ext), reinterpret_cast<uint4*>(v_ext), a.T, a.w, pos0, vec_per_row);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decode(const Args& p, void* k_ring, void* v_ring, float* state, int pos, const int* pos_dev,
                           cudaStream_t s) {
   DecodeArgs a;
+  a.pos_dev = pos_dev;
   a.q = p.q; a.k = p.k; a.v = p.v; a.k_ring = k_ring; a.v_ring = v_ring; a.state = state;
   a.out = p.out; a.gamma_swa = p.gamma_swa; a.gamma_rla = p.gamma_rla;
   a.B = p.B; a.H_q = p.H_q; a.H_kv = p.H_kv; a.w = p.w; a.pos = pos; a.group = p.group; a.phi = p.phi;

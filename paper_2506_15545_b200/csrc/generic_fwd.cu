@@ -31,12 +31,16 @@ __global__ void __launch_bounds__(NT) generic_fwd_kernel(Args a) {
   const int bh = blockIdx.y;
   const int b = bh / a.H_q, h = bh % a.H_q, hk = h / a.group;
   const int q0 = qt * BM;
-  const int T = a.T, w = a.w;
+  // T: this entry's valid query rows (variable-length batches); Tk, off: key rows and the key
+  // position of query row 0 (a resumed sequence carries its history in front of the chunk)
+  const int T = a.seq_lens ? min(a.T, a.seq_lens[b]) : a.T, w = a.w;
+  const int off = a.q_off, Tk = a.seq_lens ? T : a.Tk;
   const bool rla_on = (a.mode == RATTN_MODE_RATTN);
+  if (q0 >= T) return;
 
-  const TIO* qg = reinterpret_cast<const TIO*>(a.q) + ((size_t)b * a.H_q + h) * T * D;
-  const TIO* kg = reinterpret_cast<const TIO*>(a.k) + ((size_t)b * a.H_kv + hk) * T * D;
-  const TIO* vg = reinterpret_cast<const TIO*>(a.v) + ((size_t)b * a.H_kv + hk) * T * D;
+  const TIO* qg = reinterpret_cast<const TIO*>(a.q) + ((size_t)b * a.H_q + h) * a.T * D;
+  const TIO* kg = reinterpret_cast<const TIO*>(a.k) + ((size_t)b * a.H_kv + hk) * a.Tk * D;
+  const TIO* vg = reinterpret_cast<const TIO*>(a.v) + ((size_t)b * a.H_kv + hk) * a.Tk * D;
 
   load_tile<TIO, D, 64>(Qs, qg, q0, T, tid);
   __syncthreads();
@@ -56,16 +60,16 @@ __global__ void __launch_bounds__(NT) generic_fwd_kernel(Args a) {
   }
 
   const int q_last = min(q0 + BM, T) - 1;
-  const int n_kt = q_last / BN + 1;
+  const int n_kt = (q_last + off) / BN + 1;
   for (int kt = 0; kt < n_kt; ++kt) {
     const int j0 = kt * BN;
     // some row t in [q0, q_last] has this tile's keys inside its window / residual set
-    const bool need_swa = (j0 + BN - 1 >= q0 - w);
-    const bool need_rla = rla_on && (j0 < q_last - w);
+    const bool need_swa = (j0 + BN - 1 >= q0 + off - w);
+    const bool need_rla = rla_on && (j0 < q_last + off - w);
     if (!need_swa && !need_rla) continue;
     __syncthreads();                              // previous tile fully consumed
-    load_tile<TIO, D, 64>(Ks, kg, j0, T, tid);
-    load_tile<TIO, D, 64>(Vs, vg, j0, T, tid);
+    load_tile<TIO, D, 64>(Ks, kg, j0, Tk, tid);
+    load_tile<TIO, D, 64>(Vs, vg, j0, Tk, tid);
     __syncthreads();
     if (need_rla) feature_map_tile<D, 64>(Fk, Ks, tid, a.phi);
 
@@ -74,12 +78,12 @@ __global__ void __launch_bounds__(NT) generic_fwd_kernel(Args a) {
       tile_scores<D, 4, 4>(s, Qs, Ks, ty, tx);
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const int t = q0 + ty + 16 * i;
+        const int t = q0 + ty + 16 * i, tk = t + off;
         float mx = -INFINITY;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int jj = j0 + tx + 16 * j;
-          const bool ok = (jj <= t) && (jj >= t - w) && (t < T);
+          const bool ok = (jj <= tk) && (jj >= tk - w) && (t < T);
           s[i][j] = ok ? s[i][j] * a.scale : -INFINITY;
           mx = fmaxf(mx, s[i][j]);
         }
@@ -114,7 +118,7 @@ __global__ void __launch_bounds__(NT) generic_fwd_kernel(Args a) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const int jj = j0 + tx + 16 * j;
-          Ps[(ty + 16 * i) * LP + tx + 16 * j] = (jj < t - w && t < T) ? s[i][j] : 0.f;
+          Ps[(ty + 16 * i) * LP + tx + 16 * j] = (jj < t + off - w && t < T) ? s[i][j] : 0.f;
         }
       }
       __syncthreads();
@@ -122,9 +126,28 @@ __global__ void __launch_bounds__(NT) generic_fwd_kernel(Args a) {
     }
   }
 
+  // A resumed sequence: the tokens before the history reach every row through the incoming state,
+  // o_rla += phi(q) S_in (Eq. 4), 64 feature rows of S_in at a time.
+  if (rla_on && a.state_in) {
+    const float* Sg = a.state_in + ((size_t)b * a.H_kv + hk) * D * D;
+    for (int f0 = 0; f0 < D; f0 += 64) {
+      __syncthreads();
+      for (int i = tid; i < 64 * (D / 4); i += NT) {
+        const int r = i / (D / 4), c = (i % (D / 4)) * 4;
+        *reinterpret_cast<float4*>(Vs + r * LD + c) = *reinterpret_cast<const float4*>(Sg + (size_t)(f0 + r) * D + c);
+      }
+      for (int i = tid; i < 64 * 64; i += NT) {
+        const int r = i >> 6, c = i & 63;
+        Ps[r * LP + c] = Fq[r * LD + f0 + c];
+      }
+      __syncthreads();
+      tile_pv<D, 4, 64>(acc_r, Ps, Vs, ty, tx);
+    }
+  }
+
   // Section 3.2: two separate RMS norms, then the sum.
-  TIO* og = reinterpret_cast<TIO*>(a.out) + ((size_t)b * a.H_q + h) * T * D;
-  const size_t row_base = ((size_t)b * a.H_q + h) * T;
+  TIO* og = reinterpret_cast<TIO*>(a.out) + ((size_t)b * a.H_q + h) * a.T * D;
+  const size_t row_base = ((size_t)b * a.H_q + h) * a.T;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int t = q0 + ty + 16 * i;

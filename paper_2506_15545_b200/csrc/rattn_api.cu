@@ -80,7 +80,7 @@ static bool tensor_path(int d, int w, int dtype, int mode, unsigned flags) {
 // residuals the backward reads and the backward's own scratch, in the element type the chosen
 // kernels keep them in (bf16 on the tensor-core path, fp32 on the portable one).
 WorkspaceLayout workspace_layout(int B, int H_q, int H_kv, int T, int d, int w, int dtype, int mode,
-                                 unsigned flags) {
+                                 unsigned flags, int history) {
   WorkspaceLayout L;
   const bool tc = tensor_path(d, mode == RATTN_MODE_FULL_CAUSAL ? T : w, dtype, mode, flags);
   const bool train = (flags & RATTN_FLAG_SAVE_RESIDUALS) != 0;
@@ -94,7 +94,8 @@ WorkspaceLayout workspace_layout(int B, int H_q, int H_kv, int T, int d, int w, 
     off += align256(bytes);
     return at;
   };
-  L.n_chunks = (T + 127) / 128;
+  const int Tk = history ? w + T : T;           // key rows per head: the history precedes the chunk
+  L.n_chunks = (Tk + 127) / 128;
   const size_t states = (size_t)B * H_kv * L.n_chunks * d * d;
   const size_t rows_pad = (size_t)B * H_q * L.n_chunks * 128;
   L.status = take(true, 256);
@@ -108,6 +109,9 @@ WorkspaceLayout workspace_layout(int B, int H_q, int H_kv, int T, int d, int w, 
   L.rstate = take(tc && rla && train, states * sizeof(__nv_bfloat16));
   L.lse2p = take(tc && train, rows_pad * sizeof(float));
   L.dscp = take(tc && train, rows_pad * sizeof(float));
+  const size_t io_elem = dtype == RATTN_F32 ? sizeof(float) : sizeof(__nv_bfloat16);
+  L.k_ext = take(history != 0, (size_t)B * H_kv * Tk * d * io_elem);
+  L.v_ext = take(history != 0, (size_t)B * H_kv * Tk * d * io_elem);
   L.total = off;
   return L;
 }
@@ -136,6 +140,7 @@ static int resolve(const rattn_params* p, Args* a, bool need_T) {
   std::memset(a, 0, sizeof(*a));
   a->q = p->q; a->k = p->k; a->v = p->v; a->out = p->out;
   a->B = p->B; a->H_q = p->H_q; a->H_kv = p->H_kv; a->T = p->T; a->d = p->d;
+  a->Tk = p->T;
   a->w = (p->mode == RATTN_MODE_FULL_CAUSAL && need_T) ? p->T : p->w;
   a->group = p->H_q / p->H_kv;
   a->dtype = p->dtype; a->mode = p->mode;
@@ -145,10 +150,12 @@ static int resolve(const rattn_params* p, Args* a, bool need_T) {
   return RATTN_OK;
 }
 
-static int bind_workspace(const rattn_params* p, Args* a, bool required, unsigned flags) {
+static int bind_workspace(const rattn_params* p, Args* a, bool required, unsigned flags, int history = 0,
+                          WorkspaceLayout* layout = nullptr) {
   if (!p->workspace) return required ? RATTN_ERR_WORKSPACE : RATTN_OK;
   if (((uintptr_t)p->workspace & 255u) != 0) return RATTN_ERR_MISALIGNED;
-  const WorkspaceLayout L = workspace_layout(p->B, p->H_q, p->H_kv, p->T, p->d, p->w, p->dtype, p->mode, flags);
+  const WorkspaceLayout L = workspace_layout(p->B, p->H_q, p->H_kv, p->T, p->d, p->w, p->dtype, p->mode, flags, history);
+  if (layout) *layout = L;
   if (p->workspace_bytes < L.total) return RATTN_ERR_WORKSPACE;
   char* base = reinterpret_cast<char*>(p->workspace);
   auto at = [&](size_t off) -> char* { return off == kAbsent ? nullptr : base + off; };
@@ -182,15 +189,37 @@ static int forward_impl(const rattn_params* p, cudaStream_t s) {
   // the tensor-core kernels take the row maximum before multiplying by the scale
   if (tc && !(p->scale > 0.f)) return RATTN_ERR_UNSUPPORTED;
   const bool train = (p->flags & RATTN_FLAG_SAVE_RESIDUALS) != 0;
-  // a workspace is needed for the residuals and for the chunk states of the tensor-core path
-  rc = bind_workspace(p, &a, train || (tc && p->mode == RATTN_MODE_RATTN), p->flags);
+  // chunked prefill: the chunk continues a sequence whose last w tokens and state come with it
+  const bool resume = p->pos0 != 0 || p->state_in || p->k_ring_in || p->v_ring_in;
+  if (resume) {
+    if (p->pos0 < p->w) return RATTN_ERR_BAD_ARG;
+    if (!p->state_in || !p->k_ring_in || !p->v_ring_in) return RATTN_ERR_NULL_PTR;
+    if (misaligned(p->state_in) || misaligned(p->k_ring_in) || misaligned(p->v_ring_in)) return RATTN_ERR_MISALIGNED;
+    if (p->mode != RATTN_MODE_RATTN || train || p->seq_lens) return RATTN_ERR_UNSUPPORTED;
+  }
+  if (p->seq_lens && (((uintptr_t)p->seq_lens & 3u) != 0)) return RATTN_ERR_MISALIGNED;
+  if (p->seq_lens && train) return RATTN_ERR_UNSUPPORTED;
+  // a workspace is needed for the residuals, for the chunk states of the tensor-core path and for
+  // the history + chunk keys and values of a resumed sequence
+  WorkspaceLayout L;
+  rc = bind_workspace(p, &a, train || resume || (tc && p->mode == RATTN_MODE_RATTN), p->flags, resume ? 1 : 0, &L);
   if (rc != RATTN_OK) return rc;
+  a.seq_lens = p->seq_lens;
   a.state_out = p->state_out; a.k_ring_out = p->k_ring_out; a.v_ring_out = p->v_ring_out;
   a.training = train;
   cudaError_t e;
   if (a.status) {
     e = cudaMemsetAsync(a.status, 0, 256, s);
     if (e != cudaSuccess) return fail_cuda(e);
+  }
+  if (resume) {
+    char* base = reinterpret_cast<char*>(p->workspace);
+    void* k_ext = base + L.k_ext;
+    void* v_ext = base + L.v_ext;
+    e = launch_gather_history(a, p->k, p->v, p->k_ring_in, p->v_ring_in, k_ext, v_ext, p->pos0, s);
+    if (e != cudaSuccess) return fail_cuda(e);
+    a.k = k_ext; a.v = v_ext;
+    a.Tk = p->w + p->T; a.q_off = p->w; a.state_in = p->state_in; a.pos_shift = p->pos0 - p->w;
   }
 #ifdef RATTN_HAVE_TC
   if (tc) e = launch_tc_forward(a, s);
@@ -210,6 +239,7 @@ static int backward_impl(const rattn_params* p, cudaStream_t s) {
   int rc = resolve(p, &a, true);
   if (rc != RATTN_OK) return rc;
   if (!p->dout || !p->dq || !p->dk || !p->dv) return RATTN_ERR_NULL_PTR;
+  if (p->pos0 != 0 || p->state_in || p->seq_lens) return RATTN_ERR_UNSUPPORTED;   // training runs on whole, fresh sequences
   if (misaligned(p->dout) || misaligned(p->dq) || misaligned(p->dk) || misaligned(p->dv) ||
       misaligned(p->dgamma_swa) || misaligned(p->dgamma_rla))
     return RATTN_ERR_MISALIGNED;
@@ -294,8 +324,9 @@ int rattn_decode_step_ex(const rattn_params* p, void* k_ring, void* v_ring, floa
   if (pos < 0) return RATTN_ERR_BAD_ARG;
   if (p->mode != RATTN_MODE_RATTN) return RATTN_ERR_UNSUPPORTED;
   if (a.group > 64) return RATTN_ERR_UNSUPPORTED;
+  if (p->pos && (((uintptr_t)p->pos & 3u) != 0)) return RATTN_ERR_MISALIGNED;
   a.w = p->w;
-  cudaError_t e = launch_decode(a, k_ring, v_ring, state, pos, reinterpret_cast<cudaStream_t>(stream));
+  cudaError_t e = launch_decode(a, k_ring, v_ring, state, pos, p->pos, reinterpret_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return fail_cuda(e);
   return RATTN_OK;
 }
@@ -318,6 +349,13 @@ size_t rattn_workspace_bytes_ex(int B, int H_q, int H_kv, int T, int d, int w, i
   if (dtype != RATTN_BF16 && dtype != RATTN_F32) return 0;
   if (mode < RATTN_MODE_RATTN || mode > RATTN_MODE_FULL_CAUSAL) return 0;
   return workspace_layout(B, H_q, H_kv, T, d, w, dtype, mode, flags).total;
+}
+
+size_t rattn_workspace_bytes_chunked(int B, int H_q, int H_kv, int T, int d, int w, int dtype, unsigned flags) {
+  if (B < 1 || H_q < 1 || H_kv < 1 || T < 1 || w < 1 || (d != 64 && d != 128)) return 0;
+  if (H_q % H_kv != 0) return 0;
+  if (dtype != RATTN_BF16 && dtype != RATTN_F32) return 0;
+  return workspace_layout(B, H_q, H_kv, T, d, w, dtype, RATTN_MODE_RATTN, flags & ~RATTN_FLAG_SAVE_RESIDUALS, 1).total;
 }
 
 size_t rattn_workspace_bytes(int B, int H_q, int H_kv, int T, int d, int w, int dtype) {

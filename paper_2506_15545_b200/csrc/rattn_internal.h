@@ -25,6 +25,8 @@ struct WorkspaceLayout {
   size_t rstate;        // bf16 [B,H_kv,n_chunks,d,d]  backward: suffix sums of phi(Q)^T g_r
   size_t lse2p;         // fp32 [B*H_q, n_chunks*128]  backward: lse * log2(e), +inf in the padding
   size_t dscp;          // fp32 [B*H_q, n_chunks*128]  backward: D_t * scale, 0 in the padding
+  size_t k_ext;         // I/O type [B,H_kv,w+T,d]  chunked prefill: history + chunk keys, in time order
+  size_t v_ext;         //                          ... values
   size_t total;
   int n_chunks;         // ceil(T / 128)
 };
@@ -32,8 +34,9 @@ struct WorkspaceLayout {
 // Offset of a region the call does not use.
 constexpr size_t kAbsent = ~(size_t)0;
 
+// T: query rows of the call; history: 1 when the call resumes a sequence (chunked prefill)
 WorkspaceLayout workspace_layout(int B, int H_q, int H_kv, int T, int d, int w, int dtype, int mode,
-                                 unsigned flags);
+                                 unsigned flags, int history = 0);
 
 // Resolved arguments handed to the kernel launchers (all device pointers).
 struct Args {
@@ -42,6 +45,14 @@ struct Args {
   const void* v;
   void* out;
   int B, H_q, H_kv, T, d, w;   // w already replaced by T for FULL_CAUSAL
+  // Chunked prefill: k, v then point at the history (the w tokens before the chunk, in time
+  // order) followed by the chunk, Tk = w + T rows per head, and query row t sits at key
+  // position t + q_off (q_off = w); state_in holds the sum over the tokens before the history.
+  // A fresh sequence has Tk = T, q_off = 0, state_in = null.
+  int Tk, q_off;
+  const float* state_in;
+  const int* seq_lens;         // optional device [B]: valid tokens of each batch entry (fresh sequences only)
+  int pos_shift;               // sequence position of key row 0 (pos0 - w for a resumed sequence, else 0)
   int group;                   // H_q / H_kv
   int dtype, mode;
   int phi;                     // rattn_feature_map
@@ -80,7 +91,7 @@ struct Args {
 // Launchers; each returns the cudaError_t of its launches (cudaGetLastError).
 cudaError_t launch_generic_forward(const Args& a, cudaStream_t s);
 cudaError_t launch_generic_backward(const Args& a, cudaStream_t s);
-cudaError_t launch_decode(const Args& a, void* k_ring, void* v_ring, float* state, int pos,
+cudaError_t launch_decode(const Args& a, void* k_ring, void* v_ring, float* state, int pos, const int* pos_dev,
                           cudaStream_t s);
 // prefill -> decode hand-off: the rings, and (state_too) the state by the portable kernel
 cudaError_t launch_handoff(const Args& a, cudaStream_t s, bool state_too);
@@ -89,9 +100,10 @@ cudaError_t launch_tc_forward(const Args& a, cudaStream_t s);        // chunk st
 cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_states);
 // Running sums of phi(X_c)^T Y_c over the chunks first, first+dir, ... (n_steps of them) for every
 // K/V head (tc_state.cu).  The sum after step s goes, as bf16, to matrix out_first + dir*s of the
-// head when that index is congruent to store_phase modulo store_every; the sum after the last
-// step also goes to final_out (fp32 [n_kv,128,128]) when that is given.  Tokens at positions
-// >= row_limit (0: no limit) contribute nothing.
+// head when that index is congruent to store_phase modulo store_every.  With `handoff` the chain
+// is the forward's and also yields the decode state: per head it walks ceil((len - w) / 128) chunks
+// (len = T, or the batch entry's own length), tokens at positions >= len - w contribute nothing,
+// and the final sum goes to final_out in fp32.
 struct StateLaunch {
   const void* x;            // [n_kv * group, T, 128] bf16, mapped through phi
   const void* y;            // [n_kv * group, T, 128] bf16
@@ -99,14 +111,21 @@ struct StateLaunch {
   int T, n_kv, group, n_chunks;
   int n_steps, first, dir, out_first;
   int store_every, store_phase;
-  int row_limit;
+  int handoff;              // 1: the chain ends with the decode state (tokens before len - w, len = T or the
+  int w;                    //    entry's own length), left in final_out; the step count follows the length
   float* final_out;
+  const float* state_in;    // optional fp32 [n_kv,128,128]: the sum starts from it and matrix 0 holds it
+  const int* seq_lens;      // optional [n_kv / kv_per_batch]: valid rows of each batch entry
+  int kv_per_batch;
   int phi;                  // rattn_feature_map applied to x
   int* status;
   const char* name;         // label of the timing record
 };
 cudaError_t launch_tc_states(const StateLaunch& L, cudaStream_t s);
 cudaError_t launch_tc_backward(const Args& a, cudaStream_t s);
+// chunked prefill: k_ext/v_ext[b,hk] = the ring's tokens pos0-w .. pos0-1 in time order, then the chunk
+cudaError_t launch_gather_history(const Args& a, const void* k_chunk, const void* v_chunk, const void* k_ring,
+                                  const void* v_ring, void* k_ext, void* v_ext, int pos0, cudaStream_t s);
 
 int debug_skip_arrive();                    // always 0 outside the debug build
 void count_launches(int n);

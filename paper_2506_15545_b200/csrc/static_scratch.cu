@@ -68,7 +68,7 @@ extern "C" int rattn_forward_static(const void* q, const void* k, const void* v,
   Args a;
   std::memset(&a, 0, sizeof(a));
   a.q = q; a.k = k; a.v = v; a.out = out;
-  a.B = B; a.H_q = H_q; a.H_kv = H_kv; a.T = T; a.d = d; a.w = w;
+  a.B = B; a.H_q = H_q; a.H_kv = H_kv; a.T = T; a.Tk = T; a.d = d; a.w = w;
   a.group = H_q / H_kv;
   a.dtype = RATTN_BF16; a.mode = RATTN_MODE_RATTN;
   a.scale = scale; a.eps = 1e-6f;

@@ -1060,7 +1060,8 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
     L.x = a.q; L.y = g_r; L.out = a.rstate;
     L.T = a.T; L.n_kv = (int)nkv; L.group = a.group; L.n_chunks = a.n_chunks;
     L.n_steps = n_r; L.first = n_qt - 1; L.dir = -1; L.out_first = n_qt - wt - 2;
-    L.store_every = 1; L.store_phase = 0; L.row_limit = 0; L.final_out = nullptr;
+    L.store_every = 1; L.store_phase = 0; L.handoff = 0; L.w = a.w; L.final_out = nullptr;
+    L.state_in = nullptr; L.seq_lens = nullptr; L.kv_per_batch = 1;
     L.phi = a.phi;
     L.status = a.status; L.name = "tc_state_bwd";
     e = launch_tc_states(L, s);

@@ -15,29 +15,35 @@
 namespace rattn {
 
 cudaError_t launch_tc_forward(const Args& a, cudaStream_t s) {
-  const int n_qt = (a.T + tc::TILE - 1) / tc::TILE;
-  const int wt = a.w / tc::TILE;
+  // key-space tiles: a resumed sequence carries its w-token history in front of the chunk
+  const int n_kt = (a.Tk + tc::TILE - 1) / tc::TILE;
+  const int wt = a.w / tc::TILE, off = a.q_off / tc::TILE;
   const bool rla = (a.mode == RATTN_MODE_RATTN);
-  // S_[c] for c = 1 .. n_delta: the states some query tile reads (S_[0] = 0 is never read)
-  const int n_delta = rla ? n_qt - 1 - wt : 0;
+  // S_[c] for c = 1 .. n_delta: the states some query tile reads (S_[0] is the incoming state, zero
+  // for a fresh sequence, where it is never read)
+  const int n_delta = rla ? n_kt - 1 - wt : 0;
   const int n_kv = a.B * a.H_kv;
   const bool want_state = rla && a.state_out != nullptr;
   bool chained = false;
-  if (want_state && a.T <= a.w) {
+  if (want_state && a.Tk <= a.w && !a.seq_lens) {
     // nothing has left the window yet
     cudaError_t e = cudaMemsetAsync(a.state_out, 0, sizeof(float) * (size_t)n_kv * 128 * 128, s);
     if (e != cudaSuccess) return e;
   }
-  const int n_steps = (want_state && a.T > a.w) ? n_delta + 1 : n_delta;
-  if (n_steps > 0) {
+  const int n_steps = (want_state && (a.Tk > a.w || a.seq_lens)) ? n_delta + 1 : n_delta;
+  if (n_steps > 0 || (a.state_in && rla) || (a.seq_lens && want_state)) {
     StateLaunch L;
     L.x = a.k; L.y = a.v; L.out = a.chunk_state;
-    L.T = a.T; L.n_kv = n_kv; L.group = 1; L.n_chunks = a.n_chunks;
-    L.n_steps = n_steps; L.first = 0; L.dir = +1; L.out_first = 1;
+    L.T = a.Tk; L.n_kv = n_kv; L.group = 1; L.n_chunks = a.n_chunks;
+    L.n_steps = n_steps > 0 ? n_steps : 0; L.first = 0; L.dir = +1; L.out_first = 1;
+    // the main kernel reads S_[c] for c = off + 2p - wt only
     L.store_every = a.training ? 1 : 2;
-    L.store_phase = a.training ? 0 : (wt & 1);
-    L.row_limit = want_state ? a.T - a.w : 0;
+    L.store_phase = a.training ? 0 : ((off + wt) & 1);
+    L.handoff = want_state ? 1 : 0;
+    L.w = a.w;
     L.final_out = want_state ? a.state_out : nullptr;
+    L.state_in = a.state_in;
+    L.seq_lens = a.seq_lens; L.kv_per_batch = a.H_kv;
     L.phi = a.phi;
     L.status = a.status; L.name = "tc_state_fwd";
     cudaError_t e = launch_tc_states(L, s);

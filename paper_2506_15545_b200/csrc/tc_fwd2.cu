@@ -63,6 +63,9 @@ struct FArgs {
   int* work_counter;      // next unit to hand out (device memory, zero at launch); null: static round-robin
   int T, w, H_q, group, mode, n_chunks, n_qt, n_pairs, n_units, n_bh;
   int phi;                // rattn_feature_map
+  int off;                // key tile of query tile 0 (a resumed sequence carries w/128 history tiles in front)
+  int first_state;        // smallest chunk index whose state is stored: 1 (S_[0] = 0), or 0 with an incoming state
+  const int* seq_lens;    // optional [B]: valid query rows per batch entry
   int n_stateless;        // pairs whose tiles read no stored state; their units come first
   int wait_for_states;    // a chunk-state kernel runs ahead of this one: wait for it before the first state load
   int debug_skip_arrive;  // debug build only: tile A's row group withholds its first hand-over (a wait then runs out)
@@ -98,8 +101,10 @@ __device__ __forceinline__ Unit make_unit(const FArgs& a, int u) {
   un.bh_kv = b * (a.H_q / a.group) + un.h / a.group;
   un.wt = a.w / TILE;
   un.windowed = (a.mode != RATTN_MODE_FULL_CAUSAL);
-  un.t[0] = 2 * p;
-  un.t[1] = (2 * p + 1 < a.n_qt) ? 2 * p + 1 : -1;
+  // tile indices are key-space positions: query tile i of the call sits at key tile i + off
+  const int n_qt = a.seq_lens ? (min(a.T, a.seq_lens[b]) + TILE - 1) / TILE : a.n_qt;
+  un.t[0] = (2 * p < n_qt) ? a.off + 2 * p : -1;             // a unit without tile A is empty
+  un.t[1] = (2 * p + 1 < n_qt) ? a.off + 2 * p + 1 : -1;
   un.kt_hi = un.t[1] >= 0 ? un.t[1] : un.t[0];
   const int loA = un.windowed ? max(0, un.t[0] - un.wt) : 0;
   un.n = un.kt_hi - loA + 1;
@@ -111,7 +116,7 @@ __device__ __forceinline__ Unit make_unit(const FArgs& a, int u) {
   un.rla[0] = rla_mode && un.t[0] - un.wt >= 0;
   un.rla[1] = rla_mode && un.t[1] >= 0 && un.t[1] - un.wt >= 0;
   un.cA = un.t[0] - un.wt;
-  un.has_state = un.rla[0] && un.cA > 0;
+  un.has_state = un.rla[0] && un.cA >= a.first_state;
   return un;
 }
 
@@ -185,12 +190,13 @@ __device__ bool fwd_loader(const FMaps& tm, const FArgs& a, unsigned char* smem,
     if (!sched_next_producer(a, bars, n, &u)) return false;
     if (u < 0) break;
     const Unit un = make_unit(a, u);
+    if (un.t[0] < 0) continue;                    // beyond this batch entry's length
 #pragma unroll
     for (int X = 0; X < 2; ++X) {
       if (un.t[X] < 0) continue;
       if (cntU[X] >= 1) WAIT_OR_RETURN_W(bars->q_free[X], (cntU[X] - 1) & 1);
       mbar_arrive_expect_tx(&bars->q_full[X], TILE_BYTES);
-      load_tile(smem + F_OFF_Q + X * TILE_BYTES, &tm.q, &bars->q_full[X], un.t[X] * TILE, un.bh_q);
+      load_tile(smem + F_OFF_Q + X * TILE_BYTES, &tm.q, &bars->q_full[X], (un.t[X] - a.off) * TILE, un.bh_q);
       ++cntU[X];
     }
     for (int i = 0; i < un.n; ++i, ++kv_count) {
@@ -230,6 +236,7 @@ __device__ bool fwd_convert(const FArgs& a, unsigned char* smem, FBars* bars, in
     if (!sched_next(bars, n, true, &u)) return false;
     if (u < 0) break;
     const Unit un = make_unit(a, u);
+    if (un.t[0] < 0) continue;
     for (int i = 0; i < un.n; ++i, ++kv_count) {
       const int st = kv_count & 1, use = kv_count >> 1;
       WAIT_OR_RETURN(bars->kv_full[st], use & 1);
@@ -263,6 +270,7 @@ __device__ bool fwd_mma(const FArgs& a, unsigned char* smem, FBars* bars, uint32
     u = __shfl_sync(0xffffffffu, u, 0);
     if (u < 0) break;
     const Unit un = make_unit(a, u);
+    if (un.t[0] < 0) continue;
     const int kv0 = kv_count;
     auto stage_of = [&](int i) { return (kv0 + i) & 1; };
     auto use_of = [&](int i) { return (kv0 + i) >> 1; };
@@ -397,12 +405,13 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     if (!sched_next(bars, n, true, &u)) return false;
     if (u < 0) break;
     const Unit un = make_unit(a, u);
+    if (un.t[0] < 0) continue;
     const int kv0 = kv_count;
     kv_count += un.n;
     const int tX = X ? un.t[1] : un.t[0], i0 = X ? un.i0[1] : un.i0[0], i1 = X ? un.i1[1] : un.i1[0];
     const bool rlaX = X ? un.rla[1] : un.rla[0];
     if (tX < 0) continue;
-    const int q0 = tX * TILE;
+    const int q0 = (tX - a.off) * TILE;          // first query row of the tile (tX is its key-space index)
     const int t = q0 + r;
 
     // ---- window branch: online softmax over the key tiles of the band -------------------
@@ -788,8 +797,8 @@ extern "C" int rattn_timeline_read(unsigned long long* out, int* n) {
 
 cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_states) {
   FMaps tm;
-  if (!make_map(&tm.q, a.q, a.T, (uint64_t)a.B * a.H_q) || !make_map(&tm.k, a.k, a.T, (uint64_t)a.B * a.H_kv) ||
-      !make_map(&tm.v, a.v, a.T, (uint64_t)a.B * a.H_kv) || !make_map(&tm.out, a.out, a.T, (uint64_t)a.B * a.H_q) ||
+  if (!make_map(&tm.q, a.q, a.T, (uint64_t)a.B * a.H_q) || !make_map(&tm.k, a.k, a.Tk, (uint64_t)a.B * a.H_kv) ||
+      !make_map(&tm.v, a.v, a.Tk, (uint64_t)a.B * a.H_kv) || !make_map(&tm.out, a.out, a.T, (uint64_t)a.B * a.H_q) ||
       !make_state_map(&tm.st, a.chunk_state, a.k, (uint64_t)a.B * a.H_kv * a.n_chunks))
     return cudaErrorInvalidValue;
   FArgs t;
@@ -804,9 +813,12 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_sta
   t.n_units = t.n_pairs * t.n_bh;
   t.scale_log2 = a.scale * LOG2E; t.eps = a.eps;
   t.phi = a.phi;
-  // pairs p with 2p - w/128 <= 0 read no stored state
+  t.off = a.q_off / TILE;
+  t.first_state = a.state_in ? 0 : 1;
+  t.seq_lens = a.seq_lens;
+  // pairs p with 2p - w/128 <= 0 read no stored state (a resumed sequence has none: every tile reads one)
   t.n_stateless = 0;
-  if (a.mode == RATTN_MODE_RATTN && after_states) {
+  if (a.mode == RATTN_MODE_RATTN && after_states && !a.state_in) {
     t.n_stateless = (a.w / TILE) / 2 + 1;
     if (t.n_stateless > t.n_pairs) t.n_stateless = t.n_pairs;
   }

@@ -41,8 +41,12 @@ struct StateArgs {
   int n_chunks;
   int store_every;  // the sum after step s is stored iff (out_first + dir * s) % store_every == store_phase
   int store_phase;
-  int row_limit;    // tokens at positions >= row_limit contribute nothing (INT_MAX: no limit)
+  int handoff;      // forward chain that also yields the decode state (see StateLaunch)
+  int T, w;         // rows per head in memory, window
   float* final_out; // optional fp32 [n_kv, 128, 128]: the sum after the last step
+  const float* state_in;   // optional fp32 [n_kv, 128, 128]: the sum starts from it; matrix out_first - dir holds it
+  const int* seq_lens;     // optional: valid rows per batch entry
+  int kv_per_batch;
   int phi;          // rattn_feature_map
   int* status;
 };
@@ -57,8 +61,8 @@ __device__ __forceinline__ bool stored_step(const StateArgs& a, int s) {
   const int o = a.out_first + a.dir * s;
   return o >= 0 && (o % a.store_every) == a.store_phase;
 }
-__device__ __forceinline__ bool flushed_step(const StateArgs& a, int s) {
-  return stored_step(a, s) || (a.final_out != nullptr && s == a.n_steps - 1);
+__device__ __forceinline__ bool flushed_step(const StateArgs& a, int s, int n_steps) {
+  return stored_step(a, s) || (a.final_out != nullptr && s == n_steps - 1);
 }
 
 __global__ void __launch_bounds__(ST_THREADS, 1)
@@ -98,7 +102,19 @@ tc_state_scan_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
-  const int n_items = a.n_steps * a.group;
+  // this head's chain: the caller's step count, or -- variable-length batches -- what the entry's own
+  // length asks for; with the hand-off the tokens from len - w on are still inside the window
+  int n_steps = a.n_steps, row_limit = INT_MAX;
+  {
+    const int len = a.seq_lens ? min(a.T, a.seq_lens[kv / a.kv_per_batch]) : a.T;
+    if (a.seq_lens) {
+      const int nd = max(0, (len + TILE - 1) / TILE - 1 - a.w / TILE);
+      n_steps = (a.handoff && len > a.w) ? nd + 1 : nd;
+    }
+    if (a.handoff) row_limit = len - a.w;
+  }
+  const bool has_init = (a.state_in != nullptr);
+  const int n_items = n_steps * a.group;
   bool ok = true;
 
   if (warp < 8) {
@@ -113,7 +129,7 @@ tc_state_scan_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       // every lane maps its row (the softmax map exchanges partial results between the two lanes
       // of a row with full-warp shuffles, so no lane may skip it); rows past the limit are then cleared
       feature_map_pair_any(xh, xh, row, a.phi);
-      if (token >= a.row_limit) {
+      if (token >= row_limit) {
 #pragma unroll
         for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(xh + row * 128 + (c << 4)) = make_uint4(0, 0, 0, 0);
       }
@@ -127,15 +143,16 @@ tc_state_scan_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       const int st = it % ST_NS, use = it / ST_NS;
       const int s = it / a.group, hh = it - s * a.group;
       ok = mbar_wait_warp(&bars->phi_ready[st], use & 1, &bars->abort);
-      if (ok && hh == 0 && s > 0 && flushed_step(a, s - 1)) {
-        ok = mbar_wait_warp(&bars->acc_free, n_wait & 1, &bars->abort);   // the flush warps hold the previous sum
+      // the flush warps hold the previous sum, or are still writing the incoming state into the accumulator
+      if (ok && hh == 0 && ((s > 0 && flushed_step(a, s - 1, n_steps)) || (s == 0 && has_init))) {
+        ok = mbar_wait_warp(&bars->acc_free, n_wait & 1, &bars->abort);
         ++n_wait;
       }
       if (!ok) break;
       tc_fence_after();
-      mma_mnmn(tmem, smem_u32(smem + st * ST_STAGE), smem_u32(smem + st * ST_STAGE + TILE_BYTES), it > 0);
+      mma_mnmn(tmem, smem_u32(smem + st * ST_STAGE), smem_u32(smem + st * ST_STAGE + TILE_BYTES), it > 0 || has_init);
       mma_commit(&bars->free_[st]);
-      if (hh == a.group - 1 && flushed_step(a, s)) mma_commit(&bars->done);
+      if (hh == a.group - 1 && flushed_step(a, s, n_steps)) mma_commit(&bars->done);
     }
   } else if (warp == 9) {
     // ---- loader ---------------------------------------------------------------------------
@@ -157,8 +174,64 @@ tc_state_scan_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     unsigned char* s_out = smem + ST_OFF_OUT;
     const bool issuer = (tid == 320);
     int n_flush = 0;
-    for (int s = 0; s < a.n_steps && ok; ++s) {
-      if (!flushed_step(a, s)) continue;
+    // bf16 copy of this thread's row of the sum -> staging -> matrix `mat` of the head, one TMA store
+    auto store_row = [&](const float (&x)[4][32], int mat) {
+      if (issuer) tma_store_wait_read();                     // the staging tile has left
+      asm volatile("bar.sync 4, 128;" ::: "memory");
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          uint4 u;
+          u.x = pack_bf16(x[c][8 * e + 0], x[c][8 * e + 1]);
+          u.y = pack_bf16(x[c][8 * e + 2], x[c][8 * e + 3]);
+          u.z = pack_bf16(x[c][8 * e + 4], x[c][8 * e + 5]);
+          u.w = pack_bf16(x[c][8 * e + 6], x[c][8 * e + 7]);
+          *reinterpret_cast<uint4*>(s_out + swz(r, 4 * c + e)) = u;
+        }
+      }
+      fence_proxy_async_smem();
+      asm volatile("bar.sync 4, 128;" ::: "memory");
+      if (issuer) {
+        store_tile(&tm_out, s_out, 0, kv * a.n_chunks + mat);
+        tma_store_commit();
+      }
+    };
+    auto write_final = [&](const float (&x)[4][32]) {
+      float* dst = a.final_out + ((size_t)kv * 128 + r) * 128;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+          *reinterpret_cast<float4*>(dst + 32 * c + 4 * e) =
+              make_float4(x[c][4 * e], x[c][4 * e + 1], x[c][4 * e + 2], x[c][4 * e + 3]);
+      }
+    };
+    if (has_init || (a.final_out != nullptr && n_steps == 0)) {
+      // the chain starts from the incoming state (zero without one): into the accumulator, into the
+      // matrix in front of the first step's, and -- when no token leaves the window -- straight out
+      float x[4][32];
+      const float* src = has_init ? a.state_in + ((size_t)kv * 128 + r) * 128 : nullptr;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float4 f = src ? *reinterpret_cast<const float4*>(src + 32 * c + 4 * e) : make_float4(0.f, 0.f, 0.f, 0.f);
+          x[c][4 * e] = f.x; x[c][4 * e + 1] = f.y; x[c][4 * e + 2] = f.z; x[c][4 * e + 3] = f.w;
+        }
+      }
+      if (has_init) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_st32(t_row + 32 * c, x[c]);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&bars->acc_free);
+        if (stored_step(a, -1)) store_row(x, a.out_first - a.dir);
+      }
+      if (a.final_out != nullptr && n_steps == 0) write_final(x);
+    }
+    for (int s = 0; s < n_steps && ok; ++s) {
+      if (!flushed_step(a, s, n_steps)) continue;
       ok = mbar_wait(&bars->done, n_flush & 1, &bars->abort);
       ++n_flush;
       if (!ok) break;
@@ -169,38 +242,8 @@ tc_state_scan_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
       tmem_wait_ld();
       tc_fence_before();
       mbar_arrive(&bars->acc_free);                            // the next step may accumulate
-      if (stored_step(a, s)) {
-        if (issuer) tma_store_wait_read();                     // the staging tile has left
-        asm volatile("bar.sync 4, 128;" ::: "memory");
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            uint4 u;
-            u.x = pack_bf16(x[c][8 * e + 0], x[c][8 * e + 1]);
-            u.y = pack_bf16(x[c][8 * e + 2], x[c][8 * e + 3]);
-            u.z = pack_bf16(x[c][8 * e + 4], x[c][8 * e + 5]);
-            u.w = pack_bf16(x[c][8 * e + 6], x[c][8 * e + 7]);
-            *reinterpret_cast<uint4*>(s_out + swz(r, 4 * c + e)) = u;
-          }
-        }
-        fence_proxy_async_smem();
-        asm volatile("bar.sync 4, 128;" ::: "memory");
-        if (issuer) {
-          store_tile(&tm_out, s_out, 0, kv * a.n_chunks + a.out_first + a.dir * s);
-          tma_store_commit();
-        }
-      }
-      if (a.final_out != nullptr && s == a.n_steps - 1) {
-        float* dst = a.final_out + ((size_t)kv * 128 + r) * 128;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-#pragma unroll
-          for (int e = 0; e < 8; ++e)
-            *reinterpret_cast<float4*>(dst + 32 * c + 4 * e) =
-                make_float4(x[c][4 * e], x[c][4 * e + 1], x[c][4 * e + 2], x[c][4 * e + 3]);
-        }
-      }
+      if (stored_step(a, s)) store_row(x, a.out_first + a.dir * s);
+      if (a.final_out != nullptr && s == n_steps - 1) write_final(x);
     }
     if (issuer) tma_store_wait();
   }
@@ -217,7 +260,7 @@ tc_state_scan_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 
 // x, y: [n_kv * group, T, 128] bf16; out: [n_kv * n_chunks, 128, 128] bf16.
 cudaError_t launch_tc_states(const StateLaunch& L, cudaStream_t s) {
-  if (L.n_steps <= 0) return cudaSuccess;
+  if (L.n_steps <= 0 && !L.state_in && !(L.seq_lens && L.final_out)) return cudaSuccess;
   CUtensorMap tm_x, tm_y, tm_out;
   if (!make_map(&tm_x, L.x, L.T, (uint64_t)L.n_kv * L.group) || !make_map(&tm_y, L.y, L.T, (uint64_t)L.n_kv * L.group) ||
       !make_map(&tm_out, L.out, 128, (uint64_t)L.n_kv * L.n_chunks))
@@ -227,8 +270,10 @@ cudaError_t launch_tc_states(const StateLaunch& L, cudaStream_t s) {
   a.n_chunks = L.n_chunks; a.status = L.status;
   a.store_every = L.store_every > 0 ? L.store_every : 1;
   a.store_phase = L.store_phase;
-  a.row_limit = L.row_limit > 0 ? L.row_limit : INT_MAX;
+  a.handoff = L.handoff; a.T = L.T; a.w = L.w;
   a.final_out = L.final_out;
+  a.state_in = L.state_in;
+  a.seq_lens = L.seq_lens; a.kv_per_batch = L.kv_per_batch > 0 ? L.kv_per_batch : 1;
   a.phi = L.phi;
   cudaError_t e = cudaFuncSetAttribute(tc_state_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ST_SMEM);
   if (e != cudaSuccess) return e;

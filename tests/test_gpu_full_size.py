@@ -131,3 +131,34 @@ def test_config5_few_heads():
     """Four batch entries of the same configuration (32 K/V heads in all): the chunk-state chains
     occupy only 32 SMs while the main kernel already runs on the others."""
     _prefill_then_decode(W.C5.replace(B=4), [(0, 0), (3, 31)])
+
+
+def test_config3_prefill_in_four_chunks():
+    """B=2, H=32/8, T=8192, w=512 cut into four chunks of 2048 tokens, each resuming from the ring and
+    state the previous one handed out (tensor-core kernels throughout): sampled rows against the oracle
+    on the whole sequence, and the final state against the one-pass hand-off."""
+    wl = W.C3
+    q, k, v = W.make_qkv(wl, "cuda")
+    C = 2048
+    state = torch.zeros(wl.B, wl.H_kv, wl.d, wl.d, device="cuda")
+    k_ring = torch.zeros(wl.B, wl.H_kv, wl.w, wl.d, device="cuda", dtype=torch.bfloat16)
+    v_ring = torch.zeros_like(k_ring)
+    y = torch.empty_like(q)
+    for c in range(wl.T // C):
+        sl = slice(c * C, (c + 1) * C)
+        qc, kc, vc = (t[:, :, sl].contiguous() for t in (q, k, v))
+        kw = dict(scale=wl.scale, state_out=state, k_ring_out=k_ring, v_ring_out=v_ring)
+        if c == 0:
+            ws = R.alloc_workspace(qc, kc, wl.w, R.MODE_RATTN, 0)
+        else:
+            ws = R.alloc_workspace_chunked(qc, kc, wl.w)
+            kw.update(state_in=state, k_ring_in=k_ring, v_ring_in=v_ring, pos0=c * C)
+        y[:, :, sl] = R.rattn_forward_ex(qc, kc, vc, wl.w, workspace=ws, **kw)
+        torch.cuda.synchronize()
+        assert R.rattn_read_status(ws) == 0
+    check_sampled_forward(wl, y, q, k, v, [(0, 5), (1, 30)], n_random=48)
+    one_pass = torch.zeros_like(state)
+    ws = R.alloc_workspace(q, k, wl.w, R.MODE_RATTN, 0)
+    R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws, state_out=one_pass)
+    torch.cuda.synchronize()
+    assert (state - one_pass).abs().max().item() <= 2.0 ** -8 * max(1.0, one_pass.abs().max().item())
