@@ -650,6 +650,50 @@ def run_replicas_selftest(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """The forward's tuning parameters swept on config 2 and on the paper's own head shapes
+    (Table 1: 16 query / 4 K/V heads, 40 / 8), one JSON line per point: stored-state stride m,
+    overlap of the chunk-state kernel with the main kernel, unit order.  The chunk size is the
+    128-token MMA tile and is not swept.  Device-resident inputs, three rotating input sets."""
+    from paper_2506_15545_b200 import binding as R
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    sync = torch.cuda.synchronize
+    pk = peaks()
+    shapes = [("c2 (B=4, H=16/16, T=4096, w=512)", W.C2),
+              ("paper 3B heads 16/4 (B=4, T=4096, w=512)", W.C2.replace(H_q=16, H_kv=4)),
+              ("paper 12B heads 40/8 (B=2, T=8192, w=1024)", W.C3.replace(H_q=40, H_kv=8, w=1024))]
+    for label, wl in shapes:
+        q, k, v = W.make_qkv(wl, dev)
+        sets = [(q, k, v)] + [tuple(t.clone() for t in (q, k, v)) for _ in range(2)]
+        ws = R.alloc_workspace(q, k, wl.w, R.MODE_RATTN, 0)
+        o = torch.empty_like(q)
+        it = [0]
+
+        def fwd():
+            x = sets[it[0] % 3]
+            it[0] += 1
+            R.rattn_forward_ex(x[0], x[1], x[2], wl.w, scale=wl.scale, workspace=ws, out=o)
+
+        for m in (1, 2):
+            for overlap in (0, 1):
+                for order in (0, 1):
+                    R.rattn_tune(R.TUNE_STATE_STRIDE, m)
+                    R.rattn_tune(R.TUNE_OVERLAP, overlap)
+                    R.rattn_tune(R.TUNE_UNIT_ORDER, order)
+                    ms = timed(fwd, 40, 5, sync)
+                    assert R.rattn_read_status(ws) == 0
+                    t_roof = max(flops(wl, "fwd") / (pk["tf_burst"] * 1e12), io_bytes_fwd(wl) / (pk["hbm"] * 1e9)) * 1e3
+                    print(json.dumps({"sweep": label, "m": m, "chunk": 128, "overlap": overlap, "unit_order": order,
+                                      "ms": round(ms, 4), "tflops": round(flops(wl, "fwd") / (ms * 1e-3) / 1e12, 1),
+                                      "roofline_frac": round(t_roof / ms, 4)}), flush=True)
+        R.rattn_tune(R.TUNE_STATE_STRIDE, 0)
+        R.rattn_tune(R.TUNE_OVERLAP, 1)
+        R.rattn_tune(R.TUNE_UNIT_ORDER, 0)
+        del sets, q, k, v, ws, o
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -658,16 +702,21 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference", "replicas-selftest"])
     ap.add_argument("--case", default=None, choices=["fwd", "train", "decode"],
                     help="run one small case (for profiler captures) instead of the benchmark")
+    ap.add_argument("--sweep", action="store_true",
+                    help="sweep the forward's tuning parameters (stored-state stride, overlap, unit order)")
     ap.add_argument("--all-configs", action="store_true",
                     help="time the forward of all five named configurations instead of the benchmark")
     ap.add_argument("--c5-batch", type=int, default=32, help="batch entries of config 5's prefill to time")
     ap.add_argument("--clock-seconds", type=float, default=2.0,
                     help="after the K timed steps, repeat the step for about this long under the clock sampler")
     args = ap.parse_args()
-    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.all_configs or args.case):
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.all_configs or args.case or args.sweep):
         sys.exit(launch_replicas(sys.argv[1:], args.gpus))
     if args.impl == "replicas-selftest":
         run_replicas_selftest(args)
+        return
+    if args.sweep:
+        run_sweep(args)
         return
     if args.all_configs:
         run_all_configs(args)

@@ -290,6 +290,24 @@ uint64_t rattn_launch_count(void);
 int rattn_timing_enable(int on);
 size_t rattn_timing_read(char* buf, size_t buf_bytes);
 
+/*
+ * Tuning parameters of the tensor-core forward, process-wide (the counterpart of the paper's
+ * search over the stored-state stride m and the chunk size C, Section 3.2 "Kernel Design"; here
+ * the chunk is the 128-token MMA tile and is fixed).  rattn_tune returns the previous value,
+ * or RATTN_ERR_BAD_ARG for an unknown knob or a value out of range.  Defaults are what the
+ * sweep in profiles/ found best on B200.
+ */
+typedef enum rattn_knob {
+  RATTN_TUNE_STATE_STRIDE = 0,   /* m: 0 = automatic (2 for an inference forward, whose query-tile pairs read every
+                                    second chunk state; 1 when the backward will read them all), 1, 2 */
+  RATTN_TUNE_OVERLAP = 1,        /* 1 (default): the main kernel starts under the chunk-state kernel
+                                    (programmatic dependent launch); 0: strictly one after the other */
+  RATTN_TUNE_UNIT_ORDER = 2,     /* 0 (default): units that read no stored state first, then heaviest first;
+                                    1: heaviest first throughout */
+  RATTN_TUNE_GRID = 3            /* CTAs of the persistent forward kernel: 0 (default) = one per SM */
+} rattn_knob;
+int rattn_tune(int knob, int value);
+
 /* 1 when the tensor-core (tcgen05) forward would be chosen for these sizes. */
 int rattn_uses_tensor_path(int d, int w, int dtype, int mode, unsigned flags);
 

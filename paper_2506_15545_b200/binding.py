@@ -25,8 +25,9 @@ EXPORTS = (
     "rattn_workspace_bytes_ex", "rattn_workspace_bytes_chunked",
     "rattn_read_status", "rattn_strerror", "rattn_last_cuda_error", "rattn_launch_count",
     "rattn_uses_tensor_path", "rattn_timing_enable", "rattn_timing_read",
-    "rattn_forward_static", "rattn_static_status",
+    "rattn_forward_static", "rattn_static_status", "rattn_tune",
 )
+TUNE_STATE_STRIDE, TUNE_OVERLAP, TUNE_UNIT_ORDER, TUNE_GRID = 0, 1, 2, 3
 
 
 class RattnParams(ctypes.Structure):
@@ -106,6 +107,8 @@ def lib() -> ctypes.CDLL:
     L.rattn_forward_static.restype = ci
     L.rattn_static_status.argtypes = [vp]
     L.rattn_static_status.restype = ci
+    L.rattn_tune.argtypes = [ci, ci]
+    L.rattn_tune.restype = ci
     L.rattn_timing_enable.argtypes = [ci]
     L.rattn_timing_enable.restype = ci
     L.rattn_timing_read.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
@@ -298,6 +301,13 @@ def rattn_read_status(workspace, stream=None) -> int:
 def rattn_static_status(stream=None) -> int:
     """Status word of rattn_forward_static's last call on the current device."""
     return int(lib().rattn_static_status(_stream(stream)))
+
+
+def rattn_tune(knob: int, value: int) -> int:
+    """Sets a tuning parameter of the tensor-core forward; returns the previous value."""
+    r = int(lib().rattn_tune(knob, value))
+    _check(r if r < 0 else 0, "rattn_tune")
+    return r
 
 
 def rattn_launch_count() -> int:

@@ -18,7 +18,9 @@ template <typename T> struct Vec16;        // a 16-byte vector of I/O elements
 template <> struct Vec16<__nv_bfloat16> {
   static constexpr int N = 8;
   static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&f)[8]) {
-    uint4 u = *reinterpret_cast<const uint4*>(p);
+    unpack(*reinterpret_cast<const uint4*>(p), f);
+  }
+  static __device__ __forceinline__ void unpack(uint4 u, float (&f)[8]) {
     const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -33,6 +35,9 @@ template <> struct Vec16<float> {
   static __device__ __forceinline__ void load(const float* p, float (&f)[4]) {
     float4 u = *reinterpret_cast<const float4*>(p);
     f[0] = u.x; f[1] = u.y; f[2] = u.z; f[3] = u.w;
+  }
+  static __device__ __forceinline__ void unpack(uint4 u, float (&f)[4]) {
+    f[0] = __uint_as_float(u.x); f[1] = __uint_as_float(u.y); f[2] = __uint_as_float(u.z); f[3] = __uint_as_float(u.w);
   }
 };
 
@@ -85,33 +90,42 @@ struct DecodeArgs {
   float scale, eps;
 };
 
+// One CTA per (batch entry, K/V head); the g query heads of the group are served GH at a time.
+//   scores   thread = ring slot: the slot's whole key row is read with 16-byte loads and dotted
+//            with the GH query vectors held in shared memory (no cross-lane reduction at all)
+//   softmax  one warp per head over the w + 1 logits in shared memory
+//   P V      16 lanes x 16 bytes cover a value row; a thread keeps GH x 8 partial sums over its
+//            share of the slots; partial sums are merged through shared memory
+//   state    read-out phi(q) S and the update S += phi(k_old)^T v_old in one pass, float4
 template <typename TIO, int D>
-__global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecodeArgs a) {
-  constexpr int EPL = Vec16<TIO>::N;        // elements per lane per 16-byte load
-  constexpr int LPK = D / EPL;              // lanes that cover one key row
-  constexpr int KPW = 32 / LPK;             // key rows per warp per load
+__global__ void __launch_bounds__(DEC_THREADS, 2) decode_kernel(DecodeArgs a) {
+  constexpr int EPL = Vec16<TIO>::N;        // elements per 16-byte load
+  constexpr int LPR = D / EPL;              // lanes (loads) that cover one row
+  constexpr int RPP = DEC_THREADS / LPR;    // value rows in flight per pass of the P V phase
   constexpr int C4 = D / 4;                 // float4 columns of a state row
   constexpr int RP = DEC_THREADS / C4;      // state rows per pass
 
   extern __shared__ __align__(16) float sm[];
   const int g = a.group;
-  float* q_s = sm;                          // [g][D] raw q
+  const int w = a.w;
+  float* q_s = sm;                          // [g][D] raw q, pre-multiplied by the logit scale
   float* fq_s = q_s + g * D;                // [g][D] phi(q)
   float* k_new = fq_s + g * D;              // [D]
   float* v_new = k_new + D;
   float* k_old = v_new + D;
   float* v_old = k_old + D;
   float* fk_old = v_old + D;
-  float* s_new = fk_old + D;                // [GH] logit of the incoming token
-  float* part_m = s_new + GH;               // [WARPS][GH]
-  float* part_l = part_m + DEC_WARPS * GH;  // [WARPS][GH]
-  float* o_swa = part_l + DEC_WARPS * GH;   // [GH][D]
+  float* p_s = fk_old + D;                  // [GH][w + 1] logits, then weights (slot w = the incoming token)
+  float* red = p_s + GH * (w + 1) + ((GH * (w + 1)) & 1 ? 3 : 0) + 2;   // padded to 16 bytes below
+  red = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(red) + 15) & ~uintptr_t(15));
+  float* o_swa = red;                       // [GH][D]
   float* o_rla = o_swa + GH * D;            // [GH][D]
-  float* part_acc = o_rla + GH * D;         // [max(WARPS,RP)][GH][D]
+  float* stat = o_rla + GH * D;             // [GH] 1 / sum of weights
+  float* part = stat + 4 * GH;              // [max(DEC_WARPS, RP)][GH][D] partial sums
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = blockIdx.x / a.H_kv, hk = blockIdx.x % a.H_kv;
-  const int w = a.w, pos = a.pos_dev ? a.pos_dev[b] : a.pos;
+  const int pos = a.pos_dev ? a.pos_dev[b] : a.pos;
   const bool evict = pos - w >= 0;
   const int slot = pos % w;
   const int n_valid = pos < w ? pos : w;
@@ -124,6 +138,20 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecodeArgs a) {
   float* S = a.state + ((size_t)b * a.H_kv + hk) * (size_t)D * D;
   TIO* og = reinterpret_cast<TIO*>(a.out) + ((size_t)b * a.H_q + (size_t)hk * g) * D;
 
+  // The value ring and the state are needed only after the logits: ask L2 for them now (one request
+  // per 128-byte line), so that their HBM latency runs under the key phase.
+  {
+    const char* kb = reinterpret_cast<const char*>(kr);
+    const char* vb = reinterpret_cast<const char*>(vr);
+    const size_t v_bytes = (size_t)n_valid * D * sizeof(TIO);
+    for (size_t off = (size_t)tid * 128; off < v_bytes; off += (size_t)DEC_THREADS * 128)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(kb + off));
+    for (size_t off = (size_t)tid * 128; off < v_bytes; off += (size_t)DEC_THREADS * 128)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(vb + off));
+    const char* sb = reinterpret_cast<const char*>(S);
+    for (size_t off = (size_t)tid * 128; off < (size_t)D * D * sizeof(float); off += (size_t)DEC_THREADS * 128)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(sb + off));
+  }
   for (int i = tid; i < g * D; i += DEC_THREADS) q_s[i] = to_f(qg[i]);
   if (tid < D) {
     k_new[tid] = to_f(kg[tid]);
@@ -139,137 +167,106 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecodeArgs a) {
     else if (evict) warp_feature_map<D>(fk_old, k_old, lane, a.phi);
   }
   __syncthreads();
+  for (int i = tid; i < g * D; i += DEC_THREADS) q_s[i] *= a.scale;     // phi has seen the raw q
+  __syncthreads();
 
-  const int sub = lane / LPK, chunk = lane % LPK;
   for (int h0 = 0; h0 < g; h0 += GH) {
     const int nh = (g - h0) < GH ? (g - h0) : GH;
-    // ---- SWA over the ring (Section 2.1), online softmax per warp -------------------
-    float qr[GH][EPL], m[GH], l[GH], acc[GH][EPL];
+    // ---- SWA logits (Section 2.1): one ring slot per thread.  The slot's whole key row is read by
+    // its thread (16-byte loads, eight in flight) and dotted with the GH query vectors, which every
+    // lane reads from the same shared-memory address (a broadcast): no cross-lane reduction at all.
+    // (Eight lanes per row with coalesced 32-byte pieces and three shuffle rounds measured 60 % slower.)
+    for (int s = tid; s < n_valid; s += DEC_THREADS) {
+      float dot[GH];
 #pragma unroll
-    for (int hh = 0; hh < GH; ++hh) {
-      m[hh] = -INFINITY;
-      l[hh] = 0.f;
-#pragma unroll
-      for (int e = 0; e < EPL; ++e) {
-        qr[hh][e] = hh < nh ? q_s[(h0 + hh) * D + chunk * EPL + e] * a.scale : 0.f;
-        acc[hh][e] = 0.f;
-      }
-    }
-    constexpr int U = 4;                    // loads in flight per lane (x2 for K and V)
-    for (int s0 = warp * KPW; s0 < n_valid; s0 += DEC_WARPS * KPW * U) {
-      float kx[U][EPL], vx[U][EPL];
-      bool ok[U];
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int s = s0 + u * DEC_WARPS * KPW + sub;
-        ok[u] = s < n_valid;
-        if (ok[u]) {
-          Vec16<TIO>::load(kr + (size_t)s * D + chunk * EPL, kx[u]);
-          Vec16<TIO>::load(vr + (size_t)s * D + chunk * EPL, vx[u]);
-        } else {
-#pragma unroll
-          for (int e = 0; e < EPL; ++e) { kx[u][e] = 0.f; vx[u][e] = 0.f; }
-        }
-      }
-      // Scores of the whole batch first, then one running-maximum update and one rescale of
-      // the accumulator per batch and head (rescaling per key costs twice the arithmetic and
-      // chains every key behind the previous one).
-      float dot[U][GH];
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
+      for (int hh = 0; hh < GH; ++hh) dot[hh] = 0.f;
+      const TIO* row = kr + (size_t)s * D;
+#pragma unroll 8
+      for (int c = 0; c < LPR; ++c) {
+        float kx[EPL];
+        Vec16<TIO>::load(row + c * EPL, kx);
 #pragma unroll
         for (int hh = 0; hh < GH; ++hh) {
-          float x = 0.f;
+          if (hh < nh) {
+            const float* qh = q_s + (h0 + hh) * D + c * EPL;
 #pragma unroll
-          for (int e = 0; e < EPL; ++e) x += qr[hh][e] * kx[u][e];
-          dot[u][hh] = x;
+            for (int e = 0; e < EPL; ++e) dot[hh] += qh[e] * kx[e];
+          }
         }
       }
 #pragma unroll
-      for (int o = 1; o < LPK; o <<= 1) {
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-#pragma unroll
-          for (int hh = 0; hh < GH; ++hh) dot[u][hh] += __shfl_xor_sync(0xffffffffu, dot[u][hh], o);
-        }
-      }
+      for (int hh = 0; hh < GH; ++hh) p_s[hh * (w + 1) + s] = dot[hh];
+    }
+    if (warp == DEC_WARPS - 1) {                                 // the incoming token, one warp
 #pragma unroll
       for (int hh = 0; hh < GH; ++hh) {
-        float mb = -INFINITY;
-#pragma unroll
-        for (int u = 0; u < U; ++u) mb = fmaxf(mb, ok[u] ? dot[u][hh] : -INFINITY);
-        if (mb == -INFINITY) continue;                       // no valid key in this batch for this lane group
-        const float m_new = fmaxf(m[hh], mb);
-        const float corr = __expf(m[hh] - m_new);            // exp(-inf) = 0 on the first batch
-        float p[U];
-        float ps = 0.f;
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-          p[u] = ok[u] ? __expf(dot[u][hh] - m_new) : 0.f;
-          ps += p[u];
-        }
-        l[hh] = l[hh] * corr + ps;
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) {
-          float x = acc[hh][e] * corr;
-#pragma unroll
-          for (int u = 0; u < U; ++u) x += p[u] * vx[u][e];
-          acc[hh][e] = x;
-        }
-        m[hh] = m_new;
+        float x = 0.f;
+        if (hh < nh)
+          for (int c = lane; c < D; c += 32) x += q_s[(h0 + hh) * D + c] * k_new[c];
+        x = warp_sum(x);
+        if (lane == 0) p_s[hh * (w + 1) + w] = x;
       }
     }
-    // merge the KPW key sub-groups of the warp
-#pragma unroll
-    for (int o = LPK; o < 32; o <<= 1) {
-#pragma unroll
-      for (int hh = 0; hh < GH; ++hh) {
-        const float m_o = __shfl_xor_sync(0xffffffffu, m[hh], o);
-        const float l_o = __shfl_xor_sync(0xffffffffu, l[hh], o);
-        const float m_new = fmaxf(m[hh], m_o);
-        const float c0 = (m[hh] == -INFINITY) ? 0.f : __expf(m[hh] - m_new);
-        const float c1 = (m_o == -INFINITY) ? 0.f : __expf(m_o - m_new);
-        l[hh] = l[hh] * c0 + l_o * c1;
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) {
-          const float a_o = __shfl_xor_sync(0xffffffffu, acc[hh][e], o);
-          acc[hh][e] = acc[hh][e] * c0 + a_o * c1;
-        }
-        m[hh] = m_new;
+    __syncthreads();
+    // ---- softmax over the window, one warp per head ----------------------------------------
+    if (warp < nh) {
+      float* ph = p_s + warp * (w + 1);
+      float m = ph[w];
+      for (int s = lane; s < n_valid; s += 32) m = fmaxf(m, ph[s]);
+      m = warp_max(m);
+      float l = 0.f;
+      for (int s = lane; s < n_valid; s += 32) {
+        const float e = __expf(ph[s] - m);
+        ph[s] = e;
+        l += e;
+      }
+      l = warp_sum(l);
+      const float en = __expf(ph[w] - m);
+      if (lane == 0) {
+        ph[w] = en;
+        stat[warp] = 1.f / (l + en);
       }
     }
-    if (sub == 0) {
+    __syncthreads();
+    // ---- P V: LPR lanes cover a value row, RPP rows in flight -------------------------------
+    {
+      const int chunk = tid % LPR, r0 = tid / LPR;
+      float acc[GH][EPL];
 #pragma unroll
-      for (int hh = 0; hh < GH; ++hh) {
-        if (chunk == 0) {
-          part_m[warp * GH + hh] = m[hh];
-          part_l[warp * GH + hh] = l[hh];
+      for (int hh = 0; hh < GH; ++hh)
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc[hh][e] = 0.f;
+#pragma unroll 4
+      for (int s = r0; s < n_valid; s += RPP) {
+        float vx[EPL];
+        Vec16<TIO>::load(vr + (size_t)s * D + chunk * EPL, vx);
+#pragma unroll
+        for (int hh = 0; hh < GH; ++hh) {
+          const float p = p_s[hh * (w + 1) + s];
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) acc[hh][e] += p * vx[e];
         }
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) part_acc[(warp * GH + hh) * D + chunk * EPL + e] = acc[hh][e];
       }
-    }
-    if (warp < nh) {                        // logit of the incoming token for head h0+warp
-      float dot = 0.f;
-      for (int c = lane; c < D; c += 32) dot += q_s[(h0 + warp) * D + c] * k_new[c];
-      dot = warp_sum(dot) * a.scale;
-      if (lane == 0) s_new[warp] = dot;
+      // merge the rows held by the lanes of a warp that share `chunk`, then the warps
+#pragma unroll
+      for (int o = LPR; o < 32; o <<= 1)
+#pragma unroll
+        for (int hh = 0; hh < GH; ++hh)
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) acc[hh][e] += __shfl_xor_sync(0xffffffffu, acc[hh][e], o);
+      if (lane < LPR) {
+#pragma unroll
+        for (int hh = 0; hh < GH; ++hh)
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) part[(warp * GH + hh) * D + chunk * EPL + e] = acc[hh][e];
+      }
     }
     __syncthreads();
     for (int i = tid; i < nh * D; i += DEC_THREADS) {
       const int hh = i / D, c = i % D;
-      float M = s_new[hh];
-      for (int wv = 0; wv < DEC_WARPS; ++wv) M = fmaxf(M, part_m[wv * GH + hh]);
-      float pn = __expf(s_new[hh] - M);
-      float L = pn, O = pn * v_new[c];
-      for (int wv = 0; wv < DEC_WARPS; ++wv) {
-        const float mw = part_m[wv * GH + hh];
-        if (mw == -INFINITY) continue;
-        const float cf = __expf(mw - M);
-        L += part_l[wv * GH + hh] * cf;
-        O += part_acc[(wv * GH + hh) * D + c] * cf;
-      }
-      o_swa[hh * D + c] = O / L;
+      float O = p_s[hh * (w + 1) + w] * v_new[c];
+      for (int wv = 0; wv < DEC_WARPS; ++wv) O += part[(wv * GH + hh) * D + c];
+      o_swa[hh * D + c] = O * stat[hh];
     }
     __syncthreads();
 
@@ -298,13 +295,13 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecodeArgs a) {
       }
 #pragma unroll
       for (int hh = 0; hh < GH; ++hh)
-        *reinterpret_cast<float4*>(part_acc + ((size_t)(rl * GH + hh)) * D + c4 * 4) = ar[hh];
+        *reinterpret_cast<float4*>(part + ((size_t)(rl * GH + hh)) * D + c4 * 4) = ar[hh];
     }
     __syncthreads();
     for (int i = tid; i < nh * D; i += DEC_THREADS) {
       const int hh = i / D, c = i % D;
       float O = 0.f;
-      for (int r = 0; r < RP; ++r) O += part_acc[(r * GH + hh) * D + c];
+      for (int r = 0; r < RP; ++r) O += part[(r * GH + hh) * D + c];
       o_rla[hh * D + c] = O;
     }
     __syncthreads();
@@ -337,15 +334,15 @@ __global__ void __launch_bounds__(DEC_THREADS) decode_kernel(DecodeArgs a) {
   }
 }
 
-template <int D> constexpr size_t decode_smem_floats(int g) {
+template <int D> size_t decode_smem_floats(int g, int w) {
   constexpr int RP = DEC_THREADS / (D / 4);
   constexpr int PR = RP > DEC_WARPS ? RP : DEC_WARPS;
-  return (size_t)2 * g * D + 5 * D + GH + 2 * DEC_WARPS * GH + 2 * GH * D + (size_t)PR * GH * D;
+  return (size_t)2 * g * D + 5 * D + (size_t)GH * (w + 1) + 16 + 2 * GH * D + 4 * GH + (size_t)PR * GH * D;
 }
 
 template <typename TIO, int D>
 cudaError_t launch_dec(const DecodeArgs& a, cudaStream_t s) {
-  const size_t smem = decode_smem_floats<D>(a.group) * sizeof(float);
+  const size_t smem = decode_smem_floats<D>(a.group, a.w) * sizeof(float);
   if (smem > 227 * 1024) return cudaErrorInvalidValue;
   cudaError_t e = cudaFuncSetAttribute(decode_kernel<TIO, D>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -27,6 +27,9 @@ int debug_skip_arrive() {
 #endif
 }
 
+static std::atomic<int> g_tuning[4] = {{0}, {1}, {0}, {0}};
+int tuning(int knob) { return g_tuning[knob].load(std::memory_order_relaxed); }
+
 void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 void set_last_cuda_error(int cuda_error) { g_last_cuda_error = cuda_error; }
 
@@ -434,6 +437,12 @@ int rattn_debug_withhold_arrival(int on) {
   return RATTN_OK;
 }
 #endif
+
+int rattn_tune(int knob, int value) {
+  static const int lo[4] = {0, 0, 0, 0}, hi[4] = {2, 1, 1, 1 << 16};
+  if (knob < 0 || knob > 3 || value < lo[knob] || value > hi[knob]) return RATTN_ERR_BAD_ARG;
+  return g_tuning[knob].exchange(value, std::memory_order_relaxed);
+}
 
 int rattn_uses_tensor_path(int d, int w, int dtype, int mode, unsigned flags) {
   return tensor_path(d, w, dtype, mode, flags) ? 1 : 0;

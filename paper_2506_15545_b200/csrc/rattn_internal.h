@@ -128,6 +128,7 @@ cudaError_t launch_gather_history(const Args& a, const void* k_chunk, const void
                                   const void* v_ring, void* k_ext, void* v_ext, int pos0, cudaStream_t s);
 
 int debug_skip_arrive();                    // always 0 outside the debug build
+int tuning(int knob);                       // current value of a rattn_knob
 void count_launches(int n);
 void set_last_cuda_error(int cuda_error);   // what rattn_last_cuda_error() reports for this thread
 

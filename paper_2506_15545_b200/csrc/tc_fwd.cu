@@ -37,8 +37,10 @@ cudaError_t launch_tc_forward(const Args& a, cudaStream_t s) {
     L.T = a.Tk; L.n_kv = n_kv; L.group = 1; L.n_chunks = a.n_chunks;
     L.n_steps = n_steps > 0 ? n_steps : 0; L.first = 0; L.dir = +1; L.out_first = 1;
     // the main kernel reads S_[c] for c = off + 2p - wt only
-    L.store_every = a.training ? 1 : 2;
-    L.store_phase = a.training ? 0 : ((off + wt) & 1);
+    const int m = tuning(RATTN_TUNE_STATE_STRIDE);
+    const bool every = a.training || m == 1;
+    L.store_every = every ? 1 : 2;
+    L.store_phase = every ? 0 : ((off + wt) & 1);
     L.handoff = want_state ? 1 : 0;
     L.w = a.w;
     L.final_out = want_state ? a.state_out : nullptr;

@@ -818,7 +818,7 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_sta
   t.seq_lens = a.seq_lens;
   // pairs p with 2p - w/128 <= 0 read no stored state (a resumed sequence has none: every tile reads one)
   t.n_stateless = 0;
-  if (a.mode == RATTN_MODE_RATTN && after_states && !a.state_in) {
+  if (a.mode == RATTN_MODE_RATTN && after_states && !a.state_in && tuning(RATTN_TUNE_UNIT_ORDER) == 0) {
     t.n_stateless = (a.w / TILE) / 2 + 1;
     if (t.n_stateless > t.n_pairs) t.n_stateless = t.n_pairs;
   }
@@ -832,6 +832,7 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_sta
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(tc_fwd2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, F_SMEM);
   if (e != cudaSuccess) return e;
+  if (tuning(RATTN_TUNE_GRID) > 0 && tuning(RATTN_TUNE_GRID) < n_sm) n_sm = tuning(RATTN_TUNE_GRID);
   const int grid = t.n_units < n_sm ? t.n_units : n_sm;
   {
     KernelTimer kt("tc_fwd", s);
@@ -845,7 +846,7 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_sta
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = after_states ? 1 : 0;
+    attr[0].val.programmaticStreamSerializationAllowed = (after_states && tuning(RATTN_TUNE_OVERLAP)) ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     e = cudaLaunchKernelEx(&cfg, tc_fwd2_kernel, tm, t);
