@@ -677,7 +677,7 @@ def run_sweep(args):
 
         for m in (1, 2):
             for overlap in (0, 1):
-                for order in (0, 1):
+                for order in (1, 2):
                     R.rattn_tune(R.TUNE_STATE_STRIDE, m)
                     R.rattn_tune(R.TUNE_OVERLAP, overlap)
                     R.rattn_tune(R.TUNE_UNIT_ORDER, order)

@@ -302,8 +302,11 @@ typedef enum rattn_knob {
                                     second chunk state; 1 when the backward will read them all), 1, 2 */
   RATTN_TUNE_OVERLAP = 1,        /* 1 (default): the main kernel starts under the chunk-state kernel
                                     (programmatic dependent launch); 0: strictly one after the other */
-  RATTN_TUNE_UNIT_ORDER = 2,     /* 0 (default): units that read no stored state first, then heaviest first;
-                                    1: heaviest first throughout */
+  RATTN_TUNE_UNIT_ORDER = 2,     /* order in which the persistent forward kernel hands out its work units:
+                                    0 (default) automatic; 1 units that read no stored state first (they can run
+                                    under the chunk-state kernel), then heaviest first; 2 heaviest first
+                                    throughout; 3 the same, dealt round-robin instead of drawn from a counter.
+                                    Automatic = 1 when the state kernel leaves at least half of the SMs free. */
   RATTN_TUNE_GRID = 3            /* CTAs of the persistent forward kernel: 0 (default) = one per SM */
 } rattn_knob;
 int rattn_tune(int knob, int value);

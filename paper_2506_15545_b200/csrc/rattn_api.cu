@@ -439,7 +439,7 @@ int rattn_debug_withhold_arrival(int on) {
 #endif
 
 int rattn_tune(int knob, int value) {
-  static const int lo[4] = {0, 0, 0, 0}, hi[4] = {2, 1, 1, 1 << 16};
+  static const int lo[4] = {0, 0, 0, 0}, hi[4] = {2, 1, 3, 1 << 16};
   if (knob < 0 || knob > 3 || value < lo[knob] || value > hi[knob]) return RATTN_ERR_BAD_ARG;
   return g_tuning[knob].exchange(value, std::memory_order_relaxed);
 }

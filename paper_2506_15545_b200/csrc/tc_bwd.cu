@@ -90,10 +90,26 @@ tc_bwd_prep_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat16* __
     acc_s[e] = 0.f;
     acc_r[e] = 0.f;
   }
+  // The kernel is a pure stream (three tensors in, two out), so what matters is how many loads are in
+  // flight: the next row's three loads are issued before the current row is worked on.
+  const uint4 zero4 = make_uint4(0, 0, 0, 0);
+  uint4 us_n = zero4, ur_n = zero4, gy_n = zero4;
+  auto issue = [&](int rr) {
+    const int t = t0 + rr;
+    if (rr < ROWS_PER_CTA && t < T) {
+      const size_t row = bq * T + t;
+      us_n = *reinterpret_cast<const uint4*>(o_s + row * 128 + 8 * l16);
+      ur_n = *reinterpret_cast<const uint4*>(o_r + row * 128 + 8 * l16);
+      gy_n = *reinterpret_cast<const uint4*>(dy + row * 128 + 8 * l16);
+    }
+  };
+  issue(2 * warp + sub);
 #pragma unroll 1
   for (int rr = 2 * warp + sub; rr < ROWS_PER_CTA; rr += 16) {
     const int t = t0 + rr;
     const size_t prow = bq * t_pad + t;
+    const uint4 us = us_n, ur = ur_n, gy = gy_n;
+    issue(rr + 16);
     if (t >= T) {                                  // padding: statistics that make every weight zero
       if (l16 == 0) {
         lse2p[prow] = INFINITY;
@@ -102,9 +118,6 @@ tc_bwd_prep_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat16* __
       continue;
     }
     const size_t row = bq * T + t;
-    const uint4 us = *reinterpret_cast<const uint4*>(o_s + row * 128 + 8 * l16);
-    const uint4 ur = *reinterpret_cast<const uint4*>(o_r + row * 128 + 8 * l16);
-    const uint4 gy = *reinterpret_cast<const uint4*>(dy + row * 128 + 8 * l16);
     float vs[8], vr[8], g[8];
     {
       const __nv_bfloat162* ps = reinterpret_cast<const __nv_bfloat162*>(&us);

@@ -74,6 +74,7 @@ struct FArgs {
 
 struct FMaps {
   CUtensorMap q, k, v, st, out;
+  CUtensorMap o_swa, o_rla;   // training mode: the un-normalised branch outputs, [B*H_q, T, 128] bf16
 };
 
 // What one unit consists of; every role derives the same plan from the unit index.
@@ -406,6 +407,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     if (u < 0) break;
     const Unit un = make_unit(a, u);
     if (un.t[0] < 0) continue;
+    TL(X, 1000 + u);
     const int kv0 = kv_count;
     kv_count += un.n;
     const int tX = X ? un.t[1] : un.t[0], i0 = X ? un.i0[1] : un.i0[0], i1 = X ? un.i1[1] : un.i1[0];
@@ -521,15 +523,19 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
       inv_q = feature_map_row_any<false>(sQ, r, a.phi);
       fence_proxy_async_smem();
       mbar_arrive(&bars->phiq_ready[X]);
+      TL(X, 503);
       // this tile's own chunk: A -> last stream position, B -> its last active position
       const int ic = (X == 0) ? un.n - 1 : un.i1[1];
       feature_map_row_any<true>(smem + F_OFF_KV + ((kv0 + ic) & 1) * 2 * TILE_BYTES, r, a.phi);
       fence_proxy_async_smem();
       mbar_arrive(&bars->phik_ready[X]);
+      TL(X, 504);
     }
 
     // ---- park the normalised window output (Section 3.2, first norm) in registers ---------
+    TL(X, 500);
     WAIT_OR_RETURN(bars->o_ready[X], cntO & 1);
+    TL(X, 501);
     ++cntO;
     tc_fence_after();
     const float inv_l = 1.f / l;
@@ -555,6 +561,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     }
 
     // ---- residual branch, second part -------------------------------------------------------
+    TL(X, 502);
     if (rlaX) {
       tc_fence_before();
       mbar_arrive(&bars->stash_done[X]);
@@ -599,25 +606,39 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
 
     // ---- Section 3.2: gains, sum; outputs leave through the tile's Q buffer ---------------
     const size_t tile_row0 = (size_t)un.bh_q * a.T + q0;
+    TL(X, 530);
     const float rms_s = ms * rs;                                       // sqrt(mean square + eps)
     if (a.o_swa) {
-      // training mode: un-normalised branch outputs (bf16), 32 columns at a time, staged so
-      // that each warp writes whole 64-byte segments of its own 32 rows
+      // training mode: the un-normalised branch outputs (bf16) for the backward.  Each leaves as one
+      // whole tile: every thread writes its row into the tile's Q buffer (phi(Q_X) has been consumed),
+      // swizzled like a loaded tile, and one TMA store sends it off -- plain 16-byte global stores
+      // from 128 threads kept the load/store unit busy under the other group's feature maps.
       unsigned char* stage = sQ;
       if (rlaX) group_sync(X);
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        float x[32];
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&stash[16 * c + e]));
-          x[2 * e] = f.x * rms_s;
-          x[2 * e + 1] = f.y * rms_s;
+        for (int e = 0; e < 4; ++e) {
+          uint32_t wv[4];
+#pragma unroll
+          for (int k2 = 0; k2 < 4; ++k2) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&stash[16 * c + 4 * e + k2]));
+            wv[k2] = pack_bf16(f.x * rms_s, f.y * rms_s);
+          }
+          *reinterpret_cast<uint4*>(stage + swz(r, 4 * c + e)) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
         }
-        __syncwarp();
-        stage_bf16_block(stage, r, x);
-        __syncwarp();
-        flush_bf16_block(stage, r, a.o_swa + tile_row0 * 128 + 32 * c, a.T - q0);
+      }
+      fence_proxy_async_smem();
+      group_sync(X);
+      if (r == 0) {
+        store_tile(&tm.o_swa, stage, q0, un.bh_q);
+        tma_store_commit();
+        tma_store_wait_read();
+      }
+      group_sync(X);
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        float x[32];
         if (rlaX) {
           tmem_ld32(tO + 32 * c, x);
           tmem_wait_ld();
@@ -627,13 +648,22 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
 #pragma unroll
           for (int e = 0; e < 32; ++e) x[e] = 0.f;
         }
-        __syncwarp();
-        stage_bf16_block(stage, r, x);
-        __syncwarp();
-        flush_bf16_block(stage, r, a.o_rla + tile_row0 * 128 + 32 * c, a.T - q0);
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          *reinterpret_cast<uint4*>(stage + swz(r, 4 * c + e)) =
+              make_uint4(pack_bf16(x[8 * e], x[8 * e + 1]), pack_bf16(x[8 * e + 2], x[8 * e + 3]),
+                         pack_bf16(x[8 * e + 4], x[8 * e + 5]), pack_bf16(x[8 * e + 6], x[8 * e + 7]));
+      }
+      fence_proxy_async_smem();
+      group_sync(X);
+      if (r == 0) {
+        store_tile(&tm.o_rla, stage, q0, un.bh_q);
+        tma_store_commit();
+        tma_store_wait_read();
       }
       group_sync(X);
     }
+    TL(X, 535);
     const float* gs = a.gamma_swa ? a.gamma_swa + (size_t)un.h * 128 : nullptr;
     const float* gr = a.gamma_rla ? a.gamma_rla + (size_t)un.h * 128 : nullptr;
     // y leaves through the state tile's buffer (free once this unit's residual products are done;
@@ -705,6 +735,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     }
     if (t < a.T && a.lse) a.lse[(size_t)un.bh_q * a.T + t] = (m_ref + log2f(l)) * 0.6931471805599453f;
     mbar_arrive(&bars->y_done[X]);         // the staging buffer may take the next state tile
+    TL(X, 540);
   }
   return true;
 }
@@ -754,6 +785,8 @@ tc_fwd2_kernel(const __grid_constant__ FMaps tm, FArgs a) {
     prefetch_tensormap(&tm.v);
     prefetch_tensormap(&tm.st);
     prefetch_tensormap(&tm.out);
+    prefetch_tensormap(&tm.o_swa);
+    prefetch_tensormap(&tm.o_rla);
   }
   tc_fence_before();
   __syncthreads();
@@ -799,8 +832,15 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_sta
   FMaps tm;
   if (!make_map(&tm.q, a.q, a.T, (uint64_t)a.B * a.H_q) || !make_map(&tm.k, a.k, a.Tk, (uint64_t)a.B * a.H_kv) ||
       !make_map(&tm.v, a.v, a.Tk, (uint64_t)a.B * a.H_kv) || !make_map(&tm.out, a.out, a.T, (uint64_t)a.B * a.H_q) ||
-      !make_state_map(&tm.st, a.chunk_state, a.k, (uint64_t)a.B * a.H_kv * a.n_chunks))
+      !make_state_map(&tm.st, a.chunk_state, a.k, (uint64_t)a.B * a.H_kv * a.n_chunks) ||
+      !make_map(&tm.o_swa, a.o_swa ? (const void*)a.o_swa : a.out, a.T, (uint64_t)a.B * a.H_q) ||
+      !make_map(&tm.o_rla, a.o_rla ? (const void*)a.o_rla : a.out, a.T, (uint64_t)a.B * a.H_q))
     return cudaErrorInvalidValue;
+  int dev = 0, n_sm = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
   FArgs t;
   t.lse = a.lse;
   t.o_swa = reinterpret_cast<__nv_bfloat16*>(a.o_swa);   // the fp32-sized regions of the workspace hold bf16 here
@@ -818,18 +858,16 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_sta
   t.seq_lens = a.seq_lens;
   // pairs p with 2p - w/128 <= 0 read no stored state (a resumed sequence has none: every tile reads one)
   t.n_stateless = 0;
-  if (a.mode == RATTN_MODE_RATTN && after_states && !a.state_in && tuning(RATTN_TUNE_UNIT_ORDER) == 0) {
+  // ... which pays when the chunk-state kernel leaves many SMs free for them (it runs one CTA per K/V head)
+  const int order = tuning(RATTN_TUNE_UNIT_ORDER);
+  const bool stateless_first = order == 1 || (order == 0 && 2 * a.B * a.H_kv <= n_sm);
+  if (a.mode == RATTN_MODE_RATTN && after_states && !a.state_in && stateless_first) {
     t.n_stateless = (a.w / TILE) / 2 + 1;
     if (t.n_stateless > t.n_pairs) t.n_stateless = t.n_pairs;
   }
   t.wait_for_states = after_states ? 1 : 0;
   t.debug_skip_arrive = debug_skip_arrive();
-  t.work_counter = a.status ? a.status + 2 : nullptr;
-  int dev = 0, n_sm = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-  if (e != cudaSuccess) return e;
+  t.work_counter = (a.status && order != 3) ? a.status + 2 : nullptr;
   e = cudaFuncSetAttribute(tc_fwd2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, F_SMEM);
   if (e != cudaSuccess) return e;
   if (tuning(RATTN_TUNE_GRID) > 0 && tuning(RATTN_TUNE_GRID) < n_sm) n_sm = tuning(RATTN_TUNE_GRID);
