@@ -31,7 +31,8 @@ __host__ __device__ constexpr uint32_t kstep_mn(int k) { return (uint32_t)((k * 
 __device__ __forceinline__ uint64_t kmajor_desc(uint32_t base, int kstep) { return kmajor_base(base) + kstep_k(kstep, HALF_BYTES); }
 __device__ __forceinline__ uint64_t mnmajor_desc(uint32_t base, int kstep) { return mnmajor_base(base) + kstep_mn(kstep); }
 
-// D[128x128] (+)= A B^T-style products over a reduction of 128, 8 MMAs of K = 16.
+// D[128x128] (+)= A B^T-style products over a reduction of 128, 8 MMAs of K = 16.  (Unrolled on
+// purpose: with rolled issue loops the MMA warps, which sit on the critical path, measured 6-25 % slower.)
 __device__ __forceinline__ void mma_kk(uint32_t d, uint32_t a_base, uint32_t b_base, bool acc) {
   constexpr uint32_t idesc = instr_desc(128, 128, 0, 0);
   const uint64_t a0 = kmajor_base(a_base), b0 = kmajor_base(b_base);
@@ -357,9 +358,18 @@ __device__ __forceinline__ float feature_map_row_inplace(unsigned char* tile, in
 // phi of row r of a swizzled bf16 tile, in place, for any map.  NORMALISE = false: the softmax
 // map leaves exp(x - max) and returns 1 / sum (see feature_map_row_inplace); the element-wise
 // maps have no normalisation and return 1.
+// (The softmax map runs in its compact rolled form -- two or three passes over the row in shared
+// memory -- rather than the fully unrolled register form: the kernels that call this are larger than
+// the instruction cache, and the unrolled form alone is 16 KB of code per call site.)
 template <bool NORMALISE>
 __device__ __forceinline__ float feature_map_row_any(unsigned char* tile, int r, int phi) {
-  if (phi == RATTN_PHI_SOFTMAX) return feature_map_row_inplace<NORMALISE>(tile, r);
+  if (phi == RATTN_PHI_SOFTMAX) {
+    if (NORMALISE) {
+      feature_map_row_inplace_lr(tile, r);
+      return 1.f;
+    }
+    return feature_map_row_unnorm_inplace(tile, r);
+  }
   if (phi == RATTN_PHI_RELU) {
 #pragma unroll 4
     for (int c = 0; c < 16; ++c) {
