@@ -650,6 +650,46 @@ def run_replicas_selftest(args):
         dist.destroy_process_group()
 
 
+def run_timeline(args):
+    """Where one CTA of the forward kernel spends a work unit: the library is rebuilt with its clock
+    stamps compiled in (librattn_tl.so), one forward of the small case (B=2 of config 2; --train for
+    the training-mode forward of config 4) is run, and the stamps of CTA 7's two row groups are
+    printed as cycles since the unit began.  Stamp ids: 200+i first scores of stream position i
+    seen, 300+i row maxima done, 400+i weights handed over, 503 phi(Q) done, 504 phi(K) done,
+    501 window accumulator complete, 502 window output parked, 530 residual products complete,
+    535 residuals for the backward stored, 540 output stored."""
+    import ctypes
+    from paper_2506_15545_b200 import binding as R
+    from paper_2506_15545_b200 import build as B
+    R.LIB_PATH = B.build(timeline=True)
+    L = R.lib()
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    wl = W.C4 if args.train else W.C2.replace(B=2)
+    q, k, v = W.make_qkv(wl, dev)
+    ws = R.alloc_workspace(q, k, wl.w, R.MODE_RATTN, R.FLAG_SAVE_RESIDUALS if args.train else 0)
+    out = torch.empty_like(q)
+    buf = (ctypes.c_ulonglong * 8192)()
+    n = (ctypes.c_int * 4)()
+    for _ in range(3):
+        R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws, out=out, save_residuals=args.train)
+        torch.cuda.synchronize()
+        L.rattn_timeline_read(buf, n)
+    units = []
+    for role in range(2):
+        ev = [(int(buf[role * 2048 + 2 * i]), int(buf[role * 2048 + 2 * i + 1])) for i in range(n[role])]
+        start, marks = None, {}
+        for e, t in ev:
+            if e >= 1000:
+                start, marks = t, {"unit": e - 1000}
+            elif start is not None:
+                marks[e] = t - start
+                if e == 540:
+                    units.append({"row_group": "AB"[role], **marks})
+    print(json.dumps({"case": "timeline", "workload": workload_name(wl), "training_mode": bool(args.train),
+                      "units_of_cta_7": units}))
+
+
 def run_sweep(args):
     """The forward's tuning parameters swept on config 2 and on the paper's own head shapes
     (Table 1: 16 query / 4 K/V heads, 40 / 8), one JSON line per point: stored-state stride m,
@@ -700,7 +740,8 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference", "replicas-selftest"])
-    ap.add_argument("--case", default=None, choices=["fwd", "train", "decode"],
+    ap.add_argument("--train", action="store_true", help="with --case timeline: the training-mode forward of config 4")
+    ap.add_argument("--case", default=None, choices=["fwd", "train", "decode", "timeline"],
                     help="run one small case (for profiler captures) instead of the benchmark")
     ap.add_argument("--sweep", action="store_true",
                     help="sweep the forward's tuning parameters (stored-state stride, overlap, unit order)")
@@ -720,6 +761,9 @@ def main():
         return
     if args.all_configs:
         run_all_configs(args)
+        return
+    if args.case == "timeline":
+        run_timeline(args)
         return
     if args.case:
         run_case(args)

@@ -18,6 +18,7 @@ CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(ROOT, "_build")
 LIB = os.path.join(HERE, "librattn.so")
 LIB_DEBUG = os.path.join(HERE, "librattn_dbg.so")      # same sources with -DRATTN_DEBUG_KNOBS (include/rattn_debug.h)
+LIB_TIMELINE = os.path.join(HERE, "librattn_tl.so")    # same sources with -DRATTN_TIMELINE (bench.py --case timeline)
 
 SOURCES = ["rattn_api.cu", "generic_fwd.cu", "generic_bwd.cu", "decode.cu", "tc_fwd.cu",
            "tc_fwd2.cu", "tc_state.cu", "tc_bwd.cu", "static_scratch.cu"]
@@ -40,11 +41,13 @@ def _newest_dep_mtime() -> float:
     return max(m, os.path.getmtime(__file__))
 
 
-def _compile(src: str, verbose: bool, debug: bool = False) -> str:
-    obj = os.path.join(BUILD, src.replace(".cu", ".dbg.o" if debug else ".o"))
+def _compile(src: str, verbose: bool, debug: bool = False, timeline: bool = False) -> str:
+    obj = os.path.join(BUILD, src.replace(".cu", ".dbg.o" if debug else ".tl.o" if timeline else ".o"))
     cmd = [_nvcc(), *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
     if debug:
         cmd.insert(1, "-DRATTN_DEBUG_KNOBS")
+    if timeline:
+        cmd.insert(1, "-DRATTN_TIMELINE")
     if os.path.exists(os.path.join(CSRC, "tc_fwd.cu")):
         cmd.insert(1, "-DRATTN_HAVE_TC")
     if verbose:
@@ -58,15 +61,16 @@ def _compile(src: str, verbose: bool, debug: bool = False) -> str:
     return obj
 
 
-def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
-    """Compile every source and link librattn.so (debug: librattn_dbg.so); returns its path."""
-    lib = LIB_DEBUG if debug else LIB
+def build(force: bool = False, verbose: bool = False, debug: bool = False, timeline: bool = False) -> str:
+    """Compile every source and link librattn.so (debug: librattn_dbg.so; timeline: librattn_tl.so,
+    the forward kernel with its per-role clock stamps compiled in); returns its path."""
+    lib = LIB_DEBUG if debug else LIB_TIMELINE if timeline else LIB
     sources = [s for s in SOURCES if os.path.exists(os.path.join(CSRC, s))]
     if not force and os.path.exists(lib) and os.path.getmtime(lib) >= _newest_dep_mtime():
         return lib
     os.makedirs(BUILD, exist_ok=True)
     with concurrent.futures.ThreadPoolExecutor(max_workers=len(sources)) as ex:
-        objs = list(ex.map(lambda s: _compile(s, verbose, debug), sources))
+        objs = list(ex.map(lambda s: _compile(s, verbose, debug, timeline), sources))
     cmd = [_nvcc(), "-shared", "-o", lib, *objs, "-cudart", "static"]
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:

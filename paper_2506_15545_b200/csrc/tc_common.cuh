@@ -358,12 +358,15 @@ __device__ __forceinline__ float feature_map_row_inplace(unsigned char* tile, in
 // phi of row r of a swizzled bf16 tile, in place, for any map.  NORMALISE = false: the softmax
 // map leaves exp(x - max) and returns 1 / sum (see feature_map_row_inplace); the element-wise
 // maps have no normalisation and return 1.
-// (The softmax map runs in its compact rolled form -- two or three passes over the row in shared
-// memory -- rather than the fully unrolled register form: the kernels that call this are larger than
-// the instruction cache, and the unrolled form alone is 16 KB of code per call site.)
+// The softmax map comes in two forms: fully unrolled with the row in 128 registers (one read and one
+// write of shared memory, but 16 KB of code per call site) and compact (rolled loops, two or three
+// passes over the row in shared memory, twice the cycles).  The kernels that call this are larger
+// than the instruction cache; a caller whose launch executes much other code (the training-mode
+// forward) is faster with the compact form, the others with the unrolled one.
 template <bool NORMALISE>
-__device__ __forceinline__ float feature_map_row_any(unsigned char* tile, int r, int phi) {
+__device__ __forceinline__ float feature_map_row_any(unsigned char* tile, int r, int phi, bool compact = false) {
   if (phi == RATTN_PHI_SOFTMAX) {
+    if (!compact) return feature_map_row_inplace<NORMALISE>(tile, r);
     if (NORMALISE) {
       feature_map_row_inplace_lr(tile, r);
       return 1.f;

@@ -520,13 +520,13 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     if (rlaX) {
       // phi(Q_X) without its normalisation: everything that follows is linear in this row,
       // so 1/sum is applied to the accumulator row at the end
-      inv_q = feature_map_row_any<false>(sQ, r, a.phi);
+      inv_q = feature_map_row_any<false>(sQ, r, a.phi, a.o_swa != nullptr);
       fence_proxy_async_smem();
       mbar_arrive(&bars->phiq_ready[X]);
       TL(X, 503);
       // this tile's own chunk: A -> last stream position, B -> its last active position
       const int ic = (X == 0) ? un.n - 1 : un.i1[1];
-      feature_map_row_any<true>(smem + F_OFF_KV + ((kv0 + ic) & 1) * 2 * TILE_BYTES, r, a.phi);
+      feature_map_row_any<true>(smem + F_OFF_KV + ((kv0 + ic) & 1) * 2 * TILE_BYTES, r, a.phi, a.o_swa != nullptr);
       fence_proxy_async_smem();
       mbar_arrive(&bars->phik_ready[X]);
       TL(X, 504);
