@@ -77,6 +77,12 @@ typedef enum rattn_feature_map {
  * Parameter block of the *_ex entry points.  Zero-initialise it, then fill in.
  *   dtype      I/O element type of q,k,v,out,dout,dq,dk,dv and the decode ring.
  *              Accumulation, softmax, feature map, norms and the state are fp32.
+ *              Value range on the bf16 tensor-core path: the attention weights and v enter
+ *              the tensor cores as fp16, so |v| above 65504 saturates to 65504, |v| below
+ *              6.1e-5 (2^-14) keeps fewer than 11 bits and |v| below 6e-8 reads as zero.
+ *              Nothing detects this.  Both norms cancel a common factor of v, so a caller
+ *              whose values sit outside roughly [1e-3, 1e4] rescales v (and eps by the
+ *              square of the factor) or sets RATTN_FLAG_FORCE_GENERIC.
  *   scale      multiplies the SWA logits q.k only (the paper writes none: 1.0).  The
  *              tensor-core kernels need scale > 0 and return RATTN_ERR_UNSUPPORTED
  *              otherwise; the portable kernels (RATTN_FLAG_FORCE_GENERIC) take any finite

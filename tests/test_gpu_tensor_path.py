@@ -215,3 +215,27 @@ def test_paper_head_shapes(Hq, Hkv):
     errs = run_bwd(wl)
     for name, e in errs.items():
         assert e <= GRAD_TOL, (name, e, errs)
+
+
+@pytest.mark.parametrize("v_scale,clip", [(1.5e4, 6.0e4), (2.0 ** -9, None)])
+def test_tensor_forward_value_range(v_scale, clip):
+    """The tensor-core kernels read v through fp16 (range 6.1e-5 .. 65504 at full precision).
+    Values up to 6e4 in magnitude, and values around 2^-9 (whose tails reach fp16's subnormals),
+    still give the oracle's output: both norms divide the common scale of v out again."""
+    wl = small("tcv", 1, 4, 2, 896, 128, 256, "bf16", 4700, unit=True)
+    q, k, v = W.make_qkv(wl)
+    v = v.float() * v_scale
+    if clip is not None:
+        v = v.clamp(-clip, clip)
+        assert v.abs().max() >= 0.99 * clip
+    v = v.to(torch.bfloat16)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    ws = R.alloc_workspace(qd, kd, wl.w)
+    y = R.rattn_forward_ex(qd, kd, vd, wl.w, scale=wl.scale, workspace=ws)
+    torch.cuda.synchronize()
+    assert R.rattn_read_status(ws) == 0
+    eps = 1e-6 * v_scale * v_scale      # keeps eps in the same proportion to mean(o^2)
+    y2 = R.rattn_forward_ex(qd, kd, vd, wl.w, scale=wl.scale, workspace=ws, eps=eps)
+    ref = O.forward(np64(q), np64(k), np64(v), wl.w, wl.scale, eps, None, None, R.MODE_RATTN)
+    check(y2, ref, "bf16", f"v scale {v_scale}")
+    assert torch.isfinite(y.float()).all()
