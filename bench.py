@@ -523,6 +523,25 @@ def run_case(args):
         print(json.dumps({"case": args.case, "workload": workload_name(wl), "ms": ms,
                           "tflops": fl / (ms * 1e-3) / 1e12,
                           "kernels_ms_per_launch": {n: t / c for n, (c, t) in km.items() if c}}))
+    elif args.case == "prologue":
+        # qk-norm + rotary embedding over config 4's q and k (2 x 134 MB, larger than L2), then its gradient
+        wl = W.C4
+        q, k, _ = W.make_qkv(wl, dev)
+        gq = torch.ones(wl.d, device=dev)
+        qo, ko = torch.empty_like(q), torch.empty_like(k)
+        nbytes = 2 * (q.numel() + k.numel()) * q.element_size()
+        ms_f = timed(lambda: R.rattn_qk_prologue(q, k, q_gain=gq, k_gain=gq), args.steps, args.warmup, sync)
+        wsp = torch.empty(R.rattn_qk_prologue_workspace_bytes(wl.B, wl.H_q, wl.H_kv, wl.T, wl.d), dtype=torch.uint8,
+                          device=dev)
+        ms_b = timed(lambda: R.rattn_qk_prologue_backward(q, k, qo, ko, q_gain=gq, k_gain=gq, workspace=wsp),
+                     args.steps, args.warmup, sync)
+        hbm = peaks()["hbm"]
+        print(json.dumps({"case": "prologue", "workload": workload_name(wl),
+                          "forward": {"ms": ms_f, "gb_per_s": nbytes / ms_f / 1e6, "frac_of_hbm_peak": nbytes / ms_f / 1e6 / hbm},
+                          "backward": {"ms": ms_b, "gb_per_s": 1.5 * nbytes / ms_b / 1e6,
+                                       "frac_of_hbm_peak": 1.5 * nbytes / ms_b / 1e6 / hbm},
+                          "bytes": "forward: q, k read once and written once; backward: q, k and their output "
+                                   "gradients read, input gradients written"}))
     else:
         c5 = W.C5
         kr = torch.randn(c5.B, c5.H_kv, c5.w, c5.d, device=dev).to(torch.bfloat16)
@@ -741,7 +760,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference", "replicas-selftest"])
     ap.add_argument("--train", action="store_true", help="with --case timeline: the training-mode forward of config 4")
-    ap.add_argument("--case", default=None, choices=["fwd", "train", "decode", "timeline"],
+    ap.add_argument("--case", default=None, choices=["fwd", "train", "decode", "timeline", "prologue"],
                     help="run one small case (for profiler captures) instead of the benchmark")
     ap.add_argument("--sweep", action="store_true",
                     help="sweep the forward's tuning parameters (stored-state stride, overlap, unit order)")

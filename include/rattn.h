@@ -320,6 +320,60 @@ int rattn_tune(int knob, int value);
 /* 1 when the tensor-core (tcgen05) forward would be chosen for these sizes. */
 int rattn_uses_tensor_path(int d, int w, int dtype, int mode, unsigned flags);
 
+/*
+ * What the paper's models apply to q and k between the projections and the operator, as one
+ * pass over both tensors (one read and one write of each element instead of two of each for a
+ * norm kernel followed by a rotation kernel):
+ *
+ *   qk-norm (Table 1, "qk-norm: yes"):  n = x / sqrt(mean(x^2) + eps) * gain   per head vector,
+ *           gain fp32 [d], one for the queries and one for the keys (NULL = ones);
+ *   rotary embedding (Section 4, "Model Setup": local layers, theta = 5e5; global layers none):
+ *           features i and i + d/2 (i < d/2) of the token at sequence position p are rotated by
+ *           the angle p * theta^(-2i/d):
+ *               y_i       = n_i cos - n_{i+d/2} sin,     y_{i+d/2} = n_{i+d/2} cos + n_i sin.
+ *
+ *   q, k           inputs, [B,H_q,T,d] and [B,H_kv,T,d], element type dtype.  k (and k_out) may be
+ *                  NULL with H_kv = 0 to transform one tensor only.
+ *   q_out, k_out   results, same shapes and type; each may be the same pointer as its input.
+ *   theta          rotation base; theta <= 0 skips the rotation (global layers).
+ *   pos0, pos      row t of batch entry b sits at position (pos ? pos[b] : pos0) + t; pos is an
+ *                  optional device int32 [B] (decoding a batch whose entries have different lengths).
+ *                  Angles are formed in fp64 and reduced before the fp32 sine and cosine, so
+ *                  positions up to 2^31 keep full fp32 accuracy.
+ *   d              64 or 128.  Arithmetic is fp32; sums over a row are taken in a fixed order.
+ *
+ * rattn_qk_prologue_backward: given the same inputs (the tensors as they were BEFORE the forward
+ * pass, so not after an in-place call) and the gradients dq_out, dk_out with respect to the
+ * results, writes the gradients dq, dk with respect to q, k (each may alias its dq_out / dk_out)
+ * and, where the pointers are not NULL, the gain gradients dq_gain, dk_gain (fp32 [d],
+ * overwritten).  Gain gradients need a workspace of rattn_qk_prologue_workspace_bytes() bytes
+ * (256-byte aligned) for per-CTA partial sums, which a second kernel adds in a fixed order: the
+ * result does not depend on scheduling.
+ *
+ * Errors as for the other entry points; nothing is launched when a check fails.
+ */
+typedef struct rattn_qk_params {
+  const void* q;
+  const void* k;
+  void* q_out;
+  void* k_out;
+  const float* q_gain;
+  const float* k_gain;
+  int32_t B, H_q, H_kv, T, d;
+  int32_t dtype;                 /* rattn_dtype */
+  float eps;
+  float theta;
+  int32_t pos0;
+  int32_t reserved;
+  const int32_t* pos;
+} rattn_qk_params;
+
+int rattn_qk_prologue(const rattn_qk_params* p, void* stream);
+int rattn_qk_prologue_backward(const rattn_qk_params* p, const void* dq_out, const void* dk_out,
+                               void* dq, void* dk, float* dq_gain, float* dk_gain,
+                               void* workspace, size_t workspace_bytes, void* stream);
+size_t rattn_qk_prologue_workspace_bytes(int B, int H_q, int H_kv, int T, int d);
+
 #ifdef __cplusplus
 }
 #endif

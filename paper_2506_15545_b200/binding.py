@@ -26,6 +26,7 @@ EXPORTS = (
     "rattn_read_status", "rattn_strerror", "rattn_last_cuda_error", "rattn_launch_count",
     "rattn_uses_tensor_path", "rattn_timing_enable", "rattn_timing_read",
     "rattn_forward_static", "rattn_static_status", "rattn_tune",
+    "rattn_qk_prologue", "rattn_qk_prologue_backward", "rattn_qk_prologue_workspace_bytes",
 )
 TUNE_STATE_STRIDE, TUNE_OVERLAP, TUNE_UNIT_ORDER, TUNE_GRID = 0, 1, 2, 3
 
@@ -49,6 +50,17 @@ class RattnParams(ctypes.Structure):
         ("state_in", ctypes.c_void_p), ("k_ring_in", ctypes.c_void_p), ("v_ring_in", ctypes.c_void_p),
         ("pos0", ctypes.c_int32), ("reserved", ctypes.c_int32),
         ("seq_lens", ctypes.c_void_p), ("pos", ctypes.c_void_p),
+    ]
+
+
+class RattnQkParams(ctypes.Structure):
+    _fields_ = [
+        ("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("q_out", ctypes.c_void_p), ("k_out", ctypes.c_void_p),
+        ("q_gain", ctypes.c_void_p), ("k_gain", ctypes.c_void_p),
+        ("B", ctypes.c_int32), ("H_q", ctypes.c_int32), ("H_kv", ctypes.c_int32),
+        ("T", ctypes.c_int32), ("d", ctypes.c_int32), ("dtype", ctypes.c_int32),
+        ("eps", ctypes.c_float), ("theta", ctypes.c_float),
+        ("pos0", ctypes.c_int32), ("reserved", ctypes.c_int32), ("pos", ctypes.c_void_p),
     ]
 
 
@@ -109,6 +121,13 @@ def lib() -> ctypes.CDLL:
     L.rattn_static_status.restype = ci
     L.rattn_tune.argtypes = [ci, ci]
     L.rattn_tune.restype = ci
+    L.rattn_qk_prologue.argtypes = [ctypes.POINTER(RattnQkParams), vp]
+    L.rattn_qk_prologue.restype = ci
+    L.rattn_qk_prologue_backward.argtypes = [ctypes.POINTER(RattnQkParams), vp, vp, vp, vp, vp, vp, vp,
+                                             ctypes.c_size_t, vp]
+    L.rattn_qk_prologue_backward.restype = ci
+    L.rattn_qk_prologue_workspace_bytes.argtypes = [ci, ci, ci, ci, ci]
+    L.rattn_qk_prologue_workspace_bytes.restype = ctypes.c_size_t
     L.rattn_timing_enable.argtypes = [ci]
     L.rattn_timing_enable.restype = ci
     L.rattn_timing_read.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
@@ -331,3 +350,56 @@ def rattn_timing_read() -> dict:
         name, n, ms = line.rsplit(" ", 2)
         out[name] = (int(n), float(ms))
     return out
+
+
+def _qk_params(q, k, q_out, k_out, q_gain, k_gain, theta, eps, pos0, pos):
+    p = RattnQkParams()
+    _dense(q, k, q_out, k_out, q_gain, k_gain, pos)
+    p.q, p.q_out = q.data_ptr(), None if q_out is None else q_out.data_ptr()
+    p.B, p.H_q, p.T, p.d = q.shape
+    if k is not None:
+        p.k, p.k_out = k.data_ptr(), None if k_out is None else k_out.data_ptr()
+        p.H_kv = k.shape[1]
+    p.q_gain = None if q_gain is None else q_gain.data_ptr()
+    p.k_gain = None if k_gain is None else k_gain.data_ptr()
+    p.dtype = _dtype_code(q)
+    p.eps, p.theta, p.pos0 = eps, 0.0 if theta is None else theta, pos0
+    p.pos = None if pos is None else pos.data_ptr()
+    return p
+
+
+def rattn_qk_prologue_workspace_bytes(B, H_q, H_kv, T, d) -> int:
+    return int(lib().rattn_qk_prologue_workspace_bytes(B, H_q, H_kv, T, d))
+
+
+def rattn_qk_prologue(q, k, *, q_gain=None, k_gain=None, theta=5.0e5, eps=1e-6, pos0=0, pos=None,
+                      inplace=False, stream=None):
+    """rattn_qk_prologue: qk-norm then rotary embedding of q [B,H_q,T,d] and k [B,H_kv,T,d] (k may be
+    None).  theta None or <= 0: no rotation.  Returns (q_out, k_out); the inputs themselves if inplace."""
+    q_out = q if inplace else torch.empty_like(q)
+    k_out = None if k is None else (k if inplace else torch.empty_like(k))
+    p = _qk_params(q, k, q_out, k_out, q_gain, k_gain, theta, eps, pos0, pos)
+    _check(lib().rattn_qk_prologue(ctypes.byref(p), _stream(stream)), "rattn_qk_prologue")
+    return q_out, k_out
+
+
+def rattn_qk_prologue_backward(q, k, dq_out, dk_out, *, q_gain=None, k_gain=None, theta=5.0e5, eps=1e-6,
+                               pos0=0, pos=None, gain_grads=True, workspace=None, stream=None):
+    """rattn_qk_prologue_backward: gradients with respect to q, k (inputs as they were before the
+    forward pass) and, with gain_grads, to the two gains.  Returns (dq, dk, dq_gain, dk_gain)."""
+    _dense(dq_out, dk_out)
+    dq = torch.empty_like(q)
+    dk = None if k is None else torch.empty_like(k)
+    dqg = dkg = None
+    p = _qk_params(q, k, None, None, q_gain, k_gain, theta, eps, pos0, pos)
+    if gain_grads:
+        dqg = torch.empty(q.shape[-1], dtype=torch.float32, device=q.device)
+        dkg = None if k is None else torch.empty(q.shape[-1], dtype=torch.float32, device=q.device)
+        if workspace is None:
+            n = rattn_qk_prologue_workspace_bytes(p.B, p.H_q, p.H_kv, p.T, p.d)
+            workspace = torch.empty(n, dtype=torch.uint8, device=q.device)
+    nbytes = 0 if workspace is None else workspace.numel()
+    _check(lib().rattn_qk_prologue_backward(ctypes.byref(p), _ptr(dq_out), _ptr(dk_out), _ptr(dq), _ptr(dk),
+                                            _ptr(dqg), _ptr(dkg), _ptr(workspace), nbytes, _stream(stream)),
+           "rattn_qk_prologue_backward")
+    return dq, dk, dqg, dkg

@@ -157,3 +157,50 @@ def test_product_never_imports_the_oracle():
     for f in os.listdir(os.path.join(ROOT, "oracle")):
         if f.endswith(".py"):
             assert "paper_2506_15545_b200" not in open(os.path.join(ROOT, "oracle", f)).read()
+
+
+def test_qk_prologue_struct_and_argument_checks(B, tmp_path):
+    """rattn_qk_params has the binding's size and field offsets, and both prologue entry points
+    refuse bad arguments before any launch (there is no GPU here, so a launch would fail)."""
+    src = tmp_path / "qk.c"
+    src.write_text('#include "rattn.h"\n#include <stdio.h>\n#include <stddef.h>\n'
+                   'int main(void){printf("%zu %zu %zu %zu\\n", sizeof(rattn_qk_params),'
+                   'offsetof(rattn_qk_params, B), offsetof(rattn_qk_params, eps),'
+                   'offsetof(rattn_qk_params, pos));return 0;}\n')
+    exe = tmp_path / "qk"
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"),
+                           str(src), "-o", str(exe)])
+    size, off_b, off_eps, off_pos = map(int, subprocess.check_output([str(exe)]).split())
+    P = B.RattnQkParams
+    assert (size, off_b, off_eps, off_pos) == (ctypes.sizeof(P), P.B.offset, P.eps.offset, P.pos.offset)
+
+    L = B.lib()
+
+    def params(**kw):
+        p = P()
+        p.q = p.k = p.q_out = p.k_out = 0x1000
+        p.B, p.H_q, p.H_kv, p.T, p.d, p.dtype = 2, 4, 2, 64, 128, B.RATTN_BF16
+        p.eps, p.theta = 1e-6, 5.0e5
+        for k, v in kw.items():
+            setattr(p, k, v)
+        return p
+
+    cases = [(dict(B=0), -1), (dict(T=0), -1), (dict(H_kv=-1), -1), (dict(pos0=-5), -1),
+             (dict(eps=float("nan")), -1), (dict(eps=-1.0), -1), (dict(theta=float("inf")), -1),
+             (dict(d=96), -4), (dict(dtype=7), -4), (dict(q=None), -2), (dict(k=None), -2),
+             (dict(q_out=None), -2), (dict(k_out=None), -2), (dict(q=0x1008), -3), (dict(k_out=0x1004), -3),
+             (dict(q_gain=0x2004), -3), (dict(pos=0x3002), -3), (dict(B=70000), -1)]
+    for kw, code in cases:
+        assert L.rattn_qk_prologue(ctypes.byref(params(**kw)), None) == code, kw
+    assert L.rattn_qk_prologue(None, None) == -2
+    p = params()
+    assert L.rattn_qk_prologue_backward(ctypes.byref(p), None, 0x1000, 0x1000, 0x1000, None, None, None, 0, None) == -2
+    assert L.rattn_qk_prologue_backward(ctypes.byref(p), 0x1000, 0x1000, 0x1000, 0x1000, 0x4000, None, None, 0,
+                                        None) == -5
+    assert L.rattn_qk_prologue_backward(ctypes.byref(p), 0x1000, 0x1000, 0x1000, 0x1000, 0x4000, None, 0x5000, 16,
+                                        None) == -5
+    assert L.rattn_qk_prologue_backward(ctypes.byref(params(H_kv=0, k=None, k_out=None)), 0x1000, None, 0x1000, None,
+                                        None, 0x4000, None, 0, None) == -1
+    n = B.rattn_qk_prologue_workspace_bytes(4, 16, 16, 4096, 128)
+    assert n % 256 == 0 and 0 < n <= 2 * 2048 * 128 * 4 + 256
+    assert B.rattn_qk_prologue_workspace_bytes(4, 16, 16, 4096, 96) == 0
