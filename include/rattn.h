@@ -350,7 +350,10 @@ int rattn_uses_tensor_path(int d, int w, int dtype, int mode, unsigned flags);
  * (256-byte aligned) for per-CTA partial sums, which a second kernel adds in a fixed order: the
  * result does not depend on scheduling.
  *
- * Errors as for the other entry points; nothing is launched when a check fails.
+ * Errors as for the other entry points; nothing is launched when a check fails.  The kernels
+ * stage their data through shared memory with asynchronous copies and wait for them with a
+ * bound; rattn_qk_prologue_status (synchronises the stream) returns RATTN_ERR_TIMEOUT if such a
+ * wait has expired in any prologue call on the current device since it was last asked, else RATTN_OK.
  */
 typedef struct rattn_qk_params {
   const void* q;
@@ -373,6 +376,7 @@ int rattn_qk_prologue_backward(const rattn_qk_params* p, const void* dq_out, con
                                void* dq, void* dk, float* dq_gain, float* dk_gain,
                                void* workspace, size_t workspace_bytes, void* stream);
 size_t rattn_qk_prologue_workspace_bytes(int B, int H_q, int H_kv, int T, int d);
+int rattn_qk_prologue_status(void* stream);
 
 #ifdef __cplusplus
 }

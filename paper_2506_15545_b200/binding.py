@@ -26,7 +26,7 @@ EXPORTS = (
     "rattn_read_status", "rattn_strerror", "rattn_last_cuda_error", "rattn_launch_count",
     "rattn_uses_tensor_path", "rattn_timing_enable", "rattn_timing_read",
     "rattn_forward_static", "rattn_static_status", "rattn_tune",
-    "rattn_qk_prologue", "rattn_qk_prologue_backward", "rattn_qk_prologue_workspace_bytes",
+    "rattn_qk_prologue", "rattn_qk_prologue_backward", "rattn_qk_prologue_workspace_bytes", "rattn_qk_prologue_status",
 )
 TUNE_STATE_STRIDE, TUNE_OVERLAP, TUNE_UNIT_ORDER, TUNE_GRID = 0, 1, 2, 3
 
@@ -128,6 +128,8 @@ def lib() -> ctypes.CDLL:
     L.rattn_qk_prologue_backward.restype = ci
     L.rattn_qk_prologue_workspace_bytes.argtypes = [ci, ci, ci, ci, ci]
     L.rattn_qk_prologue_workspace_bytes.restype = ctypes.c_size_t
+    L.rattn_qk_prologue_status.argtypes = [vp]
+    L.rattn_qk_prologue_status.restype = ci
     L.rattn_timing_enable.argtypes = [ci]
     L.rattn_timing_enable.restype = ci
     L.rattn_timing_read.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
@@ -370,6 +372,10 @@ def _qk_params(q, k, q_out, k_out, q_gain, k_gain, theta, eps, pos0, pos):
 
 def rattn_qk_prologue_workspace_bytes(B, H_q, H_kv, T, d) -> int:
     return int(lib().rattn_qk_prologue_workspace_bytes(B, H_q, H_kv, T, d))
+
+
+def rattn_qk_prologue_status(stream=None) -> int:
+    return int(lib().rattn_qk_prologue_status(_stream(stream)))
 
 
 def rattn_qk_prologue(q, k, *, q_gain=None, k_gain=None, theta=5.0e5, eps=1e-6, pos0=0, pos=None,

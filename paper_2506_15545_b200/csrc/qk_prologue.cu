@@ -2,24 +2,27 @@
 // local layers rotate with theta = 5e5, global layers do not), and the gradient of that pass.
 //
 // Streaming kernels: every element is read once and written once, so the bound is HBM bandwidth.
-// A head vector of d features is held by d/16 neighbouring lanes, each with features
-// [8l, 8l+8) and [d/2 + 8l, d/2 + 8l + 8): the two halves of its 8 rotation pairs, one 16-byte
-// (bf16) or two 16-byte (fp32) loads per half.  A thread keeps one sequence position and walks
-// over the heads of a batch entry, so the 8 sines and cosines it needs are computed once and
-// used for every head; four heads are loaded before the first is stored, which keeps enough
-// loads in flight with inputs and outputs allowed to alias.
+// The unit of work is a chunk: the rows of one head that one CTA's threads cover (256 / (d/16)
+// consecutive positions, 8 KB of bf16), contiguous in memory.  Chunks travel global -> shared
+// -> global as bulk asynchronous copies through a ring of stages, so the bytes in flight do not
+// depend on registers or on where the warps are in their arithmetic; the threads transform a
+// chunk in place in shared memory.  A head vector of d features is held by d/16 neighbouring
+// lanes, each with features [8l, 8l+8) and [d/2 + 8l, d/2 + 8l + 8): the two halves of its 8
+// rotation pairs.  Chunks are ordered tensor, row block, head, and every CTA takes an equal
+// contiguous share of them: consecutive chunks share their positions, so a thread computes its
+// 8 sines and cosines once per row block.
 #include <cmath>
 #include <cstdint>
 
 #include "rattn_internal.h"
+#include "tc_ptx.cuh"
 
 namespace rattn {
 namespace {
 
 constexpr int QK_THREADS = 256;
-constexpr int QK_MAX_CTAS = 2048;     // bounds the partial sums of the gain gradients
-constexpr int QK_FWD_BATCH = 4;       // heads in flight per thread, forward
-constexpr int QK_BWD_BATCH = 2;       // backward (two tensors per head)
+constexpr int QK_MAX_CTAS = 1024;     // bounds the partial sums of the gain gradients
+constexpr int QK_CTAS_PER_SM = 3;
 
 struct Freqs {
   double inv[64];                     // theta^(-2i/d), i < d/2
@@ -32,29 +35,14 @@ struct QkArgs {
   const float* gain[2];
   float* partial;                     // backward: [2][n_cta][d] or null
   int H[2];
-  int B, T, S, nblk_t;
+  int B, T, nblk_t;
   float eps;
   int rotate;
   long long pos0;
   const int* pos;
 };
 
-struct Geometry {
-  int rpb, nblk_t, S, gx, gy;
-  int n_cta() const { return gx * gy; }
-};
-
-Geometry geometry(int B, int H_q, int H_kv, int T, int d) {
-  Geometry g;
-  g.rpb = QK_THREADS / (d / 16);
-  g.nblk_t = (T + g.rpb - 1) / g.rpb;
-  const int heads = H_q + H_kv;
-  g.S = heads / 8 < 1 ? 1 : heads / 8 > 8 ? 8 : heads / 8;
-  g.gy = B * g.S;
-  const int cap = QK_MAX_CTAS / g.gy < 1 ? 1 : QK_MAX_CTAS / g.gy;
-  g.gx = g.nblk_t < cap ? g.nblk_t : cap;
-  return g;
-}
+__device__ int g_qk_status;           // RATTN_ERR_TIMEOUT once a bounded wait has expired
 
 template <typename T> struct Io;
 template <> struct Io<__nv_bfloat16> {
@@ -130,167 +118,239 @@ __device__ __forceinline__ void load_gain(const float* gain, int lo_first, int h
   }
 }
 
-template <typename T, int D>
-__global__ void __launch_bounds__(QK_THREADS, 2) qk_prologue_kernel(const __grid_constant__ QkArgs a, const __grid_constant__ Freqs f) {
-  constexpr int LPR = D / 16, RPB = QK_THREADS / LPR, U = QK_FWD_BATCH;
-  const int l = threadIdx.x % LPR, row = threadIdx.x / LPR;
-  const int b = blockIdx.y / a.S, slice = blockIdx.y % a.S;
-  const long long p0 = a.pos ? (long long)a.pos[b] : a.pos0;
-
-  for (int tb = blockIdx.x; tb < a.nblk_t; tb += gridDim.x) {
-    const int t = tb * RPB + row;
-    const bool live = t < a.T;
-    float c[8], s[8];
-    rotation(f, 8 * l, p0 + t, a.rotate, c, s);
-
-#pragma unroll 1
-    for (int which = 0; which < 2; ++which) {
-      const int H = a.H[which];
-      if (H == 0) continue;
-      float g_lo[8], g_hi[8];
-      load_gain(a.gain[which], 8 * l, D / 2, g_lo, g_hi);
-      const void* x = a.x[which];
-      void* y = a.y[which];
-#pragma unroll 1
-      for (int h0 = slice; h0 < H; h0 += U * a.S) {
-        float lo[U][8], hi[U][8];
-        size_t at[U];
-        bool on[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-          const int h = h0 + u * a.S;
-          on[u] = live && h < H;
-          at[u] = (((size_t)b * H + (on[u] ? h : 0)) * a.T + (live ? t : 0)) * D + 8 * l;
-          if (on[u]) {
-            Io<T>::load(x, at[u], lo[u]);
-            Io<T>::load(x, at[u] + D / 2, hi[u]);
-          } else {
-            zero8(lo[u]);
-            zero8(hi[u]);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-          float ss = 0.f;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) ss += lo[u][j] * lo[u][j] + hi[u][j] * hi[u][j];
-          ss = row_sum<LPR>(ss);
-          const float r = rsqrtf(ss * (1.f / D) + a.eps);
-          float o_lo[8], o_hi[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            const float n_lo = lo[u][j] * r * g_lo[j], n_hi = hi[u][j] * r * g_hi[j];
-            o_lo[j] = n_lo * c[j] - n_hi * s[j];
-            o_hi[j] = n_hi * c[j] + n_lo * s[j];
-          }
-          if (on[u]) {
-            Io<T>::store(y, at[u], o_lo);
-            Io<T>::store(y, at[u] + D / 2, o_hi);
-          }
-        }
-      }
-    }
-  }
+// single-thread forms of the bulk copies (one issuing thread per CTA, once per chunk)
+__device__ __forceinline__ void expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(ptx::smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(ptx::smem_u32(dst)), "l"(src), "r"(bytes), "r"(ptx::smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* dst, const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+               ::"l"(dst), "r"(ptx::smem_u32(src)), "r"(bytes)
+               : "memory");
+}
+// all but the newest of this thread's store groups have finished reading shared memory
+__device__ __forceinline__ void store_wait_read_but_one() {
+  asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
 }
 
-template <typename T, int D>
-__global__ void __launch_bounds__(QK_THREADS, 2) qk_prologue_bwd_kernel(const __grid_constant__ QkArgs a, const __grid_constant__ Freqs f) {
-  constexpr int LPR = D / 16, RPB = QK_THREADS / LPR, U = QK_BWD_BATCH;
-  __shared__ float red[RPB][D];
-  __shared__ __align__(16) float gain_s[D];       // read at each use: the registers go to the loads in flight
-  const int l = threadIdx.x % LPR, row = threadIdx.x / LPR;
-  const int b = blockIdx.y / a.S, slice = blockIdx.y % a.S;
-  const long long p0 = a.pos ? (long long)a.pos[b] : a.pos0;
-  const int cta = blockIdx.y * gridDim.x + blockIdx.x, n_cta = gridDim.x * gridDim.y;
+template <typename T, bool BWD> struct Ring {
+  static constexpr int kChunk = 4096 * (int)sizeof(T);           // rows per CTA x row bytes, any d
+  static constexpr int kBufs = BWD ? 2 : 1;                      // backward: the input and its output gradient
+  static constexpr int kStages = BWD ? (sizeof(T) == 2 ? 4 : 3) : (sizeof(T) == 2 ? 8 : 4);
+  static constexpr int kRed = BWD ? 4096 * 4 : 0;                // backward: block reduction of the gain gradients
+  static constexpr int kBytes = kStages * kBufs * kChunk + kRed + 128;
+};
 
-  // q, then k: one set of gain-gradient accumulators alive at a time
-#pragma unroll 1
-  for (int which = 0; which < 2; ++which) {
-    const int H = a.H[which];
-    float acc[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) acc[i] = 0.f;
-    __syncthreads();
-    if (threadIdx.x < D) gain_s[threadIdx.x] = a.gain[which] ? a.gain[which][threadIdx.x] : 1.f;
-    __syncthreads();
-    const float* g_lo = gain_s + 8 * l;
-    const float* g_hi = gain_s + D / 2 + 8 * l;
-    const void* x = a.x[which];
-    const void* dy = a.dy[which];
-    void* dx = a.y[which];
+// One chunk: tensor `which`, batch entry b, row block tb, head h; chunks are numbered tensor,
+// batch entry, row block, head.  A cursor is set once and then stepped.
+struct Chunk {
+  int which, b, tb, h;
+};
+__device__ __forceinline__ Chunk chunk_at(const QkArgs& a, int i) {
+  Chunk c;
+  const int n0 = a.B * a.nblk_t * a.H[0];
+  c.which = i >= n0;
+  if (c.which) i -= n0;
+  const int H = a.H[c.which];
+  const int rb = i / H;
+  c.h = i - rb * H;
+  c.b = rb / a.nblk_t;
+  c.tb = rb - c.b * a.nblk_t;
+  return c;
+}
+__device__ __forceinline__ void step(const QkArgs& a, Chunk& c) {
+  if (++c.h < a.H[c.which]) return;
+  c.h = 0;
+  if (++c.tb < a.nblk_t) return;
+  c.tb = 0;
+  if (++c.b < a.B) return;
+  c.b = 0;
+  ++c.which;
+}
 
-    for (int tb = blockIdx.x; tb < a.nblk_t && H > 0; tb += gridDim.x) {
-      const int t = tb * RPB + row;
-      const bool live = t < a.T;
-      float c[8], s[8];
-      rotation(f, 8 * l, p0 + t, a.rotate, c, s);
-#pragma unroll 1
-      for (int h0 = slice; h0 < H; h0 += U * a.S) {
-        float lo[U][8], hi[U][8], e_lo[U][8], e_hi[U][8];
-        size_t at[U];
-        bool on[U];
+template <typename T, int D, bool BWD>
+__global__ void __launch_bounds__(QK_THREADS, BWD ? 2 : QK_CTAS_PER_SM)
+qk_prologue_kernel(const __grid_constant__ QkArgs a, const __grid_constant__ Freqs f) {
+  using R = Ring<T, BWD>;
+  constexpr int LPR = D / 16, RPB = QK_THREADS / LPR, ROW = D * (int)sizeof(T), S = R::kStages;
+  extern __shared__ __align__(128) unsigned char smem[];
+  unsigned char* stage = smem;                                                    // [S][kBufs][kChunk]
+  float* red = reinterpret_cast<float*>(smem + S * R::kBufs * R::kChunk);         // [RPB][D] (backward)
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + S * R::kBufs * R::kChunk + R::kRed);
+  volatile int* abort = reinterpret_cast<volatile int*>(full + S);
+
+  const int tid = threadIdx.x, l = tid % LPR, row = tid / LPR;
+  const long long n_all = (long long)a.B * a.nblk_t * (a.H[0] + a.H[1]);     // < 2^31, checked on the host
+  const int lo = (int)(n_all * blockIdx.x / gridDim.x), hi = (int)(n_all * (blockIdx.x + 1) / gridDim.x);
+
+  if (tid == 0) {
+    for (int i = 0; i < S; ++i) ptx::mbar_init(&full[i], 1);
+    *abort = 0;
+    ptx::fence_mbar_init();
+  }
+  if (BWD && a.partial != nullptr && tid < D) {
+    a.partial[((size_t)0 * gridDim.x + blockIdx.x) * D + tid] = 0.f;
+    a.partial[((size_t)1 * gridDim.x + blockIdx.x) * D + tid] = 0.f;
+  }
+  __syncthreads();
+
+  Chunk ahead = chunk_at(a, lo);                      // thread 0's cursor: the next chunk to load
+  auto issue = [&](int i) {                           // thread 0 only; i must be the cursor's chunk
+    const Chunk c = ahead;
+    step(a, ahead);
+    const int H = a.H[c.which], t0 = c.tb * RPB;
+    const int rows = a.T - t0 < RPB ? a.T - t0 : RPB;
+    const size_t at = (((size_t)c.b * H + c.h) * a.T + t0) * D * sizeof(T);
+    const int slot = (i - lo) % S;
+    unsigned char* dst = stage + (size_t)slot * R::kBufs * R::kChunk;
+    expect_tx(&full[slot], (uint32_t)(rows * ROW * R::kBufs));
+    bulk_load(dst, static_cast<const unsigned char*>(a.x[c.which]) + at, (uint32_t)(rows * ROW), &full[slot]);
+    if (BWD)
+      bulk_load(dst + R::kChunk, static_cast<const unsigned char*>(a.dy[c.which]) + at, (uint32_t)(rows * ROW),
+                &full[slot]);
+  };
+  if (tid == 0)
+    for (int i = lo; i < hi && i < lo + S - 1; ++i) issue(i);
+
+  float c[8], s[8], g_lo[8], g_hi[8], acc[16];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-          const int h = h0 + u * a.S;
-          on[u] = live && h < H;
-          at[u] = (((size_t)b * H + (on[u] ? h : 0)) * a.T + (live ? t : 0)) * D + 8 * l;
-          if (on[u]) {
-            Io<T>::load(x, at[u], lo[u]);
-            Io<T>::load(x, at[u] + D / 2, hi[u]);
-            Io<T>::load(dy, at[u], e_lo[u]);
-            Io<T>::load(dy, at[u] + D / 2, e_hi[u]);
-          } else {
-            zero8(lo[u]); zero8(hi[u]); zero8(e_lo[u]); zero8(e_hi[u]);
-          }
-        }
+  for (int j = 0; j < 16; ++j) acc[j] = 0.f;
+  int cur_which = -1, cur_rb = -1;
+
+  // per-CTA sum of the gain-gradient terms over its rows, in row order, to this CTA's partial row
+  auto flush = [&](int which) {
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-          // the rotation is orthogonal: its transpose turns by the opposite angle
-          float du_lo[8], du_hi[8];
-          float ss = 0.f, dot = 0.f;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            du_lo[j] = e_lo[u][j] * c[j] + e_hi[u][j] * s[j];
-            du_hi[j] = e_hi[u][j] * c[j] - e_lo[u][j] * s[j];
-            ss += lo[u][j] * lo[u][j] + hi[u][j] * hi[u][j];
-            dot += du_lo[j] * g_lo[j] * lo[u][j] + du_hi[j] * g_hi[j] * hi[u][j];
-          }
-          ss = row_sum<LPR>(ss);
-          dot = row_sum<LPR>(dot);
-          const float r = rsqrtf(ss * (1.f / D) + a.eps);
-          const float back = r * r * r * dot * (1.f / D);
-          float o_lo[8], o_hi[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            acc[j] += du_lo[j] * lo[u][j] * r;
-            acc[8 + j] += du_hi[j] * hi[u][j] * r;
-            o_lo[j] = r * du_lo[j] * g_lo[j] - lo[u][j] * back;
-            o_hi[j] = r * du_hi[j] * g_hi[j] - hi[u][j] * back;
-          }
-          if (on[u]) {
-            Io<T>::store(dx, at[u], o_lo);
-            Io<T>::store(dx, at[u] + D / 2, o_hi);
-          }
-        }
-      }
+    for (int j = 0; j < 8; ++j) {
+      red[row * D + 8 * l + j] = acc[j];
+      red[row * D + D / 2 + 8 * l + j] = acc[8 + j];
+      acc[j] = acc[8 + j] = 0.f;
     }
+    __syncthreads();
+    if (tid < D) {
+      float sum = 0.f;
+      for (int r = 0; r < RPB; ++r) sum += red[r * D + tid];
+      a.partial[((size_t)which * gridDim.x + blockIdx.x) * D + tid] = sum;
+    }
+    __syncthreads();
+  };
 
-    if (a.partial != nullptr) {
-      // per-CTA sum over its rows in row order, then one partial row per CTA
+  int i = lo;
+  bool ok = true;
+  Chunk ch = chunk_at(a, lo);
+  for (; i < hi; ++i, step(a, ch)) {
+    const int n = i - lo, slot = n % S;
+    if (ch.which != cur_which) {
+      if (BWD && a.partial != nullptr && cur_which >= 0) flush(cur_which);
+      load_gain(a.gain[ch.which], 8 * l, D / 2, g_lo, g_hi);
+      cur_which = ch.which;
+      cur_rb = -1;
+    }
+    const int rb = ch.b * a.nblk_t + ch.tb;
+    const int t = ch.tb * RPB + row;
+    if (rb != cur_rb) {
+      const long long p0 = a.pos ? (long long)a.pos[ch.b] : a.pos0;
+      rotation(f, 8 * l, p0 + t, a.rotate, c, s);
+      cur_rb = rb;
+    }
+    const bool live = t < a.T;
+    unsigned char* buf = stage + (size_t)slot * R::kBufs * R::kChunk + (size_t)row * ROW;
+    const bool got = ptx::mbar_wait_warp(&full[slot], (uint32_t)(n / S) & 1u, abort);
+    if (got) {
+      float x_lo[8], x_hi[8];
+      if (live) {
+        Io<T>::load(buf, 8 * l, x_lo);
+        Io<T>::load(buf, D / 2 + 8 * l, x_hi);
+      } else {
+        zero8(x_lo);
+        zero8(x_hi);
+      }
+      float ss = 0.f;
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        red[row][8 * l + j] = acc[j];
-        red[row][D / 2 + 8 * l + j] = acc[8 + j];
+      for (int j = 0; j < 8; ++j) ss += x_lo[j] * x_lo[j] + x_hi[j] * x_hi[j];
+      if (!BWD) {
+        ss = row_sum<LPR>(ss);
+        const float r = rsqrtf(ss * (1.f / D) + a.eps);
+        float o_lo[8], o_hi[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float n_lo = x_lo[j] * r * g_lo[j], n_hi = x_hi[j] * r * g_hi[j];
+          o_lo[j] = n_lo * c[j] - n_hi * s[j];
+          o_hi[j] = n_hi * c[j] + n_lo * s[j];
+        }
+        if (live) {
+          Io<T>::store(buf, 8 * l, o_lo);
+          Io<T>::store(buf, D / 2 + 8 * l, o_hi);
+        }
+      } else {
+        float e_lo[8], e_hi[8];
+        if (live) {
+          Io<T>::load(buf + R::kChunk, 8 * l, e_lo);
+          Io<T>::load(buf + R::kChunk, D / 2 + 8 * l, e_hi);
+        } else {
+          zero8(e_lo);
+          zero8(e_hi);
+        }
+        // the rotation is orthogonal: its transpose turns by the opposite angle
+        float du_lo[8], du_hi[8], dot = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          du_lo[j] = e_lo[j] * c[j] + e_hi[j] * s[j];
+          du_hi[j] = e_hi[j] * c[j] - e_lo[j] * s[j];
+          dot += du_lo[j] * g_lo[j] * x_lo[j] + du_hi[j] * g_hi[j] * x_hi[j];
+        }
+        ss = row_sum<LPR>(ss);
+        dot = row_sum<LPR>(dot);
+        const float r = rsqrtf(ss * (1.f / D) + a.eps);
+        const float back = r * r * r * dot * (1.f / D);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          acc[j] += du_lo[j] * x_lo[j] * r;
+          acc[8 + j] += du_hi[j] * x_hi[j] * r;
+          e_lo[j] = r * du_lo[j] * g_lo[j] - x_lo[j] * back;
+          e_hi[j] = r * du_hi[j] * g_hi[j] - x_hi[j] * back;
+        }
+        if (live) {
+          Io<T>::store(buf + R::kChunk, 8 * l, e_lo);
+          Io<T>::store(buf + R::kChunk, D / 2 + 8 * l, e_hi);
+        }
       }
-      __syncthreads();
-      if (threadIdx.x < D) {
-        float sum = 0.f;
-        for (int r = 0; r < RPB; ++r) sum += red[r][threadIdx.x];
-        a.partial[((size_t)which * n_cta + cta) * D + threadIdx.x] = sum;
+      ptx::fence_proxy_async_smem();
+    }
+    ok = __syncthreads_and(got) != 0;
+    if (!ok) break;
+    if (tid == 0) {
+      const int H = a.H[ch.which], t0 = ch.tb * RPB;
+      const int rows = a.T - t0 < RPB ? a.T - t0 : RPB;
+      const size_t at = (((size_t)ch.b * H + ch.h) * a.T + t0) * D * sizeof(T);
+      unsigned char* src = stage + (size_t)slot * R::kBufs * R::kChunk + (BWD ? R::kChunk : 0);
+      bulk_store(static_cast<unsigned char*>(a.y[ch.which]) + at, src, (uint32_t)(rows * ROW));
+      ptx::tma_store_commit();
+      const int next = i + S - 1;
+      if (next < hi) {
+        store_wait_read_but_one();          // the slot of chunk i - 1 has been read out
+        issue(next);
       }
-      __syncthreads();
     }
   }
+
+  if (tid == 0) {
+    ptx::tma_store_wait();
+    if (!ok) {
+      // give the loads still in flight a bounded time to land before the CTA's memory goes away
+      const int issued = i + S - 1 < hi ? i + S - 1 : hi;
+      for (int j = i; j < issued; ++j) {
+        const int n = j - lo;
+        for (int it = 0; it < ptx::kWaitPolls && !ptx::mbar_try_wait(&full[n % S], (uint32_t)(n / S) & 1u); ++it) {}
+      }
+      g_qk_status = RATTN_ERR_TIMEOUT;
+    }
+  }
+  if (BWD && ok && a.partial != nullptr && cur_which >= 0) flush(cur_which);
 }
 
 // gain gradient = sum of the per-CTA partial sums, added in an order fixed by the sizes alone
@@ -328,52 +388,62 @@ int check(const rattn_qk_params* p) {
   if (misaligned16(p->q) || misaligned16(p->k) || misaligned16(p->q_gain) || misaligned16(p->k_gain))
     return RATTN_ERR_MISALIGNED;
   if (((uintptr_t)p->pos & 3u) != 0) return RATTN_ERR_MISALIGNED;
-  if ((long long)p->B * geometry(p->B, p->H_q, p->H_kv, p->T, p->d).S > 65535) return RATTN_ERR_BAD_ARG;
+  const int rpb = QK_THREADS / (p->d / 16);
+  if ((long long)p->B * ((p->T + rpb - 1) / rpb) * ((long long)p->H_q + p->H_kv) >= (1ll << 31)) return RATTN_ERR_BAD_ARG;
   return RATTN_OK;
 }
 
-void fill(const rattn_qk_params* p, const Geometry& g, QkArgs* a, Freqs* f) {
+void fill(const rattn_qk_params* p, QkArgs* a, Freqs* f) {
   a->x[0] = p->q; a->x[1] = p->k;
   a->gain[0] = p->q_gain; a->gain[1] = p->k_gain;
   a->H[0] = p->H_q; a->H[1] = p->H_kv;
-  a->B = p->B; a->T = p->T; a->S = g.S; a->nblk_t = g.nblk_t;
+  const int rpb = QK_THREADS / (p->d / 16);
+  a->B = p->B; a->T = p->T; a->nblk_t = (p->T + rpb - 1) / rpb;
   a->eps = p->eps;
   a->rotate = p->theta > 0.f;
   a->pos0 = p->pos0;
   a->pos = p->pos;
   a->partial = nullptr;
   a->dy[0] = a->dy[1] = nullptr;
+  a->y[0] = a->y[1] = nullptr;
   for (int i = 0; i < 64; ++i)
     f->inv[i] = a->rotate && i < p->d / 2 ? std::pow((double)p->theta, -2.0 * i / p->d) : 0.0;
 }
 
-template <typename T>
-cudaError_t launch_fwd(const QkArgs& a, const Freqs& f, const Geometry& g, int d, cudaStream_t s) {
-  KernelTimer kt("qk_prologue", s);
-  const dim3 grid(g.gx, g.gy);
-  if (d == 128) qk_prologue_kernel<T, 128><<<grid, QK_THREADS, 0, s>>>(a, f);
-  else qk_prologue_kernel<T, 64><<<grid, QK_THREADS, 0, s>>>(a, f);
+// CTAs of a launch: every resident slot of the device, fewer when there are fewer chunks
+cudaError_t grid_size(const QkArgs& a, int per_sm, int* n_cta) {
+  int dev = 0, n_sm = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  long long n = (long long)a.B * a.nblk_t * (a.H[0] + a.H[1]);
+  if (n > (long long)n_sm * per_sm) n = (long long)n_sm * per_sm;
+  if (n > QK_MAX_CTAS) n = QK_MAX_CTAS;
+  *n_cta = (int)n;
+  return cudaSuccess;
+}
+
+template <typename T, int D, bool BWD>
+cudaError_t launch_one(const QkArgs& a, const Freqs& f, int n_cta, cudaStream_t s) {
+  constexpr int smem = Ring<T, BWD>::kBytes;
+  cudaError_t e = cudaFuncSetAttribute(qk_prologue_kernel<T, D, BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  KernelTimer kt(BWD ? "qk_prologue_bwd" : "qk_prologue", s);
+  qk_prologue_kernel<T, D, BWD><<<n_cta, QK_THREADS, smem, s>>>(a, f);
   count_launches(1);
   return cudaGetLastError();
 }
 
-template <typename T>
-cudaError_t launch_bwd(const QkArgs& a, const Freqs& f, const Geometry& g, int d, float* dq_gain, float* dk_gain,
-                       cudaStream_t s) {
-  const dim3 grid(g.gx, g.gy);
-  {
-    KernelTimer kt("qk_prologue_bwd", s);
-    if (d == 128) qk_prologue_bwd_kernel<T, 128><<<grid, QK_THREADS, 0, s>>>(a, f);
-    else qk_prologue_bwd_kernel<T, 64><<<grid, QK_THREADS, 0, s>>>(a, f);
-    count_launches(1);
-  }
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess || a.partial == nullptr) return e;
-  KernelTimer kt("qk_gain_reduce", s);
-  if (d == 128) qk_gain_reduce_kernel<128><<<2, 1024, 0, s>>>(a.partial, g.n_cta(), dq_gain, dk_gain);
-  else qk_gain_reduce_kernel<64><<<2, 1024, 0, s>>>(a.partial, g.n_cta(), dq_gain, dk_gain);
-  count_launches(1);
-  return cudaGetLastError();
+template <bool BWD>
+cudaError_t launch(const QkArgs& a, const Freqs& f, int d, int dtype, int n_cta, cudaStream_t s) {
+  if (dtype == RATTN_BF16)
+    return d == 128 ? launch_one<__nv_bfloat16, 128, BWD>(a, f, n_cta, s) : launch_one<__nv_bfloat16, 64, BWD>(a, f, n_cta, s);
+  return d == 128 ? launch_one<float, 128, BWD>(a, f, n_cta, s) : launch_one<float, 64, BWD>(a, f, n_cta, s);
+}
+
+int fail(cudaError_t e) {
+  set_last_cuda_error((int)e);
+  return RATTN_ERR_CUDA;
 }
 
 }  // namespace
@@ -385,8 +455,7 @@ extern "C" {
 
 size_t rattn_qk_prologue_workspace_bytes(int B, int H_q, int H_kv, int T, int d) {
   if (B < 1 || H_q < 1 || H_kv < 0 || T < 1 || (d != 64 && d != 128)) return 0;
-  const Geometry g = geometry(B, H_q, H_kv, T, d);
-  return ((size_t)2 * g.n_cta() * d * sizeof(float) + 255) / 256 * 256;
+  return (size_t)2 * QK_MAX_CTAS * d * sizeof(float);
 }
 
 int rattn_qk_prologue(const rattn_qk_params* p, void* stream) {
@@ -394,16 +463,15 @@ int rattn_qk_prologue(const rattn_qk_params* p, void* stream) {
   if (rc != RATTN_OK) return rc;
   if (!p->q_out || (p->H_kv > 0 && !p->k_out)) return RATTN_ERR_NULL_PTR;
   if (misaligned16(p->q_out) || misaligned16(p->k_out)) return RATTN_ERR_MISALIGNED;
-  const Geometry g = geometry(p->B, p->H_q, p->H_kv, p->T, p->d);
   QkArgs a;
   Freqs f;
-  fill(p, g, &a, &f);
+  fill(p, &a, &f);
   a.y[0] = p->q_out; a.y[1] = p->k_out;
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-  const cudaError_t e = p->dtype == RATTN_BF16 ? launch_fwd<__nv_bfloat16>(a, f, g, p->d, s)
-                                               : launch_fwd<float>(a, f, g, p->d, s);
-  if (e != cudaSuccess) { set_last_cuda_error((int)e); return RATTN_ERR_CUDA; }
-  return RATTN_OK;
+  int n_cta = 0;
+  cudaError_t e = grid_size(a, QK_CTAS_PER_SM, &n_cta);
+  if (e == cudaSuccess) e = launch<false>(a, f, p->d, p->dtype, n_cta, s);
+  return e == cudaSuccess ? RATTN_OK : fail(e);
 }
 
 int rattn_qk_prologue_backward(const rattn_qk_params* p, const void* dq_out, const void* dk_out, void* dq, void* dk,
@@ -416,10 +484,9 @@ int rattn_qk_prologue_backward(const rattn_qk_params* p, const void* dq_out, con
   if (misaligned16(dq_out) || misaligned16(dk_out) || misaligned16(dq) || misaligned16(dk) ||
       misaligned16(dq_gain) || misaligned16(dk_gain))
     return RATTN_ERR_MISALIGNED;
-  const Geometry g = geometry(p->B, p->H_q, p->H_kv, p->T, p->d);
   QkArgs a;
   Freqs f;
-  fill(p, g, &a, &f);
+  fill(p, &a, &f);
   a.y[0] = dq; a.y[1] = dk;
   a.dy[0] = dq_out; a.dy[1] = dk_out;
   if (dq_gain || dk_gain) {
@@ -429,11 +496,31 @@ int rattn_qk_prologue_backward(const rattn_qk_params* p, const void* dq_out, con
     a.partial = static_cast<float*>(workspace);
   }
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-  const cudaError_t e = p->dtype == RATTN_BF16
-                            ? launch_bwd<__nv_bfloat16>(a, f, g, p->d, dq_gain, dk_gain, s)
-                            : launch_bwd<float>(a, f, g, p->d, dq_gain, dk_gain, s);
-  if (e != cudaSuccess) { set_last_cuda_error((int)e); return RATTN_ERR_CUDA; }
-  return RATTN_OK;
+  int n_cta = 0;
+  cudaError_t e = grid_size(a, 2, &n_cta);
+  if (e == cudaSuccess) e = launch<true>(a, f, p->d, p->dtype, n_cta, s);
+  if (e == cudaSuccess && a.partial != nullptr) {
+    KernelTimer kt("qk_gain_reduce", s);
+    if (p->d == 128) qk_gain_reduce_kernel<128><<<2, 1024, 0, s>>>(a.partial, n_cta, dq_gain, dk_gain);
+    else qk_gain_reduce_kernel<64><<<2, 1024, 0, s>>>(a.partial, n_cta, dq_gain, dk_gain);
+    count_launches(1);
+    e = cudaGetLastError();
+  }
+  return e == cudaSuccess ? RATTN_OK : fail(e);
+}
+
+int rattn_qk_prologue_status(void* stream) {
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  int word = 0;
+  cudaError_t e = cudaMemcpyFromSymbolAsync(&word, g_qk_status, sizeof(int), 0, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e == cudaSuccess && word != 0) {
+    const int zero = 0;
+    e = cudaMemcpyToSymbolAsync(g_qk_status, &zero, sizeof(int), 0, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  }
+  if (e != cudaSuccess) return fail(e);
+  return word == 0 ? RATTN_OK : RATTN_ERR_TIMEOUT;
 }
 
 }  // extern "C"

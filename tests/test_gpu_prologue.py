@@ -52,11 +52,13 @@ def cu(t):
     (1, 2, 2, 64, 128, "f32", 2 ** 30, 5.0e5),    # a position fp32 could not even hold exactly + 1
     (2, 2, 1, 200, 128, "bf16", 0, None),         # global layer: norm only
     (2, 2, 1, 50, 64, "f32", 7, 1.0e4),           # another base
+    (3, 16, 4, 1100, 128, "bf16", 0, 5.0e5),      # more chunks than stages in every CTA
+    (2, 8, 8, 700, 64, "bf16", 3, 5.0e5),         # d = 64, bf16: 64 rows per chunk
 ])
 def test_prologue_forward(B, Hq, Hkv, T, d, dtype, pos0, theta):
     q, k, gq, gk = make(B, Hq, Hkv, T, d, dtype, 9000 + T + d)
     qo, ko = R.rattn_qk_prologue(q.cuda(), k.cuda(), q_gain=cu(gq), k_gain=cu(gk), theta=theta, pos0=pos0)
-    torch.cuda.synchronize()
+    assert R.rattn_qk_prologue_status() == 0, "a device-side wait expired"
     pos = pos0 + np.arange(T)
     close(qo, P.qk_prologue(np64(q), np64(gq), pos, theta), dtype, "q")
     close(ko, P.qk_prologue(np64(k), np64(gk), pos, theta), dtype, "k")
@@ -95,6 +97,8 @@ def test_prologue_decode_shape():
     (2, 4, 2, 300, 128, "bf16", 5.0e5),
     (1, 3, 1, 77, 64, "f32", 5.0e5),
     (2, 16, 16, 130, 128, "bf16", None),
+    (3, 16, 4, 1100, 128, "bf16", 5.0e5),         # long enough for the ring to wrap in every CTA
+    (2, 8, 8, 700, 64, "f32", 5.0e5),
 ])
 def test_prologue_backward(B, Hq, Hkv, T, d, dtype, theta):
     q, k, gq, gk = make(B, Hq, Hkv, T, d, dtype, 9300 + T)
@@ -116,6 +120,7 @@ def test_prologue_backward(B, Hq, Hkv, T, d, dtype, theta):
         assert (err <= bound).all(), (name, float(err.max()))
         assert np.abs(np64(dg) - rg).max() <= 1e-4 * np.abs(rg).max(), name
         assert torch.equal(dx, dx2) and torch.equal(dg, dg2), "run-to-run bits"
+    assert R.rattn_qk_prologue_status() == 0
     # without gain gradients no workspace is needed and the input gradients are the same bits
     out3 = R.rattn_qk_prologue_backward(q.cuda(), k.cuda(), dqo.cuda(), dko.cuda(), q_gain=cu(gq), k_gain=cu(gk),
                                         theta=theta, pos0=pos0, gain_grads=False)
