@@ -245,6 +245,14 @@ int rattn_decode_step(const void* q, const void* k, const void* v,
 int rattn_decode_step_ex(const rattn_params* p, void* k_ring, void* v_ring, float* state,
                          int pos, void* stream);
 
+/* For bf16, d = 128, w a multiple of 64 and H_q / H_kv <= 8 (unless RATTN_FLAG_FORCE_GENERIC) the
+ * decode step stages the ring and the state through shared memory with asynchronous copies and
+ * waits for them with a bound.  rattn_decode_status (synchronises the stream) returns
+ * RATTN_ERR_TIMEOUT if such a wait has expired in any decode step on the current device since it
+ * was last asked (the step then left its outputs, ring and state in an unspecified state), else
+ * RATTN_OK. */
+int rattn_decode_status(void* stream);
+
 /*
  * Bytes of workspace a call with these sizes, mode (rattn_mode) and flags (RATTN_FLAG_*)
  * needs; dtype is a rattn_dtype.  Returns 0 for invalid arguments.  The first 256 bytes hold

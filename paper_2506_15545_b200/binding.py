@@ -26,7 +26,7 @@ EXPORTS = (
     "rattn_read_status", "rattn_strerror", "rattn_last_cuda_error", "rattn_launch_count",
     "rattn_uses_tensor_path", "rattn_timing_enable", "rattn_timing_read",
     "rattn_forward_static", "rattn_static_status", "rattn_tune",
-    "rattn_qk_prologue", "rattn_qk_prologue_backward", "rattn_qk_prologue_workspace_bytes", "rattn_qk_prologue_status",
+    "rattn_qk_prologue", "rattn_qk_prologue_backward", "rattn_qk_prologue_workspace_bytes", "rattn_qk_prologue_status", "rattn_decode_status",
 )
 TUNE_STATE_STRIDE, TUNE_OVERLAP, TUNE_UNIT_ORDER, TUNE_GRID = 0, 1, 2, 3
 
@@ -128,6 +128,8 @@ def lib() -> ctypes.CDLL:
     L.rattn_qk_prologue_backward.restype = ci
     L.rattn_qk_prologue_workspace_bytes.argtypes = [ci, ci, ci, ci, ci]
     L.rattn_qk_prologue_workspace_bytes.restype = ctypes.c_size_t
+    L.rattn_decode_status.argtypes = [vp]
+    L.rattn_decode_status.restype = ci
     L.rattn_qk_prologue_status.argtypes = [vp]
     L.rattn_qk_prologue_status.restype = ci
     L.rattn_timing_enable.argtypes = [ci]
@@ -303,12 +305,13 @@ def rattn_decode_step(q, k, v, k_ring, v_ring, state, pos, out=None, stream=None
 
 
 def rattn_decode_step_ex(q, k, v, k_ring, v_ring, state, pos, *, scale=1.0, eps=1e-6,
-                         gamma_swa=None, gamma_rla=None, out=None, phi=PHI_SOFTMAX, pos_dev=None, stream=None):
+                         gamma_swa=None, gamma_rla=None, out=None, phi=PHI_SOFTMAX, pos_dev=None, flags=0,
+                         stream=None):
     """pos_dev: optional int32 device tensor [B], one position per batch entry (then `pos` is ignored)."""
     _dense(q, k, v, k_ring, v_ring, state, out, gamma_swa, gamma_rla, pos_dev)
     out = torch.empty_like(q) if out is None else out
     p = _params(q, k, v, out, k_ring.shape[2], scale, eps, gamma_swa, gamma_rla, MODE_RATTN,
-                None, 0, phi)
+                None, flags, phi)
     p.pos = None if pos_dev is None else pos_dev.data_ptr()
     _check(lib().rattn_decode_step_ex(ctypes.byref(p), _ptr(k_ring), _ptr(v_ring), _ptr(state),
                                       pos, _stream(stream)), "rattn_decode_step_ex")
@@ -372,6 +375,10 @@ def _qk_params(q, k, q_out, k_out, q_gain, k_gain, theta, eps, pos0, pos):
 
 def rattn_qk_prologue_workspace_bytes(B, H_q, H_kv, T, d) -> int:
     return int(lib().rattn_qk_prologue_workspace_bytes(B, H_q, H_kv, T, d))
+
+
+def rattn_decode_status(stream=None) -> int:
+    return int(lib().rattn_decode_status(_stream(stream)))
 
 
 def rattn_qk_prologue_status(stream=None) -> int:

@@ -21,7 +21,7 @@ LIB_DEBUG = os.path.join(HERE, "librattn_dbg.so")      # same sources with -DRAT
 LIB_TIMELINE = os.path.join(HERE, "librattn_tl.so")    # same sources with -DRATTN_TIMELINE (bench.py --case timeline)
 
 SOURCES = ["rattn_api.cu", "generic_fwd.cu", "generic_bwd.cu", "decode.cu", "tc_fwd.cu",
-           "tc_fwd2.cu", "tc_state.cu", "tc_bwd.cu", "static_scratch.cu", "qk_prologue.cu"]
+           "tc_fwd2.cu", "tc_state.cu", "tc_bwd.cu", "static_scratch.cu", "qk_prologue.cu", "decode_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC",
               "-I" + os.path.join(ROOT, "include"), "-I" + CSRC]

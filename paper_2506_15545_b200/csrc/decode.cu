@@ -511,6 +511,8 @@ cudaError_t launch_gather_history(const Args& a, const void* k_chunk, const void
 
 cudaError_t launch_decode(const Args& p, void* k_ring, void* v_ring, float* state, int pos, const int* pos_dev,
                           cudaStream_t s) {
+  if (!(p.flags & RATTN_FLAG_FORCE_GENERIC) && decode_tc_applies(p, p.w))
+    return launch_decode_tc(p, k_ring, v_ring, state, pos, pos_dev, s);
   DecodeArgs a;
   a.pos_dev = pos_dev;
   a.q = p.q; a.k = p.k; a.v = p.v; a.k_ring = k_ring; a.v_ring = v_ring; a.state = state;

@@ -147,6 +147,7 @@ static int resolve(const rattn_params* p, Args* a, bool need_T) {
   a->w = (p->mode == RATTN_MODE_FULL_CAUSAL && need_T) ? p->T : p->w;
   a->group = p->H_q / p->H_kv;
   a->dtype = p->dtype; a->mode = p->mode;
+  a->flags = p->flags;
   a->phi = p->feature_map;
   a->scale = p->scale; a->eps = p->eps;
   a->gamma_swa = p->gamma_swa; a->gamma_rla = p->gamma_rla;
@@ -332,6 +333,13 @@ int rattn_decode_step_ex(const rattn_params* p, void* k_ring, void* v_ring, floa
   cudaError_t e = launch_decode(a, k_ring, v_ring, state, pos, p->pos, reinterpret_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return fail_cuda(e);
   return RATTN_OK;
+}
+
+int rattn_decode_status(void* stream) {
+  cudaError_t e = cudaSuccess;
+  const int word = decode_tc_status(reinterpret_cast<cudaStream_t>(stream), &e);
+  if (e != cudaSuccess) return fail_cuda(e);
+  return word == 0 ? RATTN_OK : RATTN_ERR_TIMEOUT;
 }
 
 int rattn_decode_step(const void* q, const void* k, const void* v, void* k_ring, void* v_ring,

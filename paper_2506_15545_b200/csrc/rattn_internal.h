@@ -55,6 +55,7 @@ struct Args {
   int pos_shift;               // sequence position of key row 0 (pos0 - w for a resumed sequence, else 0)
   int group;                   // H_q / H_kv
   int dtype, mode;
+  unsigned flags;              // rattn_params.flags
   int phi;                     // rattn_feature_map
   float scale, eps;
   const float* gamma_swa;
@@ -93,6 +94,12 @@ cudaError_t launch_generic_forward(const Args& a, cudaStream_t s);
 cudaError_t launch_generic_backward(const Args& a, cudaStream_t s);
 cudaError_t launch_decode(const Args& a, void* k_ring, void* v_ring, float* state, int pos, const int* pos_dev,
                           cudaStream_t s);
+// The TMA-staged decode step (bf16, d = 128, w a multiple of 64, groups of up to 8 heads) and
+// its status word (RATTN_ERR_TIMEOUT once a bounded wait has expired; reading clears it).
+bool decode_tc_applies(const Args& a, int w);
+cudaError_t launch_decode_tc(const Args& a, void* k_ring, void* v_ring, float* state, int pos, const int* pos_dev,
+                             cudaStream_t s);
+int decode_tc_status(cudaStream_t s, cudaError_t* err);
 // prefill -> decode hand-off: the rings, and (state_too) the state by the portable kernel
 cudaError_t launch_handoff(const Args& a, cudaStream_t s, bool state_too);
 cudaError_t launch_tc_forward(const Args& a, cudaStream_t s);        // chunk states, then the main kernel
