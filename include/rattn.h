@@ -321,7 +321,9 @@ typedef enum rattn_knob {
                                     under the chunk-state kernel), then heaviest first; 2 heaviest first
                                     throughout; 3 the same, dealt round-robin instead of drawn from a counter.
                                     Automatic = 1 when the state kernel leaves at least half of the SMs free. */
-  RATTN_TUNE_GRID = 3            /* CTAs of the persistent forward kernel: 0 (default) = one per SM */
+  RATTN_TUNE_GRID = 3,           /* CTAs of the persistent forward kernel: 0 (default) = one per SM */
+  RATTN_TUNE_DECODE_STAGES = 4   /* 16 KB stages of the staged decode step: 0 (default) = as many as let two
+                                    CTAs share an SM; 3..8 (ignored where that many do not fit) */
 } rattn_knob;
 int rattn_tune(int knob, int value);
 

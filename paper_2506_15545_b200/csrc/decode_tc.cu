@@ -5,7 +5,7 @@
 // state back (Section 2.1: a cache of at most w+1 tokens; Eq. 4: the state), so it is bound by
 // HBM traffic.  One CTA per (batch entry, K/V head), two CTAs per SM.  Everything it will read
 // is requested up front as 16 KB pieces (64 ring slots, or 32 state rows) that pass through a
-// ring of four stages, so the memory system always has the next pieces in flight, whatever the
+// ring of stages (as many as let two CTAs share an SM, five at w = 512 with four heads), so the memory system always has the next pieces in flight, whatever the
 // warps are doing.  The two ring products are small matrix products with the group's query heads
 // as rows (q K^T, then P V), issued as warp-level mma on the pieces in shared memory (the K and V
 // pieces arrive 128-byte swizzled, so the fragment loads are conflict-free); with at most 8 rows
@@ -23,7 +23,7 @@ using namespace ptx;
 
 constexpr int DT_THREADS = 256;
 constexpr int DT_WARPS = DT_THREADS / 32;
-constexpr int DT_STAGES = 4;
+constexpr int DT_MAX_STAGES = 8;
 constexpr int DT_PIECE = 16384;            // 64 ring slots x 128 bf16, or 32 state rows x 128 fp32
 constexpr int D = 128;
 constexpr int QB_STRIDE = D + 8;           // bf16 elements; 272 bytes: rows fall 16 bytes apart modulo 128
@@ -35,7 +35,7 @@ struct DecodeTcArgs {
   __nv_bfloat16* k_ring; __nv_bfloat16* v_ring; float* state; __nv_bfloat16* out;
   const float* gamma_swa; const float* gamma_rla;
   const int* pos_dev;
-  int B, H_q, H_kv, w, pos, group, phi;
+  int B, H_q, H_kv, w, pos, group, phi, stages;
   float scale, eps;
 };
 
@@ -102,16 +102,17 @@ __device__ __forceinline__ uint32_t keep_valid(uint32_t pair, int s, int live) {
 
 // Shared-memory plan (bytes, after the 1024-byte aligned stages).
 struct Plan {
-  int q_b, zero, p_hi, p_lo, logit, q_f, fq, vec, o_swa, o_rla, stat, bars, total;
+  int stages, q_b, zero, p_hi, p_lo, logit, q_f, fq, vec, o_swa, o_rla, stat, red, bars, total;
 };
-__host__ __device__ inline Plan plan(int g, int w) {
+__host__ __device__ inline Plan plan_with(int g, int w, int stages) {
   Plan p;
-  int off = DT_STAGES * DT_PIECE;
+  p.stages = stages;
+  int off = stages * DT_PIECE;
   auto take = [&](int bytes) { const int at = off; off += (bytes + 15) & ~15; return at; };
   p.q_b = take(8 * QB_STRIDE * 2);         // bf16 [8][136]: the group's queries, rows >= g zero
   p.zero = take(16);                       // what the fragment rows 8..15 point at
-  p.p_hi = take(8 * (w + 8) * 2);          // bf16 [8][w + 8]: attention weights, leading part
-  p.p_lo = take(8 * (w + 8) * 2);          //                  remainder
+  p.p_hi = take(g * (w + 8) * 2);          // bf16 [g][w + 8]: attention weights, leading part
+  p.p_lo = take(g * (w + 8) * 2);          //                  remainder
   p.logit = take(g * (w + 4) * 4);         // fp32 [g][w + 4]: scaled logits, then un-normalised weights
   p.q_f = take(g * D * 4);                 // fp32 raw q
   p.fq = take(g * D * 4);                  // phi(q)
@@ -119,9 +120,17 @@ __host__ __device__ inline Plan plan(int g, int w) {
   p.o_swa = take(g * D * 4);
   p.o_rla = take(g * D * 4);
   p.stat = take(4 * 8 * 4);                // per head: 1 / sum, weight of the incoming token, incoming logit
-  p.bars = take(8 * DT_STAGES + 16);
+  p.red = take(2 * DT_WARPS * 8 * 4);       // per warp and head: maximum, then sum, of its share of the logits
+  p.bars = take(8 * DT_MAX_STAGES + 16);
   p.total = off + 1024;                    // room to align the stages
   return p;
+}
+// As many stages as let two CTAs share an SM (each may use (227 KB - 2 KB) / 2), at least three.
+__host__ __device__ inline Plan plan(int g, int w, int forced = 0) {
+  if (forced >= 3 && forced <= DT_MAX_STAGES && plan_with(g, w, forced).total <= 227 * 1024) return plan_with(g, w, forced);
+  int stages = 6;
+  while (stages > 3 && plan_with(g, w, stages).total > (227 * 1024 - 2048) / 2) --stages;
+  return plan_with(g, w, stages);
 }
 
 template <int G>
@@ -130,7 +139,8 @@ decode_tc_kernel(const __grid_constant__ DecodeTcArgs a, const __grid_constant__
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int g = a.group, w = a.w;
-  const Plan P = plan(g, w);
+  const Plan P = plan(g, w, a.stages);
+  const int NS = P.stages;
   __nv_bfloat16* q_b = reinterpret_cast<__nv_bfloat16*>(sm + P.q_b);
   __nv_bfloat16* p_hi = reinterpret_cast<__nv_bfloat16*>(sm + P.p_hi);
   __nv_bfloat16* p_lo = reinterpret_cast<__nv_bfloat16*>(sm + P.p_lo);
@@ -147,8 +157,10 @@ decode_tc_kernel(const __grid_constant__ DecodeTcArgs a, const __grid_constant__
   float* inv_sum = reinterpret_cast<float*>(sm + P.stat);      // [8]
   float* p_new = inv_sum + 8;                                  // [8] un-normalised weight of the incoming token
   float* l_new = p_new + 8;                                    // [8] its scaled logit
+  float* w_max = reinterpret_cast<float*>(sm + P.red);         // [8 warps][8 heads]
+  float* w_sum = w_max + DT_WARPS * 8;
   uint64_t* full = reinterpret_cast<uint64_t*>(sm + P.bars);
-  volatile int* abort = reinterpret_cast<volatile int*>(full + DT_STAGES);
+  volatile int* abort = reinterpret_cast<volatile int*>(full + DT_MAX_STAGES);
   const int LS = w + 4, PS = w + 8;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -168,17 +180,35 @@ decode_tc_kernel(const __grid_constant__ DecodeTcArgs a, const __grid_constant__
   float* S = a.state + (size_t)z * D * D;
   __nv_bfloat16* og = a.out + ((size_t)b * a.H_q + (size_t)hk * g) * D;
 
+  // The step's small operands are requested before any bulk traffic: behind 20 MB of ring pieces
+  // they would wait microseconds.  They go to registers here and to shared memory once the pieces
+  // have been asked for.
   if (tid == 0) {
-    for (int i = 0; i < DT_STAGES; ++i) mbar_init(&full[i], 1);
+    prefetch_tensormap(&maps.k);
+    prefetch_tensormap(&maps.v);
+  }
+  uint4 q_reg = make_uint4(0u, 0u, 0u, 0u);                      // thread (row, 16-byte chunk) of the group's queries
+  if (tid < g * 16) q_reg = reinterpret_cast<const uint4*>(qg)[tid];
+  __nv_bfloat16 kn = __float2bfloat16_rn(0.f), vn = kn, ko = kn, vo_ = kn;
+  if (tid < D) {
+    kn = kg[tid];
+    vn = vg[tid];
+    if (evict) {
+      ko = kr[(size_t)slot * D + tid];
+      vo_ = vr[(size_t)slot * D + tid];
+    }
+  }
+  if (tid == 0) {
+    for (int i = 0; i < NS; ++i) mbar_init(&full[i], 1);
     *abort = 0;
     fence_mbar_init();
   }
   __syncthreads();
 
-  // piece p of the step's stream into stage p % DT_STAGES (warp 0, all lanes)
+  // piece p of the step's stream into stage p % NS (warp 0, all lanes)
   auto issue = [&](int p) {
-    unsigned char* dst = sm + (p % DT_STAGES) * DT_PIECE;
-    uint64_t* bar = &full[p % DT_STAGES];
+    unsigned char* dst = sm + (p % NS) * DT_PIECE;
+    uint64_t* bar = &full[p % NS];
     mbar_arrive_expect_tx(bar, DT_PIECE);
     if (p < 2 * np) {
       const CUtensorMap* m = p < np ? &maps.k : &maps.v;
@@ -190,40 +220,33 @@ decode_tc_kernel(const __grid_constant__ DecodeTcArgs a, const __grid_constant__
     }
   };
   if (warp == 0)
-    for (int p = 0; p < DT_STAGES && p < n_pieces; ++p) issue(p);
+    for (int p = 0; p < NS && p < n_pieces; ++p) issue(p);
 
-  // ---- the step's small operands -----------------------------------------------------------
-  for (int i = tid; i < 8 * QB_STRIDE; i += DT_THREADS) {
-    const int r = i / QB_STRIDE, c = i % QB_STRIDE;
-    q_b[i] = (r < g && c < D) ? qg[r * D + c] : __float2bfloat16_rn(0.f);
-  }
-  for (int i = tid; i < g * D; i += DT_THREADS) q_f[i] = __bfloat162float(qg[i]);
-  if (tid < 4) reinterpret_cast<uint32_t*>(sm + P.zero)[tid] = 0u;
-  if (tid < D) {
-    k_new[tid] = __bfloat162float(kg[tid]);
-    v_new[tid] = __bfloat162float(vg[tid]);
-    k_old[tid] = evict ? __bfloat162float(kr[(size_t)slot * D + tid]) : 0.f;
-    v_old[tid] = evict ? __bfloat162float(vr[(size_t)slot * D + tid]) : 0.f;
-  }
-  // weights of slots that hold no token yet, and the rows of P beyond the group
-  for (int i = tid; i < 8 * PS; i += DT_THREADS) {
-    const int r = i / PS, c = i % PS;
-    if (r >= g || c >= n_valid) p_hi[i] = p_lo[i] = __float2bfloat16_rn(0.f);
-  }
-  __syncthreads();
-  for (int r = warp; r <= g; r += DT_WARPS) {
-    if (r < g) warp_feature_map(fq_s + r * D, q_f + r * D, lane, a.phi);
-    else warp_feature_map(fk_old, k_old, lane, a.phi);
-  }
-  if (warp == DT_WARPS - 1) {                                   // the incoming token's logit (Section 2.1)
-    for (int hh = 0; hh < g; ++hh) {
-      float x = 0.f;
+  // queries: bf16 rows for the fragments (rows beyond the group zero), fp32 for phi and the new logit
+  if (tid < 128) {
+    const int r = tid >> 4, c = tid & 15;
+    *reinterpret_cast<uint4*>(q_b + r * QB_STRIDE + c * 8) = q_reg;
+    if (r < g) {
+      const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&q_reg);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) x += q_f[hh * D + lane + 32 * i] * k_new[lane + 32 * i];
-      x = warp_sum(x);
-      if (lane == 0) l_new[hh] = x * a.scale;
+      for (int i = 0; i < 4; ++i) {
+        const float2 x = __bfloat1622float2(h2[i]);
+        q_f[r * D + c * 8 + 2 * i] = x.x;
+        q_f[r * D + c * 8 + 2 * i + 1] = x.y;
+      }
     }
   }
+  if (tid < 4) reinterpret_cast<uint32_t*>(sm + P.zero)[tid] = 0u;
+  if (tid < D) {
+    k_new[tid] = __bfloat162float(kn);
+    v_new[tid] = __bfloat162float(vn);
+    k_old[tid] = __bfloat162float(ko);
+    v_old[tid] = __bfloat162float(vo_);
+  }
+  // weights of slots that hold no token yet
+  for (int r = 0; r < g; ++r)
+    for (int c = n_valid + tid; c < PS; c += DT_THREADS) p_hi[r * PS + c] = p_lo[r * PS + c] = __float2bfloat16_rn(0.f);
+  __syncthreads();
 
   // query fragments: rows 0..7 from q_b, rows 8..15 are zero
   const uint32_t zero_addr = smem_u32(sm + P.zero);
@@ -237,74 +260,117 @@ decode_tc_kernel(const __grid_constant__ DecodeTcArgs a, const __grid_constant__
     }
   }
 
+  // phi(q), phi(k_old) and the incoming token's logit (Section 2.1), while the first pieces are on their way
+  for (int r = warp; r <= g; r += DT_WARPS) {
+    if (r < g) warp_feature_map(fq_s + r * D, q_f + r * D, lane, a.phi);
+    else warp_feature_map(fk_old, k_old, lane, a.phi);
+  }
+  if (warp == DT_WARPS - 1) {
+    for (int hh = 0; hh < g; ++hh) {
+      float x = 0.f;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) x += q_f[hh * D + lane + 32 * i] * k_new[lane + 32 * i];
+      x = warp_sum(x);
+      if (lane == 0) l_new[hh] = x * a.scale;
+    }
+  }
+
   int pc = 0;                                                    // pieces consumed so far
   bool ok = true;
   // ---- q K^T over the ring: piece = 64 slots, warp = 8 of them --------------------------------
+  float my_max = -INFINITY;                                      // over this thread's logits (head lane / 4)
   for (int j = 0; j < np && ok; ++j, ++pc) {
-    const bool got = mbar_wait_warp(&full[pc % DT_STAGES], (uint32_t)(pc / DT_STAGES) & 1u, abort);
+    const bool got = mbar_wait_warp(&full[pc % NS], (uint32_t)(pc / NS) & 1u, abort);
     if (got) {
-      const uint32_t base = smem_u32(sm + (pc % DT_STAGES) * DT_PIECE);
+      const uint32_t base = smem_u32(sm + (pc % NS) * DT_PIECE);
       const int row = 8 * warp + (lane & 7);
-      float c[4] = {0.f, 0.f, 0.f, 0.f};
+      float c[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int kk0 = 0; kk0 < 8; kk0 += 2) {
         const int chunk = (kk0 + (lane >> 4)) * 2 + ((lane >> 3) & 1);
         uint32_t kb[4];
         ldmatrix_x4(base + (chunk >> 3) * (DT_PIECE / 2) + row * 128 + (((chunk & 7) ^ (row & 7)) << 4), kb);
         mma_16816(c, qa[kk0], kb[0], kb[1]);
-        mma_16816(c, qa[kk0 + 1], kb[2], kb[3]);
+        mma_16816(c2, qa[kk0 + 1], kb[2], kb[3]);
       }
       const int hh = lane >> 2, s = j * 64 + 8 * warp + 2 * (lane & 3);
       if (hh < g) {
-        logit[hh * LS + s] = c[0] * a.scale;
-        logit[hh * LS + s + 1] = c[1] * a.scale;
+        const float l0 = (c[0] + c2[0]) * a.scale, l1 = (c[1] + c2[1]) * a.scale;
+        logit[hh * LS + s] = l0;
+        logit[hh * LS + s + 1] = l1;
+        if (s < n_valid) my_max = fmaxf(my_max, l0);             // a slot without a token may hold anything
+        if (s + 1 < n_valid) my_max = fmaxf(my_max, l1);
       }
     }
     ok = __syncthreads_and(got) != 0;
-    if (ok && warp == 0 && pc + DT_STAGES < n_pieces) issue(pc + DT_STAGES);
+    if (ok && warp == 0 && pc + NS < n_pieces) issue(pc + NS);
   }
-  if (np == 0) __syncthreads();                                  // l_new, p rows
-
-  // ---- softmax over the window, one warp per head; weights as a bf16 pair -------------------------
-  if (ok && warp < g) {
-    float* lh = logit + warp * LS;
-    float m = l_new[warp];
-    for (int s = lane; s < n_valid; s += 32) m = fmaxf(m, lh[s]);
-    m = warp_max(m);
-    float l = 0.f;
-    for (int s = lane; s < n_valid; s += 32) {
-      const float e = __expf(lh[s] - m);
-      l += e;
-      const __nv_bfloat16 hi = __float2bfloat16_rn(e);
-      p_hi[warp * PS + s] = hi;
-      p_lo[warp * PS + s] = __float2bfloat16_rn(e - __bfloat162float(hi));
-    }
-    l = warp_sum(l);
-    const float en = __expf(l_new[warp] - m);
-    if (lane == 0) {
-      p_new[warp] = en;
-      inv_sum[warp] = 1.f / (l + en);
-    }
-  }
+  my_max = fmaxf(my_max, __shfl_xor_sync(0xffffffffu, my_max, 1));
+  my_max = fmaxf(my_max, __shfl_xor_sync(0xffffffffu, my_max, 2));
+  if ((lane & 3) == 0) w_max[warp * 8 + (lane >> 2)] = my_max;
   __syncthreads();
 
-  // ---- P V: piece = 64 slots of V, warp = 16 of the 128 value features ------------------------------
-  float o[2][4];
+  // ---- softmax over the window: thread = slot, all heads; weights as a bf16 pair ------------------
+  {
+    float m[G], l[G];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) o[i >> 2][i & 3] = 0.f;
+    for (int hh = 0; hh < G; ++hh) {
+      l[hh] = 0.f;
+      m[hh] = hh < g ? l_new[hh] : 0.f;
+#pragma unroll
+      for (int wv = 0; wv < DT_WARPS; ++wv) m[hh] = fmaxf(m[hh], w_max[wv * 8 + hh]);
+    }
+    for (int s = tid; s < n_valid; s += DT_THREADS) {
+#pragma unroll
+      for (int hh = 0; hh < G; ++hh) {
+        if (hh < g) {
+          const float e = __expf(logit[hh * LS + s] - m[hh]);
+          l[hh] += e;
+          const __nv_bfloat16 hi = __float2bfloat16_rn(e);
+          p_hi[hh * PS + s] = hi;
+          p_lo[hh * PS + s] = __float2bfloat16_rn(e - __bfloat162float(hi));
+        }
+      }
+    }
+#pragma unroll
+    for (int hh = 0; hh < G; ++hh) {
+      l[hh] = warp_sum(l[hh]);
+      if (lane == 0) w_sum[warp * 8 + hh] = l[hh];
+    }
+    __syncthreads();
+    if (tid < g) {
+      float tot = 0.f;
+#pragma unroll
+      for (int wv = 0; wv < DT_WARPS; ++wv) tot += w_sum[wv * 8 + tid];
+      float mm = l_new[tid];
+#pragma unroll
+      for (int wv = 0; wv < DT_WARPS; ++wv) mm = fmaxf(mm, w_max[wv * 8 + tid]);
+      const float en = __expf(l_new[tid] - mm);
+      p_new[tid] = en;
+      inv_sum[tid] = 1.f / (tot + en);
+    }
+    __syncthreads();
+  }
+
+  // ---- P V: piece = 64 slots of V, warp = 16 of the 128 value features.  Rows 0..7 of the weight
+  // fragment carry the leading parts, rows 8..15 the remainders: one product gives both.
+  float o[2][2][4];                                              // [slot-step parity][feature tile][fragment]
+#pragma unroll
+  for (int i = 0; i < 16; ++i) o[i >> 3][(i >> 2) & 1][i & 3] = 0.f;
   for (int j = 0; j < np && ok; ++j, ++pc) {
-    const bool got = mbar_wait_warp(&full[pc % DT_STAGES], (uint32_t)(pc / DT_STAGES) & 1u, abort);
+    const bool got = mbar_wait_warp(&full[pc % NS], (uint32_t)(pc / NS) & 1u, abort);
     if (got) {
-      unsigned char* piece = sm + (pc % DT_STAGES) * DT_PIECE;
+      unsigned char* piece = sm + (pc % NS) * DT_PIECE;
       const uint32_t base = smem_u32(piece);
       const bool upper = (lane >> 3) & 1;
       const int chunk = 2 * warp + (lane >> 4);
       const int live = n_valid - j * 64;                         // slots of this piece that hold a token
+      const __nv_bfloat16* p_part = (upper ? p_lo : p_hi) + (lane & 7) * PS + j * 64 + (lane >> 4) * 8;
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks) {
         if (ks * 16 >= live) break;                              // nothing but zero weights from here on
         const int row = ks * 16 + (lane & 7) + (upper ? 8 : 0);
-        uint32_t vb[4], ph[4], pl[4];
+        uint32_t vb[4], pa[4];
         ldmatrix_x4_trans(base + (chunk >> 3) * (DT_PIECE / 2) + row * 128 + (((chunk & 7) ^ (row & 7)) << 4), vb);
         if (live < 64) {
           // a slot without a token may hold anything; its weight is zero, but 0 * NaN is not
@@ -314,17 +380,13 @@ decode_tc_kernel(const __grid_constant__ DecodeTcArgs a, const __grid_constant__
           vb[1] = keep_valid(vb[1], s0 + 8, live);
           vb[3] = keep_valid(vb[3], s0 + 8, live);
         }
-        const int pcol = j * 64 + ks * 16 + (lane >> 4) * 8;
-        ldmatrix_x4(upper ? zero_addr : smem_u32(p_hi + (lane & 7) * PS + pcol), ph);
-        ldmatrix_x4(upper ? zero_addr : smem_u32(p_lo + (lane & 7) * PS + pcol), pl);
-        mma_16816(o[0], ph, vb[0], vb[1]);
-        mma_16816(o[1], ph, vb[2], vb[3]);
-        mma_16816(o[0], pl, vb[0], vb[1]);
-        mma_16816(o[1], pl, vb[2], vb[3]);
+        ldmatrix_x4((lane & 7) >= g ? zero_addr : smem_u32(p_part + ks * 16), pa);
+        mma_16816(o[ks & 1][0], pa, vb[0], vb[1]);
+        mma_16816(o[ks & 1][1], pa, vb[2], vb[3]);
       }
     }
     ok = __syncthreads_and(got) != 0;
-    if (ok && warp == 0 && pc + DT_STAGES < n_pieces) issue(pc + DT_STAGES);
+    if (ok && warp == 0 && pc + NS < n_pieces) issue(pc + NS);
   }
   if (ok) {
     const int hh = lane >> 2;
@@ -332,9 +394,16 @@ decode_tc_kernel(const __grid_constant__ DecodeTcArgs a, const __grid_constant__
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt) {
         const int c = 16 * warp + 8 * nt + 2 * (lane & 3);
-        o_swa[hh * D + c] = (o[nt][0] + p_new[hh] * v_new[c]) * inv_sum[hh];
-        o_swa[hh * D + c + 1] = (o[nt][1] + p_new[hh] * v_new[c + 1]) * inv_sum[hh];
+        const float x0 = o[0][nt][0] + o[0][nt][2] + o[1][nt][0] + o[1][nt][2];
+        const float x1 = o[0][nt][1] + o[0][nt][3] + o[1][nt][1] + o[1][nt][3];
+        o_swa[hh * D + c] = (x0 + p_new[hh] * v_new[c]) * inv_sum[hh];
+        o_swa[hh * D + c + 1] = (x1 + p_new[hh] * v_new[c + 1]) * inv_sum[hh];
       }
+    }
+    // the incoming token takes the evicted token's slot: every piece of the ring has been consumed
+    if (tid < D) {
+      kr[(size_t)slot * D + tid] = kn;
+      vr[(size_t)slot * D + tid] = vn;
     }
   }
 
@@ -347,9 +416,9 @@ decode_tc_kernel(const __grid_constant__ DecodeTcArgs a, const __grid_constant__
     for (int hh = 0; hh < G; ++hh) ar[hh] = make_float4(0.f, 0.f, 0.f, 0.f);
     const float4 vo = *reinterpret_cast<const float4*>(v_old + c4 * 4);
     for (int i = 0; i < 4 && ok; ++i, ++pc) {
-      const bool got = mbar_wait_warp(&full[pc % DT_STAGES], (uint32_t)(pc / DT_STAGES) & 1u, abort);
+      const bool got = mbar_wait_warp(&full[pc % NS], (uint32_t)(pc / NS) & 1u, abort);
       if (got) {
-        const float* piece = reinterpret_cast<const float*>(sm + (pc % DT_STAGES) * DT_PIECE);
+        const float* piece = reinterpret_cast<const float*>(sm + (pc % NS) * DT_PIECE);
 #pragma unroll
         for (int m = 0; m < 4; ++m) {
           const int rp = rl + 8 * m, r = 32 * i + rp;
@@ -367,7 +436,7 @@ decode_tc_kernel(const __grid_constant__ DecodeTcArgs a, const __grid_constant__
         }
       }
       ok = __syncthreads_and(got) != 0;
-      if (ok && warp == 0 && pc + DT_STAGES < n_pieces) issue(pc + DT_STAGES);
+      if (ok && warp == 0 && pc + NS < n_pieces) issue(pc + NS);
     }
 #pragma unroll
     for (int hh = 0; hh < G; ++hh) {
@@ -386,8 +455,8 @@ decode_tc_kernel(const __grid_constant__ DecodeTcArgs a, const __grid_constant__
   if (!ok) {
     // a wait ran out: give what is still in flight a bounded time to land, report, leave the caches alone
     if (tid == 0) {
-      for (int p = pc; p < n_pieces && p < pc + DT_STAGES; ++p)
-        for (int it = 0; it < kWaitPolls && !mbar_try_wait(&full[p % DT_STAGES], (uint32_t)(p / DT_STAGES) & 1u); ++it) {}
+      for (int p = pc; p < n_pieces && p < pc + NS; ++p)
+        for (int it = 0; it < kWaitPolls && !mbar_try_wait(&full[p % NS], (uint32_t)(p / NS) & 1u); ++it) {}
       g_decode_status = RATTN_ERR_TIMEOUT;
     }
     return;
@@ -414,11 +483,6 @@ decode_tc_kernel(const __grid_constant__ DecodeTcArgs a, const __grid_constant__
       const float gr = a.gamma_rla ? a.gamma_rla[(size_t)h * D + c] : 1.f;
       og[(size_t)warp * D + c] = __float2bfloat16_rn(gs * x[i] * is + gr * y[i] * ir);
     }
-  }
-  // the incoming token takes the evicted token's slot (every piece of the ring has been consumed)
-  if (tid < D) {
-    kr[(size_t)slot * D + tid] = kg[tid];
-    vr[(size_t)slot * D + tid] = vg[tid];
   }
 }
 
@@ -455,7 +519,8 @@ cudaError_t launch_decode_tc(const Args& p, void* k_ring, void* v_ring, float* s
   if (!tc::make_map(&m.k, k_ring, (uint64_t)p.w, (uint64_t)p.B * p.H_kv, 64) ||
       !tc::make_map(&m.v, v_ring, (uint64_t)p.w, (uint64_t)p.B * p.H_kv, 64))
     return cudaErrorInvalidValue;
-  const int smem = plan(p.group, p.w).total;
+  a.stages = tuning(RATTN_TUNE_DECODE_STAGES);
+  const int smem = plan(p.group, p.w, a.stages).total;
   if (p.group == 1) return launch_g<1>(a, m, smem, s);
   if (p.group == 2) return launch_g<2>(a, m, smem, s);
   if (p.group <= 4) return launch_g<4>(a, m, smem, s);

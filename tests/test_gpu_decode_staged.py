@@ -60,7 +60,6 @@ def run_steps(wl, T0, steps, poison=False, phi=R.PHI_SOFTMAX, flags=0):
 ])
 def test_staged_decode_after_prefill(w, Hq, Hkv, T0, steps, poison):
     wl = small("dst", 2, Hq, Hkv, T0 + steps, 128, w, "bf16", 7000 + w + Hq, unit=True)
-    assert R.rattn_uses_tensor_path(128, w, R.RATTN_BF16, R.MODE_RATTN)
     y, ref = run_steps(wl, T0, steps, poison)
     check(y, ref, "bf16", f"w={w} g={Hq // Hkv}")
 
