@@ -459,7 +459,7 @@ def run_ours(args, wl):
         "tokens_per_s": c5.B / (ms_d * 1e-3),
         "roofline_denominator": f"{pk['hbm']} GB/s HBM copy, {pk['src']}",
     }
-    del rings
+    torch.cuda.empty_cache()
     result["extra"] = extra
 
     # ---- end to end: host buffers in, gradients out, through the same calls ----------
