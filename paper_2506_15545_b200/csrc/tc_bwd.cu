@@ -60,121 +60,227 @@ struct BwdArgs {
   do { if (!mbar_wait_warp(&(bar), (parity), &bars->abort)) return false; } while (0)
 
 // ------------------------------------------------------------------------------ prep
-// One warp per row; lane owns 4 consecutive features.  Writes g_s, g_r (bf16), D and, when
-// asked, accumulates the gain gradients.
-__global__ void __launch_bounds__(256)
-tc_bwd_prep_kernel(const __nv_bfloat16* __restrict__ dy, const __nv_bfloat16* __restrict__ o_s,
-                   const __nv_bfloat16* __restrict__ o_r, const float* __restrict__ gamma_s,
-                   const float* __restrict__ gamma_r, __nv_bfloat16* __restrict__ g_s,
-                   __nv_bfloat16* __restrict__ g_r, float* __restrict__ delta, float* __restrict__ dgamma_s,
-                   float* __restrict__ dgamma_r, const float* __restrict__ lse, float* __restrict__ lse2p,
-                   float* __restrict__ dscp, size_t n_rows_pad, int T, int t_pad, int H_q, float eps, float scale,
-                   int rla_on) {
-  // Half a warp per row, a lane owns 8 consecutive features; the 64 rows of a CTA lie inside one
-  // (batch, head) pair because t_pad is a multiple of 128.  With n = o / r (r the rms incl. eps),
-  // gh = dy * gain, A = gh . o:   g = (gh - n * (A / (128 r))) / r,   D = g . o = (A - A ss / (128 r^2)) / r,
-  // so each branch needs two row sums (ss = o . o and A), all four reduced in one shuffle round.
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int sub = lane >> 4, l16 = lane & 15;
-  constexpr int ROWS_PER_CTA = 64;
-  const size_t row0 = (size_t)blockIdx.x * ROWS_PER_CTA;
-  if (row0 >= n_rows_pad) return;
-  const size_t bq = row0 / t_pad;
-  const int t0 = (int)(row0 - bq * t_pad);
-  const int h = (int)(bq % H_q);
-  float gs[8], gr[8], acc_s[8], acc_r[8];
+// A pure stream: dO and the two un-normalised branch outputs in, g_s and g_r out (bf16), plus the
+// per-row statistics; bound by HBM.  The unit is a chunk of 32 rows of one head (8 KB per tensor,
+// contiguous), which travels global -> shared -> global as bulk asynchronous copies through a ring
+// of stages, so the bytes in flight do not depend on where the warps are; the rows are transformed
+// in place in shared memory (g_s over o_swa, g_r over o_rla).  Eight neighbouring lanes hold a row:
+// lane l has features [8l, 8l+8) and [64+8l, 64+8l+8).  Every CTA takes an equal contiguous share of
+// the chunks (head-major), so it meets few heads and keeps its gain-gradient sums in registers.
+// With n = o / r (r the rms incl. eps), gh = dy * gain, A = gh . o:
+//   g = (gh - n * (A / (128 r))) / r,   D = g . o = (A - A ss / (128 r^2)) / r,
+// so each branch needs two row sums (ss = o . o and A).
+constexpr int PREP_THREADS = 256;
+constexpr int PREP_ROWS = 32;                       // rows of a chunk
+constexpr int PREP_CHUNK = PREP_ROWS * 256;         // bytes of a chunk of one tensor
+constexpr int PREP_STAGES = 4;
+constexpr int PREP_SMEM = PREP_STAGES * 3 * PREP_CHUNK + 128;
+
+struct PrepArgs {
+  const __nv_bfloat16* dy; const __nv_bfloat16* o_s; const __nv_bfloat16* o_r;
+  const float* gamma_s; const float* gamma_r;
+  __nv_bfloat16* g_s; __nv_bfloat16* g_r;
+  float* delta; float* dgamma_s; float* dgamma_r;
+  const float* lse; float* lse2p; float* dscp;
+  int* status;
+  int n_heads, T, t_pad, H_q, rla_on;
+  float eps, scale;
+};
+
+__device__ __forceinline__ void unpack8(const unsigned char* p, float (&x)[8]) {
+  const uint4 u = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
-  for (int e = 0; e < 8; ++e) {
-    gs[e] = gamma_s ? __ldg(gamma_s + (size_t)h * 128 + 8 * l16 + e) : 1.f;
-    gr[e] = gamma_r ? __ldg(gamma_r + (size_t)h * 128 + 8 * l16 + e) : 1.f;
-    acc_s[e] = 0.f;
-    acc_r[e] = 0.f;
+  for (int i = 0; i < 4; ++i) {
+    x[2 * i] = __uint_as_float(w[i] << 16);
+    x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
   }
-  // The kernel is a pure stream (three tensors in, two out), so what matters is how many loads are in
-  // flight: the next row's three loads are issued before the current row is worked on.
-  const uint4 zero4 = make_uint4(0, 0, 0, 0);
-  uint4 us_n = zero4, ur_n = zero4, gy_n = zero4;
-  auto issue = [&](int rr) {
-    const int t = t0 + rr;
-    if (rr < ROWS_PER_CTA && t < T) {
-      const size_t row = bq * T + t;
-      us_n = *reinterpret_cast<const uint4*>(o_s + row * 128 + 8 * l16);
-      ur_n = *reinterpret_cast<const uint4*>(o_r + row * 128 + 8 * l16);
-      gy_n = *reinterpret_cast<const uint4*>(dy + row * 128 + 8 * l16);
+}
+
+__global__ void __launch_bounds__(PREP_THREADS, 2) tc_bwd_prep_kernel(const __grid_constant__ PrepArgs a) {
+  extern __shared__ __align__(128) unsigned char psm[];
+  uint64_t* full = reinterpret_cast<uint64_t*>(psm + PREP_STAGES * 3 * PREP_CHUNK);
+  volatile int* abort = reinterpret_cast<volatile int*>(full + PREP_STAGES);
+  const int tid = threadIdx.x, l = tid & 7, row = tid >> 3;
+  const int cph = a.t_pad / PREP_ROWS;                              // chunks per head
+  const long long n_all = (long long)a.n_heads * cph;
+  const int lo = (int)(n_all * blockIdx.x / gridDim.x), hi = (int)(n_all * (blockIdx.x + 1) / gridDim.x);
+  const int n_in = a.rla_on ? 3 : 2;                                // tensors read per chunk
+
+  if (tid == 0) {
+    for (int i = 0; i < PREP_STAGES; ++i) mbar_init(&full[i], 1);
+    *abort = 0;
+    fence_mbar_init();
+  }
+  __syncthreads();
+
+  // chunk i: head i / cph, rows t0 .. t0 + 31 of it; rows at or beyond T are padding (nothing is copied)
+  auto rows_of = [&](int i) { const int t0 = (i % cph) * PREP_ROWS; return a.T - t0 < 0 ? 0 : a.T - t0 < PREP_ROWS ? a.T - t0 : PREP_ROWS; };
+  // Thread 0 keeps the ring fed: the next chunk with data goes into stage (chunks issued so far) % stages.
+  int cursor = lo, n_issued = 0;
+  auto issue_next = [&]() {
+    while (cursor < hi && rows_of(cursor) == 0) ++cursor;
+    if (cursor >= hi) return;
+    const int i = cursor++, rows = rows_of(i);
+    const size_t at = ((size_t)(i / cph) * a.T + (size_t)(i % cph) * PREP_ROWS) * 128;
+    unsigned char* dst = psm + (size_t)(n_issued % PREP_STAGES) * 3 * PREP_CHUNK;
+    uint64_t* bar = &full[n_issued % PREP_STAGES];
+    ++n_issued;
+    const uint32_t bytes = (uint32_t)rows * 256;
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes * n_in) : "memory");
+    const __nv_bfloat16* src[3] = {a.dy, a.o_s, a.o_r};
+    for (int k = 0; k < n_in; ++k)
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                   ::"r"(smem_u32(dst + k * PREP_CHUNK)), "l"(src[k] + at), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+  };
+  if (tid == 0)
+    for (int k = 0; k < PREP_STAGES - 1; ++k) issue_next();
+
+  float gs_lo[8], gs_hi[8], gr_lo[8], gr_hi[8], acc_s[16], acc_r[16];
+#pragma unroll
+  for (int e = 0; e < 16; ++e) acc_s[e] = acc_r[e] = 0.f;
+  int cur_h = -1;
+  auto flush = [&]() {                                              // this CTA's sums for head cur_h
+    if (cur_h < 0) return;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      if (a.dgamma_s) {
+        atomicAdd(a.dgamma_s + (size_t)cur_h * 128 + 8 * l + e, acc_s[e]);
+        atomicAdd(a.dgamma_s + (size_t)cur_h * 128 + 64 + 8 * l + e, acc_s[8 + e]);
+      }
+      if (a.dgamma_r && a.rla_on) {
+        atomicAdd(a.dgamma_r + (size_t)cur_h * 128 + 8 * l + e, acc_r[e]);
+        atomicAdd(a.dgamma_r + (size_t)cur_h * 128 + 64 + 8 * l + e, acc_r[8 + e]);
+      }
+      acc_s[e] = acc_s[8 + e] = acc_r[e] = acc_r[8 + e] = 0.f;
     }
   };
-  issue(2 * warp + sub);
-#pragma unroll 1
-  for (int rr = 2 * warp + sub; rr < ROWS_PER_CTA; rr += 16) {
-    const int t = t0 + rr;
-    const size_t prow = bq * t_pad + t;
-    const uint4 us = us_n, ur = ur_n, gy = gy_n;
-    issue(rr + 16);
-    if (t >= T) {                                  // padding: statistics that make every weight zero
-      if (l16 == 0) {
-        lse2p[prow] = INFINITY;
-        dscp[prow] = 0.f;
-      }
+
+  int i = lo, n_cons = 0;                                           // n_cons: chunks with data consumed so far
+  bool ok = true;
+  for (; i < hi; ++i) {
+    const int bq = i / cph, t0 = (i % cph) * PREP_ROWS, rows = rows_of(i);
+    const int t = t0 + row;
+    const size_t prow = (size_t)bq * a.t_pad + t;
+    if (rows == 0) {                                                // padding only: statistics that make every weight zero
+      if (l == 0) { a.lse2p[prow] = INFINITY; a.dscp[prow] = 0.f; }
       continue;
     }
-    const size_t row = bq * T + t;
-    float vs[8], vr[8], g[8];
-    {
-      const __nv_bfloat162* ps = reinterpret_cast<const __nv_bfloat162*>(&us);
-      const __nv_bfloat162* pr = reinterpret_cast<const __nv_bfloat162*>(&ur);
-      const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&gy);
+    const int h = bq % a.H_q;
+    if (h != cur_h) {
+      if (a.dgamma_s || a.dgamma_r) flush();
+      cur_h = h;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 fs = __bfloat1622float2(ps[e]), fr = __bfloat1622float2(pr[e]), f = __bfloat1622float2(hp[e]);
-        vs[2 * e] = fs.x; vs[2 * e + 1] = fs.y;
-        vr[2 * e] = fr.x; vr[2 * e + 1] = fr.y;
-        g[2 * e] = f.x;   g[2 * e + 1] = f.y;
+      for (int e = 0; e < 8; ++e) {
+        gs_lo[e] = a.gamma_s ? __ldg(a.gamma_s + (size_t)h * 128 + 8 * l + e) : 1.f;
+        gs_hi[e] = a.gamma_s ? __ldg(a.gamma_s + (size_t)h * 128 + 64 + 8 * l + e) : 1.f;
+        gr_lo[e] = a.gamma_r ? __ldg(a.gamma_r + (size_t)h * 128 + 8 * l + e) : 1.f;
+        gr_hi[e] = a.gamma_r ? __ldg(a.gamma_r + (size_t)h * 128 + 64 + 8 * l + e) : 1.f;
       }
     }
-    float ss = 0.f, sr = 0.f, As = 0.f, Ar = 0.f;
+    const int slot = n_cons % PREP_STAGES;
+    unsigned char* buf = psm + (size_t)slot * 3 * PREP_CHUNK + row * 256 + 16 * l;
+    const bool live = row < rows;
+    // the row's log-sum-exp is asked for before the wait, so that its latency passes under it
+    const float lse_row = (live && l == 0) ? __ldg(a.lse + (size_t)bq * a.T + t) : 0.f;
+    const bool got = mbar_wait_warp(&full[slot], (uint32_t)(n_cons / PREP_STAGES) & 1u, abort);
+    if (got) {
+      float g_lo[8], g_hi[8], s_lo[8], s_hi[8], r_lo[8], r_hi[8];
+      if (live) {
+        unpack8(buf, g_lo); unpack8(buf + 128, g_hi);
+        unpack8(buf + PREP_CHUNK, s_lo); unpack8(buf + PREP_CHUNK + 128, s_hi);
+      }
+      if (live && a.rla_on) { unpack8(buf + 2 * PREP_CHUNK, r_lo); unpack8(buf + 2 * PREP_CHUNK + 128, r_hi); }
+      if (!live || !a.rla_on) {
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      ss += vs[e] * vs[e];
-      sr += vr[e] * vr[e];
-      As += g[e] * gs[e] * vs[e];
-      Ar += g[e] * gr[e] * vr[e];
-    }
-    const unsigned half_mask = sub ? 0xffff0000u : 0x0000ffffu;   // the other half may be on a padding row
+        for (int e = 0; e < 8; ++e) r_lo[e] = r_hi[e] = 0.f;
+      }
+      if (!live) {
 #pragma unroll
-    for (int o = 8; o > 0; o >>= 1) {
-      ss += __shfl_xor_sync(half_mask, ss, o);
-      sr += __shfl_xor_sync(half_mask, sr, o);
-      As += __shfl_xor_sync(half_mask, As, o);
-      Ar += __shfl_xor_sync(half_mask, Ar, o);
-    }
-    const float is = rsqrtf(ss * (1.f / 128.f) + eps), ir = rsqrtf(sr * (1.f / 128.f) + eps);
-    const float cs = As * is * is * (1.f / 128.f), cr = Ar * ir * ir * (1.f / 128.f);   // mean(gh n) / r
-    uint32_t ws[4], wr[4];
+        for (int e = 0; e < 8; ++e) g_lo[e] = g_hi[e] = s_lo[e] = s_hi[e] = 0.f;
+      }
+      float ss = 0.f, sr = 0.f, As = 0.f, Ar = 0.f;
 #pragma unroll
-    for (int e = 0; e < 8; e += 2) {
-      ws[e >> 1] = pack_bf16((g[e] * gs[e] - vs[e] * cs) * is, (g[e + 1] * gs[e + 1] - vs[e + 1] * cs) * is);
-      wr[e >> 1] = pack_bf16((g[e] * gr[e] - vr[e] * cr) * ir, (g[e + 1] * gr[e + 1] - vr[e + 1] * cr) * ir);
-      acc_s[e] += g[e] * vs[e] * is;
-      acc_s[e + 1] += g[e + 1] * vs[e + 1] * is;
-      acc_r[e] += g[e] * vr[e] * ir;
-      acc_r[e + 1] += g[e + 1] * vr[e + 1] * ir;
+      for (int e = 0; e < 8; ++e) {
+        ss += s_lo[e] * s_lo[e] + s_hi[e] * s_hi[e];
+        sr += r_lo[e] * r_lo[e] + r_hi[e] * r_hi[e];
+        As += g_lo[e] * gs_lo[e] * s_lo[e] + g_hi[e] * gs_hi[e] * s_hi[e];
+        Ar += g_lo[e] * gr_lo[e] * r_lo[e] + g_hi[e] * gr_hi[e] * r_hi[e];
+      }
+#pragma unroll
+      for (int o = 1; o < 8; o <<= 1) {
+        ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        sr += __shfl_xor_sync(0xffffffffu, sr, o);
+        As += __shfl_xor_sync(0xffffffffu, As, o);
+        Ar += __shfl_xor_sync(0xffffffffu, Ar, o);
+      }
+      const float is = rsqrtf(ss * (1.f / 128.f) + a.eps), ir = rsqrtf(sr * (1.f / 128.f) + a.eps);
+      const float cs = As * is * is * (1.f / 128.f), cr = Ar * ir * ir * (1.f / 128.f);   // mean(gh n) / r
+      if (live) {
+        uint32_t w_lo[4], w_hi[4];
+#pragma unroll
+        for (int e = 0; e < 8; e += 2) {
+          w_lo[e >> 1] = pack_bf16((g_lo[e] * gs_lo[e] - s_lo[e] * cs) * is, (g_lo[e + 1] * gs_lo[e + 1] - s_lo[e + 1] * cs) * is);
+          w_hi[e >> 1] = pack_bf16((g_hi[e] * gs_hi[e] - s_hi[e] * cs) * is, (g_hi[e + 1] * gs_hi[e + 1] - s_hi[e + 1] * cs) * is);
+        }
+        *reinterpret_cast<uint4*>(buf + PREP_CHUNK) = make_uint4(w_lo[0], w_lo[1], w_lo[2], w_lo[3]);
+        *reinterpret_cast<uint4*>(buf + PREP_CHUNK + 128) = make_uint4(w_hi[0], w_hi[1], w_hi[2], w_hi[3]);
+        if (a.rla_on) {
+#pragma unroll
+          for (int e = 0; e < 8; e += 2) {
+            w_lo[e >> 1] = pack_bf16((g_lo[e] * gr_lo[e] - r_lo[e] * cr) * ir, (g_lo[e + 1] * gr_lo[e + 1] - r_lo[e + 1] * cr) * ir);
+            w_hi[e >> 1] = pack_bf16((g_hi[e] * gr_hi[e] - r_hi[e] * cr) * ir, (g_hi[e + 1] * gr_hi[e + 1] - r_hi[e + 1] * cr) * ir);
+          }
+          *reinterpret_cast<uint4*>(buf + 2 * PREP_CHUNK) = make_uint4(w_lo[0], w_lo[1], w_lo[2], w_lo[3]);
+          *reinterpret_cast<uint4*>(buf + 2 * PREP_CHUNK + 128) = make_uint4(w_hi[0], w_hi[1], w_hi[2], w_hi[3]);
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          acc_s[e] += g_lo[e] * s_lo[e] * is;
+          acc_s[8 + e] += g_hi[e] * s_hi[e] * is;
+          acc_r[e] += g_lo[e] * r_lo[e] * ir;
+          acc_r[8 + e] += g_hi[e] * r_hi[e] * ir;
+        }
+      }
+      if (l == 0) {
+        if (live) {
+          const size_t grow = (size_t)bq * a.T + t;
+          const float dl = (As - cs * ss) * is;                     // D_t = g_s . o_swa
+          a.delta[grow] = dl;
+          a.lse2p[prow] = lse_row * LOG2E;
+          a.dscp[prow] = dl * a.scale;
+        } else {
+          a.lse2p[prow] = INFINITY;
+          a.dscp[prow] = 0.f;
+        }
+      }
+      fence_proxy_async_smem();
     }
-    *reinterpret_cast<uint4*>(g_s + row * 128 + 8 * l16) = make_uint4(ws[0], ws[1], ws[2], ws[3]);
-    *reinterpret_cast<uint4*>(g_r + row * 128 + 8 * l16) = make_uint4(wr[0], wr[1], wr[2], wr[3]);
-    if (l16 == 0) {
-      const float dl = (As - cs * ss) * is;        // D_t = g_s . o_swa
-      delta[row] = dl;
-      lse2p[prow] = lse[row] * LOG2E;
-      dscp[prow] = dl * scale;
+    ok = __syncthreads_and(got) != 0;
+    if (!ok) break;
+    if (tid == 0) {
+      const size_t at = ((size_t)bq * a.T + t0) * 128;
+      unsigned char* src = psm + (size_t)slot * 3 * PREP_CHUNK;
+      const uint32_t bytes = (uint32_t)rows * 256;
+      asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(a.g_s + at), "r"(smem_u32(src + PREP_CHUNK)), "r"(bytes) : "memory");
+      if (a.rla_on)
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(a.g_r + at), "r"(smem_u32(src + 2 * PREP_CHUNK)), "r"(bytes) : "memory");
+      tma_store_commit();
+      asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the stage of the chunk before this one has been read out
+      issue_next();
+    }
+    ++n_cons;
+  }
+  if (tid == 0) {
+    tma_store_wait();
+    if (!ok) {
+      // give the copies still in flight a bounded time to land before the CTA's memory goes away
+      for (int n = n_cons; n < n_issued; ++n)
+        for (int it = 0; it < kWaitPolls && !mbar_try_wait(&full[n % PREP_STAGES], (uint32_t)(n / PREP_STAGES) & 1u); ++it) {}
+      atomicExch(a.status, RATTN_ERR_TIMEOUT);
     }
   }
-  if (dgamma_s || dgamma_r) {
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      if (dgamma_s) atomicAdd(dgamma_s + (size_t)h * 128 + 8 * l16 + e, acc_s[e]);
-      if (dgamma_r && rla_on) atomicAdd(dgamma_r + (size_t)h * 128 + 8 * l16 + e, acc_r[e]);
-    }
-  }
+  if (ok && (a.dgamma_s || a.dgamma_r)) flush();
 }
 
 // ================================================================================ dq
@@ -1046,14 +1152,27 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
     if (e != cudaSuccess) return e;
   }
   const int t_pad = a.n_chunks * TILE;
-  const size_t n_rows_pad = (size_t)a.B * a.H_q * t_pad;
   {
+    PrepArgs pa;
+    pa.dy = reinterpret_cast<const __nv_bfloat16*>(a.dout);
+    pa.o_s = reinterpret_cast<const __nv_bfloat16*>(a.o_swa);
+    pa.o_r = reinterpret_cast<const __nv_bfloat16*>(a.o_rla);
+    pa.gamma_s = a.gamma_swa; pa.gamma_r = a.gamma_rla;
+    pa.g_s = g_s; pa.g_r = g_r;
+    pa.delta = a.delta; pa.dgamma_s = a.dgamma_swa; pa.dgamma_r = a.dgamma_rla;
+    pa.lse = a.lse; pa.lse2p = a.lse2p; pa.dscp = a.dscp;
+    pa.status = a.status;
+    pa.n_heads = a.B * a.H_q; pa.T = a.T; pa.t_pad = t_pad; pa.H_q = a.H_q; pa.rla_on = rla_on ? 1 : 0;
+    pa.eps = a.eps; pa.scale = a.scale;
+    int dev = 0, n_sm = 0;
+    e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_bwd_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PREP_SMEM);
+    if (e != cudaSuccess) return e;
+    const long long n_chunks_all = (long long)pa.n_heads * (t_pad / PREP_ROWS);
+    const int grid = (int)(n_chunks_all < 2ll * n_sm ? n_chunks_all : 2ll * n_sm);
     KernelTimer kt("tc_bwd_prep", s);
-    tc_bwd_prep_kernel<<<(unsigned)((n_rows_pad + 63) / 64), 256, 0, s>>>(
-        reinterpret_cast<const __nv_bfloat16*>(a.dout), reinterpret_cast<const __nv_bfloat16*>(a.o_swa),
-        reinterpret_cast<const __nv_bfloat16*>(a.o_rla), a.gamma_swa, a.gamma_rla, g_s, g_r,
-        a.delta, a.dgamma_swa, a.dgamma_rla, a.lse, a.lse2p, a.dscp, n_rows_pad, a.T, t_pad, a.H_q, a.eps, a.scale,
-        rla_on ? 1 : 0);
+    tc_bwd_prep_kernel<<<grid, PREP_THREADS, PREP_SMEM, s>>>(pa);
   }
   count_launches(1);
 
