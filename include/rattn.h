@@ -163,7 +163,11 @@ typedef struct rattn_params {
  * (rattn_workspace_bytes_ex(..., RATTN_MODE_RATTN, 0) bytes) and obtains it with
  * cudaMallocAsync / cudaFreeAsync on `stream` (the device's stream-ordered pool; no
  * synchronisation).  Callers that must control every allocation use rattn_forward_ex
- * with their own workspace.
+ * with their own workspace.  That scratch, and the status word in it, are gone when the call
+ * returns, so the word is latched into the library before the scratch is freed:
+ * rattn_forward_status (synchronises the stream) returns RATTN_ERR_TIMEOUT if a bounded
+ * device-side wait has expired in any rattn_forward call on the current device since it was
+ * last asked, else RATTN_OK.
  */
 int rattn_forward(const void* q, const void* k, const void* v,
                   int B, int H_q, int H_kv, int T, int d, int w,
@@ -205,6 +209,7 @@ int rattn_static_status(void* stream);
 
 /* Forward with the full parameter block (dtype, scale, gains, mode, workspace,
  * residuals for the backward, prefill -> decode hand-off). */
+int rattn_forward_status(void* stream);
 int rattn_forward_ex(const rattn_params* p, void* stream);
 
 /*

@@ -26,7 +26,7 @@ EXPORTS = (
     "rattn_read_status", "rattn_strerror", "rattn_last_cuda_error", "rattn_launch_count",
     "rattn_uses_tensor_path", "rattn_timing_enable", "rattn_timing_read",
     "rattn_forward_static", "rattn_static_status", "rattn_tune",
-    "rattn_qk_prologue", "rattn_qk_prologue_backward", "rattn_qk_prologue_workspace_bytes", "rattn_qk_prologue_status", "rattn_decode_status",
+    "rattn_qk_prologue", "rattn_qk_prologue_backward", "rattn_qk_prologue_workspace_bytes", "rattn_qk_prologue_status", "rattn_decode_status", "rattn_forward_status",
 )
 TUNE_STATE_STRIDE, TUNE_OVERLAP, TUNE_UNIT_ORDER, TUNE_GRID, TUNE_DECODE_STAGES = 0, 1, 2, 3, 4
 
@@ -128,6 +128,8 @@ def lib() -> ctypes.CDLL:
     L.rattn_qk_prologue_backward.restype = ci
     L.rattn_qk_prologue_workspace_bytes.argtypes = [ci, ci, ci, ci, ci]
     L.rattn_qk_prologue_workspace_bytes.restype = ctypes.c_size_t
+    L.rattn_forward_status.argtypes = [vp]
+    L.rattn_forward_status.restype = ci
     L.rattn_decode_status.argtypes = [vp]
     L.rattn_decode_status.restype = ci
     L.rattn_qk_prologue_status.argtypes = [vp]
@@ -375,6 +377,11 @@ def _qk_params(q, k, q_out, k_out, q_gain, k_gain, theta, eps, pos0, pos):
 
 def rattn_qk_prologue_workspace_bytes(B, H_q, H_kv, T, d) -> int:
     return int(lib().rattn_qk_prologue_workspace_bytes(B, H_q, H_kv, T, d))
+
+
+def rattn_forward_status(stream=None) -> int:
+    """RATTN_ERR_TIMEOUT if a bounded wait expired in a rattn_forward call since the last query."""
+    return int(lib().rattn_forward_status(_stream(stream)))
 
 
 def rattn_decode_status(stream=None) -> int:

@@ -269,10 +269,34 @@ static int backward_impl(const rattn_params* p, cudaStream_t s) {
 
 using namespace rattn;
 
+namespace {
+// rattn_forward's scratch, status word included, is freed before the call returns: a one-thread
+// kernel copies a non-zero word into this one first (sticky until rattn_forward_status reads it).
+__device__ int g_forward_status;
+__global__ void latch_status_kernel(const int* word) {
+  if (*word != 0) g_forward_status = *word;
+}
+
+}  // namespace
+
 extern "C" {
 
 int rattn_forward_ex(const rattn_params* p, void* stream) {
   return forward_impl(p, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int rattn_forward_status(void* stream) {
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  int word = 0;
+  cudaError_t e = cudaMemcpyFromSymbolAsync(&word, g_forward_status, sizeof(int), 0, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e == cudaSuccess && word != 0) {
+    const int zero = 0;
+    e = cudaMemcpyToSymbolAsync(g_forward_status, &zero, sizeof(int), 0, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  }
+  if (e != cudaSuccess) return fail_cuda(e);
+  return word == 0 ? RATTN_OK : RATTN_ERR_TIMEOUT;
 }
 
 int rattn_forward(const void* q, const void* k, const void* v, int B, int H_q, int H_kv, int T,
@@ -296,6 +320,10 @@ int rattn_forward(const void* q, const void* k, const void* v, int B, int H_q, i
   p.workspace = ws;
   p.workspace_bytes = bytes;
   rc = forward_impl(&p, s);
+  if (rc == RATTN_OK) {
+    latch_status_kernel<<<1, 1, 0, s>>>(static_cast<const int*>(ws));
+    count_launches(1);
+  }
   e = cudaFreeAsync(ws, s);
   if (rc == RATTN_OK && e != cudaSuccess) return fail_cuda(e);
   return rc;

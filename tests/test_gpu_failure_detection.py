@@ -68,3 +68,33 @@ def test_expired_wait_is_reported_and_the_context_stays_usable(dbg):
     y = R.rattn_forward_ex(qd, kd, vd, wl.w, scale=wl.scale, workspace=ws)
     assert R.rattn_read_status(ws) == 0
     assert torch.equal(y, out)
+
+
+def test_plain_forward_latches_its_status_before_freeing_its_scratch(dbg):
+    """rattn_forward takes its scratch from the stream-ordered pool and frees it before it returns, so
+    the status word in it is copied into the library first: rattn_forward_status reports the expired
+    wait, is clear again afterwards, and the next call is correct."""
+    vp, ci = ctypes.c_void_p, ctypes.c_int
+    dbg.rattn_forward.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, vp, vp]
+    dbg.rattn_forward.restype = ci
+    dbg.rattn_forward_status.argtypes = [vp]
+    dbg.rattn_forward_status.restype = ci
+    wl = small("fdp", 1, 1, 1, 256, 128, 128, "bf16", 8200, unit=True, scale=1.0)
+    q, k, v = W.make_qkv(wl)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    out = torch.zeros_like(qd)
+    stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    call = lambda: dbg.rattn_forward(qd.data_ptr(), kd.data_ptr(), vd.data_ptr(), 1, 1, 1, wl.T, 128, wl.w,
+                                     out.data_ptr(), stream)
+    assert dbg.rattn_forward_status(stream) == 0
+    dbg.rattn_debug_withhold_arrival(1)
+    assert call() == 0
+    assert dbg.rattn_forward_status(stream) == RATTN_ERR_TIMEOUT
+    assert dbg.rattn_forward_status(stream) == 0          # reading clears it
+    dbg.rattn_debug_withhold_arrival(0)
+    assert call() == 0
+    assert dbg.rattn_forward_status(stream) == 0
+    check(out, O.forward(np64(q), np64(k), np64(v), wl.w, 1.0), "bf16", "after the time-out")
+    # the product library's own word was never touched
+    y = R.rattn_forward(qd, kd, vd, wl.w)
+    assert R.rattn_forward_status() == 0 and torch.equal(y, out)
