@@ -16,6 +16,7 @@
  *   - Positions are 0-indexed.  The window holds w+1 keys including the current one.
  *   - Tensors are dense, row-major, innermost dimension d:
  *       q, out, dout, dq : [B, H_q,  T, d]      k, v, dk, dv : [B, H_kv, T, d]
+ *     (or, with rattn_params.layout = RATTN_LAYOUT_BTHD, [B, T, H_q, d] and [B, T, H_kv, d])
  *   - All data pointers are DEVICE pointers unless a parameter says "host".
  *     They must be 16-byte aligned.  The caller owns every buffer; the library
  *     keeps no reference after the call returns, allocates no device memory
@@ -65,6 +66,16 @@ typedef enum rattn_feature_map {
   RATTN_PHI_RELU = 1,            /* max(x, 0), element-wise */
   RATTN_PHI_IDENTITY = 2         /* x */
 } rattn_feature_map;
+
+/* Memory layout of the operator's tensors (rattn_params.layout).  The projections of a transformer
+ * layer produce [B, T, H * d]; RATTN_LAYOUT_BTHD reads and writes that directly (through the strides of
+ * the TMA tensor maps on the tensor-core path), so no transposing copy is needed around the operator.
+ * Applies to q, out, dout, dq (H = H_q) and k, v, dk, dv (H = H_kv) of rattn_forward_ex and
+ * rattn_backward_ex; decode tokens, rings, states and gains keep their layouts. */
+typedef enum rattn_layout {
+  RATTN_LAYOUT_BHTD = 0,         /* [B, H, T, d], the default */
+  RATTN_LAYOUT_BTHD = 1          /* [B, T, H, d] */
+} rattn_layout;
 
 /* Path selection for rattn_params.flags. */
 #define RATTN_FLAG_FORCE_GENERIC 1u  /* use the portable fp32-FMA kernels even where the
@@ -147,7 +158,7 @@ typedef struct rattn_params {
   const void* k_ring_in;         /* [B,H_kv,w,d]: tokens pos0-w .. pos0-1 at slot j % w */
   const void* v_ring_in;
   int32_t pos0;                  /* tokens that precede this call's T tokens; 0 or >= w */
-  int32_t reserved;
+  int32_t layout;                /* rattn_layout of q, k, v, out, dout, dq, dk, dv */
   const int32_t* seq_lens;       /* optional device [B]: valid tokens of each batch entry, 1 <= len <= T
                                     (fresh sequences only); NULL: all T */
   const int32_t* pos;            /* decode only: optional device [B] positions, one per batch entry

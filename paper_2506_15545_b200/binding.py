@@ -18,6 +18,7 @@ RATTN_BF16, RATTN_F32 = 0, 1
 MODE_RATTN, MODE_SWA_ONLY, MODE_FULL_CAUSAL = 0, 1, 2
 FLAG_FORCE_GENERIC, FLAG_SAVE_RESIDUALS = 1, 2
 PHI_SOFTMAX, PHI_RELU, PHI_IDENTITY = 0, 1, 2
+LAYOUT_BHTD, LAYOUT_BTHD = 0, 1
 
 EXPORTS = (
     "rattn_forward", "rattn_forward_ex", "rattn_backward", "rattn_backward_ex",
@@ -48,7 +49,7 @@ class RattnParams(ctypes.Structure):
         ("dgamma_rla", ctypes.c_void_p),
         ("flags", ctypes.c_uint32), ("feature_map", ctypes.c_int32),
         ("state_in", ctypes.c_void_p), ("k_ring_in", ctypes.c_void_p), ("v_ring_in", ctypes.c_void_p),
-        ("pos0", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("pos0", ctypes.c_int32), ("layout", ctypes.c_int32),
         ("seq_lens", ctypes.c_void_p), ("pos", ctypes.c_void_p),
     ]
 
@@ -189,27 +190,38 @@ def alloc_workspace_chunked(q, k, w, flags=0) -> torch.Tensor:
     return torch.empty(n, dtype=torch.uint8, device=q.device)
 
 
-def alloc_workspace(q, k, w, mode=None, flags=None) -> torch.Tensor:
+def alloc_workspace(q, k, w, mode=None, flags=None, layout=LAYOUT_BHTD) -> torch.Tensor:
     """A uint8 device tensor for these shapes: exactly rattn_workspace_bytes_ex() bytes when
     mode and flags are given, else rattn_workspace_bytes() (enough for any mode and flags)."""
-    B, H_q, T, d = q.shape
-    if mode is None and flags is None:
-        n = rattn_workspace_bytes(B, H_q, k.shape[1], T, d, w, _dtype_code(q))
+    if layout == LAYOUT_BTHD:
+        B, T, H_q, d = q.shape
+        H_kv = k.shape[2]
     else:
-        n = rattn_workspace_bytes_ex(B, H_q, k.shape[1], T, d, w, _dtype_code(q), mode or 0, flags or 0)
+        B, H_q, T, d = q.shape
+        H_kv = k.shape[1]
+    if mode is None and flags is None:
+        n = rattn_workspace_bytes(B, H_q, H_kv, T, d, w, _dtype_code(q))
+    else:
+        n = rattn_workspace_bytes_ex(B, H_q, H_kv, T, d, w, _dtype_code(q), mode or 0, flags or 0)
     return torch.empty(n, dtype=torch.uint8, device=q.device)
 
 
-def _params(q, k, v, out, w, scale, eps, gamma_swa, gamma_rla, mode, workspace, flags, phi=PHI_SOFTMAX):
+def _params(q, k, v, out, w, scale, eps, gamma_swa, gamma_rla, mode, workspace, flags, phi=PHI_SOFTMAX,
+            layout=LAYOUT_BHTD):
     p = RattnParams()
     p.feature_map = phi
+    p.layout = layout
     p.q, p.k, p.v, p.out = q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr()
-    if q.dim() == 4:
+    if q.dim() == 4 and layout == LAYOUT_BTHD:
+        p.B, p.T, p.H_q, p.d = q.shape
+        p.H_kv = k.shape[2]
+    elif q.dim() == 4:
         p.B, p.H_q, p.T, p.d = q.shape
+        p.H_kv = k.shape[1]
     else:
         p.B, p.H_q, p.d = q.shape
         p.T = 1
-    p.H_kv = k.shape[1]
+        p.H_kv = k.shape[1]
     p.w = w
     p.dtype = _dtype_code(q)
     p.mode = mode
@@ -248,13 +260,14 @@ def rattn_forward_static(q, k, v, w, scale=1.0, out=None, stream=None):
 def rattn_forward_ex(q, k, v, w, *, scale=1.0, eps=1e-6, gamma_swa=None, gamma_rla=None,
                      mode=MODE_RATTN, workspace=None, save_residuals=False, state_out=None,
                      k_ring_out=None, v_ring_out=None, out=None, flags=0, phi=PHI_SOFTMAX, state_in=None,
-                     k_ring_in=None, v_ring_in=None, pos0=0, seq_lens=None, stream=None):
+                     k_ring_in=None, v_ring_in=None, pos0=0, seq_lens=None, layout=LAYOUT_BHTD, stream=None):
+    """layout=LAYOUT_BTHD: q, out are [B, T, H_q, d] and k, v [B, T, H_kv, d]."""
     _dense(q, k, v, out, gamma_swa, gamma_rla, workspace, state_out, k_ring_out, v_ring_out, state_in,
            k_ring_in, v_ring_in, seq_lens)
     out = torch.empty_like(q) if out is None else out
     if save_residuals:
         flags |= FLAG_SAVE_RESIDUALS
-    p = _params(q, k, v, out, w, scale, eps, gamma_swa, gamma_rla, mode, workspace, flags, phi)
+    p = _params(q, k, v, out, w, scale, eps, gamma_swa, gamma_rla, mode, workspace, flags, phi, layout)
     p.state_out = None if state_out is None else state_out.data_ptr()
     p.k_ring_out = None if k_ring_out is None else k_ring_out.data_ptr()
     p.v_ring_out = None if v_ring_out is None else v_ring_out.data_ptr()
@@ -282,12 +295,12 @@ def rattn_backward(q, k, v, dout, workspace, w, dq=None, dk=None, dv=None, strea
 
 def rattn_backward_ex(q, k, v, dout, w, workspace, *, scale=1.0, eps=1e-6, gamma_swa=None,
                       gamma_rla=None, mode=MODE_RATTN, dq=None, dk=None, dv=None,
-                      dgamma_swa=None, dgamma_rla=None, flags=0, phi=PHI_SOFTMAX, stream=None):
+                      dgamma_swa=None, dgamma_rla=None, flags=0, phi=PHI_SOFTMAX, layout=LAYOUT_BHTD, stream=None):
     _dense(q, k, v, dout, workspace, gamma_swa, gamma_rla, dq, dk, dv, dgamma_swa, dgamma_rla)
     dq = torch.empty_like(q) if dq is None else dq
     dk = torch.empty_like(k) if dk is None else dk
     dv = torch.empty_like(v) if dv is None else dv
-    p = _params(q, k, v, dq, w, scale, eps, gamma_swa, gamma_rla, mode, workspace, flags, phi)
+    p = _params(q, k, v, dq, w, scale, eps, gamma_swa, gamma_rla, mode, workspace, flags, phi, layout)
     p.dout, p.dq, p.dk, p.dv = dout.data_ptr(), dq.data_ptr(), dk.data_ptr(), dv.data_ptr()
     p.dgamma_swa = None if dgamma_swa is None else dgamma_swa.data_ptr()
     p.dgamma_rla = None if dgamma_rla is None else dgamma_rla.data_ptr()

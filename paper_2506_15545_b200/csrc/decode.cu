@@ -361,14 +361,17 @@ __global__ void __launch_bounds__(256) handoff_state_kernel(const TIO* __restric
                                                             const TIO* __restrict__ v,
                                                             float* __restrict__ state, int T, int w, int phi,
                                                             const int* __restrict__ len, int H_kv,
-                                                            const float* __restrict__ state_in) {
+                                                            const float* __restrict__ state_in, int layout) {
   constexpr int ROWS = 8, TOK = 32;
   __shared__ float fk[TOK][ROWS];
   __shared__ float vs[TOK][D];
   const int bh = blockIdx.y, r0 = blockIdx.x * ROWS;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const TIO* kg = k + (size_t)bh * T * D;
-  const TIO* vg = v + (size_t)bh * T * D;
+  // head (b, hk) of [B, H_kv, T, D] (layout 0) or [B, T, H_kv, D] (layout 1): first row and row pitch
+  const size_t head0 = layout ? ((size_t)(bh / H_kv) * T * H_kv + bh % H_kv) * D : (size_t)bh * T * D;
+  const size_t pitch = layout ? (size_t)H_kv * D : (size_t)D;
+  const TIO* kg = k + head0;
+  const TIO* vg = v + head0;
   const int n = (len ? min(T, len[bh / H_kv]) : T) - w;   // tokens 0..n-1 have left every window
   // thread -> (row, column group): 8 rows x 32 column lanes, D/32 columns each
   const int row = tid / 32, cl = tid % 32;
@@ -384,7 +387,7 @@ __global__ void __launch_bounds__(256) handoff_state_kernel(const TIO* __restric
       float m = -INFINITY;
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
-        x[c] = j < n ? to_f(kg[(size_t)j * D + lane + 32 * c]) : 0.f;
+        x[c] = j < n ? to_f(kg[(size_t)j * pitch + lane + 32 * c]) : 0.f;
         m = fmaxf(m, x[c]);
       }
       m = warp_max(m);
@@ -405,7 +408,7 @@ __global__ void __launch_bounds__(256) handoff_state_kernel(const TIO* __restric
       for (int c = 0; c < D / 32; ++c) {
         const int col = lane + 32 * c;
         if (col >= r0 && col < r0 + ROWS) fk[jj][col - r0] = x[c] * inv;
-        vs[jj][col] = j < n ? to_f(vg[(size_t)j * D + col]) : 0.f;
+        vs[jj][col] = j < n ? to_f(vg[(size_t)j * pitch + col]) : 0.f;
       }
     }
     __syncthreads();
@@ -424,8 +427,10 @@ __global__ void __launch_bounds__(256) handoff_state_kernel(const TIO* __restric
 template <typename TIO>
 __global__ void handoff_ring_kernel(const TIO* __restrict__ k, const TIO* __restrict__ v,
                                     TIO* __restrict__ kr, TIO* __restrict__ vr, int T, int w, int D,
-                                    const int* __restrict__ len, int H_kv, int pos_shift) {
+                                    const int* __restrict__ len, int H_kv, int pos_shift, int layout) {
   const int bh = blockIdx.y;
+  const size_t head0 = layout ? ((size_t)(bh / H_kv) * T * H_kv + bh % H_kv) * D : (size_t)bh * T * D;
+  const size_t pitch = layout ? (size_t)H_kv * D : (size_t)D;
   const int slot = blockIdx.x;
   // Row j of k, v is the token at sequence position j + pos_shift (a resumed sequence's rows start
   // before the chunk); the ring keeps position p at slot p % w.  The newest row that maps to this slot:
@@ -436,8 +441,8 @@ __global__ void handoff_ring_kernel(const TIO* __restrict__ k, const TIO* __rest
   for (int c = threadIdx.x; c < D; c += blockDim.x) {
     const size_t dst = ((size_t)bh * w + slot) * D + c;
     if (valid) {
-      kr[dst] = k[((size_t)bh * T + j) * D + c];
-      vr[dst] = v[((size_t)bh * T + j) * D + c];
+      kr[dst] = k[head0 + (size_t)j * pitch + c];
+      vr[dst] = v[head0 + (size_t)j * pitch + c];
     } else {
       kr[dst] = from_f<TIO>(0.f);
       vr[dst] = from_f<TIO>(0.f);
@@ -453,7 +458,7 @@ cudaError_t launch_handoff_t(const Args& a, cudaStream_t s, bool state_too) {
     KernelTimer kt("handoff_state", s);
     handoff_state_kernel<TIO, D><<<grid, 256, 0, s>>>(reinterpret_cast<const TIO*>(a.k),
                                                       reinterpret_cast<const TIO*>(a.v),
-                                                      a.state_out, a.Tk, a.w, a.phi, a.seq_lens, a.H_kv, a.state_in);
+                                                      a.state_out, a.Tk, a.w, a.phi, a.seq_lens, a.H_kv, a.state_in, a.kv_layout);
     count_launches(1);
   }
   if (a.k_ring_out && a.v_ring_out) {
@@ -463,7 +468,7 @@ cudaError_t launch_handoff_t(const Args& a, cudaStream_t s, bool state_too) {
                                                  reinterpret_cast<const TIO*>(a.v),
                                                  reinterpret_cast<TIO*>(a.k_ring_out),
                                                  reinterpret_cast<TIO*>(a.v_ring_out), a.Tk, a.w, D, a.seq_lens,
-                                                 a.H_kv, a.pos_shift);
+                                                 a.H_kv, a.pos_shift, a.kv_layout);
     count_launches(1);
   }
   return cudaGetLastError();
@@ -473,8 +478,11 @@ cudaError_t launch_handoff_t(const Args& a, cudaStream_t s, bool state_too) {
 __global__ void gather_history_kernel(const uint4* __restrict__ k_chunk, const uint4* __restrict__ v_chunk,
                                       const uint4* __restrict__ k_ring, const uint4* __restrict__ v_ring,
                                       uint4* __restrict__ k_ext, uint4* __restrict__ v_ext, int T, int w, int pos0,
-                                      int vec_per_row) {
+                                      int vec_per_row, int H_kv, int layout) {
   const int bh = blockIdx.y;
+  // the chunk is the caller's tensor: [B, H_kv, T, d] (layout 0) or [B, T, H_kv, d] (layout 1), in 16-byte vectors
+  const size_t head0 = layout ? ((size_t)(bh / H_kv) * T * H_kv + bh % H_kv) * vec_per_row : (size_t)bh * T * vec_per_row;
+  const size_t pitch = layout ? (size_t)H_kv * vec_per_row : (size_t)vec_per_row;
   const size_t n_ext = (size_t)(w + T) * vec_per_row;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_ext; i += (size_t)gridDim.x * blockDim.x) {
     const int e = (int)(i / vec_per_row), c = (int)(i % vec_per_row);
@@ -484,8 +492,8 @@ __global__ void gather_history_kernel(const uint4* __restrict__ k_chunk, const u
       kk = k_ring[((size_t)bh * w + slot) * vec_per_row + c];
       vv = v_ring[((size_t)bh * w + slot) * vec_per_row + c];
     } else {
-      kk = k_chunk[((size_t)bh * T + (e - w)) * vec_per_row + c];
-      vv = v_chunk[((size_t)bh * T + (e - w)) * vec_per_row + c];
+      kk = k_chunk[head0 + (size_t)(e - w) * pitch + c];
+      vv = v_chunk[head0 + (size_t)(e - w) * pitch + c];
     }
     k_ext[(size_t)bh * n_ext + i] = kk;
     v_ext[(size_t)bh * n_ext + i] = vv;
@@ -504,7 +512,7 @@ cudaError_t launch_gather_history(const Args& a, const void* k_chunk, const void
   gather_history_kernel<<<grid, 256, 0, s>>>(
       reinterpret_cast<const uint4*>(k_chunk), reinterpret_cast<const uint4*>(v_chunk),
       reinterpret_cast<const uint4*>(k_ring), reinterpret_cast<const uint4*>(v_ring),
-      reinterpret_cast<uint4*>(k_ext), reinterpret_cast<uint4*>(v_ext), a.T, a.w, pos0, vec_per_row);
+      reinterpret_cast<uint4*>(k_ext), reinterpret_cast<uint4*>(v_ext), a.T, a.w, pos0, vec_per_row, a.H_kv, a.layout);
   count_launches(1);
   return cudaGetLastError();
 }

@@ -38,7 +38,9 @@ __global__ void __launch_bounds__(256) bwd_preprocess_kernel(Args a, float* __re
   if (row >= n_rows) return;
   const int h = (int)((row / a.T) % a.H_q);
   constexpr int E = D / 32;
-  const TIO* dy = reinterpret_cast<const TIO*>(a.dout) + row * D;
+  const int bq_ = (int)(row / a.T), t_ = (int)(row - (size_t)bq_ * a.T);
+  const TIO* dy = reinterpret_cast<const TIO*>(a.dout) + head_base<D>(bq_ / a.H_q, bq_ % a.H_q, a.H_q, a.T, a.layout) +
+                  (size_t)t_ * row_pitch<D>(a.H_q, a.layout);
   float xs[E], xr[E], g[E];
   float ss = 0.f, sr = 0.f;
 #pragma unroll
@@ -109,11 +111,12 @@ __global__ void __launch_bounds__(NT) bwd_dq_kernel(Args a, const float* __restr
   const int q0 = qt * BQ, T = a.T, w = a.w;
   const bool rla_on = (a.mode == RATTN_MODE_RATTN);
   const size_t row_base = ((size_t)b * a.H_q + h) * T;
-  const TIO* qg = reinterpret_cast<const TIO*>(a.q) + row_base * D;
-  const TIO* kg = reinterpret_cast<const TIO*>(a.k) + ((size_t)b * a.H_kv + hk) * T * D;
-  const TIO* vg = reinterpret_cast<const TIO*>(a.v) + ((size_t)b * a.H_kv + hk) * T * D;
+  const size_t q_pitch = row_pitch<D>(a.H_q, a.layout), kv_pitch = row_pitch<D>(a.H_kv, a.layout);
+  const TIO* qg = reinterpret_cast<const TIO*>(a.q) + head_base<D>(b, h, a.H_q, T, a.layout);
+  const TIO* kg = reinterpret_cast<const TIO*>(a.k) + head_base<D>(b, hk, a.H_kv, T, a.layout);
+  const TIO* vg = reinterpret_cast<const TIO*>(a.v) + head_base<D>(b, hk, a.H_kv, T, a.layout);
 
-  load_tile<TIO, D, BQ>(Qs, qg, q0, T, tid);
+  load_tile<TIO, D, BQ>(Qs, qg, q0, T, tid, q_pitch);
   load_tile<float, D, BQ>(Gs, do_s + row_base * D, q0, T, tid);
   load_tile<float, D, BQ>(Gr, do_r + row_base * D, q0, T, tid);
   if (tid < BQ) {
@@ -141,8 +144,8 @@ __global__ void __launch_bounds__(NT) bwd_dq_kernel(Args a, const float* __restr
     const bool need_rla = rla_on && (j0 < q_last - w);
     if (!need_swa && !need_rla) continue;
     __syncthreads();
-    load_tile<TIO, D, BK>(Ks, kg, j0, T, tid);
-    load_tile<TIO, D, BK>(Vs, vg, j0, T, tid);
+    load_tile<TIO, D, BK>(Ks, kg, j0, T, tid, kv_pitch);
+    load_tile<TIO, D, BK>(Vs, vg, j0, T, tid, kv_pitch);
     __syncthreads();
     if (need_rla) feature_map_tile<D, BK>(Fk, Ks, tid, a.phi);
     if (need_swa) {
@@ -181,7 +184,7 @@ __global__ void __launch_bounds__(NT) bwd_dq_kernel(Args a, const float* __restr
     }
   }
   // dq += gradient through phi: phi(q) * (dphi_q - <dphi_q, phi(q)>) for the softmax map
-  TIO* dqg = reinterpret_cast<TIO*>(a.dq) + row_base * D;
+  TIO* dqg = reinterpret_cast<TIO*>(a.dq) + head_base<D>(b, h, a.H_q, T, a.layout);
 #pragma unroll
   for (int i = 0; i < 2; ++i) {
     const int r = ty + 16 * i, t = q0 + r;
@@ -205,7 +208,7 @@ __global__ void __launch_bounds__(NT) bwd_dq_kernel(Args a, const float* __restr
           o.z += feature_map_grad(a.phi, f[c].z, dfq[i][c].z, dot);
           o.w += feature_map_grad(a.phi, f[c].w, dfq[i][c].w, dot);
         }
-        store4<TIO>(dqg + (size_t)t * D + tx * 4 + 64 * c, o);
+        store4<TIO>(dqg + (size_t)t * q_pitch + tx * 4 + 64 * c, o);
       }
     }
   }
@@ -234,12 +237,13 @@ __global__ void __launch_bounds__(NT) bwd_dkv_kernel(Args a, const float* __rest
   const int bhk = blockIdx.y, b = bhk / a.H_kv, hk = bhk % a.H_kv;
   const int j0 = kt * BK, T = a.T, w = a.w;
   const bool rla_on = (a.mode == RATTN_MODE_RATTN);
-  const size_t kv_base = ((size_t)b * a.H_kv + hk) * T;
-  const TIO* kg = reinterpret_cast<const TIO*>(a.k) + kv_base * D;
-  const TIO* vg = reinterpret_cast<const TIO*>(a.v) + kv_base * D;
+  const size_t q_pitch = row_pitch<D>(a.H_q, a.layout), kv_pitch = row_pitch<D>(a.H_kv, a.layout);
+  const size_t kv_head = head_base<D>(b, hk, a.H_kv, T, a.layout);
+  const TIO* kg = reinterpret_cast<const TIO*>(a.k) + kv_head;
+  const TIO* vg = reinterpret_cast<const TIO*>(a.v) + kv_head;
 
-  load_tile<TIO, D, BK>(Ks, kg, j0, T, tid);
-  load_tile<TIO, D, BK>(Vs, vg, j0, T, tid);
+  load_tile<TIO, D, BK>(Ks, kg, j0, T, tid, kv_pitch);
+  load_tile<TIO, D, BK>(Vs, vg, j0, T, tid, kv_pitch);
   __syncthreads();
   if (rla_on) feature_map_tile<D, BK>(Fk, Ks, tid, a.phi);
 
@@ -257,14 +261,14 @@ __global__ void __launch_bounds__(NT) bwd_dkv_kernel(Args a, const float* __rest
   for (int hh = 0; hh < a.group; ++hh) {
     const int h = hk * a.group + hh;
     const size_t row_base = ((size_t)b * a.H_q + h) * T;
-    const TIO* qg = reinterpret_cast<const TIO*>(a.q) + row_base * D;
+    const TIO* qg = reinterpret_cast<const TIO*>(a.q) + head_base<D>(b, h, a.H_q, T, a.layout);
     for (int qt = j0 / BQ; qt < n_qt; ++qt) {
       const int q0 = qt * BQ, q_last = min(q0 + BQ, T) - 1;
       const bool need_swa = (j0 <= q_last) && (j0 + BK - 1 >= q0 - w);
       const bool need_rla = rla_on && (j0 < q_last - w);
       if (!need_swa && !need_rla) continue;
       __syncthreads();
-      load_tile<TIO, D, BQ>(Qs, qg, q0, T, tid);
+      load_tile<TIO, D, BQ>(Qs, qg, q0, T, tid, q_pitch);
       load_tile<float, D, BQ>(Gs, do_s + row_base * D, q0, T, tid);
       if (need_rla) load_tile<float, D, BQ>(Gr, do_r + row_base * D, q0, T, tid);
       if (tid < BQ) {
@@ -330,8 +334,8 @@ __global__ void __launch_bounds__(NT) bwd_dkv_kernel(Args a, const float* __rest
       }
     }
   }
-  TIO* dkg = reinterpret_cast<TIO*>(a.dk) + kv_base * D;
-  TIO* dvg = reinterpret_cast<TIO*>(a.dv) + kv_base * D;
+  TIO* dkg = reinterpret_cast<TIO*>(a.dk) + kv_head;
+  TIO* dvg = reinterpret_cast<TIO*>(a.dv) + kv_head;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int r = ty + 16 * i, jj = j0 + r;
@@ -355,8 +359,8 @@ __global__ void __launch_bounds__(NT) bwd_dkv_kernel(Args a, const float* __rest
           o.z += feature_map_grad(a.phi, f[c].z, dfk[i][c].z, dot);
           o.w += feature_map_grad(a.phi, f[c].w, dfk[i][c].w, dot);
         }
-        store4<TIO>(dkg + (size_t)jj * D + tx * 4 + 64 * c, o);
-        store4<TIO>(dvg + (size_t)jj * D + tx * 4 + 64 * c, dv[i][c]);
+        store4<TIO>(dkg + (size_t)jj * kv_pitch + tx * 4 + 64 * c, o);
+        store4<TIO>(dvg + (size_t)jj * kv_pitch + tx * 4 + 64 * c, dv[i][c]);
       }
     }
   }

@@ -34,15 +34,25 @@ template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16*
   *reinterpret_cast<uint2*>(p) = u;
 }
 
-// Copy a [ROWS, D] tile (rows row0.., zero beyond n_rows) into padded fp32 shared memory.
+// Where head (b, h) of a caller's tensor with H heads and T rows per head starts, and the distance
+// between its rows, in elements: [B, H, T, D] (layout 0) or [B, T, H, D] (layout 1).
+template <int D>
+__device__ __forceinline__ size_t head_base(int b, int h, int H, int T, int layout) {
+  return layout ? ((size_t)b * T * H + h) * D : ((size_t)b * H + h) * (size_t)T * D;
+}
+template <int D>
+__device__ __forceinline__ size_t row_pitch(int H, int layout) { return layout ? (size_t)H * D : (size_t)D; }
+
+// Copy a [ROWS, D] tile (rows row0.., zero beyond n_rows; `pitch` elements between rows) into padded fp32
+// shared memory.
 template <typename TIO, int D, int ROWS>
-__device__ __forceinline__ void load_tile(float* dst, const TIO* src, int row0, int n_rows, int tid) {
+__device__ __forceinline__ void load_tile(float* dst, const TIO* src, int row0, int n_rows, int tid, size_t pitch = D) {
   constexpr int LD = D + PAD;
   constexpr int V4 = D / 4;
   for (int i = tid; i < ROWS * V4; i += NT) {
     int r = i / V4, c = (i % V4) * 4;
     float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (row0 + r < n_rows) x = load4<TIO>(src + (size_t)(row0 + r) * D + c);
+    if (row0 + r < n_rows) x = load4<TIO>(src + (size_t)(row0 + r) * pitch + c);
     *reinterpret_cast<float4*>(dst + r * LD + c) = x;
   }
 }

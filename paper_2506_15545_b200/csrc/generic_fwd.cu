@@ -38,11 +38,12 @@ __global__ void __launch_bounds__(NT) generic_fwd_kernel(Args a) {
   const bool rla_on = (a.mode == RATTN_MODE_RATTN);
   if (q0 >= T) return;
 
-  const TIO* qg = reinterpret_cast<const TIO*>(a.q) + ((size_t)b * a.H_q + h) * a.T * D;
-  const TIO* kg = reinterpret_cast<const TIO*>(a.k) + ((size_t)b * a.H_kv + hk) * a.Tk * D;
-  const TIO* vg = reinterpret_cast<const TIO*>(a.v) + ((size_t)b * a.H_kv + hk) * a.Tk * D;
+  const size_t q_pitch = row_pitch<D>(a.H_q, a.layout), kv_pitch = row_pitch<D>(a.H_kv, a.kv_layout);
+  const TIO* qg = reinterpret_cast<const TIO*>(a.q) + head_base<D>(b, h, a.H_q, a.T, a.layout);
+  const TIO* kg = reinterpret_cast<const TIO*>(a.k) + head_base<D>(b, hk, a.H_kv, a.Tk, a.kv_layout);
+  const TIO* vg = reinterpret_cast<const TIO*>(a.v) + head_base<D>(b, hk, a.H_kv, a.Tk, a.kv_layout);
 
-  load_tile<TIO, D, 64>(Qs, qg, q0, T, tid);
+  load_tile<TIO, D, 64>(Qs, qg, q0, T, tid, q_pitch);
   __syncthreads();
   if (rla_on) feature_map_tile<D, 64>(Fq, Qs, tid, a.phi);
 
@@ -68,8 +69,8 @@ __global__ void __launch_bounds__(NT) generic_fwd_kernel(Args a) {
     const bool need_rla = rla_on && (j0 < q_last + off - w);
     if (!need_swa && !need_rla) continue;
     __syncthreads();                              // previous tile fully consumed
-    load_tile<TIO, D, 64>(Ks, kg, j0, Tk, tid);
-    load_tile<TIO, D, 64>(Vs, vg, j0, Tk, tid);
+    load_tile<TIO, D, 64>(Ks, kg, j0, Tk, tid, kv_pitch);
+    load_tile<TIO, D, 64>(Vs, vg, j0, Tk, tid, kv_pitch);
     __syncthreads();
     if (need_rla) feature_map_tile<D, 64>(Fk, Ks, tid, a.phi);
 
@@ -146,7 +147,7 @@ __global__ void __launch_bounds__(NT) generic_fwd_kernel(Args a) {
   }
 
   // Section 3.2: two separate RMS norms, then the sum.
-  TIO* og = reinterpret_cast<TIO*>(a.out) + ((size_t)b * a.H_q + h) * a.T * D;
+  TIO* og = reinterpret_cast<TIO*>(a.out) + head_base<D>(b, h, a.H_q, a.T, a.layout);
   const size_t row_base = ((size_t)b * a.H_q + h) * a.T;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -183,7 +184,7 @@ __global__ void __launch_bounds__(NT) generic_fwd_kernel(Args a) {
           y.z += gr.z * acc_r[i][c].z * rinv_r;
           y.w += gr.w * acc_r[i][c].w * rinv_r;
         }
-        store4<TIO>(og + (size_t)t * D + col, y);
+        store4<TIO>(og + (size_t)t * q_pitch + col, y);
         if (a.o_swa) *reinterpret_cast<float4*>(a.o_swa + (row_base + t) * D + col) = acc_s[i][c];
         if (a.o_rla) *reinterpret_cast<float4*>(a.o_rla + (row_base + t) * D + col) = acc_r[i][c];
       }

@@ -135,6 +135,7 @@ static int resolve(const rattn_params* p, Args* a, bool need_T) {
   if (p->dtype != RATTN_BF16 && p->dtype != RATTN_F32) return RATTN_ERR_UNSUPPORTED;
   if (p->mode < RATTN_MODE_RATTN || p->mode > RATTN_MODE_FULL_CAUSAL) return RATTN_ERR_UNSUPPORTED;
   if (p->feature_map < RATTN_PHI_SOFTMAX || p->feature_map > RATTN_PHI_IDENTITY) return RATTN_ERR_UNSUPPORTED;
+  if (p->layout != RATTN_LAYOUT_BHTD && p->layout != RATTN_LAYOUT_BTHD) return RATTN_ERR_UNSUPPORTED;
   if (!(p->eps > 0.f) || !(p->scale == p->scale)) return RATTN_ERR_BAD_ARG;
   if (!p->q || !p->k || !p->v || !p->out) return RATTN_ERR_NULL_PTR;
   if (misaligned(p->q) || misaligned(p->k) || misaligned(p->v) || misaligned(p->out) ||
@@ -148,6 +149,7 @@ static int resolve(const rattn_params* p, Args* a, bool need_T) {
   a->group = p->H_q / p->H_kv;
   a->dtype = p->dtype; a->mode = p->mode;
   a->flags = p->flags;
+  a->layout = a->kv_layout = p->layout;
   a->phi = p->feature_map;
   a->scale = p->scale; a->eps = p->eps;
   a->gamma_swa = p->gamma_swa; a->gamma_rla = p->gamma_rla;
@@ -223,6 +225,7 @@ static int forward_impl(const rattn_params* p, cudaStream_t s) {
     e = launch_gather_history(a, p->k, p->v, p->k_ring_in, p->v_ring_in, k_ext, v_ext, p->pos0, s);
     if (e != cudaSuccess) return fail_cuda(e);
     a.k = k_ext; a.v = v_ext;
+    a.kv_layout = RATTN_LAYOUT_BHTD;                       // the gathered history + chunk is dense per head
     a.Tk = p->w + p->T; a.q_off = p->w; a.state_in = p->state_in; a.pos_shift = p->pos0 - p->w;
   }
 #ifdef RATTN_HAVE_TC

@@ -56,6 +56,8 @@ struct Args {
   int group;                   // H_q / H_kv
   int dtype, mode;
   unsigned flags;              // rattn_params.flags
+  int layout;                  // rattn_layout of q, out, dout, dq (and of k, v, dk, dv unless kv_layout says otherwise)
+  int kv_layout;               // layout of the k, v the kernels read: dense when they are the gathered history + chunk
   int phi;                     // rattn_feature_map
   float scale, eps;
   const float* gamma_swa;
@@ -114,6 +116,9 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_sta
 struct StateLaunch {
   const void* x;            // [n_kv * group, T, 128] bf16, mapped through phi
   const void* y;            // [n_kv * group, T, 128] bf16
+  // x and y as the caller's tensors: heads per batch entry and head layout (rattn_layout); 0 heads = a dense
+  // internal tensor of n_kv * group matrices
+  int x_heads, x_layout, y_heads, y_layout;
   void* out;                // [n_kv * n_chunks, 128, 128] bf16
   int T, n_kv, group, n_chunks;
   int n_steps, first, dir, out_first;

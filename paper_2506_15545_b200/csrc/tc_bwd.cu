@@ -77,7 +77,7 @@ constexpr int PREP_STAGES = 4;
 constexpr int PREP_SMEM = PREP_STAGES * 3 * PREP_CHUNK + 128;
 
 struct PrepArgs {
-  const __nv_bfloat16* dy; const __nv_bfloat16* o_s; const __nv_bfloat16* o_r;
+  const __nv_bfloat16* o_s; const __nv_bfloat16* o_r;
   const float* gamma_s; const float* gamma_r;
   __nv_bfloat16* g_s; __nv_bfloat16* g_r;
   float* delta; float* dgamma_s; float* dgamma_r;
@@ -97,7 +97,8 @@ __device__ __forceinline__ void unpack8(const unsigned char* p, float (&x)[8]) {
   }
 }
 
-__global__ void __launch_bounds__(PREP_THREADS, 2) tc_bwd_prep_kernel(const __grid_constant__ PrepArgs a) {
+__global__ void __launch_bounds__(PREP_THREADS, 2)
+tc_bwd_prep_kernel(const __grid_constant__ PrepArgs a, const __grid_constant__ CUtensorMap dy_map) {
   extern __shared__ __align__(128) unsigned char psm[];
   uint64_t* full = reinterpret_cast<uint64_t*>(psm + PREP_STAGES * 3 * PREP_CHUNK);
   volatile int* abort = reinterpret_cast<volatile int*>(full + PREP_STAGES);
@@ -108,6 +109,7 @@ __global__ void __launch_bounds__(PREP_THREADS, 2) tc_bwd_prep_kernel(const __gr
   const int n_in = a.rla_on ? 3 : 2;                                // tensors read per chunk
 
   if (tid == 0) {
+    prefetch_tensormap(&dy_map);
     for (int i = 0; i < PREP_STAGES; ++i) mbar_init(&full[i], 1);
     *abort = 0;
     fence_mbar_init();
@@ -127,9 +129,15 @@ __global__ void __launch_bounds__(PREP_THREADS, 2) tc_bwd_prep_kernel(const __gr
     uint64_t* bar = &full[n_issued % PREP_STAGES];
     ++n_issued;
     const uint32_t bytes = (uint32_t)rows * 256;
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes * n_in) : "memory");
-    const __nv_bfloat16* src[3] = {a.dy, a.o_s, a.o_r};
-    for (int k = 0; k < n_in; ++k)
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                 ::"r"(smem_u32(bar)), "r"((uint32_t)PREP_CHUNK + bytes * (n_in - 1)) : "memory");
+    // dO is the caller's tensor (either head layout): a tiled copy of 32 whole rows, rows beyond T read as zero
+    const int bq_ = i / cph, b_ = bq_ / a.H_q, h_ = bq_ - b_ * a.H_q;
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(&dy_map), "r"(smem_u32(bar)), "r"(0), "r"((i % cph) * PREP_ROWS), "r"(h_), "r"(b_)
+                 : "memory");
+    const __nv_bfloat16* src[3] = {nullptr, a.o_s, a.o_r};
+    for (int k = 1; k < n_in; ++k)
       asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                    ::"r"(smem_u32(dst + k * PREP_CHUNK)), "l"(src[k] + at), "r"(bytes), "r"(smem_u32(bar)) : "memory");
   };
@@ -332,7 +340,8 @@ __device__ __forceinline__ DqItem dq_item(const BwdArgs& a, int idx, int n_qt) {
 }
 
 struct DqMaps {
-  CUtensorMap q, k, v, gs, gr, st, dq;
+  UMap q, k, v, dq;             // the caller's tensors (either head layout)
+  CUtensorMap gs, gr, st;
 };
 
 __device__ bool dq_loader(const DqMaps& tm, const BwdArgs& a, unsigned char* smem, DqBars* bars, int n_items, int n_qt) {
@@ -636,13 +645,13 @@ tc_bwd_dq_kernel(const __grid_constant__ DqMaps tm, BwdArgs a, int n_items, int 
     tmem_relinquish();
   }
   if (tid == 288) {
-    prefetch_tensormap(&tm.q);
-    prefetch_tensormap(&tm.k);
-    prefetch_tensormap(&tm.v);
+    prefetch_map(&tm.q);
+    prefetch_map(&tm.k);
+    prefetch_map(&tm.v);
     prefetch_tensormap(&tm.gs);
     prefetch_tensormap(&tm.gr);
     prefetch_tensormap(&tm.st);
-    prefetch_tensormap(&tm.dq);
+    prefetch_map(&tm.dq);
   }
   tc_fence_before();
   __syncthreads();
@@ -704,7 +713,8 @@ struct KvBars {
 };
 
 struct KvMaps {
-  CUtensorMap k, v, rs, qh, gsh, grh, dk, dv;
+  UMap k, v, qh, dk, dv;        // the caller's tensors (either head layout)
+  CUtensorMap rs, gsh, grh;
 };
 
 // One key tile (j, K/V head) of the persistent CTA's work list, and how its half-tile items
@@ -1099,14 +1109,14 @@ tc_bwd_dkv_kernel(const __grid_constant__ KvMaps tm, BwdArgs a, int n_items) {
     tmem_relinquish();
   }
   if (tid == 288) {
-    prefetch_tensormap(&tm.k);
-    prefetch_tensormap(&tm.v);
+    prefetch_map(&tm.k);
+    prefetch_map(&tm.v);
     prefetch_tensormap(&tm.rs);
-    prefetch_tensormap(&tm.qh);
+    prefetch_map(&tm.qh);
     prefetch_tensormap(&tm.gsh);
     prefetch_tensormap(&tm.grh);
-    prefetch_tensormap(&tm.dk);
-    prefetch_tensormap(&tm.dv);
+    prefetch_map(&tm.dk);
+    prefetch_map(&tm.dv);
   }
   tc_fence_before();
   __syncthreads();
@@ -1154,7 +1164,6 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
   const int t_pad = a.n_chunks * TILE;
   {
     PrepArgs pa;
-    pa.dy = reinterpret_cast<const __nv_bfloat16*>(a.dout);
     pa.o_s = reinterpret_cast<const __nv_bfloat16*>(a.o_swa);
     pa.o_r = reinterpret_cast<const __nv_bfloat16*>(a.o_rla);
     pa.gamma_s = a.gamma_swa; pa.gamma_r = a.gamma_rla;
@@ -1171,16 +1180,21 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
     if (e != cudaSuccess) return e;
     const long long n_chunks_all = (long long)pa.n_heads * (t_pad / PREP_ROWS);
     const int grid = (int)(n_chunks_all < 2ll * n_sm ? n_chunks_all : 2ll * n_sm);
+    CUtensorMap dy_map;
+    if (!make_row_map(&dy_map, a.dout, a.T, a.H_q, a.B, a.layout, PREP_ROWS)) return cudaErrorInvalidValue;
     KernelTimer kt("tc_bwd_prep", s);
-    tc_bwd_prep_kernel<<<grid, PREP_THREADS, PREP_SMEM, s>>>(pa);
+    tc_bwd_prep_kernel<<<grid, PREP_THREADS, PREP_SMEM, s>>>(pa, dy_map);
   }
   count_launches(1);
 
-  CUtensorMap tm_q, tm_k, tm_v, tm_gs, tm_gr, tm_st, tm_rs, tm_dq, tm_dk, tm_dv;
+  UMap tm_q, tm_k, tm_v, tm_dq, tm_dk, tm_dv;
+  CUtensorMap tm_gs, tm_gr, tm_st, tm_rs;
   const uint64_t nq = (uint64_t)a.B * a.H_q, nkv = (uint64_t)a.B * a.H_kv;
-  if (!make_map(&tm_q, a.q, a.T, nq) || !make_map(&tm_k, a.k, a.T, nkv) || !make_map(&tm_v, a.v, a.T, nkv) ||
+  if (!make_user_map(&tm_q, a.q, a.T, a.H_q, a.B, a.layout) || !make_user_map(&tm_k, a.k, a.T, a.H_kv, a.B, a.layout) ||
+      !make_user_map(&tm_v, a.v, a.T, a.H_kv, a.B, a.layout) ||
       !make_map(&tm_gs, g_s, a.T, nq) || !make_map(&tm_gr, g_r, a.T, nq) ||
-      !make_map(&tm_dq, a.dq, a.T, nq) || !make_map(&tm_dk, a.dk, a.T, nkv) || !make_map(&tm_dv, a.dv, a.T, nkv) ||
+      !make_user_map(&tm_dq, a.dq, a.T, a.H_q, a.B, a.layout) || !make_user_map(&tm_dk, a.dk, a.T, a.H_kv, a.B, a.layout) ||
+      !make_user_map(&tm_dv, a.dv, a.T, a.H_kv, a.B, a.layout) ||
       !make_state_map(&tm_st, a.chunk_state, a.k, nkv * a.n_chunks) || !make_state_map(&tm_rs, a.rstate, a.k, nkv * a.n_chunks))
     return cudaErrorInvalidValue;
 
@@ -1190,6 +1204,7 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
   {
     StateLaunch L;
     L.x = a.q; L.y = g_r; L.out = a.rstate;
+    L.x_heads = a.H_q; L.x_layout = a.layout; L.y_heads = 0; L.y_layout = 0;
     L.T = a.T; L.n_kv = (int)nkv; L.group = a.group; L.n_chunks = a.n_chunks;
     L.n_steps = n_r; L.first = n_qt - 1; L.dir = -1; L.out_first = n_qt - wt - 2;
     L.store_every = 1; L.store_phase = 0; L.handoff = 0; L.w = a.w; L.final_out = nullptr;
@@ -1227,7 +1242,8 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
   }
   KvMaps km;
   km.k = tm_k; km.v = tm_v; km.rs = tm_rs; km.dk = tm_dk; km.dv = tm_dv;
-  if (!make_map(&km.qh, a.q, a.T, nq, 64) || !make_map(&km.gsh, g_s, a.T, nq, 64) || !make_map(&km.grh, g_r, a.T, nq, 64))
+  if (!make_user_map(&km.qh, a.q, a.T, a.H_q, a.B, a.layout, 64) || !make_map(&km.gsh, g_s, a.T, nq, 64) ||
+      !make_map(&km.grh, g_r, a.T, nq, 64))
     return cudaErrorInvalidValue;
   {
     int dev = 0, n_sm = 0;

@@ -79,6 +79,24 @@ __device__ __forceinline__ void mma_ts_h(uint32_t d, uint32_t a_tmem, uint32_t b
   for (int k = 0; k < 4; ++k)
     mma_bf16_ts(d, a_tmem + (k < 2 ? 8 * k : 32 + 8 * (k - 2)), b0 + kstep_mn(k), idesc, (acc || k > 0) ? 1u : 0u);
 }
+// A caller's tensor (q, k, v, out and the gradients): its heads may be dense ([B, H, T, d]) or interleaved
+// ([B, T, H, d]), so its map has four dimensions (d, T, H, B) and a matrix index z = b * H + h is split.
+struct alignas(64) UMap {
+  CUtensorMap m;
+  int H;
+};
+__device__ __forceinline__ void prefetch_map(const UMap* tm) { prefetch_tensormap(&tm->m); }
+__device__ __forceinline__ void load_tile(unsigned char* dst, const UMap* tm, uint64_t* bar, int row, int z) {
+  const int b = z / tm->H, h = z - b * tm->H;
+  tma_load_4d(dst, &tm->m, bar, 0, row, h, b);
+  tma_load_4d(dst + HALF_BYTES, &tm->m, bar, 64, row, h, b);
+}
+// `tm` must have a [64 columns x 64 rows] box
+__device__ __forceinline__ void load_half_tile(unsigned char* dst, const UMap* tm, uint64_t* bar, int row, int z) {
+  const int b = z / tm->H, h = z - b * tm->H;
+  tma_load_4d(dst, &tm->m, bar, 0, row, h, b);
+  tma_load_4d(dst + HT_HALF, &tm->m, bar, 64, row, h, b);
+}
 __device__ __forceinline__ void load_tile(unsigned char* dst, const CUtensorMap* tm, uint64_t* bar, int row, int z) {
   tma_load_3d(dst, tm, bar, 0, row, z);
   tma_load_3d(dst + HALF_BYTES, tm, bar, 64, row, z);
@@ -179,6 +197,16 @@ __device__ __forceinline__ uint32_t swz(int r, int c) {
 
 // One [128 x 128] bf16 tile staged in shared memory (swizzled like a loaded tile) goes to
 // rows row0.. of matrix z of a tensor map: two 64-column boxes; rows past the end are clipped.
+__device__ __forceinline__ void store_tile(const UMap* tm, const unsigned char* tile, int row0, int z) {
+  const int b = z / tm->H, h = z - b * tm->H;
+  tma_store_4d(&tm->m, tile, 0, row0, h, b);
+  tma_store_4d(&tm->m, tile + HALF_BYTES, 64, row0, h, b);
+}
+// one 64-column half of a staged tile
+__device__ __forceinline__ void store_half(const UMap* tm, const unsigned char* half, int x, int row0, int z) {
+  const int b = z / tm->H, h = z - b * tm->H;
+  tma_store_4d(&tm->m, half, x, row0, h, b);
+}
 __device__ __forceinline__ void store_tile(const CUtensorMap* tm, const unsigned char* tile, int row0, int z) {
   tma_store_3d(tm, tile, 0, row0, z);
   tma_store_3d(tm, tile + HALF_BYTES, 64, row0, z);
@@ -408,6 +436,36 @@ inline bool make_map(CUtensorMap* m, const void* base, uint64_t rows, uint64_t n
   const cuuint32_t estr[3] = {1, 1, 1};
   return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// A caller's tensor with T rows per head, H heads, B batch entries: [B, H, T, 128] (layout 0) or
+// [B, T, H, 128] (layout 1), bf16; box = 64 columns x box_rows rows of one head.
+inline bool make_user_map(UMap* u, const void* base, uint64_t T, uint64_t H, uint64_t B, int layout,
+                          uint32_t box_rows = 128) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  u->H = (int)H;
+  const cuuint64_t dims[4] = {128, T, H, B};
+  const cuuint64_t row = 128 * 2;
+  const cuuint64_t strides[3] = {layout ? H * row : row, layout ? row : T * row, T * H * row};
+  const cuuint32_t box[4] = {64, box_rows, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(&u->m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// The same tensor read as whole rows: box = 128 columns x box_rows rows of one head, no swizzle.
+inline bool make_row_map(CUtensorMap* m, const void* base, uint64_t T, uint64_t H, uint64_t B, int layout,
+                         uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[4] = {128, T, H, B};
+  const cuuint64_t row = 128 * 2;
+  const cuuint64_t strides[3] = {layout ? H * row : row, layout ? row : T * row, T * H * row};
+  const cuuint32_t box[4] = {128, box_rows, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 // [n_mats, 128, 128] bf16 chunk states.  Modes without a linear branch keep none: the kernels

@@ -34,6 +34,7 @@ cudaError_t launch_tc_forward(const Args& a, cudaStream_t s) {
   if (n_steps > 0 || (a.state_in && rla) || (a.seq_lens && want_state)) {
     StateLaunch L;
     L.x = a.k; L.y = a.v; L.out = a.chunk_state;
+    L.x_heads = L.y_heads = a.H_kv; L.x_layout = L.y_layout = a.kv_layout;
     L.T = a.Tk; L.n_kv = n_kv; L.group = 1; L.n_chunks = a.n_chunks;
     L.n_steps = n_steps > 0 ? n_steps : 0; L.first = 0; L.dir = +1; L.out_first = 1;
     // the main kernel reads S_[c] for c = off + 2p - wt only

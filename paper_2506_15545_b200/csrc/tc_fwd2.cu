@@ -73,7 +73,8 @@ struct FArgs {
 };
 
 struct FMaps {
-  CUtensorMap q, k, v, st, out;
+  UMap q, k, v, out;          // the caller's tensors (either head layout)
+  CUtensorMap st;
   CUtensorMap o_swa, o_rla;   // training mode: the un-normalised branch outputs, [B*H_q, T, 128] bf16
 };
 
@@ -714,7 +715,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
         fence_proxy_async_smem();
         group_sync(X);
         if (r == 0) {
-          tma_store_3d(&tm.out, sY, 64 * hf, q0, un.bh_q);
+          store_half(&tm.out, sY, 64 * hf, q0, un.bh_q);
           tma_store_commit();
         }
         // The Q buffer (phi(Q_X) has long been consumed) is released only once the last store is
@@ -780,11 +781,11 @@ tc_fwd2_kernel(const __grid_constant__ FMaps tm, FArgs a) {
     tmem_relinquish();
   }
   if (tid == 288) {
-    prefetch_tensormap(&tm.q);
-    prefetch_tensormap(&tm.k);
-    prefetch_tensormap(&tm.v);
+    prefetch_map(&tm.q);
+    prefetch_map(&tm.k);
+    prefetch_map(&tm.v);
     prefetch_tensormap(&tm.st);
-    prefetch_tensormap(&tm.out);
+    prefetch_map(&tm.out);
     prefetch_tensormap(&tm.o_swa);
     prefetch_tensormap(&tm.o_rla);
   }
@@ -830,8 +831,8 @@ extern "C" int rattn_timeline_read(unsigned long long* out, int* n) {
 
 cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_states) {
   FMaps tm;
-  if (!make_map(&tm.q, a.q, a.T, (uint64_t)a.B * a.H_q) || !make_map(&tm.k, a.k, a.Tk, (uint64_t)a.B * a.H_kv) ||
-      !make_map(&tm.v, a.v, a.Tk, (uint64_t)a.B * a.H_kv) || !make_map(&tm.out, a.out, a.T, (uint64_t)a.B * a.H_q) ||
+  if (!make_user_map(&tm.q, a.q, a.T, a.H_q, a.B, a.layout) || !make_user_map(&tm.k, a.k, a.Tk, a.H_kv, a.B, a.kv_layout) ||
+      !make_user_map(&tm.v, a.v, a.Tk, a.H_kv, a.B, a.kv_layout) || !make_user_map(&tm.out, a.out, a.T, a.H_q, a.B, a.layout) ||
       !make_state_map(&tm.st, a.chunk_state, a.k, (uint64_t)a.B * a.H_kv * a.n_chunks) ||
       !make_map(&tm.o_swa, a.o_swa ? (const void*)a.o_swa : a.out, a.T, (uint64_t)a.B * a.H_q) ||
       !make_map(&tm.o_rla, a.o_rla ? (const void*)a.o_rla : a.out, a.T, (uint64_t)a.B * a.H_q))

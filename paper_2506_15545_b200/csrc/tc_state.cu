@@ -66,7 +66,7 @@ __device__ __forceinline__ bool flushed_step(const StateArgs& a, int s, int n_st
 }
 
 __global__ void __launch_bounds__(ST_THREADS, 1)
-tc_state_scan_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_y,
+tc_state_scan_kernel(const __grid_constant__ UMap tm_x, const __grid_constant__ UMap tm_y,
                      const __grid_constant__ CUtensorMap tm_out, StateArgs a) {
   extern __shared__ __align__(1024) unsigned char smem[];
   StBars* bars = reinterpret_cast<StBars*>(smem + ST_OFF_BAR);
@@ -94,8 +94,8 @@ tc_state_scan_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
     tmem_relinquish();
   }
   if (tid == 288) {
-    prefetch_tensormap(&tm_x);
-    prefetch_tensormap(&tm_y);
+    prefetch_map(&tm_x);
+    prefetch_map(&tm_y);
     prefetch_tensormap(&tm_out);
   }
   tc_fence_before();
@@ -261,8 +261,13 @@ tc_state_scan_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_cons
 // x, y: [n_kv * group, T, 128] bf16; out: [n_kv * n_chunks, 128, 128] bf16.
 cudaError_t launch_tc_states(const StateLaunch& L, cudaStream_t s) {
   if (L.n_steps <= 0 && !L.state_in && !(L.seq_lens && L.final_out)) return cudaSuccess;
-  CUtensorMap tm_x, tm_y, tm_out;
-  if (!make_map(&tm_x, L.x, L.T, (uint64_t)L.n_kv * L.group) || !make_map(&tm_y, L.y, L.T, (uint64_t)L.n_kv * L.group) ||
+  UMap tm_x, tm_y;
+  CUtensorMap tm_out;
+  const uint64_t n_mats = (uint64_t)L.n_kv * L.group;
+  auto user = [&](UMap* m, const void* base, int heads, int layout) {
+    return heads > 0 ? make_user_map(m, base, L.T, heads, n_mats / heads, layout) : make_user_map(m, base, L.T, n_mats, 1, 0);
+  };
+  if (!user(&tm_x, L.x, L.x_heads, L.x_layout) || !user(&tm_y, L.y, L.y_heads, L.y_layout) ||
       !make_map(&tm_out, L.out, 128, (uint64_t)L.n_kv * L.n_chunks))
     return cudaErrorInvalidValue;
   StateArgs a;
