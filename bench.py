@@ -561,7 +561,12 @@ def run_case(args):
         ms_b = timed(lambda: R.rattn_qk_prologue_backward(q, k, qo, ko, q_gain=gq, k_gain=gq, workspace=wsp),
                      args.steps, args.warmup, sync)
         hbm = peaks()["hbm"]
+        qt, kt = q.transpose(1, 2).contiguous(), k.transpose(1, 2).contiguous()       # [B, T, H, d]
+        ms_ft = timed(lambda: R.rattn_qk_prologue(qt, kt, q_gain=gq, k_gain=gq, layout=R.LAYOUT_BTHD), args.steps,
+                      args.warmup, sync)
         print(json.dumps({"case": "prologue", "workload": workload_name(wl),
+                          "forward_bthd": {"ms": ms_ft, "gb_per_s": nbytes / ms_ft / 1e6,
+                                           "frac_of_hbm_peak": nbytes / ms_ft / 1e6 / hbm},
                           "forward": {"ms": ms_f, "gb_per_s": nbytes / ms_f / 1e6, "frac_of_hbm_peak": nbytes / ms_f / 1e6 / hbm},
                           "backward": {"ms": ms_b, "gb_per_s": 1.5 * nbytes / ms_b / 1e6,
                                        "frac_of_hbm_peak": 1.5 * nbytes / ms_b / 1e6 / hbm},

@@ -366,6 +366,8 @@ int rattn_uses_tensor_path(int d, int w, int dtype, int mode, unsigned flags);
  *                  optional device int32 [B] (decoding a batch whose entries have different lengths).
  *                  Angles are formed in fp64 and reduced before the fp32 sine and cosine, so
  *                  positions up to 2^31 keep full fp32 accuracy.
+ *   layout         RATTN_LAYOUT_BHTD (default) or RATTN_LAYOUT_BTHD: q as [B,T,H_q,d], k as [B,T,H_kv,d],
+ *                  the layout the projections write; the results and gradients have the same layout.
  *   d              64 or 128.  Arithmetic is fp32; sums over a row are taken in a fixed order.
  *
  * rattn_qk_prologue_backward: given the same inputs (the tensors as they were BEFORE the forward
@@ -393,7 +395,7 @@ typedef struct rattn_qk_params {
   float eps;
   float theta;
   int32_t pos0;
-  int32_t reserved;
+  int32_t layout;                /* rattn_layout of q, k, their outputs and gradients */
   const int32_t* pos;
 } rattn_qk_params;
 

@@ -61,7 +61,7 @@ class RattnQkParams(ctypes.Structure):
         ("B", ctypes.c_int32), ("H_q", ctypes.c_int32), ("H_kv", ctypes.c_int32),
         ("T", ctypes.c_int32), ("d", ctypes.c_int32), ("dtype", ctypes.c_int32),
         ("eps", ctypes.c_float), ("theta", ctypes.c_float),
-        ("pos0", ctypes.c_int32), ("reserved", ctypes.c_int32), ("pos", ctypes.c_void_p),
+        ("pos0", ctypes.c_int32), ("layout", ctypes.c_int32), ("pos", ctypes.c_void_p),
     ]
 
 
@@ -372,14 +372,17 @@ def rattn_timing_read() -> dict:
     return out
 
 
-def _qk_params(q, k, q_out, k_out, q_gain, k_gain, theta, eps, pos0, pos):
+def _qk_params(q, k, q_out, k_out, q_gain, k_gain, theta, eps, pos0, pos, layout=LAYOUT_BHTD):
     p = RattnQkParams()
     _dense(q, k, q_out, k_out, q_gain, k_gain, pos)
     p.q, p.q_out = q.data_ptr(), None if q_out is None else q_out.data_ptr()
-    p.B, p.H_q, p.T, p.d = q.shape
+    hd = 2 if layout == LAYOUT_BTHD else 1              # which dimension counts the heads
+    p.layout = layout
+    p.B, p.d = q.shape[0], q.shape[3]
+    p.H_q, p.T = q.shape[hd], q.shape[3 - hd]
     if k is not None:
         p.k, p.k_out = k.data_ptr(), None if k_out is None else k_out.data_ptr()
-        p.H_kv = k.shape[1]
+        p.H_kv = k.shape[hd]
     p.q_gain = None if q_gain is None else q_gain.data_ptr()
     p.k_gain = None if k_gain is None else k_gain.data_ptr()
     p.dtype = _dtype_code(q)
@@ -406,25 +409,25 @@ def rattn_qk_prologue_status(stream=None) -> int:
 
 
 def rattn_qk_prologue(q, k, *, q_gain=None, k_gain=None, theta=5.0e5, eps=1e-6, pos0=0, pos=None,
-                      inplace=False, stream=None):
+                      inplace=False, layout=LAYOUT_BHTD, stream=None):
     """rattn_qk_prologue: qk-norm then rotary embedding of q [B,H_q,T,d] and k [B,H_kv,T,d] (k may be
     None).  theta None or <= 0: no rotation.  Returns (q_out, k_out); the inputs themselves if inplace."""
     q_out = q if inplace else torch.empty_like(q)
     k_out = None if k is None else (k if inplace else torch.empty_like(k))
-    p = _qk_params(q, k, q_out, k_out, q_gain, k_gain, theta, eps, pos0, pos)
+    p = _qk_params(q, k, q_out, k_out, q_gain, k_gain, theta, eps, pos0, pos, layout)
     _check(lib().rattn_qk_prologue(ctypes.byref(p), _stream(stream)), "rattn_qk_prologue")
     return q_out, k_out
 
 
 def rattn_qk_prologue_backward(q, k, dq_out, dk_out, *, q_gain=None, k_gain=None, theta=5.0e5, eps=1e-6,
-                               pos0=0, pos=None, gain_grads=True, workspace=None, stream=None):
+                               pos0=0, pos=None, gain_grads=True, workspace=None, layout=LAYOUT_BHTD, stream=None):
     """rattn_qk_prologue_backward: gradients with respect to q, k (inputs as they were before the
     forward pass) and, with gain_grads, to the two gains.  Returns (dq, dk, dq_gain, dk_gain)."""
     _dense(dq_out, dk_out)
     dq = torch.empty_like(q)
     dk = None if k is None else torch.empty_like(k)
     dqg = dkg = None
-    p = _qk_params(q, k, None, None, q_gain, k_gain, theta, eps, pos0, pos)
+    p = _qk_params(q, k, None, None, q_gain, k_gain, theta, eps, pos0, pos, layout)
     if gain_grads:
         dqg = torch.empty(q.shape[-1], dtype=torch.float32, device=q.device)
         dkg = None if k is None else torch.empty(q.shape[-1], dtype=torch.float32, device=q.device)

@@ -35,6 +35,10 @@ struct QkArgs {
   const float* gain[2];
   float* partial;                     // backward: [2][n_cta][d] or null
   int H[2];
+  float inv_H[2];                     // 1 / H
+  int n_chunks[2];                    // chunks of q, of k
+  int tbl_tokens;                     // [B,T,H,d]: positions a rotation table holds
+  int layout;                         // rattn_layout of x, y, dy
   int B, T, nblk_t;
   float eps;
   int rotate;
@@ -146,24 +150,56 @@ template <typename T, bool BWD> struct Ring {
   static constexpr int kBytes = kStages * kBufs * kChunk + kRed + 128;
 };
 
-// One chunk: tensor `which`, batch entry b, row block tb, head h; chunks are numbered tensor,
-// batch entry, row block, head.  A cursor is set once and then stepped.
-struct Chunk {
-  int which, b, tb, h;
+// Chunks and their order.
+//   [B, H, T, d]: a chunk = RPB consecutive positions of one head; chunks are numbered tensor, batch entry,
+//                 row block, head, so consecutive chunks share their positions and a thread forms its 8
+//                 sines and cosines once per row block.
+//   [B, T, H, d]: memory is a sequence of head vectors in (b, t, h) order; a chunk = RPB consecutive ones
+//                 (a few positions' worth).  The sines and cosines of a chunk's positions are formed once
+//                 per CTA, one chunk ahead, in a small shared-memory table.
+// A cursor is set once and then stepped.
+struct Cursor {
+  int which;            // 0: q, 1: k
+  int b, tb, h;         // [B, H, T, d]
+  int c;                // [B, T, H, d]: chunk inside the tensor; its first head vector is head h0 of
+  int h0, t0, b0;       //               position t0 of batch entry b0
 };
-__device__ __forceinline__ Chunk chunk_at(const QkArgs& a, int i) {
-  Chunk c;
-  const int n0 = a.B * a.nblk_t * a.H[0];
-  c.which = i >= n0;
-  if (c.which) i -= n0;
+// x / H for 0 <= x < 8192 without an integer division ((x + 0.5) / H is at least 0.5 / H away from an integer)
+__device__ __forceinline__ int small_div(int x, float inv_H) { return __float2int_rd(((float)x + 0.5f) * inv_H); }
+template <int RPB>
+__device__ __forceinline__ Cursor cursor_at(const QkArgs& a, int i) {
+  Cursor c;
+  c.which = i >= a.n_chunks[0];
+  if (c.which) i -= a.n_chunks[0];
+  c.c = i;
   const int H = a.H[c.which];
+  {
+    const long long bt = (long long)i * RPB / H;
+    c.h0 = (int)((long long)i * RPB - bt * H);
+    c.b0 = (int)(bt / a.T);
+    c.t0 = (int)(bt - (long long)c.b0 * a.T);
+  }
   const int rb = i / H;
   c.h = i - rb * H;
   c.b = rb / a.nblk_t;
   c.tb = rb - c.b * a.nblk_t;
   return c;
 }
-__device__ __forceinline__ void step(const QkArgs& a, Chunk& c) {
+template <bool BTHD, int RPB>
+__device__ __forceinline__ void step(const QkArgs& a, Cursor& c) {
+  if (BTHD) {
+    if (++c.c >= a.n_chunks[c.which]) {
+      c.c = c.h0 = c.t0 = c.b0 = 0;
+      ++c.which;
+      return;
+    }
+    c.h0 += RPB;                                   // the next run of RPB head vectors
+    const int carry = small_div(c.h0, a.inv_H[c.which]);
+    c.h0 -= carry * a.H[c.which];
+    c.t0 += carry;
+    while (c.t0 >= a.T) { c.t0 -= a.T; ++c.b0; }
+    return;
+  }
   if (++c.h < a.H[c.which]) return;
   c.h = 0;
   if (++c.tb < a.nblk_t) return;
@@ -172,8 +208,21 @@ __device__ __forceinline__ void step(const QkArgs& a, Chunk& c) {
   c.b = 0;
   ++c.which;
 }
+// byte offset of the cursor's chunk in its tensor and the rows of it that exist
+template <int RPB, int ROW, bool BTHD>
+__device__ __forceinline__ void where(const QkArgs& a, const Cursor& c, size_t* at, int* rows) {
+  const int H = a.H[c.which];
+  if (!BTHD) {
+    *rows = a.T - c.tb * RPB < RPB ? a.T - c.tb * RPB : RPB;
+    *at = (((size_t)c.b * H + c.h) * a.T + (size_t)c.tb * RPB) * ROW;
+  } else {
+    const int n_vec = a.B * a.T * H, v0 = c.c * RPB;          // < 2^31, checked on the host
+    *rows = n_vec - v0 < RPB ? n_vec - v0 : RPB;
+    *at = (size_t)v0 * ROW;
+  }
+}
 
-template <typename T, int D, bool BWD>
+template <typename T, int D, bool BWD, bool BTHD>
 __global__ void __launch_bounds__(QK_THREADS, BWD ? 2 : QK_CTAS_PER_SM)
 qk_prologue_kernel(const __grid_constant__ QkArgs a, const __grid_constant__ Freqs f) {
   using R = Ring<T, BWD>;
@@ -183,9 +232,10 @@ qk_prologue_kernel(const __grid_constant__ QkArgs a, const __grid_constant__ Fre
   float* red = reinterpret_cast<float*>(smem + S * R::kBufs * R::kChunk);         // [RPB][D] (backward)
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + S * R::kBufs * R::kChunk + R::kRed);
   volatile int* abort = reinterpret_cast<volatile int*>(full + S);
+  float2* tbl = reinterpret_cast<float2*>(smem + R::kBytes);                      // [2][tbl_tokens][D/2] (cos, sin)
 
   const int tid = threadIdx.x, l = tid % LPR, row = tid / LPR;
-  const long long n_all = (long long)a.B * a.nblk_t * (a.H[0] + a.H[1]);     // < 2^31, checked on the host
+  const long long n_all = (long long)a.n_chunks[0] + a.n_chunks[1];           // < 2^31, checked on the host
   const int lo = (int)(n_all * blockIdx.x / gridDim.x), hi = (int)(n_all * (blockIdx.x + 1) / gridDim.x);
 
   if (tid == 0) {
@@ -199,13 +249,13 @@ qk_prologue_kernel(const __grid_constant__ QkArgs a, const __grid_constant__ Fre
   }
   __syncthreads();
 
-  Chunk ahead = chunk_at(a, lo);                      // thread 0's cursor: the next chunk to load
+  Cursor ahead = cursor_at<RPB>(a, lo);                    // thread 0's cursor: the next chunk to load
   auto issue = [&](int i) {                           // thread 0 only; i must be the cursor's chunk
-    const Chunk c = ahead;
-    step(a, ahead);
-    const int H = a.H[c.which], t0 = c.tb * RPB;
-    const int rows = a.T - t0 < RPB ? a.T - t0 : RPB;
-    const size_t at = (((size_t)c.b * H + c.h) * a.T + t0) * D * sizeof(T);
+    const Cursor c = ahead;
+    step<BTHD, RPB>(a, ahead);
+    size_t at;
+    int rows;
+    where<RPB, ROW, BTHD>(a, c, &at, &rows);
     const int slot = (i - lo) % S;
     unsigned char* dst = stage + (size_t)slot * R::kBufs * R::kChunk;
     expect_tx(&full[slot], (uint32_t)(rows * ROW * R::kBufs));
@@ -239,10 +289,38 @@ qk_prologue_kernel(const __grid_constant__ QkArgs a, const __grid_constant__ Fre
     __syncthreads();
   };
 
+  // [B, T, H, d]: cos and sin of every (position, pair) of the cursor's chunk into table `buf`, one entry per
+  // thread and round (a chunk of RPB head vectors spans RPB / H positions, plus one when it straddles)
+  const bool tabled = BTHD && a.rotate;
+  auto fill_table = [&](const Cursor& cx, int buf) {
+    constexpr double kTwoPi = 6.283185307179586476925286766559;
+    size_t at_;
+    int rows_;
+    where<RPB, ROW, BTHD>(a, cx, &at_, &rows_);
+    const int n_tok = small_div(cx.h0 + rows_ - 1, a.inv_H[cx.which]) + 1;
+    for (int e = tid; e < n_tok * (D / 2); e += QK_THREADS) {
+      const int tok = e / (D / 2), pair = e % (D / 2);
+      int t = cx.t0 + tok, b = cx.b0;
+      while (t >= a.T) { t -= a.T; ++b; }
+      const long long position = (a.pos ? (long long)a.pos[b] : a.pos0) + t;
+      double ang = (double)position * f.inv[pair];
+      ang -= kTwoPi * rint(ang * (1.0 / kTwoPi));
+      float sn, cs;
+      sincosf((float)ang, &sn, &cs);
+      tbl[((size_t)buf * a.tbl_tokens + tok) * (D / 2) + pair] = make_float2(cs, sn);
+    }
+  };
+  Cursor ch = cursor_at<RPB>(a, lo);
+  if (tabled && lo < hi) fill_table(ch, 0);
+  if (!a.rotate) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) { c[j] = 1.f; s[j] = 0.f; }
+  }
+  __syncthreads();
+
   int i = lo;
   bool ok = true;
-  Chunk ch = chunk_at(a, lo);
-  for (; i < hi; ++i, step(a, ch)) {
+  for (; i < hi; ++i, step<BTHD, RPB>(a, ch)) {
     const int n = i - lo, slot = n % S;
     if (ch.which != cur_which) {
       if (BWD && a.partial != nullptr && cur_which >= 0) flush(cur_which);
@@ -250,14 +328,30 @@ qk_prologue_kernel(const __grid_constant__ QkArgs a, const __grid_constant__ Fre
       cur_which = ch.which;
       cur_rb = -1;
     }
-    const int rb = ch.b * a.nblk_t + ch.tb;
-    const int t = ch.tb * RPB + row;
-    if (rb != cur_rb) {
-      const long long p0 = a.pos ? (long long)a.pos[ch.b] : a.pos0;
-      rotation(f, 8 * l, p0 + t, a.rotate, c, s);
-      cur_rb = rb;
+    size_t ch_at;
+    int ch_rows;
+    where<RPB, ROW, BTHD>(a, ch, &ch_at, &ch_rows);
+    if (!BTHD) {
+      const int rb = ch.b * a.nblk_t + ch.tb;
+      if (rb != cur_rb && a.rotate) {
+        const long long p0 = a.pos ? (long long)a.pos[ch.b] : a.pos0;
+        rotation(f, 8 * l, p0 + ch.tb * RPB + row, a.rotate, c, s);
+        cur_rb = rb;
+      }
+    } else if (tabled) {
+      // the next chunk's table while this chunk's data is on its way; this chunk's was written one
+      // iteration ago (or before the loop) and the barrier in between made it visible
+      if (i + 1 < hi) {
+        Cursor nx = ch;
+        step<BTHD, RPB>(a, nx);
+        fill_table(nx, (n + 1) & 1);
+      }
+      const int tok = small_div(ch.h0 + row, a.inv_H[ch.which]);
+      const float2* e = tbl + ((size_t)(n & 1) * a.tbl_tokens + (row < ch_rows ? tok : 0)) * (D / 2) + 8 * l;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { c[j] = e[j].x; s[j] = e[j].y; }
     }
-    const bool live = t < a.T;
+    const bool live = row < ch_rows;
     unsigned char* buf = stage + (size_t)slot * R::kBufs * R::kChunk + (size_t)row * ROW;
     const bool got = ptx::mbar_wait_warp(&full[slot], (uint32_t)(n / S) & 1u, abort);
     if (got) {
@@ -324,9 +418,8 @@ qk_prologue_kernel(const __grid_constant__ QkArgs a, const __grid_constant__ Fre
     ok = __syncthreads_and(got) != 0;
     if (!ok) break;
     if (tid == 0) {
-      const int H = a.H[ch.which], t0 = ch.tb * RPB;
-      const int rows = a.T - t0 < RPB ? a.T - t0 : RPB;
-      const size_t at = (((size_t)ch.b * H + ch.h) * a.T + t0) * D * sizeof(T);
+      const int rows = ch_rows;
+      const size_t at = ch_at;
       unsigned char* src = stage + (size_t)slot * R::kBufs * R::kChunk + (BWD ? R::kChunk : 0);
       bulk_store(static_cast<unsigned char*>(a.y[ch.which]) + at, src, (uint32_t)(rows * ROW));
       ptx::tma_store_commit();
@@ -388,8 +481,12 @@ int check(const rattn_qk_params* p) {
   if (misaligned16(p->q) || misaligned16(p->k) || misaligned16(p->q_gain) || misaligned16(p->k_gain))
     return RATTN_ERR_MISALIGNED;
   if (((uintptr_t)p->pos & 3u) != 0) return RATTN_ERR_MISALIGNED;
+  if (p->layout != RATTN_LAYOUT_BHTD && p->layout != RATTN_LAYOUT_BTHD) return RATTN_ERR_UNSUPPORTED;
   const int rpb = QK_THREADS / (p->d / 16);
   if ((long long)p->B * ((p->T + rpb - 1) / rpb) * ((long long)p->H_q + p->H_kv) >= (1ll << 31)) return RATTN_ERR_BAD_ARG;
+  if (p->layout == RATTN_LAYOUT_BTHD && ((long long)p->B * p->T * (p->H_q > p->H_kv ? p->H_q : p->H_kv) >= (1ll << 31) ||
+                                         p->H_q > 4096 || p->H_kv > 4096))
+    return RATTN_ERR_BAD_ARG;
   return RATTN_OK;
 }
 
@@ -397,8 +494,19 @@ void fill(const rattn_qk_params* p, QkArgs* a, Freqs* f) {
   a->x[0] = p->q; a->x[1] = p->k;
   a->gain[0] = p->q_gain; a->gain[1] = p->k_gain;
   a->H[0] = p->H_q; a->H[1] = p->H_kv;
+  a->inv_H[0] = 1.f / (float)p->H_q; a->inv_H[1] = p->H_kv > 0 ? 1.f / (float)p->H_kv : 0.f;
   const int rpb = QK_THREADS / (p->d / 16);
   a->B = p->B; a->T = p->T; a->nblk_t = (p->T + rpb - 1) / rpb;
+  a->layout = p->layout;
+  a->tbl_tokens = 0;
+  for (int w = 0; w < 2; ++w) {     // [B,H,T,d]: row blocks x heads; [B,T,H,d]: runs of rpb head vectors
+    a->n_chunks[w] = p->layout == RATTN_LAYOUT_BHTD ? p->B * a->nblk_t * a->H[w]
+                                                    : (int)(((long long)p->B * p->T * a->H[w] + rpb - 1) / rpb);
+    if (p->layout != RATTN_LAYOUT_BHTD && a->H[w] > 0 && p->theta > 0.f) {
+      const int tokens = (rpb + a->H[w] - 1) / a->H[w] + 1;      // positions a chunk can touch
+      if (tokens > a->tbl_tokens) a->tbl_tokens = tokens;
+    }
+  }
   a->eps = p->eps;
   a->rotate = p->theta > 0.f;
   a->pos0 = p->pos0;
@@ -416,22 +524,28 @@ cudaError_t grid_size(const QkArgs& a, int per_sm, int* n_cta) {
   cudaError_t e = cudaGetDevice(&dev);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
-  long long n = (long long)a.B * a.nblk_t * (a.H[0] + a.H[1]);
+  long long n = (long long)a.n_chunks[0] + a.n_chunks[1];
   if (n > (long long)n_sm * per_sm) n = (long long)n_sm * per_sm;
   if (n > QK_MAX_CTAS) n = QK_MAX_CTAS;
   *n_cta = (int)n;
   return cudaSuccess;
 }
 
-template <typename T, int D, bool BWD>
-cudaError_t launch_one(const QkArgs& a, const Freqs& f, int n_cta, cudaStream_t s) {
-  constexpr int smem = Ring<T, BWD>::kBytes;
-  cudaError_t e = cudaFuncSetAttribute(qk_prologue_kernel<T, D, BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+template <typename T, int D, bool BWD, bool BTHD>
+cudaError_t launch_layout(const QkArgs& a, const Freqs& f, int n_cta, cudaStream_t s) {
+  const int smem = Ring<T, BWD>::kBytes + 2 * a.tbl_tokens * (D / 2) * (int)sizeof(float2);
+  cudaError_t e = cudaFuncSetAttribute(qk_prologue_kernel<T, D, BWD, BTHD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
   KernelTimer kt(BWD ? "qk_prologue_bwd" : "qk_prologue", s);
-  qk_prologue_kernel<T, D, BWD><<<n_cta, QK_THREADS, smem, s>>>(a, f);
+  qk_prologue_kernel<T, D, BWD, BTHD><<<n_cta, QK_THREADS, smem, s>>>(a, f);
   count_launches(1);
   return cudaGetLastError();
+}
+
+template <typename T, int D, bool BWD>
+cudaError_t launch_one(const QkArgs& a, const Freqs& f, int n_cta, cudaStream_t s) {
+  return a.layout == RATTN_LAYOUT_BHTD ? launch_layout<T, D, BWD, false>(a, f, n_cta, s)
+                                       : launch_layout<T, D, BWD, true>(a, f, n_cta, s);
 }
 
 template <bool BWD>

@@ -163,27 +163,35 @@ def test_prologue_argument_checks():
 
 
 # ---------------------------------------------------------------- a stack of attention layers
-def gpu_layer(x, lay, *, H_q, H_kv, d, w, local, scale, dt, flags=0):
+def gpu_layer(x, lay, *, H_q, H_kv, d, w, local, scale, dt, layout, flags=0):
     """The oracle's layer with the library's kernels for the prologue and the operator, and torch
-    for what surrounds them (RMS norm of the layer input, the four projections, the residual add)."""
+    for what surrounds them (RMS norm of the layer input, the four projections, the residual add).
+    With the [B, T, H, d] layout the projections' outputs are used as they are: no transposing copy."""
     Wq, Wk, Wv, Wo, gq, gk = lay
     B, T, D = x.shape
     h = F.rms_norm(x, (D,), eps=1e-6).to(dt)
-    heads = lambda z, H: z.reshape(B, T, H, d).transpose(1, 2).contiguous()
+    if layout == R.LAYOUT_BTHD:
+        heads = lambda z, H: z.reshape(B, T, H, d)
+        merge = lambda y: y.reshape(B, T, H_q * d)
+    else:
+        heads = lambda z, H: z.reshape(B, T, H, d).transpose(1, 2).contiguous()
+        merge = lambda y: y.transpose(1, 2).reshape(B, T, H_q * d)
     q, k, v = heads(h @ Wq.to(dt), H_q), heads(h @ Wk.to(dt), H_kv), heads(h @ Wv.to(dt), H_kv)
-    R.rattn_qk_prologue(q, k, q_gain=gq, k_gain=gk, theta=P.THETA_LOCAL if local else None, inplace=True)
+    R.rattn_qk_prologue(q, k, q_gain=gq, k_gain=gk, theta=P.THETA_LOCAL if local else None, inplace=True,
+                        layout=layout)
     mode = R.MODE_RATTN if local else R.MODE_FULL_CAUSAL
-    ws = R.alloc_workspace(q, k, w, mode, flags)
-    y = R.rattn_forward_ex(q, k, v, w, scale=scale, mode=mode, workspace=ws, flags=flags)
+    ws = R.alloc_workspace(q, k, w, mode, flags, layout=layout)
+    y = R.rattn_forward_ex(q, k, v, w, scale=scale, mode=mode, workspace=ws, flags=flags, layout=layout)
     assert R.rattn_read_status(ws) == 0
-    return x + (y.transpose(1, 2).reshape(B, T, H_q * d) @ Wo.to(dt)).float()
+    return x + (merge(y) @ Wo.to(dt)).float()
 
 
+@pytest.mark.parametrize("layout", [R.LAYOUT_BHTD, R.LAYOUT_BTHD])
 @pytest.mark.parametrize("dtype,D,H_q,H_kv,d,T,w,tol", [
     ("f32", 128, 4, 2, 64, 160, 32, 2e-4),       # portable fp32 kernels
     ("bf16", 256, 4, 2, 128, 640, 128, 3e-2),    # tensor-core kernels
 ])
-def test_local_local_local_global_stack(dtype, D, H_q, H_kv, d, T, w, tol):
+def test_local_local_local_global_stack(dtype, D, H_q, H_kv, d, T, w, tol, layout):
     """Three local layers (RAttention with rotary q, k) and one global layer (full causal attention,
     no rotary), Section 4 "Model Setup", on synthetic weights: relative Frobenius error of the
     final residual stream.  bf16: every layer rounds q, k, v, y to bf16 and the operator's own error
@@ -205,6 +213,37 @@ def test_local_local_local_global_stack(dtype, D, H_q, H_kv, d, T, w, tol):
         if dtype == "bf16":
             assert R.rattn_uses_tensor_path(d, w, R.RATTN_BF16, R.MODE_RATTN)
         y = gpu_layer(y, tuple(t.cuda() for t in lay), H_q=H_q, H_kv=H_kv, d=d, w=w, local=(l + 1) % 4 != 0,
-                      scale=scale, dt=dt)
+                      scale=scale, dt=dt, layout=layout)
     torch.cuda.synchronize()
     assert rel_fro(np64(y), ref) <= tol, rel_fro(np64(y), ref)
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,T,d,dtype,theta", [
+    (2, 16, 4, 300, 128, "bf16", 5.0e5),      # 16 and 4 heads: two and eight positions per chunk
+    (1, 40, 8, 130, 128, "f32", 5.0e5),       # 40 heads: a chunk is part of one position's heads
+    (2, 3, 1, 77, 64, "bf16", 5.0e5),         # head counts that do not divide the chunk
+    (2, 4, 2, 200, 128, "bf16", None),
+])
+def test_prologue_in_bthd_layout(B, Hq, Hkv, T, d, dtype, theta):
+    """[B, T, H, d] tensors: forward outputs and input gradients carry the same bits as the default layout
+    (the same arithmetic per head vector); gain gradients are summed in another order."""
+    q, k, gq, gk = make(B, Hq, Hkv, T, d, dtype, 9700 + T)
+    g = torch.Generator().manual_seed(78)
+    dqo = torch.randn(q.shape, generator=g).to(q.dtype)
+    dko = torch.randn(k.shape, generator=g).to(k.dtype)
+    tr = lambda x: x.transpose(1, 2).contiguous()
+    pos = torch.arange(B, dtype=torch.int32) * 1000 + 17
+    kw = dict(q_gain=cu(gq), k_gain=cu(gk), theta=theta, pos=pos.cuda())
+    qa, ka = R.rattn_qk_prologue(q.cuda(), k.cuda(), **kw)
+    qb, kb = R.rattn_qk_prologue(tr(q).cuda(), tr(k).cuda(), layout=R.LAYOUT_BTHD, **kw)
+    assert torch.equal(tr(qb), qa) and torch.equal(tr(kb), ka)
+    ga = R.rattn_qk_prologue_backward(q.cuda(), k.cuda(), dqo.cuda(), dko.cuda(), **kw)
+    gb = R.rattn_qk_prologue_backward(tr(q).cuda(), tr(k).cuda(), tr(dqo).cuda(), tr(dko).cuda(),
+                                      layout=R.LAYOUT_BTHD, **kw)
+    assert torch.equal(tr(gb[0]), ga[0]) and torch.equal(tr(gb[1]), ga[1])
+    for x, y in ((ga[2], gb[2]), (ga[3], gb[3])):
+        assert (x - y).abs().max() <= 1e-4 * x.abs().max()
+    assert R.rattn_qk_prologue_status() == 0
+    for b in range(B):
+        p = int(pos[b]) + np.arange(T)
+        close(tr(qb)[b], P.qk_prologue(np64(q[b]), np64(gq), p, theta), dtype, f"q entry {b}")
