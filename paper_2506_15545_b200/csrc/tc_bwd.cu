@@ -703,11 +703,11 @@ constexpr int KV_OFF_STAGE = 4 * TILE_BYTES;               // KV_NS x [Q_h 16 KB
 constexpr int KV_OFF_STAT = KV_OFF_STAGE + KV_NS * TILE_BYTES;   // KV_NS x (lse2[64], D*scale[64]) fp32
 constexpr int KV_OFF_BAR = KV_OFF_STAT + KV_NS * 512;
 constexpr int KV_SMEM = KV_OFF_BAR + 256;
-constexpr int KV_THREADS = 320;                            // 2 row groups, MMA warp, loader warp
+constexpr int KV_THREADS = 352;                            // 2 row groups, score warp, loader warp, accumulate warp
 
 struct KvBars {
   uint64_t kv_full, kphi_ready, full[KV_NS], acc_done[KV_NS], s_full[2], p_ready[2], phiq_ready[2],
-      r_acc_done, fold_done, all_done, acc_free, drain;
+      r_acc_done, fold_done, all_done, acc_free, drain, drain2;
   uint32_t tmem_base;
   int abort;
 };
@@ -799,24 +799,68 @@ __device__ bool kv_loader(const KvMaps& tm, const BwdArgs& a, unsigned char* sme
   return true;
 }
 
-__device__ bool kv_mma(const BwdArgs& a, unsigned char* smem, KvBars* bars, uint32_t tmem, int n_items) {
+// The products are issued by two warps: the score warp issues S^T and dP^T of every item, the accumulate
+// warp everything that writes the dV / dK accumulators, so that the waits of one (a wait that is already
+// satisfied still costs an issuing warp some 300 cycles) pass under the products of the other.  A third
+// issuer (S^T and dP^T apart) measured no faster: what then limits an item is the chain scores -> row
+// group -> accumulate on its TMEM slot, of which there are two.  Order between the two warps:
+//   scores(n) -> row group -> p_ready -> accumulate(n)        (existing barriers)
+//   accumulate(n - 2) complete -> scores(n) may overwrite the TMEM slot they share   (acc_done of n - 2's stage)
+__device__ bool kv_mma_scores(const BwdArgs& a, unsigned char* smem, KvBars* bars, uint32_t tmem, int n_items) {
   const uint32_t sK = smem_u32(smem + KV_OFF_K), sV = smem_u32(smem + KV_OFF_V), sKphi = smem_u32(smem + KV_OFF_KPHI);
   const uint32_t sStage = smem_u32(smem + KV_OFF_STAGE);
-  const uint32_t tV = tmem, tK = tmem + 128;
   const uint32_t tS[2] = {tmem + 256, tmem + 384}, tP[2] = {tmem + 320, tmem + 448};
   KvCount c = {0, 0, 0, 0};
   int cq[2] = {0, 0};                                      // phi(Q_h) hand-overs per TMEM slot
 
   for (int idx = blockIdx.x; idx < n_items; idx += gridDim.x, ++c.it) {
     const KvPlan pl = kv_plan(a, idx);
-    bool accV = false, accK = false;
+    // K_j, V_j have landed (which also means every product of the previous key tile has completed)
     WAIT_OR_RETURN_W(bars->kv_full, c.it & 1);
     if (pl.n_R > 0) WAIT_OR_RETURN_W(bars->kphi_ready, c.cr & 1);
+    if (pl.has_inter) ++c.seq;                             // the reverse state's ring slot (accumulate warp)
+    const int seq0 = c.seq, gi0 = c.gi;
+    for (int n = 0; n < pl.N; ++n) {
+      const int st = (seq0 + n) % KV_NS, use = (seq0 + n) / KV_NS, slot = (gi0 + n) & 1;
+      const uint32_t sQh = sStage + st * TILE_BYTES, sGh = sQh + HT_BYTES;
+      WAIT_OR_RETURN_W(bars->full[st], use & 1);
+      if (pl.is_r(n)) {
+        WAIT_OR_RETURN_W(bars->phiq_ready[slot], cq[slot] & 1);
+        ++cq[slot];
+      }
+      if (n >= 2) {                                        // the slot's previous item has been accumulated
+        const int st2 = (seq0 + n - 2) % KV_NS, use2 = (seq0 + n - 2) / KV_NS;
+        WAIT_OR_RETURN_W(bars->acc_done[st2], use2 & 1);
+      }
+      tc_fence_after();
+      mma_k_kh(tS[slot], pl.is_r(n) ? sKphi : sK, sQh);     // S^T  = K Q_h^T   (phi(K) phi(Q_h)^T)
+      mma_k_kh(tP[slot], sV, sGh);                           // dP^T = V g_h^T
+      mma_commit(&bars->s_full[slot]);
+    }
+    c.seq += pl.N;
+    c.gi += pl.N;
+    if (pl.n_R > 0) ++c.cr;
+  }
+  return true;
+}
+
+__device__ bool kv_mma_accum(const BwdArgs& a, unsigned char* smem, KvBars* bars, uint32_t tmem, int n_items) {
+  const uint32_t sV = smem_u32(smem + KV_OFF_V), sKphi = smem_u32(smem + KV_OFF_KPHI);
+  const uint32_t sStage = smem_u32(smem + KV_OFF_STAGE);
+  const uint32_t tV = tmem, tK = tmem + 128;
+  const uint32_t tS[2] = {tmem + 256, tmem + 384}, tP[2] = {tmem + 320, tmem + 448};
+  KvCount c = {0, 0, 0, 0};
+
+  for (int idx = blockIdx.x; idx < n_items; idx += gridDim.x, ++c.it) {
+    const KvPlan pl = kv_plan(a, idx);
+    bool accV = false, accK = false;
     // the previous key tile's epilogue has read the two accumulators
     bool acc_ok = (c.it == 0);
     if (pl.has_inter) {
       const int st = c.seq % KV_NS, use = c.seq / KV_NS;
       ++c.seq;
+      WAIT_OR_RETURN_W(bars->kv_full, c.it & 1);
+      WAIT_OR_RETURN_W(bars->kphi_ready, c.cr & 1);
       WAIT_OR_RETURN_W(bars->full[st], use & 1);
       if (!acc_ok) { WAIT_OR_RETURN_W(bars->acc_free, (c.it - 1) & 1); acc_ok = true; }
       tc_fence_after();
@@ -826,36 +870,18 @@ __device__ bool kv_mma(const BwdArgs& a, unsigned char* smem, KvBars* bars, uint
       accV = accK = true;
     }
     const int seq0 = c.seq, gi0 = c.gi;
-    for (int n = 0; n <= pl.N; ++n) {
-      if (n < pl.N) {
-        const int st = (seq0 + n) % KV_NS, use = (seq0 + n) / KV_NS, slot = (gi0 + n) & 1;
-        const uint32_t sQh = sStage + st * TILE_BYTES, sGh = sQh + HT_BYTES;
-        WAIT_OR_RETURN_W(bars->full[st], use & 1);
-        if (pl.is_r(n)) {
-          WAIT_OR_RETURN_W(bars->phiq_ready[slot], cq[slot] & 1);
-          ++cq[slot];
-        }
-        // The slot's previous user needs no wait here: its row groups were waited for before its
-        // accumulate products were issued, and those precede these scores in the tensor pipe,
-        // which executes in issue order.
-        tc_fence_after();
-        mma_k_kh(tS[slot], pl.is_r(n) ? sKphi : sK, sQh);   // S^T  = K Q_h^T   (phi(K) phi(Q_h)^T)
-        mma_k_kh(tP[slot], sV, sGh);                         // dP^T = V g_h^T
-        mma_commit(&bars->s_full[slot]);
-      }
-      if (n >= 1) {
-        const int m = n - 1, st = (seq0 + m) % KV_NS, slot = (gi0 + m) & 1;
-        const uint32_t sQh = sStage + st * TILE_BYTES, sGh = sQh + HT_BYTES;
-        WAIT_OR_RETURN_W(bars->p_ready[slot], ((gi0 + m) >> 1) & 1);
-        if (m == pl.n_R && pl.n_R > 0) WAIT_OR_RETURN_W(bars->fold_done, c.cr & 1);
-        if (!acc_ok) { WAIT_OR_RETURN_W(bars->acc_free, (c.it - 1) & 1); acc_ok = true; }
-        tc_fence_after();
-        mma_ts_h(tV, tS[slot], sGh, accV);                   // dV += P^T g_h
-        mma_ts_h(tK, tP[slot], sQh, accK);                   // dK += dS^T Q_h   (dphi_k += dA^T phi(Q_h))
-        accV = accK = true;
-        mma_commit(&bars->acc_done[st]);
-        if (m == pl.n_R - 1) mma_commit(&bars->r_acc_done);
-      }
+    for (int m = 0; m < pl.N; ++m) {
+      const int st = (seq0 + m) % KV_NS, slot = (gi0 + m) & 1;
+      const uint32_t sQh = sStage + st * TILE_BYTES, sGh = sQh + HT_BYTES;
+      WAIT_OR_RETURN_W(bars->p_ready[slot], ((gi0 + m) >> 1) & 1);
+      if (m == pl.n_R && pl.n_R > 0) WAIT_OR_RETURN_W(bars->fold_done, c.cr & 1);
+      if (!acc_ok) { WAIT_OR_RETURN_W(bars->acc_free, (c.it - 1) & 1); acc_ok = true; }
+      tc_fence_after();
+      mma_ts_h(tV, tS[slot], sGh, accV);                   // dV += P^T g_h
+      mma_ts_h(tK, tP[slot], sQh, accK);                   // dK += dS^T Q_h   (dphi_k += dA^T phi(Q_h))
+      accV = accK = true;
+      mma_commit(&bars->acc_done[st]);
+      if (m == pl.n_R - 1) mma_commit(&bars->r_acc_done);
     }
     c.seq += pl.N;
     c.gi += pl.N;
@@ -1101,6 +1127,7 @@ tc_bwd_dkv_kernel(const __grid_constant__ KvMaps tm, BwdArgs a, int n_items) {
     mbar_init(&bars->all_done, 1);
     mbar_init(&bars->acc_free, 256);
     mbar_init(&bars->drain, 1);
+    mbar_init(&bars->drain2, 1);
     bars->abort = 0;
     fence_mbar_init();
   }
@@ -1126,11 +1153,12 @@ tc_bwd_dkv_kernel(const __grid_constant__ KvMaps tm, BwdArgs a, int n_items) {
   bool ok = true;
   if (warp < 8) {
     ok = kv_rows(tm, a, smem, bars, tmem, warp >> 2, tid & 127, n_items);
-  } else if (warp == 8) {
-    ok = kv_mma(a, smem, bars, tmem, n_items);
-    if (!ok) {
-      mma_commit(&bars->drain);
-      for (int it = 0; it < (1 << 16) && !mbar_try_wait(&bars->drain, 0); ++it) {}
+  } else if (warp == 8 || warp == 10) {
+    ok = warp == 8 ? kv_mma_scores(a, smem, bars, tmem, n_items) : kv_mma_accum(a, smem, bars, tmem, n_items);
+    if (!ok) {                                             // let this warp's products in flight finish
+      uint64_t* drain = warp == 8 ? &bars->drain : &bars->drain2;
+      mma_commit(drain);
+      for (int it = 0; it < (1 << 16) && !mbar_try_wait(drain, 0); ++it) {}
     }
   } else if (warp == 9) {
     ok = kv_loader(tm, a, smem, bars, n_items);
