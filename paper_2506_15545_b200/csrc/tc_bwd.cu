@@ -312,7 +312,7 @@ constexpr int DQ_SMEM = DQ_OFF_BAR + 256;
 constexpr int DQ_THREADS = 320;            // 2 row groups, MMA warp, loader warp
 
 struct DqBars {
-  uint64_t qg_full, kv_full[2], kv_free[2], s_full, ds_full, phik_ready, o_done, acc_free, drain;
+  uint64_t qg_full, kv_full[2], kv_free[2], s_full, ds_full, phik_ready, o_done, acc_free, q_read, drain;
   uint32_t tmem_base;
   int abort;
 };
@@ -358,7 +358,10 @@ __device__ bool dq_loader(const DqMaps& tm, const BwdArgs& a, unsigned char* sme
     if (n >= 1) WAIT_OR_RETURN_W(bars->qg_full, (n - 1) & 1);
     mbar_arrive_expect_tx(&bars->qg_full, 2 * TILE_BYTES);
     // Q into the buffer last used two items ago: free once that item's epilogue has left it
-    if (n >= 2) WAIT_OR_RETURN_W(bars->acc_free, (n - 2) & 1);
+    if (n >= 2) {
+      WAIT_OR_RETURN_W(bars->acc_free, (n - 2) & 1);
+      WAIT_OR_RETURN_W(bars->q_read, (n - 2) & 1);      // and its dQ, staged there, has left
+    }
     load_tile(smem + ((n & 1) ? DQ_OFF_Q1 : DQ_OFF_Q), &tm.q, &bars->qg_full, it.q0, it.bh_q);
     // g_s: its one buffer is free once every product of the previous item has completed
     // (o_done completes twice for an item with a residual part, once otherwise)
@@ -442,6 +445,7 @@ __device__ bool dq_rows(const DqMaps& tm, const BwdArgs& a, unsigned char* smem,
   const uint32_t tS = tmem + lane_off, tP = tmem + 128 + lane_off, tQ = tmem + 256 + lane_off,
                  tF = tmem + 384 + lane_off;
   int kc = 0, n = 0, cs = 0, co = 0;                       // ring uses, items, score hand-overs, o_done completions
+  bool store_pending = false;                              // this thread issued a dQ store whose read-out it has not confirmed
   for (int idx = blockIdx.x; idx < n_items; idx += gridDim.x, ++n) {
     const DqItem it = dq_item(a, idx, n_qt);
     const int n_kt = it.n_kt;
@@ -485,6 +489,11 @@ __device__ bool dq_rows(const DqMaps& tm, const BwdArgs& a, unsigned char* smem,
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&bars->ds_full);
+      if (i == 0 && store_pending) {                         // the previous item's dQ has left its Q buffer by now
+        tma_store_wait_read();
+        mbar_arrive(&bars->q_read);
+        store_pending = false;
+      }
     }
     kc += n_kt;
 
@@ -602,17 +611,19 @@ __device__ bool dq_rows(const DqMaps& tm, const BwdArgs& a, unsigned char* smem,
         *reinterpret_cast<uint4*>(sQ + swz(r, 4 * c + e)) = u;
       }
     }
-    fence_proxy_async_smem();
     tc_fence_before();
+    mbar_arrive(&bars->acc_free);          // the dQ / dphi_q columns have been read
+    fence_proxy_async_smem();
     rows_sync();
     if (r == 0) {
+      // nobody waits for the store to read the Q buffer out: the loader refills that buffer two items
+      // on, after q_read, which this thread confirms once the next item's first key tile is behind it
       store_tile(&tm.dq, sQ, it.q0, it.bh_q);
       tma_store_commit();
-      tma_store_wait_read();
+      store_pending = true;
     }
-    rows_sync();
-    mbar_arrive(&bars->acc_free);          // dQ / dphi_q columns and this Q buffer may be reused
   }
+  if (store_pending) tma_store_wait();     // the last store has completed before the CTA may go
   return true;
 }
 
@@ -636,6 +647,7 @@ tc_bwd_dq_kernel(const __grid_constant__ DqMaps tm, BwdArgs a, int n_items, int 
     mbar_init(&bars->phik_ready, 256);
     mbar_init(&bars->o_done, 1);
     mbar_init(&bars->acc_free, 128);
+    mbar_init(&bars->q_read, 1);
     mbar_init(&bars->drain, 1);
     bars->abort = 0;
     fence_mbar_init();
@@ -707,7 +719,7 @@ constexpr int KV_THREADS = 352;                            // 2 row groups, scor
 
 struct KvBars {
   uint64_t kv_full, kphi_ready, full[KV_NS], acc_done[KV_NS], s_full[2], p_ready[2], phiq_ready[2],
-      r_acc_done, fold_done, all_done, acc_free, drain, drain2;
+      r_acc_done, fold_done, all_done, acc_free, out_read, drain, drain2;
   uint32_t tmem_base;
   int abort;
 };
@@ -763,10 +775,14 @@ __device__ bool kv_loader(const KvMaps& tm, const BwdArgs& a, unsigned char* sme
     mbar_arrive_expect_tx(&bars->kv_full, 2 * TILE_BYTES);
     load_tile(smem + KV_OFF_K, &tm.k, &bars->kv_full, j0, pl.bh_kv);
     load_tile(smem + KV_OFF_V, &tm.v, &bars->kv_full, j0, pl.bh_kv);
+    // dK of the previous key tile left through the ring slot this tile uses third: its store must
+    // have read the slot out first
+    const int gate_seq = c.seq + 2;
     auto ring = [&](int& st) -> bool {                     // next ring slot, once its previous user is consumed
       st = c.seq % KV_NS;
       const int use = c.seq / KV_NS;
       if (use >= 1) WAIT_OR_RETURN_W(bars->acc_done[st], (use - 1) & 1);
+      if (c.it >= 1 && c.seq == gate_seq) WAIT_OR_RETURN_W(bars->out_read, (c.it - 1) & 1);
       ++c.seq;
       return true;
     };
@@ -915,6 +931,11 @@ __device__ bool kv_rows(const KvMaps& tm, const BwdArgs& a, unsigned char* smem,
       fence_proxy_async_smem();
       mbar_arrive(&bars->kphi_ready);
     }
+    // the previous key tile's dK has long left its ring slot by now: tell the loader
+    if (gg == 0 && r == 0 && cnt.it >= 1) {
+      tma_store_wait_read();
+      mbar_arrive(&bars->out_read);
+    }
   }
   const int seq0 = cnt.seq + (pl.has_inter ? 1 : 0), gi0 = cnt.gi;
 
@@ -1058,12 +1079,16 @@ __device__ bool kv_rows(const KvMaps& tm, const BwdArgs& a, unsigned char* smem,
     }
   }
 
-  // every product has completed: group 0 stores dK (staged in the phi(K) tile), group 1 dV
-  // (staged in its own tile), each written by one TMA store
+  // every product has completed: group 1 stores dV, staged in its own tile; group 0 stores dK, staged
+  // in the ring slot that the next key tile uses third (its last user was this tile's last item), so
+  // that nobody has to wait for a store to read its source out: phi(K) of the next tile goes to its
+  // own tile at once, and the loader waits for out_read before it refills that slot
   if (gg < 2) {
     WAIT_OR_RETURN(bars->all_done, cnt.it & 1);
     tc_fence_after();
-    unsigned char* sOut = smem + (gg == 0 ? KV_OFF_KPHI : KV_OFF_OUT);
+    if (gg == 1 && r == 0) tma_store_wait_read();            // the previous dV has left the staging tile
+    if (gg == 1) group_sync(1);
+    unsigned char* sOut = gg == 0 ? smem + KV_OFF_STAGE + ((seq0 + pl.N + 2) % KV_NS) * TILE_BYTES : smem + KV_OFF_OUT;
     const uint32_t tOut = gg == 0 ? tK : tV;
 #pragma unroll 1
     for (int cc = 0; cc < 4; ++cc) {
@@ -1080,24 +1105,21 @@ __device__ bool kv_rows(const KvMaps& tm, const BwdArgs& a, unsigned char* smem,
         *reinterpret_cast<uint4*>(sOut + swz(r, 4 * cc + e)) = u;
       }
     }
-    fence_proxy_async_smem();
     tc_fence_before();
+    mbar_arrive(&bars->acc_free);                              // the accumulators have been read
+    fence_proxy_async_smem();
     group_sync(gg);
     if (r == 0) {
       store_tile(gg == 0 ? &tm.dk : &tm.dv, sOut, pl.j * TILE, bh_kv);
       tma_store_commit();
-      tma_store_wait_read();
     }
-    // both staging tiles have been read by their stores before either group goes on (the next
-    // key tile's phi(K) is written by both groups into the tile that staged dK)
-    asm volatile("bar.sync 6, 256;" ::: "memory");
-    mbar_arrive(&bars->acc_free);
   }
   cnt.seq = seq0 + pl.N;
   cnt.gi += pl.N;
   if (pl.n_R > 0) ++cnt.cr;
   ++cnt.it;
   }
+  if (r == 0) tma_store_wait();                               // this thread's last store has completed
   return true;
 }
 
@@ -1126,6 +1148,7 @@ tc_bwd_dkv_kernel(const __grid_constant__ KvMaps tm, BwdArgs a, int n_items) {
     mbar_init(&bars->fold_done, 128);
     mbar_init(&bars->all_done, 1);
     mbar_init(&bars->acc_free, 256);
+    mbar_init(&bars->out_read, 1);
     mbar_init(&bars->drain, 1);
     mbar_init(&bars->drain2, 1);
     bars->abort = 0;
