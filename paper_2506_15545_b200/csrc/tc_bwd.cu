@@ -1091,19 +1091,22 @@ __device__ bool kv_rows(const KvMaps& tm, const BwdArgs& a, unsigned char* smem,
     unsigned char* sOut = gg == 0 ? smem + KV_OFF_STAGE + ((seq0 + pl.N + 2) % KV_NS) * TILE_BYTES : smem + KV_OFF_OUT;
     const uint32_t tOut = gg == 0 ? tK : tV;
 #pragma unroll 1
-    for (int cc = 0; cc < 4; ++cc) {
-      float x[32];
-      tmem_ld32(tOut + 32 * cc, x);
+    for (int cc = 0; cc < 4; cc += 2) {                        // two loads in flight
+      float x[2][32];
+      tmem_ld32(tOut + 32 * cc, x[0]);
+      tmem_ld32(tOut + 32 * (cc + 1), x[1]);
       tmem_wait_ld();
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        uint4 u;
-        u.x = pack_bf16(x[8 * e + 0], x[8 * e + 1]);
-        u.y = pack_bf16(x[8 * e + 2], x[8 * e + 3]);
-        u.z = pack_bf16(x[8 * e + 4], x[8 * e + 5]);
-        u.w = pack_bf16(x[8 * e + 6], x[8 * e + 7]);
-        *reinterpret_cast<uint4*>(sOut + swz(r, 4 * cc + e)) = u;
-      }
+      for (int h2 = 0; h2 < 2; ++h2)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          uint4 u;
+          u.x = pack_bf16(x[h2][8 * e + 0], x[h2][8 * e + 1]);
+          u.y = pack_bf16(x[h2][8 * e + 2], x[h2][8 * e + 3]);
+          u.z = pack_bf16(x[h2][8 * e + 4], x[h2][8 * e + 5]);
+          u.w = pack_bf16(x[h2][8 * e + 6], x[h2][8 * e + 7]);
+          *reinterpret_cast<uint4*>(sOut + swz(r, 4 * (cc + h2) + e)) = u;
+        }
     }
     tc_fence_before();
     mbar_arrive(&bars->acc_free);                              // the accumulators have been read
