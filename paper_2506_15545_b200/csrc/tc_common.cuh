@@ -261,6 +261,11 @@ __device__ __forceinline__ float max32(const float (&x)[32]) {
   }
   return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
 }
+// columns whose keep bit is clear become -inf: no part in the maximum, weight exactly zero
+__device__ __forceinline__ void mask32(float (&x)[32], uint32_t keep) {
+#pragma unroll
+  for (int e = 0; e < 32; ++e) x[e] = (keep >> e) & 1u ? x[e] : -INFINITY;
+}
 __device__ __forceinline__ float max32_masked(const float (&x)[32], uint32_t keep) {
   float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll

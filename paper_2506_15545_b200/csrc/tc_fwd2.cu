@@ -45,7 +45,7 @@ constexpr int SCHED_SLOTS = 4;
 constexpr int SCHED_READERS = 256 + 1 + 64;      // row threads, the MMA warp's lane 0, the converter threads
 
 struct FBars {
-  uint64_t q_full[2], q_free[2], kv_full[2], v_ready[2], kv_free[2], x_full, x_free;
+  uint64_t q_full[2], q_free[2], k_full[2], v_full[2], v_ready[2], k_free[2], v_free[2], x_full, x_free;
   uint64_t s_full[2], p_ready[2], o_ready[2], stash_done[2], phiq_ready[2], phik_ready[2], o_free[2], y_done[2], drain;
   uint64_t sched_full[SCHED_SLOTS], sched_free[SCHED_SLOTS];
   int sched_unit[SCHED_SLOTS];
@@ -137,6 +137,13 @@ __device__ int g_timeline_n[4];
 #define TL(role, id) do { } while (0)
 #endif
 
+// the MMA warp's own events cost it issue slots: they are a second switch (-DRATTN_TIMELINE_MMA)
+#ifdef RATTN_TIMELINE_MMA
+#define TLM(role, id) TL(role, id)
+#else
+#define TLM(role, id) do { } while (0)
+#endif
+
 #define WAIT_OR_RETURN(bar, parity) \
   do { if (!mbar_wait(&(bar), (parity), &bars->abort)) return false; } while (0)
 #define WAIT_OR_RETURN_W(bar, parity) \
@@ -203,11 +210,16 @@ __device__ bool fwd_loader(const FMaps& tm, const FArgs& a, unsigned char* smem,
     }
     for (int i = 0; i < un.n; ++i, ++kv_count) {
       const int st = kv_count & 1, use = kv_count >> 1;
-      if (use >= 1) WAIT_OR_RETURN_W(bars->kv_free[st], (use - 1) & 1);
+      // K and V of a stage are released separately: a K tile has served its last scores one
+      // stream position before its V tile has served its last product, and the next K load
+      // needs that head start to arrive in time
       unsigned char* dst = smem + F_OFF_KV + st * 2 * TILE_BYTES;
-      mbar_arrive_expect_tx(&bars->kv_full[st], 2 * TILE_BYTES);
-      load_tile(dst, &tm.k, &bars->kv_full[st], (un.kt_hi - i) * TILE, un.bh_kv);
-      load_tile(dst + TILE_BYTES, &tm.v, &bars->kv_full[st], (un.kt_hi - i) * TILE, un.bh_kv);
+      if (use >= 1) WAIT_OR_RETURN_W(bars->k_free[st], (use - 1) & 1);
+      mbar_arrive_expect_tx(&bars->k_full[st], TILE_BYTES);
+      load_tile(dst, &tm.k, &bars->k_full[st], (un.kt_hi - i) * TILE, un.bh_kv);
+      if (use >= 1) WAIT_OR_RETURN_W(bars->v_free[st], (use - 1) & 1);
+      mbar_arrive_expect_tx(&bars->v_full[st], TILE_BYTES);
+      load_tile(dst + TILE_BYTES, &tm.v, &bars->v_full[st], (un.kt_hi - i) * TILE, un.bh_kv);
     }
     if (un.has_state) {
       if (cntX >= 1) WAIT_OR_RETURN_W(bars->x_free, (cntX - 1) & 1);
@@ -241,7 +253,7 @@ __device__ bool fwd_convert(const FArgs& a, unsigned char* smem, FBars* bars, in
     if (un.t[0] < 0) continue;
     for (int i = 0; i < un.n; ++i, ++kv_count) {
       const int st = kv_count & 1, use = kv_count >> 1;
-      WAIT_OR_RETURN(bars->kv_full[st], use & 1);
+      WAIT_OR_RETURN(bars->v_full[st], use & 1);
       unsigned char* tile = smem + F_OFF_KV + st * 2 * TILE_BYTES + TILE_BYTES;
 #pragma unroll 4
       for (int c = cid; c < TILE_BYTES / 16; c += 64) {
@@ -265,6 +277,7 @@ __device__ bool fwd_mma(const FArgs& a, unsigned char* smem, FBars* bars, uint32
   const uint32_t sKV = smem_u32(smem + F_OFF_KV), sX = smem_u32(smem + F_OFF_X);
   const uint32_t tS[2] = {tmem, tmem + 128}, tO[2] = {tmem + 256, tmem + 384};
   int kv_count = 0, cntU[2] = {0, 0}, cntX = 0, cntP[2] = {0, 0}, cntR[2] = {0, 0}, cntK[2] = {0, 0};
+  TL_DECL(blockIdx.x == 7 && (threadIdx.x & 31) == 0);
 
   for (int n = 0;; ++n) {
     int u;
@@ -286,7 +299,9 @@ __device__ bool fwd_mma(const FArgs& a, unsigned char* smem, FBars* bars, uint32
       ++cntU[X];
     }
     // first scores of each tile
-    WAIT_OR_RETURN_W(bars->kv_full[stage_of(0)], use_of(0) & 1);
+    // stream positions whose stage the residual branch still reads (chunks cA, cB)
+    auto kept = [&](int i) { return (un.rla[0] && i == un.n - 1) || (un.rla[1] && i == un.i1[1]); };
+    WAIT_OR_RETURN_W(bars->k_full[stage_of(0)], use_of(0) & 1);
     tc_fence_after();
 #pragma unroll
     for (int X = 1; X >= 0; --X) {
@@ -295,27 +310,35 @@ __device__ bool fwd_mma(const FArgs& a, unsigned char* smem, FBars* bars, uint32
         mma_commit(&bars->s_full[X]);
       }
     }
+    if (!kept(0)) mma_commit(&bars->k_free[stage_of(0)]);
     for (int i = 0; i < un.n; ++i) {
+      // The operands of this position are awaited once and ahead of the weights, so that the
+      // products and the next scores go out the moment a row group hands its weights over
+      // (a wait costs this warp a few hundred cycles even when it is already satisfied).
+      WAIT_OR_RETURN_W(bars->v_ready[stage_of(i)], use_of(i) & 1);
+      if (i + 1 < un.n) WAIT_OR_RETURN_W(bars->k_full[stage_of(i + 1)], use_of(i + 1) & 1);
 #pragma unroll
       for (int X = 0; X < 2; ++X) {
         if (active(un, X, i)) {
+          TLM(2, 10 * i + X);
           WAIT_OR_RETURN_W(bars->p_ready[X], cntP[X] & 1);
           ++cntP[X];
-          WAIT_OR_RETURN_W(bars->v_ready[stage_of(i)], use_of(i) & 1);
+          TLM(2, 200 + 10 * i + X);
           tc_fence_after();
           mma_pv(tO[X], tS[X], sV(i), i > un.i0[X]);                             // O_X += P V
           if (i == un.i1[X]) mma_commit(&bars->o_ready[X]);
+          TLM(2, 300 + 10 * i + X);
         }
         if (i + 1 < un.n && active(un, X, i + 1)) {
-          WAIT_OR_RETURN_W(bars->kv_full[stage_of(i + 1)], use_of(i + 1) & 1);
           tc_fence_after();
           mma_kk(tS[X], sQ[X], sK(i + 1), false);                                // S_X = Q_X K^T (after P V in pipe order)
           mma_commit(&bars->s_full[X]);
+          TLM(2, 500 + 10 * i + X);
         }
       }
-      // the stage is released here unless the residual branch still reads it
-      const bool keep = (un.rla[0] && i == un.n - 1) || (un.rla[1] && i == un.i1[1]);
-      if (!keep) mma_commit(&bars->kv_free[stage_of(i)]);
+      // K of the next position has served all its scores, V of this one all its products
+      if (i + 1 < un.n && !kept(i + 1)) mma_commit(&bars->k_free[stage_of(i + 1)]);
+      if (!kept(i)) mma_commit(&bars->v_free[stage_of(i)]);
     }
     // ---- residual branch ---------------------------------------------------------------
     const int iA = un.n - 1, iB = un.i1[1];          // stream positions of chunks cA, cB
@@ -382,10 +405,17 @@ __device__ bool fwd_mma(const FArgs& a, unsigned char* smem, FBars* bars, uint32
       if (un.rla[0]) { ++cntR[0]; ++cntK[0]; }
       if (un.rla[1]) { ++cntR[1]; ++cntK[1]; }
       // the chunk stages
-      if (un.rla[0]) mma_commit(&bars->kv_free[stage_of(iA)]);
-      if (un.rla[1] && !(un.rla[0] && iB == iA)) mma_commit(&bars->kv_free[stage_of(iB)]);
+      if (un.rla[0]) {
+        mma_commit(&bars->k_free[stage_of(iA)]);
+        mma_commit(&bars->v_free[stage_of(iA)]);
+      }
+      if (un.rla[1] && !(un.rla[0] && iB == iA)) {
+        mma_commit(&bars->k_free[stage_of(iB)]);
+        mma_commit(&bars->v_free[stage_of(iB)]);
+      }
     }
     kv_count += un.n;
+    TLM(2, 1000 + u);
   }
   return true;
 }
@@ -433,15 +463,23 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
       tc_fence_after();
       const bool diag = (kt == tX), bound = un.windowed && (kt == tX - un.wt);
       const int c_lo = bound ? wq : 0, c_hi = diag ? wq : 3;     // chunks with kept columns
-      // pass 1 over the scores: row maximum
-      float mx = -INFINITY;
-#pragma unroll 1
-      for (int c = c_lo; c <= c_hi; ++c) {
-        float x[32];
-        tmem_ld32(tS + 32 * c, x);
-        tmem_wait_ld();
-        mx = fmaxf(mx, ((diag || bound) && c == wq) ? max32_masked(x, keep_bits(r, c, diag, bound)) : max32(x));
+      // The whole score row is read once (128 registers; the row groups run with a raised
+      // register allowance, see the kernel body) and kept for both the maximum and the weights.
+      float x[4][32];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32(tS + 32 * c, x[c]);      // dropped chunks too: four loads in flight
+      tmem_wait_ld();
+      if (diag || bound) {
+        // the one chunk this warp keeps partly: dropped columns become -inf (weight zero)
+        const uint32_t keep = keep_bits(r, wq, diag, bound);
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (c == wq) mask32(x[c], keep);
       }
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        if (c >= c_lo && c <= c_hi) mx = fmaxf(mx, max32(x[c]));
       mx *= a.scale_log2;                                              // scale > 0
       // lazy rescale: the reference maximum only moves when the row maximum grew by more than 2^8
       const float m_new = fmaxf(m_ref, mx);
@@ -464,42 +502,28 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
         m_ref = m_new;
       }
       TL(X, 300 + i);
-      // pass 2: weights, written back (fp16, two per column) over score columns already consumed
-      float psum = 0.f;
-#pragma unroll 1
+      // weights, written back (fp16, two per column) over the score columns
+      const float2 sc2 = make_float2(a.scale_log2, a.scale_log2), nm2 = make_float2(-m_ref, -m_ref);
+      float2 ps0 = make_float2(0.f, 0.f), ps1 = make_float2(0.f, 0.f);
+#pragma unroll
       for (int c = 0; c < 4; ++c) {
         uint32_t pk[16];
         if (c < c_lo || c > c_hi) {
 #pragma unroll
           for (int e = 0; e < 16; ++e) pk[e] = 0u;
         } else {
-          float x[32];
-          tmem_ld32(tS + 32 * c, x);
-          tmem_wait_ld();
-          float ps[4] = {0.f, 0.f, 0.f, 0.f};
-          if ((diag || bound) && c == wq) {
-            const uint32_t keep = keep_bits(r, c, diag, bound);
 #pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              const float p0 = (keep >> (2 * e)) & 1u ? ex2(x[2 * e] * a.scale_log2 - m_ref) : 0.f;
-              const float p1 = (keep >> (2 * e + 1)) & 1u ? ex2(x[2 * e + 1] * a.scale_log2 - m_ref) : 0.f;
-              ps[2 * (e & 1)] += p0;
-              ps[2 * (e & 1) + 1] += p1;
-              pk[e] = pack_f16(p0, p1);
-            }
-          } else {
-#pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              const float p0 = ex2(x[2 * e] * a.scale_log2 - m_ref), p1 = ex2(x[2 * e + 1] * a.scale_log2 - m_ref);
-              ps[2 * (e & 1)] += p0;
-              ps[2 * (e & 1) + 1] += p1;
-              pk[e] = pack_f16(p0, p1);
-            }
+          for (int e = 0; e < 16; ++e) {
+            const float2 y = __ffma2_rn(make_float2(x[c][2 * e], x[c][2 * e + 1]), sc2, nm2);
+            const float2 pp = make_float2(ex2(y.x), ex2(y.y));
+            if (e & 1) ps1 = __fadd2_rn(ps1, pp);
+            else ps0 = __fadd2_rn(ps0, pp);
+            pk[e] = pack_f16(pp.x, pp.y);
           }
-          psum += (ps[0] + ps[1]) + (ps[2] + ps[3]);
         }
         tmem_st16(tS + 16 * c, pk);
       }
+      const float psum = (ps0.x + ps0.y) + (ps1.x + ps1.y);
       l += psum;
       tmem_wait_st();
       tc_fence_before();
@@ -606,7 +630,6 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     }
 
     // ---- Section 3.2: gains, sum; outputs leave through the tile's Q buffer ---------------
-    const size_t tile_row0 = (size_t)un.bh_q * a.T + q0;
     TL(X, 530);
     const float rms_s = ms * rs;                                       // sqrt(mean square + eps)
     if (a.o_swa) {
@@ -754,9 +777,11 @@ tc_fwd2_kernel(const __grid_constant__ FMaps tm, FArgs a) {
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bars->q_full[i], 1);
       mbar_init(&bars->q_free[i], 128);
-      mbar_init(&bars->kv_full[i], 1);
+      mbar_init(&bars->k_full[i], 1);
+      mbar_init(&bars->v_full[i], 1);
       mbar_init(&bars->v_ready[i], 64);
-      mbar_init(&bars->kv_free[i], 1);
+      mbar_init(&bars->k_free[i], 1);
+      mbar_init(&bars->v_free[i], 1);
       mbar_init(&bars->s_full[i], 1);
       mbar_init(&bars->p_ready[i], 128);
       mbar_init(&bars->o_ready[i], 1);
@@ -794,7 +819,11 @@ tc_fwd2_kernel(const __grid_constant__ FMaps tm, FArgs a) {
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
 
+  // Registers follow the work: the row groups keep a whole score row (128 values) live, the
+  // other four warps need few.  2 x 128 x 208 + 128 x 88 = 384 x 168, the CTA's allocation.
   bool ok = true;
+  if (warp < 8) setmaxnreg_inc<208>();
+  else setmaxnreg_dec<88>();
   if (warp < 8) {
     ok = fwd_rows(tm, a, smem, bars, tmem, warp >> 2, tid & 127);
   } else if (warp == 8) {

@@ -186,6 +186,14 @@ __device__ __forceinline__ void mma_commit(uint64_t* bar) {
       ::"r"(smem_u32(bar))
       : "memory");
 }
+// Register re-allocation between the warp groups of a CTA (all four warps of an aligned group
+// execute the same instruction).  The increase blocks until the registers are free, so the sum
+// over the groups must stay within the CTA's allocation.
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
