@@ -825,9 +825,11 @@ __device__ bool kv_loader(const KvMaps& tm, const BwdArgs& a, unsigned char* sme
 __device__ bool kv_mma_scores(const BwdArgs& a, unsigned char* smem, KvBars* bars, uint32_t tmem, int n_items) {
   const uint32_t sK = smem_u32(smem + KV_OFF_K), sV = smem_u32(smem + KV_OFF_V), sKphi = smem_u32(smem + KV_OFF_KPHI);
   const uint32_t sStage = smem_u32(smem + KV_OFF_STAGE);
-  const uint32_t tS[2] = {tmem + 256, tmem + 384}, tP[2] = {tmem + 320, tmem + 448};
+  // slot s: [S^T | dP^T] at columns 256 + 128 s and 320 + 128 s (computed, not looked up: an array
+  // indexed by the slot would live in local memory)
+  const uint32_t tS0 = tmem + 256, tP0 = tmem + 320;
   KvCount c = {0, 0, 0, 0};
-  int cq[2] = {0, 0};                                      // phi(Q_h) hand-overs per TMEM slot
+  int cq0 = 0, cq1 = 0;                                    // phi(Q_h) hand-overs per TMEM slot
 
   for (int idx = blockIdx.x; idx < n_items; idx += gridDim.x, ++c.it) {
     const KvPlan pl = kv_plan(a, idx);
@@ -841,16 +843,16 @@ __device__ bool kv_mma_scores(const BwdArgs& a, unsigned char* smem, KvBars* bar
       const uint32_t sQh = sStage + st * TILE_BYTES, sGh = sQh + HT_BYTES;
       WAIT_OR_RETURN_W(bars->full[st], use & 1);
       if (pl.is_r(n)) {
-        WAIT_OR_RETURN_W(bars->phiq_ready[slot], cq[slot] & 1);
-        ++cq[slot];
+        WAIT_OR_RETURN_W(bars->phiq_ready[slot], (slot ? cq1 : cq0) & 1);
+        if (slot) ++cq1; else ++cq0;
       }
       if (n >= 2) {                                        // the slot's previous item has been accumulated
         const int st2 = (seq0 + n - 2) % KV_NS, use2 = (seq0 + n - 2) / KV_NS;
         WAIT_OR_RETURN_W(bars->acc_done[st2], use2 & 1);
       }
       tc_fence_after();
-      mma_k_kh(tS[slot], pl.is_r(n) ? sKphi : sK, sQh);     // S^T  = K Q_h^T   (phi(K) phi(Q_h)^T)
-      mma_k_kh(tP[slot], sV, sGh);                           // dP^T = V g_h^T
+      mma_k_kh(tS0 + 128 * slot, pl.is_r(n) ? sKphi : sK, sQh);   // S^T  = K Q_h^T   (phi(K) phi(Q_h)^T)
+      mma_k_kh(tP0 + 128 * slot, sV, sGh);                         // dP^T = V g_h^T
       mma_commit(&bars->s_full[slot]);
     }
     c.seq += pl.N;
@@ -864,7 +866,7 @@ __device__ bool kv_mma_accum(const BwdArgs& a, unsigned char* smem, KvBars* bars
   const uint32_t sV = smem_u32(smem + KV_OFF_V), sKphi = smem_u32(smem + KV_OFF_KPHI);
   const uint32_t sStage = smem_u32(smem + KV_OFF_STAGE);
   const uint32_t tV = tmem, tK = tmem + 128;
-  const uint32_t tS[2] = {tmem + 256, tmem + 384}, tP[2] = {tmem + 320, tmem + 448};
+  const uint32_t tS0 = tmem + 256, tP0 = tmem + 320;
   KvCount c = {0, 0, 0, 0};
 
   for (int idx = blockIdx.x; idx < n_items; idx += gridDim.x, ++c.it) {
@@ -893,8 +895,8 @@ __device__ bool kv_mma_accum(const BwdArgs& a, unsigned char* smem, KvBars* bars
       if (m == pl.n_R && pl.n_R > 0) WAIT_OR_RETURN_W(bars->fold_done, c.cr & 1);
       if (!acc_ok) { WAIT_OR_RETURN_W(bars->acc_free, (c.it - 1) & 1); acc_ok = true; }
       tc_fence_after();
-      mma_ts_h(tV, tS[slot], sGh, accV);                   // dV += P^T g_h
-      mma_ts_h(tK, tP[slot], sQh, accK);                   // dK += dS^T Q_h   (dphi_k += dA^T phi(Q_h))
+      mma_ts_h(tV, tS0 + 128 * slot, sGh, accV);           // dV += P^T g_h
+      mma_ts_h(tK, tP0 + 128 * slot, sQh, accK);           // dK += dS^T Q_h   (dphi_k += dA^T phi(Q_h))
       accV = accK = true;
       mma_commit(&bars->acc_done[st]);
       if (m == pl.n_R - 1) mma_commit(&bars->r_acc_done);

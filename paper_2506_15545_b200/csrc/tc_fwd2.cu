@@ -820,10 +820,10 @@ tc_fwd2_kernel(const __grid_constant__ FMaps tm, FArgs a) {
   const uint32_t tmem = bars->tmem_base;
 
   // Registers follow the work: the row groups keep a whole score row (128 values) live, the
-  // other four warps need few.  2 x 128 x 208 + 128 x 88 = 384 x 168, the CTA's allocation.
+  // other four warps need few.  2 x 128 x 192 + 128 x 120 = 384 x 168, the CTA's allocation; with this split neither side spills.
   bool ok = true;
-  if (warp < 8) setmaxnreg_inc<208>();
-  else setmaxnreg_dec<88>();
+  if (warp < 8) setmaxnreg_inc<192>();
+  else setmaxnreg_dec<120>();
   if (warp < 8) {
     ok = fwd_rows(tm, a, smem, bars, tmem, warp >> 2, tid & 127);
   } else if (warp == 8) {
