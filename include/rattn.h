@@ -338,12 +338,8 @@ typedef enum rattn_knob {
                                     throughout; 3 the same, dealt round-robin instead of drawn from a counter.
                                     Automatic = 1 when the state kernel leaves at least half of the SMs free. */
   RATTN_TUNE_GRID = 3,           /* CTAs of the persistent forward kernel: 0 (default) = one per SM */
-  RATTN_TUNE_DECODE_STAGES = 4,  /* 16 KB stages of the staged decode step: 0 (default) = as many as let two
+  RATTN_TUNE_DECODE_STAGES = 4   /* 16 KB stages of the staged decode step: 0 (default) = as many as let two
                                     CTAs share an SM; 3..8 (ignored where that many do not fit) */
-  RATTN_TUNE_HEAD_PAIRS = 5      /* grouped heads (H_q / H_kv even): a work unit of the forward is one query tile of
-                                    two heads of a group (they share every K/V tile, phi(K) of the chunk and one
-                                    stored state) instead of two adjacent query tiles of one head: 0 (default)
-                                    and 1 = on where the group allows it, 2 = off */
 } rattn_knob;
 int rattn_tune(int knob, int value);
 

@@ -27,7 +27,7 @@ int debug_skip_arrive() {
 #endif
 }
 
-static std::atomic<int> g_tuning[6] = {{0}, {1}, {0}, {0}, {0}, {0}};
+static std::atomic<int> g_tuning[5] = {{0}, {1}, {0}, {0}, {0}};
 int tuning(int knob) { return g_tuning[knob].load(std::memory_order_relaxed); }
 
 void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
@@ -478,8 +478,8 @@ int rattn_debug_withhold_arrival(int on) {
 #endif
 
 int rattn_tune(int knob, int value) {
-  static const int lo[6] = {0, 0, 0, 0, 0, 0}, hi[6] = {2, 1, 3, 1 << 16, 8, 2};
-  if (knob < 0 || knob > 5 || value < lo[knob] || value > hi[knob]) return RATTN_ERR_BAD_ARG;
+  static const int lo[5] = {0, 0, 0, 0, 0}, hi[5] = {2, 1, 3, 1 << 16, 8};
+  if (knob < 0 || knob > 4 || value < lo[knob] || value > hi[knob]) return RATTN_ERR_BAD_ARG;
   return g_tuning[knob].exchange(value, std::memory_order_relaxed);
 }
 

@@ -134,7 +134,6 @@ struct StateLaunch {
   const char* name;         // label of the timing record
 };
 cudaError_t launch_tc_states(const StateLaunch& L, cudaStream_t s);
-bool head_pair_units(const Args& a);        // the forward's work units are pairs of heads, not pairs of tiles
 cudaError_t launch_tc_backward(const Args& a, cudaStream_t s);
 // chunked prefill: k_ext/v_ext[b,hk] = the ring's tokens pos0-w .. pos0-1 in time order, then the chunk
 cudaError_t launch_gather_history(const Args& a, const void* k_chunk, const void* v_chunk, const void* k_ring,

@@ -67,9 +67,6 @@ struct FArgs {
   int first_state;        // smallest chunk index whose state is stored: 1 (S_[0] = 0), or 0 with an incoming state
   const int* seq_lens;    // optional [B]: valid query rows per batch entry
   int n_stateless;        // pairs whose tiles read no stored state; their units come first
-  int head_pairs;         // 1: a unit is one query tile of two heads that share a K/V head (grouped heads),
-                          // 0: two adjacent query tiles of one head
-  int n_pos;              // positions a unit index runs over: query tiles (head pairs) or pairs of query tiles
   int wait_for_states;    // a chunk-state kernel runs ahead of this one: wait for it before the first state load
   int debug_skip_arrive;  // debug build only: tile A's row group withholds its first hand-over (a wait then runs out)
   float scale_log2, eps;
@@ -83,9 +80,7 @@ struct FMaps {
 
 // What one unit consists of; every role derives the same plan from the unit index.
 struct Unit {
-  int bh_q, bh_kv, h;       // tile A's query head (batch-major index, head within the entry), the K/V head
-  int bh_q1, h1;            // tile B's query head: the same one, or its neighbour in the group (head-pair units)
-  bool same_pos;            // head-pair unit: both tiles sit at the same position and share band, chunk and state
+  int bh_q, bh_kv, h;
   int t[2];                 // tile index of A, B (B: -1 when the sequence ends after A)
   int kt_hi, n;             // key tiles kt_hi, kt_hi-1, ..., kt_hi-n+1
   int i0[2], i1[2];         // stream positions each tile is active on (inclusive)
@@ -101,25 +96,17 @@ __device__ __forceinline__ Unit make_unit(const FArgs& a, int u) {
   // Order: first the pairs that read no stored state (they can run while the chunk-state kernel
   // is still at work), then the others, heaviest first.
   const int pr = u / a.n_bh;
-  const int p = pr < a.n_stateless ? pr : a.n_pos - 1 - (pr - a.n_stateless);
-  un.same_pos = a.head_pairs != 0;
-  // head-pair units: n_bh counts pairs of adjacent heads (2j, 2j+1), which an even group keeps under one K/V head
-  un.bh_q = un.same_pos ? 2 * (u % a.n_bh) : u % a.n_bh;
-  un.bh_q1 = un.same_pos ? un.bh_q + 1 : un.bh_q;
+  un.bh_q = u % a.n_bh;
+  const int p = pr < a.n_stateless ? pr : a.n_pairs - 1 - (pr - a.n_stateless);
   const int b = un.bh_q / a.H_q;
   un.h = un.bh_q % a.H_q;
-  un.h1 = un.bh_q1 % a.H_q;
   un.bh_kv = b * (a.H_q / a.group) + un.h / a.group;
   un.wt = a.w / TILE;
   un.windowed = (a.mode != RATTN_MODE_FULL_CAUSAL);
   // tile indices are key-space positions: query tile i of the call sits at key tile i + off
   const int n_qt = a.seq_lens ? (min(a.T, a.seq_lens[b]) + TILE - 1) / TILE : a.n_qt;
-  if (un.same_pos) {
-    un.t[0] = un.t[1] = (p < n_qt) ? a.off + p : -1;
-  } else {
-    un.t[0] = (2 * p < n_qt) ? a.off + 2 * p : -1;           // a unit without tile A is empty
-    un.t[1] = (2 * p + 1 < n_qt) ? a.off + 2 * p + 1 : -1;
-  }
+  un.t[0] = (2 * p < n_qt) ? a.off + 2 * p : -1;             // a unit without tile A is empty
+  un.t[1] = (2 * p + 1 < n_qt) ? a.off + 2 * p + 1 : -1;
   un.kt_hi = un.t[1] >= 0 ? un.t[1] : un.t[0];
   const int loA = un.windowed ? max(0, un.t[0] - un.wt) : 0;
   un.n = un.kt_hi - loA + 1;
@@ -218,7 +205,7 @@ __device__ bool fwd_loader(const FMaps& tm, const FArgs& a, unsigned char* smem,
       if (un.t[X] < 0) continue;
       if (cntU[X] >= 1) WAIT_OR_RETURN_W(bars->q_free[X], (cntU[X] - 1) & 1);
       mbar_arrive_expect_tx(&bars->q_full[X], TILE_BYTES);
-      load_tile(smem + F_OFF_Q + X * TILE_BYTES, &tm.q, &bars->q_full[X], (un.t[X] - a.off) * TILE, X ? un.bh_q1 : un.bh_q);
+      load_tile(smem + F_OFF_Q + X * TILE_BYTES, &tm.q, &bars->q_full[X], (un.t[X] - a.off) * TILE, un.bh_q);
       ++cntU[X];
     }
     for (int i = 0; i < un.n; ++i, ++kv_count) {
@@ -404,24 +391,19 @@ __device__ bool fwd_mma(const FArgs& a, unsigned char* smem, FBars* bars, uint32
           tc_fence_after();
           mma_pv(tO[1], tS[1], sV(iA), un.has_state);
         }
-        if (un.same_pos) {
-          // head-pair unit: tile B's chunk is tile A's, the one (masked) term above was all of it
-          mma_commit(&bars->o_ready[1]);
-        } else {
-          WAIT_OR_RETURN_W(bars->phik_ready[1], cntK[1] & 1);
-          tc_fence_after();
-          mma_kk(tS[1], sQ[1], sK(iB), false);                                   // phi(Q_B) phi(K_cB)^T
-          mma_commit(&bars->s_full[1]);
-          WAIT_OR_RETURN_W(bars->p_ready[1], cntP[1] & 1);
-          ++cntP[1];
-          tc_fence_after();
-          mma_pv(tO[1], tS[1], sV(iB), un.rla[0]);
-          mma_commit(&bars->o_ready[1]);
-        }
+        WAIT_OR_RETURN_W(bars->phik_ready[1], cntK[1] & 1);
+        tc_fence_after();
+        mma_kk(tS[1], sQ[1], sK(iB), false);                                     // phi(Q_B) phi(K_cB)^T
+        mma_commit(&bars->s_full[1]);
+        WAIT_OR_RETURN_W(bars->p_ready[1], cntP[1] & 1);
+        ++cntP[1];
+        tc_fence_after();
+        mma_pv(tO[1], tS[1], sV(iB), un.rla[0]);
+        mma_commit(&bars->o_ready[1]);
       }
       if (un.has_state) mma_commit(&bars->x_free);
       if (un.rla[0]) { ++cntR[0]; ++cntK[0]; }
-      if (un.rla[1]) { ++cntR[1]; if (!un.same_pos) ++cntK[1]; }
+      if (un.rla[1]) { ++cntR[1]; ++cntK[1]; }
       // the chunk stages
       if (un.rla[0]) {
         mma_commit(&bars->k_free[stage_of(iA)]);
@@ -461,7 +443,6 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     kv_count += un.n;
     const int tX = X ? un.t[1] : un.t[0], i0 = X ? un.i0[1] : un.i0[0], i1 = X ? un.i1[1] : un.i1[0];
     const bool rlaX = X ? un.rla[1] : un.rla[0];
-    const int bhX = X ? un.bh_q1 : un.bh_q, hX = X ? un.h1 : un.h;      // this tile's query head
     if (tX < 0) continue;
     const int q0 = (tX - a.off) * TILE;          // first query row of the tile (tX is its key-space index)
     const int t = q0 + r;
@@ -569,13 +550,10 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
       mbar_arrive(&bars->phiq_ready[X]);
       TL(X, 503);
       // this tile's own chunk: A -> last stream position, B -> its last active position
-      // (in a head-pair unit both tiles have the same chunk: tile A's group maps it)
-      if (!(un.same_pos && X == 1)) {
-        const int ic = (X == 0) ? un.n - 1 : un.i1[1];
-        feature_map_row_any<true>(smem + F_OFF_KV + ((kv0 + ic) & 1) * 2 * TILE_BYTES, r, a.phi, a.o_swa != nullptr);
-        fence_proxy_async_smem();
-        mbar_arrive(&bars->phik_ready[X]);
-      }
+      const int ic = (X == 0) ? un.n - 1 : un.i1[1];
+      feature_map_row_any<true>(smem + F_OFF_KV + ((kv0 + ic) & 1) * 2 * TILE_BYTES, r, a.phi, a.o_swa != nullptr);
+      fence_proxy_async_smem();
+      mbar_arrive(&bars->phik_ready[X]);
       TL(X, 504);
     }
 
@@ -612,7 +590,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
     if (rlaX) {
       tc_fence_before();
       mbar_arrive(&bars->stash_done[X]);
-      const int n_terms = (X == 1 && un.rla[0] && !un.same_pos) ? 2 : 1;
+      const int n_terms = (X == 1 && un.rla[0]) ? 2 : 1;
 #pragma unroll 1
       for (int term = 0; term < n_terms; ++term) {
         const bool masked = (term == n_terms - 1);                     // B's first term takes chunk cA whole
@@ -677,7 +655,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
       fence_proxy_async_smem();
       group_sync(X);
       if (r == 0) {
-        store_tile(&tm.o_swa, stage, q0, bhX);
+        store_tile(&tm.o_swa, stage, q0, un.bh_q);
         tma_store_commit();
         tma_store_wait_read();
       }
@@ -703,15 +681,15 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
       fence_proxy_async_smem();
       group_sync(X);
       if (r == 0) {
-        store_tile(&tm.o_rla, stage, q0, bhX);
+        store_tile(&tm.o_rla, stage, q0, un.bh_q);
         tma_store_commit();
         tma_store_wait_read();
       }
       group_sync(X);
     }
     TL(X, 535);
-    const float* gs = a.gamma_swa ? a.gamma_swa + (size_t)hX * 128 : nullptr;
-    const float* gr = a.gamma_rla ? a.gamma_rla + (size_t)hX * 128 : nullptr;
+    const float* gs = a.gamma_swa ? a.gamma_swa + (size_t)un.h * 128 : nullptr;
+    const float* gr = a.gamma_rla ? a.gamma_rla + (size_t)un.h * 128 : nullptr;
     // y leaves through the state tile's buffer (free once this unit's residual products are done;
     // 16 KB per row group), one 64-column half at a time, so that the tile's Q buffer and the
     // K/V stages can take the next unit's loads while the epilogue runs.  The branches on "gains
@@ -760,7 +738,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
         fence_proxy_async_smem();
         group_sync(X);
         if (r == 0) {
-          store_half(&tm.out, sY, 64 * hf, q0, bhX);
+          store_half(&tm.out, sY, 64 * hf, q0, un.bh_q);
           tma_store_commit();
         }
         // The Q buffer (phi(Q_X) has long been consumed) is released only once the last store is
@@ -779,7 +757,7 @@ __device__ bool fwd_rows(const FMaps& tm, const FArgs& a, unsigned char* smem, F
       if (rlaX) emit_y(std::false_type{}, std::true_type{});
       else emit_y(std::false_type{}, std::false_type{});
     }
-    if (t < a.T && a.lse) a.lse[(size_t)bhX * a.T + t] = (m_ref + log2f(l)) * 0.6931471805599453f;
+    if (t < a.T && a.lse) a.lse[(size_t)un.bh_q * a.T + t] = (m_ref + log2f(l)) * 0.6931471805599453f;
     mbar_arrive(&bars->y_done[X]);         // the staging buffer may take the next state tile
     TL(X, 540);
   }
@@ -880,13 +858,6 @@ extern "C" int rattn_timeline_read(unsigned long long* out, int* n) {
 }
 #endif
 
-// Grouped heads: two query heads of a group work on the same query tile position, so that they share
-// the whole band of K/V tiles, the chunk's phi(K) and one stored state (every chunk state is then read).
-bool head_pair_units(const Args& a) {
-  const int knob = tuning(RATTN_TUNE_HEAD_PAIRS);
-  return knob != 2 && a.group >= 2 && a.group % 2 == 0;
-}
-
 cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_states) {
   FMaps tm;
   if (!make_user_map(&tm.q, a.q, a.T, a.H_q, a.B, a.layout) || !make_user_map(&tm.k, a.k, a.Tk, a.H_kv, a.B, a.kv_layout) ||
@@ -908,10 +879,8 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_sta
   t.T = a.T; t.w = a.w; t.H_q = a.H_q; t.group = a.group; t.mode = a.mode; t.n_chunks = a.n_chunks;
   t.n_qt = (a.T + TILE - 1) / TILE;
   t.n_pairs = (t.n_qt + 1) / 2;
-  t.head_pairs = head_pair_units(a) ? 1 : 0;
-  t.n_pos = t.head_pairs ? t.n_qt : t.n_pairs;
-  t.n_bh = t.head_pairs ? a.B * a.H_q / 2 : a.B * a.H_q;
-  t.n_units = t.n_pos * t.n_bh;
+  t.n_bh = a.B * a.H_q;
+  t.n_units = t.n_pairs * t.n_bh;
   t.scale_log2 = a.scale * LOG2E; t.eps = a.eps;
   t.phi = a.phi;
   t.off = a.q_off / TILE;
@@ -923,8 +892,8 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_sta
   const int order = tuning(RATTN_TUNE_UNIT_ORDER);
   const bool stateless_first = order == 1 || (order == 0 && 2 * a.B * a.H_kv <= n_sm);
   if (a.mode == RATTN_MODE_RATTN && after_states && !a.state_in && stateless_first) {
-    t.n_stateless = t.head_pairs ? a.w / TILE + 1 : (a.w / TILE) / 2 + 1;
-    if (t.n_stateless > t.n_pos) t.n_stateless = t.n_pos;
+    t.n_stateless = (a.w / TILE) / 2 + 1;
+    if (t.n_stateless > t.n_pairs) t.n_stateless = t.n_pairs;
   }
   t.wait_for_states = after_states ? 1 : 0;
   t.debug_skip_arrive = debug_skip_arrive();

@@ -59,7 +59,7 @@ def test_tensor_core_kernels(phi, T, w, Hq, Hkv):
     assert R.rattn_uses_tensor_path(128, w)
     wl = small("fmt", 2, Hq, Hkv, T, 128, w, "bf16", 7100 + T + phi, unit=True)
     y, ref, grads, want = fwd_bwd(wl, phi, 0)
-    check_bf16_heavy_tails(y, ref, f"phi={phi}")      # signed weights: outputs beyond |y| = 4 occur (see the helper)
+    check(y, ref, "bf16", f"phi={phi}")
     for name, a, b in zip(("dq", "dk", "dv"), grads, want):
         assert np.isfinite(np64(a)).all(), name
         assert rel_fro(np64(a), b) <= GRAD_TOL, (name, rel_fro(np64(a), b))

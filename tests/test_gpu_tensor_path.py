@@ -63,20 +63,6 @@ def test_tensor_forward_large_logits_trigger_rescale():
     check(y, ref, "bf16", "large logits")
 
 
-@pytest.mark.parametrize("knob", [0, 2])
-@pytest.mark.parametrize("T,w,Hq,Hkv", [(1280, 256, 4, 2), (1100, 128, 4, 1), (2048, 512, 6, 1), (900, 256, 3, 1)])
-def test_tensor_forward_grouped_heads_unit_shapes(knob, T, w, Hq, Hkv):
-    """Grouped heads: work units of two heads on one query tile (knob 0, where the group is even) and of two
-    query tiles of one head (knob 2; also what an odd group gets) compute the same operator."""
-    wl = small("tcgqa", 2, Hq, Hkv, T, 128, w, "bf16", 4400 + T + w + Hq, unit=True)
-    prev = R.rattn_tune(R.TUNE_HEAD_PAIRS, knob)
-    try:
-        y, ref, _ = run(wl)
-    finally:
-        R.rattn_tune(R.TUNE_HEAD_PAIRS, prev)
-    check(y, ref, "bf16", f"head-pair knob {knob}, T={T} w={w} heads {Hq}/{Hkv}")
-
-
 def test_tensor_forward_c2_like_heads():
     """Config 2's sequence (T=4096, w=512, unit-RMS q/k, scale 1/sqrt(128)) on two heads."""
     wl = W.C2.replace(B=1, H_q=2, H_kv=2)
