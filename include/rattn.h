@@ -195,7 +195,7 @@ int rattn_forward(const void* q, const void* k, const void* v,
  * framework's allocator, a latency-bound loop that must stay clear of the driver's
  * allocation lock.  Where the tensor-core path applies (d = 128, w % 128 == 0) its chunk
  * states go into a fixed array inside the library instead: RATTN_STATIC_MAX_CHUNK_STATES
- * matrices of 128 x 128 bf16 (2 MiB in all, held by every GPU that loads the library until
+ * matrices of 128 x 128 bf16 (2 MiB in all, plus 512 bytes of status and progress words, held by every GPU that loads the library until
  * the process exits).  The call is refused with RATTN_ERR_STATIC_LIMIT when
  * B * H_kv * ceil(T / 128) exceeds that number; other shapes run the portable kernel,
  * which needs no scratch, so they are never refused for size.
@@ -272,7 +272,8 @@ int rattn_decode_status(void* stream);
 /*
  * Bytes of workspace a call with these sizes, mode (rattn_mode) and flags (RATTN_FLAG_*)
  * needs; dtype is a rattn_dtype.  Returns 0 for invalid arguments.  The first 256 bytes hold
- * the device status word.  What the rest holds depends on the call:
+ * the device status word (on the tensor-core kernels in mode RATTN one progress word per K/V
+ * head follows it, rounded up to 256 bytes).  What the rest holds depends on the call:
  *   inference, portable kernels        nothing more (256 bytes in all);
  *   inference, tensor-core kernels     the chunk states of the linear branch (Eq. 2; the
  *                                      paper's stored states): bf16 [B,H_kv,ceil(T/128),d,d],
@@ -338,8 +339,12 @@ typedef enum rattn_knob {
                                     throughout; 3 the same, dealt round-robin instead of drawn from a counter.
                                     Automatic = 1 when the state kernel leaves at least half of the SMs free. */
   RATTN_TUNE_GRID = 3,           /* CTAs of the persistent forward kernel: 0 (default) = one per SM */
-  RATTN_TUNE_DECODE_STAGES = 4   /* 16 KB stages of the staged decode step: 0 (default) = as many as let two
+  RATTN_TUNE_DECODE_STAGES = 4,  /* 16 KB stages of the staged decode step: 0 (default) = as many as let two
                                     CTAs share an SM; 3..8 (ignored where that many do not fit) */
+  RATTN_TUNE_STATE_PROGRESS = 5  /* the main kernel takes the chunk states as the chunk-state kernel publishes them
+                                    (one progress word per K/V head, work units in sequence order) instead of
+                                    waiting for that whole kernel: 0 (default) automatic = on for long chains on
+                                    few K/V heads (T >= 6144, 4 B H_kv <= SMs); 1 on; 2 off */
 } rattn_knob;
 int rattn_tune(int knob, int value);
 

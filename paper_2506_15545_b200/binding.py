@@ -29,7 +29,7 @@ EXPORTS = (
     "rattn_forward_static", "rattn_static_status", "rattn_tune",
     "rattn_qk_prologue", "rattn_qk_prologue_backward", "rattn_qk_prologue_workspace_bytes", "rattn_qk_prologue_status", "rattn_decode_status", "rattn_forward_status",
 )
-TUNE_STATE_STRIDE, TUNE_OVERLAP, TUNE_UNIT_ORDER, TUNE_GRID, TUNE_DECODE_STAGES = 0, 1, 2, 3, 4
+TUNE_STATE_STRIDE, TUNE_OVERLAP, TUNE_UNIT_ORDER, TUNE_GRID, TUNE_DECODE_STAGES, TUNE_STATE_PROGRESS = 0, 1, 2, 3, 4, 5
 
 
 class RattnParams(ctypes.Structure):

@@ -27,7 +27,7 @@ int debug_skip_arrive() {
 #endif
 }
 
-static std::atomic<int> g_tuning[5] = {{0}, {1}, {0}, {0}, {0}};
+static std::atomic<int> g_tuning[6] = {{0}, {1}, {0}, {0}, {0}, {0}};
 int tuning(int knob) { return g_tuning[knob].load(std::memory_order_relaxed); }
 
 void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
@@ -101,7 +101,8 @@ WorkspaceLayout workspace_layout(int B, int H_q, int H_kv, int T, int d, int w, 
   L.n_chunks = (Tk + 127) / 128;
   const size_t states = (size_t)B * H_kv * L.n_chunks * d * d;
   const size_t rows_pad = (size_t)B * H_q * L.n_chunks * 128;
-  L.status = take(true, 256);
+  L.status_bytes = 256 + ((tc && rla) ? align256(sizeof(int) * (size_t)B * H_kv) : 0);
+  L.status = take(true, L.status_bytes);
   L.lse = take(train, rows * sizeof(float));
   L.o_swa = take(train, rows * d * branch_elem);
   L.o_rla = take(train, rows * d * branch_elem);
@@ -166,6 +167,7 @@ static int bind_workspace(const rattn_params* p, Args* a, bool required, unsigne
   char* base = reinterpret_cast<char*>(p->workspace);
   auto at = [&](size_t off) -> char* { return off == kAbsent ? nullptr : base + off; };
   a->status = reinterpret_cast<int*>(at(L.status));
+  a->state_ready = L.status_bytes > 256 ? a->status + 64 : nullptr;
   a->lse = reinterpret_cast<float*>(at(L.lse));
   a->o_swa = reinterpret_cast<float*>(at(L.o_swa));
   a->o_rla = reinterpret_cast<float*>(at(L.o_rla));
@@ -215,7 +217,7 @@ static int forward_impl(const rattn_params* p, cudaStream_t s) {
   a.training = train;
   cudaError_t e;
   if (a.status) {
-    e = cudaMemsetAsync(a.status, 0, 256, s);
+    e = cudaMemsetAsync(a.status, 0, L.status_bytes, s);
     if (e != cudaSuccess) return fail_cuda(e);
   }
   if (resume) {
@@ -478,8 +480,8 @@ int rattn_debug_withhold_arrival(int on) {
 #endif
 
 int rattn_tune(int knob, int value) {
-  static const int lo[5] = {0, 0, 0, 0, 0}, hi[5] = {2, 1, 3, 1 << 16, 8};
-  if (knob < 0 || knob > 4 || value < lo[knob] || value > hi[knob]) return RATTN_ERR_BAD_ARG;
+  static const int lo[6] = {0, 0, 0, 0, 0, 0}, hi[6] = {2, 1, 3, 1 << 16, 8, 2};
+  if (knob < 0 || knob > 5 || value < lo[knob] || value > hi[knob]) return RATTN_ERR_BAD_ARG;
   return g_tuning[knob].exchange(value, std::memory_order_relaxed);
 }
 

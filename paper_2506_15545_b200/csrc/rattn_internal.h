@@ -14,7 +14,9 @@ namespace rattn {
 // Byte offsets inside the caller's workspace.  Every region is 256-byte aligned; a region the
 // call's mode and flags do not need has offset kAbsent and takes no room.
 struct WorkspaceLayout {
-  size_t status;        // 256 bytes; word 0 = device status, word 1 = detail code
+  size_t status;        // 256 bytes; word 0 = device status, word 1 = detail code; behind it, on the tensor-core
+                        // path with a linear branch, one progress word per K/V head (status_bytes in all)
+  size_t status_bytes;  // what a forward clears before its kernels
   size_t lse;           // fp32 [B,H_q,T]      log-sum-exp of the SWA logits (natural log)
   size_t o_swa;         // fp32 [B,H_q,T,d]    un-normalised SWA branch output (bf16 on the tensor-core path)
   size_t o_rla;         // fp32 [B,H_q,T,d]    un-normalised RLA branch output (likewise)
@@ -74,6 +76,8 @@ struct Args {
   int n_chunks;
   int* status;                 // device status block (may be null when no workspace): word 0 status,
                                // word 1 detail, word 2 the forward's work counter
+  int* state_ready;            // [B*H_kv], zero at launch: chunk states the chunk-state kernel has stored so far
+                               // (null: the main kernel waits for that whole kernel instead)
   bool training;               // the backward will read every chunk state
   // hand-off
   float* state_out;
@@ -131,6 +135,7 @@ struct StateLaunch {
   int kv_per_batch;
   int phi;                  // rattn_feature_map applied to x
   int* status;
+  int* ready;               // optional [n_kv] (forward chain): matrices stored so far, published after each store
   const char* name;         // label of the timing record
 };
 cudaError_t launch_tc_states(const StateLaunch& L, cudaStream_t s);

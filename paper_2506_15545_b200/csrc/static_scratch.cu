@@ -17,10 +17,10 @@ namespace rattn {
 namespace {
 
 constexpr size_t kMatrices = RATTN_STATIC_MAX_CHUNK_STATES;
-constexpr size_t kStatusBytes = 256;
+constexpr size_t kStatusBytes = 512;                       // status block + one progress word per K/V head (at most kMatrices)
 constexpr size_t kStateBytes = kMatrices * 128 * 128 * sizeof(__nv_bfloat16);
 
-// [status block, 256 B | chunk states, bf16]
+// [status block, 256 B | progress words, 256 B | chunk states, bf16]
 static __device__ __align__(256) unsigned char g_static_scratch[kStatusBytes + kStateBytes];
 
 constexpr int kMaxDevices = 64;
@@ -85,6 +85,7 @@ extern "C" int rattn_forward_static(const void* q, const void* k, const void* v,
   e = scratch_address(&base);
   if (e != cudaSuccess) return cuda_failure(e);
   a.status = reinterpret_cast<int*>(base);
+  a.state_ready = reinterpret_cast<int*>(base + 256);
   a.chunk_state = reinterpret_cast<__nv_bfloat16*>(base + kStatusBytes);
   a.n_chunks = n_chunks;
   // The array keeps whatever the previous call left.  Only the status block (status word and

@@ -1259,6 +1259,7 @@ cudaError_t launch_tc_backward(const Args& a, cudaStream_t s) {
   // R_c for c = 0 .. n_r-1: walk the query tiles from the last one down to wt+1
   {
     StateLaunch L;
+    L.ready = nullptr;
     L.x = a.q; L.y = g_r; L.out = a.rstate;
     L.x_heads = a.H_q; L.x_layout = a.layout; L.y_heads = 0; L.y_layout = 0;
     L.T = a.T; L.n_kv = (int)nkv; L.group = a.group; L.n_chunks = a.n_chunks;

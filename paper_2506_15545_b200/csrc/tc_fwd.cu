@@ -25,6 +25,17 @@ cudaError_t launch_tc_forward(const Args& a, cudaStream_t s) {
   const int n_kv = a.B * a.H_kv;
   const bool want_state = rla && a.state_out != nullptr;
   bool chained = false;
+  // The main kernel can take the chunk states as the chain publishes them instead of waiting for the whole
+  // chain.  That pays where the chain is long and leaves most SMs to the main kernel, which otherwise runs out
+  // of work that needs no state (config 3: 16 chains of 64 chunks); elsewhere publishing only slows the chain.
+  bool progress = a.state_ready != nullptr;
+  if (progress) {
+    const int knob = tuning(RATTN_TUNE_STATE_PROGRESS);
+    int dev = 0, n_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      n_sm = 0;
+    progress = knob == 1 || (knob == 0 && 4 * n_kv <= n_sm && n_kt >= 48);
+  }
   if (want_state && a.Tk <= a.w && !a.seq_lens) {
     // nothing has left the window yet
     cudaError_t e = cudaMemsetAsync(a.state_out, 0, sizeof(float) * (size_t)n_kv * 128 * 128, s);
@@ -49,11 +60,14 @@ cudaError_t launch_tc_forward(const Args& a, cudaStream_t s) {
     L.seq_lens = a.seq_lens; L.kv_per_batch = a.H_kv;
     L.phi = a.phi;
     L.status = a.status; L.name = "tc_state_fwd";
+    L.ready = progress ? a.state_ready : nullptr;
     cudaError_t e = launch_tc_states(L, s);
     if (e != cudaSuccess) return e;
     chained = true;
   }
-  return launch_tc_forward_main(a, s, chained);
+  Args m = a;
+  if (!progress) m.state_ready = nullptr;            // the main kernel waits for the whole chain instead
+  return launch_tc_forward_main(m, s, chained);
 }
 
 }  // namespace rattn

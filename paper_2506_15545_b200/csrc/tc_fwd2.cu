@@ -68,6 +68,8 @@ struct FArgs {
   const int* seq_lens;    // optional [B]: valid query rows per batch entry
   int n_stateless;        // pairs whose tiles read no stored state; their units come first
   int wait_for_states;    // a chunk-state kernel runs ahead of this one: wait for it before the first state load
+  const int* state_ready; // ... or, per K/V head, for the number of states it has published so far (null: the former)
+  int ascending;          // units in sequence order, the order in which their states appear
   int debug_skip_arrive;  // debug build only: tile A's row group withholds its first hand-over (a wait then runs out)
   float scale_log2, eps;
 };
@@ -97,7 +99,7 @@ __device__ __forceinline__ Unit make_unit(const FArgs& a, int u) {
   // is still at work), then the others, heaviest first.
   const int pr = u / a.n_bh;
   un.bh_q = u % a.n_bh;
-  const int p = pr < a.n_stateless ? pr : a.n_pairs - 1 - (pr - a.n_stateless);
+  const int p = (a.ascending || pr < a.n_stateless) ? pr : a.n_pairs - 1 - (pr - a.n_stateless);
   const int b = un.bh_q / a.H_q;
   un.h = un.bh_q % a.H_q;
   un.bh_kv = b * (a.H_q / a.group) + un.h / a.group;
@@ -191,6 +193,21 @@ __device__ __forceinline__ bool sched_next(FBars* bars, int n, bool arrives, int
 }
 
 // ----------------------------------------------------------------------------- loader
+// Bounded wait (whole warp) until a progress word of another kernel reaches `need`; the TMA loads
+// that follow are ordered behind the acquiring read.
+__device__ __forceinline__ bool wait_published(const int* word, int need, volatile int* abort) {
+#pragma unroll 1
+  for (int it = 0; it < (1 << 20); ++it) {
+    if (ld_acquire_gpu(word) >= need) {
+      fence_proxy_async_all();
+      return true;
+    }
+    if ((it & 15) == 15 && *abort) return false;
+    __nanosleep(200);
+  }
+  *abort = 1;
+  return false;
+}
 __device__ bool fwd_loader(const FMaps& tm, const FArgs& a, unsigned char* smem, FBars* bars) {
   int kv_count = 0, cntU[2] = {0, 0}, cntX = 0;
   bool states_ready = (a.wait_for_states == 0);
@@ -229,7 +246,10 @@ __device__ bool fwd_loader(const FMaps& tm, const FArgs& a, unsigned char* smem,
         const int done_before = cntU[X] - (un.t[X] >= 0 ? 1 : 0);      // epilogues of tile X before this unit
         if (done_before >= 1) WAIT_OR_RETURN_W(bars->y_done[X], (done_before - 1) & 1);
       }
-      if (!states_ready) {
+      if (a.state_ready) {
+        // the chunk-state kernel, still running beside this one, has stored and published S_[cA]
+        if (!wait_published(a.state_ready + un.bh_kv, un.cA + 1, &bars->abort)) return false;
+      } else if (!states_ready) {
         // the chunk-state kernel launched ahead of this one has completed and its stores are visible
         asm volatile("griddepcontrol.wait;" ::: "memory");
         states_ready = true;
@@ -239,6 +259,8 @@ __device__ bool fwd_loader(const FMaps& tm, const FArgs& a, unsigned char* smem,
       ++cntX;
     }
   }
+  // not to end before the kernel whose states were taken as they appeared
+  if (a.state_ready && a.wait_for_states) asm volatile("griddepcontrol.wait;" ::: "memory");
   return true;
 }
 
@@ -896,6 +918,10 @@ cudaError_t launch_tc_forward_main(const Args& a, cudaStream_t s, bool after_sta
     if (t.n_stateless > t.n_pairs) t.n_stateless = t.n_pairs;
   }
   t.wait_for_states = after_states ? 1 : 0;
+  t.state_ready = (after_states && a.mode == RATTN_MODE_RATTN) ? a.state_ready : nullptr;
+  // with per-head progress words the units can follow the chain; worth it where the order above would
+  // have put the units without a state first anyway (few K/V heads, many SMs free beside the chain)
+  t.ascending = (t.state_ready && t.n_stateless > 0) ? 1 : 0;
   t.debug_skip_arrive = debug_skip_arrive();
   t.work_counter = (a.status && order != 3) ? a.status + 2 : nullptr;
   e = cudaFuncSetAttribute(tc_fwd2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, F_SMEM);

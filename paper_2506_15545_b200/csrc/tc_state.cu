@@ -49,6 +49,7 @@ struct StateArgs {
   int kv_per_batch;
   int phi;          // rattn_feature_map
   int* status;
+  int* ready;       // optional [n_kv]: number of leading output matrices stored so far (forward chain)
 };
 
 struct StBars {
@@ -175,8 +176,22 @@ tc_state_scan_kernel(const __grid_constant__ UMap tm_x, const __grid_constant__ 
     const bool issuer = (tid == 320);
     int n_flush = 0;
     // bf16 copy of this thread's row of the sum -> staging -> matrix `mat` of the head, one TMA store
+    int pending = 0;                                         // matrices stored, not yet published
+    auto publish = [&]() {
+      tma_store_wait();
+      fence_proxy_async_all();
+      __threadfence();
+      st_release_gpu(a.ready + kv, pending);
+      pending = 0;
+    };
     auto store_row = [&](const float (&x)[4][32], int mat) {
-      if (issuer) tma_store_wait_read();                     // the staging tile has left
+      if (issuer) {
+        // The kernel that reads the states runs beside this one and takes them as they appear.  The
+        // matrix stored last is published here, one flush later, when its store has long completed
+        // (it must be in memory, not merely read out of the staging tile, before its index is shown).
+        if (a.ready && pending) publish();
+        else tma_store_wait_read();                          // the staging tile has left
+      }
       asm volatile("bar.sync 4, 128;" ::: "memory");
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
@@ -195,6 +210,7 @@ tc_state_scan_kernel(const __grid_constant__ UMap tm_x, const __grid_constant__ 
       if (issuer) {
         store_tile(&tm_out, s_out, 0, kv * a.n_chunks + mat);
         tma_store_commit();
+        pending = mat + 1;
       }
     };
     auto write_final = [&](const float (&x)[4][32]) {
@@ -245,7 +261,10 @@ tc_state_scan_kernel(const __grid_constant__ UMap tm_x, const __grid_constant__ 
       if (stored_step(a, s)) store_row(x, a.out_first + a.dir * s);
       if (a.final_out != nullptr && s == n_steps - 1) write_final(x);
     }
-    if (issuer) tma_store_wait();
+    if (issuer) {
+      if (a.ready && pending) publish();
+      else tma_store_wait();
+    }
   }
   if (!ok && a.status) atomicExch(a.status, 1);
   tc_fence_before();
@@ -280,6 +299,7 @@ cudaError_t launch_tc_states(const StateLaunch& L, cudaStream_t s) {
   a.state_in = L.state_in;
   a.seq_lens = L.seq_lens; a.kv_per_batch = L.kv_per_batch > 0 ? L.kv_per_batch : 1;
   a.phi = L.phi;
+  a.ready = (L.dir > 0 && L.group == 1) ? L.ready : nullptr;
   cudaError_t e = cudaFuncSetAttribute(tc_state_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ST_SMEM);
   if (e != cudaSuccess) return e;
   {

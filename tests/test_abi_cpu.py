@@ -80,11 +80,12 @@ def test_strerror_and_workspace_bytes(B):
 
 def test_workspace_size_follows_mode_and_flags(B):
     """An inference forward keeps only what it uses: the status block on the portable kernels,
-    status + bf16 chunk states on the tensor-core kernels; training adds the residuals."""
+    status + one progress word per K/V head + bf16 chunk states on the tensor-core kernels; training
+    adds the residuals."""
     c5 = (32, 32, 8, 32768, 128, 512)
     infer = B.rattn_workspace_bytes_ex(*c5, B.RATTN_BF16, B.MODE_RATTN, 0)
     states = 32 * 8 * 256 * 128 * 128 * 2
-    assert infer == 256 + states                                         # 2.1 GB, not 78 GB
+    assert infer == 256 + 1024 + states                                  # 2.1 GB, not 78 GB
     assert B.rattn_workspace_bytes_ex(*c5, B.RATTN_BF16, B.MODE_SWA_ONLY, 0) == 256
     assert B.rattn_workspace_bytes_ex(*c5, B.RATTN_BF16, B.MODE_RATTN, B.FLAG_FORCE_GENERIC) == 256
     train = B.rattn_workspace_bytes_ex(*c5, B.RATTN_BF16, B.MODE_RATTN, B.FLAG_SAVE_RESIDUALS)
@@ -94,7 +95,7 @@ def test_workspace_size_follows_mode_and_flags(B):
     assert B.rattn_workspace_bytes(*c5) == max(train, train_generic)     # the bound covers every case
     assert B.rattn_workspace_bytes_ex(*c5, B.RATTN_BF16, 7, 0) == 0      # unknown mode
     few = (1, 4, 2, 1024, 128, 128)
-    assert B.rattn_workspace_bytes_ex(*few, B.RATTN_BF16, B.MODE_RATTN, 0) == 256 + 2 * 8 * 128 * 128 * 2
+    assert B.rattn_workspace_bytes_ex(*few, B.RATTN_BF16, B.MODE_RATTN, 0) == 256 + 256 + 2 * 8 * 128 * 128 * 2
 
 
 def _p(bind, **kw):

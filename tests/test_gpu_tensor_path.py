@@ -63,6 +63,27 @@ def test_tensor_forward_large_logits_trigger_rescale():
     check(y, ref, "bf16", "large logits")
 
 
+@pytest.mark.parametrize("T,w,Hq,Hkv", [(1280, 256, 4, 2), (1100, 128, 4, 1), (2048, 512, 2, 2), (4096, 128, 2, 1)])
+def test_tensor_forward_states_taken_as_published(T, w, Hq, Hkv):
+    """The main kernel reading each chunk state as soon as the chunk-state kernel has published it
+    (knob forced on; by default only long chains on few heads do this) computes the same operator,
+    with the same bits as the default schedule: only the order of the work units differs."""
+    wl = small("tcprog", 2, Hq, Hkv, T, 128, w, "bf16", 4500 + T + w, unit=True)
+    y0, ref, _ = run(wl)
+    prev = R.rattn_tune(R.TUNE_STATE_PROGRESS, 1)
+    try:
+        y1, _, _ = run(wl)
+        y2, _, _ = run(wl, save=True)
+    finally:
+        R.rattn_tune(R.TUNE_STATE_PROGRESS, prev)
+    # (with gains an output beyond |y| = 8 occurs in these inputs, where half a bf16 step alone is 3e-2:
+    # the bound that takes the output format into account, as for the element-wise maps)
+    from test_gpu_feature_maps import check_bf16_heavy_tails
+    check_bf16_heavy_tails(y1, ref, f"progress words, T={T} w={w}")
+    check_bf16_heavy_tails(y2, ref, f"progress words, training mode, T={T} w={w}")
+    assert torch.equal(y0, y1)
+
+
 def test_tensor_forward_c2_like_heads():
     """Config 2's sequence (T=4096, w=512, unit-RMS q/k, scale 1/sqrt(128)) on two heads."""
     wl = W.C2.replace(B=1, H_q=2, H_kv=2)
@@ -72,8 +93,9 @@ def test_tensor_forward_c2_like_heads():
 
 def test_tensor_residuals_match_portable_path():
     """The residuals the training-mode forward leaves for the backward: log-sum-exp (fp32, first
-    region after the 256-byte status block) and the un-normalised window output (second region;
-    fp32 on the portable path, bf16 on the tensor-core path) agree between the two paths."""
+    region after the status block: 256 bytes, plus 256 bytes of per-head progress words on the
+    tensor-core path) and the un-normalised window output (second region; fp32 on the portable
+    path, bf16 on the tensor-core path) agree between the two paths."""
     wl = small("tcs", 1, 2, 1, 512, 128, 128, "bf16", 4300, unit=True)
     y, ref, (q, k, v, ws) = run(wl, save=True)
     ws2 = torch.zeros_like(ws)
@@ -82,12 +104,13 @@ def test_tensor_residuals_match_portable_path():
                             flags=R.FLAG_FORCE_GENERIC)
     torch.cuda.synchronize()
     n = 2 * 512
-    f1 = ws[256:].view(torch.float32)
+    head1 = 512                                   # status block + progress words (one K/V head: 256 bytes)
+    f1 = ws[head1:].view(torch.float32)
     f2 = ws2[256:].view(torch.float32)
     lse1, lse2 = f1[:n], f2[:n]
     assert (lse1 - lse2).abs().max() < 2e-2
     off = (n * 4 + 255) // 256 * 256
-    o1 = ws[256 + off:256 + off + n * 128 * 2].view(torch.bfloat16).float()
+    o1 = ws[head1 + off:head1 + off + n * 128 * 2].view(torch.bfloat16).float()
     o2 = f2[off // 4:off // 4 + n * 128]
     assert (o1 - o2).abs().max() < 3e-2
     check(y, ref, "bf16")
