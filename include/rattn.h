@@ -344,7 +344,7 @@ typedef enum rattn_knob {
   RATTN_TUNE_STATE_PROGRESS = 5  /* the main kernel takes the chunk states as the chunk-state kernel publishes them
                                     (one progress word per K/V head, work units in sequence order) instead of
                                     waiting for that whole kernel: 0 (default) automatic = on for long chains on
-                                    few K/V heads (T >= 6144, 4 B H_kv <= SMs); 1 on; 2 off */
+                                    few K/V heads with windows up to 512 (T >= 6144, 4 B H_kv <= SMs); 1 on; 2 off */
 } rattn_knob;
 int rattn_tune(int knob, int value);
 

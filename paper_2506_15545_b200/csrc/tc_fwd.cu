@@ -28,13 +28,15 @@ cudaError_t launch_tc_forward(const Args& a, cudaStream_t s) {
   // The main kernel can take the chunk states as the chain publishes them instead of waiting for the whole
   // chain.  That pays where the chain is long and leaves most SMs to the main kernel, which otherwise runs out
   // of work that needs no state (config 3: 16 chains of 64 chunks); elsewhere publishing only slows the chain.
+  // With wide windows the units without a state are many and heavy already, and taking the units in sequence
+  // order (light ones first) costs more at the tail than the earlier start gains (measured from w = 1024 on).
   bool progress = a.state_ready != nullptr;
   if (progress) {
     const int knob = tuning(RATTN_TUNE_STATE_PROGRESS);
     int dev = 0, n_sm = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
       n_sm = 0;
-    progress = knob == 1 || (knob == 0 && 4 * n_kv <= n_sm && n_kt >= 48);
+    progress = knob == 1 || (knob == 0 && 4 * n_kv <= n_sm && n_kt >= 48 && wt <= 4);
   }
   if (want_state && a.Tk <= a.w && !a.seq_lens) {
     // nothing has left the window yet
