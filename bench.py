@@ -35,7 +35,7 @@ METRIC = "RAttention fwd+bwd TFLOP/s (T=4096,w=512,d=128,bf16)"
 # ncu capture each on the small training case `--case train`, B = 2), in MB per batch entry of
 # this head configuration; it scales with the batch.  See profiles/.  Set an entry to None when
 # its kernel changes after the capture.
-NCU_TRAFFIC_MB_PER_BATCH_ENTRY = {"tc_fwd": 89.9, "tc_bwd_dq": 106.7, "tc_bwd_dkv": 117.9}
+NCU_TRAFFIC_MB_PER_BATCH_ENTRY = {"tc_fwd": 90.3, "tc_bwd_dq": 107.1, "tc_bwd_dkv": 117.4}
 
 
 # --------------------------------------------------------------------------- work model
