@@ -58,6 +58,20 @@ def test_chunked_prefill_equals_one_pass(d, w, chunks, dtype, Hq, Hkv):
         assert torch.equal(k_ring[:, :, j % w].cpu(), k[:, :, j]) and torch.equal(v_ring[:, :, j % w].cpu(), v[:, :, j])
 
 
+def test_serving_paths_with_states_taken_as_published():
+    """The same chunked prefill (a resumed chunk's chain starts from the incoming state, which is its
+    first published matrix) and variable-length batch (every entry's chain has its own length) with
+    the main kernel reading each chunk state as soon as it is published, which by default only long
+    sequences on few heads do."""
+    prev = R.rattn_tune(R.TUNE_STATE_PROGRESS, 1)
+    try:
+        test_chunked_prefill_equals_one_pass(128, 128, (256, 200, 131), "bf16", 4, 2)
+        test_chunked_prefill_equals_one_pass(128, 256, (768, 640, 300), "bf16", 2, 1)
+        test_variable_length_batch(128, 128, "bf16")
+    finally:
+        R.rattn_tune(R.TUNE_STATE_PROGRESS, prev)
+
+
 def test_chunked_prefill_argument_checks():
     wl = small("cpa", 1, 2, 1, 32, 64, 16, "bf16", 1)
     q, k, v = (t.cuda() for t in W.make_qkv(wl))
