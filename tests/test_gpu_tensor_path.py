@@ -84,6 +84,28 @@ def test_tensor_forward_states_taken_as_published(T, w, Hq, Hkv):
     assert torch.equal(y0, y1)
 
 
+def test_states_taken_as_published_never_read_stale_memory():
+    """With the main kernel reading chunk states while the chunk-state kernel is still writing them, a
+    state read before it was complete would show as whatever the workspace held before: poison it
+    between calls and demand the bits of the schedule that waits for the whole chain, every time."""
+    wl = small("tcstale", 1, 4, 1, 4096, 128, 128, "bf16", 4600, unit=True)
+    q, k, v = (t.cuda() for t in W.make_qkv(wl))
+    ws = R.alloc_workspace(q, k, wl.w)
+    prev = R.rattn_tune(R.TUNE_STATE_PROGRESS, 2)
+    try:
+        want = R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws).clone()
+        R.rattn_tune(R.TUNE_STATE_PROGRESS, 1)
+        out = torch.empty_like(q)
+        for it in range(12):
+            ws.fill_(0x5A if it % 2 else 0xFF)
+            R.rattn_forward_ex(q, k, v, wl.w, scale=wl.scale, workspace=ws, out=out)
+            torch.cuda.synchronize()
+            assert R.rattn_read_status(ws) == 0
+            assert torch.equal(out, want), it
+    finally:
+        R.rattn_tune(R.TUNE_STATE_PROGRESS, prev)
+
+
 def test_tensor_forward_c2_like_heads():
     """Config 2's sequence (T=4096, w=512, unit-RMS q/k, scale 1/sqrt(128)) on two heads."""
     wl = W.C2.replace(B=1, H_q=2, H_kv=2)
